@@ -1,0 +1,460 @@
+"""CPU checker for greedy Tandem + SPEED decoding (Tandem Transformers, arXiv 2402.08644).
+
+THIS IS TEST INFRASTRUCTURE, NOT A PRODUCT PATH.  It is a plain, slow, fp64 numpy restatement of the
+paper's equations, used by the tests, by the smoke check and by the benchmark's CPU-baseline leg to
+decide whether the CUDA library computes the right thing.  It shares no code with the CUDA path and
+must never be imported by it.
+
+What it computes, in the paper's notation (x = large-model representations, y = small-model
+representations, y_hat = projected large representations, gamma = block length):
+
+  * Eq. 1 (Section 3, "Standard (Decoder) Transformer"): causal decoder, both as a brute-force
+    whole-sequence forward (no cache) and as an incremental pass over a key/value cache.
+  * Eq. 2 (Section 3, "Tandem Transformer"): y_hat = FF_Tandem(x^(l(j))); small layer j attends the
+    projected large representations for positions the large model has processed and its own
+    representations for the rest.  Brute force and cached.
+  * Section 3, "Inference", Figures 2 and 3: prompt handling (large model reads the prompt without
+    its last token), block-mode large pass, the free token.
+  * Section 3.1: draft gamma tokens, verify the block, first mismatch, take the large model's token
+    there, continue with the large model's representations of all previous tokens.
+
+Readings taken where the paper is silent or inconsistent (numbers match the design notes):
+  R1  Boundary.  Eq. 2 prints k = floor(i/gamma)*gamma, which would let a token at a multiple of gamma
+      attend the large model's representation of itself.  The training bullets of Section 3 and
+      Figure 3 say that the current block, including the query token, uses the small model's own
+      keys/values.  Here the boundary is simply the number of positions the large model has processed;
+      a query always sees its own key/value.  Inside SPEED the boundary is ragged (Section 3.1: "all
+      the previous tokens").
+  R2  x^(l) is the residual stream after l large layers; l = 0 is the embedding output.
+  R3  y_hat replaces y as the *layer input* at that position: K = LN1_S(y_hat) Wk^T, V likewise.
+  R4  Pre-LayerNorm blocks (gain and bias, eps 1e-5, biased variance), exact-erf GELU, no linear
+      biases, learned absolute position embeddings, untied output head.
+  R6  FF_Tandem MLP variant: hidden width given by the shape, GELU, no biases.
+  R7  The large model reads prompt[0..P-2]; prompt[P-1] is the pending token the small model starts from.
+  R8  "Deemed incorrect" = the draft differs from the arg-max of the large model's logits (greedy).
+  R9  Arg-max ties go to the lowest token id.  The decision is taken on logits rounded to float32,
+      the precision in which the CUDA path holds its logits.
+  R10 The verify pass has gamma+1 rows (pending token + gamma drafts) and can emit up to gamma+1 tokens.
+  R11 Accept lengths are per sequence; sequences are independent.
+  R12 A sequence stops after exactly max_new tokens; surplus tokens of the last iteration are dropped.
+  R13 accept_mode 1 keeps all gamma drafts whatever the comparison says (equal to stand-alone Tandem
+      with the free token, Figure 2); accept_mode 2 takes a pseudo-random accept length from a
+      counter-based hash (test only).
+
+Pins: every function here is pinned by tests/test_oracle_*.py (library decoder layer, brute force vs
+cache, SPEED == plain greedy, self-tandem, block == single-token passes, schedule fixtures from
+Figures 2 and 3, hand-made accept cases).  The absolute logit values of a random-init *Tandem* pair
+have no value printed in the paper to compare with: for those, parity unpinned beyond the invariants.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+from scipy.special import erf
+
+LN_EPS = 1e-5
+
+ACCEPT_NATURAL = 0
+ACCEPT_ALL = 1
+ACCEPT_HASH = 2
+
+
+# ----------------------------------------------------------------------------------------------
+# Elementary pieces (Eq. 1's Atn and FF, written out)
+# ----------------------------------------------------------------------------------------------
+
+def layer_norm(x: np.ndarray, gain: np.ndarray, bias: np.ndarray) -> np.ndarray:
+    """LayerNorm over the last axis: (x - mean) / sqrt(var + eps) * gain + bias, biased variance."""
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + LN_EPS) * gain + bias
+
+
+def gelu(x: np.ndarray) -> np.ndarray:
+    """Exact GELU: x * Phi(x)."""
+    return 0.5 * x * (1.0 + erf(x / math.sqrt(2.0)))
+
+
+def softmax(s: np.ndarray) -> np.ndarray:
+    """Softmax over the last axis."""
+    e = np.exp(s - s.max(axis=-1, keepdims=True))
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def attend(q: np.ndarray, K: np.ndarray, V: np.ndarray, n_heads: int) -> np.ndarray:
+    """Multi-head attention of ONE query q[d] over a context K[n][d], V[n][d]: per head,
+    softmax(q_h . k_h / sqrt(d_h)) weighted sum of v_h; heads concatenated."""
+    d = q.shape[0]
+    dh = d // n_heads
+    out = np.empty(d, dtype=q.dtype)
+    for h in range(n_heads):
+        sl = slice(h * dh, (h + 1) * dh)
+        scores = K[:, sl] @ q[sl] / math.sqrt(dh)
+        out[sl] = softmax(scores) @ V[:, sl]
+    return out
+
+
+def argmax_decision(logits: np.ndarray) -> int:
+    """Greedy token: arg-max of the float32-rounded logits, lowest id on ties (R9)."""
+    return int(np.argmax(logits.astype(np.float32)))
+
+
+def splitmix64(x: int) -> int:
+    """One round of the public splitmix64 mixing function on a 64-bit counter."""
+    m = 0xFFFFFFFFFFFFFFFF
+    x = (x + 0x9E3779B97F4A7C15) & m
+    z = x
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & m
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & m
+    return z ^ (z >> 31)
+
+
+def hashed_accept_length(mode_seed: int, seq: int, iteration: int, gamma: int) -> int:
+    """accept_mode 2 (R13): a = mix(mix(mix(seed) ^ seq) ^ iteration) mod (gamma + 1)."""
+    return splitmix64(splitmix64(splitmix64(mode_seed) ^ seq) ^ iteration) % (gamma + 1)
+
+
+# ----------------------------------------------------------------------------------------------
+# Weights
+# ----------------------------------------------------------------------------------------------
+
+class Decoder:
+    """Weights of one decoder (prefix 'L' or 'S' in the weight dict), cast to the compute dtype."""
+
+    def __init__(self, weights: Dict[str, np.ndarray], prefix: str, n_layers: int, n_heads: int,
+                 dtype=np.float64):
+        g = lambda name: np.asarray(weights[f"{prefix}.{name}"], dtype=dtype)
+        self.n_layers, self.n_heads = n_layers, n_heads
+        self.emb, self.pos = g("emb"), g("pos")
+        self.layers = []
+        for l in range(n_layers):
+            self.layers.append({k: g(f"{l}.{k}") for k in
+                                ("ln1_g", "ln1_b", "wq", "wk", "wv", "wo", "ln2_g", "ln2_b", "w1", "w2")})
+        self.lnf_g, self.lnf_b, self.w_out = g("lnf_g"), g("lnf_b"), g("w_out")
+
+    def embed(self, token: int, index: int) -> np.ndarray:
+        """x^(0) = Emb(t) + Pos(index)   (Eq. 1, R4)."""
+        return self.emb[token] + self.pos[index]
+
+    def feed_forward(self, l: int, h: np.ndarray) -> np.ndarray:
+        """h + GELU(LN2(h) W1^T) W2^T   (the FF of Eq. 1, R4)."""
+        p = self.layers[l]
+        return h + gelu(layer_norm(h, p["ln2_g"], p["ln2_b"]) @ p["w1"].T) @ p["w2"].T
+
+    def logits(self, h: np.ndarray) -> np.ndarray:
+        return layer_norm(h, self.lnf_g, self.lnf_b) @ self.w_out.T
+
+
+class TandemProjection:
+    """FF_Tandem^(j) for every small layer j (Eq. 2, first line)."""
+
+    def __init__(self, weights: Dict[str, np.ndarray], n_small_layers: int, kind: int, dtype=np.float64):
+        self.kind = kind
+        self.w = []
+        for j in range(n_small_layers):
+            if kind == 0:
+                self.w.append((np.asarray(weights[f"T.{j}.w_t"], dtype=dtype),))
+            else:
+                self.w.append((np.asarray(weights[f"T.{j}.w_t1"], dtype=dtype),
+                               np.asarray(weights[f"T.{j}.w_t2"], dtype=dtype)))
+
+    def __call__(self, j: int, x: np.ndarray) -> np.ndarray:
+        if self.kind == 0:
+            return x @ self.w[j][0].T
+        return gelu(x @ self.w[j][0].T) @ self.w[j][1].T
+
+
+# ----------------------------------------------------------------------------------------------
+# Brute force: whole-sequence forwards with no cache (the plain definitions)
+# ----------------------------------------------------------------------------------------------
+
+def decoder_full_forward(dec: Decoder, ids: Sequence[int]) -> Tuple[List[np.ndarray], np.ndarray]:
+    """Eq. 1 over a whole sequence, recomputing everything.  Returns ([x^(0), ..., x^(L)], logits),
+    each x^(l) of shape [S][d], logits [S][V]."""
+    S = len(ids)
+    h = np.stack([dec.embed(int(t), i) for i, t in enumerate(ids)]) if S else np.zeros((0, dec.emb.shape[1]))
+    reps = [h]
+    for l in range(dec.n_layers):
+        p = dec.layers[l]
+        a = layer_norm(h, p["ln1_g"], p["ln1_b"])
+        q, k, v = a @ p["wq"].T, a @ p["wk"].T, a @ p["wv"].T
+        o = np.stack([attend(q[i], k[: i + 1], v[: i + 1], dec.n_heads) for i in range(S)]) if S else h
+        h = h + o @ p["wo"].T
+        h = dec.feed_forward(l, h)
+        reps.append(h)
+    return reps, dec.logits(h)
+
+
+def tandem_small_full_forward(small: Decoder, proj: TandemProjection, layer_map: Sequence[int],
+                              large_reps: List[np.ndarray], boundary: int, ids: Sequence[int]) -> np.ndarray:
+    """Eq. 2 by brute force for positions boundary .. len(ids)-1 (the ones the small model runs on).
+
+    `large_reps[l]` holds x^(l) for at least the first `boundary` positions.  For small layer j the
+    context representation at position p is y_hat_p = FF_Tandem^(j)(x_p^(l(j))) if p < boundary, else
+    the small model's own y_p^(j) (R1); keys and values are LN1_S(context) Wk^T / Wv^T (R3).
+    Returns the small model's logits for positions boundary .. len(ids)-1."""
+    S = len(ids)
+    own = list(range(boundary, S))
+    y = np.stack([small.embed(int(ids[p]), p) for p in own])
+    for j in range(small.n_layers):
+        p_ = small.layers[j]
+        if boundary > 0:
+            ctx = np.concatenate([proj(j, large_reps[layer_map[j]][:boundary]), y], axis=0)
+        else:
+            ctx = y
+        a_ctx = layer_norm(ctx, p_["ln1_g"], p_["ln1_b"])
+        k, v = a_ctx @ p_["wk"].T, a_ctx @ p_["wv"].T
+        q = layer_norm(y, p_["ln1_g"], p_["ln1_b"]) @ p_["wq"].T
+        o = np.stack([attend(q[r], k[: p + 1], v[: p + 1], small.n_heads) for r, p in enumerate(own)])
+        y = y + o @ p_["wo"].T
+        y = small.feed_forward(j, y)
+    return small.logits(y)
+
+
+# ----------------------------------------------------------------------------------------------
+# Incremental passes over key/value caches
+# ----------------------------------------------------------------------------------------------
+
+class KVCache:
+    """Per layer, keys and values by absolute position.  `truncate` implements rollback."""
+
+    def __init__(self, n_layers: int):
+        self.k: List[List[np.ndarray]] = [[] for _ in range(n_layers)]
+        self.v: List[List[np.ndarray]] = [[] for _ in range(n_layers)]
+
+    def length(self, layer: int = 0) -> int:
+        return len(self.k[layer])
+
+    def append(self, layer: int, k: np.ndarray, v: np.ndarray) -> None:
+        self.k[layer].append(k)
+        self.v[layer].append(v)
+
+    def truncate(self, n: int) -> None:
+        for l in range(len(self.k)):
+            del self.k[l][n:]
+            del self.v[l][n:]
+
+
+def large_block_pass(dec: Decoder, cache: KVCache, tokens: Sequence[int], start: int
+                     ) -> Tuple[List[np.ndarray], np.ndarray]:
+    """Block mode (Section 3, "Inference"; Section 3.1): the large model processes `tokens` at
+    positions start, start+1, ... together.  Row r attends cache positions 0 .. start+r (causal
+    inside the block).  Appends the rows' keys/values to the cache.
+    Returns ([x^(0), ..., x^(L)] each [rows][d], logits [rows][V])."""
+    assert cache.length() == start
+    R = len(tokens)
+    h = np.stack([dec.embed(int(t), start + r) for r, t in enumerate(tokens)])
+    reps = [h]
+    for l in range(dec.n_layers):
+        p = dec.layers[l]
+        a = layer_norm(h, p["ln1_g"], p["ln1_b"])
+        q, k, v = a @ p["wq"].T, a @ p["wk"].T, a @ p["wv"].T
+        for r in range(R):
+            cache.append(l, k[r], v[r])
+        K, V = np.stack(cache.k[l]), np.stack(cache.v[l])
+        o = np.stack([attend(q[r], K[: start + r + 1], V[: start + r + 1], dec.n_heads) for r in range(R)])
+        h = h + o @ p["wo"].T
+        h = dec.feed_forward(l, h)
+        reps.append(h)
+    return reps, dec.logits(h)
+
+
+class TandemOracle:
+    """Greedy Tandem + SPEED for ONE sequence, step by step (Section 3.1)."""
+
+    def __init__(self, shape, weights: Dict[str, np.ndarray], dtype=np.float64):
+        self.shape = shape
+        self.large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
+        self.small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype)
+        self.proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
+        self.layer_map = list(shape.layer_map)
+        self.tokens: List[int] = []           # committed tokens c[0..n-1]; c[n-1] is pending
+        self.large_cache = KVCache(shape.large.n_layers)
+        self.derived = KVCache(shape.small.n_layers)   # large-derived region of the small model's K/V
+        self.own = KVCache(shape.small.n_layers)       # the small model's own K/V for the current block
+        self.n_large_runs = 0
+        self.n_small_runs = 0
+        self.iteration = 0
+        self.schedule: List[Tuple[str, List[int]]] = []   # (model, positions) per run, for Figures 2/3
+
+    # --- Eq. 2, first line, then the small layer's key/value maps (R3) --------------------------
+    def _project_rows(self, reps: List[np.ndarray], rows: range) -> None:
+        for j in range(self.small.n_layers):
+            p = self.small.layers[j]
+            for r in rows:
+                y_hat = self.proj(j, reps[self.layer_map[j]][r])
+                a = layer_norm(y_hat, p["ln1_g"], p["ln1_b"])
+                self.derived.append(j, a @ p["wk"].T, a @ p["wv"].T)
+
+    # --- prompt (Section 3 "Inference"; Figure 3; R7) --------------------------------------------
+    def prefill(self, prompt: Sequence[int]) -> None:
+        assert len(prompt) >= 1
+        self.tokens = [int(t) for t in prompt]
+        m = len(prompt) - 1
+        if m > 0:
+            reps, _ = large_block_pass(self.large, self.large_cache, self.tokens[:m], 0)
+            self._project_rows(reps, range(m))
+            self.schedule.append(("L", list(range(m))))
+
+    # --- one token through the small model over the mixed context (Eq. 2, lines 2-3) --------------
+    def _small_step(self, token: int, index: int) -> np.ndarray:
+        sm = self.small
+        y = sm.embed(token, index)
+        for j in range(sm.n_layers):
+            p = sm.layers[j]
+            a = layer_norm(y, p["ln1_g"], p["ln1_b"])
+            self.own.append(j, a @ p["wk"].T, a @ p["wv"].T)
+            K = np.stack(self.derived.k[j] + self.own.k[j])
+            V = np.stack(self.derived.v[j] + self.own.v[j])
+            assert K.shape[0] == index + 1
+            y = y + attend(a @ p["wq"].T, K, V, sm.n_heads) @ p["wo"].T
+            y = sm.feed_forward(j, y)
+        self.n_small_runs += 1
+        self.schedule.append(("S", [index]))
+        return sm.logits(y)
+
+    def draft(self, gamma: int, forced: Optional[Sequence[int]] = None) -> Tuple[List[int], List[np.ndarray]]:
+        """gamma autoregressive small-model steps starting from the pending token (Section 3.1).
+        Returns (own arg-max drafts, logits per step).  If `forced` is given, step s+1 is fed
+        forced[s] instead of its own arg-max (teacher forcing, used by replay tests)."""
+        n = len(self.tokens)
+        assert self.derived.length() == n - 1 and self.own.length() == 0
+        u = self.tokens[-1]
+        drafts, all_logits = [], []
+        for s in range(gamma):
+            lg = self._small_step(u, n - 1 + s)
+            d = argmax_decision(lg)
+            drafts.append(d)
+            all_logits.append(lg)
+            u = int(forced[s]) if forced is not None else d
+        return drafts, all_logits
+
+    def verify(self, drafts: Sequence[int]) -> Tuple[List[int], np.ndarray, List[np.ndarray]]:
+        """The large model processes the pending token and the drafts as one block (R10).
+        Returns (targets g[0..gamma], logits [gamma+1][V], reps)."""
+        n = len(self.tokens)
+        rows = [self.tokens[-1]] + [int(d) for d in drafts]
+        reps, logits = large_block_pass(self.large, self.large_cache, rows, n - 1)
+        self.n_large_runs += 1
+        self.schedule.append(("L", list(range(n - 1, n - 1 + len(rows)))))
+        return [argmax_decision(logits[r]) for r in range(len(rows))], logits, reps
+
+    @staticmethod
+    def accept_length(drafts: Sequence[int], targets: Sequence[int], mode: int = ACCEPT_NATURAL,
+                      mode_seed: int = 0, seq: int = 0, iteration: int = 0) -> int:
+        """Number of drafts kept: the length of the longest prefix on which draft r equals the large
+        model's token for the same position (Section 3.1, R8); or gamma (mode 1); or hashed (mode 2)."""
+        gamma = len(drafts)
+        if mode == ACCEPT_ALL:
+            return gamma
+        if mode == ACCEPT_HASH:
+            return hashed_accept_length(mode_seed, seq, iteration, gamma)
+        a = 0
+        while a < gamma and int(drafts[a]) == int(targets[a]):
+            a += 1
+        return a
+
+    def commit(self, a: int, drafts: Sequence[int], targets: Sequence[int], reps: List[np.ndarray]) -> List[int]:
+        """Keep drafts[0..a-1], then the large model's token for the next position; roll the large
+        cache back to the kept rows; project the kept rows for the small model; drop the small
+        model's own keys/values (Section 3.1)."""
+        n = len(self.tokens)
+        emitted = [int(d) for d in drafts[:a]] + [int(targets[a])]
+        self.tokens += emitted
+        self.large_cache.truncate(n + a)            # rows 0..a stay: positions n-1 .. n-1+a
+        self._project_rows(reps, range(a + 1))
+        self.own.truncate(0)
+        self.iteration += 1
+        return emitted
+
+    def step(self, gamma: int, mode: int = ACCEPT_NATURAL, mode_seed: int = 0, seq: int = 0) -> dict:
+        drafts, s_logits = self.draft(gamma)
+        targets, l_logits, reps = self.verify(drafts)
+        a = self.accept_length(drafts, targets, mode, mode_seed, seq, self.iteration)
+        emitted = self.commit(a, drafts, targets, reps)
+        return {"drafts": drafts, "targets": targets, "accept_len": a, "emitted": emitted,
+                "small_logits": s_logits, "large_logits": l_logits, "n_committed": len(self.tokens)}
+
+    def generate(self, prompt: Sequence[int], gamma: int, max_new: int, mode: int = ACCEPT_NATURAL,
+                 mode_seed: int = 0, seq: int = 0) -> Tuple[List[int], List[int]]:
+        """Full response (R12).  Returns (max_new tokens, accept length of every iteration)."""
+        self.prefill(prompt)
+        P = len(prompt)
+        accepts = []
+        while len(self.tokens) - P < max_new:
+            accepts.append(self.step(gamma, mode, mode_seed, seq)["accept_len"])
+        return self.tokens[P:P + max_new], accepts
+
+
+# ----------------------------------------------------------------------------------------------
+# Independent reference loops used as pins
+# ----------------------------------------------------------------------------------------------
+
+def plain_greedy(shape, weights: Dict[str, np.ndarray], prompt: Sequence[int], max_new: int,
+                 dtype=np.float64) -> List[int]:
+    """Greedy decoding of the large model alone by full recompute: tok[t] = argmax M_L(prompt ++ tok[<t]).
+    This is the definition that SPEED's output must equal (abstract; Section 3.1)."""
+    dec = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
+    seq = [int(t) for t in prompt]
+    for _ in range(max_new):
+        _, logits = decoder_full_forward(dec, seq)
+        seq.append(argmax_decision(logits[-1]))
+    return seq[len(prompt):]
+
+
+def plain_greedy_cached(shape, weights: Dict[str, np.ndarray], prompt: Sequence[int], max_new: int,
+                        dtype=np.float64) -> List[int]:
+    """The same tokens with a key/value cache and one-row block passes (used where full recompute
+    is too slow; pinned against `plain_greedy` on small cases)."""
+    dec = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
+    cache = KVCache(dec.n_layers)
+    seq = [int(t) for t in prompt]
+    if len(seq) > 1:
+        large_block_pass(dec, cache, seq[:-1], 0)
+    out = []
+    for _ in range(max_new):
+        _, logits = large_block_pass(dec, cache, [seq[-1]], len(seq) - 1)
+        seq.append(argmax_decision(logits[0]))
+        out.append(seq[-1])
+    return out
+
+
+def standalone_tandem_free_token(shape, weights: Dict[str, np.ndarray], prompt: Sequence[int], gamma: int,
+                                 max_new: int, dtype=np.float64) -> List[int]:
+    """Stand-alone Tandem decoding with the free token, written directly from Figure 2 and the
+    "Representation Generation + Token Prediction" variant of Section 3, by brute force (no cache,
+    no accept logic).  The prompt itself is read as in Figure 3 (R7).
+
+    Each round: the small model, reading the large model's representations of everything but the
+    last token, appends gamma tokens one at a time; then the large model reads the whole sequence
+    and appends its own prediction of the next token."""
+    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
+    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype)
+    proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
+    seq = [int(t) for t in prompt]
+    P = len(seq)
+    while len(seq) - P < max_new:
+        boundary = len(seq) - 1
+        reps, _ = decoder_full_forward(large, seq[:boundary])
+        for _ in range(gamma):
+            lg = tandem_small_full_forward(small, proj, shape.layer_map, reps, boundary, seq)
+            seq.append(argmax_decision(lg[-1]))
+        _, logits = decoder_full_forward(large, seq)
+        seq.append(argmax_decision(logits[-1]))
+    return seq[P:P + max_new]
+
+
+def generate_batch(shape, weights: Dict[str, np.ndarray], prompts: Sequence[Sequence[int]], gamma: int,
+                   max_new: int, mode: int = ACCEPT_NATURAL, mode_seed: int = 0, dtype=np.float64):
+    """Independent sequences (R11).  Returns (tokens per sequence, accept lengths per sequence,
+    (large runs, small runs) per sequence)."""
+    toks, accs, runs = [], [], []
+    for b, p in enumerate(prompts):
+        o = TandemOracle(shape, weights, dtype)
+        t, a = o.generate(p, gamma, max_new, mode, mode_seed, b)
+        toks.append(t)
+        accs.append(a)
+        runs.append((o.n_large_runs, o.n_small_runs))
+    return toks, accs, runs

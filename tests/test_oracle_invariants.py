@@ -1,0 +1,234 @@
+"""Pins for the checker's algorithmic paths: what the paper and the mathematics fix.
+
+I1  greedy Tandem + SPEED emits exactly plain greedy decoding of the large model (abstract, Section 3.1)
+I2  one block pass over gamma+1 tokens equals gamma+1 single-token passes (Section 3 "Inference")
+I3  with no large-processed positions the small model is a plain decoder (Section 1: gamma -> infinity)
+I4  gamma = 0 is a plain greedy step of the large model (Section 1: gamma = 0)
+I5  self-tandem (small == large, identity FF_Tandem, l(j) = j): Eq. 2 collapses to Eq. 1 for ANY boundary
+I6  cached mixed-context path equals brute-force recomputation of Eq. 2
+plus the schedule of Figures 2 and 3, hand-made accept cases, forced modes and run counts.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import tandem_oracle as O
+from paper_2402_08644_b200 import synth
+from helpers import toy_shape, toy_weights
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _prompt(shape, n, seed=0):
+    return [int(t) for t in synth.make_prompts(1, n, shape.large.vocab, seed)[0]]
+
+
+@pytest.mark.parametrize("gamma", [1, 2, 3, 4, 5, 8])
+@pytest.mark.parametrize("kind", [synth.FF_TANDEM_LINEAR, synth.FF_TANDEM_MLP])
+def test_I1_speed_equals_plain_greedy(gamma, kind):
+    shape = toy_shape(kind=kind, hidden=24 if kind else 0)
+    w = toy_weights(shape, seed=gamma)
+    prompt = _prompt(shape, 6, seed=gamma)
+    want = O.plain_greedy(shape, w, prompt, 12)
+    got, accepts = O.TandemOracle(shape, w).generate(prompt, gamma, 12)
+    assert got == want
+    assert all(0 <= a <= gamma for a in accepts)
+
+
+def test_I1_holds_for_a_garbage_small_model_and_a_one_token_prompt():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=3)
+    for k in w:
+        if k.startswith("S.") and not synth.is_norm_param(k):
+            w[k] = w[k] * 40.0          # nonsense drafts
+    for P in (1, 2, 9):
+        prompt = _prompt(shape, P, seed=P)
+        assert O.TandemOracle(shape, w).generate(prompt, 3, 10)[0] == O.plain_greedy(shape, w, prompt, 10)
+    assert O.plain_greedy_cached(shape, w, _prompt(shape, 5), 9) == O.plain_greedy(shape, w, _prompt(shape, 5), 9)
+
+
+def test_I2_block_pass_equals_single_token_passes_and_full_forward():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=7)
+    dec = O.Decoder(w, "L", shape.large.n_layers, shape.large.n_heads)
+    ids = _prompt(shape, 11)
+    c1, c2 = O.KVCache(dec.n_layers), O.KVCache(dec.n_layers)
+    O.large_block_pass(dec, c1, ids[:6], 0)
+    O.large_block_pass(dec, c2, ids[:6], 0)
+    reps_b, logits_b = O.large_block_pass(dec, c1, ids[6:], 6)
+    rows = [O.large_block_pass(dec, c2, [t], 6 + r) for r, t in enumerate(ids[6:])]
+    for r, (reps_s, logits_s) in enumerate(rows):
+        assert np.allclose(logits_b[r], logits_s[0], atol=1e-10)
+        for l in range(dec.n_layers + 1):
+            assert np.allclose(reps_b[l][r], reps_s[l][0], atol=1e-10)
+    for l in range(dec.n_layers):
+        assert np.allclose(np.stack(c1.k[l]), np.stack(c2.k[l]), atol=1e-10)
+        assert np.allclose(np.stack(c1.v[l]), np.stack(c2.v[l]), atol=1e-10)
+    full_reps, full_logits = O.decoder_full_forward(dec, ids)
+    assert np.allclose(full_logits[6:], logits_b, atol=1e-10)
+    assert np.allclose(full_reps[2][6:], reps_b[2], atol=1e-10)
+    assert np.abs(full_logits).max() > 0.5
+
+
+def test_I3_no_large_context_means_plain_small_decoder():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=9)
+    ids = _prompt(shape, 7)
+    o = O.TandemOracle(shape, w)
+    o.prefill(ids[:1])                         # one-token prompt: the large model has seen nothing
+    _, logits = o.draft(6, forced=ids[1:7])
+    small = O.Decoder(w, "S", shape.small.n_layers, shape.small.n_heads)
+    _, want = O.decoder_full_forward(small, ids[:6])
+    assert np.allclose(np.stack(logits), want, atol=1e-10)
+
+
+def test_I4_gamma_zero_is_a_plain_large_step():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=2)
+    prompt = _prompt(shape, 5)
+    got, accepts = O.TandemOracle(shape, w).generate(prompt, 0, 7)
+    assert got == O.plain_greedy(shape, w, prompt, 7)
+    assert accepts == [0] * 7
+
+
+@pytest.mark.parametrize("gamma", [1, 3, 4])
+def test_I5_self_tandem_accepts_everything(gamma):
+    dims = synth.ModelDims(3, 32, 4, 64, 50, 64)
+    shape = synth.self_tandem_shape(dims)
+    w = synth.make_self_tandem_weights(shape, seed=4, std=0.35)
+    synth.perturb_norm_params(w, 4)
+    for k in list(w):                          # keep the copy exact after perturbing the norms
+        if k.startswith("S."):
+            w[k] = w["L." + k[2:]].copy()
+    prompt = _prompt(shape, 5)
+    o = O.TandemOracle(shape, w)
+    o.prefill(prompt)
+    for it in range(4):
+        res = o.step(gamma)
+        assert res["accept_len"] == gamma
+        assert res["drafts"] == res["targets"][:gamma]
+        for s in range(gamma):                 # the small model's logits are the large model's
+            assert np.allclose(res["small_logits"][s], res["large_logits"][s], atol=1e-9)
+    assert o.tokens[5:] == O.plain_greedy(shape, w, prompt, 4 * (gamma + 1))
+
+
+@pytest.mark.parametrize("kind", [synth.FF_TANDEM_LINEAR, synth.FF_TANDEM_MLP])
+def test_I6_cached_mixed_context_equals_brute_force_eq2(kind):
+    shape = toy_shape(kind=kind, hidden=20 if kind else 0, layer_map=(1, 3))
+    w = toy_weights(shape, seed=11)
+    prompt = _prompt(shape, 6)
+    o = O.TandemOracle(shape, w)
+    o.prefill(prompt)
+    large = O.Decoder(w, "L", shape.large.n_layers, shape.large.n_heads)
+    small = O.Decoder(w, "S", shape.small.n_layers, shape.small.n_heads)
+    proj = O.TandemProjection(w, shape.small.n_layers, kind)
+    for it in range(4):
+        n = len(o.tokens)
+        drafts, s_logits = o.draft(3)
+        seq = o.tokens + drafts[:-1]                      # inputs of the three draft steps
+        reps, _ = O.decoder_full_forward(large, o.tokens[: n - 1])
+        want = O.tandem_small_full_forward(small, proj, shape.layer_map, reps, n - 1, seq)
+        assert np.allclose(np.stack(s_logits), want, atol=1e-10)
+        targets, l_logits, xs = o.verify(drafts)
+        a = (it * 2) % 4                                  # 0, 2, 0, 2 ... plus 3 below: ragged rollback
+        if it == 3:
+            a = 3
+        o.commit(a, drafts, targets, xs)
+        # provenance: every derived key equals a from-scratch projection of the large model's reps
+        reps_now, _ = O.decoder_full_forward(large, o.tokens[:-1])
+        for j in range(small.n_layers):
+            p = small.layers[j]
+            ctx = O.layer_norm(proj(j, reps_now[shape.layer_map[j]]), p["ln1_g"], p["ln1_b"])
+            assert np.allclose(np.stack(o.derived.k[j]), ctx @ p["wk"].T, atol=1e-10)
+            assert np.allclose(np.stack(o.derived.v[j]), ctx @ p["wv"].T, atol=1e-10)
+        assert o.large_cache.length() == len(o.tokens) - 1 and o.own.length() == 0
+
+
+def test_brute_force_eq2_is_sensitive_to_the_boundary():
+    """The mixed context matters: moving the boundary changes the small model's logits (so the
+    equalities above are not satisfied by a path that ignores the large model)."""
+    shape = toy_shape()
+    w = toy_weights(shape, seed=13)
+    ids = _prompt(shape, 8)
+    large = O.Decoder(w, "L", shape.large.n_layers, shape.large.n_heads)
+    small = O.Decoder(w, "S", shape.small.n_layers, shape.small.n_heads)
+    proj = O.TandemProjection(w, shape.small.n_layers, 0)
+    reps, _ = O.decoder_full_forward(large, ids)
+    a = O.tandem_small_full_forward(small, proj, shape.layer_map, reps, 6, ids)[-1]
+    b = O.tandem_small_full_forward(small, proj, shape.layer_map, reps, 3, ids)[-1]
+    assert np.abs(a - b).max() > 1e-3
+
+
+def test_accept_all_equals_standalone_tandem_with_free_token():
+    for kind, gamma in ((synth.FF_TANDEM_LINEAR, 2), (synth.FF_TANDEM_MLP, 3)):
+        shape = toy_shape(kind=kind, hidden=12 if kind else 0)
+        w = toy_weights(shape, seed=21 + gamma)
+        prompt = _prompt(shape, 5, seed=gamma)
+        got, accepts = O.TandemOracle(shape, w).generate(prompt, gamma, 11, mode=O.ACCEPT_ALL)
+        assert got == O.standalone_tandem_free_token(shape, w, prompt, gamma, 11)
+        assert accepts == [gamma] * len(accepts)
+        assert got != O.plain_greedy(shape, w, prompt, 11)     # it is a different decoder
+
+
+def _read_schedule(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                m, a, b = line.split()
+                rows.append((m, list(range(int(a), int(b) + 1))))
+    return rows
+
+
+def test_schedule_matches_figures_2_and_3():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=1)
+    fig2 = _read_schedule("fig2_schedule_gamma2.txt")
+    o = O.TandemOracle(shape, w)
+    o.prefill(_prompt(shape, 9))
+    for _ in range(3):
+        o.step(2, mode=O.ACCEPT_ALL)
+    assert o.schedule == fig2
+    fig3 = _read_schedule("fig3_prompt_schedule_gamma2.txt")
+    o = O.TandemOracle(shape, w)
+    o.prefill(_prompt(shape, 8))
+    o.draft(2)
+    assert o.schedule == fig3
+
+
+def test_accept_length_hand_cases():
+    A = O.TandemOracle.accept_length
+    assert A([5, 6, 7], [5, 6, 7, 9]) == 3          # all verified: i = gamma + 1
+    assert A([5, 6, 7], [4, 6, 7, 9]) == 0          # first draft wrong, later matches do not count
+    assert A([5, 6, 7], [5, 1, 7, 9]) == 1
+    assert A([5, 6, 7], [5, 6, 1, 9]) == 2
+    assert A([], [3]) == 0
+    assert A([5, 6, 7], [0, 0, 0, 0], mode=O.ACCEPT_ALL) == 3
+    a = A([5, 6, 7], [0, 0, 0, 0], mode=O.ACCEPT_HASH, mode_seed=5, seq=2, iteration=9)
+    assert a == O.hashed_accept_length(5, 2, 9, 3) and 0 <= a <= 3
+
+
+def test_commit_emits_prefix_plus_correction_and_rolls_back():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=17)
+    o = O.TandemOracle(shape, w)
+    o.prefill(_prompt(shape, 4))
+    drafts, _ = o.draft(3)
+    targets, _, reps = o.verify(drafts)
+    assert o.large_cache.length() == 3 + 4
+    emitted = o.commit(1, drafts, targets, reps)
+    assert emitted == [drafts[0], targets[1]]
+    assert len(o.tokens) == 6 and o.large_cache.length() == 5 and o.derived.length() == 5
+
+
+def test_hash_mode_still_emits_valid_lengths_and_counts_runs():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=19)
+    prompts = [list(p) for p in synth.make_prompts(3, [4, 7, 2], shape.large.vocab, 5)]
+    toks, accs, runs = O.generate_batch(shape, w, prompts, 3, 10, mode=O.ACCEPT_HASH, mode_seed=77)
+    assert [len(t) for t in toks] == [10, 10, 10]
+    assert accs[0] != accs[1]                      # the hash depends on the sequence index
+    for a, (nl, ns) in zip(accs, runs):
+        assert nl == len(a) and ns == 3 * len(a)   # one large run and gamma small runs per iteration
+        assert sum(x + 1 for x in a) >= 10 > sum(x + 1 for x in a[:-1])

@@ -1,0 +1,134 @@
+"""Pins for the checker's elementary pieces: closed forms, textbook special cases and library routines.
+
+Each test is chosen so that one plausible mistake (a dropped term, a wrong sign, a transposed operand,
+a wrong axis) makes it fail."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import tandem_oracle as O
+from paper_2402_08644_b200 import synth
+from helpers import toy_shape, toy_weights
+
+
+def test_softmax_rows_sum_to_one_and_shift_invariant():
+    rng = np.random.default_rng(0)
+    s = rng.normal(size=(7, 33)) * 5
+    p = O.softmax(s)
+    assert np.allclose(p.sum(-1), 1.0, atol=1e-14)
+    assert np.allclose(O.softmax(s + 123.0), p, atol=1e-13)
+    # closed form for two logits: sigmoid of the difference
+    assert np.isclose(O.softmax(np.array([0.3, -1.1]))[0], 1 / (1 + math.exp(-1.4)))
+
+
+def test_gelu_closed_forms():
+    assert O.gelu(np.array(0.0)) == 0.0
+    assert np.isclose(O.gelu(np.array(1.0)), 0.8413447460685429, atol=1e-15)   # Phi(1)
+    x = np.linspace(-6, 6, 101)
+    assert np.allclose(O.gelu(x) - O.gelu(-x), x, atol=1e-14)                  # odd part is x/2 * 2
+    assert np.isclose(O.gelu(np.array(12.0)), 12.0)
+    assert abs(O.gelu(np.array(-12.0))) < 1e-12
+    t = torch.tensor(x, dtype=torch.float64)
+    assert np.allclose(O.gelu(x), torch.nn.functional.gelu(t).numpy(), atol=1e-14)
+
+
+def test_layer_norm_special_cases_and_library():
+    rng = np.random.default_rng(1)
+    g, b = rng.normal(size=16), rng.normal(size=16)
+    const = np.full((3, 16), 4.25)
+    assert np.allclose(O.layer_norm(const, g, b), np.broadcast_to(b, (3, 16)), atol=1e-12)
+    x = rng.normal(size=(5, 16)) * 3 + 1
+    ref = torch.nn.functional.layer_norm(torch.tensor(x), (16,), torch.tensor(g), torch.tensor(b), eps=1e-5)
+    assert np.allclose(O.layer_norm(x, g, b), ref.numpy(), atol=1e-13)
+    # unit gain, zero bias: rows have zero mean and (almost) unit biased variance
+    y = O.layer_norm(x, np.ones(16), np.zeros(16))
+    assert np.allclose(y.mean(-1), 0, atol=1e-13)
+    assert np.allclose((y ** 2).mean(-1), x.var(-1) / (x.var(-1) + 1e-5), atol=1e-12)
+
+
+def test_attend_uniform_keys_is_mean_of_values():
+    rng = np.random.default_rng(2)
+    q = rng.normal(size=12)
+    K = np.tile(rng.normal(size=12), (9, 1))
+    V = rng.normal(size=(9, 12))
+    assert np.allclose(O.attend(q, K, V, 3), V.mean(0), atol=1e-13)
+
+
+def test_attend_single_key_returns_its_value_and_matches_library():
+    rng = np.random.default_rng(3)
+    q = rng.normal(size=16)
+    K, V = rng.normal(size=(1, 16)), rng.normal(size=(1, 16))
+    assert np.allclose(O.attend(q, K, V, 4), V[0])
+    n, H, dh = 11, 4, 4
+    K, V = rng.normal(size=(n, 16)), rng.normal(size=(n, 16))
+    tq = torch.tensor(q).view(1, H, 1, dh)
+    tk = torch.tensor(K).view(n, H, dh).permute(1, 0, 2).unsqueeze(0)
+    tv = torch.tensor(V).view(n, H, dh).permute(1, 0, 2).unsqueeze(0)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv).reshape(16).numpy()
+    assert np.allclose(O.attend(q, K, V, H), ref, atol=1e-13)
+
+
+def test_argmax_ties_go_to_lowest_id_in_float32():
+    assert O.argmax_decision(np.array([0.1, 0.7, 0.7, 0.2])) == 1
+    # two values that differ only below float32 resolution tie after rounding
+    assert O.argmax_decision(np.array([0.0, 1.0, 1.0 + 1e-12])) == 1
+    assert O.argmax_decision(np.array([0.0, 1.0, 1.0 + 1e-6])) == 2
+
+
+def _torch_decoder_logits(shape, w, ids):
+    """The same decoder assembled from torch.nn building blocks (pre-LN TransformerEncoderLayer with a
+    causal mask, exact GELU, biases zeroed) in float64."""
+    d = shape.large
+    layers = []
+    for l in range(d.n_layers):
+        lay = torch.nn.TransformerEncoderLayer(d.d_model, d.n_heads, d.d_ff, dropout=0.0, activation="gelu",
+                                               batch_first=True, norm_first=True, dtype=torch.float64)
+        g = lambda k: torch.tensor(w[f"L.{l}.{k}"], dtype=torch.float64)
+        with torch.no_grad():
+            lay.self_attn.in_proj_weight.copy_(torch.cat([g("wq"), g("wk"), g("wv")], 0))
+            lay.self_attn.in_proj_bias.zero_()
+            lay.self_attn.out_proj.weight.copy_(g("wo"))
+            lay.self_attn.out_proj.bias.zero_()
+            lay.linear1.weight.copy_(g("w1")); lay.linear1.bias.zero_()
+            lay.linear2.weight.copy_(g("w2")); lay.linear2.bias.zero_()
+            lay.norm1.weight.copy_(g("ln1_g")); lay.norm1.bias.copy_(g("ln1_b"))
+            lay.norm2.weight.copy_(g("ln2_g")); lay.norm2.bias.copy_(g("ln2_b"))
+        lay.eval()
+        layers.append(lay)
+    S = len(ids)
+    t = lambda k: torch.tensor(w[k], dtype=torch.float64)
+    h = (t("L.emb")[torch.tensor(ids)] + t("L.pos")[:S]).unsqueeze(0)
+    mask = torch.triu(torch.full((S, S), float("-inf"), dtype=torch.float64), diagonal=1)
+    reps = [h[0].numpy().copy()]
+    with torch.no_grad():
+        for lay in layers:
+            h = lay(h, src_mask=mask)
+            reps.append(h[0].numpy().copy())
+        out = torch.nn.functional.layer_norm(h[0], (d.d_model,), t("L.lnf_g"), t("L.lnf_b"), eps=1e-5)
+        logits = out @ t("L.w_out").T
+    return reps, logits.numpy()
+
+
+def test_decoder_full_forward_matches_torch_transformer_layers():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=5)
+    ids = synth.make_prompts(1, 13, shape.large.vocab, seed=3)[0]
+    dec = O.Decoder(w, "L", shape.large.n_layers, shape.large.n_heads)
+    reps, logits = O.decoder_full_forward(dec, ids)
+    ref_reps, ref_logits = _torch_decoder_logits(shape, w, [int(i) for i in ids])
+    for a, b in zip(reps, ref_reps):
+        assert np.allclose(a, b, atol=1e-10, rtol=1e-10)
+    assert np.allclose(logits, ref_logits, atol=1e-10, rtol=1e-10)
+    assert np.abs(logits).max() > 0.5   # the comparison is not vacuous
+
+
+def test_splitmix64_matches_published_sequence_head():
+    # First outputs of the public-domain splitmix64 generator started from state 0 (Vigna's
+    # reference values, widely reproduced): next() adds the golden-ratio increment, then mixes.
+    assert O.splitmix64(0) == 0xE220A8397B1DCDAF
+    assert O.splitmix64(0x9E3779B97F4A7C15) == 0x6E789E6AA1B965F4
+    for g in (1, 3, 7):
+        vals = {O.hashed_accept_length(11, 0, it, g) for it in range(200)}
+        assert vals == set(range(g + 1))
