@@ -1,0 +1,319 @@
+#!/usr/bin/env python
+"""Benchmark of the Tandem + SPEED hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input: the prompt pass (large model over
+the prompt, FF_Tandem projection of every prompt position) followed by Tandem + SPEED greedy decoding of
+`max_new` tokens per sequence (draft, block verify, projection, accept/rollback, repeated).  The default
+workload is the "Small Tandem" configuration: bf16, batch 1, 512-token random prompt, gamma 3, 256 new
+tokens, natural acceptance.  The metric is generated tokens per second of the whole job.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload small|tiny|medium]
+
+With N > 1 (under torchrun) every rank runs an independent replica (sequences are independent units; there
+is no collective on the path); the value is all ranks' tokens over the slowest rank's time.
+
+`--impl reference` times the CPU checker (oracle/) on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2402_08644_b200 import synth  # noqa: E402
+
+METRIC = "tandem_speed_decode_tokens_per_s"
+UNIT = "tokens/s"
+
+WORKLOADS = {
+    # name: (config name, batch, prompt length, gamma, new tokens, max_pos)
+    "tiny": ("tiny", 1, 32, 4, 64, 128),
+    "small": ("small", 1, 512, 3, 256, 1024),
+    "medium": ("medium", 8, 2048, 3, 256, 2560),
+}
+
+
+def workload_desc(name):
+    cfgname, B, P, gamma, new, _ = WORKLOADS[name]
+    return (f"{cfgname}: batch {B}, prompt {P} uniform-random ids, gamma {gamma}, {new} new tokens, "
+            f"natural acceptance, random-init N(0,0.02) weights seed 0")
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes_per_iteration(shape, B, gamma, T):
+    """Weights of the large model once, of the small model gamma times, FF_Tandem and the small key/value maps
+    once, plus both KV streams at context length T (bf16)."""
+    esz = 2 if shape.dtype == synth.DTYPE_BF16 else 4
+    def model(d):
+        return d.n_layers * (4 * d.d_model ** 2 + 2 * d.d_model * d.d_ff) + d.d_model * d.vocab
+    L, S = shape.large, shape.small
+    proj = S.n_layers * (S.d_model * L.d_model + 2 * S.d_model ** 2) if shape.ff_tandem_kind == 0 else \
+        S.n_layers * (shape.hidden * L.d_model + S.d_model * shape.hidden + 2 * S.d_model ** 2)
+    kv = B * T * (L.n_layers * 2 * L.d_model + gamma * S.n_layers * 2 * S.d_model)
+    return esz * (model(L) + gamma * model(S) + proj + kv)
+
+
+def run_reference(args):
+    """The CPU checker as it stands, on the host cores, on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import tandem_oracle as O
+    cfgname, B, P, gamma, new, max_pos = WORKLOADS[args.workload]
+    shape = synth.named_config(cfgname, max_pos)
+    weights = synth.make_weights(shape, seed=0)
+    prompt = [int(t) for t in synth.make_prompts(B, P, shape.large.vocab, seed=0)[0]]
+    sample_new = min(new, 8)
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        o = O.TandemOracle(shape, weights)
+        o.prefill(prompt)
+        t1 = time.perf_counter()
+        while len(o.tokens) - P < sample_new:
+            o.step(gamma)
+        t2 = time.perf_counter()
+        if it >= args.warmup:
+            # scale the sample to the full workload: one prompt pass plus `new` tokens at the sampled decode rate
+            times.append((t1 - t0) + (t2 - t1) * new / (len(o.tokens) - P))
+    sec = float(np.mean(times))
+    value = B * new / sec
+    cores = os.cpu_count()
+    sample = (f"sequence 0 of the workload: full {P}-token prompt pass + {sample_new} new tokens per step, decode time "
+              f"scaled to {new} tokens; numpy fp64")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_desc(args.workload)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def cpu_baseline(shape, weights, prompt, gamma, new):
+    from oracle import tandem_oracle as O
+    P = len(prompt)
+    sample_new = min(new, 24)
+    t0 = time.perf_counter()
+    o = O.TandemOracle(shape, weights)
+    o.prefill(prompt)
+    t1 = time.perf_counter()
+    while len(o.tokens) - P < sample_new:
+        o.step(gamma)
+    t2 = time.perf_counter()
+    sec = (t1 - t0) + (t2 - t1) * new / (len(o.tokens) - P)
+    return {"value": new / sec, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+            "sample": (f"sequence 0: full {P}-token prompt pass ({t1 - t0:.1f} s) + {sample_new} new tokens "
+                       f"({t2 - t1:.1f} s), decode time scaled to {new} tokens; numpy fp64 with its BLAS threads")}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="small", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the accept-all / greedy / per-kernel passes")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2402_08644_b200 import binding, build as _build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+
+    cfgname, B, P, gamma, new, max_pos = WORKLOADS[args.workload]
+    shape = synth.named_config(cfgname, max_pos)
+    weights = synth.make_weights(shape, seed=0)
+    prompts = [[int(t) for t in p] for p in synth.make_prompts(B, P, shape.large.vocab, seed=rank)]
+    t = binding.Tandem(shape, weights, max_batch=B, max_seq=P + new + gamma + 1, gamma_max=gamma, device=local_rank,
+                       max_prefill_rows=B * P)
+    stream = torch.cuda.current_stream()
+
+    def step(mode=0):
+        t.tandem_prefill(prompts)
+        return t.tandem_speculative_generate(gamma, new, mode)
+
+    for _ in range(args.warmup):
+        out, lens, stats = step()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-timed region: K steps between events on the stream the library launches on ----
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    barrier()
+    launches0 = t.tandem_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
+    ev[0].record(stream)
+    iters = 0
+    for k in range(args.steps):
+        t.tandem_prefill(prompts)
+        ev[2 * k + 1].record(stream)
+        out, lens, stats = t.tandem_speculative_generate(gamma, new, 0)
+        ev[2 * k + 2].record(stream)
+        iters += stats["iterations"]
+    barrier()
+    clocks = sampler.stop()
+    launches = t.tandem_launch_count() - launches0
+    total_ms = ev[0].elapsed_time(ev[-1])
+    prefill_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(args.steps)) / args.steps
+    decode_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(args.steps)) / args.steps
+    ms_per_step = total_ms / args.steps
+    if world > 1:
+        tm = torch.tensor([ms_per_step], device="cuda")
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        ms_per_step = float(tm.item())
+    value = world * B * new / (ms_per_step * 1e-3)
+
+    # ---- end to end through the public calls with host buffers, wall clock, copies included ----
+    barrier()
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        out, lens, stats = step()
+    torch.cuda.synchronize()
+    e2e_sec = (time.perf_counter() - t0) / args.steps
+    if world > 1:
+        tm = torch.tensor([e2e_sec], device="cuda")
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        e2e_sec = float(tm.item())
+    rows = B * (P - 1)
+    h2d = 4 * (3 * rows + 2 * (rows // 16 + B) + 2 * B)          # row token/sequence/position, query groups, n, pending
+    d2h = 4 * (B * new + B + 16) + stats["iterations"] * 20      # tokens, lengths, histogram; 5 counters per iteration
+    e2e = {"value": world * B * new / e2e_sec, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if shape.dtype == synth.DTYPE_BF16 else "f32", "data": "synthetic",
+            "config": {"workload": workload_desc(args.workload), "parallelism": f"replicas x{world}",
+                       "l2": "per-iteration working set (weights + KV) exceeds the 126 MB L2; no flush needed"},
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "prefill_ms": prefill_ms, "decode_ms": decode_ms, "decode_tokens_per_s": B * new / (decode_ms * 1e-3),
+            "iterations_per_step": iters / args.steps, "accept_hist": stats["accept_hist"]}
+
+    if rank == 0 and not args.no_extras:
+        peak, peak_kind = read_peaks()
+        # whole-iteration view: algorithmic bytes of one draft/verify iteration over the measured time per iteration
+        T_avg = P + new / 2
+        it_bytes = algorithmic_bytes_per_iteration(shape, B, gamma, T_avg)
+        it_ms = decode_ms / (iters / args.steps)
+        line["iteration"] = {"algorithmic_gb": it_bytes / 1e9, "ms": it_ms, "achieved_gbs": it_bytes / 1e9 / (it_ms * 1e-3),
+                             "frac_of_peak": it_bytes / 1e9 / (it_ms * 1e-3) / peak}
+        # per-kernel pass: the same step with every launch bracketed by events (slower; not the timed value)
+        t.tandem_profile_enable(200000)
+        step()
+        prof = t.tandem_profile_read()
+        t.tandem_profile_enable(0)
+        tot = sum(v["ms"] for v in prof.values()) or 1.0
+        line["kernels"] = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / tot, 4),
+                               "avg_us": round(1e3 * v["ms"] / max(1, v["launches"]), 3)} for k, v in prof.items()}
+        dom = max((k for k in prof if k != "gemm_tiled" and k != "attn_prompt"), key=lambda k: prof[k]["ms"])
+        g = prof[dom]
+        achieved = g["work"] / 1e9 / (g["ms"] * 1e-3) if g["ms"] > 0 else 0.0
+        line["roofline"] = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                            "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind,
+                            "launches": g["launches"], "avg_launch_us": 1e3 * g["ms"] / max(1, g["launches"]),
+                            "algorithmic_bytes_per_launch": g["work"] / max(1, g["launches"])}
+        # context: accept-all timing mode and plain greedy decoding of the large model alone
+        t.tandem_prefill(prompts); torch.cuda.synchronize()
+        t0 = time.perf_counter(); t.tandem_speculative_generate(gamma, new, 1); torch.cuda.synchronize()
+        line["accept_all_decode_tokens_per_s"] = B * new / (time.perf_counter() - t0)
+        t.tandem_prefill(prompts); torch.cuda.synchronize()
+        t0 = time.perf_counter(); t.tandem_large_greedy_generate(new); torch.cuda.synchronize()
+        line["large_greedy_decode_tokens_per_s"] = B * new / (time.perf_counter() - t0)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(shape, weights, prompts[0], gamma, new)
+    t.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,227 @@
+/*
+ * tandem.h - C boundary of the B200 (sm_100a) Tandem + SPEED greedy decoding library.
+ *
+ * The library implements the inference loop of "Tandem Transformers for Inference Efficient LLMs"
+ * (arXiv 2402.08644): a large decoder M_L that runs in block mode, a per-layer projection FF_Tandem
+ * that turns M_L's representations into keys/values of a small decoder M_S, M_S drafting gamma tokens
+ * autoregressively over that large-derived context plus its own keys/values, and M_L verifying the
+ * drafts (Section 3, Eq. 1 and Eq. 2; Section 3.1).
+ *
+ * Conventions common to every call
+ *  - Plain C types only.  Every pointer argument says whether it is a HOST or a DEVICE pointer.
+ *  - Every weight matrix is row-major [out_features][in_features] (y = x W^T), embedding / position
+ *    tables are [rows][d_model], the output head is [vocab][d_model].  Matrices and tables are in the
+ *    context's dtype (fp32 or bf16); LayerNorm gains and biases are always fp32.
+ *  - Model form (the paper leaves it open): pre-LayerNorm blocks with gain and bias, eps 1e-5,
+ *    exact GELU, no linear biases, learned absolute position embeddings, untied output head.
+ *  - Ownership: the caller owns the weights, the arena and every host buffer.  The library allocates
+ *    no device memory: all of its state (both KV caches, workspaces, device-side loop state) lives in
+ *    the caller's arena.  Weights and arena must stay valid until tandem_destroy.
+ *  - Errors: every call returns a tandem_status; nothing throws or aborts.  Arguments are validated
+ *    before any GPU work is launched; on error, out-parameters are left untouched.
+ *  - A context is bound to one device and one stream and is not thread-safe.  All GPU work is enqueued
+ *    on that stream.
+ *  - Greedy decisions: arg-max over fp32 logits, lowest token id on ties.
+ */
+#ifndef TANDEM_B200_H
+#define TANDEM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define TANDEM_API __attribute__((visibility("default")))
+#else
+#define TANDEM_API
+#endif
+
+typedef struct tandem_ctx tandem_ctx; /* opaque; one per (model pair, device) */
+
+typedef enum {
+    TANDEM_OK = 0,
+    TANDEM_ERR_INVALID_ARG = 1,     /* null pointer, negative size, unknown enum value */
+    TANDEM_ERR_SHAPE = 2,           /* unsupported dims (see tandem_create) */
+    TANDEM_ERR_ARENA_TOO_SMALL = 3,
+    TANDEM_ERR_CAPACITY = 4,        /* batch > max_batch, or positions would exceed max_seq / max_pos */
+    TANDEM_ERR_STATE = 5,           /* call order, e.g. a step before a prefill */
+    TANDEM_ERR_CUDA = 6,            /* a CUDA call failed; tandem_last_cuda_error() names it */
+    TANDEM_ERR_TIMEOUT = 7,         /* a bounded device-side wait expired */
+    TANDEM_ERR_UNIMPLEMENTED = 8
+} tandem_status;
+
+enum { TANDEM_DTYPE_FP32 = 0, TANDEM_DTYPE_BF16 = 1 };
+enum { TANDEM_FF_LINEAR = 0, TANDEM_FF_MLP = 1 };
+/* accept_mode: 0 = compare drafts with M_L's arg-max (Section 3.1); 1 = keep all gamma drafts (equals
+ * stand-alone Tandem with the free token, Figure 2); 2 = accept length drawn from a counter-based hash
+ * of (mode_seed, sequence, iteration), for tests of ragged accept lengths. */
+enum { TANDEM_ACCEPT_NATURAL = 0, TANDEM_ACCEPT_ALL = 1, TANDEM_ACCEPT_HASH = 2 };
+
+#define TANDEM_GAMMA_LIMIT 15 /* largest block length gamma a context can be created for */
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, d_ff, vocab, max_pos;
+} tandem_dims;
+
+typedef struct {
+    tandem_dims large, small;    /* M_L and M_S; both vocabularies must be equal */
+    int32_t ff_tandem_kind;      /* TANDEM_FF_LINEAR (the paper's choice, Section 3) or TANDEM_FF_MLP */
+    int32_t ff_tandem_hidden;    /* MLP only: hidden width; 0 = small.d_model */
+    const int32_t* layer_map;    /* HOST [small.n_layers]: l(j) of Eq. 2, the number of large layers after
+                                    which the residual stream feeds small layer j; 0 = embedding output;
+                                    values in [0, large.n_layers] */
+    int32_t dtype;               /* TANDEM_DTYPE_* : storage type of weights, activations and KV caches */
+    int32_t max_batch;           /* sequences per prefill */
+    int32_t max_seq;             /* KV-cache capacity in positions per sequence */
+    int32_t gamma_max;           /* largest gamma used with this context, 0..TANDEM_GAMMA_LIMIT */
+    int32_t max_prefill_rows;    /* workspace rows for the prompt pass; 0 = max_batch * max_seq */
+    int32_t device;              /* CUDA device ordinal */
+    void* stream;                /* cudaStream_t to enqueue on; NULL = the legacy default stream */
+} tandem_config;
+
+/* DEVICE pointers in this fixed order (n_ptrs must match):
+ *   for model in (large, small):  emb[V][d], pos[max_pos][d],
+ *       per layer: ln1_g[d], ln1_b[d], wq[d][d], wk[d][d], wv[d][d], wo[d][d], ln2_g[d], ln2_b[d],
+ *                  w1[d_ff][d], w2[d][d_ff],
+ *       lnf_g[d], lnf_b[d], w_out[V][d]
+ *   then per small layer j:  linear: w_t[d_S][d_L]      MLP: w_t1[hidden][d_L], w_t2[d_S][hidden]
+ * All pointers 16-byte aligned. */
+typedef struct {
+    const void* const* ptrs; /* HOST array of DEVICE pointers */
+    int32_t n_ptrs;
+} tandem_weights;
+
+/* HOST buffers owned by the caller; any member may be NULL (then it is not filled). */
+typedef struct {
+    int32_t* drafts;      /* [batch][gamma]      the small model's draft tokens d_1..d_gamma */
+    int32_t* targets;     /* [batch][gamma+1]    M_L's arg-max for the same positions and the next one */
+    int32_t* accept_len;  /* [batch]             number of drafts kept this iteration */
+    int32_t* n_committed; /* [batch]             committed tokens (prompt included) after the iteration */
+} tandem_step_result;
+
+typedef struct {
+    int64_t iterations;   /* draft+verify iterations run by the call */
+    int64_t large_runs;   /* M_L passes (one per iteration; the paper's "primary model runs", Table 6) */
+    int64_t small_runs;   /* M_S passes (gamma per iteration; "secondary model runs") */
+    int64_t emitted;      /* tokens returned over all sequences */
+    int64_t accept_hist[TANDEM_GAMMA_LIMIT + 1]; /* iterations of live sequences by accept length */
+    int64_t kernel_launches; /* kernels of this library enqueued by the call */
+} tandem_stats;
+
+/* Bytes of device memory tandem_create needs for this configuration (KV caches of both models,
+ * including the small model's large-derived region; workspaces; loop state). */
+TANDEM_API tandem_status tandem_query_arena(const tandem_config* cfg, size_t* bytes /* HOST out */);
+
+/* Builds a context over caller-owned weights and arena (DEVICE, 256-byte aligned, arena_bytes >= the
+ * queried size).  Supported shapes: d_model % n_heads == 0; head size 32, 64 or 128; d_model, d_ff and
+ * ff_tandem_hidden multiples of 8; max_batch * (gamma_max + 1) <= 256.  Zero-fills the arena's state. */
+TANDEM_API tandem_status tandem_create(const tandem_config* cfg, const tandem_weights* weights,
+                            void* arena /* DEVICE */, size_t arena_bytes, tandem_ctx** out /* HOST out */);
+
+/* Waits for the context's stream and releases host resources.  Never frees caller memory. */
+TANDEM_API tandem_status tandem_destroy(tandem_ctx* ctx);
+
+/* Prompt pass (Section 3 "Inference"; Figure 3): for each sequence b, M_L processes
+ * prompt[b][0 .. len_b-2] as a standard causal decoder (Eq. 1) and fills its KV cache; FF_Tandem and the
+ * small layers' key/value maps turn x^(l(j)) of those positions into the small model's large-derived
+ * keys/values (Eq. 2, first line).  The last prompt token becomes the pending token that M_S starts
+ * from.  Resets all per-sequence state.  prompt_ids: HOST, the prompts concatenated; prompt_lens:
+ * HOST [batch], each >= 1.  Needs len_b <= max_seq, <= both max_pos, and the total number of processed
+ * rows <= max_prefill_rows.  Asynchronous on the context's stream (the host arrays are copied before
+ * the call returns). */
+TANDEM_API tandem_status tandem_prefill(tandem_ctx* ctx, int32_t batch, const int32_t* prompt_ids,
+                             const int32_t* prompt_lens);
+
+/* One Tandem + SPEED iteration for every sequence (Section 3.1):
+ *   draft   M_S runs gamma times from the pending token; each step attends the large-derived keys/values
+ *           of positions M_L has processed plus M_S's own keys/values of the current block (Eq. 2);
+ *   verify  M_L processes the pending token and the gamma drafts as one block of gamma+1 rows (Eq. 1 in
+ *           block mode), extending its KV cache;
+ *   project FF_Tandem writes the small model's keys/values for the block's positions;
+ *   accept  per sequence: a = length of the longest prefix of drafts equal to M_L's arg-max; the sequence
+ *           gains d_1..d_a and M_L's token for the next position, which becomes pending; both caches
+ *           roll back to the kept positions (a length update; no data moves).
+ * 0 <= gamma <= gamma_max.  result may be NULL (the call is then asynchronous); filling it waits for
+ * the stream.  Fails with TANDEM_ERR_CAPACITY, launching nothing, if a sequence could outgrow max_seq. */
+TANDEM_API tandem_status tandem_block_step(tandem_ctx* ctx, int32_t gamma, int32_t accept_mode, uint64_t mode_seed,
+                                tandem_step_result* result /* HOST, nullable */);
+
+/* Repeats tandem_block_step until every sequence has max_new_tokens new tokens (surplus tokens of the
+ * last iteration are dropped; finished sequences stay frozen).  out_ids: HOST [batch][max_new_tokens];
+ * out_lens: HOST [batch] (nullable); stats: HOST, nullable.  Synchronous.  Must follow a prefill; may be
+ * called again to continue the same sequences. */
+TANDEM_API tandem_status tandem_speculative_generate(tandem_ctx* ctx, int32_t gamma, int32_t max_new_tokens,
+                                          int32_t accept_mode, uint64_t mode_seed, int32_t* out_ids,
+                                          int32_t* out_lens, tandem_stats* stats);
+
+/* Baseline and invariant hook: plain greedy decoding of M_L alone, one token per pass (the output that
+ * Tandem + SPEED must reproduce; abstract and Section 3.1).  Same buffers as above.  Leaves the small
+ * model's keys/values stale: call tandem_prefill again before the next speculative call. */
+TANDEM_API tandem_status tandem_large_greedy_generate(tandem_ctx* ctx, int32_t max_new_tokens, int32_t* out_ids,
+                                           int32_t* out_lens, tandem_stats* stats);
+
+/* Test hook: copies internal results of the LAST iteration to the host as fp32 / int32.  Synchronous.
+ *   what = 0  large logits      [batch][gamma+1][vocab]              (last verify pass)
+ *   what = 1  small logits      [gamma][batch][vocab]                (last draft steps)
+ *   what = 2  large hidden      [batch][gamma+1][d_large]            (final residual stream, last verify)
+ *   what = 3  large keys        [n][d_large]  for (layer, seq), n = positions M_L has processed
+ *   what = 4  large values      same
+ *   what = 5  small keys        [n][d_small]  for (layer, seq): the large-derived region
+ *   what = 6  small values      same
+ *   what = 7  committed counts  int32 [batch]
+ * bytes must equal the size of the selected item. */
+TANDEM_API tandem_status tandem_debug_read(tandem_ctx* ctx, int32_t what, int32_t layer, int32_t seq,
+                                void* host_dst, size_t bytes);
+
+/* Measurement hooks.  tandem_profile_enable(ctx, n > 0) brackets each of the next n kernel launches with a
+ * pair of CUDA events on the context's stream (this slows the stream down: never leave it on while timing
+ * throughput); n = 0 switches it off.  tandem_profile_read waits for the stream and sums, per kernel class
+ * (tandem_profile_class_name(i), i = 0 .. until it returns NULL), the elapsed milliseconds, the launches and
+ * the algorithmic work of the recorded launches (bytes for the memory-bound classes, flops for gemm_tiled),
+ * then clears the record.  ms, launches, work: HOST [n_classes].  tandem_launch_count: kernels enqueued by
+ * the context since tandem_create. */
+TANDEM_API tandem_status tandem_profile_enable(tandem_ctx* ctx, int32_t max_launches);
+TANDEM_API tandem_status tandem_profile_read(tandem_ctx* ctx, int32_t n_classes, double* ms, int64_t* launches,
+                                             double* work);
+TANDEM_API const char* tandem_profile_class_name(int32_t cls);
+TANDEM_API int64_t tandem_launch_count(tandem_ctx* ctx);
+
+/* Stand-alone kernels of the path (the attention / projection micro-benchmark).
+ *
+ * tandem_decode_attention: one query per (sequence, head) of the small model attends a mixed context
+ * (Eq. 2, second line): `derived_len` positions whose keys/values came from M_L through FF_Tandem,
+ * followed by `own_len` positions computed by M_S itself.  All pointers DEVICE, bf16.
+ *   q, out           [batch][n_heads][d_head]
+ *   k_derived, v_derived  [batch][n_heads][derived_len][d_head]
+ *   k_own, v_own     [batch][n_heads][own_len][d_head]
+ *   scratch          split-K partial results, fp32, at least tandem_decode_attention_scratch_bytes(...)
+ * d_head in {32, 64, 128}.  The context is cut into fixed chunks by absolute position; each chunk yields
+ * (max, sum, weighted values) and a second kernel merges the chunks in position order. */
+TANDEM_API size_t tandem_decode_attention_scratch_bytes(int32_t batch, int32_t n_heads, int32_t d_head,
+                                             int32_t derived_len, int32_t own_len);
+TANDEM_API tandem_status tandem_decode_attention(const void* q, const void* k_derived, const void* v_derived,
+                                      const void* k_own, const void* v_own, void* out, void* scratch,
+                                      size_t scratch_bytes, int32_t batch, int32_t n_heads, int32_t d_head,
+                                      int32_t derived_len, int32_t own_len, void* stream);
+
+/* tandem_ff_tandem_project: the linear FF_Tandem of Eq. 2 (first line) followed by the small layer's
+ * LayerNorm and key/value maps, written as bf16 keys/values.  All pointers DEVICE.
+ *   x [rows][d_large] bf16;  w_t [d_small][d_large] bf16;  ln_g, ln_b [d_small] fp32;
+ *   wk, wv [d_small][d_small] bf16;  k_out, v_out [rows][d_small] bf16;
+ *   scratch: fp32, at least rows * d_small * 4 + rows * d_small * 2 bytes.  rows <= 256. */
+TANDEM_API tandem_status tandem_ff_tandem_project(const void* x, const void* w_t, const void* ln_g, const void* ln_b,
+                                       const void* wk, const void* wv, void* k_out, void* v_out,
+                                       void* scratch, size_t scratch_bytes, int32_t rows, int32_t d_large,
+                                       int32_t d_small, void* stream);
+
+TANDEM_API const char* tandem_status_string(tandem_status s);
+/* Name of the last failing CUDA call's error for this thread (valid after TANDEM_ERR_CUDA). */
+TANDEM_API const char* tandem_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TANDEM_B200_H */

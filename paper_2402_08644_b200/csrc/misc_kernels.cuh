@@ -1,0 +1,155 @@
+// Row set-up, embedding, LayerNorm, casts, arg-max, and the verify / accept / rollback kernel.
+#pragma once
+#include <math.h>
+#include "common.cuh"
+
+namespace tandem {
+
+// Device-resident loop state (all int32 arrays live in the caller's arena).
+struct LoopState {
+    int* n;            // [B] committed tokens per sequence (prompt included); position n-1 is pending
+    int* pending;      // [B] the pending token c[n-1]
+    int* drafts;       // [B][gamma_limit]   d_1..d_gamma of the current iteration
+    int* targets;      // [B][gamma_limit+1] the large model's arg-max per block row
+    int* accept_len;   // [B]
+    int* emitted;      // [B] tokens written to out_ids since the generate call began
+    int* done;         // [B]
+    int* out_ids;      // [B][out_cap]
+    int* counters;     // [0] iteration index since prefill, [1] live sequences, [2] error flags,
+                       // [3] max_b n_b, [4] sum_b n_b (both refreshed by every verify)
+    unsigned long long* hist;   // [gamma_limit+1] accept-length histogram of live sequences
+    int out_cap;
+    int gamma_limit;
+};
+
+// Decode rows: sequence b contributes rows r0 .. r0+nq-1 of its block (row 0 = pending token, row r = draft r).
+// Row m = b*nq + (r - r0):  token, sequence, absolute position n_b - 1 + r.
+__global__ void setup_rows_kernel(LoopState st, int batch, int r0, int nq, int* row_tok, int* row_seq, int* row_pos) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= batch * nq) return;
+    const int b = m / nq, r = r0 + (m - b * nq);
+    row_tok[m] = (r == 0) ? st.pending[b] : st.drafts[b * st.gamma_limit + r - 1];
+    row_seq[m] = b;
+    row_pos[m] = st.n[b] - 1 + r;
+}
+
+// x^(0) = Emb(t) + Pos(index)  (Eq. 1); fp32 residual stream.  grid: rows; block: 128.
+template <typename T>
+__global__ void embed_kernel(const int* __restrict__ row_tok, const int* __restrict__ row_pos, const T* __restrict__ emb,
+                             const T* __restrict__ pos, float* __restrict__ h, int d) {
+    const int m = blockIdx.x;
+    const T* er = emb + (size_t)row_tok[m] * d;
+    const T* pr = pos + (size_t)row_pos[m] * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)m * d + i] = to_float(er[i]) + to_float(pr[i]);
+}
+
+__device__ __forceinline__ float block_sum_128(float v, float* red) {
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    return red[0] + red[1] + red[2] + red[3];
+}
+
+// LayerNorm of fp32 rows (biased variance, eps 1e-5), output in the storage type.  grid: rows; block: 128.
+template <typename T>
+__global__ void __launch_bounds__(128) layernorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+                                                        const float* __restrict__ bias, T* __restrict__ out, int d) {
+    __shared__ float red[4];
+    const float* xr = x + (size_t)blockIdx.x * d;
+    float s = 0.f;
+    for (int i = threadIdx.x; i < d; i += 128) s += xr[i];
+    const float mu = block_sum_128(s, red) / d;
+    float v = 0.f;
+    for (int i = threadIdx.x; i < d; i += 128) { const float c = xr[i] - mu; v = fmaf(c, c, v); }
+    const float rstd = 1.0f / sqrtf(block_sum_128(v, red) / d + 1e-5f);
+    for (int i = threadIdx.x; i < d; i += 128)
+        out[(size_t)blockIdx.x * d + i] = from_float<T>((xr[i] - mu) * rstd * gain[i] + bias[i]);
+}
+
+template <typename T>
+__global__ void cast_rows_kernel(const float* __restrict__ x, T* __restrict__ out, size_t n) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = from_float<T>(x[i]);
+}
+
+// Arg-max of fp32 rows, lowest index on ties.  grid: rows; block: 256.
+// Row m belongs to sequence m / nq; the result goes to dst[(m / nq) * seq_stride + m % nq + off].
+__global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restrict__ logits, int V, int* dst, int nq, int seq_stride, int off) {
+    __shared__ float sv[8];
+    __shared__ int si[8];
+    const float* lr = logits + (size_t)blockIdx.x * V;
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int i = threadIdx.x; i < V; i += 256) {
+        const float v = lr[i];
+        if (v > best || (v == best && i < bi)) { best = v; bi = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = best; si[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w)
+            if (sv[w] > best || (sv[w] == best && si[w] < bi)) { best = sv[w]; bi = si[w]; }
+        const int m = blockIdx.x;
+        dst[(size_t)(m / nq) * seq_stride + (m % nq) + off] = bi;
+    }
+}
+
+// Verify / accept / rollback (Section 3.1), one thread per sequence, one CTA.
+//   a = longest prefix of drafts equal to the large model's tokens (or forced);
+//   the sequence gains d_1..d_a and g_{a+1}; n advances; g_{a+1} becomes pending.
+// Rolling the caches back is the update of n: positions >= n-1 are rewritten by the next iteration.
+__global__ void verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed, int max_new) {
+    const int b = threadIdx.x;
+    const int iteration = st.counters[0];
+    __syncthreads();
+    if (b < batch && !st.done[b]) {
+        const int* d = st.drafts + b * st.gamma_limit;
+        const int* g = st.targets + b * (st.gamma_limit + 1);
+        int a = 0;
+        if (mode == 1) a = gamma;
+        else if (mode == 2) a = (int)(splitmix64(splitmix64(splitmix64(seed) ^ (unsigned long long)b) ^ (unsigned long long)iteration) % (unsigned long long)(gamma + 1));
+        else { while (a < gamma && d[a] == g[a]) ++a; }
+        st.accept_len[b] = a;
+        atomicAdd(st.hist + a, 1ull);
+        const int em = st.emitted[b];
+        const int room = max_new - em;
+        const int take = min(a + 1, room);
+        int last = st.pending[b];
+        for (int i = 0; i < take; ++i) {
+            last = (i < a) ? d[i] : g[a];
+            if (em + i < st.out_cap) st.out_ids[(size_t)b * st.out_cap + em + i] = last;
+        }
+        st.emitted[b] = em + take;
+        st.n[b] += take;
+        st.pending[b] = last;
+        if (em + take >= max_new) { st.done[b] = 1; atomicSub(st.counters + 1, 1); }
+    }
+    __syncthreads();
+    if (b == 0) {
+        st.counters[0] = iteration + 1;
+        int n_max = 0, n_sum = 0;
+        for (int i = 0; i < batch; ++i) { n_max = max(n_max, st.n[i]); n_sum += st.n[i]; }
+        st.counters[3] = n_max;
+        st.counters[4] = n_sum;
+    }
+}
+
+// Test hook: gathers K or V of one (layer, sequence) from [H][t_max][dh] into fp32 [n][H*dh].
+template <typename T>
+__global__ void gather_kv_kernel(const T* __restrict__ cache_seq, float* __restrict__ dst, int n, int n_heads, int d_head, int t_max) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int d = n_heads * d_head;
+    if (i >= (size_t)n * d) return;
+    const int t = (int)(i / d), c = (int)(i - (size_t)t * d);
+    const int h = c / d_head, el = c - h * d_head;
+    dst[i] = to_float(cache_seq[((size_t)h * t_max + t) * d_head + el]);
+}
+
+}  // namespace tandem

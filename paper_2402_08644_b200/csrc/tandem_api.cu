@@ -1,0 +1,911 @@
+// Host side of the C boundary: context, arena layout, pass scheduling, and the exported entry points.
+#include <cuda_runtime.h>
+#include <limits.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "../../include/tandem.h"
+#include "attention.cuh"
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "misc_kernels.cuh"
+
+using namespace tandem;
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+#define CK(call)                                                                                  \
+    do {                                                                                          \
+        cudaError_t err__ = (call);                                                               \
+        if (err__ != cudaSuccess) {                                                               \
+            snprintf(g_cuda_err, sizeof(g_cuda_err), "%s at %s:%d", cudaGetErrorString(err__), __FILE__, __LINE__); \
+            return TANDEM_ERR_CUDA;                                                               \
+        }                                                                                         \
+    } while (0)
+#define TRY(expr)                             \
+    do {                                      \
+        tandem_status st__ = (expr);          \
+        if (st__ != TANDEM_OK) return st__;   \
+    } while (0)
+
+size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+struct Layout {   // byte offsets into the arena
+    size_t kv_large, kv_small;
+    size_t st_n, st_pending, st_drafts, st_targets, st_accept, st_emitted, st_done, st_out, st_counters, st_hist;
+    size_t row_tok, row_seq, row_pos, grp_row0, grp_cnt;
+    size_t h_large, h_small, a, q, o, f, xb, t1, yhat, a_s, logits_large, logits_small, part_ml, part_acc, dbg;
+    size_t total;
+    int max_rows, dec_rows, max_groups, n_chunks_max;
+    size_t kv_large_layer, kv_small_layer;   // elements per (layer, k-or-v)
+};
+
+struct Model {
+    tandem_dims d;
+    int wbase;
+    size_t kv_off;          // arena offset of this model's KV cache
+    size_t kv_layer_elems;  // elements per (layer, K or V): B * H * T * dh
+};
+
+}  // namespace
+
+enum { PC_GEMM_SMALLM = 0, PC_GEMM_TILED, PC_ATTN_SPLIT, PC_ATTN_MERGE, PC_ATTN_PROMPT, PC_LAYERNORM, PC_ROWS, PC_ARGMAX,
+       PC_VERIFY, PC_COUNT };
+
+struct Prof {   // optional per-launch timing with CUDA events (measurement hook)
+    bool on = false;
+    std::vector<cudaEvent_t> ev;
+    std::vector<int> cls;
+    std::vector<double> bytes;
+    size_t used = 0;   // events used (two per launch)
+};
+
+struct tandem_ctx {
+    Prof prof;
+    tandem_config cfg;
+    std::vector<int32_t> layer_map;
+    std::vector<const void*> w;
+    Layout lay;
+    Model large, small;
+    int tbase;          // first FF_Tandem weight index
+    int hidden;
+    unsigned char* arena;
+    cudaStream_t stream;
+    size_t esz;         // storage element size
+    // host trackers
+    int batch;          // sequences of the current prefill (0 = none)
+    int n_ub;           // upper bound on max_b n_b (exact after every synchronising call)
+    long long n_sum;    // sum_b n_b at the last synchronisation (accounting only)
+    int32_t* pinned;    // staging for prefill row arrays and small read-backs
+    size_t pinned_ints;
+    int64_t launches = 0;
+    int last_gamma = 0;
+    LoopState st;
+};
+
+namespace {
+// Brackets one launch with two events when profiling is on.
+struct ProfScope {
+    tandem_ctx& c;
+    bool active;
+    ProfScope(tandem_ctx& ctx, int cls, double bytes) : c(ctx), active(false) {
+        Prof& p = c.prof;
+        if (p.on && p.used + 2 <= p.ev.size()) {
+            active = true;
+            p.cls.push_back(cls);
+            p.bytes.push_back(bytes);
+            cudaEventRecord(p.ev[p.used], c.stream);
+        }
+    }
+    ~ProfScope() {
+        if (active) { cudaEventRecord(c.prof.ev[c.prof.used + 1], c.stream); c.prof.used += 2; }
+    }
+};
+}  // namespace
+
+namespace {
+
+int dims_ok(const tandem_dims& d) {
+    if (d.n_layers < 1 || d.d_model < 8 || d.n_heads < 1 || d.d_ff < 8 || d.vocab < 1 || d.max_pos < 1) return 0;
+    if (d.d_model % d.n_heads) return 0;
+    const int dh = d.d_model / d.n_heads;
+    if (dh != 32 && dh != 64 && dh != 128) return 0;
+    if (d.d_model % 8 || d.d_ff % 8) return 0;
+    return 1;
+}
+
+tandem_status validate(const tandem_config* c) {
+    if (!c || !c->layer_map) return TANDEM_ERR_INVALID_ARG;
+    if (c->dtype != TANDEM_DTYPE_FP32 && c->dtype != TANDEM_DTYPE_BF16) return TANDEM_ERR_INVALID_ARG;
+    if (c->ff_tandem_kind != TANDEM_FF_LINEAR && c->ff_tandem_kind != TANDEM_FF_MLP) return TANDEM_ERR_INVALID_ARG;
+    if (c->max_batch < 1 || c->max_seq < 2 || c->gamma_max < 0 || c->gamma_max > TANDEM_GAMMA_LIMIT) return TANDEM_ERR_INVALID_ARG;
+    if (c->max_prefill_rows < 0 || c->ff_tandem_hidden < 0 || c->device < 0) return TANDEM_ERR_INVALID_ARG;
+    if (!dims_ok(c->large) || !dims_ok(c->small)) return TANDEM_ERR_SHAPE;
+    if (c->large.vocab != c->small.vocab) return TANDEM_ERR_SHAPE;
+    if (c->ff_tandem_hidden % 8) return TANDEM_ERR_SHAPE;
+    if ((long long)c->max_batch * (c->gamma_max + 1) > 256) return TANDEM_ERR_SHAPE;
+    for (int j = 0; j < c->small.n_layers; ++j)
+        if (c->layer_map[j] < 0 || c->layer_map[j] > c->large.n_layers) return TANDEM_ERR_INVALID_ARG;
+    return TANDEM_OK;
+}
+
+Layout make_layout(const tandem_config& c) {
+    Layout L;
+    memset(&L, 0, sizeof(L));
+    const size_t esz = c.dtype == TANDEM_DTYPE_BF16 ? 2 : 4;
+    const size_t B = c.max_batch, T = c.max_seq, GL = TANDEM_GAMMA_LIMIT;
+    const int hidden = c.ff_tandem_hidden > 0 ? c.ff_tandem_hidden : c.small.d_model;
+    L.dec_rows = c.max_batch * (c.gamma_max + 1);
+    const long long pre = c.max_prefill_rows > 0 ? c.max_prefill_rows : (long long)c.max_batch * c.max_seq;
+    L.max_rows = (int)std::max<long long>(pre, L.dec_rows);
+    L.max_groups = L.max_rows / ATT_NQ + c.max_batch + 1;
+    L.n_chunks_max = cdiv(c.max_seq, ATT_CH);
+    const size_t dmax = std::max(std::max(c.large.d_model, c.small.d_model), hidden);
+    const size_t fmax = std::max(c.large.d_ff, c.small.d_ff);
+    const size_t hmax = std::max(c.large.n_heads, c.small.n_heads);
+    const size_t R = L.max_rows, RD = L.dec_rows, V = c.large.vocab;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    L.kv_large_layer = B * T * c.large.d_model;
+    L.kv_small_layer = B * T * c.small.d_model;
+    L.kv_large = take((size_t)c.large.n_layers * 2 * L.kv_large_layer * esz);
+    L.kv_small = take((size_t)c.small.n_layers * 2 * L.kv_small_layer * esz);
+    L.st_n = take(B * 4); L.st_pending = take(B * 4); L.st_drafts = take(B * GL * 4);
+    L.st_targets = take(B * (GL + 1) * 4); L.st_accept = take(B * 4); L.st_emitted = take(B * 4);
+    L.st_done = take(B * 4); L.st_out = take(B * T * 4); L.st_counters = take(16 * 4); L.st_hist = take((GL + 1) * 8);
+    L.row_tok = take(R * 4); L.row_seq = take(R * 4); L.row_pos = take(R * 4);
+    L.grp_row0 = take((size_t)L.max_groups * 4); L.grp_cnt = take((size_t)L.max_groups * 4);
+    L.h_large = take(R * c.large.d_model * 4);
+    L.h_small = take(B * c.small.d_model * 4);
+    L.a = take(R * dmax * esz); L.q = take(R * dmax * esz); L.o = take(R * dmax * esz);
+    L.f = take(R * fmax * esz);
+    L.xb = take(R * c.large.d_model * esz); L.t1 = take(R * hidden * esz);
+    L.yhat = take(R * c.small.d_model * 4); L.a_s = take(R * c.small.d_model * esz);
+    L.logits_large = take(RD * V * 4);
+    L.logits_small = take((size_t)std::max(1, c.gamma_max) * B * V * 4);
+    L.part_ml = take(RD * hmax * L.n_chunks_max * 2 * 4);
+    L.part_acc = take(RD * dmax * L.n_chunks_max * 4);
+    L.dbg = take(T * dmax * 4);
+    L.total = off;
+    return L;
+}
+
+int n_weight_ptrs(const tandem_config& c) {
+    const int per_t = c.ff_tandem_kind == TANDEM_FF_LINEAR ? 1 : 2;
+    return (5 + 10 * c.large.n_layers) + (5 + 10 * c.small.n_layers) + per_t * c.small.n_layers;
+}
+
+enum { W_LN1G = 0, W_LN1B, W_WQ, W_WK, W_WV, W_WO, W_LN2G, W_LN2B, W_W1, W_W2 };
+inline const void* w_emb(const tandem_ctx& c, const Model& m) { return c.w[m.wbase]; }
+inline const void* w_pos(const tandem_ctx& c, const Model& m) { return c.w[m.wbase + 1]; }
+inline const void* w_layer(const tandem_ctx& c, const Model& m, int l, int k) { return c.w[m.wbase + 2 + 10 * l + k]; }
+inline const void* w_tail(const tandem_ctx& c, const Model& m, int k) { return c.w[m.wbase + 2 + 10 * m.d.n_layers + k]; }
+inline const void* w_tandem(const tandem_ctx& c, int j, int k) {
+    return c.w[c.tbase + (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR ? j : 2 * j + k)];
+}
+
+template <typename P> P* at(tandem_ctx& c, size_t off) { return reinterpret_cast<P*>(c.arena + off); }
+
+constexpr int MAX_DEVICES = 64;
+int cur_dev() {   // opt-in shared-memory sizes are per device
+    int d = 0;
+    cudaGetDevice(&d);
+    return (d >= 0 && d < MAX_DEVICES) ? d : 0;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// launch helpers
+// ---------------------------------------------------------------------------------------------------
+
+template <typename T, int MT, int EPI>
+void launch_smallm(tandem_ctx& c, const T* x, int ldx, int M, int K, const WSegs& ws, int N, const EpiArgs& e) {
+    static bool attr_set[MAX_DEVICES] = {};
+    const size_t smem = (size_t)MT * GS_KC * sizeof(T);
+    const int dev = cur_dev();
+    if (!attr_set[dev]) {
+        cudaFuncSetAttribute(gemm_smallm_kernel<T, MT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_set[dev] = true;
+    }
+    dim3 grid(cdiv(N, GS_WARPS * GS_COLS), cdiv(M, MT));
+    ProfScope ps(c, PC_GEMM_SMALLM, ((double)N * K + (double)M * K + (double)M * N) * sizeof(T));
+    gemm_smallm_kernel<T, MT, EPI><<<grid, GS_THREADS, smem, c.stream>>>(x, ldx, M, K, ws, N, e);
+    c.launches++;
+}
+
+template <typename T, int EPI>
+void launch_gemm(tandem_ctx& c, bool decode, const T* x, int ldx, int M, int K, const WSegs& ws, int N, const EpiArgs& e) {
+    if (M <= 0) return;
+    if (decode) {
+        if (M <= 1) launch_smallm<T, 1, EPI>(c, x, ldx, M, K, ws, N, e);
+        else if (M <= 2) launch_smallm<T, 2, EPI>(c, x, ldx, M, K, ws, N, e);
+        else if (M <= 4) launch_smallm<T, 4, EPI>(c, x, ldx, M, K, ws, N, e);
+        else launch_smallm<T, 8, EPI>(c, x, ldx, M, K, ws, N, e);
+    } else {
+        dim3 grid(cdiv(N, GT_BN), cdiv(M, GT_BM));
+        ProfScope ps(c, PC_GEMM_TILED, 2.0 * M * (double)N * K);   // flops, not bytes: this one is compute-bound
+        gemm_tiled_kernel<T, EPI><<<grid, GT_THREADS, 0, c.stream>>>(x, ldx, M, K, ws, N, e);
+        c.launches++;
+    }
+}
+
+WSegs segs1(const void* w, int n) { WSegs s; s.w[0] = w; s.w[1] = s.w[2] = nullptr; s.seg_rows = n; return s; }
+WSegs segs3(const void* a, const void* b, const void* c3, int n) { WSegs s; s.w[0] = a; s.w[1] = b; s.w[2] = c3; s.seg_rows = n; return s; }
+
+template <typename T, int DH>
+void set_attn_attrs() {
+    cudaFuncSetAttribute(attn_kernel<T, DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<T, DH>());
+    cudaFuncSetAttribute(attn_kernel<T, DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<T, DH>());
+}
+
+template <typename T, int DH>
+void launch_attn_dh(tandem_ctx& c, const AttnArgs& a, int M, int groups, bool loop, int n_chunks, double kv_bytes) {
+    static bool attr_set[MAX_DEVICES] = {};
+    const int dev = cur_dev();
+    cudaStream_t s = c.stream;
+    if (!attr_set[dev]) { set_attn_attrs<T, DH>(); attr_set[dev] = true; }
+    if (loop) {
+        ProfScope ps(c, PC_ATTN_PROMPT, kv_bytes);
+        attn_kernel<T, DH, true><<<dim3(1, a.n_heads, groups), ATT_THREADS, attn_smem_bytes<T, DH>(), s>>>(a);
+        c.launches += 1;
+    } else {
+        {
+            ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
+            attn_kernel<T, DH, false><<<dim3(n_chunks, a.n_heads, groups), ATT_THREADS, attn_smem_bytes<T, DH>(), s>>>(a);
+        }
+        ProfScope ps(c, PC_ATTN_MERGE, (double)M * a.n_heads * n_chunks * (DH + 2) * 4.0);
+        attn_merge_kernel<T, DH><<<dim3(M, a.n_heads), DH, 0, s>>>(a);
+        c.launches += 2;
+    }
+}
+
+template <typename T>
+void launch_attn(tandem_ctx& c, int d_head, const AttnArgs& a, int M, int groups, bool loop, int n_chunks, double kv_bytes) {
+    if (d_head == 32) launch_attn_dh<T, 32>(c, a, M, groups, loop, n_chunks, kv_bytes);
+    else if (d_head == 64) launch_attn_dh<T, 64>(c, a, M, groups, loop, n_chunks, kv_bytes);
+    else launch_attn_dh<T, 128>(c, a, M, groups, loop, n_chunks, kv_bytes);
+}
+
+template <typename T>
+void launch_layernorm(tandem_ctx& c, int M, const float* x, const void* gain, const void* bias, T* out, int d) {
+    ProfScope ps(c, PC_LAYERNORM, (double)M * d * (4.0 + sizeof(T)));
+    layernorm_kernel<T><<<M, 128, 0, c.stream>>>(x, static_cast<const float*>(gain), static_cast<const float*>(bias), out, d);
+    c.launches++;
+}
+
+// Describes the rows of one pass.
+struct Rows {
+    int M;            // rows
+    int groups;       // attention groups
+    int nq;           // rows per group when group arrays are not used (decode)
+    bool decode;      // decode kernels (split attention, streaming GEMM) or prompt kernels
+    int n_chunks;     // split attention grid size along the context
+    double kv_positions;   // context positions read by one attention launch, summed over sequences (accounting only)
+};
+
+template <typename T>
+T* kv_ptr(tandem_ctx& c, const Model& m, int layer, int which) {
+    return at<T>(c, m.kv_off) + ((size_t)layer * 2 + which) * m.kv_layer_elems;
+}
+
+EpiArgs epi_plain(void* out, int ldo) {
+    EpiArgs e; memset(&e, 0, sizeof(e)); e.out = out; e.ldo = ldo; return e;
+}
+
+template <typename T>
+EpiArgs epi_cache(tandem_ctx& c, const Model& m, int layer, void* q_out) {
+    EpiArgs e; memset(&e, 0, sizeof(e));
+    e.out = q_out; e.ldo = m.d.d_model;
+    e.kcache = kv_ptr<T>(c, m, layer, 0); e.vcache = kv_ptr<T>(c, m, layer, 1);
+    e.row_seq = at<int>(c, c.lay.row_seq); e.row_pos = at<int>(c, c.lay.row_pos);
+    e.n_heads = m.d.n_heads; e.d_head = m.d.d_model / m.d.n_heads; e.t_max = c.cfg.max_seq; e.seg = m.d.d_model;
+    return e;
+}
+
+// Eq. 2, first line, for small layer j, then that layer's LayerNorm and key/value maps: writes the
+// small model's large-derived keys/values for the rows' positions.
+template <typename T>
+void project_layer(tandem_ctx& c, int j, const Rows& r) {
+    const int dL = c.large.d.d_model, dS = c.small.d.d_model;
+    T* xb = at<T>(c, c.lay.xb);
+    float* yhat = at<float>(c, c.lay.yhat);
+    T* a_s = at<T>(c, c.lay.a_s);
+    if (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR) {
+        launch_gemm<T, EPI_STORE_F32>(c, r.decode, xb, dL, r.M, dL, segs1(w_tandem(c, j, 0), dS), dS, epi_plain(yhat, dS));
+    } else {
+        T* t1 = at<T>(c, c.lay.t1);
+        launch_gemm<T, EPI_GELU>(c, r.decode, xb, dL, r.M, dL, segs1(w_tandem(c, j, 0), c.hidden), c.hidden, epi_plain(t1, c.hidden));
+        launch_gemm<T, EPI_STORE_F32>(c, r.decode, t1, c.hidden, r.M, c.hidden, segs1(w_tandem(c, j, 1), dS), dS, epi_plain(yhat, dS));
+    }
+    launch_layernorm<T>(c, r.M, yhat, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), a_s, dS);
+    launch_gemm<T, EPI_KV>(c, r.decode, a_s, dS, r.M, dS,
+                           segs3(w_layer(c, c.small, j, W_WK), w_layer(c, c.small, j, W_WV), nullptr, dS), 2 * dS,
+                           epi_cache<T>(c, c.small, j, nullptr));
+}
+
+template <typename T>
+void project_after(tandem_ctx& c, int n_large_layers_done, const Rows& r) {
+    bool any = false;
+    for (int j = 0; j < c.small.d.n_layers; ++j) any |= (c.layer_map[j] == n_large_layers_done);
+    if (!any) return;
+    const size_t n = (size_t)r.M * c.large.d.d_model;
+    {
+        ProfScope ps(c, PC_ROWS, (double)n * (4.0 + sizeof(T)));
+        cast_rows_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, c.stream>>>(at<float>(c, c.lay.h_large), at<T>(c, c.lay.xb), n);
+        c.launches++;
+    }
+    for (int j = 0; j < c.small.d.n_layers; ++j)
+        if (c.layer_map[j] == n_large_layers_done) project_layer<T>(c, j, r);
+}
+
+// One decoder layer (Eq. 1; the same form serves the small model's layers in Eq. 2) on residual stream h.
+template <typename T>
+void decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r) {
+    const int d = m.d.d_model, dff = m.d.d_ff, H = m.d.n_heads, dh = d / H;
+    T* a = at<T>(c, c.lay.a);
+    T* q = at<T>(c, c.lay.q);
+    T* o = at<T>(c, c.lay.o);
+    T* f = at<T>(c, c.lay.f);
+    launch_layernorm<T>(c, r.M, h, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), a, d);
+    launch_gemm<T, EPI_QKV>(c, r.decode, a, d, r.M, d, segs3(w_layer(c, m, l, W_WQ), w_layer(c, m, l, W_WK), w_layer(c, m, l, W_WV), d),
+                            3 * d, epi_cache<T>(c, m, l, q));
+    AttnArgs aa; memset(&aa, 0, sizeof(aa));
+    aa.q = q; aa.ldq = d; aa.kcache = kv_ptr<T>(c, m, l, 0); aa.vcache = kv_ptr<T>(c, m, l, 1);
+    aa.out = o; aa.ldo = d; aa.row_seq = at<int>(c, c.lay.row_seq); aa.row_pos = at<int>(c, c.lay.row_pos);
+    if (!r.decode) { aa.grp_row0 = at<int>(c, c.lay.grp_row0); aa.grp_cnt = at<int>(c, c.lay.grp_cnt); }
+    aa.nq = r.nq; aa.n_heads = H; aa.t_max = c.cfg.max_seq;
+    aa.part_ml = at<float>(c, c.lay.part_ml); aa.part_acc = at<float>(c, c.lay.part_acc);
+    aa.n_chunks_max = c.lay.n_chunks_max; aa.scale = 1.0f / sqrtf((float)dh);
+    launch_attn<T>(c, dh, aa, r.M, r.groups, !r.decode, r.n_chunks, r.kv_positions * 2.0 * d * sizeof(T));
+    launch_gemm<T, EPI_RESID>(c, r.decode, o, d, r.M, d, segs1(w_layer(c, m, l, W_WO), d), d, epi_plain(h, d));
+    launch_layernorm<T>(c, r.M, h, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), a, d);
+    launch_gemm<T, EPI_GELU>(c, r.decode, a, d, r.M, d, segs1(w_layer(c, m, l, W_W1), dff), dff, epi_plain(f, dff));
+    launch_gemm<T, EPI_RESID>(c, r.decode, f, dff, r.M, dff, segs1(w_layer(c, m, l, W_W2), d), d, epi_plain(h, d));
+}
+
+// Final LayerNorm, output head, arg-max.  dst[(m / nq) * seq_stride + m % nq + off].
+template <typename T>
+void head_argmax(tandem_ctx& c, const Model& m, float* h, const Rows& r, float* logits, int* dst, int seq_stride, int off) {
+    const int d = m.d.d_model, V = m.d.vocab;
+    T* a = at<T>(c, c.lay.a);
+    launch_layernorm<T>(c, r.M, h, w_tail(c, m, 0), w_tail(c, m, 1), a, d);
+    launch_gemm<T, EPI_STORE_F32>(c, r.decode, a, d, r.M, d, segs1(w_tail(c, m, 2), V), V, epi_plain(logits, V));
+    ProfScope ps(c, PC_ARGMAX, (double)r.M * V * 4.0);
+    argmax_rows_kernel<<<r.M, 256, 0, c.stream>>>(logits, V, dst, r.nq, seq_stride, off);
+    c.launches++;
+}
+
+// The large model over the current rows (block mode in decode, whole prompt otherwise).
+template <typename T>
+void large_pass(tandem_ctx& c, const Rows& r, bool project, bool head) {
+    float* h = at<float>(c, c.lay.h_large);
+    {
+        ProfScope ps(c, PC_ROWS, (double)r.M * c.large.d.d_model * (4.0 + 2 * sizeof(T)));
+        embed_kernel<T><<<r.M, 128, 0, c.stream>>>(at<int>(c, c.lay.row_tok), at<int>(c, c.lay.row_pos), (const T*)w_emb(c, c.large),
+                                                   (const T*)w_pos(c, c.large), h, c.large.d.d_model);
+        c.launches++;
+    }
+    if (project) project_after<T>(c, 0, r);
+    for (int l = 0; l < c.large.d.n_layers; ++l) {
+        decoder_layer<T>(c, c.large, l, h, r);
+        if (project) project_after<T>(c, l + 1, r);
+    }
+    if (head)
+        head_argmax<T>(c, c.large, h, r, at<float>(c, c.lay.logits_large), c.st.targets, TANDEM_GAMMA_LIMIT + 1, 0);
+}
+
+Rows decode_rows(tandem_ctx& c, int r_last, int nq) {
+    Rows r;
+    r.M = c.batch * nq; r.groups = c.batch; r.nq = nq; r.decode = true;
+    r.n_chunks = std::min(c.lay.n_chunks_max, (c.n_ub - 1 + r_last) / ATT_CH + 1);
+    r.kv_positions = (double)c.n_sum + (double)c.batch * r_last;
+    return r;
+}
+
+void setup_rows(tandem_ctx& c, int r0, int nq) {
+    const int M = c.batch * nq;
+    ProfScope ps(c, PC_ROWS, (double)M * 12.0);
+    setup_rows_kernel<<<cdiv(M, 128), 128, 0, c.stream>>>(c.st, c.batch, r0, nq, at<int>(c, c.lay.row_tok), at<int>(c, c.lay.row_seq), at<int>(c, c.lay.row_pos));
+    c.launches++;
+}
+
+// Draft step s: one token per sequence through the small model over the mixed context (Eq. 2, lines 2-3).
+template <typename T>
+void small_step(tandem_ctx& c, int s) {
+    setup_rows(c, s, 1);
+    Rows r = decode_rows(c, s, 1);
+    float* y = at<float>(c, c.lay.h_small);
+    {
+        ProfScope ps(c, PC_ROWS, (double)r.M * c.small.d.d_model * (4.0 + 2 * sizeof(T)));
+        embed_kernel<T><<<r.M, 128, 0, c.stream>>>(at<int>(c, c.lay.row_tok), at<int>(c, c.lay.row_pos), (const T*)w_emb(c, c.small),
+                                                   (const T*)w_pos(c, c.small), y, c.small.d.d_model);
+        c.launches++;
+    }
+    for (int j = 0; j < c.small.d.n_layers; ++j) decoder_layer<T>(c, c.small, j, y, r);
+    float* logits = at<float>(c, c.lay.logits_small) + (size_t)s * c.batch * c.small.d.vocab;
+    head_argmax<T>(c, c.small, y, r, logits, c.st.drafts, TANDEM_GAMMA_LIMIT, s);
+}
+
+template <typename T>
+void iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
+    for (int s = 0; s < gamma; ++s) small_step<T>(c, s);
+    setup_rows(c, 0, gamma + 1);
+    large_pass<T>(c, decode_rows(c, gamma, gamma + 1), true, true);
+    {
+        ProfScope ps(c, PC_VERIFY, (double)c.batch * (2 * gamma + 8) * 4.0);
+        verify_kernel<<<1, 256, 0, c.stream>>>(c.st, c.batch, gamma, mode, seed, max_new);
+        c.launches++;
+    }
+    c.last_gamma = gamma;
+}
+
+template <typename T>
+void greedy_iteration(tandem_ctx& c, int max_new) {
+    setup_rows(c, 0, 1);
+    large_pass<T>(c, decode_rows(c, 0, 1), false, true);
+    {
+        ProfScope ps(c, PC_VERIFY, (double)c.batch * 8 * 4.0);
+        verify_kernel<<<1, 256, 0, c.stream>>>(c.st, c.batch, 0, 0, 0ull, max_new);
+        c.launches++;
+    }
+    c.last_gamma = 0;
+}
+
+tandem_status check_launch() {
+    CK(cudaGetLastError());
+    return TANDEM_OK;
+}
+
+tandem_status begin_call(tandem_ctx* c) {
+    if (!c) return TANDEM_ERR_INVALID_ARG;
+    CK(cudaSetDevice(c->cfg.device));
+    return TANDEM_OK;
+}
+
+__global__ void reset_call_kernel(LoopState st, int batch) {
+    const int b = threadIdx.x;
+    if (b < batch) { st.emitted[b] = 0; st.done[b] = 0; }
+    if (b == 0) st.counters[1] = batch;
+}
+
+}  // namespace
+
+// =====================================================================================================
+// exported entry points
+// =====================================================================================================
+
+extern "C" const char* tandem_status_string(tandem_status s) {
+    switch (s) {
+        case TANDEM_OK: return "ok";
+        case TANDEM_ERR_INVALID_ARG: return "invalid argument";
+        case TANDEM_ERR_SHAPE: return "unsupported shape";
+        case TANDEM_ERR_ARENA_TOO_SMALL: return "arena too small";
+        case TANDEM_ERR_CAPACITY: return "capacity exceeded";
+        case TANDEM_ERR_STATE: return "call out of order";
+        case TANDEM_ERR_CUDA: return "CUDA error";
+        case TANDEM_ERR_TIMEOUT: return "device wait timed out";
+        case TANDEM_ERR_UNIMPLEMENTED: return "not implemented";
+    }
+    return "unknown status";
+}
+
+extern "C" const char* tandem_last_cuda_error(void) { return g_cuda_err; }
+
+extern "C" tandem_status tandem_query_arena(const tandem_config* cfg, size_t* bytes) {
+    if (!bytes) return TANDEM_ERR_INVALID_ARG;
+    TRY(validate(cfg));
+    *bytes = make_layout(*cfg).total;
+    return TANDEM_OK;
+}
+
+extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_weights* weights, void* arena,
+                                       size_t arena_bytes, tandem_ctx** out) {
+    if (!out || !weights || !weights->ptrs || !arena) return TANDEM_ERR_INVALID_ARG;
+    TRY(validate(cfg));
+    if (weights->n_ptrs != n_weight_ptrs(*cfg)) return TANDEM_ERR_INVALID_ARG;
+    for (int i = 0; i < weights->n_ptrs; ++i)
+        if (!weights->ptrs[i] || ((uintptr_t)weights->ptrs[i] & 15)) return TANDEM_ERR_INVALID_ARG;
+    if ((uintptr_t)arena & 255) return TANDEM_ERR_INVALID_ARG;
+    Layout lay = make_layout(*cfg);
+    if (arena_bytes < lay.total) return TANDEM_ERR_ARENA_TOO_SMALL;
+    CK(cudaSetDevice(cfg->device));
+
+    tandem_ctx* c = new (std::nothrow) tandem_ctx();
+    if (!c) return TANDEM_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->layer_map.assign(cfg->layer_map, cfg->layer_map + cfg->small.n_layers);
+    c->cfg.layer_map = c->layer_map.data();
+    c->w.assign(weights->ptrs, weights->ptrs + weights->n_ptrs);
+    c->lay = lay;
+    c->arena = static_cast<unsigned char*>(arena);
+    c->stream = static_cast<cudaStream_t>(cfg->stream);
+    c->esz = cfg->dtype == TANDEM_DTYPE_BF16 ? 2 : 4;
+    c->hidden = cfg->ff_tandem_hidden > 0 ? cfg->ff_tandem_hidden : cfg->small.d_model;
+    c->large.d = cfg->large; c->large.wbase = 0; c->large.kv_off = lay.kv_large; c->large.kv_layer_elems = lay.kv_large_layer;
+    c->small.d = cfg->small; c->small.wbase = 5 + 10 * cfg->large.n_layers; c->small.kv_off = lay.kv_small; c->small.kv_layer_elems = lay.kv_small_layer;
+    c->tbase = c->small.wbase + 5 + 10 * cfg->small.n_layers;
+    c->batch = 0; c->n_ub = 0; c->launches = 0; c->last_gamma = 0;
+    c->pinned_ints = (size_t)3 * lay.max_rows + 2 * lay.max_groups + 4 * cfg->max_batch + 64;
+    c->pinned = nullptr;
+    LoopState& st = c->st;
+    st.n = at<int>(*c, lay.st_n); st.pending = at<int>(*c, lay.st_pending); st.drafts = at<int>(*c, lay.st_drafts);
+    st.targets = at<int>(*c, lay.st_targets); st.accept_len = at<int>(*c, lay.st_accept); st.emitted = at<int>(*c, lay.st_emitted);
+    st.done = at<int>(*c, lay.st_done); st.out_ids = at<int>(*c, lay.st_out); st.counters = at<int>(*c, lay.st_counters);
+    st.hist = at<unsigned long long>(*c, lay.st_hist);
+    st.out_cap = cfg->max_seq; st.gamma_limit = TANDEM_GAMMA_LIMIT;
+    cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&c->pinned), c->pinned_ints * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->arena + lay.st_n, 0, lay.h_large - lay.st_n, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "%s in tandem_create", cudaGetErrorString(e));
+        if (c->pinned) cudaFreeHost(c->pinned);
+        delete c;
+        return TANDEM_ERR_CUDA;
+    }
+    *out = c;
+    return TANDEM_OK;
+}
+
+extern "C" tandem_status tandem_destroy(tandem_ctx* c) {
+    if (!c) return TANDEM_ERR_INVALID_ARG;
+    cudaSetDevice(c->cfg.device);
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (c->pinned) cudaFreeHost(c->pinned);
+    for (cudaEvent_t ev : c->prof.ev) cudaEventDestroy(ev);
+    delete c;
+    if (e != cudaSuccess) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "%s in tandem_destroy", cudaGetErrorString(e));
+        return TANDEM_ERR_CUDA;
+    }
+    return TANDEM_OK;
+}
+
+extern "C" tandem_status tandem_prefill(tandem_ctx* c, int32_t batch, const int32_t* prompt_ids, const int32_t* prompt_lens) {
+    TRY(begin_call(c));
+    if (!prompt_ids || !prompt_lens || batch < 1) return TANDEM_ERR_INVALID_ARG;
+    if (batch > c->cfg.max_batch) return TANDEM_ERR_CAPACITY;
+    const int pos_cap = std::min(c->cfg.max_seq, std::min(c->cfg.large.max_pos, c->cfg.small.max_pos));
+    long long rows = 0, total = 0;
+    int n_max = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (prompt_lens[b] < 1) return TANDEM_ERR_INVALID_ARG;
+        if (prompt_lens[b] > pos_cap) return TANDEM_ERR_CAPACITY;
+        rows += prompt_lens[b] - 1;
+        total += prompt_lens[b];
+        n_max = std::max(n_max, prompt_lens[b]);
+    }
+    if (rows > c->lay.max_rows) return TANDEM_ERR_CAPACITY;
+    for (long long i = 0; i < total; ++i)
+        if (prompt_ids[i] < 0 || prompt_ids[i] >= c->cfg.large.vocab) return TANDEM_ERR_INVALID_ARG;
+
+    CK(cudaStreamSynchronize(c->stream));   // staging buffer free again
+    const int M = (int)rows;
+    int32_t* p_tok = c->pinned;
+    int32_t* p_seq = p_tok + c->lay.max_rows;
+    int32_t* p_pos = p_seq + c->lay.max_rows;
+    int32_t* p_g0 = p_pos + c->lay.max_rows;
+    int32_t* p_gc = p_g0 + c->lay.max_groups;
+    int32_t* p_n = p_gc + c->lay.max_groups;
+    int32_t* p_pend = p_n + c->cfg.max_batch;
+    int m = 0, groups = 0;
+    long long off = 0;
+    for (int b = 0; b < batch; ++b) {
+        const int len = prompt_lens[b];
+        for (int p = 0; p < len - 1; ++p) {
+            if (p % ATT_NQ == 0) { p_g0[groups] = m; p_gc[groups] = std::min(ATT_NQ, len - 1 - p); ++groups; }
+            p_tok[m] = prompt_ids[off + p]; p_seq[m] = b; p_pos[m] = p; ++m;
+        }
+        p_n[b] = len;
+        p_pend[b] = prompt_ids[off + len - 1];
+        off += len;
+    }
+    cudaStream_t s = c->stream;
+    if (M > 0) {
+        CK(cudaMemcpyAsync(c->arena + c->lay.row_tok, p_tok, (size_t)M * 4, cudaMemcpyHostToDevice, s));
+        CK(cudaMemcpyAsync(c->arena + c->lay.row_seq, p_seq, (size_t)M * 4, cudaMemcpyHostToDevice, s));
+        CK(cudaMemcpyAsync(c->arena + c->lay.row_pos, p_pos, (size_t)M * 4, cudaMemcpyHostToDevice, s));
+        CK(cudaMemcpyAsync(c->arena + c->lay.grp_row0, p_g0, (size_t)groups * 4, cudaMemcpyHostToDevice, s));
+        CK(cudaMemcpyAsync(c->arena + c->lay.grp_cnt, p_gc, (size_t)groups * 4, cudaMemcpyHostToDevice, s));
+    }
+    CK(cudaMemsetAsync(c->arena + c->lay.st_n, 0, c->lay.row_tok - c->lay.st_n, s));
+    CK(cudaMemcpyAsync(c->st.n, p_n, (size_t)batch * 4, cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(c->st.pending, p_pend, (size_t)batch * 4, cudaMemcpyHostToDevice, s));
+    c->batch = batch;
+    c->n_ub = n_max;
+    c->n_sum = total;
+    if (M > 0) {
+        Rows r; r.M = M; r.groups = groups; r.nq = 0; r.decode = false; r.n_chunks = 0; r.kv_positions = (double)rows;
+        if (c->cfg.dtype == TANDEM_DTYPE_BF16) large_pass<bf16>(*c, r, true, false);
+        else large_pass<float>(*c, r, true, false);
+    }
+    return check_launch();
+}
+
+namespace {
+
+tandem_status capacity_for(tandem_ctx* c, int extra_tokens, int gamma) {
+    const int pos_cap = std::min(c->cfg.max_seq, std::min(c->cfg.large.max_pos, c->cfg.small.max_pos));
+    // rows of the last iteration reach position (n_ub + extra - 1) + gamma
+    if ((long long)c->n_ub + extra_tokens + gamma > pos_cap) return TANDEM_ERR_CAPACITY;
+    return TANDEM_OK;
+}
+
+}  // namespace
+
+extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t accept_mode, uint64_t mode_seed,
+                                           tandem_step_result* result) {
+    TRY(begin_call(c));
+    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 2) return TANDEM_ERR_INVALID_ARG;
+    if (c->batch == 0) return TANDEM_ERR_STATE;
+    TRY(capacity_for(c, 0, gamma));
+    reset_call_kernel<<<1, 256, 0, c->stream>>>(c->st, c->batch);
+    c->launches++;
+    if (c->cfg.dtype == TANDEM_DTYPE_BF16) iteration<bf16>(*c, gamma, accept_mode, mode_seed, INT_MAX);
+    else iteration<float>(*c, gamma, accept_mode, mode_seed, INT_MAX);
+    c->n_ub += gamma + 1;
+    c->n_sum += (long long)c->batch * (gamma + 1);
+    TRY(check_launch());
+    if (result) {
+        int32_t* cnt = c->pinned;   // staging is idle outside prefill
+        CK(cudaMemcpyAsync(cnt, c->st.counters, 5 * 4, cudaMemcpyDeviceToHost, c->stream));
+        const int B = c->batch, GL = TANDEM_GAMMA_LIMIT;
+        std::vector<int32_t> d((size_t)B * GL), t((size_t)B * (GL + 1));
+        if (result->drafts) CK(cudaMemcpyAsync(d.data(), c->st.drafts, d.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+        if (result->targets) CK(cudaMemcpyAsync(t.data(), c->st.targets, t.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+        if (result->accept_len) CK(cudaMemcpyAsync(result->accept_len, c->st.accept_len, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+        if (result->n_committed) CK(cudaMemcpyAsync(result->n_committed, c->st.n, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+        c->n_ub = cnt[3];
+        c->n_sum = cnt[4];
+        for (int b = 0; b < B; ++b) {
+            if (result->drafts) for (int i = 0; i < gamma; ++i) result->drafts[b * gamma + i] = d[(size_t)b * GL + i];
+            if (result->targets) for (int i = 0; i <= gamma; ++i) result->targets[b * (gamma + 1) + i] = t[(size_t)b * (GL + 1) + i];
+        }
+    }
+    return TANDEM_OK;
+}
+
+namespace {
+
+tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_new, int mode, uint64_t seed,
+                           int32_t* out_ids, int32_t* out_lens, tandem_stats* stats) {
+    if (!out_ids || max_new < 1) return TANDEM_ERR_INVALID_ARG;
+    if (c->batch == 0) return TANDEM_ERR_STATE;
+    if (max_new > c->cfg.max_seq) return TANDEM_ERR_CAPACITY;
+    TRY(capacity_for(c, max_new, gamma));
+    const int B = c->batch;
+    const int64_t launches0 = c->launches;
+    reset_call_kernel<<<1, 256, 0, c->stream>>>(c->st, B);
+    c->launches++;
+    CK(cudaMemsetAsync(c->st.hist, 0, (TANDEM_GAMMA_LIMIT + 1) * 8, c->stream));
+    int32_t* live = c->pinned;   // staging is idle outside prefill
+    int64_t iters = 0;
+    for (;;) {
+        if (speculative) {
+            if (c->cfg.dtype == TANDEM_DTYPE_BF16) iteration<bf16>(*c, gamma, mode, seed, max_new);
+            else iteration<float>(*c, gamma, mode, seed, max_new);
+        } else {
+            if (c->cfg.dtype == TANDEM_DTYPE_BF16) greedy_iteration<bf16>(*c, max_new);
+            else greedy_iteration<float>(*c, max_new);
+        }
+        ++iters;
+        CK(cudaMemcpyAsync(live, c->st.counters, 5 * 4, cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+        c->n_ub = live[3];
+        c->n_sum = live[4];
+        if (live[1] <= 0) break;
+        if (iters > (int64_t)max_new + 1) return TANDEM_ERR_STATE;   // every iteration emits at least one token
+    }
+    TRY(check_launch());
+    CK(cudaMemcpy2DAsync(out_ids, (size_t)max_new * 4, c->st.out_ids, (size_t)c->st.out_cap * 4, (size_t)max_new * 4, B,
+                         cudaMemcpyDeviceToHost, c->stream));
+    std::vector<unsigned long long> hist(TANDEM_GAMMA_LIMIT + 1);
+    CK(cudaMemcpyAsync(hist.data(), c->st.hist, hist.size() * 8, cudaMemcpyDeviceToHost, c->stream));
+    if (out_lens) CK(cudaMemcpyAsync(out_lens, c->st.emitted, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (stats) {
+        memset(stats, 0, sizeof(*stats));
+        stats->iterations = iters;
+        stats->large_runs = iters;
+        stats->small_runs = speculative ? iters * gamma : 0;
+        stats->emitted = (int64_t)B * max_new;
+        for (int i = 0; i <= TANDEM_GAMMA_LIMIT; ++i) stats->accept_hist[i] = (int64_t)hist[i];
+        stats->kernel_launches = c->launches - launches0;
+    }
+    return TANDEM_OK;
+}
+
+}  // namespace
+
+extern "C" tandem_status tandem_speculative_generate(tandem_ctx* c, int32_t gamma, int32_t max_new_tokens, int32_t accept_mode,
+                                                     uint64_t mode_seed, int32_t* out_ids, int32_t* out_lens, tandem_stats* stats) {
+    TRY(begin_call(c));
+    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 2) return TANDEM_ERR_INVALID_ARG;
+    return run_generate(c, true, gamma, max_new_tokens, accept_mode, mode_seed, out_ids, out_lens, stats);
+}
+
+extern "C" tandem_status tandem_large_greedy_generate(tandem_ctx* c, int32_t max_new_tokens, int32_t* out_ids, int32_t* out_lens,
+                                                      tandem_stats* stats) {
+    TRY(begin_call(c));
+    return run_generate(c, false, 0, max_new_tokens, 0, 0ull, out_ids, out_lens, stats);
+}
+
+extern "C" int64_t tandem_launch_count(tandem_ctx* c) { return c ? c->launches : -1; }
+
+extern "C" const char* tandem_profile_class_name(int32_t cls) {
+    static const char* names[PC_COUNT] = {"gemm_smallm", "gemm_tiled", "attn_split", "attn_merge", "attn_prompt",
+                                          "layernorm", "rows", "argmax", "verify"};
+    return (cls >= 0 && cls < PC_COUNT) ? names[cls] : nullptr;
+}
+
+extern "C" tandem_status tandem_profile_enable(tandem_ctx* c, int32_t max_launches) {
+    TRY(begin_call(c));
+    if (max_launches < 0) return TANDEM_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(c->stream));
+    Prof& p = c->prof;
+    p.on = max_launches > 0;
+    p.used = 0;
+    p.cls.clear();
+    p.bytes.clear();
+    while (p.ev.size() < (size_t)2 * max_launches) {
+        cudaEvent_t e;
+        CK(cudaEventCreate(&e));
+        p.ev.push_back(e);
+    }
+    return TANDEM_OK;
+}
+
+extern "C" tandem_status tandem_profile_read(tandem_ctx* c, int32_t n_classes, double* ms, int64_t* launches, double* work) {
+    TRY(begin_call(c));
+    if (!ms || !launches || !work || n_classes < 1) return TANDEM_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(c->stream));
+    for (int i = 0; i < n_classes; ++i) { ms[i] = 0; launches[i] = 0; work[i] = 0; }
+    Prof& p = c->prof;
+    for (size_t i = 0; i + 1 < p.used; i += 2) {
+        const int cls = p.cls[i / 2];
+        if (cls >= n_classes) continue;
+        float t = 0.f;
+        CK(cudaEventElapsedTime(&t, p.ev[i], p.ev[i + 1]));
+        ms[cls] += t;
+        launches[cls] += 1;
+        work[cls] += p.bytes[i / 2];
+    }
+    p.used = 0;
+    p.cls.clear();
+    p.bytes.clear();
+    return TANDEM_OK;
+}
+
+extern "C" tandem_status tandem_debug_read(tandem_ctx* c, int32_t what, int32_t layer, int32_t seq, void* host_dst, size_t bytes) {
+    TRY(begin_call(c));
+    if (!host_dst) return TANDEM_ERR_INVALID_ARG;
+    if (c->batch == 0) return TANDEM_ERR_STATE;
+    const int B = c->batch, g = c->last_gamma, V = c->cfg.large.vocab;
+    CK(cudaStreamSynchronize(c->stream));
+    if (what == 0 || what == 1 || what == 2) {
+        size_t n;
+        const void* src;
+        if (what == 0) { n = (size_t)B * (g + 1) * V; src = c->arena + c->lay.logits_large; }
+        else if (what == 1) { n = (size_t)g * B * V; src = c->arena + c->lay.logits_small; }
+        else { n = (size_t)B * (g + 1) * c->cfg.large.d_model; src = c->arena + c->lay.h_large; }
+        if (bytes != n * 4) return TANDEM_ERR_INVALID_ARG;
+        if (n) CK(cudaMemcpy(host_dst, src, bytes, cudaMemcpyDeviceToHost));
+        return TANDEM_OK;
+    }
+    if (what >= 3 && what <= 6) {
+        const Model& m = (what <= 4) ? c->large : c->small;
+        if (layer < 0 || layer >= m.d.n_layers || seq < 0 || seq >= B) return TANDEM_ERR_INVALID_ARG;
+        int n_b = 0;
+        CK(cudaMemcpy(&n_b, c->st.n + seq, 4, cudaMemcpyDeviceToHost));
+        const int n = n_b - 1, d = m.d.d_model, H = m.d.n_heads, dh = d / H;
+        if (bytes != (size_t)n * d * 4) return TANDEM_ERR_INVALID_ARG;
+        if (n == 0) return TANDEM_OK;
+        const int which = (what == 3 || what == 5) ? 0 : 1;
+        float* dbg = at<float>(*c, c->lay.dbg);
+        const size_t total = (size_t)n * d;
+        const size_t seq_off = (size_t)seq * H * c->cfg.max_seq * dh;
+        if (c->cfg.dtype == TANDEM_DTYPE_BF16)
+            gather_kv_kernel<bf16><<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(kv_ptr<bf16>(*c, m, layer, which) + seq_off, dbg, n, H, dh, c->cfg.max_seq);
+        else
+            gather_kv_kernel<float><<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(kv_ptr<float>(*c, m, layer, which) + seq_off, dbg, n, H, dh, c->cfg.max_seq);
+        TRY(check_launch());
+        CK(cudaMemcpyAsync(host_dst, dbg, bytes, cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+        return TANDEM_OK;
+    }
+    if (what == 7) {
+        if (bytes != (size_t)B * 4) return TANDEM_ERR_INVALID_ARG;
+        CK(cudaMemcpy(host_dst, c->st.n, bytes, cudaMemcpyDeviceToHost));
+        return TANDEM_OK;
+    }
+    return TANDEM_ERR_INVALID_ARG;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// stand-alone kernels
+// ---------------------------------------------------------------------------------------------------
+
+namespace {
+struct AttnScratch { size_t ml, acc, rows, total; int n_chunks; };
+AttnScratch attn_scratch_layout(int batch, int H, int dh, int derived_len, int own_len) {
+    AttnScratch s;
+    s.n_chunks = cdiv(derived_len + own_len, ATT_CH);
+    size_t off = 0;
+    s.ml = off; off = align_up(off + (size_t)batch * H * s.n_chunks * 2 * 4);
+    s.acc = off; off = align_up(off + (size_t)batch * H * s.n_chunks * dh * 4);
+    s.rows = off; off = align_up(off + (size_t)batch * 2 * 4);
+    s.total = off;
+    return s;
+}
+__global__ void iota_rows_kernel(int* row_seq, int* row_pos, int n, int pos) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) { row_seq[i] = i; row_pos[i] = pos; }
+}
+}  // namespace
+
+extern "C" size_t tandem_decode_attention_scratch_bytes(int32_t batch, int32_t n_heads, int32_t d_head, int32_t derived_len, int32_t own_len) {
+    if (batch < 1 || n_heads < 1 || d_head < 1 || derived_len < 0 || own_len < 0 || derived_len + own_len < 1) return 0;
+    return attn_scratch_layout(batch, n_heads, d_head, derived_len, own_len).total;
+}
+
+extern "C" tandem_status tandem_decode_attention(const void* q, const void* k_derived, const void* v_derived, const void* k_own,
+                                                 const void* v_own, void* out, void* scratch, size_t scratch_bytes, int32_t batch,
+                                                 int32_t n_heads, int32_t d_head, int32_t derived_len, int32_t own_len, void* stream) {
+    if (!q || !out || !scratch) return TANDEM_ERR_INVALID_ARG;
+    if (batch < 1 || n_heads < 1 || derived_len < 0 || own_len < 0 || derived_len + own_len < 1) return TANDEM_ERR_INVALID_ARG;
+    if ((derived_len > 0 && (!k_derived || !v_derived)) || (own_len > 0 && (!k_own || !v_own))) return TANDEM_ERR_INVALID_ARG;
+    if (d_head != 32 && d_head != 64 && d_head != 128) return TANDEM_ERR_SHAPE;
+    if ((long long)batch * n_heads > 65535 * 16) return TANDEM_ERR_SHAPE;
+    if (((uintptr_t)q | (uintptr_t)k_derived | (uintptr_t)v_derived | (uintptr_t)k_own | (uintptr_t)v_own | (uintptr_t)out | (uintptr_t)scratch) & 15)
+        return TANDEM_ERR_INVALID_ARG;
+    const AttnScratch sl = attn_scratch_layout(batch, n_heads, d_head, derived_len, own_len);
+    if (scratch_bytes < sl.total) return TANDEM_ERR_ARENA_TOO_SMALL;
+    if (batch > 65535) return TANDEM_ERR_SHAPE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned char* sc = static_cast<unsigned char*>(scratch);
+    int* row_seq = reinterpret_cast<int*>(sc + sl.rows);
+    int* row_pos = row_seq + batch;
+    iota_rows_kernel<<<cdiv(batch, 256), 256, 0, s>>>(row_seq, row_pos, batch, derived_len + own_len - 1);
+    AttnArgs a; memset(&a, 0, sizeof(a));
+    a.q = q; a.ldq = n_heads * d_head; a.kcache = k_derived; a.vcache = v_derived; a.k2 = k_own; a.v2 = v_own;
+    a.split = derived_len; a.t_max = derived_len; a.t_max2 = own_len;
+    a.out = out; a.ldo = n_heads * d_head; a.row_seq = row_seq; a.row_pos = row_pos; a.nq = 1; a.n_heads = n_heads;
+    a.part_ml = reinterpret_cast<float*>(sc + sl.ml); a.part_acc = reinterpret_cast<float*>(sc + sl.acc);
+    a.n_chunks_max = sl.n_chunks; a.scale = 1.0f / sqrtf((float)d_head);
+    tandem_ctx tmp;   // only the stream and the launch counter are used by the launch helpers
+    tmp.stream = s;
+    launch_attn<bf16>(tmp, d_head, a, batch, batch, false, sl.n_chunks, 0.0);
+    return check_launch();
+}
+
+extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t, const void* ln_g, const void* ln_b, const void* wk,
+                                                  const void* wv, void* k_out, void* v_out, void* scratch, size_t scratch_bytes,
+                                                  int32_t rows, int32_t d_large, int32_t d_small, void* stream) {
+    if (!x || !w_t || !ln_g || !ln_b || !wk || !wv || !k_out || !v_out || !scratch) return TANDEM_ERR_INVALID_ARG;
+    if (rows < 1 || rows > 256 || d_large < 8 || d_small < 8) return TANDEM_ERR_INVALID_ARG;
+    if (d_large % 8 || d_small % 8) return TANDEM_ERR_SHAPE;
+    const size_t need = align_up((size_t)rows * d_small * 4) + align_up((size_t)rows * d_small * 2) + align_up((size_t)rows * 8);
+    if (scratch_bytes < need) return TANDEM_ERR_ARENA_TOO_SMALL;
+    if (((uintptr_t)x | (uintptr_t)w_t | (uintptr_t)wk | (uintptr_t)wv | (uintptr_t)k_out | (uintptr_t)v_out | (uintptr_t)scratch) & 15)
+        return TANDEM_ERR_INVALID_ARG;
+    tandem_ctx tmp;   // only the stream and the launch counter are used by the launch helpers
+    tmp.stream = static_cast<cudaStream_t>(stream);
+    unsigned char* sc = static_cast<unsigned char*>(scratch);
+    float* yhat = reinterpret_cast<float*>(sc);
+    bf16* a_s = reinterpret_cast<bf16*>(sc + align_up((size_t)rows * d_small * 4));
+    int* row_seq = reinterpret_cast<int*>(sc + align_up((size_t)rows * d_small * 4) + align_up((size_t)rows * d_small * 2));
+    int* row_pos = row_seq + rows;
+    iota_rows_kernel<<<cdiv(rows, 256), 256, 0, tmp.stream>>>(row_seq, row_pos, rows, 0);
+    launch_gemm<bf16, EPI_STORE_F32>(tmp, true, static_cast<const bf16*>(x), d_large, rows, d_large, segs1(w_t, d_small), d_small, epi_plain(yhat, d_small));
+    launch_layernorm<bf16>(tmp, rows, yhat, ln_g, ln_b, a_s, d_small);
+    EpiArgs e; memset(&e, 0, sizeof(e));
+    e.kcache = k_out; e.vcache = v_out; e.row_seq = row_seq; e.row_pos = row_pos; e.n_heads = 1; e.d_head = d_small; e.t_max = 1; e.seg = d_small;
+    launch_gemm<bf16, EPI_KV>(tmp, true, a_s, d_small, rows, d_small, segs3(wk, wv, nullptr, d_small), 2 * d_small, e);
+    return check_launch();
+}

@@ -1,0 +1,315 @@
+"""GPU parity: the CUDA library, called through its C boundary, against the CPU checker on the same seeded
+inputs.  Token ids, accept lengths and counts must match bit for bit in fp32 mode; logits and hidden states
+within 1e-4 (fp32) or 2e-2 (bf16).  In bf16 an arg-max can legitimately flip when the checker's top two logits
+are closer than the logit tolerance, so bf16 runs are compared by replay (teacher forcing on the GPU's tokens)."""
+import numpy as np
+import pytest
+
+from oracle import tandem_oracle as O
+from paper_2402_08644_b200 import binding, build, synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-4
+TOL_BF16 = 2e-2
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    return binding.load_library()
+
+
+def gpu_toy_shape(kind=synth.FF_TANDEM_LINEAR, dtype=synth.DTYPE_FP32, max_pos=320, layer_map=None, hidden=0,
+                  large=(3, 128, 4, 256), small=(2, 64, 2, 136), vocab=97):
+    L = synth.ModelDims(large[0], large[1], large[2], large[3], vocab, max_pos)
+    S = synth.ModelDims(small[0], small[1], small[2], small[3], vocab, max_pos)
+    return synth.make_shape(L, S, kind, hidden, layer_map, dtype)
+
+
+def toy_weights(shape, seed, std=0.08):
+    w = synth.make_weights(shape, seed, std)
+    synth.perturb_norm_params(w, seed)
+    return w
+
+
+def prompts_for(shape, lens, seed):
+    return [[int(t) for t in p] for p in synth.make_prompts(len(lens), list(lens), shape.large.vocab, seed)]
+
+
+# ------------------------------------------------------------------------------------------------
+# fp32 mode: strict equality
+# ------------------------------------------------------------------------------------------------
+
+def test_config1_tiny_fp32_end_to_end_bit_exact():
+    """The Tiny Tandem configuration exactly: seed 0, batch 1, 32-token prompt, gamma 4, 64 new tokens."""
+    shape = synth.named_config("tiny")
+    w = synth.make_weights(shape, seed=0, std=0.02)
+    prompt = prompts_for(shape, [32], seed=0)
+    want, accepts, runs = O.generate_batch(shape, w, prompt, 4, 64)
+    t = binding.Tandem(shape, w, max_batch=1, max_seq=128, gamma_max=4)
+    t.tandem_prefill(prompt)
+    got, lens, stats = t.tandem_speculative_generate(4, 64)
+    assert got[0].tolist() == want[0]
+    assert lens.tolist() == [64]
+    assert stats["iterations"] == len(accepts[0]) and stats["large_runs"] == runs[0][0] and stats["small_runs"] == runs[0][1]
+    hist = np.bincount(accepts[0], minlength=5).tolist()
+    assert stats["accept_hist"] == hist
+    assert stats["kernel_launches"] > 0
+    # and the plain greedy decoding of the large model, on the GPU, gives the same tokens
+    t.tandem_prefill(prompt)
+    greedy, _, _ = t.tandem_large_greedy_generate(64)
+    assert greedy[0].tolist() == want[0]
+    t.close()
+
+
+@pytest.mark.parametrize("kind,gamma,mode", [(synth.FF_TANDEM_LINEAR, 3, 0), (synth.FF_TANDEM_MLP, 4, 2),
+                                             (synth.FF_TANDEM_LINEAR, 1, 1), (synth.FF_TANDEM_MLP, 7, 2),
+                                             (synth.FF_TANDEM_LINEAR, 0, 0)])
+def test_fp32_ragged_batch_steps_match_oracle(kind, gamma, mode):
+    """Step by step on a ragged batch (prompt lengths 1, 2, 17, 130 cross a chunk boundary): drafts, targets,
+    accept lengths, committed counts bit-exact; logits, hidden states and both KV caches within 1e-4."""
+    shape = gpu_toy_shape(kind=kind, hidden=40 if kind else 0, layer_map=(1, 3))
+    w = toy_weights(shape, seed=10 + gamma)
+    lens = [1, 2, 17, 130]
+    prompts = prompts_for(shape, lens, seed=gamma)
+    t = binding.Tandem(shape, w, max_batch=4, max_seq=320, gamma_max=max(gamma, 1))
+    t.tandem_prefill(prompts)
+    oracles = [O.TandemOracle(shape, w) for _ in prompts]
+    for o, p in zip(oracles, prompts):
+        o.prefill(p)
+    seed = 1234
+    for it in range(5):
+        res = t.tandem_block_step(gamma, mode, seed)
+        s_logits = t.tandem_debug_read(binding.READ_SMALL_LOGITS, gamma)
+        l_logits = t.tandem_debug_read(binding.READ_LARGE_LOGITS, gamma)
+        hidden = t.tandem_debug_read(binding.READ_LARGE_HIDDEN, gamma)
+        for b, o in enumerate(oracles):
+            drafts, sl = o.draft(gamma)
+            targets, ll, reps = o.verify(drafts)
+            a = o.accept_length(drafts, targets, mode, seed, b, o.iteration)
+            o.commit(a, drafts, targets, reps)
+            assert res["drafts"][b].tolist() == drafts
+            assert res["targets"][b].tolist() == targets
+            assert res["accept_len"][b] == a
+            assert res["n_committed"][b] == len(o.tokens)
+            for s in range(gamma):
+                assert np.abs(s_logits[s, b] - sl[s]).max() < TOL_FP32
+            assert np.abs(l_logits[b] - ll).max() < TOL_FP32
+            assert np.abs(hidden[b] - reps[-1]).max() < TOL_FP32
+    for b, o in enumerate(oracles):
+        for layer in range(shape.large.n_layers):
+            k = t.tandem_debug_read(binding.READ_LARGE_K, layer=layer, seq=b)
+            v = t.tandem_debug_read(binding.READ_LARGE_V, layer=layer, seq=b)
+            assert k.shape[0] == len(o.tokens) - 1 == o.large_cache.length()
+            assert np.abs(k - np.stack(o.large_cache.k[layer])).max() < TOL_FP32
+            assert np.abs(v - np.stack(o.large_cache.v[layer])).max() < TOL_FP32
+        for layer in range(shape.small.n_layers):
+            k = t.tandem_debug_read(binding.READ_SMALL_K, layer=layer, seq=b)
+            v = t.tandem_debug_read(binding.READ_SMALL_V, layer=layer, seq=b)
+            assert np.abs(k - np.stack(o.derived.k[layer])).max() < TOL_FP32
+            assert np.abs(v - np.stack(o.derived.v[layer])).max() < TOL_FP32
+    t.close()
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_fp32_generate_matches_oracle_all_modes(mode):
+    shape = gpu_toy_shape(kind=synth.FF_TANDEM_MLP, hidden=48)
+    w = toy_weights(shape, seed=5)
+    prompts = prompts_for(shape, [9, 1, 33], seed=8)
+    want, accepts, runs = O.generate_batch(shape, w, prompts, 3, 21, mode=mode, mode_seed=99)
+    t = binding.Tandem(shape, w, max_batch=3, max_seq=96, gamma_max=3)
+    t.tandem_prefill(prompts)
+    got, lens, stats = t.tandem_speculative_generate(3, 21, mode, 99)
+    assert got.tolist() == want
+    assert lens.tolist() == [21, 21, 21]
+    hist = np.zeros(4, dtype=np.int64)
+    for a in accepts:
+        hist += np.bincount(a, minlength=4)
+    assert stats["accept_hist"] == hist.tolist()
+    assert stats["iterations"] == max(len(a) for a in accepts)
+    t.close()
+
+
+def test_fp32_self_tandem_accepts_every_draft():
+    """Small model == large model, identity FF_Tandem, l(j) = j: Eq. 2 collapses to Eq. 1, so with the natural
+    comparison every draft is accepted and the small model's logits equal the large model's."""
+    dims = synth.ModelDims(3, 128, 4, 256, 97, 128)
+    shape = synth.self_tandem_shape(dims)
+    w = synth.make_self_tandem_weights(shape, seed=4, std=0.08)
+    prompts = prompts_for(shape, [7, 40], seed=2)
+    t = binding.Tandem(shape, w, max_batch=2, max_seq=128, gamma_max=4)
+    t.tandem_prefill(prompts)
+    for it in range(4):
+        res = t.tandem_block_step(4)
+        assert res["accept_len"].tolist() == [4, 4]
+        sl = t.tandem_debug_read(binding.READ_SMALL_LOGITS, 4)
+        ll = t.tandem_debug_read(binding.READ_LARGE_LOGITS, 4)
+        for s in range(4):
+            assert np.abs(sl[s] - ll[:, s]).max() < TOL_FP32
+    t.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# bf16 mode
+# ------------------------------------------------------------------------------------------------
+
+def _near_tie(logits, token, delta):
+    lg = logits.astype(np.float32)
+    return lg.max() - lg[token] <= delta
+
+
+def _replay_compare(shape, w, prompts, gamma, iters, tol, delta):
+    """Runs `iters` GPU iterations; the checker follows the GPU's tokens (teacher forcing).  Returns the
+    number of GPU decisions that differ from the checker's arg-max (each must be a near-tie)."""
+    t = binding.Tandem(shape, w, max_batch=len(prompts), max_seq=shape.large.max_pos, gamma_max=gamma)
+    t.tandem_prefill(prompts)
+    oracles = [O.TandemOracle(shape, w) for _ in prompts]
+    for o, p in zip(oracles, prompts):
+        o.prefill(p)
+    flips = 0
+    for it in range(iters):
+        res = t.tandem_block_step(gamma)
+        s_logits = t.tandem_debug_read(binding.READ_SMALL_LOGITS, gamma)
+        l_logits = t.tandem_debug_read(binding.READ_LARGE_LOGITS, gamma)
+        for b, o in enumerate(oracles):
+            g_drafts = res["drafts"][b].tolist()
+            g_targets = res["targets"][b].tolist()
+            drafts, sl = o.draft(gamma, forced=g_drafts)
+            for s in range(gamma):
+                assert np.abs(s_logits[s, b] - sl[s]).max() < tol
+                if drafts[s] != g_drafts[s]:
+                    assert _near_tie(sl[s], g_drafts[s], delta)
+                    flips += 1
+            targets, ll, reps = o.verify(g_drafts)
+            assert np.abs(l_logits[b] - ll).max() < tol
+            for r in range(gamma + 1):
+                if targets[r] != g_targets[r]:
+                    assert _near_tie(ll[r], g_targets[r], delta)
+                    flips += 1
+            # the accept rule itself is integer work: the checker's rule on the GPU's ids must give the GPU's length
+            a = o.accept_length(g_drafts, g_targets)
+            assert res["accept_len"][b] == a
+            o.commit(a, g_drafts, g_targets, reps)
+            assert res["n_committed"][b] == len(o.tokens)
+    t.close()
+    return flips
+
+
+def test_bf16_toy_replay_within_tolerance():
+    shape = gpu_toy_shape(dtype=synth.DTYPE_BF16, layer_map=(2, 3))
+    w = toy_weights(shape, seed=31)
+    for k in w:                                    # bf16-representable values everywhere they are stored as bf16
+        if not synth.is_norm_param(k):
+            w[k] = synth.round_to_bf16(w[k])
+    flips = _replay_compare(shape, w, prompts_for(shape, [5, 140, 1], seed=6), 3, 4, TOL_BF16, 2 * TOL_BF16)
+    assert flips <= 6
+
+
+def test_bf16_small_config_widths_replay():
+    """Config "small" (12x1024 / 4x512, vocab 32000, bf16) with a shortened prompt so the checker stays fast."""
+    shape = synth.named_config("small", max_pos=192)
+    w = synth.make_weights(shape, seed=3)
+    flips = _replay_compare(shape, w, prompts_for(shape, [150], seed=4), 3, 3, TOL_BF16, 2 * TOL_BF16)
+    assert flips <= 3
+
+
+@pytest.mark.parametrize("dtype", [synth.DTYPE_FP32, synth.DTYPE_BF16])
+def test_gpu_speed_equals_gpu_greedy_bit_exact(dtype):
+    """On the GPU itself: Tandem + SPEED (block passes of gamma+1 rows, ragged rollback) returns exactly the
+    tokens of one-row greedy decoding of the large model, for every accept pattern."""
+    shape = gpu_toy_shape(dtype=dtype)
+    w = toy_weights(shape, seed=77)
+    prompts = prompts_for(shape, [3, 129, 64], seed=1)
+    t = binding.Tandem(shape, w, max_batch=3, max_seq=320, gamma_max=5)
+    t.tandem_prefill(prompts)
+    greedy, _, _ = t.tandem_large_greedy_generate(40)
+    for gamma, mode in ((5, 0), (2, 0), (4, 0)):
+        t.tandem_prefill(prompts)
+        got, _, stats = t.tandem_speculative_generate(gamma, 40, mode)
+        assert got.tolist() == greedy.tolist()
+    t.close()
+
+
+def test_bf16_small_config_speed_equals_greedy_full_prompt():
+    """Config "small" at its full prompt length (512) and gamma 3: GPU SPEED == GPU greedy, and the natural
+    accept histogram is what the call reports."""
+    shape = synth.named_config("small", max_pos=640)
+    w = synth.make_weights(shape, seed=0)
+    prompts = prompts_for(shape, [512], seed=0)
+    t = binding.Tandem(shape, w, max_batch=1, max_seq=640, gamma_max=3)
+    t.tandem_prefill(prompts)
+    greedy, _, _ = t.tandem_large_greedy_generate(48)
+    t.tandem_prefill(prompts)
+    got, lens, stats = t.tandem_speculative_generate(3, 48)
+    assert got.tolist() == greedy.tolist()
+    assert sum((a + 1) * c for a, c in enumerate(stats["accept_hist"])) >= 48
+    t.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# stand-alone kernels (the attention / projection micro-benchmark shapes, scaled down)
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("B,H,dh,Td,To", [(1, 16, 64, 1024, 4), (3, 4, 64, 129, 4), (2, 2, 32, 0, 3), (2, 3, 128, 127, 0),
+                                          (1, 16, 64, 1, 1), (8, 16, 64, 2048, 4), (1, 2, 64, 128, 1)])
+def test_decode_attention_mixed_context_matches_oracle(B, H, dh, Td, To):
+    import torch
+    g = torch.Generator().manual_seed(B * 1000 + Td)
+    mk = lambda *s: torch.randn(*s, generator=g).to(torch.bfloat16)
+    q, kd, vd, ko, vo = mk(B, H, dh), mk(B, H, Td, dh), mk(B, H, Td, dh), mk(B, H, To, dh), mk(B, H, To, dh)
+    out = binding.tandem_decode_attention(*(x.cuda() for x in (q, kd, vd, ko, vo))).float().cpu().numpy()
+    f = lambda x: x.float().numpy().astype(np.float64)
+    for b in range(B):
+        for h in range(H):
+            K = np.concatenate([f(kd[b, h]), f(ko[b, h])], 0)
+            V = np.concatenate([f(vd[b, h]), f(vo[b, h])], 0)
+            want = O.attend(f(q[b, h]), K, V, 1)
+            assert np.abs(out[b, h] - want).max() < TOL_BF16
+
+
+@pytest.mark.parametrize("rows,dL,dS", [(4, 256, 64), (13, 4096, 1024), (1, 128, 128)])
+def test_ff_tandem_project_matches_oracle(rows, dL, dS):
+    import torch
+    g = torch.Generator().manual_seed(rows)
+    bf = lambda t: t.to(torch.bfloat16)
+    x = bf(torch.randn(rows, dL, generator=g))
+    w_t, wk, wv = (bf(torch.randn(dS, k, generator=g) * 0.02) for k in (dL, dS, dS))   # the benchmark's init scale
+    ln_g = 1 + 0.1 * torch.randn(dS, generator=g)
+    ln_b = 0.1 * torch.randn(dS, generator=g)
+    k, v = binding.tandem_ff_tandem_project(*(t.cuda() for t in (x, w_t, ln_g, ln_b, wk, wv)))
+    f = lambda t: t.float().numpy().astype(np.float64)
+    a = O.layer_norm(f(x) @ f(w_t).T, f(ln_g), f(ln_b))
+    assert np.abs(k.float().cpu().numpy() - a @ f(wk).T).max() < TOL_BF16
+    assert np.abs(v.float().cpu().numpy() - a @ f(wv).T).max() < TOL_BF16
+
+
+# ------------------------------------------------------------------------------------------------
+# error behaviour: validated on the host, nothing launched
+# ------------------------------------------------------------------------------------------------
+
+def test_errors_are_reported_not_launched():
+    shape = gpu_toy_shape()
+    w = toy_weights(shape, seed=1)
+    t = binding.Tandem(shape, w, max_batch=2, max_seq=40, gamma_max=3)
+    with pytest.raises(binding.TandemError) as e:
+        t.batch = 1
+        t.tandem_block_step(2)
+    assert e.value.status == 5                      # step before prefill
+    with pytest.raises(binding.TandemError) as e:
+        t.tandem_prefill(prompts_for(shape, [4, 4, 4], 0))
+    assert e.value.status == 4                      # batch > max_batch
+    with pytest.raises(binding.TandemError) as e:
+        t.tandem_prefill(prompts_for(shape, [41], 0))
+    assert e.value.status == 4                      # prompt longer than max_seq
+    t.tandem_prefill(prompts_for(shape, [30, 8], 0))
+    with pytest.raises(binding.TandemError) as e:
+        t.tandem_block_step(4)
+    assert e.value.status == 1                      # gamma > gamma_max
+    with pytest.raises(binding.TandemError) as e:
+        t.tandem_speculative_generate(3, 10)
+    assert e.value.status == 4                      # 30 + 10 + 3 > 40
+    got, _, _ = t.tandem_speculative_generate(3, 7) # fits exactly
+    want, _, _ = O.generate_batch(shape, w, prompts_for(shape, [30, 8], 0), 3, 7)
+    assert got.tolist() == want
+    t.close()
