@@ -207,6 +207,34 @@ TANDEM_API tandem_status tandem_decode_attention(const void* q, const void* k_de
                                       size_t scratch_bytes, int32_t batch, int32_t n_heads, int32_t d_head,
                                       int32_t derived_len, int32_t own_len, void* stream);
 
+/* tandem_decode_attention_static: the same attention for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of the kernel above, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a host callback or another
+ * library's hook, in a process whose memory pool is owned by a framework that hands out no raw buffers,
+ * or in a service that must not touch the allocator after start-up because an allocation can block on,
+ * or synchronise with, other work on the device.  Such a caller still passes its inputs and its output,
+ * but the split-K partial results go to a buffer built into the library: a file-scope __device__ array of
+ * TANDEM_STATIC_SCRATCH_BYTES that every GPU loading the library holds until the process exits.
+ *
+ * Same arguments, layouts and results as tandem_decode_attention, minus scratch.  Differences:
+ *  - Shapes whose partial results need more than TANDEM_STATIC_SCRATCH_BYTES
+ *    (tandem_decode_attention_scratch_bytes tells) are refused with TANDEM_ERR_CAPACITY before anything is
+ *    launched; tandem_last_cuda_error() then holds a sentence with both sizes.
+ *  - The first call on each device looks up the device address of the built-in buffer (with that device
+ *    current - make the device that owns the tensors current before calling).  Make that first call before
+ *    any stream capture is begun on the device.  Later calls only launch.
+ *  - The call itself allocates nothing on host or device and frees nothing.
+ *  - All calls on a device share the one buffer, and it keeps whatever the previous call left there.  The
+ *    kernels overwrite every partial result they later read, so nothing needs clearing between calls; but
+ *    two calls that can overlap on the GPU (different streams, or one stream and a graph) race on it and
+ *    give wrong results.  Keep calls to this entry point on one stream, or order them with events. */
+#define TANDEM_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+TANDEM_API tandem_status tandem_decode_attention_static(const void* q, const void* k_derived, const void* v_derived,
+                                                        const void* k_own, const void* v_own, void* out,
+                                                        int32_t batch, int32_t n_heads, int32_t d_head,
+                                                        int32_t derived_len, int32_t own_len, void* stream);
+
 /* tandem_ff_tandem_project: the linear FF_Tandem of Eq. 2 (first line) followed by the small layer's
  * LayerNorm and key/value maps, written as bf16 keys/values.  All pointers DEVICE.
  *   x [rows][d_large] bf16;  w_t [d_small][d_large] bf16;  ln_g, ln_b [d_small] fp32;

@@ -27,7 +27,7 @@ EXPORTS = ["tandem_query_arena", "tandem_create", "tandem_destroy", "tandem_pref
            "tandem_speculative_generate", "tandem_large_greedy_generate", "tandem_debug_read",
            "tandem_decode_attention_scratch_bytes", "tandem_decode_attention", "tandem_ff_tandem_project",
            "tandem_status_string", "tandem_last_cuda_error", "tandem_profile_enable", "tandem_profile_read",
-           "tandem_profile_class_name", "tandem_launch_count"]
+           "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static"]
 
 
 class TandemError(RuntimeError):
@@ -91,6 +91,7 @@ def load_library():
     lib.tandem_decode_attention_scratch_bytes.restype = sz
     lib.tandem_decode_attention.argtypes = [vp] * 7 + [sz] + [i32] * 5 + [vp]
     lib.tandem_ff_tandem_project.argtypes = [vp] * 9 + [sz] + [i32] * 3 + [vp]
+    lib.tandem_decode_attention_static.argtypes = [vp] * 6 + [i32] * 5 + [vp]
     lib.tandem_profile_enable.argtypes = [vp, i32]
     lib.tandem_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_double)]
     lib.tandem_profile_class_name.argtypes = [i32]
@@ -279,6 +280,26 @@ def tandem_decode_attention(q, k_derived, v_derived, k_own, v_own, out=None, scr
                                        ptr(scratch), scratch.numel(), B, H, dh, Td, To,
                                        C.c_void_p(torch.cuda.current_stream(q.device).cuda_stream or None)),
            "tandem_decode_attention")
+    return out
+
+
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+
+
+def tandem_decode_attention_static(q, k_derived, v_derived, k_own, v_own, out):
+    """tandem_decode_attention without a scratch argument, for callers that may not allocate device memory:
+    the partial results live in a buffer built into the library (at most STATIC_SCRATCH_BYTES are needed, else
+    TandemError with status CAPACITY).  `out` is required, so this wrapper allocates nothing either.  Calls
+    share that buffer: keep them on one stream.  Make the first call on a device outside any stream capture."""
+    import torch
+    lib = load_library()
+    B, H, dh = q.shape
+    Td, To = k_derived.shape[2], k_own.shape[2]
+    ptr = lambda t: C.c_void_p(t.data_ptr() if t.numel() else None)
+    _check(lib.tandem_decode_attention_static(ptr(q), ptr(k_derived), ptr(v_derived), ptr(k_own), ptr(v_own), ptr(out),
+                                              B, H, dh, Td, To,
+                                              C.c_void_p(torch.cuda.current_stream(q.device).cuda_stream or None)),
+           "tandem_decode_attention_static")
     return out
 
 

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -882,6 +883,54 @@ extern "C" tandem_status tandem_decode_attention(const void* q, const void* k_de
     tmp.stream = s;
     launch_attn<bf16>(tmp, d_head, a, batch, batch, false, sl.n_chunks, 0.0);
     return check_launch();
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Decode attention for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------------------------
+
+// Split-K partial results and row indices of tandem_decode_attention_static live here instead of in a
+// caller-provided buffer.  Every GPU that loads this library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_attn_scratch[TANDEM_STATIC_SCRATCH_BYTES];
+
+namespace {
+// In host code the array's name is only a handle for the runtime, not a device address: the address
+// a kernel may use comes from cudaGetSymbolAddress, asked once per device with that device current.
+void* g_static_scratch_addr[MAX_DEVICES] = {};
+std::mutex g_static_scratch_mutex;
+
+tandem_status static_scratch_for_current_device(void** out) {
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return TANDEM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        CK(cudaGetSymbolAddress(&p, g_static_attn_scratch));
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return TANDEM_OK;
+}
+}  // namespace
+
+extern "C" tandem_status tandem_decode_attention_static(const void* q, const void* k_derived, const void* v_derived,
+                                                        const void* k_own, const void* v_own, void* out, int32_t batch,
+                                                        int32_t n_heads, int32_t d_head, int32_t derived_len, int32_t own_len,
+                                                        void* stream) {
+    if (batch < 1 || n_heads < 1 || d_head < 1 || derived_len < 0 || own_len < 0 || derived_len + own_len < 1)
+        return TANDEM_ERR_INVALID_ARG;
+    const size_t need = attn_scratch_layout(batch, n_heads, d_head, derived_len, own_len).total;
+    if (need > (size_t)TANDEM_STATIC_SCRATCH_BYTES) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err),
+                 "tandem_decode_attention_static: this shape needs %zu bytes of split-K scratch, the built-in buffer holds %d; "
+                 "use tandem_decode_attention with your own scratch", need, TANDEM_STATIC_SCRATCH_BYTES);
+        return TANDEM_ERR_CAPACITY;
+    }
+    void* scratch = nullptr;
+    TRY(static_scratch_for_current_device(&scratch));
+    return tandem_decode_attention(q, k_derived, v_derived, k_own, v_own, out, scratch, (size_t)TANDEM_STATIC_SCRATCH_BYTES, batch,
+                                   n_heads, d_head, derived_len, own_len, stream);
 }
 
 extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t, const void* ln_g, const void* ln_b, const void* wk,
