@@ -15,8 +15,10 @@ struct LoopState {
     int* emitted;      // [B] tokens written to out_ids since the generate call began
     int* done;         // [B]
     int* out_ids;      // [B][out_cap]
-    int* counters;     // [0] iteration index since prefill, [1] live sequences, [2] error flags,
-                       // [3] max_b n_b, [4] sum_b n_b (both refreshed by every verify)
+    int* counters;     // [0] iteration index since prefill (advances while sequences are live), [1] live sequences,
+                       // [2] error flags, [3] max_b n_b, [4] sum_b n_b, [5] live iterations of the current call,
+                       // [6] verify kernels executed since the context was created (the host's ticket)
+    volatile int* host_flags;   // mapped pinned host memory: [0] ticket, [1] live, [2] n_max, [3] n_sum, [4] iterations
     unsigned long long* hist;   // [gamma_limit+1] accept-length histogram of live sequences
     int out_cap;
     int gamma_limit;
@@ -108,6 +110,7 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restric
 __global__ void verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed, int max_new) {
     const int b = threadIdx.x;
     const int iteration = st.counters[0];
+    const int live_before = st.counters[1];
     __syncthreads();
     if (b < batch && !st.done[b]) {
         const int* d = st.drafts + b * st.gamma_limit;
@@ -133,11 +136,20 @@ __global__ void verify_kernel(LoopState st, int batch, int gamma, int mode, unsi
     }
     __syncthreads();
     if (b == 0) {
-        st.counters[0] = iteration + 1;
+        if (live_before > 0) { st.counters[0] = iteration + 1; st.counters[5] += 1; }
         int n_max = 0, n_sum = 0;
         for (int i = 0; i < batch; ++i) { n_max = max(n_max, st.n[i]); n_sum += st.n[i]; }
         st.counters[3] = n_max;
         st.counters[4] = n_sum;
+        const int ticket = st.counters[6] + 1;
+        st.counters[6] = ticket;
+        // publish to the host: data first, then the ticket it polls on
+        st.host_flags[1] = st.counters[1];
+        st.host_flags[2] = n_max;
+        st.host_flags[3] = n_sum;
+        st.host_flags[4] = st.counters[5];
+        __threadfence_system();
+        st.host_flags[0] = ticket;
     }
 }
 

@@ -2,7 +2,9 @@
 #include <cuda_runtime.h>
 #include <limits.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
+#include <time.h>
 
 #include <algorithm>
 #include <mutex>
@@ -89,6 +91,20 @@ struct tandem_ctx {
     int64_t launches = 0;
     int last_gamma = 0;
     LoopState st;
+    // CUDA graphs of one iteration, keyed by everything baked into the captured launches
+    struct GraphEntry {
+        int kind, gamma, mode, max_new, batch, chunks;
+        uint64_t seed;
+        bool warm;
+        cudaGraphExec_t exec;
+        int64_t kernels;
+    };
+    std::vector<GraphEntry> graphs;
+    cudaStream_t cap_stream = nullptr;   // capture happens here (the caller's stream may be the legacy default stream)
+    bool use_graphs = true;
+    int chunks_launch = 1;               // attention grid size along the context for the current iteration
+    int32_t* hflags = nullptr;           // mapped pinned host memory the verify kernel publishes to
+    int64_t ticket = 0;                  // verify kernels enqueued since creation
 };
 
 namespace {
@@ -404,7 +420,8 @@ void large_pass(tandem_ctx& c, const Rows& r, bool project, bool head) {
 Rows decode_rows(tandem_ctx& c, int r_last, int nq) {
     Rows r;
     r.M = c.batch * nq; r.groups = c.batch; r.nq = nq; r.decode = true;
-    r.n_chunks = std::min(c.lay.n_chunks_max, (c.n_ub - 1 + r_last) / ATT_CH + 1);
+    (void)r_last;
+    r.n_chunks = c.chunks_launch;
     r.kv_positions = (double)c.n_sum + (double)c.batch * r_last;
     return r;
 }
@@ -463,6 +480,81 @@ tandem_status check_launch() {
     return TANDEM_OK;
 }
 
+void enqueue_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t seed, int max_new) {
+    const bool bf = c.cfg.dtype == TANDEM_DTYPE_BF16;
+    if (kind == 0) { if (bf) iteration<bf16>(c, gamma, mode, seed, max_new); else iteration<float>(c, gamma, mode, seed, max_new); }
+    else { if (bf) greedy_iteration<bf16>(c, max_new); else greedy_iteration<float>(c, max_new); }
+}
+
+// Enqueues one iteration on the context's stream: eagerly the first time a launch shape is seen (and whenever
+// per-launch profiling is on), as a CUDA graph afterwards.  kind 0 = draft + verify, 1 = plain greedy M_L.
+tandem_status launch_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t seed, int max_new) {
+    const int need = (c.n_ub - 1 + gamma) / ATT_CH + 1;
+    c.chunks_launch = std::min(c.lay.n_chunks_max, (need + 3) / 4 * 4);
+    c.ticket++;
+    if (c.prof.on || !c.use_graphs) {
+        enqueue_iteration(c, kind, gamma, mode, seed, max_new);
+        return check_launch();
+    }
+    tandem_ctx::GraphEntry* g = nullptr;
+    for (auto& e : c.graphs)
+        if (e.kind == kind && e.gamma == gamma && e.mode == mode && e.max_new == max_new && e.batch == c.batch &&
+            e.chunks == c.chunks_launch && e.seed == seed) { g = &e; break; }
+    if (!g) {
+        c.graphs.push_back({kind, gamma, mode, max_new, c.batch, c.chunks_launch, seed, false, nullptr, 0});
+        g = &c.graphs.back();
+    }
+    if (!g->warm) {   // first use: run eagerly (sets kernel attributes, surfaces launch errors outside a capture)
+        g->warm = true;
+        enqueue_iteration(c, kind, gamma, mode, seed, max_new);
+        return check_launch();
+    }
+    if (!g->exec) {
+        cudaStream_t user = c.stream;
+        const int64_t l0 = c.launches;
+        CK(cudaStreamBeginCapture(c.cap_stream, cudaStreamCaptureModeThreadLocal));
+        c.stream = c.cap_stream;
+        enqueue_iteration(c, kind, gamma, mode, seed, max_new);
+        c.stream = user;
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamEndCapture(c.cap_stream, &graph);
+        g->kernels = c.launches - l0;
+        c.launches = l0;
+        if (e == cudaSuccess) e = cudaGraphInstantiate(&g->exec, graph, 0);
+        if (graph) cudaGraphDestroy(graph);
+        if (e != cudaSuccess) {
+            g->exec = nullptr;
+            snprintf(g_cuda_err, sizeof(g_cuda_err), "%s while capturing an iteration", cudaGetErrorString(e));
+            return TANDEM_ERR_CUDA;
+        }
+    }
+    CK(cudaGraphLaunch(g->exec, c.stream));
+    c.launches += g->kernels;
+    return TANDEM_OK;
+}
+
+// Waits (bounded) until the verify kernel with the given ticket has published its results to the host.
+tandem_status wait_ticket(tandem_ctx& c, int64_t ticket) {
+    volatile int32_t* hf = c.hflags;
+    struct timespec t0, t1;
+    clock_gettime(CLOCK_MONOTONIC, &t0);
+    for (unsigned spin = 0; (int64_t)hf[0] < ticket; ++spin) {
+        if ((spin & 1023) == 1023) {
+            if (cudaStreamQuery(c.stream) != cudaErrorNotReady && (int64_t)hf[0] < ticket) {
+                // the stream drained (or failed) without publishing: report instead of spinning forever
+                cudaError_t e = cudaStreamSynchronize(c.stream);
+                if ((int64_t)hf[0] >= ticket) break;
+                snprintf(g_cuda_err, sizeof(g_cuda_err), "%s while waiting for an iteration", cudaGetErrorString(e));
+                return e == cudaSuccess ? TANDEM_ERR_TIMEOUT : TANDEM_ERR_CUDA;
+            }
+            clock_gettime(CLOCK_MONOTONIC, &t1);
+            if (t1.tv_sec - t0.tv_sec > 60) return TANDEM_ERR_TIMEOUT;
+        }
+    }
+    __sync_synchronize();
+    return TANDEM_OK;
+}
+
 tandem_status begin_call(tandem_ctx* c) {
     if (!c) return TANDEM_ERR_INVALID_ARG;
     CK(cudaSetDevice(c->cfg.device));
@@ -472,11 +564,10 @@ tandem_status begin_call(tandem_ctx* c) {
 __global__ void reset_call_kernel(LoopState st, int batch) {
     const int b = threadIdx.x;
     if (b < batch) { st.emitted[b] = 0; st.done[b] = 0; }
-    if (b == 0) st.counters[1] = batch;
+    if (b == 0) { st.counters[1] = batch; st.counters[5] = 0; }
 }
 
 }  // namespace
-
 // =====================================================================================================
 // exported entry points
 // =====================================================================================================
@@ -541,11 +632,22 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
     st.hist = at<unsigned long long>(*c, lay.st_hist);
     st.out_cap = cfg->max_seq; st.gamma_limit = TANDEM_GAMMA_LIMIT;
     cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&c->pinned), c->pinned_ints * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&c->hflags), 16 * sizeof(int32_t), cudaHostAllocMapped);
+    if (e == cudaSuccess) {
+        memset(c->hflags, 0, 16 * sizeof(int32_t));
+        int* dptr = nullptr;
+        e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&dptr), c->hflags, 0);
+        st.host_flags = dptr;
+    }
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
+    c->use_graphs = getenv("TANDEM_NO_GRAPH") == nullptr;
     if (e == cudaSuccess) e = cudaMemsetAsync(c->arena + lay.st_n, 0, lay.h_large - lay.st_n, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "%s in tandem_create", cudaGetErrorString(e));
         if (c->pinned) cudaFreeHost(c->pinned);
+        if (c->hflags) cudaFreeHost(c->hflags);
+        if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
         delete c;
         return TANDEM_ERR_CUDA;
     }
@@ -559,6 +661,9 @@ extern "C" tandem_status tandem_destroy(tandem_ctx* c) {
     cudaError_t e = cudaStreamSynchronize(c->stream);
     if (c->pinned) cudaFreeHost(c->pinned);
     for (cudaEvent_t ev : c->prof.ev) cudaEventDestroy(ev);
+    for (auto& g : c->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
+    if (c->hflags) cudaFreeHost(c->hflags);
+    if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     delete c;
     if (e != cudaSuccess) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "%s in tandem_destroy", cudaGetErrorString(e));
@@ -585,7 +690,9 @@ extern "C" tandem_status tandem_prefill(tandem_ctx* c, int32_t batch, const int3
     for (long long i = 0; i < total; ++i)
         if (prompt_ids[i] < 0 || prompt_ids[i] >= c->cfg.large.vocab) return TANDEM_ERR_INVALID_ARG;
 
-    CK(cudaStreamSynchronize(c->stream));   // staging buffer free again
+    CK(cudaStreamSynchronize(c->stream));   // staging buffer free again; no verify kernel in flight
+    c->ticket = 0;                          // the device-side ticket is cleared with the rest of the loop state below
+    c->hflags[0] = 0;
     const int M = (int)rows;
     int32_t* p_tok = c->pinned;
     int32_t* p_seq = p_tok + c->lay.max_rows;
@@ -647,11 +754,9 @@ extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t
     TRY(capacity_for(c, 0, gamma));
     reset_call_kernel<<<1, 256, 0, c->stream>>>(c->st, c->batch);
     c->launches++;
-    if (c->cfg.dtype == TANDEM_DTYPE_BF16) iteration<bf16>(*c, gamma, accept_mode, mode_seed, INT_MAX);
-    else iteration<float>(*c, gamma, accept_mode, mode_seed, INT_MAX);
+    TRY(launch_iteration(*c, 0, gamma, accept_mode, mode_seed, INT_MAX));
     c->n_ub += gamma + 1;
     c->n_sum += (long long)c->batch * (gamma + 1);
-    TRY(check_launch());
     if (result) {
         int32_t* cnt = c->pinned;   // staging is idle outside prefill
         CK(cudaMemcpyAsync(cnt, c->st.counters, 5 * 4, cudaMemcpyDeviceToHost, c->stream));
@@ -685,24 +790,42 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
     reset_call_kernel<<<1, 256, 0, c->stream>>>(c->st, B);
     c->launches++;
     CK(cudaMemsetAsync(c->st.hist, 0, (TANDEM_GAMMA_LIMIT + 1) * 8, c->stream));
-    int32_t* live = c->pinned;   // staging is idle outside prefill
-    int64_t iters = 0;
-    for (;;) {
-        if (speculative) {
-            if (c->cfg.dtype == TANDEM_DTYPE_BF16) iteration<bf16>(*c, gamma, mode, seed, max_new);
-            else iteration<float>(*c, gamma, mode, seed, max_new);
-        } else {
-            if (c->cfg.dtype == TANDEM_DTYPE_BF16) greedy_iteration<bf16>(*c, max_new);
-            else greedy_iteration<float>(*c, max_new);
+    // Iterations are enqueued ahead of the host's knowledge of their outcome.  None can be the last one before
+    // ceil(max_new / (gamma + 1)); after that at most DEPTH iterations are in flight beyond the last one whose
+    // result the host has seen (surplus iterations find every sequence frozen and change nothing).
+    const int DEPTH = 3;
+    const int kind = speculative ? 0 : 1;
+    const int64_t ticket0 = c->ticket;
+    const int min_iters = (max_new + gamma) / (gamma + 1);
+    const int n_known0 = c->n_ub;
+    int64_t enq = 0, seen = 0;   // iterations of this call enqueued / observed
+    int n_known = n_known0;      // max_b n_b after the last observed iteration
+    bool finished = false;
+    while (!finished) {
+        if (enq >= min_iters && enq - seen >= DEPTH) {
+            TRY(wait_ticket(*c, ticket0 + enq - DEPTH + 1));
         }
-        ++iters;
-        CK(cudaMemcpyAsync(live, c->st.counters, 5 * 4, cudaMemcpyDeviceToHost, c->stream));
-        CK(cudaStreamSynchronize(c->stream));
-        c->n_ub = live[3];
-        c->n_sum = live[4];
-        if (live[1] <= 0) break;
-        if (iters > (int64_t)max_new + 1) return TANDEM_ERR_STATE;   // every iteration emits at least one token
+        // take whatever has been published so far
+        const int64_t pub = (int64_t)((volatile int32_t*)c->hflags)[0] - ticket0;
+        if (pub > seen) {
+            __sync_synchronize();
+            seen = std::min<int64_t>(pub, enq);
+            n_known = c->hflags[2];
+            c->n_sum = c->hflags[3];
+            if (seen >= min_iters && c->hflags[1] <= 0) finished = true;
+        }
+        if (finished) break;
+        if (enq > (int64_t)max_new + DEPTH + 1) return TANDEM_ERR_STATE;   // every live iteration emits a token
+        c->n_ub = std::min<long long>((long long)n_known + (enq - seen) * (gamma + 1), (long long)n_known0 + max_new);
+        TRY(launch_iteration(*c, kind, gamma, mode, seed, max_new));
+        ++enq;
     }
+    int32_t* cnt = c->pinned;   // staging is idle outside prefill
+    CK(cudaMemcpyAsync(cnt, c->st.counters, 8 * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    c->n_ub = cnt[3];
+    c->n_sum = cnt[4];
+    const int64_t iters = cnt[5];
     TRY(check_launch());
     CK(cudaMemcpy2DAsync(out_ids, (size_t)max_new * 4, c->st.out_ids, (size_t)c->st.out_cap * 4, (size_t)max_new * 4, B,
                          cudaMemcpyDeviceToHost, c->stream));
