@@ -197,9 +197,10 @@ TANDEM_API int64_t tandem_launch_count(tandem_ctx* ctx);
  *   q, out           [batch][n_heads][d_head]
  *   k_derived, v_derived  [batch][n_heads][derived_len][d_head]
  *   k_own, v_own     [batch][n_heads][own_len][d_head]
- *   scratch          split-K partial results, fp32, at least tandem_decode_attention_scratch_bytes(...)
+ *   scratch          split-K partial results and merge tickets, at least tandem_decode_attention_scratch_bytes(...)
  * d_head in {32, 64, 128}.  The context is cut into fixed chunks by absolute position; each chunk yields
- * (max, sum, weighted values) and a second kernel merges the chunks in position order. */
+ * (max, sum, weighted values), and the CTA of a (sequence, head) that finishes last merges the chunks in
+ * position order. */
 TANDEM_API size_t tandem_decode_attention_scratch_bytes(int32_t batch, int32_t n_heads, int32_t d_head,
                                              int32_t derived_len, int32_t own_len);
 TANDEM_API tandem_status tandem_decode_attention(const void* q, const void* k_derived, const void* v_derived,
@@ -226,7 +227,8 @@ TANDEM_API tandem_status tandem_decode_attention(const void* q, const void* k_de
  *    any stream capture is begun on the device.  Later calls only launch.
  *  - The call itself allocates nothing on host or device and frees nothing.
  *  - All calls on a device share the one buffer, and it keeps whatever the previous call left there.  The
- *    kernels overwrite every partial result they later read, so nothing needs clearing between calls; but
+ *    kernels overwrite every partial result they later read and each call clears the merge tickets itself
+ *    (a memset on the stream), so the caller clears nothing between calls; but
  *    two calls that can overlap on the GPU (different streams, or one stream and a graph) race on it and
  *    give wrong results.  Keep calls to this entry point on one stream, or order them with events. */
 #define TANDEM_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
@@ -236,10 +238,15 @@ TANDEM_API tandem_status tandem_decode_attention_static(const void* q, const voi
                                                         int32_t derived_len, int32_t own_len, void* stream);
 
 /* tandem_ff_tandem_project: the linear FF_Tandem of Eq. 2 (first line) followed by the small layer's
- * LayerNorm and key/value maps, written as bf16 keys/values.  All pointers DEVICE.
+ * LayerNorm and key/value maps, written as bf16 keys/values.  All pointers DEVICE, 16-byte aligned.
  *   x [rows][d_large] bf16;  w_t [d_small][d_large] bf16;  ln_g, ln_b [d_small] fp32;
  *   wk, wv [d_small][d_small] bf16;  k_out, v_out [rows][d_small] bf16;
- *   scratch: fp32, at least rows * d_small * 4 + rows * d_small * 2 bytes.  rows <= 256. */
+ *   scratch: at least tandem_ff_tandem_project_scratch_bytes(rows, d_small) bytes (the fp32 projection,
+ *   split-K partial sums and their tickets).  rows <= 256; d_large, d_small multiples of 8.
+ * Up to 64 rows the two GEMMs stream their weights once on the tensor cores with the LayerNorm fused into
+ * the second one's operand load and the key/value write as its epilogue; above that they are tiled GEMMs
+ * with a LayerNorm kernel in between. */
+TANDEM_API size_t tandem_ff_tandem_project_scratch_bytes(int32_t rows, int32_t d_small);
 TANDEM_API tandem_status tandem_ff_tandem_project(const void* x, const void* w_t, const void* ln_g, const void* ln_b,
                                        const void* wk, const void* wv, void* k_out, void* v_out,
                                        void* scratch, size_t scratch_bytes, int32_t rows, int32_t d_large,

@@ -26,6 +26,7 @@ STATUS_NAMES = ["OK", "INVALID_ARG", "SHAPE", "ARENA_TOO_SMALL", "CAPACITY", "ST
 EXPORTS = ["tandem_query_arena", "tandem_create", "tandem_destroy", "tandem_prefill", "tandem_block_step",
            "tandem_speculative_generate", "tandem_large_greedy_generate", "tandem_debug_read",
            "tandem_decode_attention_scratch_bytes", "tandem_decode_attention", "tandem_ff_tandem_project",
+           "tandem_ff_tandem_project_scratch_bytes",
            "tandem_status_string", "tandem_last_cuda_error", "tandem_profile_enable", "tandem_profile_read",
            "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static"]
 
@@ -91,6 +92,8 @@ def load_library():
     lib.tandem_decode_attention_scratch_bytes.restype = sz
     lib.tandem_decode_attention.argtypes = [vp] * 7 + [sz] + [i32] * 5 + [vp]
     lib.tandem_ff_tandem_project.argtypes = [vp] * 9 + [sz] + [i32] * 3 + [vp]
+    lib.tandem_ff_tandem_project_scratch_bytes.argtypes = [i32] * 2
+    lib.tandem_ff_tandem_project_scratch_bytes.restype = sz
     lib.tandem_decode_attention_static.argtypes = [vp] * 6 + [i32] * 5 + [vp]
     lib.tandem_profile_enable.argtypes = [vp, i32]
     lib.tandem_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_double)]
@@ -101,7 +104,8 @@ def load_library():
         fn = getattr(lib, name)
         if name.endswith("_string") or name.endswith("_cuda_error") or name.endswith("_class_name"):
             fn.restype = C.c_char_p
-        elif name not in ("tandem_decode_attention_scratch_bytes", "tandem_launch_count"):
+        elif name not in ("tandem_decode_attention_scratch_bytes", "tandem_ff_tandem_project_scratch_bytes",
+                          "tandem_launch_count"):
             fn.restype = C.c_int
     lib.tandem_status_string.argtypes = [C.c_int]
     lib.tandem_last_cuda_error.argtypes = []
@@ -312,7 +316,7 @@ def tandem_ff_tandem_project(x, w_t, ln_g, ln_b, wk, wv, scratch=None):
     k = torch.empty(rows, d_s, dtype=torch.bfloat16, device=x.device)
     v = torch.empty_like(k)
     if scratch is None:
-        scratch = torch.empty(rows * d_s * 6 + rows * 8 + 1024, dtype=torch.uint8, device=x.device)
+        scratch = torch.empty(lib.tandem_ff_tandem_project_scratch_bytes(rows, d_s), dtype=torch.uint8, device=x.device)
     ptr = lambda t: C.c_void_p(t.data_ptr())
     _check(lib.tandem_ff_tandem_project(ptr(x), ptr(w_t), ptr(ln_g), ptr(ln_b), ptr(wk), ptr(wv), ptr(k), ptr(v),
                                         ptr(scratch), scratch.numel(), rows, d_l, d_s,

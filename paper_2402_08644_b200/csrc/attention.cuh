@@ -9,13 +9,14 @@
 //   * the prompt pass (LOOP = true): a group of consecutive queries sweeps all chunks up to its last position.
 //
 // The context is cut into chunks of ATT_CH positions anchored at absolute position 0.  In split mode one
-// CTA handles one chunk and writes (max, sum, weighted values) per query; attn_merge_kernel combines the
-// chunks in position order.  A query's arithmetic never depends on how many other queries ride along,
+// CTA handles one chunk and writes (max, sum, weighted values) per query; the CTA of a (group, head)
+// that finishes last combines the chunks in position order.  A query's arithmetic never depends on how many other queries ride along,
 // so a block pass and single-token passes produce identical bits.
 #pragma once
 #include <limits.h>
 #include <math.h>
 #include "common.cuh"
+#include "tc_common.cuh"
 
 namespace tandem {
 
@@ -37,6 +38,7 @@ struct AttnArgs {
     float* part_acc;                     //             [M][H][n_chunks_max][DH]
     int n_chunks_max;
     float scale;
+    int* merge_counters;                 // split mode: [groups][H], zero between launches
 };
 
 template <typename T, int DH>
@@ -54,6 +56,9 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
     constexpr int QS = ATT_THREADS / DH;        // query stride of the value phase
     constexpr int QPT = (ATT_NQ + QS - 1) / QS; // queries per thread in the value phase
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int s_last;
+    pdl_launch_dependents();   // the next kernel may start fetching its weights
+    pdl_wait();                // queries and keys/values come from earlier kernels
     T* ks = reinterpret_cast<T*>(smem_raw);
     T* vs = ks + ATT_CH * LD;
     float* qs = reinterpret_cast<float*>(vs + ATT_CH * LD);
@@ -172,31 +177,48 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
             }
         }
     }
+    T* og = static_cast<T*>(a.out);
     if (LOOP) {
-        T* og = static_cast<T*>(a.out);
 #pragma unroll
         for (int i = 0; i < QPT; ++i) {
             const int qi = qsub + i * QS;
             if (qi < cnt) og[(size_t)(row0 + qi) * a.ldo + h * DH + e] = from_float<T>(racc[i] / rl[i]);
         }
+    } else {
+        // The CTA that finishes last for this (group, head) merges every query's chunks in position order.
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            const int active = min((int)gridDim.x, pos_last / ATT_CH + 1);   // CTAs that got this far
+            int* counter = a.merge_counters + (size_t)g * a.n_heads + h;
+            const int t = atomicAdd(counter, 1);
+            s_last = (t == active - 1);
+            if (t == active - 1) *counter = 0;   // ready for the next launch
+        }
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+#pragma unroll
+        for (int i = 0; i < QPT; ++i) {
+            const int qi = qsub + i * QS;
+            if (qi >= cnt) continue;
+            const int nc = (pos_first + qi) / ATT_CH + 1;
+            const size_t base = ((size_t)(row0 + qi) * a.n_heads + h) * a.n_chunks_max;
+            float mx = -INFINITY;
+#pragma unroll 8
+            for (int c = 0; c < nc; ++c) mx = fmaxf(mx, __ldcg(a.part_ml + (base + c) * 2));
+            float l = 0.f, o = 0.f;
+#pragma unroll 4
+            for (int c = 0; c < nc; ++c) {
+                const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (base + c) * 2));
+                const float pa = __ldcg(a.part_acc + (base + c) * DH + e);
+                const float f = expf(ml.x - mx);
+                l = fmaf(ml.y, f, l);
+                o = fmaf(pa, f, o);
+            }
+            og[(size_t)(row0 + qi) * a.ldo + h * DH + e] = from_float<T>(o / l);
+        }
     }
-}
-
-// grid: (rows, heads); block: DH threads.  Merges a query's chunks in position order.
-template <typename T, int DH>
-__global__ void attn_merge_kernel(AttnArgs a) {
-    const int row = blockIdx.x, h = blockIdx.y, e = threadIdx.x;
-    const int nc = a.row_pos[row] / ATT_CH + 1;
-    const size_t base = ((size_t)row * a.n_heads + h) * a.n_chunks_max;
-    float mx = -INFINITY;
-    for (int c = 0; c < nc; ++c) mx = fmaxf(mx, a.part_ml[(base + c) * 2]);
-    float l = 0.f, o = 0.f;
-    for (int c = 0; c < nc; ++c) {
-        const float f = expf(a.part_ml[(base + c) * 2] - mx);
-        l = fmaf(a.part_ml[(base + c) * 2 + 1], f, l);
-        o = fmaf(a.part_acc[(base + c) * DH + e], f, o);
-    }
-    static_cast<T*>(a.out)[(size_t)row * a.ldo + h * DH + e] = from_float<T>(o / l);
 }
 
 }  // namespace tandem

@@ -1,0 +1,477 @@
+// bf16 GEMMs  y[m][n] = sum_k x[m][k] * W[n][k]  on the tcgen05 tensor cores, fp32 accumulation in TMEM.
+//
+//  gemm_tc_decode_kernel   few rows (<= 64): the weight matrix is the MMA's A operand (128 output features
+//                          per tile on the TMEM lanes), the token rows are the B operand (16..64 columns).
+//                          The job is streaming W once from HBM: every CTA owns one (tile, K-slice) unit so
+//                          that all SMs pull weights, tiles arrive by TMA through a ring of stages, and the
+//                          K-slices of a tile are summed in slice order by the CTA that finishes last.
+//                          The token rows are written into the B stages by the CTA's own threads, which is
+//                          where the LayerNorm (or the fp32 -> bf16 cast) of the residual stream is fused.
+//                          The weight loads are issued before the kernel waits for its predecessor in the
+//                          stream (programmatic dependent launch), so they overlap its tail.
+//  gemm_tc_tiled_kernel    many rows (prompt pass): 128 x 128 output tiles, both operands by TMA.
+//
+// An output element's reduction order depends on (N, K) only, never on the number of rows, so a block
+// pass and a one-row pass give identical bits.
+#pragma once
+#include <limits.h>
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "tc_common.cuh"
+
+namespace tandem {
+
+enum { PRO_BF16 = 0, PRO_LN = 1, PRO_CAST = 2 };   // how the token rows become the bf16 B operand
+constexpr int EPI_ARGMAX = 6;                       // fp32 store plus the (max, index) of each row within the tile
+enum { TC_ERR_SLOT = 1, TC_ERR_OPERANDS = 2, TC_ERR_ACCUM = 3 };   // which bounded wait gave up
+
+struct TcDecodeArgs {
+    const void* x;          // PRO_BF16: bf16 [rows][ldx];  PRO_LN / PRO_CAST: float [rows][ldx]
+    int ldx;
+    const float* ln_g;      // PRO_LN: LayerNorm gain / bias [K]
+    const float* ln_b;
+    int rows, K, N;         // N = output features over all segments
+    int seg_rows;           // output features per weight segment (one tensor map each)
+    int tiles_per_seg;      // ceil(seg_rows / 128)
+    int splits;             // K-slices per tile; grid = tiles * splits
+    int stream_weights;     // 1: weights are read once per pass and should not stay in L2
+    float* partials;        // [tiles * splits][NB][128] fp32, used when splits > 1
+    int* tile_counters;     // [tiles], zero between launches
+    int* err_flag;          // nullable
+    float* amax_val;        // EPI_ARGMAX: [rows][amax_stride] best value per tile
+    int* amax_idx;          //             and its output feature
+    int amax_stride;
+    EpiArgs e;
+};
+
+constexpr int TCD_THREADS = 192;   // warps 0-3: B operand + epilogue; warp 4: TMA; warp 5: TMEM + MMA issue
+template <int NB> struct TcdCfg {
+    static constexpr int STAGES = NB <= 32 ? 5 : 4;
+    static constexpr int A_BYTES = 128 * 128;       // 128 weight rows x 64 bf16
+    static constexpr int B_BYTES = NB * 128;        // NB token rows x 64 bf16
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024
+    static constexpr int TMEM_COLS = NB <= 32 ? 32 : 64;
+};
+
+__device__ __forceinline__ void tc_report(int* err_flag, int code) {
+    if (err_flag) atomicExch(err_flag, code);
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
+}
+
+template <int NB, int PRO, int EPI>
+__global__ void __launch_bounds__(TCD_THREADS)
+gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap tm0, const __grid_constant__ CUtensorMap tm1,
+                      const __grid_constant__ CUtensorMap tm2) {
+    using C = TcdCfg<NB>;
+    extern __shared__ __align__(1024) unsigned char smem_dyn[];
+    __shared__ __align__(8) uint64_t s_full[C::STAGES];
+    __shared__ __align__(8) uint64_t s_empty[C::STAGES];
+    __shared__ __align__(8) uint64_t s_accum;
+    __shared__ uint32_t s_tmem;
+    __shared__ int s_last;
+    __shared__ float s_mu[NB], s_rstd[NB];
+    __shared__ float s_av[4][NB];
+    __shared__ int s_ai[4][NB];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t ring0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // shared-space address of stage 0
+    unsigned char* ring = smem_dyn + (ring0 - smem_u32(smem_dyn));         // the same place as a generic pointer
+
+    const int S = a.splits;
+    const int unit = blockIdx.x;
+    const int tile = unit / S, sp = unit - tile * S;
+    const int seg = tile / a.tiles_per_seg;
+    const int n_local0 = (tile - seg * a.tiles_per_seg) * 128;
+    const int KB = (a.K + 63) >> 6;
+    const int kb_base = KB / S, kb_rem = KB - kb_base * S;
+    const int kb0 = sp * kb_base + min(sp, kb_rem);
+    const int nkb = kb_base + (sp < kb_rem ? 1 : 0);
+
+    if (warp == 5) {
+        if (lane == 0) {
+            for (int s = 0; s < C::STAGES; ++s) {
+                mbar_init(smem_u32(&s_full[s]), 5);    // the TMA thread's arrive + one arrive per B-operand warp
+                mbar_init(smem_u32(&s_empty[s]), 1);   // the MMA thread's commit
+            }
+            mbar_init(smem_u32(&s_accum), 1);
+            mbar_init_fence();
+        }
+        __syncwarp();
+        tmem_alloc(smem_u32(&s_tmem), C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = s_tmem;
+    pdl_launch_dependents();
+
+    if (warp == 4) {
+        // ---- weight tiles: independent of every earlier kernel, so no wait on the predecessor here ----
+        if (lane == 0) {
+            const CUtensorMap* tm = seg == 0 ? &tm0 : (seg == 1 ? &tm1 : &tm2);
+            tma_prefetch_desc(tm);
+            const uint64_t pol = l2_policy_evict_first();
+            for (int i = 0; i < nkb; ++i) {
+                const int st = i % C::STAGES;
+                if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
+                    tc_report(a.err_flag, TC_ERR_SLOT);
+                    break;
+                }
+                const uint32_t bar = smem_u32(&s_full[st]);
+                mbar_arrive_expect_tx(bar, C::A_BYTES);
+                if (a.stream_weights) tma_load_2d(ring0 + st * C::STAGE_BYTES, tm, (kb0 + i) * 64, n_local0, bar, pol);
+                else tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES, tm, (kb0 + i) * 64, n_local0, bar);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        // ---- MMA issue: one thread ----
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(128, NB);
+            for (int i = 0; i < nkb; ++i) {
+                const int st = i % C::STAGES;
+                if (!mbar_wait(smem_u32(&s_full[st]), (i / C::STAGES) & 1)) {
+                    tc_report(a.err_flag, TC_ERR_OPERANDS);
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint64_t da = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES);
+                const uint64_t db = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES + C::A_BYTES);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)   // 4 x 16 elements of K per stage
+                    umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
+                umma_commit(smem_u32(&s_empty[st]));
+            }
+            umma_commit(smem_u32(&s_accum));
+        }
+        __syncwarp();
+    } else {
+        // ---- warps 0-3: token rows into the B stages, then the epilogue ----
+        pdl_wait();   // x (and everything the epilogue touches) comes from earlier kernels
+        if (PRO == PRO_LN) {
+            // Row statistics, one warp per row in a fixed lane-strided order (so they do not depend on how many
+            // rows ride along).  Rows of up to 1024 elements stay in registers between the two passes.
+            const int K4 = a.K >> 2;
+            for (int r = warp; r < a.rows; r += 4) {
+                const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx);
+                float mu, var;
+                if (K4 <= 256) {
+                    float4 t[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) t[u] = (lane + 32 * u < K4) ? __ldcg(xr + lane + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    float s = 0.f;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) s += (t[u].x + t[u].y) + (t[u].z + t[u].w);
+                    mu = warp_sum(s) / (float)a.K;
+                    float q = 0.f;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (lane + 32 * u < K4) {
+                            const float d0 = t[u].x - mu, d1 = t[u].y - mu, d2 = t[u].z - mu, d3 = t[u].w - mu;
+                            q = fmaf(d0, d0, q); q = fmaf(d1, d1, q); q = fmaf(d2, d2, q); q = fmaf(d3, d3, q);
+                        }
+                    }
+                    var = warp_sum(q) / (float)a.K;
+                } else {
+                    float s = 0.f;
+#pragma unroll 8
+                    for (int k4 = lane; k4 < K4; k4 += 32) { const float4 t = __ldcg(xr + k4); s += (t.x + t.y) + (t.z + t.w); }
+                    mu = warp_sum(s) / (float)a.K;
+                    float q = 0.f;
+#pragma unroll 8
+                    for (int k4 = lane; k4 < K4; k4 += 32) {
+                        const float4 t = __ldcg(xr + k4);
+                        const float d0 = t.x - mu, d1 = t.y - mu, d2 = t.z - mu, d3 = t.w - mu;
+                        q = fmaf(d0, d0, q); q = fmaf(d1, d1, q); q = fmaf(d2, d2, q); q = fmaf(d3, d3, q);
+                    }
+                    var = warp_sum(q) / (float)a.K;
+                }
+                if (lane == 0) { s_mu[r] = mu; s_rstd[r] = 1.0f / sqrtf(var + 1e-5f); }
+            }
+            bar_sync(1, 128);
+        }
+        for (int i = 0; i < nkb; ++i) {
+            const int st = i % C::STAGES;
+            if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
+                tc_report(a.err_flag, TC_ERR_SLOT);
+                break;
+            }
+            unsigned char* bt = ring + st * C::STAGE_BYTES + C::A_BYTES;
+            for (int idx = tid; idx < NB * 8; idx += 128) {
+                const int r = idx >> 3, c = idx & 7;
+                const int k = (kb0 + i) * 64 + c * 8;
+                uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                if (r < a.rows && k < a.K) {
+                    if (PRO == PRO_BF16) {
+                        val = __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k));
+                    } else {
+                        const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
+                        float4 u0 = __ldcg(xp), u1 = __ldcg(xp + 1);
+                        if (PRO == PRO_LN) {
+                            const float mu = s_mu[r], rs = s_rstd[r];
+                            const float4 g0 = __ldg(reinterpret_cast<const float4*>(a.ln_g + k)), g1 = __ldg(reinterpret_cast<const float4*>(a.ln_g + k) + 1);
+                            const float4 b0 = __ldg(reinterpret_cast<const float4*>(a.ln_b + k)), b1 = __ldg(reinterpret_cast<const float4*>(a.ln_b + k) + 1);
+                            u0.x = (u0.x - mu) * rs * g0.x + b0.x; u0.y = (u0.y - mu) * rs * g0.y + b0.y;
+                            u0.z = (u0.z - mu) * rs * g0.z + b0.z; u0.w = (u0.w - mu) * rs * g0.w + b0.w;
+                            u1.x = (u1.x - mu) * rs * g1.x + b1.x; u1.y = (u1.y - mu) * rs * g1.y + b1.y;
+                            u1.z = (u1.z - mu) * rs * g1.z + b1.z; u1.w = (u1.w - mu) * rs * g1.w + b1.w;
+                        }
+                        val.x = pack_bf16x2(u0.x, u0.y); val.y = pack_bf16x2(u0.z, u0.w);
+                        val.z = pack_bf16x2(u1.x, u1.y); val.w = pack_bf16x2(u1.z, u1.w);
+                    }
+                }
+                // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
+                *reinterpret_cast<uint4*>(bt + r * 128 + ((c ^ (r & 7)) << 4)) = val;
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_full[st]));
+        }
+
+        if (!mbar_wait(smem_u32(&s_accum), 0)) tc_report(a.err_flag, TC_ERR_ACCUM);
+        tc_fence_after_sync();
+        float v[NB];
+#pragma unroll
+        for (int c0 = 0; c0 < NB; c0 += 16) {
+            float t[16];
+            tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c0, t);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[c0 + i] = t[i];
+        }
+        const int tl = warp * 32 + lane;             // output feature within the tile = TMEM lane
+        const int n_local = n_local0 + tl;
+        const bool valid = n_local < a.seg_rows;
+        const int n = seg * a.seg_rows + n_local;
+        bool finish = true;
+        if (S > 1) {
+            float* mine = a.partials + (size_t)unit * NB * 128 + tl;
+#pragma unroll
+            for (int j = 0; j < NB; ++j)
+                if (j < a.rows) mine[j * 128] = v[j];
+            __threadfence();
+            bar_sync(1, 128);
+            if (tid == 0) {
+                const int t = atomicAdd(a.tile_counters + tile, 1);
+                s_last = (t == S - 1);
+                if (t == S - 1) a.tile_counters[tile] = 0;   // ready for the next launch
+            }
+            bar_sync(1, 128);
+            finish = s_last != 0;
+            if (finish) {
+                __threadfence();
+                const float* base = a.partials + (size_t)tile * S * NB * 128 + tl;
+                constexpr int U = NB <= 16 ? 4 : (NB <= 32 ? 2 : 1);   // slices fetched together; summed in slice order
+#pragma unroll
+                for (int j = 0; j < NB; ++j) v[j] = 0.f;
+                for (int s0 = 0; s0 < S; s0 += U) {
+                    float t[U][NB];
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+#pragma unroll
+                        for (int j = 0; j < NB; ++j)
+                            t[u][j] = (s0 + u < S && j < a.rows) ? __ldcg(base + ((size_t)(s0 + u) * NB + j) * 128) : 0.f;
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+#pragma unroll
+                        for (int j = 0; j < NB; ++j)
+                            if (s0 + u < S) v[j] += t[u][j];
+                }
+            }
+        }
+        if (finish) {
+            if (EPI == EPI_ARGMAX) {
+                float* out = static_cast<float*>(a.e.out);
+#pragma unroll
+                for (int j = 0; j < NB; ++j) {
+                    if (j < a.rows) {
+                        float bv = valid ? v[j] : -INFINITY;
+                        int bi = valid ? n : INT_MAX;
+                        if (valid) out[(size_t)j * a.e.ldo + n] = v[j];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+                        }
+                        if (lane == 0) { s_av[warp][j] = bv; s_ai[warp][j] = bi; }
+                    }
+                }
+                bar_sync(1, 128);
+                if (tid < a.rows) {
+                    float bv = s_av[0][tid];
+                    int bi = s_ai[0][tid];
+                    for (int w = 1; w < 4; ++w)
+                        if (s_av[w][tid] > bv || (s_av[w][tid] == bv && s_ai[w][tid] < bi)) { bv = s_av[w][tid]; bi = s_ai[w][tid]; }
+                    a.amax_val[(size_t)tid * a.amax_stride + tile] = bv;
+                    a.amax_idx[(size_t)tid * a.amax_stride + tile] = bi;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < NB; ++j)
+                    if (j < a.rows && valid) epilogue<bf16, EPI>(a.e, j, n, v[j]);
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem, C::TMEM_COLS);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Many rows: 128 x 128 output tiles, A = token rows, B = weight rows, both by TMA.
+// ---------------------------------------------------------------------------------------------------
+
+struct TcTiledArgs {
+    int M, K, N;
+    int seg_rows, tiles_per_seg;
+    int* err_flag;
+    EpiArgs e;
+};
+
+constexpr int TCT_THREADS = 192;
+constexpr int TCT_STAGES = 6;
+constexpr int TCT_TILE_BYTES = 128 * 128;
+constexpr int TCT_STAGE_BYTES = 2 * TCT_TILE_BYTES;
+constexpr int TCT_SMEM_BYTES = TCT_STAGES * TCT_STAGE_BYTES + 1024;
+constexpr int TCT_TMEM_COLS = 128;
+
+// Sixteen consecutive output features of one row.  n_local0 is a multiple of 16.
+template <int EPI>
+__device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int seg, int seg_rows, int n_local0, const float (&v)[16]) {
+    const int n0 = seg * seg_rows + n_local0;
+    if (n_local0 + 16 > seg_rows || (e.ldo & 7) || (seg_rows & 7)) {
+        for (int i = 0; i < 16; ++i)
+            if (n_local0 + i < seg_rows) epilogue<bf16, EPI>(e, m, n0 + i, v[i]);
+        return;
+    }
+    if (EPI == EPI_STORE_F32 || EPI == EPI_RESID) {
+        float4* p = reinterpret_cast<float4*>(static_cast<float*>(e.out) + (size_t)m * e.ldo + n0);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float4 t = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            if (EPI == EPI_RESID) { const float4 o = p[i]; t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w; }
+            p[i] = t;
+        }
+        return;
+    }
+    uint4 lo, hi;
+    if (EPI == EPI_GELU) {
+        lo.x = pack_bf16x2(gelu_exact(v[0]), gelu_exact(v[1])); lo.y = pack_bf16x2(gelu_exact(v[2]), gelu_exact(v[3]));
+        lo.z = pack_bf16x2(gelu_exact(v[4]), gelu_exact(v[5])); lo.w = pack_bf16x2(gelu_exact(v[6]), gelu_exact(v[7]));
+        hi.x = pack_bf16x2(gelu_exact(v[8]), gelu_exact(v[9])); hi.y = pack_bf16x2(gelu_exact(v[10]), gelu_exact(v[11]));
+        hi.z = pack_bf16x2(gelu_exact(v[12]), gelu_exact(v[13])); hi.w = pack_bf16x2(gelu_exact(v[14]), gelu_exact(v[15]));
+    } else {
+        lo.x = pack_bf16x2(v[0], v[1]); lo.y = pack_bf16x2(v[2], v[3]); lo.z = pack_bf16x2(v[4], v[5]); lo.w = pack_bf16x2(v[6], v[7]);
+        hi.x = pack_bf16x2(v[8], v[9]); hi.y = pack_bf16x2(v[10], v[11]); hi.z = pack_bf16x2(v[12], v[13]); hi.w = pack_bf16x2(v[14], v[15]);
+    }
+    bf16* dst;
+    if (EPI == EPI_STORE || EPI == EPI_GELU) {
+        dst = static_cast<bf16*>(e.out) + (size_t)m * e.ldo + n0;
+    } else {   // EPI_QKV / EPI_KV: the query goes to its buffer, keys and values straight into the cache
+        int s = seg;
+        if (EPI == EPI_QKV && s == 0) {
+            dst = static_cast<bf16*>(e.out) + (size_t)m * e.ldo + n_local0;
+        } else {
+            if (EPI == EPI_QKV) s -= 1;
+            const int h = n_local0 / e.d_head, el = n_local0 - h * e.d_head;
+            const size_t idx = (((size_t)e.row_seq[m] * e.n_heads + h) * e.t_max + e.row_pos[m]) * e.d_head + el;
+            dst = static_cast<bf16*>(s == 0 ? e.kcache : e.vcache) + idx;
+        }
+    }
+    reinterpret_cast<uint4*>(dst)[0] = lo;
+    reinterpret_cast<uint4*>(dst)[1] = hi;
+}
+
+// grid: (tiles over all segments, ceil(M / 128)); dynamic smem TCT_SMEM_BYTES.
+template <int EPI>
+__global__ void __launch_bounds__(TCT_THREADS)
+gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tm0,
+                     const __grid_constant__ CUtensorMap tm1, const __grid_constant__ CUtensorMap tm2) {
+    extern __shared__ __align__(1024) unsigned char smem_dyn[];
+    __shared__ __align__(8) uint64_t s_full[TCT_STAGES];
+    __shared__ __align__(8) uint64_t s_empty[TCT_STAGES];
+    __shared__ __align__(8) uint64_t s_accum;
+    __shared__ uint32_t s_tmem;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t ring0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    const int tile = blockIdx.x;
+    const int seg = tile / a.tiles_per_seg;
+    const int n_local0 = (tile - seg * a.tiles_per_seg) * 128;
+    const int m0 = blockIdx.y * 128;
+    const int KB = (a.K + 63) >> 6;
+
+    if (warp == 5) {
+        if (lane == 0) {
+            for (int s = 0; s < TCT_STAGES; ++s) { mbar_init(smem_u32(&s_full[s]), 1); mbar_init(smem_u32(&s_empty[s]), 1); }
+            mbar_init(smem_u32(&s_accum), 1);
+            mbar_init_fence();
+        }
+        __syncwarp();
+        tmem_alloc(smem_u32(&s_tmem), TCT_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = s_tmem;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            const CUtensorMap* tw = seg == 0 ? &tm0 : (seg == 1 ? &tm1 : &tm2);
+            tma_prefetch_desc(&tmx);
+            tma_prefetch_desc(tw);
+            for (int i = 0; i < KB; ++i) {
+                const int st = i % TCT_STAGES;
+                if (i >= TCT_STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / TCT_STAGES) - 1) & 1)) {
+                    tc_report(a.err_flag, TC_ERR_SLOT);
+                    break;
+                }
+                const uint32_t bar = smem_u32(&s_full[st]);
+                mbar_arrive_expect_tx(bar, TCT_STAGE_BYTES);
+                tma_load_2d_nohint(ring0 + st * TCT_STAGE_BYTES, &tmx, i * 64, m0, bar);
+                tma_load_2d_nohint(ring0 + st * TCT_STAGE_BYTES + TCT_TILE_BYTES, tw, i * 64, n_local0, bar);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
+            for (int i = 0; i < KB; ++i) {
+                const int st = i % TCT_STAGES;
+                if (!mbar_wait(smem_u32(&s_full[st]), (i / TCT_STAGES) & 1)) {
+                    tc_report(a.err_flag, TC_ERR_OPERANDS);
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint64_t da = umma_desc_k_sw128(ring0 + st * TCT_STAGE_BYTES);
+                const uint64_t db = umma_desc_k_sw128(ring0 + st * TCT_STAGE_BYTES + TCT_TILE_BYTES);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
+                umma_commit(smem_u32(&s_empty[st]));
+            }
+            umma_commit(smem_u32(&s_accum));
+        }
+        __syncwarp();
+    } else {
+        if (!mbar_wait(smem_u32(&s_accum), 0)) tc_report(a.err_flag, TC_ERR_ACCUM);
+        tc_fence_after_sync();
+        const int m = m0 + warp * 32 + lane;   // output row = TMEM lane
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 16) {
+            float t[16];
+            tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c0, t);   // warp-wide: every lane takes part
+            if (m < a.M && n_local0 + c0 < a.seg_rows) epilogue16<EPI>(a.e, m, seg, a.seg_rows, n_local0 + c0, t);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc(tmem, TCT_TMEM_COLS);
+}
+
+}  // namespace tandem

@@ -1,7 +1,9 @@
 // Row set-up, embedding, LayerNorm, casts, arg-max, and the verify / accept / rollback kernel.
 #pragma once
 #include <math.h>
+#include <limits.h>
 #include "common.cuh"
+#include "tc_common.cuh"
 
 namespace tandem {
 
@@ -43,6 +45,66 @@ __global__ void embed_kernel(const int* __restrict__ row_tok, const int* __restr
     const T* er = emb + (size_t)row_tok[m] * d;
     const T* pr = pos + (size_t)row_pos[m] * d;
     for (int i = threadIdx.x; i < d; i += blockDim.x) h[(size_t)m * d + i] = to_float(er[i]) + to_float(pr[i]);
+}
+
+// Arg-max of one row from the per-tile (value, index) pairs an output-head GEMM left behind; lowest index
+// on ties.  Warp-wide; every lane returns the result.
+__device__ __forceinline__ int argmax_from_tiles(const float* val, const int* idx, int n_tiles) {
+    const int lane = threadIdx.x & 31;
+    float bv = -INFINITY;
+    int bi = INT_MAX;
+    for (int t0 = lane; t0 < n_tiles; t0 += 256) {   // eight loads in flight per lane
+        float v[8];
+        int ix[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int t = t0 + 32 * u;
+            v[u] = t < n_tiles ? __ldcg(val + t) : -INFINITY;
+            ix[u] = t < n_tiles ? __ldcg(idx + t) : INT_MAX;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (v[u] > bv || (v[u] == bv && ix[u] < bi)) { bv = v[u]; bi = ix[u]; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    return bi == INT_MAX ? 0 : bi;
+}
+
+// Start of a pass over decode rows: row set-up and x^(0) = Emb(t) + Pos(index) in one kernel (Eq. 1).
+// Row m = b*nq + (r - r0) carries block row r of sequence b (row 0 = pending token, row r = draft r).
+// The token of block row fin_r is not known yet as an id: it is the arg-max of the small model's last
+// output-head GEMM, finished here from its per-tile results and recorded as draft fin_r.  grid: rows; block: 128.
+template <typename T>
+__global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, int nq, int fin_r, const float* amax_val,
+                                                         const int* amax_idx, int amax_stride, int n_tiles, int* row_tok,
+                                                         int* row_seq, int* row_pos, const T* __restrict__ emb,
+                                                         const T* __restrict__ pos, float* __restrict__ h, int d) {
+    __shared__ int s_tok, s_pos;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int m = blockIdx.x;
+    const int b = m / nq, r = r0 + (m - b * nq);
+    if (threadIdx.x < 32) {
+        int tok;
+        if (r == 0) tok = st.pending[b];
+        else if (r == fin_r) tok = argmax_from_tiles(amax_val + (size_t)b * amax_stride, amax_idx + (size_t)b * amax_stride, n_tiles);
+        else tok = st.drafts[b * st.gamma_limit + r - 1];
+        if (threadIdx.x == 0) {
+            if (r == fin_r && r > 0) st.drafts[b * st.gamma_limit + r - 1] = tok;
+            const int p = st.n[b] - 1 + r;
+            s_tok = tok; s_pos = p;
+            row_tok[m] = tok; row_seq[m] = b; row_pos[m] = p;
+        }
+    }
+    __syncthreads();
+    const T* er = emb + (size_t)s_tok * d;
+    const T* pr = pos + (size_t)s_pos * d;
+    for (int i = threadIdx.x; i < d; i += 128) h[(size_t)m * d + i] = to_float(er[i]) + to_float(pr[i]);
 }
 
 __device__ __forceinline__ float block_sum_128(float v, float* red) {
@@ -107,7 +169,21 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restric
 //   a = longest prefix of drafts equal to the large model's tokens (or forced);
 //   the sequence gains d_1..d_a and g_{a+1}; n advances; g_{a+1} becomes pending.
 // Rolling the caches back is the update of n: positions >= n-1 are rewritten by the next iteration.
-__global__ void verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed, int max_new) {
+// When amax_val is given, the large model's arg-max per block row is first finished from the per-tile results of
+// its output-head GEMM.  block: 256.
+__global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed,
+                                                     int max_new, const float* amax_val, const int* amax_idx, int amax_stride,
+                                                     int n_tiles) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (amax_val != nullptr) {
+        const int rows = batch * (gamma + 1);
+        for (int m = threadIdx.x >> 5; m < rows; m += 8) {
+            const int tok = argmax_from_tiles(amax_val + (size_t)m * amax_stride, amax_idx + (size_t)m * amax_stride, n_tiles);
+            if ((threadIdx.x & 31) == 0) st.targets[(m / (gamma + 1)) * (st.gamma_limit + 1) + m % (gamma + 1)] = tok;
+        }
+        __syncthreads();
+    }
     const int b = threadIdx.x;
     const int iteration = st.counters[0];
     const int live_before = st.counters[1];

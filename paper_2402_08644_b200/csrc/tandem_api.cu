@@ -15,6 +15,7 @@
 #include "attention.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
 #include "misc_kernels.cuh"
 
 using namespace tandem;
@@ -39,14 +40,19 @@ thread_local char g_cuda_err[256] = "";
 
 size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 int cdiv(int a, int b) { return (a + b - 1) / b; }
+constexpr int TC_MAX_UNITS = 512;
+// Columns of the tensor-core decode GEMM's B operand for a number of token rows (0: too many rows for it).
+int tc_nb(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 48 ? 48 : rows <= 64 ? 64 : 0; }   // most (tile, K-slice) units of a split-K launch of the tensor-core decode GEMM
 
 struct Layout {   // byte offsets into the arena
     size_t kv_large, kv_small;
     size_t st_n, st_pending, st_drafts, st_targets, st_accept, st_emitted, st_done, st_out, st_counters, st_hist;
     size_t row_tok, row_seq, row_pos, grp_row0, grp_cnt;
+    size_t tc_counters, attn_counters;   // inside the zero-filled state block
     size_t h_large, h_small, a, q, o, f, xb, t1, yhat, a_s, logits_large, logits_small, part_ml, part_acc, dbg;
+    size_t tc_partials, amax_val_large, amax_idx_large, amax_val_small, amax_idx_small;
     size_t total;
-    int max_rows, dec_rows, max_groups, n_chunks_max;
+    int max_rows, dec_rows, max_groups, n_chunks_max, vocab_tiles;
     size_t kv_large_layer, kv_small_layer;   // elements per (layer, k-or-v)
 };
 
@@ -60,7 +66,7 @@ struct Model {
 }  // namespace
 
 enum { PC_GEMM_SMALLM = 0, PC_GEMM_TILED, PC_ATTN_SPLIT, PC_ATTN_MERGE, PC_ATTN_PROMPT, PC_LAYERNORM, PC_ROWS, PC_ARGMAX,
-       PC_VERIFY, PC_COUNT };
+       PC_VERIFY, PC_GEMM_TC_DECODE, PC_GEMM_TC_TILED, PC_COUNT };
 
 struct Prof {   // optional per-launch timing with CUDA events (measurement hook)
     bool on = false;
@@ -105,6 +111,12 @@ struct tandem_ctx {
     int chunks_launch = 1;               // attention grid size along the context for the current iteration
     int32_t* hflags = nullptr;           // mapped pinned host memory the verify kernel publishes to
     int64_t ticket = 0;                  // verify kernels enqueued since creation
+    // tensor-core path (bf16 only)
+    bool tc = false;                     // weights have tensor maps; GEMMs run on tcgen05
+    bool use_pdl = true;                 // programmatic dependent launch between the decode kernels
+    int tc_target = 148;                 // CTAs a split-K decode GEMM aims for
+    std::vector<CUtensorMap> wmap;       // one per weight pointer (matrices only), box 128 rows x 64 columns
+    std::vector<char> wmap_ok;
 };
 
 namespace {
@@ -179,6 +191,8 @@ Layout make_layout(const tandem_config& c) {
     L.st_done = take(B * 4); L.st_out = take(B * T * 4); L.st_counters = take(16 * 4); L.st_hist = take((GL + 1) * 8);
     L.row_tok = take(R * 4); L.row_seq = take(R * 4); L.row_pos = take(R * 4);
     L.grp_row0 = take((size_t)L.max_groups * 4); L.grp_cnt = take((size_t)L.max_groups * 4);
+    L.tc_counters = take(TC_MAX_UNITS * 4);
+    L.attn_counters = take(B * hmax * 4);
     L.h_large = take(R * c.large.d_model * 4);
     L.h_small = take(B * c.small.d_model * 4);
     L.a = take(R * dmax * esz); L.q = take(R * dmax * esz); L.o = take(R * dmax * esz);
@@ -190,6 +204,10 @@ Layout make_layout(const tandem_config& c) {
     L.part_ml = take(RD * hmax * L.n_chunks_max * 2 * 4);
     L.part_acc = take(RD * dmax * L.n_chunks_max * 4);
     L.dbg = take(T * dmax * 4);
+    L.vocab_tiles = cdiv(c.large.vocab, 128);
+    L.tc_partials = take((size_t)TC_MAX_UNITS * tc_nb(L.dec_rows) * 128 * 4);
+    L.amax_val_large = take(RD * L.vocab_tiles * 4); L.amax_idx_large = take(RD * L.vocab_tiles * 4);
+    L.amax_val_small = take(B * L.vocab_tiles * 4); L.amax_idx_small = take(B * L.vocab_tiles * 4);
     L.total = off;
     return L;
 }
@@ -204,9 +222,16 @@ inline const void* w_emb(const tandem_ctx& c, const Model& m) { return c.w[m.wba
 inline const void* w_pos(const tandem_ctx& c, const Model& m) { return c.w[m.wbase + 1]; }
 inline const void* w_layer(const tandem_ctx& c, const Model& m, int l, int k) { return c.w[m.wbase + 2 + 10 * l + k]; }
 inline const void* w_tail(const tandem_ctx& c, const Model& m, int k) { return c.w[m.wbase + 2 + 10 * m.d.n_layers + k]; }
-inline const void* w_tandem(const tandem_ctx& c, int j, int k) {
-    return c.w[c.tbase + (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR ? j : 2 * j + k)];
-}
+
+inline int wi_layer(const Model& m, int l, int k) { return m.wbase + 2 + 10 * l + k; }
+inline int wi_tail(const Model& m, int k) { return m.wbase + 2 + 10 * m.d.n_layers + k; }
+inline int wi_tandem(const tandem_ctx& c, int j, int k) { return c.tbase + (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR ? j : 2 * j + k); }
+
+// A linear map given by the indices of up to three weight matrices stacked along the output features.
+struct Lin { int i0, i1, i2, seg_rows, K; };
+inline Lin lin1(int i0, int rows, int K) { Lin l = {i0, -1, -1, rows, K}; return l; }
+inline Lin lin3(int i0, int i1, int i2, int rows, int K) { Lin l = {i0, i1, i2, rows, K}; return l; }
+inline int lin_n(const Lin& l) { return (1 + (l.i1 >= 0) + (l.i2 >= 0)) * l.seg_rows; }
 
 template <typename P> P* at(tandem_ctx& c, size_t off) { return reinterpret_cast<P*>(c.arena + off); }
 
@@ -236,14 +261,164 @@ void launch_smallm(tandem_ctx& c, const T* x, int ldx, int M, int K, const WSegs
     c.launches++;
 }
 
+// ---------------------------------------------------------------------------------------------------
+// tensor-core GEMMs: tensor maps and launches
+// ---------------------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (the library does not link libcuda).
+EncodeTiledFn tmap_encoder() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
+        return q == cudaDriverEntryPointSuccess ? reinterpret_cast<EncodeTiledFn>(p) : nullptr;
+    }();
+    return fn;
+}
+
+// bf16 matrix [rows][cols] with leading dimension ld (elements), tiles of 128 rows x 64 columns, 128-byte swizzle.
+// base 16-byte aligned, ld a multiple of 8.
+bool make_tmap_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+    EncodeTiledFn enc = tmap_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {ld * 2};
+    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct TcW {              // up to three weight matrices stacked along the output features
+    CUtensorMap tm[3];
+    int n_segs, seg_rows, K;
+};
+struct TcScratch { float* partials; int* counters; int* err; };
+
+TcW tcw(const tandem_ctx& c, int i0, int i1, int i2, int seg_rows, int K) {
+    TcW w;
+    w.tm[0] = c.wmap[i0];
+    w.tm[1] = c.wmap[i1 >= 0 ? i1 : i0];
+    w.tm[2] = c.wmap[i2 >= 0 ? i2 : i0];
+    w.n_segs = 1 + (i1 >= 0) + (i2 >= 0);
+    w.seg_rows = seg_rows; w.K = K;
+    return w;
+}
+
+TcScratch tc_scratch(tandem_ctx& c) {
+    TcScratch s;
+    s.partials = reinterpret_cast<float*>(c.arena + c.lay.tc_partials);
+    s.counters = reinterpret_cast<int*>(c.arena + c.lay.tc_counters);
+    s.err = c.st.counters + 2;
+    return s;
+}
+
+template <typename... KArgs, typename... Args>
+void launch_ex(tandem_ctx& c, bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (pdl && c.use_pdl) ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    c.launches++;
+}
+
+template <int NB, int PRO, int EPI>
+void launch_tc_decode_nb(tandem_ctx& c, const TcDecodeArgs& a, const TcW& w, int units) {
+    using C = TcdCfg<NB>;
+    static bool attr_set[MAX_DEVICES] = {};
+    const int dev = cur_dev();
+    if (!attr_set[dev]) {
+        cudaFuncSetAttribute(gemm_tc_decode_kernel<NB, PRO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+        attr_set[dev] = true;
+    }
+    launch_ex(c, true, gemm_tc_decode_kernel<NB, PRO, EPI>, dim3(units), dim3(TCD_THREADS), (size_t)C::SMEM_BYTES, a, w.tm[0], w.tm[1], w.tm[2]);
+}
+
+// y = prologue(x) W^T for rows <= 64 on the tensor cores, streaming W once.
+template <int PRO, int EPI>
+void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx, const void* ln_g, const void* ln_b, int rows,
+                      const TcW& w, bool stream_weights, const EpiArgs& e, float* amax_val = nullptr, int* amax_idx = nullptr,
+                      int amax_stride = 0) {
+    if (rows <= 0) return;
+    TcDecodeArgs a;
+    memset(&a, 0, sizeof(a));
+    a.x = x; a.ldx = ldx; a.ln_g = static_cast<const float*>(ln_g); a.ln_b = static_cast<const float*>(ln_b);
+    a.rows = rows; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
+    const int tiles = w.n_segs * a.tiles_per_seg, KB = cdiv(w.K, 64);
+    int S = 1;
+    if (tiles < c.tc_target) S = std::min(KB, cdiv(c.tc_target, tiles));
+    while (S > 1 && tiles * S > TC_MAX_UNITS) --S;
+    a.splits = S;
+    a.stream_weights = stream_weights ? 1 : 0;
+    a.partials = sc.partials; a.tile_counters = sc.counters; a.err_flag = sc.err;
+    a.amax_val = amax_val; a.amax_idx = amax_idx; a.amax_stride = amax_stride;
+    a.e = e;
+    const size_t xsz = PRO == PRO_BF16 ? 2 : 4;
+    ProfScope ps(c, PC_GEMM_TC_DECODE, 2.0 * a.N * w.K + (double)rows * w.K * xsz + (double)rows * a.N * (EPI == EPI_STORE_F32 || EPI == EPI_ARGMAX || EPI == EPI_RESID ? 4.0 : 2.0));
+    const int units = tiles * S;
+    if (rows <= 16) launch_tc_decode_nb<16, PRO, EPI>(c, a, w, units);
+    else if (rows <= 32) launch_tc_decode_nb<32, PRO, EPI>(c, a, w, units);
+    else if (rows <= 48) launch_tc_decode_nb<48, PRO, EPI>(c, a, w, units);
+    else launch_tc_decode_nb<64, PRO, EPI>(c, a, w, units);
+}
+
+// y = x W^T for many rows on the tensor cores; x bf16 [M][ldx].
+template <int EPI>
+tandem_status launch_tc_tiled(tandem_ctx& c, const bf16* x, int ldx, int M, const TcW& w, const EpiArgs& e, int* err) {
+    if (M <= 0) return TANDEM_OK;
+    static bool attr_set[MAX_DEVICES] = {};
+    const int dev = cur_dev();
+    if (!attr_set[dev]) {
+        cudaFuncSetAttribute(gemm_tc_tiled_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TCT_SMEM_BYTES);
+        attr_set[dev] = true;
+    }
+    CUtensorMap tmx;
+    if (!make_tmap_bf16(&tmx, x, (uint64_t)M, (uint64_t)w.K, (uint64_t)ldx)) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed for an activation buffer");
+        return TANDEM_ERR_CUDA;
+    }
+    TcTiledArgs a;
+    memset(&a, 0, sizeof(a));
+    a.M = M; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
+    a.err_flag = err; a.e = e;
+    ProfScope ps(c, PC_GEMM_TC_TILED, 2.0 * M * (double)a.N * w.K);   // flops
+    launch_ex(c, false, gemm_tc_tiled_kernel<EPI>, dim3(w.n_segs * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)TCT_SMEM_BYTES,
+              a, tmx, w.tm[0], w.tm[1], w.tm[2]);
+    return TANDEM_OK;
+}
+
+WSegs segs_of(const tandem_ctx& c, const Lin& l) {
+    WSegs s;
+    s.w[0] = c.w[l.i0];
+    s.w[1] = l.i1 >= 0 ? c.w[l.i1] : nullptr;
+    s.w[2] = l.i2 >= 0 ? c.w[l.i2] : nullptr;
+    s.seg_rows = l.seg_rows;
+    return s;
+}
+
+// y = x W^T with a fused epilogue.  decode: few rows, streaming kernel; otherwise the prompt-pass kernels
+// (tensor cores for bf16 when the context has tensor maps).
 template <typename T, int EPI>
-void launch_gemm(tandem_ctx& c, bool decode, const T* x, int ldx, int M, int K, const WSegs& ws, int N, const EpiArgs& e) {
+void launch_gemm(tandem_ctx& c, bool decode, const T* x, int ldx, int M, const Lin& l, const EpiArgs& e) {
     if (M <= 0) return;
+    const WSegs ws = segs_of(c, l);
+    const int N = lin_n(l), K = l.K;
     if (decode) {
         if (M <= 1) launch_smallm<T, 1, EPI>(c, x, ldx, M, K, ws, N, e);
         else if (M <= 2) launch_smallm<T, 2, EPI>(c, x, ldx, M, K, ws, N, e);
         else if (M <= 4) launch_smallm<T, 4, EPI>(c, x, ldx, M, K, ws, N, e);
         else launch_smallm<T, 8, EPI>(c, x, ldx, M, K, ws, N, e);
+    } else if (sizeof(T) == 2 && c.tc) {
+        launch_tc_tiled<EPI>(c, reinterpret_cast<const bf16*>(x), ldx, M, tcw(c, l.i0, l.i1, l.i2, l.seg_rows, l.K), e, c.st.counters + 2);
     } else {
         dim3 grid(cdiv(N, GT_BN), cdiv(M, GT_BM));
         ProfScope ps(c, PC_GEMM_TILED, 2.0 * M * (double)N * K);   // flops, not bytes: this one is compute-bound
@@ -252,9 +427,6 @@ void launch_gemm(tandem_ctx& c, bool decode, const T* x, int ldx, int M, int K, 
     }
 }
 
-WSegs segs1(const void* w, int n) { WSegs s; s.w[0] = w; s.w[1] = s.w[2] = nullptr; s.seg_rows = n; return s; }
-WSegs segs3(const void* a, const void* b, const void* c3, int n) { WSegs s; s.w[0] = a; s.w[1] = b; s.w[2] = c3; s.seg_rows = n; return s; }
-
 template <typename T, int DH>
 void set_attn_attrs() {
     cudaFuncSetAttribute(attn_kernel<T, DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<T, DH>());
@@ -262,31 +434,24 @@ void set_attn_attrs() {
 }
 
 template <typename T, int DH>
-void launch_attn_dh(tandem_ctx& c, const AttnArgs& a, int M, int groups, bool loop, int n_chunks, double kv_bytes) {
+void launch_attn_dh(tandem_ctx& c, const AttnArgs& a, int groups, bool loop, int n_chunks, double kv_bytes) {
     static bool attr_set[MAX_DEVICES] = {};
     const int dev = cur_dev();
-    cudaStream_t s = c.stream;
     if (!attr_set[dev]) { set_attn_attrs<T, DH>(); attr_set[dev] = true; }
     if (loop) {
         ProfScope ps(c, PC_ATTN_PROMPT, kv_bytes);
-        attn_kernel<T, DH, true><<<dim3(1, a.n_heads, groups), ATT_THREADS, attn_smem_bytes<T, DH>(), s>>>(a);
-        c.launches += 1;
+        launch_ex(c, false, attn_kernel<T, DH, true>, dim3(1, a.n_heads, groups), dim3(ATT_THREADS), attn_smem_bytes<T, DH>(), a);
     } else {
-        {
-            ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
-            attn_kernel<T, DH, false><<<dim3(n_chunks, a.n_heads, groups), ATT_THREADS, attn_smem_bytes<T, DH>(), s>>>(a);
-        }
-        ProfScope ps(c, PC_ATTN_MERGE, (double)M * a.n_heads * n_chunks * (DH + 2) * 4.0);
-        attn_merge_kernel<T, DH><<<dim3(M, a.n_heads), DH, 0, s>>>(a);
-        c.launches += 2;
+        ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
+        launch_ex(c, true, attn_kernel<T, DH, false>, dim3(n_chunks, a.n_heads, groups), dim3(ATT_THREADS), attn_smem_bytes<T, DH>(), a);
     }
 }
 
 template <typename T>
-void launch_attn(tandem_ctx& c, int d_head, const AttnArgs& a, int M, int groups, bool loop, int n_chunks, double kv_bytes) {
-    if (d_head == 32) launch_attn_dh<T, 32>(c, a, M, groups, loop, n_chunks, kv_bytes);
-    else if (d_head == 64) launch_attn_dh<T, 64>(c, a, M, groups, loop, n_chunks, kv_bytes);
-    else launch_attn_dh<T, 128>(c, a, M, groups, loop, n_chunks, kv_bytes);
+void launch_attn(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, bool loop, int n_chunks, double kv_bytes) {
+    if (d_head == 32) launch_attn_dh<T, 32>(c, a, groups, loop, n_chunks, kv_bytes);
+    else if (d_head == 64) launch_attn_dh<T, 64>(c, a, groups, loop, n_chunks, kv_bytes);
+    else launch_attn_dh<T, 128>(c, a, groups, loop, n_chunks, kv_bytes);
 }
 
 template <typename T>
@@ -325,6 +490,20 @@ EpiArgs epi_cache(tandem_ctx& c, const Model& m, int layer, void* q_out) {
     return e;
 }
 
+template <typename T>
+void attention(tandem_ctx& c, const Model& m, int l, const T* q, T* o, const Rows& r) {
+    const int d = m.d.d_model, H = m.d.n_heads, dh = d / H;
+    AttnArgs aa; memset(&aa, 0, sizeof(aa));
+    aa.q = q; aa.ldq = d; aa.kcache = kv_ptr<T>(c, m, l, 0); aa.vcache = kv_ptr<T>(c, m, l, 1);
+    aa.out = o; aa.ldo = d; aa.row_seq = at<int>(c, c.lay.row_seq); aa.row_pos = at<int>(c, c.lay.row_pos);
+    if (!r.decode) { aa.grp_row0 = at<int>(c, c.lay.grp_row0); aa.grp_cnt = at<int>(c, c.lay.grp_cnt); }
+    aa.nq = r.nq; aa.n_heads = H; aa.t_max = c.cfg.max_seq;
+    aa.part_ml = at<float>(c, c.lay.part_ml); aa.part_acc = at<float>(c, c.lay.part_acc);
+    aa.n_chunks_max = c.lay.n_chunks_max; aa.scale = 1.0f / sqrtf((float)dh);
+    aa.merge_counters = at<int>(c, c.lay.attn_counters);
+    launch_attn<T>(c, dh, aa, r.groups, !r.decode, r.n_chunks, r.kv_positions * 2.0 * d * sizeof(T));
+}
+
 // Eq. 2, first line, for small layer j, then that layer's LayerNorm and key/value maps: writes the
 // small model's large-derived keys/values for the rows' positions.
 template <typename T>
@@ -334,15 +513,14 @@ void project_layer(tandem_ctx& c, int j, const Rows& r) {
     float* yhat = at<float>(c, c.lay.yhat);
     T* a_s = at<T>(c, c.lay.a_s);
     if (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR) {
-        launch_gemm<T, EPI_STORE_F32>(c, r.decode, xb, dL, r.M, dL, segs1(w_tandem(c, j, 0), dS), dS, epi_plain(yhat, dS));
+        launch_gemm<T, EPI_STORE_F32>(c, r.decode, xb, dL, r.M, lin1(wi_tandem(c, j, 0), dS, dL), epi_plain(yhat, dS));
     } else {
         T* t1 = at<T>(c, c.lay.t1);
-        launch_gemm<T, EPI_GELU>(c, r.decode, xb, dL, r.M, dL, segs1(w_tandem(c, j, 0), c.hidden), c.hidden, epi_plain(t1, c.hidden));
-        launch_gemm<T, EPI_STORE_F32>(c, r.decode, t1, c.hidden, r.M, c.hidden, segs1(w_tandem(c, j, 1), dS), dS, epi_plain(yhat, dS));
+        launch_gemm<T, EPI_GELU>(c, r.decode, xb, dL, r.M, lin1(wi_tandem(c, j, 0), c.hidden, dL), epi_plain(t1, c.hidden));
+        launch_gemm<T, EPI_STORE_F32>(c, r.decode, t1, c.hidden, r.M, lin1(wi_tandem(c, j, 1), dS, c.hidden), epi_plain(yhat, dS));
     }
     launch_layernorm<T>(c, r.M, yhat, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), a_s, dS);
-    launch_gemm<T, EPI_KV>(c, r.decode, a_s, dS, r.M, dS,
-                           segs3(w_layer(c, c.small, j, W_WK), w_layer(c, c.small, j, W_WV), nullptr, dS), 2 * dS,
+    launch_gemm<T, EPI_KV>(c, r.decode, a_s, dS, r.M, lin3(wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS),
                            epi_cache<T>(c, c.small, j, nullptr));
 }
 
@@ -364,26 +542,19 @@ void project_after(tandem_ctx& c, int n_large_layers_done, const Rows& r) {
 // One decoder layer (Eq. 1; the same form serves the small model's layers in Eq. 2) on residual stream h.
 template <typename T>
 void decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r) {
-    const int d = m.d.d_model, dff = m.d.d_ff, H = m.d.n_heads, dh = d / H;
+    const int d = m.d.d_model, dff = m.d.d_ff;
     T* a = at<T>(c, c.lay.a);
     T* q = at<T>(c, c.lay.q);
     T* o = at<T>(c, c.lay.o);
     T* f = at<T>(c, c.lay.f);
     launch_layernorm<T>(c, r.M, h, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), a, d);
-    launch_gemm<T, EPI_QKV>(c, r.decode, a, d, r.M, d, segs3(w_layer(c, m, l, W_WQ), w_layer(c, m, l, W_WK), w_layer(c, m, l, W_WV), d),
-                            3 * d, epi_cache<T>(c, m, l, q));
-    AttnArgs aa; memset(&aa, 0, sizeof(aa));
-    aa.q = q; aa.ldq = d; aa.kcache = kv_ptr<T>(c, m, l, 0); aa.vcache = kv_ptr<T>(c, m, l, 1);
-    aa.out = o; aa.ldo = d; aa.row_seq = at<int>(c, c.lay.row_seq); aa.row_pos = at<int>(c, c.lay.row_pos);
-    if (!r.decode) { aa.grp_row0 = at<int>(c, c.lay.grp_row0); aa.grp_cnt = at<int>(c, c.lay.grp_cnt); }
-    aa.nq = r.nq; aa.n_heads = H; aa.t_max = c.cfg.max_seq;
-    aa.part_ml = at<float>(c, c.lay.part_ml); aa.part_acc = at<float>(c, c.lay.part_acc);
-    aa.n_chunks_max = c.lay.n_chunks_max; aa.scale = 1.0f / sqrtf((float)dh);
-    launch_attn<T>(c, dh, aa, r.M, r.groups, !r.decode, r.n_chunks, r.kv_positions * 2.0 * d * sizeof(T));
-    launch_gemm<T, EPI_RESID>(c, r.decode, o, d, r.M, d, segs1(w_layer(c, m, l, W_WO), d), d, epi_plain(h, d));
+    launch_gemm<T, EPI_QKV>(c, r.decode, a, d, r.M, lin3(wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, d),
+                            epi_cache<T>(c, m, l, q));
+    attention<T>(c, m, l, q, o, r);
+    launch_gemm<T, EPI_RESID>(c, r.decode, o, d, r.M, lin1(wi_layer(m, l, W_WO), d, d), epi_plain(h, d));
     launch_layernorm<T>(c, r.M, h, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), a, d);
-    launch_gemm<T, EPI_GELU>(c, r.decode, a, d, r.M, d, segs1(w_layer(c, m, l, W_W1), dff), dff, epi_plain(f, dff));
-    launch_gemm<T, EPI_RESID>(c, r.decode, f, dff, r.M, dff, segs1(w_layer(c, m, l, W_W2), d), d, epi_plain(h, d));
+    launch_gemm<T, EPI_GELU>(c, r.decode, a, d, r.M, lin1(wi_layer(m, l, W_W1), dff, d), epi_plain(f, dff));
+    launch_gemm<T, EPI_RESID>(c, r.decode, f, dff, r.M, lin1(wi_layer(m, l, W_W2), d, dff), epi_plain(h, d));
 }
 
 // Final LayerNorm, output head, arg-max.  dst[(m / nq) * seq_stride + m % nq + off].
@@ -392,7 +563,7 @@ void head_argmax(tandem_ctx& c, const Model& m, float* h, const Rows& r, float* 
     const int d = m.d.d_model, V = m.d.vocab;
     T* a = at<T>(c, c.lay.a);
     launch_layernorm<T>(c, r.M, h, w_tail(c, m, 0), w_tail(c, m, 1), a, d);
-    launch_gemm<T, EPI_STORE_F32>(c, r.decode, a, d, r.M, d, segs1(w_tail(c, m, 2), V), V, epi_plain(logits, V));
+    launch_gemm<T, EPI_STORE_F32>(c, r.decode, a, d, r.M, lin1(wi_tail(m, 2), V, d), epi_plain(logits, V));
     ProfScope ps(c, PC_ARGMAX, (double)r.M * V * 4.0);
     argmax_rows_kernel<<<r.M, 256, 0, c.stream>>>(logits, V, dst, r.nq, seq_stride, off);
     c.launches++;
@@ -420,7 +591,6 @@ void large_pass(tandem_ctx& c, const Rows& r, bool project, bool head) {
 Rows decode_rows(tandem_ctx& c, int r_last, int nq) {
     Rows r;
     r.M = c.batch * nq; r.groups = c.batch; r.nq = nq; r.decode = true;
-    (void)r_last;
     r.n_chunks = c.chunks_launch;
     r.kv_positions = (double)c.n_sum + (double)c.batch * r_last;
     return r;
@@ -450,16 +620,19 @@ void small_step(tandem_ctx& c, int s) {
     head_argmax<T>(c, c.small, y, r, logits, c.st.drafts, TANDEM_GAMMA_LIMIT, s);
 }
 
+void launch_verify(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new, bool from_tiles) {
+    ProfScope ps(c, PC_VERIFY, (double)c.batch * (2 * gamma + 8) * 4.0);
+    launch_ex(c, true, verify_kernel, dim3(1), dim3(256), 0, c.st, c.batch, gamma, mode, (unsigned long long)seed, max_new,
+              from_tiles ? (const float*)at<float>(c, c.lay.amax_val_large) : (const float*)nullptr,
+              from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_large) : (const int*)nullptr, c.lay.vocab_tiles, c.lay.vocab_tiles);
+}
+
 template <typename T>
 void iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
     for (int s = 0; s < gamma; ++s) small_step<T>(c, s);
     setup_rows(c, 0, gamma + 1);
     large_pass<T>(c, decode_rows(c, gamma, gamma + 1), true, true);
-    {
-        ProfScope ps(c, PC_VERIFY, (double)c.batch * (2 * gamma + 8) * 4.0);
-        verify_kernel<<<1, 256, 0, c.stream>>>(c.st, c.batch, gamma, mode, seed, max_new);
-        c.launches++;
-    }
+    launch_verify(c, gamma, mode, seed, max_new, false);
     c.last_gamma = gamma;
 }
 
@@ -467,11 +640,106 @@ template <typename T>
 void greedy_iteration(tandem_ctx& c, int max_new) {
     setup_rows(c, 0, 1);
     large_pass<T>(c, decode_rows(c, 0, 1), false, true);
-    {
-        ProfScope ps(c, PC_VERIFY, (double)c.batch * 8 * 4.0);
-        verify_kernel<<<1, 256, 0, c.stream>>>(c.st, c.batch, 0, 0, 0ull, max_new);
-        c.launches++;
+    launch_verify(c, 0, 0, 0ull, max_new, false);
+    c.last_gamma = 0;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// bf16 decode on the tensor cores: five kernels per decoder layer, chained by programmatic dependent launch
+// ---------------------------------------------------------------------------------------------------
+
+// Row set-up + embedding for block rows r0 .. r0+nq-1 of every sequence; fin_r: block row whose token is the
+// arg-max the small model's last head GEMM left as per-tile results (-1: none).
+void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r) {
+    ProfScope ps(c, PC_ROWS, (double)c.batch * nq * m.d.d_model * 8.0);
+    launch_ex(c, true, step_begin_kernel<bf16>, dim3(c.batch * nq), dim3(128), 0, c.st, r0, nq, fin_r,
+              (const float*)at<float>(c, c.lay.amax_val_small), (const int*)at<int>(c, c.lay.amax_idx_small), c.lay.vocab_tiles,
+              c.lay.vocab_tiles, at<int>(c, c.lay.row_tok), at<int>(c, c.lay.row_seq), at<int>(c, c.lay.row_pos),
+              (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model);
+}
+
+void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r, bool stream_w) {
+    const int d = m.d.d_model, dff = m.d.d_ff;
+    bf16* q = at<bf16>(c, c.lay.q);
+    bf16* o = at<bf16>(c, c.lay.o);
+    bf16* f = at<bf16>(c, c.lay.f);
+    const TcScratch sc = tc_scratch(c);
+    launch_tc_decode<PRO_LN, EPI_QKV>(c, sc, h, d, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), r.M,
+                                      tcw(c, wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, d), stream_w,
+                                      epi_cache<bf16>(c, m, l, q));
+    attention<bf16>(c, m, l, q, o, r);
+    launch_tc_decode<PRO_BF16, EPI_RESID>(c, sc, o, d, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_WO), -1, -1, d, d), stream_w,
+                                          epi_plain(h, d));
+    launch_tc_decode<PRO_LN, EPI_GELU>(c, sc, h, d, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), r.M,
+                                       tcw(c, wi_layer(m, l, W_W1), -1, -1, dff, d), stream_w, epi_plain(f, dff));
+    launch_tc_decode<PRO_BF16, EPI_RESID>(c, sc, f, dff, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_W2), -1, -1, d, dff), stream_w,
+                                          epi_plain(h, d));
+}
+
+// Final LayerNorm + output head; leaves fp32 logits and the per-tile (max, index) pairs that the next kernel
+// (the next pass's row set-up, or the verify kernel) turns into token ids.
+void tc_head(tandem_ctx& c, const Model& m, float* h, const Rows& r, float* logits, size_t amax_val_off, size_t amax_idx_off, bool stream_w) {
+    launch_tc_decode<PRO_LN, EPI_ARGMAX>(c, tc_scratch(c), h, m.d.d_model, w_tail(c, m, 0), w_tail(c, m, 1), r.M,
+                                         tcw(c, wi_tail(m, 2), -1, -1, m.d.vocab, m.d.d_model), stream_w, epi_plain(logits, m.d.vocab),
+                                         at<float>(c, amax_val_off), at<int>(c, amax_idx_off), c.lay.vocab_tiles);
+}
+
+// FF_Tandem of the block's rows after n large layers (Eq. 2, first line) for every small layer fed from there,
+// then that layer's LayerNorm and key/value maps with the cache write as the GEMM epilogue.
+void tc_project_after(tandem_ctx& c, int n_large_layers_done, const Rows& r) {
+    const int dL = c.large.d.d_model, dS = c.small.d.d_model;
+    const TcScratch sc = tc_scratch(c);
+    float* h = at<float>(c, c.lay.h_large);
+    float* yhat = at<float>(c, c.lay.yhat);
+    for (int j = 0; j < c.small.d.n_layers; ++j) {
+        if (c.layer_map[j] != n_large_layers_done) continue;
+        if (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR) {
+            launch_tc_decode<PRO_CAST, EPI_STORE_F32>(c, sc, h, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, dS, dL), true,
+                                                      epi_plain(yhat, dS));
+        } else {
+            bf16* t1 = at<bf16>(c, c.lay.t1);
+            launch_tc_decode<PRO_CAST, EPI_GELU>(c, sc, h, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, c.hidden, dL), true,
+                                                 epi_plain(t1, c.hidden));
+            launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, t1, c.hidden, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 1), -1, -1, dS, c.hidden),
+                                                      true, epi_plain(yhat, dS));
+        }
+        launch_tc_decode<PRO_LN, EPI_KV>(c, sc, yhat, dS, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), r.M,
+                                         tcw(c, wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS), true,
+                                         epi_cache<bf16>(c, c.small, j, nullptr));
     }
+}
+
+void tc_small_step(tandem_ctx& c, int s) {
+    float* y = at<float>(c, c.lay.h_small);
+    tc_begin(c, c.small, y, s, 1, s > 0 ? s : -1);
+    const Rows r = decode_rows(c, s, 1);
+    for (int j = 0; j < c.small.d.n_layers; ++j) tc_decoder_layer(c, c.small, j, y, r, false);
+    float* logits = at<float>(c, c.lay.logits_small) + (size_t)s * c.batch * c.small.d.vocab;
+    tc_head(c, c.small, y, r, logits, c.lay.amax_val_small, c.lay.amax_idx_small, false);
+}
+
+void tc_large_block(tandem_ctx& c, int gamma, bool project) {
+    float* h = at<float>(c, c.lay.h_large);
+    tc_begin(c, c.large, h, 0, gamma + 1, gamma > 0 ? gamma : -1);
+    const Rows r = decode_rows(c, gamma, gamma + 1);
+    if (project) tc_project_after(c, 0, r);
+    for (int l = 0; l < c.large.d.n_layers; ++l) {
+        tc_decoder_layer(c, c.large, l, h, r, true);
+        if (project) tc_project_after(c, l + 1, r);
+    }
+    tc_head(c, c.large, h, r, at<float>(c, c.lay.logits_large), c.lay.amax_val_large, c.lay.amax_idx_large, true);
+}
+
+void tc_iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
+    for (int s = 0; s < gamma; ++s) tc_small_step(c, s);
+    tc_large_block(c, gamma, true);
+    launch_verify(c, gamma, mode, seed, max_new, true);
+    c.last_gamma = gamma;
+}
+
+void tc_greedy_iteration(tandem_ctx& c, int max_new) {
+    tc_large_block(c, 0, false);
+    launch_verify(c, 0, 0, 0ull, max_new, true);
     c.last_gamma = 0;
 }
 
@@ -482,6 +750,10 @@ tandem_status check_launch() {
 
 void enqueue_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t seed, int max_new) {
     const bool bf = c.cfg.dtype == TANDEM_DTYPE_BF16;
+    if (bf && c.tc && tc_nb(c.batch * (gamma + 1)) != 0) {
+        if (kind == 0) tc_iteration(c, gamma, mode, seed, max_new); else tc_greedy_iteration(c, max_new);
+        return;
+    }
     if (kind == 0) { if (bf) iteration<bf16>(c, gamma, mode, seed, max_new); else iteration<float>(c, gamma, mode, seed, max_new); }
     else { if (bf) greedy_iteration<bf16>(c, max_new); else greedy_iteration<float>(c, max_new); }
 }
@@ -641,6 +913,39 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
     }
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
     c->use_graphs = getenv("TANDEM_NO_GRAPH") == nullptr;
+    c->use_pdl = getenv("TANDEM_NO_PDL") == nullptr;
+    if (const char* t = getenv("TANDEM_TC_TARGET")) c->tc_target = std::max(1, std::min(TC_MAX_UNITS, atoi(t)));
+    if (e == cudaSuccess && cfg->dtype == TANDEM_DTYPE_BF16 && getenv("TANDEM_NO_TC") == nullptr) {
+        // one tensor map per weight matrix: [out_features][in_features], 128 x 64 tiles
+        c->wmap.resize(c->w.size());
+        c->wmap_ok.assign(c->w.size(), 0);
+        bool ok = tmap_encoder() != nullptr;
+        auto add = [&](int idx, int rows, int cols) {
+            if (ok && make_tmap_bf16(&c->wmap[idx], c->w[idx], (uint64_t)rows, (uint64_t)cols, (uint64_t)cols)) c->wmap_ok[idx] = 1;
+            else ok = false;
+        };
+        for (const Model* m : {&c->large, &c->small}) {
+            const int d = m->d.d_model, dff = m->d.d_ff;
+            for (int l = 0; l < m->d.n_layers; ++l) {
+                add(wi_layer(*m, l, W_WQ), d, d); add(wi_layer(*m, l, W_WK), d, d); add(wi_layer(*m, l, W_WV), d, d);
+                add(wi_layer(*m, l, W_WO), d, d); add(wi_layer(*m, l, W_W1), dff, d); add(wi_layer(*m, l, W_W2), d, dff);
+            }
+            add(wi_tail(*m, 2), m->d.vocab, d);
+        }
+        for (int j = 0; j < cfg->small.n_layers; ++j) {
+            if (cfg->ff_tandem_kind == TANDEM_FF_LINEAR) add(wi_tandem(*c, j, 0), cfg->small.d_model, cfg->large.d_model);
+            else { add(wi_tandem(*c, j, 0), c->hidden, cfg->large.d_model); add(wi_tandem(*c, j, 1), cfg->small.d_model, c->hidden); }
+        }
+        if (!ok) {
+            snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled unavailable or failed for a weight matrix");
+            if (c->pinned) cudaFreeHost(c->pinned);
+            if (c->hflags) cudaFreeHost(c->hflags);
+            if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+            delete c;
+            return TANDEM_ERR_CUDA;
+        }
+        c->tc = true;
+    }
     if (e == cudaSuccess) e = cudaMemsetAsync(c->arena + lay.st_n, 0, lay.h_large - lay.st_n, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) {
@@ -864,7 +1169,7 @@ extern "C" int64_t tandem_launch_count(tandem_ctx* c) { return c ? c->launches :
 
 extern "C" const char* tandem_profile_class_name(int32_t cls) {
     static const char* names[PC_COUNT] = {"gemm_smallm", "gemm_tiled", "attn_split", "attn_merge", "attn_prompt",
-                                          "layernorm", "rows", "argmax", "verify"};
+                                          "layernorm", "rows", "argmax", "verify", "gemm_tc_decode", "gemm_tc_tiled"};
     return (cls >= 0 && cls < PC_COUNT) ? names[cls] : nullptr;
 }
 
@@ -956,7 +1261,7 @@ extern "C" tandem_status tandem_debug_read(tandem_ctx* c, int32_t what, int32_t 
 // ---------------------------------------------------------------------------------------------------
 
 namespace {
-struct AttnScratch { size_t ml, acc, rows, total; int n_chunks; };
+struct AttnScratch { size_t ml, acc, rows, counters, total; int n_chunks; };
 AttnScratch attn_scratch_layout(int batch, int H, int dh, int derived_len, int own_len) {
     AttnScratch s;
     s.n_chunks = cdiv(derived_len + own_len, ATT_CH);
@@ -964,6 +1269,7 @@ AttnScratch attn_scratch_layout(int batch, int H, int dh, int derived_len, int o
     s.ml = off; off = align_up(off + (size_t)batch * H * s.n_chunks * 2 * 4);
     s.acc = off; off = align_up(off + (size_t)batch * H * s.n_chunks * dh * 4);
     s.rows = off; off = align_up(off + (size_t)batch * 2 * 4);
+    s.counters = off; off = align_up(off + (size_t)batch * H * 4);
     s.total = off;
     return s;
 }
@@ -995,6 +1301,7 @@ extern "C" tandem_status tandem_decode_attention(const void* q, const void* k_de
     unsigned char* sc = static_cast<unsigned char*>(scratch);
     int* row_seq = reinterpret_cast<int*>(sc + sl.rows);
     int* row_pos = row_seq + batch;
+    CK(cudaMemsetAsync(sc + sl.counters, 0, (size_t)batch * n_heads * 4, s));   // the chunk-merge tickets start at zero
     iota_rows_kernel<<<cdiv(batch, 256), 256, 0, s>>>(row_seq, row_pos, batch, derived_len + own_len - 1);
     AttnArgs a; memset(&a, 0, sizeof(a));
     a.q = q; a.ldq = n_heads * d_head; a.kcache = k_derived; a.vcache = v_derived; a.k2 = k_own; a.v2 = v_own;
@@ -1002,9 +1309,11 @@ extern "C" tandem_status tandem_decode_attention(const void* q, const void* k_de
     a.out = out; a.ldo = n_heads * d_head; a.row_seq = row_seq; a.row_pos = row_pos; a.nq = 1; a.n_heads = n_heads;
     a.part_ml = reinterpret_cast<float*>(sc + sl.ml); a.part_acc = reinterpret_cast<float*>(sc + sl.acc);
     a.n_chunks_max = sl.n_chunks; a.scale = 1.0f / sqrtf((float)d_head);
+    a.merge_counters = reinterpret_cast<int*>(sc + sl.counters);
     tandem_ctx tmp;   // only the stream and the launch counter are used by the launch helpers
     tmp.stream = s;
-    launch_attn<bf16>(tmp, d_head, a, batch, batch, false, sl.n_chunks, 0.0);
+    tmp.use_pdl = false;
+    launch_attn<bf16>(tmp, d_head, a, batch, false, sl.n_chunks, 0.0);
     return check_launch();
 }
 
@@ -1056,28 +1365,67 @@ extern "C" tandem_status tandem_decode_attention_static(const void* q, const voi
                                    n_heads, d_head, derived_len, own_len, stream);
 }
 
+namespace {
+struct ProjScratch { size_t yhat, a_s, rows, partials, counters, total; };
+ProjScratch proj_scratch_layout(int rows, int d_small) {
+    ProjScratch p;
+    size_t off = 0;
+    p.yhat = off; off = align_up(off + (size_t)rows * d_small * 4);
+    p.a_s = off; off = align_up(off + (size_t)rows * d_small * 2);
+    p.rows = off; off = align_up(off + (size_t)rows * 8);
+    p.counters = off; off = align_up(off + (size_t)TC_MAX_UNITS * 4);
+    p.partials = off; off = align_up(off + (size_t)TC_MAX_UNITS * std::max(16, tc_nb(rows)) * 128 * 4);
+    p.total = off;
+    return p;
+}
+}  // namespace
+
+extern "C" size_t tandem_ff_tandem_project_scratch_bytes(int32_t rows, int32_t d_small) {
+    if (rows < 1 || rows > 256 || d_small < 8) return 0;
+    return proj_scratch_layout(rows, d_small).total;
+}
+
 extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t, const void* ln_g, const void* ln_b, const void* wk,
                                                   const void* wv, void* k_out, void* v_out, void* scratch, size_t scratch_bytes,
                                                   int32_t rows, int32_t d_large, int32_t d_small, void* stream) {
     if (!x || !w_t || !ln_g || !ln_b || !wk || !wv || !k_out || !v_out || !scratch) return TANDEM_ERR_INVALID_ARG;
     if (rows < 1 || rows > 256 || d_large < 8 || d_small < 8) return TANDEM_ERR_INVALID_ARG;
     if (d_large % 8 || d_small % 8) return TANDEM_ERR_SHAPE;
-    const size_t need = align_up((size_t)rows * d_small * 4) + align_up((size_t)rows * d_small * 2) + align_up((size_t)rows * 8);
-    if (scratch_bytes < need) return TANDEM_ERR_ARENA_TOO_SMALL;
-    if (((uintptr_t)x | (uintptr_t)w_t | (uintptr_t)wk | (uintptr_t)wv | (uintptr_t)k_out | (uintptr_t)v_out | (uintptr_t)scratch) & 15)
+    const ProjScratch pl = proj_scratch_layout(rows, d_small);
+    if (scratch_bytes < pl.total) return TANDEM_ERR_ARENA_TOO_SMALL;
+    if (((uintptr_t)x | (uintptr_t)w_t | (uintptr_t)wk | (uintptr_t)wv | (uintptr_t)k_out | (uintptr_t)v_out | (uintptr_t)scratch |
+         (uintptr_t)ln_g | (uintptr_t)ln_b) & 15)
         return TANDEM_ERR_INVALID_ARG;
-    tandem_ctx tmp;   // only the stream and the launch counter are used by the launch helpers
+    tandem_ctx tmp;   // only the stream, the launch counter and the launch options are used by the launch helpers
     tmp.stream = static_cast<cudaStream_t>(stream);
+    tmp.use_pdl = false;
     unsigned char* sc = static_cast<unsigned char*>(scratch);
-    float* yhat = reinterpret_cast<float*>(sc);
-    bf16* a_s = reinterpret_cast<bf16*>(sc + align_up((size_t)rows * d_small * 4));
-    int* row_seq = reinterpret_cast<int*>(sc + align_up((size_t)rows * d_small * 4) + align_up((size_t)rows * d_small * 2));
+    float* yhat = reinterpret_cast<float*>(sc + pl.yhat);
+    bf16* a_s = reinterpret_cast<bf16*>(sc + pl.a_s);
+    int* row_seq = reinterpret_cast<int*>(sc + pl.rows);
     int* row_pos = row_seq + rows;
+    TcW wt, wkv;
+    if (!make_tmap_bf16(&wt.tm[0], w_t, (uint64_t)d_small, (uint64_t)d_large, (uint64_t)d_large) ||
+        !make_tmap_bf16(&wkv.tm[0], wk, (uint64_t)d_small, (uint64_t)d_small, (uint64_t)d_small) ||
+        !make_tmap_bf16(&wkv.tm[1], wv, (uint64_t)d_small, (uint64_t)d_small, (uint64_t)d_small)) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled unavailable or failed");
+        return TANDEM_ERR_CUDA;
+    }
+    wt.tm[1] = wt.tm[2] = wt.tm[0]; wt.n_segs = 1; wt.seg_rows = d_small; wt.K = d_large;
+    wkv.tm[2] = wkv.tm[0]; wkv.n_segs = 2; wkv.seg_rows = d_small; wkv.K = d_small;
     iota_rows_kernel<<<cdiv(rows, 256), 256, 0, tmp.stream>>>(row_seq, row_pos, rows, 0);
-    launch_gemm<bf16, EPI_STORE_F32>(tmp, true, static_cast<const bf16*>(x), d_large, rows, d_large, segs1(w_t, d_small), d_small, epi_plain(yhat, d_small));
-    launch_layernorm<bf16>(tmp, rows, yhat, ln_g, ln_b, a_s, d_small);
     EpiArgs e; memset(&e, 0, sizeof(e));
     e.kcache = k_out; e.vcache = v_out; e.row_seq = row_seq; e.row_pos = row_pos; e.n_heads = 1; e.d_head = d_small; e.t_max = 1; e.seg = d_small;
-    launch_gemm<bf16, EPI_KV>(tmp, true, a_s, d_small, rows, d_small, segs3(wk, wv, nullptr, d_small), 2 * d_small, e);
+    if (tc_nb(rows) != 0) {
+        // few rows: weights streamed once per GEMM; LayerNorm fused into the second GEMM's operand load
+        CK(cudaMemsetAsync(sc + pl.counters, 0, (size_t)TC_MAX_UNITS * 4, tmp.stream));
+        TcScratch ts; ts.partials = reinterpret_cast<float*>(sc + pl.partials); ts.counters = reinterpret_cast<int*>(sc + pl.counters); ts.err = nullptr;
+        launch_tc_decode<PRO_BF16, EPI_STORE_F32>(tmp, ts, x, d_large, nullptr, nullptr, rows, wt, true, epi_plain(yhat, d_small));
+        launch_tc_decode<PRO_LN, EPI_KV>(tmp, ts, yhat, d_small, ln_g, ln_b, rows, wkv, true, e);
+    } else {
+        TRY(launch_tc_tiled<EPI_STORE_F32>(tmp, static_cast<const bf16*>(x), d_large, rows, wt, epi_plain(yhat, d_small), nullptr));
+        launch_layernorm<bf16>(tmp, rows, yhat, ln_g, ln_b, a_s, d_small);
+        TRY(launch_tc_tiled<EPI_KV>(tmp, a_s, d_small, rows, wkv, e, nullptr));
+    }
     return check_launch();
 }
