@@ -241,8 +241,8 @@ TANDEM_API tandem_status tandem_decode_attention_static(const void* q, const voi
  * LayerNorm and key/value maps, written as bf16 keys/values.  All pointers DEVICE, 16-byte aligned.
  *   x [rows][d_large] bf16;  w_t [d_small][d_large] bf16;  ln_g, ln_b [d_small] fp32;
  *   wk, wv [d_small][d_small] bf16;  k_out, v_out [rows][d_small] bf16;
- *   scratch: at least tandem_ff_tandem_project_scratch_bytes(rows, d_small) bytes (the fp32 projection,
- *   split-K partial sums and their tickets).  rows <= 256; d_large, d_small multiples of 8.
+ *   scratch: at least tandem_ff_tandem_project_scratch_bytes(rows, d_small) bytes (the fp32 projection
+ *   and, above 64 rows, its normalised bf16 copy).  rows <= 256; d_large, d_small multiples of 8.
  * Up to 64 rows the two GEMMs stream their weights once on the tensor cores with the LayerNorm fused into
  * the second one's operand load and the key/value write as its epilogue; above that they are tiled GEMMs
  * with a LayerNorm kernel in between. */

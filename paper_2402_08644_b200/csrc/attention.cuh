@@ -57,8 +57,10 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
     constexpr int QPT = (ATT_NQ + QS - 1) / QS; // queries per thread in the value phase
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_last;
+    TC_PROBE_INIT(LOOP ? 201 : 200);
     pdl_launch_dependents();   // the next kernel may start fetching its weights
     pdl_wait();                // queries and keys/values come from earlier kernels
+    if (threadIdx.x == 0) TC_PROBE(1);
     T* ks = reinterpret_cast<T*>(smem_raw);
     T* vs = ks + ATT_CH * LD;
     float* qs = reinterpret_cast<float*>(vs + ATT_CH * LD);
@@ -114,6 +116,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
         cp_async_commit();
         cp_async_wait_all();
         __syncthreads();
+        if (threadIdx.x == 0) TC_PROBE(2);
 
         // scores: thread t owns key t0+t for every query
         for (int t = tid; t < nt; t += ATT_THREADS) {
@@ -138,6 +141,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
         }
         __syncthreads();
 
+        if (threadIdx.x == 0) TC_PROBE(3);
         // per query: chunk max, exponentials, chunk sum
         for (int qi = warp; qi < cnt; qi += ATT_THREADS / 32) {
             float m = -INFINITY;
@@ -156,6 +160,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
         }
         __syncthreads();
 
+        if (threadIdx.x == 0) TC_PROBE(4);
         // weighted values: thread owns element e for queries qsub, qsub+QS, ...
 #pragma unroll
         for (int i = 0; i < QPT; ++i) {
@@ -186,8 +191,10 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
         }
     } else {
         // The CTA that finishes last for this (group, head) merges every query's chunks in position order.
+        if (threadIdx.x == 0) TC_PROBE(5);
         __threadfence();
         __syncthreads();
+        if (threadIdx.x == 0) TC_PROBE(6);
         if (tid == 0) {
             const int active = min((int)gridDim.x, pos_last / ATT_CH + 1);   // CTAs that got this far
             int* counter = a.merge_counters + (size_t)g * a.n_heads + h;
@@ -196,6 +203,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
             if (t == active - 1) *counter = 0;   // ready for the next launch
         }
         __syncthreads();
+        if (threadIdx.x == 0) TC_PROBE(7);
         if (!s_last) return;
         __threadfence();
 #pragma unroll
@@ -218,7 +226,250 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
             }
             og[(size_t)(row0 + qi) * a.ldo + h * DH + e] = from_float<T>(o / l);
         }
+        if (threadIdx.x == 0) TC_PROBE(8);
     }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Decode attention, bf16, built for short dependent chains: a cluster of ATD_CLUSTER CTAs serves one
+// (sequence, head).  CTA `rank` takes the 128-position chunks rank, rank + 8, ... (anchored at absolute
+// position 0) through a cp.async ring, keeps an online-softmax state per query, and the cluster merges
+// its eight states in rank order through distributed shared memory: no global scratch, no second kernel.
+// DH / 8 threads share a key (16 bytes each); a query's arithmetic does not depend on the other queries.
+// ---------------------------------------------------------------------------------------------------
+constexpr int ATD_THREADS = 128;
+constexpr int ATD_CLUSTER = 8;
+
+template <int DH> struct AtdCfg {
+    static constexpr int TPK = DH / 8;              // threads per key
+    static constexpr int KPP = ATD_THREADS / TPK;   // keys per pass
+    static constexpr int PPC = ATT_CH / KPP;        // passes per chunk
+    static constexpr int STAGES = DH <= 64 ? 3 : 2;
+    static constexpr int TILE_ELEMS = ATT_CH * DH;  // one chunk of keys (or values)
+    static constexpr int STAGE_ELEMS = 2 * TILE_ELEMS;
+};
+template <int DH, int QG>
+constexpr size_t attn_decode_smem_bytes() {
+    return (size_t)AtdCfg<DH>::STAGES * AtdCfg<DH>::STAGE_ELEMS * sizeof(bf16) +
+           sizeof(float) * ((size_t)2 * ATT_NQ * DH + 2 * ATT_NQ + 2 * 4 * QG + (size_t)4 * QG * DH);
+}
+
+// grid: (ATD_CLUSTER, heads, sequences) in clusters of ATD_CLUSTER along x; block: ATD_THREADS.
+template <int DH, int QG>
+__global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
+    using C = AtdCfg<DH>;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    bf16* ring = reinterpret_cast<bf16*>(smem_raw);
+    float* qs = reinterpret_cast<float*>(ring + (size_t)C::STAGES * C::STAGE_ELEMS);   // [ATT_NQ][DH]
+    float* racc = qs + ATT_NQ * DH;       // running weighted values [ATT_NQ][DH]
+    float* rm = racc + ATT_NQ * DH;       // running max [ATT_NQ]
+    float* rl = rm + ATT_NQ;              // running sum [ATT_NQ]
+    float* red = rl + ATT_NQ;             // [2][4][QG] per-warp chunk max / sum
+    float* pv = red + 2 * 4 * QG;         // [4][QG][DH] per-warp weighted values
+    TC_PROBE_INIT(210);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rank = blockIdx.x, h = blockIdx.y, g = blockIdx.z;
+    const int part = tid % C::TPK, kslot = tid / C::TPK;
+    pdl_launch_dependents();
+    pdl_wait();   // queries and the newest keys/values come from earlier kernels
+    if (tid == 0) TC_PROBE(1);
+    const int cnt = a.nq, row0 = g * a.nq;
+    const int b = a.row_seq[row0];
+    const int pos_first = a.row_pos[row0];
+    const int pos_last = pos_first + cnt - 1;
+    const int n_chunks = pos_last / ATT_CH + 1;
+    const int n_mine = rank < n_chunks ? (n_chunks - rank + ATD_CLUSTER - 1) / ATD_CLUSTER : 0;
+    const size_t head_base = ((size_t)b * a.n_heads + h) * a.t_max;
+    const size_t head_base2 = ((size_t)b * a.n_heads + h) * a.t_max2;
+    const int split = a.k2 ? a.split : INT_MAX;
+
+    auto issue = [&](int it) {
+        const int t0 = (rank + it * ATD_CLUSTER) * ATT_CH;
+        const int nt = min(ATT_CH, pos_last + 1 - t0);
+        bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
+        bf16* vs = ks + C::TILE_ELEMS;
+        for (int i = tid; i < nt * C::TPK; i += ATD_THREADS) {
+            const int t = i / C::TPK, v = i - t * C::TPK;
+            const int ta = t0 + t;
+            const bf16 *kg, *vg;
+            if (ta < split) {
+                kg = static_cast<const bf16*>(a.kcache) + (head_base + ta) * DH;
+                vg = static_cast<const bf16*>(a.vcache) + (head_base + ta) * DH;
+            } else {
+                kg = static_cast<const bf16*>(a.k2) + (head_base2 + (ta - split)) * DH;
+                vg = static_cast<const bf16*>(a.v2) + (head_base2 + (ta - split)) * DH;
+            }
+            cp_async16(ks + t * DH + v * 8, kg + v * 8);
+            cp_async16(vs + t * DH + v * 8, vg + v * 8);
+        }
+        // positions past the last query: zeros, so that a zero weight times them stays zero
+        for (int i = nt * C::TPK + tid; i < ATT_CH * C::TPK; i += ATD_THREADS) {
+            *reinterpret_cast<uint4*>(ks + i * 8) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(vs + i * 8) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+#pragma unroll
+    for (int it = 0; it < C::STAGES - 1; ++it) {
+        if (it < n_mine) issue(it);
+        cp_async_commit();
+    }
+    const bf16* qg = static_cast<const bf16*>(a.q);
+    for (int i = tid; i < cnt * DH; i += ATD_THREADS) {
+        const int qi = i / DH, el = i - qi * DH;
+        qs[i] = to_float(qg[(size_t)(row0 + qi) * a.ldq + h * DH + el]);
+    }
+    for (int i = tid; i < ATT_NQ * DH; i += ATD_THREADS) racc[i] = 0.f;
+    if (tid < ATT_NQ) { rm[tid] = -INFINITY; rl[tid] = 0.f; }
+    if (tid == 0) TC_PROBE(2);
+
+    for (int it = 0; it < n_mine; ++it) {
+        if (it + C::STAGES - 1 < n_mine) issue(it + C::STAGES - 1);
+        cp_async_commit();
+        asm volatile("cp.async.wait_group %0;" ::"n"(C::STAGES - 1) : "memory");
+        __syncthreads();
+        if (tid == 0 && it == 0) TC_PROBE(3);
+        const int t0 = (rank + it * ATD_CLUSTER) * ATT_CH;
+        const bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
+        const bf16* vs = ks + C::TILE_ELEMS;
+        for (int q0 = 0; q0 < cnt; q0 += QG) {
+            float qreg[QG][8];
+#pragma unroll
+            for (int qi = 0; qi < QG; ++qi)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) qreg[qi][j] = (q0 + qi < cnt) ? qs[(q0 + qi) * DH + part * 8 + j] : 0.f;
+            float sc[QG][C::PPC];
+            float mloc[QG];
+#pragma unroll
+            for (int qi = 0; qi < QG; ++qi) mloc[qi] = -INFINITY;
+#pragma unroll
+            for (int p = 0; p < C::PPC; ++p) {
+                const int key = p * C::KPP + kslot;
+                float kf[8];
+                load_vec(ks + key * DH + part * 8, kf);
+#pragma unroll
+                for (int qi = 0; qi < QG; ++qi) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) d = fmaf(qreg[qi][j], kf[j], d);
+#pragma unroll
+                    for (int o = 1; o < C::TPK; o <<= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+                    const bool live = (q0 + qi < cnt) && (t0 + key <= pos_first + q0 + qi);
+                    sc[qi][p] = live ? d * a.scale : -INFINITY;
+                    mloc[qi] = fmaxf(mloc[qi], sc[qi][p]);
+                }
+            }
+#pragma unroll
+            for (int qi = 0; qi < QG; ++qi) {
+#pragma unroll
+                for (int o = C::TPK; o < 32; o <<= 1) mloc[qi] = fmaxf(mloc[qi], __shfl_xor_sync(0xffffffffu, mloc[qi], o));
+                if (lane == 0) red[warp * QG + qi] = mloc[qi];
+            }
+            __syncthreads();
+            float acc[QG][8];
+#pragma unroll
+            for (int qi = 0; qi < QG; ++qi) {
+                const float mc = fmaxf(fmaxf(red[qi], red[QG + qi]), fmaxf(red[2 * QG + qi], red[3 * QG + qi]));
+                float ls = 0.f;
+#pragma unroll
+                for (int p = 0; p < C::PPC; ++p) {
+                    const float pr = mc > -INFINITY ? expf(sc[qi][p] - mc) : 0.f;
+                    sc[qi][p] = pr;
+                    ls += pr;
+                }
+#pragma unroll
+                for (int o = C::TPK; o < 32; o <<= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+                if (lane == 0) red[4 * QG + warp * QG + qi] = ls;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[qi][j] = 0.f;
+            }
+#pragma unroll
+            for (int p = 0; p < C::PPC; ++p) {
+                const int key = p * C::KPP + kslot;
+                float vf[8];
+                load_vec(vs + key * DH + part * 8, vf);
+#pragma unroll
+                for (int qi = 0; qi < QG; ++qi)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[qi][j] = fmaf(sc[qi][p], vf[j], acc[qi][j]);
+            }
+#pragma unroll
+            for (int qi = 0; qi < QG; ++qi)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+#pragma unroll
+                    for (int o = C::TPK; o < 32; o <<= 1) acc[qi][j] += __shfl_xor_sync(0xffffffffu, acc[qi][j], o);
+                    if (lane < C::TPK) pv[(warp * QG + qi) * DH + lane * 8 + j] = acc[qi][j];
+                }
+            __syncthreads();
+            // fold the chunk into the running state: thread (query slot, element)
+            float m_new[(QG * DH + ATD_THREADS - 1) / ATD_THREADS], l_new[(QG * DH + ATD_THREADS - 1) / ATD_THREADS];
+#pragma unroll
+            for (int u = 0; u < (QG * DH + ATD_THREADS - 1) / ATD_THREADS; ++u) {
+                const int idx = tid + u * ATD_THREADS;
+                const int qi = idx / DH, e = idx - qi * DH;
+                m_new[u] = 0.f; l_new[u] = 0.f;
+                if (qi < QG && q0 + qi < cnt) {
+                    const float mc = fmaxf(fmaxf(red[qi], red[QG + qi]), fmaxf(red[2 * QG + qi], red[3 * QG + qi]));
+                    const float lc = ((red[4 * QG + qi] + red[5 * QG + qi]) + red[6 * QG + qi]) + red[7 * QG + qi];
+                    const float oc = ((pv[qi * DH + e] + pv[(QG + qi) * DH + e]) + pv[(2 * QG + qi) * DH + e]) + pv[(3 * QG + qi) * DH + e];
+                    const float mo = rm[q0 + qi], lo = rl[q0 + qi];
+                    const float mn = fmaxf(mo, mc);
+                    const float fo = mo > -INFINITY ? expf(mo - mn) : 0.f;
+                    const float fn = mc > -INFINITY ? expf(mc - mn) : 0.f;
+                    racc[(q0 + qi) * DH + e] = racc[(q0 + qi) * DH + e] * fo + oc * fn;
+                    m_new[u] = mn; l_new[u] = lo * fo + lc * fn;
+                }
+            }
+            __syncthreads();
+#pragma unroll
+            for (int u = 0; u < (QG * DH + ATD_THREADS - 1) / ATD_THREADS; ++u) {
+                const int idx = tid + u * ATD_THREADS;
+                const int qi = idx / DH, e = idx - qi * DH;
+                if (e == 0 && qi < QG && q0 + qi < cnt) { rm[q0 + qi] = m_new[u]; rl[q0 + qi] = l_new[u]; }
+            }
+        }
+        __syncthreads();   // the stage may be refilled, the state re-read
+    }
+    if (tid == 0) TC_PROBE(4);
+    cluster_sync_all();
+    if (tid == 0) TC_PROBE(5);
+    // merge the cluster's states in rank order: CTA `rank` finishes queries rank, rank + 8, ...
+    float res[(ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER];
+#pragma unroll
+    for (int u = 0; u < (ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER; ++u) {
+        const int qi = rank + u * ATD_CLUSTER;
+        res[u] = 0.f;
+        if (qi < cnt && tid < DH) {
+            float mr[ATD_CLUSTER], lr[ATD_CLUSTER], ar[ATD_CLUSTER];
+#pragma unroll
+            for (int r = 0; r < ATD_CLUSTER; ++r) {
+                mr[r] = ld_dsmem_f32(smem_u32(rm + qi), r);
+                lr[r] = ld_dsmem_f32(smem_u32(rl + qi), r);
+                ar[r] = ld_dsmem_f32(smem_u32(racc + qi * DH + tid), r);
+            }
+            float mx = mr[0];
+#pragma unroll
+            for (int r = 1; r < ATD_CLUSTER; ++r) mx = fmaxf(mx, mr[r]);
+            float l = 0.f, o = 0.f;
+#pragma unroll
+            for (int r = 0; r < ATD_CLUSTER; ++r) {
+                const float f = mr[r] > -INFINITY ? expf(mr[r] - mx) : 0.f;
+                l = fmaf(lr[r], f, l);
+                o = fmaf(ar[r], f, o);
+            }
+            res[u] = o / l;
+        }
+    }
+    cluster_arrive();   // done reading the peers' states
+#pragma unroll
+    for (int u = 0; u < (ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER; ++u) {
+        const int qi = rank + u * ATD_CLUSTER;
+        if (qi < cnt && tid < DH) static_cast<bf16*>(a.out)[(size_t)(row0 + qi) * a.ldo + h * DH + tid] = __float2bfloat16_rn(res[u]);
+    }
+    if (tid == 0) TC_PROBE(6);
+    cluster_wait();   // nobody leaves while its state may still be read
+    if (tid == 0) TC_PROBE(7);
 }
 
 }  // namespace tandem

@@ -4,7 +4,8 @@
 //                          per tile on the TMEM lanes), the token rows are the B operand (16..64 columns).
 //                          The job is streaming W once from HBM: every CTA owns one (tile, K-slice) unit so
 //                          that all SMs pull weights, tiles arrive by TMA through a ring of stages, and the
-//                          K-slices of a tile are summed in slice order by the CTA that finishes last.
+//                          K-slices of a tile sit in one thread-block cluster and are summed in slice order
+//                          through distributed shared memory.
 //                          The token rows are written into the B stages by the CTA's own threads, which is
 //                          where the LayerNorm (or the fp32 -> bf16 cast) of the residual stream is fused.
 //                          The weight loads are issued before the kernel waits for its predecessor in the
@@ -33,10 +34,8 @@ struct TcDecodeArgs {
     int rows, K, N;         // N = output features over all segments
     int seg_rows;           // output features per weight segment (one tensor map each)
     int tiles_per_seg;      // ceil(seg_rows / 128)
-    int splits;             // K-slices per tile; grid = tiles * splits
+    int splits;             // K-slices per tile: 1, 2, 4 or 8 = the cluster size; grid = tiles * splits
     int stream_weights;     // 1: weights are read once per pass and should not stay in L2
-    float* partials;        // [tiles * splits][NB][128] fp32, used when splits > 1
-    int* tile_counters;     // [tiles], zero between launches
     int* err_flag;          // nullable
     float* amax_val;        // EPI_ARGMAX: [rows][amax_stride] best value per tile
     int* amax_idx;          //             and its output feature
@@ -61,7 +60,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&p);
 }
+__device__ __forceinline__ float4 ln_apply(float4 x, float mu, float rs, float4 g, float4 b) {
+    return make_float4((x.x - mu) * rs * g.x + b.x, (x.y - mu) * rs * g.y + b.y, (x.z - mu) * rs * g.z + b.z, (x.w - mu) * rs * g.w + b.w);
+}
 
+// grid: tiles * splits CTAs in clusters of `splits` (the K-slices of one tile); dynamic smem TcdCfg<NB>::SMEM_BYTES.
 template <int NB, int PRO, int EPI>
 __global__ void __launch_bounds__(TCD_THREADS)
 gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap tm0, const __grid_constant__ CUtensorMap tm1,
@@ -72,7 +75,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     __shared__ __align__(8) uint64_t s_empty[C::STAGES];
     __shared__ __align__(8) uint64_t s_accum;
     __shared__ uint32_t s_tmem;
-    __shared__ int s_last;
     __shared__ float s_mu[NB], s_rstd[NB];
     __shared__ float s_av[4][NB];
     __shared__ int s_ai[4][NB];
@@ -83,13 +85,18 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 
     const int S = a.splits;
     const int unit = blockIdx.x;
-    const int tile = unit / S, sp = unit - tile * S;
+    const int tile = unit / S, sp = unit - tile * S;                       // sp = this CTA's rank in its cluster
     const int seg = tile / a.tiles_per_seg;
     const int n_local0 = (tile - seg * a.tiles_per_seg) * 128;
     const int KB = (a.K + 63) >> 6;
     const int kb_base = KB / S, kb_rem = KB - kb_base * S;
     const int kb0 = sp * kb_base + min(sp, kb_rem);
     const int nkb = kb_base + (sp < kb_rem ? 1 : 0);
+    const int K4 = a.K >> 2;
+    // LayerNorm rows short enough to sit in registers (8 float4 per lane) and a K-slice that fits the ring
+    // without reuse: the B operand is then written straight from the registers that gave the statistics.
+    const bool ln_regs = PRO == PRO_LN && K4 <= 256 && nkb <= C::STAGES;
+    TC_PROBE_INIT(100 + PRO * 10 + EPI);
 
     if (warp == 5) {
         if (lane == 0) {
@@ -109,6 +116,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     tc_fence_after_sync();
     const uint32_t tmem = s_tmem;
     pdl_launch_dependents();
+    if (tid == 0) TC_PROBE(1);
 
     if (warp == 4) {
         // ---- weight tiles: independent of every earlier kernel, so no wait on the predecessor here ----
@@ -127,6 +135,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 if (a.stream_weights) tma_load_2d(ring0 + st * C::STAGE_BYTES, tm, (kb0 + i) * 64, n_local0, bar, pol);
                 else tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES, tm, (kb0 + i) * 64, n_local0, bar);
             }
+            TC_PROBE(2);
         }
         __syncwarp();
     } else if (warp == 5) {
@@ -140,6 +149,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                     break;
                 }
                 tc_fence_after_sync();
+                if (i == 0) TC_PROBE(3);
                 const uint64_t da = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES);
                 const uint64_t db = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES + C::A_BYTES);
 #pragma unroll
@@ -148,19 +158,77 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 umma_commit(smem_u32(&s_empty[st]));
             }
             umma_commit(smem_u32(&s_accum));
+            TC_PROBE(4);
         }
         __syncwarp();
+    } else if (ln_regs) {
+        // ---- warps 0-3, short LayerNorm rows: one pass over x.  Lane L holds the row's float4 number L + 32u in
+        // t[u], i.e. K-block 2u + (L >= 16), 16-byte chunk (L & 15) / 2, half L & 1. ----
+        float4 gq[C::STAGES], bq[C::STAGES];   // gain / bias of this lane's slot in each of the CTA's K-blocks
+#pragma unroll
+        for (int i = 0; i < C::STAGES; ++i) {
+            const int k4 = ((kb0 + i) >> 1) * 32 + lane;
+            const bool mine = i < nkb && ((kb0 + i) & 1) == (lane >> 4) && k4 < K4;
+            gq[i] = mine ? __ldg(reinterpret_cast<const float4*>(a.ln_g) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            bq[i] = mine ? __ldg(reinterpret_cast<const float4*>(a.ln_b) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        pdl_wait();   // x comes from earlier kernels; gains and biases above are parameters
+        if (tid == 0) TC_PROBE(5);
+        for (int r = warp; r < a.rows; r += 4) {
+            const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx);
+            float4 t[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) t[u] = (lane + 32 * u < K4) ? __ldcg(xr + lane + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float s = 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) s += (t[u].x + t[u].y) + (t[u].z + t[u].w);
+            const float mu = warp_sum(s) / (float)a.K;
+            if (tid == 0) TC_PROBE(13);
+            float q = 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (lane + 32 * u < K4) {
+                    const float d0 = t[u].x - mu, d1 = t[u].y - mu, d2 = t[u].z - mu, d3 = t[u].w - mu;
+                    q = fmaf(d0, d0, q); q = fmaf(d1, d1, q); q = fmaf(d2, d2, q); q = fmaf(d3, d3, q);
+                }
+            }
+            const float rs = 1.0f / sqrtf(warp_sum(q) / (float)a.K + 1e-5f);
+            if (tid == 0) TC_PROBE(14);
+#pragma unroll
+            for (int i = 0; i < C::STAGES; ++i) {
+                const int kb = kb0 + i;
+                if (i < nkb && (kb & 1) == (lane >> 4)) {
+                    const int u = kb >> 1;
+                    float4 xv = t[0];
+#pragma unroll
+                    for (int uu = 1; uu < 8; ++uu) if (u == uu) xv = t[uu];
+                    uint2 val = make_uint2(0u, 0u);   // beyond K the weights are zero-filled; so is x
+                    if (u * 32 + lane < K4) {
+                        const float4 y = ln_apply(xv, mu, rs, gq[i], bq[i]);
+                        val.x = pack_bf16x2(y.x, y.y); val.y = pack_bf16x2(y.z, y.w);
+                    }
+                    const int c = (lane & 15) >> 1;
+                    unsigned char* bt = ring + i * C::STAGE_BYTES + C::A_BYTES;
+                    *reinterpret_cast<uint2*>(bt + r * 128 + ((c ^ (r & 7)) << 4) + ((lane & 1) << 3)) = val;
+                }
+            }
+        }
+        // rows >= a.rows of the B tiles stay as they are: a column of the product depends on its own row only
+        if (tid == 0) TC_PROBE(15);
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0)
+            for (int i = 0; i < nkb; ++i) mbar_arrive(smem_u32(&s_full[i]));
+        if (tid == 0) TC_PROBE(6);
     } else {
-        // ---- warps 0-3: token rows into the B stages, then the epilogue ----
+        // ---- warps 0-3, general case: statistics (LayerNorm), then the K-blocks one by one ----
         pdl_wait();   // x (and everything the epilogue touches) comes from earlier kernels
+        if (tid == 0) TC_PROBE(5);
         if (PRO == PRO_LN) {
-            // Row statistics, one warp per row in a fixed lane-strided order (so they do not depend on how many
-            // rows ride along).  Rows of up to 1024 elements stay in registers between the two passes.
-            const int K4 = a.K >> 2;
-            for (int r = warp; r < a.rows; r += 4) {
+            for (int r = warp; r < a.rows; r += 4) {   // one warp per row, fixed lane-strided order
                 const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx);
                 float mu, var;
-                if (K4 <= 256) {
+                if (K4 <= 256) {   // the same arithmetic as the register path above
                     float4 t[8];
 #pragma unroll
                     for (int u = 0; u < 8; ++u) t[u] = (lane + 32 * u < K4) ? __ldcg(xr + lane + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -195,47 +263,72 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             }
             bar_sync(1, 128);
         }
-        for (int i = 0; i < nkb; ++i) {
-            const int st = i % C::STAGES;
-            if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
-                tc_report(a.err_flag, TC_ERR_SLOT);
-                break;
-            }
-            unsigned char* bt = ring + st * C::STAGE_BYTES + C::A_BYTES;
-            for (int idx = tid; idx < NB * 8; idx += 128) {
-                const int r = idx >> 3, c = idx & 7;
-                const int k = (kb0 + i) * 64 + c * 8;
-                uint4 val = make_uint4(0u, 0u, 0u, 0u);
-                if (r < a.rows && k < a.K) {
-                    if (PRO == PRO_BF16) {
-                        val = __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k));
-                    } else {
-                        const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
-                        float4 u0 = __ldcg(xp), u1 = __ldcg(xp + 1);
-                        if (PRO == PRO_LN) {
-                            const float mu = s_mu[r], rs = s_rstd[r];
-                            const float4 g0 = __ldg(reinterpret_cast<const float4*>(a.ln_g + k)), g1 = __ldg(reinterpret_cast<const float4*>(a.ln_g + k) + 1);
-                            const float4 b0 = __ldg(reinterpret_cast<const float4*>(a.ln_b + k)), b1 = __ldg(reinterpret_cast<const float4*>(a.ln_b + k) + 1);
-                            u0.x = (u0.x - mu) * rs * g0.x + b0.x; u0.y = (u0.y - mu) * rs * g0.y + b0.y;
-                            u0.z = (u0.z - mu) * rs * g0.z + b0.z; u0.w = (u0.w - mu) * rs * g0.w + b0.w;
-                            u1.x = (u1.x - mu) * rs * g1.x + b1.x; u1.y = (u1.y - mu) * rs * g1.y + b1.y;
-                            u1.z = (u1.z - mu) * rs * g1.z + b1.z; u1.w = (u1.w - mu) * rs * g1.w + b1.w;
-                        }
-                        val.x = pack_bf16x2(u0.x, u0.y); val.y = pack_bf16x2(u0.z, u0.w);
-                        val.z = pack_bf16x2(u1.x, u1.y); val.w = pack_bf16x2(u1.z, u1.w);
+        constexpr int CPT = NB * 8 / 128;   // 16-byte chunks of one B tile per thread
+        for (int i0 = 0; i0 < nkb; i0 += C::STAGES) {
+            // a ring's worth of K-blocks at a time: all loads first, so their latencies overlap
+            uint4 raw[PRO == PRO_BF16 ? C::STAGES : 1][CPT];
+            if (PRO == PRO_BF16) {
+#pragma unroll
+                for (int g = 0; g < C::STAGES; ++g)
+#pragma unroll
+                    for (int ch = 0; ch < CPT; ++ch) {
+                        const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
+                        const int k = (kb0 + i0 + g) * 64 + c * 8;
+                        raw[g][ch] = (i0 + g < nkb && r < a.rows && k < a.K)
+                                         ? __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k))
+                                         : make_uint4(0u, 0u, 0u, 0u);
                     }
-                }
-                // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
-                *reinterpret_cast<uint4*>(bt + r * 128 + ((c ^ (r & 7)) << 4)) = val;
             }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&s_full[st]));
+            bool dead = false;
+#pragma unroll
+            for (int g = 0; g < C::STAGES; ++g) {
+                const int i = i0 + g;
+                if (i >= nkb || dead) continue;
+                const int st = g;   // i0 is a multiple of STAGES
+                if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
+                    tc_report(a.err_flag, TC_ERR_SLOT);
+                    dead = true;
+                    continue;
+                }
+                unsigned char* bt = ring + st * C::STAGE_BYTES + C::A_BYTES;
+#pragma unroll
+                for (int ch = 0; ch < CPT; ++ch) {
+                    const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
+                    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                    if (PRO == PRO_BF16) {
+                        val = raw[g][ch];
+                    } else {
+                        const int k = (kb0 + i) * 64 + c * 8;
+                        if (r < a.rows && k < a.K) {
+                            const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
+                            float4 u0 = __ldcg(xp), u1 = __ldcg(xp + 1);
+                            if (PRO == PRO_LN) {
+                                const float mu = s_mu[r], rs = s_rstd[r];
+                                u0 = ln_apply(u0, mu, rs, __ldg(reinterpret_cast<const float4*>(a.ln_g + k)), __ldg(reinterpret_cast<const float4*>(a.ln_b + k)));
+                                u1 = ln_apply(u1, mu, rs, __ldg(reinterpret_cast<const float4*>(a.ln_g + k) + 1), __ldg(reinterpret_cast<const float4*>(a.ln_b + k) + 1));
+                            }
+                            val.x = pack_bf16x2(u0.x, u0.y); val.y = pack_bf16x2(u0.z, u0.w);
+                            val.z = pack_bf16x2(u1.x, u1.y); val.w = pack_bf16x2(u1.z, u1.w);
+                        }
+                    }
+                    // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
+                    *reinterpret_cast<uint4*>(bt + r * 128 + ((c ^ (r & 7)) << 4)) = val;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s_full[st]));
+            }
         }
+        if (tid == 0) TC_PROBE(6);
+    }
 
+    // ---- epilogue: warps 0-3 own TMEM lanes 32 * warp .. +31 = output features of the tile ----
+    float v[NB];
+    const int tl = warp * 32 + lane;
+    if (warp < 4) {
         if (!mbar_wait(smem_u32(&s_accum), 0)) tc_report(a.err_flag, TC_ERR_ACCUM);
         tc_fence_after_sync();
-        float v[NB];
+        if (tid == 0) TC_PROBE(7);
 #pragma unroll
         for (int c0 = 0; c0 < NB; c0 += 16) {
             float t[16];
@@ -243,47 +336,13 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[c0 + i] = t[i];
         }
-        const int tl = warp * 32 + lane;             // output feature within the tile = TMEM lane
-        const int n_local = n_local0 + tl;
-        const bool valid = n_local < a.seg_rows;
-        const int n = seg * a.seg_rows + n_local;
-        bool finish = true;
-        if (S > 1) {
-            float* mine = a.partials + (size_t)unit * NB * 128 + tl;
-#pragma unroll
-            for (int j = 0; j < NB; ++j)
-                if (j < a.rows) mine[j * 128] = v[j];
-            __threadfence();
-            bar_sync(1, 128);
-            if (tid == 0) {
-                const int t = atomicAdd(a.tile_counters + tile, 1);
-                s_last = (t == S - 1);
-                if (t == S - 1) a.tile_counters[tile] = 0;   // ready for the next launch
-            }
-            bar_sync(1, 128);
-            finish = s_last != 0;
-            if (finish) {
-                __threadfence();
-                const float* base = a.partials + (size_t)tile * S * NB * 128 + tl;
-                constexpr int U = NB <= 16 ? 4 : (NB <= 32 ? 2 : 1);   // slices fetched together; summed in slice order
-#pragma unroll
-                for (int j = 0; j < NB; ++j) v[j] = 0.f;
-                for (int s0 = 0; s0 < S; s0 += U) {
-                    float t[U][NB];
-#pragma unroll
-                    for (int u = 0; u < U; ++u)
-#pragma unroll
-                        for (int j = 0; j < NB; ++j)
-                            t[u][j] = (s0 + u < S && j < a.rows) ? __ldcg(base + ((size_t)(s0 + u) * NB + j) * 128) : 0.f;
-#pragma unroll
-                    for (int u = 0; u < U; ++u)
-#pragma unroll
-                        for (int j = 0; j < NB; ++j)
-                            if (s0 + u < S) v[j] += t[u][j];
-                }
-            }
-        }
-        if (finish) {
+        if (tid == 0) TC_PROBE(8);
+    }
+    if (S == 1) {
+        if (warp < 4) {
+            const int n_local = n_local0 + tl;
+            const bool valid = n_local < a.seg_rows;
+            const int n = seg * a.seg_rows + n_local;
             if (EPI == EPI_ARGMAX) {
                 float* out = static_cast<float*>(a.e.out);
 #pragma unroll
@@ -316,10 +375,55 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                     if (j < a.rows && valid) epilogue<bf16, EPI>(a.e, j, n, v[j]);
             }
         }
+    } else {
+        // The cluster's CTAs hold the K-slices of one tile.  Each parks its partial tile in its own shared memory
+        // (the ring is free: every MMA has completed), then CTA `sp` sums columns [sp*128/S, (sp+1)*128/S) over
+        // the slices in slice order, reading the other CTAs' shared memory, and runs the epilogue for them.
+        float* red = reinterpret_cast<float*>(ring);   // [NB][128]
+        if (warp < 4) {
+#pragma unroll
+            for (int j = 0; j < NB; ++j)
+                if (j < a.rows) red[j * 128 + tl] = v[j];
+        }
+        cluster_sync_all();
+        if (tid == 0) TC_PROBE(9);
+        if (warp < 4 && EPI != EPI_ARGMAX) {
+            const int CW = 128 / S;                       // columns this CTA finishes
+            const int col = sp * CW + (tid & (CW - 1));
+            const int n_local = n_local0 + col;
+            const bool valid = n_local < a.seg_rows;
+            const int n = seg * a.seg_rows + n_local;
+            const uint32_t red0 = ring0 + col * 4;
+            float accs[NB / 2];                            // 128 / CW = S row groups: rows tid / CW, + S, ...
+#pragma unroll
+            for (int it = 0; it < NB / 2; ++it) {
+                const int j = tid / CW + it * S;
+                accs[it] = 0.f;
+                if (j < a.rows) {
+                    float part[8];
+#pragma unroll
+                    for (int ss = 0; ss < 8; ++ss) part[ss] = ss < S ? ld_dsmem_f32(red0 + j * 512, ss) : 0.f;
+#pragma unroll
+                    for (int ss = 0; ss < 8; ++ss) if (ss < S) accs[it] += part[ss];   // slice order
+                }
+            }
+            cluster_arrive();   // done reading the peers' shared memory
+            if (tid == 0) TC_PROBE(10);
+#pragma unroll
+            for (int it = 0; it < NB / 2; ++it) {
+                const int j = tid / CW + it * S;
+                if (j < a.rows && valid) epilogue<bf16, EPI>(a.e, j, n, accs[it]);
+            }
+        } else {
+            cluster_arrive();
+        }
+        cluster_wait();   // nobody leaves while its shared memory may still be read
     }
+    if (tid == 0) TC_PROBE(11);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 5) tmem_dealloc(tmem, C::TMEM_COLS);
+    if (tid == 0) TC_PROBE(12);
 }
 
 // ---------------------------------------------------------------------------------------------------

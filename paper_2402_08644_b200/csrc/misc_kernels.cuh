@@ -85,8 +85,10 @@ __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, i
                                                          int* row_seq, int* row_pos, const T* __restrict__ emb,
                                                          const T* __restrict__ pos, float* __restrict__ h, int d) {
     __shared__ int s_tok, s_pos;
+    TC_PROBE_INIT(300);
     pdl_launch_dependents();
     pdl_wait();
+    if (threadIdx.x == 0) TC_PROBE(1);
     const int m = blockIdx.x;
     const int b = m / nq, r = r0 + (m - b * nq);
     if (threadIdx.x < 32) {
@@ -105,6 +107,7 @@ __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, i
     const T* er = emb + (size_t)s_tok * d;
     const T* pr = pos + (size_t)s_pos * d;
     for (int i = threadIdx.x; i < d; i += 128) h[(size_t)m * d + i] = to_float(er[i]) + to_float(pr[i]);
+    if (threadIdx.x == 0) TC_PROBE(2);
 }
 
 __device__ __forceinline__ float block_sum_128(float v, float* red) {
@@ -174,8 +177,10 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restric
 __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed,
                                                      int max_new, const float* amax_val, const int* amax_idx, int amax_stride,
                                                      int n_tiles) {
+    TC_PROBE_INIT(400);
     pdl_launch_dependents();
     pdl_wait();
+    if (threadIdx.x == 0) TC_PROBE(1);
     if (amax_val != nullptr) {
         const int rows = batch * (gamma + 1);
         for (int m = threadIdx.x >> 5; m < rows; m += 8) {
@@ -226,6 +231,7 @@ __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, in
         st.host_flags[4] = st.counters[5];
         __threadfence_system();
         st.host_flags[0] = ticket;
+        TC_PROBE(2);
     }
 }
 

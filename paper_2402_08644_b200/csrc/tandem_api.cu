@@ -40,17 +40,16 @@ thread_local char g_cuda_err[256] = "";
 
 size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 int cdiv(int a, int b) { return (a + b - 1) / b; }
-constexpr int TC_MAX_UNITS = 512;
 // Columns of the tensor-core decode GEMM's B operand for a number of token rows (0: too many rows for it).
-int tc_nb(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 48 ? 48 : rows <= 64 ? 64 : 0; }   // most (tile, K-slice) units of a split-K launch of the tensor-core decode GEMM
+int tc_nb(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 48 ? 48 : rows <= 64 ? 64 : 0; }
 
 struct Layout {   // byte offsets into the arena
     size_t kv_large, kv_small;
     size_t st_n, st_pending, st_drafts, st_targets, st_accept, st_emitted, st_done, st_out, st_counters, st_hist;
     size_t row_tok, row_seq, row_pos, grp_row0, grp_cnt;
-    size_t tc_counters, attn_counters;   // inside the zero-filled state block
+    size_t attn_counters;   // inside the zero-filled state block
     size_t h_large, h_small, a, q, o, f, xb, t1, yhat, a_s, logits_large, logits_small, part_ml, part_acc, dbg;
-    size_t tc_partials, amax_val_large, amax_idx_large, amax_val_small, amax_idx_small;
+    size_t amax_val_large, amax_idx_large, amax_val_small, amax_idx_small;
     size_t total;
     int max_rows, dec_rows, max_groups, n_chunks_max, vocab_tiles;
     size_t kv_large_layer, kv_small_layer;   // elements per (layer, k-or-v)
@@ -191,7 +190,6 @@ Layout make_layout(const tandem_config& c) {
     L.st_done = take(B * 4); L.st_out = take(B * T * 4); L.st_counters = take(16 * 4); L.st_hist = take((GL + 1) * 8);
     L.row_tok = take(R * 4); L.row_seq = take(R * 4); L.row_pos = take(R * 4);
     L.grp_row0 = take((size_t)L.max_groups * 4); L.grp_cnt = take((size_t)L.max_groups * 4);
-    L.tc_counters = take(TC_MAX_UNITS * 4);
     L.attn_counters = take(B * hmax * 4);
     L.h_large = take(R * c.large.d_model * 4);
     L.h_small = take(B * c.small.d_model * 4);
@@ -205,7 +203,6 @@ Layout make_layout(const tandem_config& c) {
     L.part_acc = take(RD * dmax * L.n_chunks_max * 4);
     L.dbg = take(T * dmax * 4);
     L.vocab_tiles = cdiv(c.large.vocab, 128);
-    L.tc_partials = take((size_t)TC_MAX_UNITS * tc_nb(L.dec_rows) * 128 * 4);
     L.amax_val_large = take(RD * L.vocab_tiles * 4); L.amax_idx_large = take(RD * L.vocab_tiles * 4);
     L.amax_val_small = take(B * L.vocab_tiles * 4); L.amax_idx_small = take(B * L.vocab_tiles * 4);
     L.total = off;
@@ -297,7 +294,7 @@ struct TcW {              // up to three weight matrices stacked along the outpu
     CUtensorMap tm[3];
     int n_segs, seg_rows, K;
 };
-struct TcScratch { float* partials; int* counters; int* err; };
+struct TcScratch { int* err; };
 
 TcW tcw(const tandem_ctx& c, int i0, int i1, int i2, int seg_rows, int K) {
     TcW w;
@@ -311,22 +308,29 @@ TcW tcw(const tandem_ctx& c, int i0, int i1, int i2, int seg_rows, int K) {
 
 TcScratch tc_scratch(tandem_ctx& c) {
     TcScratch s;
-    s.partials = reinterpret_cast<float*>(c.arena + c.lay.tc_partials);
-    s.counters = reinterpret_cast<int*>(c.arena + c.lay.tc_counters);
     s.err = c.st.counters + 2;
     return s;
 }
 
 template <typename... KArgs, typename... Args>
-void launch_ex(tandem_ctx& c, bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+void launch_ex(tandem_ctx& c, bool pdl, int cluster, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c.stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (pdl && c.use_pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (cluster > 1) {   // consecutive blocks along x form a thread-block cluster
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = (pdl && c.use_pdl) ? 1 : 0;
+    cfg.numAttrs = n;
     cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
     c.launches++;
 }
@@ -340,7 +344,7 @@ void launch_tc_decode_nb(tandem_ctx& c, const TcDecodeArgs& a, const TcW& w, int
         cudaFuncSetAttribute(gemm_tc_decode_kernel<NB, PRO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
         attr_set[dev] = true;
     }
-    launch_ex(c, true, gemm_tc_decode_kernel<NB, PRO, EPI>, dim3(units), dim3(TCD_THREADS), (size_t)C::SMEM_BYTES, a, w.tm[0], w.tm[1], w.tm[2]);
+    launch_ex(c, true, a.splits, gemm_tc_decode_kernel<NB, PRO, EPI>, dim3(units), dim3(TCD_THREADS), (size_t)C::SMEM_BYTES, a, w.tm[0], w.tm[1], w.tm[2]);
 }
 
 // y = prologue(x) W^T for rows <= 64 on the tensor cores, streaming W once.
@@ -354,12 +358,14 @@ void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx
     a.x = x; a.ldx = ldx; a.ln_g = static_cast<const float*>(ln_g); a.ln_b = static_cast<const float*>(ln_b);
     a.rows = rows; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
     const int tiles = w.n_segs * a.tiles_per_seg, KB = cdiv(w.K, 64);
+    // K-slices per tile = cluster size: the smallest power of two that puts tiles * S CTAs at or above the target
+    // (about one per SM), at most 8 and at most one per 64-element K-block.  The head GEMM keeps whole tiles.
     int S = 1;
-    if (tiles < c.tc_target) S = std::min(KB, cdiv(c.tc_target, tiles));
-    while (S > 1 && tiles * S > TC_MAX_UNITS) --S;
+    if (EPI != EPI_ARGMAX)
+        while (S < 8 && tiles * S < c.tc_target && 2 * S <= KB) S *= 2;
     a.splits = S;
     a.stream_weights = stream_weights ? 1 : 0;
-    a.partials = sc.partials; a.tile_counters = sc.counters; a.err_flag = sc.err;
+    a.err_flag = sc.err;
     a.amax_val = amax_val; a.amax_idx = amax_idx; a.amax_stride = amax_stride;
     a.e = e;
     const size_t xsz = PRO == PRO_BF16 ? 2 : 4;
@@ -391,7 +397,7 @@ tandem_status launch_tc_tiled(tandem_ctx& c, const bf16* x, int ldx, int M, cons
     a.M = M; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
     a.err_flag = err; a.e = e;
     ProfScope ps(c, PC_GEMM_TC_TILED, 2.0 * M * (double)a.N * w.K);   // flops
-    launch_ex(c, false, gemm_tc_tiled_kernel<EPI>, dim3(w.n_segs * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)TCT_SMEM_BYTES,
+    launch_ex(c, false, 1, gemm_tc_tiled_kernel<EPI>, dim3(w.n_segs * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)TCT_SMEM_BYTES,
               a, tmx, w.tm[0], w.tm[1], w.tm[2]);
     return TANDEM_OK;
 }
@@ -440,10 +446,10 @@ void launch_attn_dh(tandem_ctx& c, const AttnArgs& a, int groups, bool loop, int
     if (!attr_set[dev]) { set_attn_attrs<T, DH>(); attr_set[dev] = true; }
     if (loop) {
         ProfScope ps(c, PC_ATTN_PROMPT, kv_bytes);
-        launch_ex(c, false, attn_kernel<T, DH, true>, dim3(1, a.n_heads, groups), dim3(ATT_THREADS), attn_smem_bytes<T, DH>(), a);
+        launch_ex(c, false, 1, attn_kernel<T, DH, true>, dim3(1, a.n_heads, groups), dim3(ATT_THREADS), attn_smem_bytes<T, DH>(), a);
     } else {
         ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
-        launch_ex(c, true, attn_kernel<T, DH, false>, dim3(n_chunks, a.n_heads, groups), dim3(ATT_THREADS), attn_smem_bytes<T, DH>(), a);
+        launch_ex(c, true, 1, attn_kernel<T, DH, false>, dim3(n_chunks, a.n_heads, groups), dim3(ATT_THREADS), attn_smem_bytes<T, DH>(), a);
     }
 }
 
@@ -452,6 +458,26 @@ void launch_attn(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, bool 
     if (d_head == 32) launch_attn_dh<T, 32>(c, a, groups, loop, n_chunks, kv_bytes);
     else if (d_head == 64) launch_attn_dh<T, 64>(c, a, groups, loop, n_chunks, kv_bytes);
     else launch_attn_dh<T, 128>(c, a, groups, loop, n_chunks, kv_bytes);
+}
+
+// bf16 decode attention: one cluster of ATD_CLUSTER CTAs per (sequence, head); no scratch.
+template <int DH, int QG>
+void launch_attn_decode_dq(tandem_ctx& c, const AttnArgs& a, int groups, double kv_bytes) {
+    static bool attr_set[MAX_DEVICES] = {};
+    const int dev = cur_dev();
+    if (!attr_set[dev]) {
+        cudaFuncSetAttribute(attn_decode_kernel<DH, QG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_decode_smem_bytes<DH, QG>());
+        attr_set[dev] = true;
+    }
+    ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
+    launch_ex(c, true, ATD_CLUSTER, attn_decode_kernel<DH, QG>, dim3(ATD_CLUSTER, a.n_heads, groups), dim3(ATD_THREADS),
+              attn_decode_smem_bytes<DH, QG>(), a);
+}
+void launch_attn_decode(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, double kv_bytes) {
+    const bool one = a.nq == 1;
+    if (d_head == 32) { if (one) launch_attn_decode_dq<32, 1>(c, a, groups, kv_bytes); else launch_attn_decode_dq<32, 4>(c, a, groups, kv_bytes); }
+    else if (d_head == 64) { if (one) launch_attn_decode_dq<64, 1>(c, a, groups, kv_bytes); else launch_attn_decode_dq<64, 4>(c, a, groups, kv_bytes); }
+    else { if (one) launch_attn_decode_dq<128, 1>(c, a, groups, kv_bytes); else launch_attn_decode_dq<128, 4>(c, a, groups, kv_bytes); }
 }
 
 template <typename T>
@@ -501,7 +527,8 @@ void attention(tandem_ctx& c, const Model& m, int l, const T* q, T* o, const Row
     aa.part_ml = at<float>(c, c.lay.part_ml); aa.part_acc = at<float>(c, c.lay.part_acc);
     aa.n_chunks_max = c.lay.n_chunks_max; aa.scale = 1.0f / sqrtf((float)dh);
     aa.merge_counters = at<int>(c, c.lay.attn_counters);
-    launch_attn<T>(c, dh, aa, r.groups, !r.decode, r.n_chunks, r.kv_positions * 2.0 * d * sizeof(T));
+    if (r.decode && sizeof(T) == 2 && r.groups <= 65535) launch_attn_decode(c, dh, aa, r.groups, r.kv_positions * 2.0 * d * sizeof(T));
+    else launch_attn<T>(c, dh, aa, r.groups, !r.decode, r.n_chunks, r.kv_positions * 2.0 * d * sizeof(T));
 }
 
 // Eq. 2, first line, for small layer j, then that layer's LayerNorm and key/value maps: writes the
@@ -622,7 +649,7 @@ void small_step(tandem_ctx& c, int s) {
 
 void launch_verify(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new, bool from_tiles) {
     ProfScope ps(c, PC_VERIFY, (double)c.batch * (2 * gamma + 8) * 4.0);
-    launch_ex(c, true, verify_kernel, dim3(1), dim3(256), 0, c.st, c.batch, gamma, mode, (unsigned long long)seed, max_new,
+    launch_ex(c, true, 1, verify_kernel, dim3(1), dim3(256), 0, c.st, c.batch, gamma, mode, (unsigned long long)seed, max_new,
               from_tiles ? (const float*)at<float>(c, c.lay.amax_val_large) : (const float*)nullptr,
               from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_large) : (const int*)nullptr, c.lay.vocab_tiles, c.lay.vocab_tiles);
 }
@@ -652,7 +679,7 @@ void greedy_iteration(tandem_ctx& c, int max_new) {
 // arg-max the small model's last head GEMM left as per-tile results (-1: none).
 void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r) {
     ProfScope ps(c, PC_ROWS, (double)c.batch * nq * m.d.d_model * 8.0);
-    launch_ex(c, true, step_begin_kernel<bf16>, dim3(c.batch * nq), dim3(128), 0, c.st, r0, nq, fin_r,
+    launch_ex(c, true, 1, step_begin_kernel<bf16>, dim3(c.batch * nq), dim3(128), 0, c.st, r0, nq, fin_r,
               (const float*)at<float>(c, c.lay.amax_val_small), (const int*)at<int>(c, c.lay.amax_idx_small), c.lay.vocab_tiles,
               c.lay.vocab_tiles, at<int>(c, c.lay.row_tok), at<int>(c, c.lay.row_seq), at<int>(c, c.lay.row_pos),
               (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model);
@@ -914,7 +941,7 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
     c->use_graphs = getenv("TANDEM_NO_GRAPH") == nullptr;
     c->use_pdl = getenv("TANDEM_NO_PDL") == nullptr;
-    if (const char* t = getenv("TANDEM_TC_TARGET")) c->tc_target = std::max(1, std::min(TC_MAX_UNITS, atoi(t)));
+    if (const char* t = getenv("TANDEM_TC_TARGET")) c->tc_target = std::max(1, atoi(t));
     if (e == cudaSuccess && cfg->dtype == TANDEM_DTYPE_BF16 && getenv("TANDEM_NO_TC") == nullptr) {
         // one tensor map per weight matrix: [out_features][in_features], 128 x 64 tiles
         c->wmap.resize(c->w.size());
@@ -1366,15 +1393,13 @@ extern "C" tandem_status tandem_decode_attention_static(const void* q, const voi
 }
 
 namespace {
-struct ProjScratch { size_t yhat, a_s, rows, partials, counters, total; };
+struct ProjScratch { size_t yhat, a_s, rows, total; };
 ProjScratch proj_scratch_layout(int rows, int d_small) {
     ProjScratch p;
     size_t off = 0;
     p.yhat = off; off = align_up(off + (size_t)rows * d_small * 4);
     p.a_s = off; off = align_up(off + (size_t)rows * d_small * 2);
     p.rows = off; off = align_up(off + (size_t)rows * 8);
-    p.counters = off; off = align_up(off + (size_t)TC_MAX_UNITS * 4);
-    p.partials = off; off = align_up(off + (size_t)TC_MAX_UNITS * std::max(16, tc_nb(rows)) * 128 * 4);
     p.total = off;
     return p;
 }
@@ -1418,8 +1443,7 @@ extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
     e.kcache = k_out; e.vcache = v_out; e.row_seq = row_seq; e.row_pos = row_pos; e.n_heads = 1; e.d_head = d_small; e.t_max = 1; e.seg = d_small;
     if (tc_nb(rows) != 0) {
         // few rows: weights streamed once per GEMM; LayerNorm fused into the second GEMM's operand load
-        CK(cudaMemsetAsync(sc + pl.counters, 0, (size_t)TC_MAX_UNITS * 4, tmp.stream));
-        TcScratch ts; ts.partials = reinterpret_cast<float*>(sc + pl.partials); ts.counters = reinterpret_cast<int*>(sc + pl.counters); ts.err = nullptr;
+        TcScratch ts; ts.err = nullptr;
         launch_tc_decode<PRO_BF16, EPI_STORE_F32>(tmp, ts, x, d_large, nullptr, nullptr, rows, wt, true, epi_plain(yhat, d_small));
         launch_tc_decode<PRO_LN, EPI_KV>(tmp, ts, yhat, d_small, ln_g, ln_b, rows, wkv, true, e);
     } else {

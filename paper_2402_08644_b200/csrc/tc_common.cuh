@@ -9,6 +9,12 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// Measurement hooks: checkpoints that a profiling build may define to record timestamps; nothing otherwise.
+#ifndef TC_PROBE
+#define TC_PROBE_INIT(tag)
+#define TC_PROBE(slot)
+#endif
+
 namespace tandem {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -130,6 +136,23 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
         : "r"(taddr) : "memory");
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---- thread-block clusters ----------------------------------------------------------------------
+// Barrier over every thread of every CTA in the cluster, with release/acquire ordering of shared memory.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+// The same barrier in two halves: arrive once this CTA no longer reads its peers' shared memory, wait before exit.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+// Reads a float at the same shared-memory offset in the cluster's CTA number `rank`.
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t local_smem_addr, int rank) {
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_smem_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
 }
 
 // Named barrier among a subset of the CTA's warps.
