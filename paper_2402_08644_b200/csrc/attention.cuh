@@ -235,10 +235,13 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
 // (sequence, head).  CTA `rank` takes the 128-position chunks rank, rank + 8, ... (anchored at absolute
 // position 0) through a cp.async ring, keeps an online-softmax state per query, and the cluster merges
 // its eight states in rank order through distributed shared memory: no global scratch, no second kernel.
+// The probabilities use the fast exponential (2^x hardware approximation), well inside the bf16 tolerance.
 // DH / 8 threads share a key (16 bytes each); a query's arithmetic does not depend on the other queries.
 // ---------------------------------------------------------------------------------------------------
-constexpr int ATD_THREADS = 128;
+constexpr int ATD_THREADS = 256;
+constexpr int ATD_WARPS = ATD_THREADS / 32;
 constexpr int ATD_CLUSTER = 8;
+constexpr int ATD_QPC = (ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER;   // queries a CTA finishes at most
 
 template <int DH> struct AtdCfg {
     static constexpr int TPK = DH / 8;              // threads per key
@@ -251,21 +254,24 @@ template <int DH> struct AtdCfg {
 template <int DH, int QG>
 constexpr size_t attn_decode_smem_bytes() {
     return (size_t)AtdCfg<DH>::STAGES * AtdCfg<DH>::STAGE_ELEMS * sizeof(bf16) +
-           sizeof(float) * ((size_t)2 * ATT_NQ * DH + 2 * ATT_NQ + 2 * 4 * QG + (size_t)4 * QG * DH);
+           sizeof(float) * ((size_t)2 * ATT_NQ * DH + 2 * ATT_NQ + 2 * ATD_WARPS * QG + (size_t)ATD_WARPS * QG * DH +
+                            (size_t)ATD_CLUSTER * ATD_QPC * (DH + 2));
 }
 
 // grid: (ATD_CLUSTER, heads, sequences) in clusters of ATD_CLUSTER along x; block: ATD_THREADS.
 template <int DH, int QG>
 __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     using C = AtdCfg<DH>;
+    constexpr int NW = ATD_WARPS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     bf16* ring = reinterpret_cast<bf16*>(smem_raw);
     float* qs = reinterpret_cast<float*>(ring + (size_t)C::STAGES * C::STAGE_ELEMS);   // [ATT_NQ][DH]
     float* racc = qs + ATT_NQ * DH;       // running weighted values [ATT_NQ][DH]
     float* rm = racc + ATT_NQ * DH;       // running max [ATT_NQ]
     float* rl = rm + ATT_NQ;              // running sum [ATT_NQ]
-    float* red = rl + ATT_NQ;             // [2][4][QG] per-warp chunk max / sum
-    float* pv = red + 2 * 4 * QG;         // [4][QG][DH] per-warp weighted values
+    float* red = rl + ATT_NQ;             // [2][NW][QG] per-warp chunk max / sum
+    float* pv = red + 2 * NW * QG;        // [NW][QG][DH] per-warp weighted values
+    float* inbox = pv + NW * QG * DH;     // [ATD_CLUSTER][ATD_QPC][DH + 2] states sent by the cluster's CTAs
     TC_PROBE_INIT(210);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -275,6 +281,12 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     pdl_wait();   // queries and the newest keys/values come from earlier kernels
     if (tid == 0) TC_PROBE(1);
     const int cnt = a.nq, row0 = g * a.nq;
+    // queries first (their address needs nothing else), then the position that fixes the chunks
+    const bf16* qg = static_cast<const bf16*>(a.q);
+    for (int i = tid; i < cnt * DH; i += ATD_THREADS) {
+        const int qi = i / DH, el = i - qi * DH;
+        qs[i] = to_float(qg[(size_t)(row0 + qi) * a.ldq + h * DH + el]);
+    }
     const int b = a.row_seq[row0];
     const int pos_first = a.row_pos[row0];
     const int pos_last = pos_first + cnt - 1;
@@ -313,11 +325,6 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     for (int it = 0; it < C::STAGES - 1; ++it) {
         if (it < n_mine) issue(it);
         cp_async_commit();
-    }
-    const bf16* qg = static_cast<const bf16*>(a.q);
-    for (int i = tid; i < cnt * DH; i += ATD_THREADS) {
-        const int qi = i / DH, el = i - qi * DH;
-        qs[i] = to_float(qg[(size_t)(row0 + qi) * a.ldq + h * DH + el]);
     }
     for (int i = tid; i < ATT_NQ * DH; i += ATD_THREADS) racc[i] = 0.f;
     if (tid < ATT_NQ) { rm[tid] = -INFINITY; rl[tid] = 0.f; }
@@ -366,20 +373,23 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
                 if (lane == 0) red[warp * QG + qi] = mloc[qi];
             }
             __syncthreads();
+            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(8);
             float acc[QG][8];
 #pragma unroll
             for (int qi = 0; qi < QG; ++qi) {
-                const float mc = fmaxf(fmaxf(red[qi], red[QG + qi]), fmaxf(red[2 * QG + qi], red[3 * QG + qi]));
+                float mc = red[qi];
+#pragma unroll
+                for (int w = 1; w < NW; ++w) mc = fmaxf(mc, red[w * QG + qi]);
                 float ls = 0.f;
 #pragma unroll
                 for (int p = 0; p < C::PPC; ++p) {
-                    const float pr = mc > -INFINITY ? expf(sc[qi][p] - mc) : 0.f;
+                    const float pr = mc > -INFINITY ? __expf(sc[qi][p] - mc) : 0.f;
                     sc[qi][p] = pr;
                     ls += pr;
                 }
 #pragma unroll
                 for (int o = C::TPK; o < 32; o <<= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
-                if (lane == 0) red[4 * QG + warp * QG + qi] = ls;
+                if (lane == 0) red[NW * QG + warp * QG + qi] = ls;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[qi][j] = 0.f;
             }
@@ -402,74 +412,73 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
                     if (lane < C::TPK) pv[(warp * QG + qi) * DH + lane * 8 + j] = acc[qi][j];
                 }
             __syncthreads();
+            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(9);
             // fold the chunk into the running state: thread (query slot, element)
-            float m_new[(QG * DH + ATD_THREADS - 1) / ATD_THREADS], l_new[(QG * DH + ATD_THREADS - 1) / ATD_THREADS];
+            constexpr int FU = (QG * DH + ATD_THREADS - 1) / ATD_THREADS;
+            float m_new[FU], l_new[FU];
 #pragma unroll
-            for (int u = 0; u < (QG * DH + ATD_THREADS - 1) / ATD_THREADS; ++u) {
+            for (int u = 0; u < FU; ++u) {
                 const int idx = tid + u * ATD_THREADS;
                 const int qi = idx / DH, e = idx - qi * DH;
                 m_new[u] = 0.f; l_new[u] = 0.f;
                 if (qi < QG && q0 + qi < cnt) {
-                    const float mc = fmaxf(fmaxf(red[qi], red[QG + qi]), fmaxf(red[2 * QG + qi], red[3 * QG + qi]));
-                    const float lc = ((red[4 * QG + qi] + red[5 * QG + qi]) + red[6 * QG + qi]) + red[7 * QG + qi];
-                    const float oc = ((pv[qi * DH + e] + pv[(QG + qi) * DH + e]) + pv[(2 * QG + qi) * DH + e]) + pv[(3 * QG + qi) * DH + e];
+                    float mc = red[qi], lc = red[NW * QG + qi], oc = pv[qi * DH + e];
+#pragma unroll
+                    for (int w = 1; w < NW; ++w) {   // warp order
+                        mc = fmaxf(mc, red[w * QG + qi]);
+                        lc += red[NW * QG + w * QG + qi];
+                        oc += pv[(w * QG + qi) * DH + e];
+                    }
                     const float mo = rm[q0 + qi], lo = rl[q0 + qi];
                     const float mn = fmaxf(mo, mc);
-                    const float fo = mo > -INFINITY ? expf(mo - mn) : 0.f;
-                    const float fn = mc > -INFINITY ? expf(mc - mn) : 0.f;
+                    const float fo = mo > -INFINITY ? __expf(mo - mn) : 0.f;
+                    const float fn = mc > -INFINITY ? __expf(mc - mn) : 0.f;
                     racc[(q0 + qi) * DH + e] = racc[(q0 + qi) * DH + e] * fo + oc * fn;
                     m_new[u] = mn; l_new[u] = lo * fo + lc * fn;
                 }
             }
             __syncthreads();
 #pragma unroll
-            for (int u = 0; u < (QG * DH + ATD_THREADS - 1) / ATD_THREADS; ++u) {
+            for (int u = 0; u < FU; ++u) {
                 const int idx = tid + u * ATD_THREADS;
                 const int qi = idx / DH, e = idx - qi * DH;
                 if (e == 0 && qi < QG && q0 + qi < cnt) { rm[q0 + qi] = m_new[u]; rl[q0 + qi] = l_new[u]; }
             }
+            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(10);
         }
         __syncthreads();   // the stage may be refilled, the state re-read
     }
+    __syncthreads();       // a CTA without chunks comes straight from initialising its state
     if (tid == 0) TC_PROBE(4);
+    // Query qi is finished by CTA qi % 8: every CTA sends it its state for that query (remote shared-memory stores),
+    // one cluster barrier makes the states visible, and the owner merges them in rank order.  Nobody touches a
+    // peer's shared memory after the barrier.
+    for (int i = tid; i < cnt * (DH + 2); i += ATD_THREADS) {
+        const int qi = i / (DH + 2), e = i - qi * (DH + 2);
+        const float val = e < DH ? racc[qi * DH + e] : (e == DH ? rm[qi] : rl[qi]);
+        st_dsmem_f32(smem_u32(inbox + ((size_t)rank * ATD_QPC + qi / ATD_CLUSTER) * (DH + 2) + e), qi % ATD_CLUSTER, val);
+    }
     cluster_sync_all();
     if (tid == 0) TC_PROBE(5);
-    // merge the cluster's states in rank order: CTA `rank` finishes queries rank, rank + 8, ...
-    float res[(ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER];
 #pragma unroll
-    for (int u = 0; u < (ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER; ++u) {
+    for (int u = 0; u < ATD_QPC; ++u) {
         const int qi = rank + u * ATD_CLUSTER;
-        res[u] = 0.f;
         if (qi < cnt && tid < DH) {
-            float mr[ATD_CLUSTER], lr[ATD_CLUSTER], ar[ATD_CLUSTER];
+            float mx = -INFINITY;
 #pragma unroll
-            for (int r = 0; r < ATD_CLUSTER; ++r) {
-                mr[r] = ld_dsmem_f32(smem_u32(rm + qi), r);
-                lr[r] = ld_dsmem_f32(smem_u32(rl + qi), r);
-                ar[r] = ld_dsmem_f32(smem_u32(racc + qi * DH + tid), r);
-            }
-            float mx = mr[0];
-#pragma unroll
-            for (int r = 1; r < ATD_CLUSTER; ++r) mx = fmaxf(mx, mr[r]);
+            for (int r = 0; r < ATD_CLUSTER; ++r) mx = fmaxf(mx, inbox[((size_t)r * ATD_QPC + u) * (DH + 2) + DH]);
             float l = 0.f, o = 0.f;
 #pragma unroll
             for (int r = 0; r < ATD_CLUSTER; ++r) {
-                const float f = mr[r] > -INFINITY ? expf(mr[r] - mx) : 0.f;
-                l = fmaf(lr[r], f, l);
-                o = fmaf(ar[r], f, o);
+                const float* st = inbox + ((size_t)r * ATD_QPC + u) * (DH + 2);
+                const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
+                l = fmaf(st[DH + 1], f, l);
+                o = fmaf(st[tid], f, o);
             }
-            res[u] = o / l;
+            static_cast<bf16*>(a.out)[(size_t)(row0 + qi) * a.ldo + h * DH + tid] = __float2bfloat16_rn(o / l);
         }
     }
-    cluster_arrive();   // done reading the peers' states
-#pragma unroll
-    for (int u = 0; u < (ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER; ++u) {
-        const int qi = rank + u * ATD_CLUSTER;
-        if (qi < cnt && tid < DH) static_cast<bf16*>(a.out)[(size_t)(row0 + qi) * a.ldo + h * DH + tid] = __float2bfloat16_rn(res[u]);
-    }
     if (tid == 0) TC_PROBE(6);
-    cluster_wait();   // nobody leaves while its state may still be read
-    if (tid == 0) TC_PROBE(7);
 }
 
 }  // namespace tandem

@@ -4,8 +4,9 @@
 //                          per tile on the TMEM lanes), the token rows are the B operand (16..64 columns).
 //                          The job is streaming W once from HBM: every CTA owns one (tile, K-slice) unit so
 //                          that all SMs pull weights, tiles arrive by TMA through a ring of stages, and the
-//                          K-slices of a tile sit in one thread-block cluster and are summed in slice order
-//                          through distributed shared memory.
+//                          K-slices of a tile sit in one thread-block cluster: each CTA sends its partial
+//                          sums to the CTA that finishes those columns (remote shared-memory stores), which
+//                          adds them in slice order.
 //                          The token rows are written into the B stages by the CTA's own threads, which is
 //                          where the LayerNorm (or the fp32 -> bf16 cast) of the residual stream is fused.
 //                          The weight loads are issued before the kernel waits for its predecessor in the
@@ -45,11 +46,12 @@ struct TcDecodeArgs {
 
 constexpr int TCD_THREADS = 192;   // warps 0-3: B operand + epilogue; warp 4: TMA; warp 5: TMEM + MMA issue
 template <int NB> struct TcdCfg {
-    static constexpr int STAGES = NB <= 32 ? 5 : 4;
+    static constexpr int STAGES = NB <= 16 ? 5 : (NB <= 32 ? 4 : 3);   // two CTAs fit on an SM
     static constexpr int A_BYTES = 128 * 128;       // 128 weight rows x 64 bf16
     static constexpr int B_BYTES = NB * 128;        // NB token rows x 64 bf16
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024
+    static constexpr int INBOX_BYTES = NB * 128 * 4;   // the K-slices' partial sums for this CTA's share of the columns
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + INBOX_BYTES + 1024;   // + slack to align the ring to 1024
     static constexpr int TMEM_COLS = NB <= 32 ? 32 : 64;
 };
 
@@ -96,6 +98,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     // LayerNorm rows short enough to sit in registers (8 float4 per lane) and a K-slice that fits the ring
     // without reuse: the B operand is then written straight from the registers that gave the statistics.
     const bool ln_regs = PRO == PRO_LN && K4 <= 256 && nkb <= C::STAGES;
+    float hres[EPI == EPI_RESID ? NB : 1];   // EPI_RESID: the residual values this thread's outputs are added to
     TC_PROBE_INIT(100 + PRO * 10 + EPI);
 
     if (warp == 5) {
@@ -161,10 +164,10 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             TC_PROBE(4);
         }
         __syncwarp();
-    } else if (ln_regs) {
-        // ---- warps 0-3, short LayerNorm rows: one pass over x.  Lane L holds the row's float4 number L + 32u in
-        // t[u], i.e. K-block 2u + (L >= 16), 16-byte chunk (L & 15) / 2, half L & 1. ----
-        float4 gq[C::STAGES], bq[C::STAGES];   // gain / bias of this lane's slot in each of the CTA's K-blocks
+    } else {
+    // ---- warps 0-3: token rows into the B stages (then the epilogue) ----
+    float4 gq[C::STAGES], bq[C::STAGES];   // register path: gain / bias of this lane's slot in each of the CTA's K-blocks
+    if (ln_regs) {
 #pragma unroll
         for (int i = 0; i < C::STAGES; ++i) {
             const int k4 = ((kb0 + i) >> 1) * 32 + lane;
@@ -172,8 +175,30 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             gq[i] = mine ? __ldg(reinterpret_cast<const float4*>(a.ln_g) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
             bq[i] = mine ? __ldg(reinterpret_cast<const float4*>(a.ln_b) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        pdl_wait();   // x comes from earlier kernels; gains and biases above are parameters
-        if (tid == 0) TC_PROBE(5);
+    }
+    pdl_wait();   // x, and everything the epilogue touches, comes from earlier kernels; gains and biases are parameters
+    if (tid == 0) TC_PROBE(5);
+    if (EPI == EPI_RESID) {
+        // the residual-stream values this thread will add to: fetched now, off the critical path
+        const float* hp = static_cast<const float*>(a.e.out);
+        if (S == 1) {
+            const int nl = n_local0 + tid;
+#pragma unroll
+            for (int j = 0; j < NB; ++j)
+                hres[j] = (j < a.rows && nl < a.seg_rows) ? __ldcg(hp + (size_t)j * a.e.ldo + seg * a.seg_rows + nl) : 0.f;
+        } else {
+            const int CW = 128 / S;
+            const int nl = n_local0 + sp * CW + (tid & (CW - 1));
+#pragma unroll
+            for (int it = 0; it < NB / 2; ++it) {
+                const int j = tid / CW + it * S;
+                hres[it] = (j < a.rows && nl < a.seg_rows) ? __ldcg(hp + (size_t)j * a.e.ldo + seg * a.seg_rows + nl) : 0.f;
+            }
+        }
+    }
+    if (ln_regs) {
+        // short LayerNorm rows: one pass over x.  Lane L holds the row's float4 number L + 32u in
+        // t[u], i.e. K-block 2u + (L >= 16), 16-byte chunk (L & 15) / 2, half L & 1.
         for (int r = warp; r < a.rows; r += 4) {
             const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx);
             float4 t[8];
@@ -221,9 +246,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             for (int i = 0; i < nkb; ++i) mbar_arrive(smem_u32(&s_full[i]));
         if (tid == 0) TC_PROBE(6);
     } else {
-        // ---- warps 0-3, general case: statistics (LayerNorm), then the K-blocks one by one ----
-        pdl_wait();   // x (and everything the epilogue touches) comes from earlier kernels
-        if (tid == 0) TC_PROBE(5);
+        // general case: statistics (LayerNorm), then the K-blocks a ring's worth at a time
         if (PRO == PRO_LN) {
             for (int r = warp; r < a.rows; r += 4) {   // one warp per row, fixed lane-strided order
                 const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx);
@@ -321,6 +344,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         }
         if (tid == 0) TC_PROBE(6);
     }
+    }
 
     // ---- epilogue: warps 0-3 own TMEM lanes 32 * warp .. +31 = output features of the tile ----
     float v[NB];
@@ -369,6 +393,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                     a.amax_val[(size_t)tid * a.amax_stride + tile] = bv;
                     a.amax_idx[(size_t)tid * a.amax_stride + tile] = bi;
                 }
+            } else if (EPI == EPI_RESID) {
+                float* out = static_cast<float*>(a.e.out);
+#pragma unroll
+                for (int j = 0; j < NB; ++j)
+                    if (j < a.rows && valid) out[(size_t)j * a.e.ldo + n] = hres[j] + v[j];
             } else {
 #pragma unroll
                 for (int j = 0; j < NB; ++j)
@@ -376,48 +405,39 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             }
         }
     } else {
-        // The cluster's CTAs hold the K-slices of one tile.  Each parks its partial tile in its own shared memory
-        // (the ring is free: every MMA has completed), then CTA `sp` sums columns [sp*128/S, (sp+1)*128/S) over
-        // the slices in slice order, reading the other CTAs' shared memory, and runs the epilogue for them.
-        float* red = reinterpret_cast<float*>(ring);   // [NB][128]
+        // The cluster's CTAs hold the K-slices of one tile, and CTA `r` finishes columns [r*128/S, (r+1)*128/S).
+        // Every CTA sends each column's partial sums to the inbox of the CTA that finishes it (remote shared-memory
+        // stores), one cluster barrier makes them visible, and each CTA sums its inbox in slice order.  Nobody
+        // touches a peer's shared memory after the barrier, so CTAs may leave as they finish.
+        const int CW = 128 / S;
+        const uint32_t inbox0 = ring0 + C::STAGES * C::STAGE_BYTES;           // [S][NB][CW] fp32
         if (warp < 4) {
+            const int dst = tl / CW, cw = tl & (CW - 1);
 #pragma unroll
             for (int j = 0; j < NB; ++j)
-                if (j < a.rows) red[j * 128 + tl] = v[j];
+                if (j < a.rows) st_dsmem_f32(inbox0 + ((sp * NB + j) * CW + cw) * 4, dst, v[j]);
         }
         cluster_sync_all();
         if (tid == 0) TC_PROBE(9);
         if (warp < 4 && EPI != EPI_ARGMAX) {
-            const int CW = 128 / S;                       // columns this CTA finishes
-            const int col = sp * CW + (tid & (CW - 1));
-            const int n_local = n_local0 + col;
+            const float* inbox = reinterpret_cast<const float*>(ring + C::STAGES * C::STAGE_BYTES);
+            const int cw = tid & (CW - 1);
+            const int n_local = n_local0 + sp * CW + cw;
             const bool valid = n_local < a.seg_rows;
             const int n = seg * a.seg_rows + n_local;
-            const uint32_t red0 = ring0 + col * 4;
-            float accs[NB / 2];                            // 128 / CW = S row groups: rows tid / CW, + S, ...
 #pragma unroll
-            for (int it = 0; it < NB / 2; ++it) {
+            for (int it = 0; it < NB / 2; ++it) {       // 128 / CW = S row groups: rows tid / CW, + S, ...
                 const int j = tid / CW + it * S;
-                accs[it] = 0.f;
-                if (j < a.rows) {
-                    float part[8];
+                if (j < a.rows && valid) {
+                    float acc = 0.f;
 #pragma unroll
-                    for (int ss = 0; ss < 8; ++ss) part[ss] = ss < S ? ld_dsmem_f32(red0 + j * 512, ss) : 0.f;
-#pragma unroll
-                    for (int ss = 0; ss < 8; ++ss) if (ss < S) accs[it] += part[ss];   // slice order
+                    for (int ss = 0; ss < 8; ++ss) if (ss < S) acc += inbox[(ss * NB + j) * CW + cw];   // slice order
+                    if (EPI == EPI_RESID) static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = hres[it] + acc;
+                    else epilogue<bf16, EPI>(a.e, j, n, acc);
                 }
             }
-            cluster_arrive();   // done reading the peers' shared memory
-            if (tid == 0) TC_PROBE(10);
-#pragma unroll
-            for (int it = 0; it < NB / 2; ++it) {
-                const int j = tid / CW + it * S;
-                if (j < a.rows && valid) epilogue<bf16, EPI>(a.e, j, n, accs[it]);
-            }
-        } else {
-            cluster_arrive();
         }
-        cluster_wait();   // nobody leaves while its shared memory may still be read
+        if (tid == 0) TC_PROBE(10);
     }
     if (tid == 0) TC_PROBE(11);
     tc_fence_before_sync();

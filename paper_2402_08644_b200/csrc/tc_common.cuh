@@ -155,6 +155,13 @@ __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_smem_addr, int rank
     return v;
 }
 
+// Writes a float to the same shared-memory offset in the cluster's CTA number `rank`.
+__device__ __forceinline__ void st_dsmem_f32(uint32_t local_smem_addr, int rank, float v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_smem_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
 // Named barrier among a subset of the CTA's warps.
 __device__ __forceinline__ void bar_sync(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 
