@@ -197,10 +197,12 @@ TANDEM_API int64_t tandem_launch_count(tandem_ctx* ctx);
  *   q, out           [batch][n_heads][d_head]
  *   k_derived, v_derived  [batch][n_heads][derived_len][d_head]
  *   k_own, v_own     [batch][n_heads][own_len][d_head]
- *   scratch          split-K partial results and merge tickets, at least tandem_decode_attention_scratch_bytes(...)
- * d_head in {32, 64, 128}.  The context is cut into fixed chunks by absolute position; each chunk yields
- * (max, sum, weighted values), and the CTA of a (sequence, head) that finishes last merges the chunks in
- * position order. */
+ *   scratch          work space of at least tandem_decode_attention_scratch_bytes(...) bytes (the kernel reads
+ *                    every row's sequence and position from two int arrays that the call fills there)
+ * d_head in {32, 64, 128}; batch <= 65535.  The context is cut into 128-position chunks by absolute position.
+ * A cluster of eight CTAs serves one (sequence, head): CTA r takes chunks r, r + 8, ..., each warp keeps an
+ * online-softmax state for its share of the positions, and the states are merged in a fixed order through
+ * the cluster's shared memory, so a query's result does not depend on what else is in the launch. */
 TANDEM_API size_t tandem_decode_attention_scratch_bytes(int32_t batch, int32_t n_heads, int32_t d_head,
                                              int32_t derived_len, int32_t own_len);
 TANDEM_API tandem_status tandem_decode_attention(const void* q, const void* k_derived, const void* v_derived,
@@ -215,23 +217,23 @@ TANDEM_API tandem_status tandem_decode_attention(const void* q, const void* k_de
  * library's hook, in a process whose memory pool is owned by a framework that hands out no raw buffers,
  * or in a service that must not touch the allocator after start-up because an allocation can block on,
  * or synchronise with, other work on the device.  Such a caller still passes its inputs and its output,
- * but the split-K partial results go to a buffer built into the library: a file-scope __device__ array of
- * TANDEM_STATIC_SCRATCH_BYTES that every GPU loading the library holds until the process exits.
+ * but the kernel's work space (the per-row sequence / position arrays) is a buffer built into the library:
+ * a file-scope __device__ array of TANDEM_STATIC_SCRATCH_BYTES that every GPU loading the library holds
+ * until the process exits.
  *
  * Same arguments, layouts and results as tandem_decode_attention, minus scratch.  Differences:
- *  - Shapes whose partial results need more than TANDEM_STATIC_SCRATCH_BYTES
- *    (tandem_decode_attention_scratch_bytes tells) are refused with TANDEM_ERR_CAPACITY before anything is
- *    launched; tandem_last_cuda_error() then holds a sentence with both sizes.
+ *  - Batches whose work space exceeds TANDEM_STATIC_SCRATCH_BYTES (tandem_decode_attention_scratch_bytes
+ *    tells; 8 bytes per sequence, so 8192 sequences fit) are refused with TANDEM_ERR_CAPACITY before anything
+ *    is launched; tandem_last_cuda_error() then holds a sentence with both sizes.
  *  - The first call on each device looks up the device address of the built-in buffer (with that device
  *    current - make the device that owns the tensors current before calling).  Make that first call before
  *    any stream capture is begun on the device.  Later calls only launch.
  *  - The call itself allocates nothing on host or device and frees nothing.
- *  - All calls on a device share the one buffer, and it keeps whatever the previous call left there.  The
- *    kernels overwrite every partial result they later read and each call clears the merge tickets itself
- *    (a memset on the stream), so the caller clears nothing between calls; but
- *    two calls that can overlap on the GPU (different streams, or one stream and a graph) race on it and
- *    give wrong results.  Keep calls to this entry point on one stream, or order them with events. */
-#define TANDEM_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+ *  - All calls on a device share the one buffer, and it keeps whatever the previous call left there.  Each call
+ *    rewrites the part it reads, so the caller clears nothing between calls; but two calls that can overlap
+ *    on the GPU (different streams, or one stream and a graph) race on it and give wrong results.  Keep calls
+ *    to this entry point on one stream, or order them with events. */
+#define TANDEM_STATIC_SCRATCH_BYTES (64 * 1024)
 TANDEM_API tandem_status tandem_decode_attention_static(const void* q, const void* k_derived, const void* v_derived,
                                                         const void* k_own, const void* v_own, void* out,
                                                         int32_t batch, int32_t n_heads, int32_t d_head,

@@ -287,13 +287,13 @@ def tandem_decode_attention(q, k_derived, v_derived, k_own, v_own, out=None, scr
     return out
 
 
-STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+STATIC_SCRATCH_BYTES = 64 * 1024
 
 
 def tandem_decode_attention_static(q, k_derived, v_derived, k_own, v_own, out):
     """tandem_decode_attention without a scratch argument, for callers that may not allocate device memory:
-    the partial results live in a buffer built into the library (at most STATIC_SCRATCH_BYTES are needed, else
-    TandemError with status CAPACITY).  `out` is required, so this wrapper allocates nothing either.  Calls
+    the kernel's work space (8 bytes per sequence) is a buffer built into the library (at most STATIC_SCRATCH_BYTES
+    are needed, else TandemError with status CAPACITY).  `out` is required, so this wrapper allocates nothing either.  Calls
     share that buffer: keep them on one stream.  Make the first call on a device outside any stream capture."""
     import torch
     lib = load_library()

@@ -231,31 +231,35 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Decode attention, bf16, built for short dependent chains: a cluster of ATD_CLUSTER CTAs serves one
-// (sequence, head).  CTA `rank` takes the 128-position chunks rank, rank + 8, ... (anchored at absolute
-// position 0) through a cp.async ring, keeps an online-softmax state per query, and the cluster merges
-// its eight states in rank order through distributed shared memory: no global scratch, no second kernel.
-// The probabilities use the fast exponential (2^x hardware approximation), well inside the bf16 tolerance.
-// DH / 8 threads share a key (16 bytes each); a query's arithmetic does not depend on the other queries.
+// Decode attention, bf16, built for short dependent chains and for streaming: a cluster of ATD_CLUSTER CTAs
+// serves one (sequence, head).  CTA `rank` takes the 128-position chunks rank, rank + 8, ... (anchored at
+// absolute position 0); inside a chunk warp w owns positions 16w .. 16w+15.  Every warp runs on its own: it
+// fetches its rows through a private cp.async ring, keeps an online-softmax state per query in registers and
+// never waits for another warp until the end, where the CTA folds its warps' states in warp order, sends the
+// result to the CTA that finishes the query (remote shared-memory stores), and that CTA merges the eight
+// states in rank order.  No global scratch, no second kernel.  DH / 8 lanes share a key (16 bytes each); a
+// query's arithmetic does not depend on the other queries.  The probabilities use the fast exponential
+// (2^x hardware approximation), well inside the bf16 tolerance.
 // ---------------------------------------------------------------------------------------------------
 constexpr int ATD_THREADS = 256;
 constexpr int ATD_WARPS = ATD_THREADS / 32;
 constexpr int ATD_CLUSTER = 8;
 constexpr int ATD_QPC = (ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER;   // queries a CTA finishes at most
+constexpr int ATD_WROWS = ATT_CH / ATD_WARPS;                       // positions of a chunk per warp (16)
 
 template <int DH> struct AtdCfg {
-    static constexpr int TPK = DH / 8;              // threads per key
-    static constexpr int KPP = ATD_THREADS / TPK;   // keys per pass
-    static constexpr int PPC = ATT_CH / KPP;        // passes per chunk
+    static constexpr int TPK = DH / 8;               // lanes per key
+    static constexpr int KPW = 32 / TPK;             // keys per warp pass
+    static constexpr int PPW = ATD_WROWS / KPW;      // passes per chunk
     static constexpr int STAGES = DH <= 64 ? 3 : 2;
-    static constexpr int TILE_ELEMS = ATT_CH * DH;  // one chunk of keys (or values)
+    static constexpr int TILE_ELEMS = ATD_WROWS * DH;   // a warp's keys (or values) of one chunk
     static constexpr int STAGE_ELEMS = 2 * TILE_ELEMS;
+    static constexpr int UNITS = ATD_WROWS * TPK / 32;  // 16-byte units per lane per tile
 };
 template <int DH, int QG>
 constexpr size_t attn_decode_smem_bytes() {
-    return (size_t)AtdCfg<DH>::STAGES * AtdCfg<DH>::STAGE_ELEMS * sizeof(bf16) +
-           sizeof(float) * ((size_t)2 * ATT_NQ * DH + 2 * ATT_NQ + 2 * ATD_WARPS * QG + (size_t)ATD_WARPS * QG * DH +
-                            (size_t)ATD_CLUSTER * ATD_QPC * (DH + 2));
+    return (size_t)ATD_WARPS * AtdCfg<DH>::STAGES * AtdCfg<DH>::STAGE_ELEMS * sizeof(bf16) +
+           sizeof(float) * ((size_t)ATT_NQ * DH + (size_t)ATD_WARPS * QG * (DH + 2) + (size_t)ATD_CLUSTER * ATD_QPC * (DH + 2));
 }
 
 // grid: (ATD_CLUSTER, heads, sequences) in clusters of ATD_CLUSTER along x; block: ATD_THREADS.
@@ -264,24 +268,20 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     using C = AtdCfg<DH>;
     constexpr int NW = ATD_WARPS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    bf16* ring = reinterpret_cast<bf16*>(smem_raw);
-    float* qs = reinterpret_cast<float*>(ring + (size_t)C::STAGES * C::STAGE_ELEMS);   // [ATT_NQ][DH]
-    float* racc = qs + ATT_NQ * DH;       // running weighted values [ATT_NQ][DH]
-    float* rm = racc + ATT_NQ * DH;       // running max [ATT_NQ]
-    float* rl = rm + ATT_NQ;              // running sum [ATT_NQ]
-    float* red = rl + ATT_NQ;             // [2][NW][QG] per-warp chunk max / sum
-    float* pv = red + 2 * NW * QG;        // [NW][QG][DH] per-warp weighted values
-    float* inbox = pv + NW * QG * DH;     // [ATD_CLUSTER][ATD_QPC][DH + 2] states sent by the cluster's CTAs
+    bf16* ring_all = reinterpret_cast<bf16*>(smem_raw);
+    float* qs = reinterpret_cast<float*>(ring_all + (size_t)NW * C::STAGES * C::STAGE_ELEMS);   // [ATT_NQ][DH]
+    float* wst = qs + ATT_NQ * DH;                 // [NW][QG][DH + 2] the warps' states of the current query group
+    float* inbox = wst + NW * QG * (DH + 2);       // [ATD_CLUSTER][ATD_QPC][DH + 2] states sent by the cluster's CTAs
     TC_PROBE_INIT(210);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = blockIdx.x, h = blockIdx.y, g = blockIdx.z;
-    const int part = tid % C::TPK, kslot = tid / C::TPK;
+    const int part = lane % C::TPK, kslot = lane / C::TPK;
+    bf16* ring = ring_all + (size_t)warp * C::STAGES * C::STAGE_ELEMS;
     pdl_launch_dependents();
     pdl_wait();   // queries and the newest keys/values come from earlier kernels
     if (tid == 0) TC_PROBE(1);
     const int cnt = a.nq, row0 = g * a.nq;
-    // queries first (their address needs nothing else), then the position that fixes the chunks
     const bf16* qg = static_cast<const bf16*>(a.q);
     for (int i = tid; i < cnt * DH; i += ATD_THREADS) {
         const int qi = i / DH, el = i - qi * DH;
@@ -296,62 +296,69 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     const size_t head_base2 = ((size_t)b * a.n_heads + h) * a.t_max2;
     const int split = a.k2 ? a.split : INT_MAX;
 
+    // this warp's rows of its CTA's it-th chunk into stage it % STAGES
     auto issue = [&](int it) {
-        const int t0 = (rank + it * ATD_CLUSTER) * ATT_CH;
-        const int nt = min(ATT_CH, pos_last + 1 - t0);
+        const int t0 = (rank + it * ATD_CLUSTER) * ATT_CH + warp * ATD_WROWS;
         bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
         bf16* vs = ks + C::TILE_ELEMS;
-        for (int i = tid; i < nt * C::TPK; i += ATD_THREADS) {
-            const int t = i / C::TPK, v = i - t * C::TPK;
+#pragma unroll
+        for (int u = 0; u < C::UNITS; ++u) {
+            const int idx = lane + 32 * u;
+            const int t = idx / C::TPK, v = idx - t * C::TPK;
             const int ta = t0 + t;
-            const bf16 *kg, *vg;
-            if (ta < split) {
-                kg = static_cast<const bf16*>(a.kcache) + (head_base + ta) * DH;
-                vg = static_cast<const bf16*>(a.vcache) + (head_base + ta) * DH;
-            } else {
-                kg = static_cast<const bf16*>(a.k2) + (head_base2 + (ta - split)) * DH;
-                vg = static_cast<const bf16*>(a.v2) + (head_base2 + (ta - split)) * DH;
+            if (ta <= pos_last) {
+                const bf16 *kg, *vg;
+                if (ta < split) {
+                    kg = static_cast<const bf16*>(a.kcache) + (head_base + ta) * DH;
+                    vg = static_cast<const bf16*>(a.vcache) + (head_base + ta) * DH;
+                } else {
+                    kg = static_cast<const bf16*>(a.k2) + (head_base2 + (ta - split)) * DH;
+                    vg = static_cast<const bf16*>(a.v2) + (head_base2 + (ta - split)) * DH;
+                }
+                cp_async16(ks + idx * 8, kg + v * 8);
+                cp_async16(vs + idx * 8, vg + v * 8);
+            } else {   // past the last query: zeros, so that a zero weight times them stays zero
+                *reinterpret_cast<uint4*>(ks + idx * 8) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(vs + idx * 8) = make_uint4(0u, 0u, 0u, 0u);
             }
-            cp_async16(ks + t * DH + v * 8, kg + v * 8);
-            cp_async16(vs + t * DH + v * 8, vg + v * 8);
-        }
-        // positions past the last query: zeros, so that a zero weight times them stays zero
-        for (int i = nt * C::TPK + tid; i < ATT_CH * C::TPK; i += ATD_THREADS) {
-            *reinterpret_cast<uint4*>(ks + i * 8) = make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(vs + i * 8) = make_uint4(0u, 0u, 0u, 0u);
         }
     };
-#pragma unroll
-    for (int it = 0; it < C::STAGES - 1; ++it) {
-        if (it < n_mine) issue(it);
-        cp_async_commit();
-    }
-    for (int i = tid; i < ATT_NQ * DH; i += ATD_THREADS) racc[i] = 0.f;
-    if (tid < ATT_NQ) { rm[tid] = -INFINITY; rl[tid] = 0.f; }
+    __syncthreads();   // qs written
     if (tid == 0) TC_PROBE(2);
 
-    for (int it = 0; it < n_mine; ++it) {
-        if (it + C::STAGES - 1 < n_mine) issue(it + C::STAGES - 1);
-        cp_async_commit();
-        asm volatile("cp.async.wait_group %0;" ::"n"(C::STAGES - 1) : "memory");
-        __syncthreads();
-        if (tid == 0 && it == 0) TC_PROBE(3);
-        const int t0 = (rank + it * ATD_CLUSTER) * ATT_CH;
-        const bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
-        const bf16* vs = ks + C::TILE_ELEMS;
-        for (int q0 = 0; q0 < cnt; q0 += QG) {
-            float qreg[QG][8];
+    for (int q0 = 0; q0 < cnt; q0 += QG) {
 #pragma unroll
-            for (int qi = 0; qi < QG; ++qi)
+        for (int it = 0; it < C::STAGES - 1; ++it) {
+            if (it < n_mine) issue(it);
+            cp_async_commit();
+        }
+        float qreg[QG][8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) qreg[qi][j] = (q0 + qi < cnt) ? qs[(q0 + qi) * DH + part * 8 + j] : 0.f;
-            float sc[QG][C::PPC];
-            float mloc[QG];
+        for (int qi = 0; qi < QG; ++qi)
 #pragma unroll
-            for (int qi = 0; qi < QG; ++qi) mloc[qi] = -INFINITY;
+            for (int j = 0; j < 8; ++j) qreg[qi][j] = (q0 + qi < cnt) ? qs[(q0 + qi) * DH + part * 8 + j] : 0.f;
+        float m[QG], l[QG], acc[QG][8];
 #pragma unroll
-            for (int p = 0; p < C::PPC; ++p) {
-                const int key = p * C::KPP + kslot;
+        for (int qi = 0; qi < QG; ++qi) {
+            m[qi] = -INFINITY; l[qi] = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[qi][j] = 0.f;
+        }
+        for (int it = 0; it < n_mine; ++it) {
+            if (it + C::STAGES - 1 < n_mine) issue(it + C::STAGES - 1);
+            cp_async_commit();
+            asm volatile("cp.async.wait_group %0;" ::"n"(C::STAGES - 1) : "memory");
+            __syncwarp();
+            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(3);
+            const int t0 = (rank + it * ATD_CLUSTER) * ATT_CH + warp * ATD_WROWS;
+            const bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
+            const bf16* vs = ks + C::TILE_ELEMS;
+            float sc[QG][C::PPW], mc[QG];
+#pragma unroll
+            for (int qi = 0; qi < QG; ++qi) mc[qi] = -INFINITY;
+#pragma unroll
+            for (int p = 0; p < C::PPW; ++p) {
+                const int key = p * C::KPW + kslot;
                 float kf[8];
                 load_vec(ks + key * DH + part * 8, kf);
 #pragma unroll
@@ -363,39 +370,30 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
                     for (int o = 1; o < C::TPK; o <<= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
                     const bool live = (q0 + qi < cnt) && (t0 + key <= pos_first + q0 + qi);
                     sc[qi][p] = live ? d * a.scale : -INFINITY;
-                    mloc[qi] = fmaxf(mloc[qi], sc[qi][p]);
+                    mc[qi] = fmaxf(mc[qi], sc[qi][p]);
                 }
             }
 #pragma unroll
             for (int qi = 0; qi < QG; ++qi) {
 #pragma unroll
-                for (int o = C::TPK; o < 32; o <<= 1) mloc[qi] = fmaxf(mloc[qi], __shfl_xor_sync(0xffffffffu, mloc[qi], o));
-                if (lane == 0) red[warp * QG + qi] = mloc[qi];
-            }
-            __syncthreads();
-            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(8);
-            float acc[QG][8];
-#pragma unroll
-            for (int qi = 0; qi < QG; ++qi) {
-                float mc = red[qi];
-#pragma unroll
-                for (int w = 1; w < NW; ++w) mc = fmaxf(mc, red[w * QG + qi]);
+                for (int o = C::TPK; o < 32; o <<= 1) mc[qi] = fmaxf(mc[qi], __shfl_xor_sync(0xffffffffu, mc[qi], o));
+                const float mn = fmaxf(m[qi], mc[qi]);
+                const float f = m[qi] > -INFINITY ? __expf(m[qi] - mn) : 0.f;
+                m[qi] = mn;
                 float ls = 0.f;
 #pragma unroll
-                for (int p = 0; p < C::PPC; ++p) {
-                    const float pr = mc > -INFINITY ? __expf(sc[qi][p] - mc) : 0.f;
+                for (int p = 0; p < C::PPW; ++p) {
+                    const float pr = mn > -INFINITY ? __expf(sc[qi][p] - mn) : 0.f;
                     sc[qi][p] = pr;
                     ls += pr;
                 }
+                l[qi] = l[qi] * f + ls;   // this lane's keys only; the key slots are added up at the end
 #pragma unroll
-                for (int o = C::TPK; o < 32; o <<= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
-                if (lane == 0) red[NW * QG + warp * QG + qi] = ls;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc[qi][j] = 0.f;
+                for (int j = 0; j < 8; ++j) acc[qi][j] *= f;
             }
 #pragma unroll
-            for (int p = 0; p < C::PPC; ++p) {
-                const int key = p * C::KPP + kslot;
+            for (int p = 0; p < C::PPW; ++p) {
+                const int key = p * C::KPW + kslot;
                 float vf[8];
                 load_vec(vs + key * DH + part * 8, vf);
 #pragma unroll
@@ -403,60 +401,51 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) acc[qi][j] = fmaf(sc[qi][p], vf[j], acc[qi][j]);
             }
-#pragma unroll
-            for (int qi = 0; qi < QG; ++qi)
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-#pragma unroll
-                    for (int o = C::TPK; o < 32; o <<= 1) acc[qi][j] += __shfl_xor_sync(0xffffffffu, acc[qi][j], o);
-                    if (lane < C::TPK) pv[(warp * QG + qi) * DH + lane * 8 + j] = acc[qi][j];
-                }
-            __syncthreads();
-            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(9);
-            // fold the chunk into the running state: thread (query slot, element)
-            constexpr int FU = (QG * DH + ATD_THREADS - 1) / ATD_THREADS;
-            float m_new[FU], l_new[FU];
-#pragma unroll
-            for (int u = 0; u < FU; ++u) {
-                const int idx = tid + u * ATD_THREADS;
-                const int qi = idx / DH, e = idx - qi * DH;
-                m_new[u] = 0.f; l_new[u] = 0.f;
-                if (qi < QG && q0 + qi < cnt) {
-                    float mc = red[qi], lc = red[NW * QG + qi], oc = pv[qi * DH + e];
-#pragma unroll
-                    for (int w = 1; w < NW; ++w) {   // warp order
-                        mc = fmaxf(mc, red[w * QG + qi]);
-                        lc += red[NW * QG + w * QG + qi];
-                        oc += pv[(w * QG + qi) * DH + e];
-                    }
-                    const float mo = rm[q0 + qi], lo = rl[q0 + qi];
-                    const float mn = fmaxf(mo, mc);
-                    const float fo = mo > -INFINITY ? __expf(mo - mn) : 0.f;
-                    const float fn = mc > -INFINITY ? __expf(mc - mn) : 0.f;
-                    racc[(q0 + qi) * DH + e] = racc[(q0 + qi) * DH + e] * fo + oc * fn;
-                    m_new[u] = mn; l_new[u] = lo * fo + lc * fn;
-                }
-            }
-            __syncthreads();
-#pragma unroll
-            for (int u = 0; u < FU; ++u) {
-                const int idx = tid + u * ATD_THREADS;
-                const int qi = idx / DH, e = idx - qi * DH;
-                if (e == 0 && qi < QG && q0 + qi < cnt) { rm[q0 + qi] = m_new[u]; rl[q0 + qi] = l_new[u]; }
-            }
-            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(10);
+            __syncwarp();   // the stage may be refilled by this warp's next issue
+            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(8);
         }
-        __syncthreads();   // the stage may be refilled, the state re-read
-    }
-    __syncthreads();       // a CTA without chunks comes straight from initialising its state
-    if (tid == 0) TC_PROBE(4);
-    // Query qi is finished by CTA qi % 8: every CTA sends it its state for that query (remote shared-memory stores),
-    // one cluster barrier makes the states visible, and the owner merges them in rank order.  Nobody touches a
-    // peer's shared memory after the barrier.
-    for (int i = tid; i < cnt * (DH + 2); i += ATD_THREADS) {
-        const int qi = i / (DH + 2), e = i - qi * (DH + 2);
-        const float val = e < DH ? racc[qi * DH + e] : (e == DH ? rm[qi] : rl[qi]);
-        st_dsmem_f32(smem_u32(inbox + ((size_t)rank * ATD_QPC + qi / ATD_CLUSTER) * (DH + 2) + e), qi % ATD_CLUSTER, val);
+        // the warp's state: add up its key slots (lanes that share `part`), lanes 0 .. TPK-1 publish it
+#pragma unroll
+        for (int qi = 0; qi < QG; ++qi) {
+#pragma unroll
+            for (int o = C::TPK; o < 32; o <<= 1) {
+                l[qi] += __shfl_xor_sync(0xffffffffu, l[qi], o);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[qi][j] += __shfl_xor_sync(0xffffffffu, acc[qi][j], o);
+            }
+            if (lane < C::TPK) {
+                float* st = wst + (size_t)(warp * QG + qi) * (DH + 2);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) st[lane * 8 + j] = acc[qi][j];
+                if (lane == 0) { st[DH] = m[qi]; st[DH + 1] = l[qi]; }
+            }
+        }
+        __syncthreads();
+        if (tid == 0 && q0 == 0) TC_PROBE(4);
+        // fold the warps' states in warp order and send the CTA's state of query qi to CTA qi % 8
+        for (int i = tid; i < QG * (DH + 2); i += ATD_THREADS) {
+            const int qi = i / (DH + 2), e = i - qi * (DH + 2);
+            const int qa = q0 + qi;
+            if (qa < cnt) {
+                float mx = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < NW; ++w) mx = fmaxf(mx, wst[(size_t)(w * QG + qi) * (DH + 2) + DH]);
+                float val;
+                if (e == DH) {
+                    val = mx;
+                } else {
+                    val = 0.f;
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) {
+                        const float* st = wst + (size_t)(w * QG + qi) * (DH + 2);
+                        const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
+                        val = fmaf(e < DH ? st[e] : st[DH + 1], f, val);
+                    }
+                }
+                st_dsmem_f32(smem_u32(inbox + ((size_t)rank * ATD_QPC + qa / ATD_CLUSTER) * (DH + 2) + e), qa % ATD_CLUSTER, val);
+            }
+        }
+        __syncthreads();   // wst is rewritten by the next query group
     }
     cluster_sync_all();
     if (tid == 0) TC_PROBE(5);

@@ -134,6 +134,76 @@ __global__ void __launch_bounds__(128) layernorm_kernel(const float* __restrict_
         out[(size_t)blockIdx.x * d + i] = from_float<T>((xr[i] - mu) * rstd * gain[i] + bias[i]);
 }
 
+// Decode-path LayerNorm of fp32 rows to bf16 for the tensor-core GEMMs: the row sits in registers between the
+// passes (up to 4096 elements), loads and stores are 16 / 8 bytes wide.  grid: rows; block: 128; d % 4 == 0.
+__global__ void __launch_bounds__(128) layernorm_rows_bf16_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+                                                                  const float* __restrict__ bias, bf16* __restrict__ out, int d) {
+    __shared__ float red[4];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int d4 = d >> 2;
+    const float4* xr = reinterpret_cast<const float4*>(x + (size_t)blockIdx.x * d);
+    uint2* orow = reinterpret_cast<uint2*>(out + (size_t)blockIdx.x * d);
+    if (d4 <= 8 * 128) {
+        float4 t[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) t[u] = (threadIdx.x + 128 * u < d4) ? __ldcg(xr + threadIdx.x + 128 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float s = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += (t[u].x + t[u].y) + (t[u].z + t[u].w);
+        const float mu = block_sum_128(s, red) / d;
+        float q = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (threadIdx.x + 128 * u < d4) {
+                const float d0 = t[u].x - mu, d1 = t[u].y - mu, d2 = t[u].z - mu, d3 = t[u].w - mu;
+                q = fmaf(d0, d0, q); q = fmaf(d1, d1, q); q = fmaf(d2, d2, q); q = fmaf(d3, d3, q);
+            }
+        }
+        const float rs = 1.0f / sqrtf(block_sum_128(q, red) / d + 1e-5f);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int k4 = threadIdx.x + 128 * u;
+            if (k4 < d4) {
+                const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + k4), b = __ldg(reinterpret_cast<const float4*>(bias) + k4);
+                const __nv_bfloat162 lo = __floats2bfloat162_rn((t[u].x - mu) * rs * g.x + b.x, (t[u].y - mu) * rs * g.y + b.y);
+                const __nv_bfloat162 hi = __floats2bfloat162_rn((t[u].z - mu) * rs * g.z + b.z, (t[u].w - mu) * rs * g.w + b.w);
+                orow[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+            }
+        }
+    } else {
+        float s = 0.f;
+        for (int k4 = threadIdx.x; k4 < d4; k4 += 128) { const float4 t = __ldcg(xr + k4); s += (t.x + t.y) + (t.z + t.w); }
+        const float mu = block_sum_128(s, red) / d;
+        float q = 0.f;
+        for (int k4 = threadIdx.x; k4 < d4; k4 += 128) {
+            const float4 t = __ldcg(xr + k4);
+            const float d0 = t.x - mu, d1 = t.y - mu, d2 = t.z - mu, d3 = t.w - mu;
+            q = fmaf(d0, d0, q); q = fmaf(d1, d1, q); q = fmaf(d2, d2, q); q = fmaf(d3, d3, q);
+        }
+        const float rs = 1.0f / sqrtf(block_sum_128(q, red) / d + 1e-5f);
+        for (int k4 = threadIdx.x; k4 < d4; k4 += 128) {
+            const float4 t = __ldcg(xr + k4);
+            const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + k4), b = __ldg(reinterpret_cast<const float4*>(bias) + k4);
+            const __nv_bfloat162 lo = __floats2bfloat162_rn((t.x - mu) * rs * g.x + b.x, (t.y - mu) * rs * g.y + b.y);
+            const __nv_bfloat162 hi = __floats2bfloat162_rn((t.z - mu) * rs * g.z + b.z, (t.w - mu) * rs * g.w + b.w);
+            orow[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+        }
+    }
+}
+
+// fp32 rows to bf16, 4 elements per thread; n % 4 == 0.  Decode path (waits for its predecessor in the stream).
+__global__ void cast_rows_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ out, size_t n4) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n4) {
+        const float4 t = __ldcg(reinterpret_cast<const float4*>(x) + i);
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(t.x, t.y), hi = __floats2bfloat162_rn(t.z, t.w);
+        reinterpret_cast<uint2*>(out)[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    }
+}
+
 template <typename T>
 __global__ void cast_rows_kernel(const float* __restrict__ x, T* __restrict__ out, size_t n) {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;

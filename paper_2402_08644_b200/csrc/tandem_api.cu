@@ -685,20 +685,43 @@ void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r
               (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model);
 }
 
+// Whether LayerNorm (or the fp32 -> bf16 cast) is fused into the GEMM's operand load.  Fused, every CTA of the
+// GEMM normalises the rows it needs itself: right for a couple of sequences and short rows, wasteful beyond.
+// The choice depends on the batch and the model only, never on the number of rows, so a block pass and a
+// one-row pass take the same route.
+bool tc_fused_prologue(const tandem_ctx& c, int K) { return c.batch <= 2 && K <= 1024; }
+
+// y = LayerNorm(h) W^T with the given epilogue; h fp32 [rows][K].
+template <int EPI>
+void tc_ln_gemm(tandem_ctx& c, const float* h, const void* ln_g, const void* ln_b, int rows, const TcW& w, bool stream_w,
+                const EpiArgs& e, float* amax_val = nullptr, int* amax_idx = nullptr, int amax_stride = 0) {
+    const TcScratch sc = tc_scratch(c);
+    if (tc_fused_prologue(c, w.K)) {
+        launch_tc_decode<PRO_LN, EPI>(c, sc, h, w.K, ln_g, ln_b, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
+        return;
+    }
+    bf16* a = at<bf16>(c, c.lay.a);
+    {
+        ProfScope ps(c, PC_LAYERNORM, (double)rows * w.K * 6.0);
+        launch_ex(c, true, 1, layernorm_rows_bf16_kernel, dim3(rows), dim3(128), 0, h, static_cast<const float*>(ln_g),
+                  static_cast<const float*>(ln_b), a, w.K);
+    }
+    launch_tc_decode<PRO_BF16, EPI>(c, sc, a, w.K, nullptr, nullptr, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
+}
+
 void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r, bool stream_w) {
     const int d = m.d.d_model, dff = m.d.d_ff;
     bf16* q = at<bf16>(c, c.lay.q);
     bf16* o = at<bf16>(c, c.lay.o);
     bf16* f = at<bf16>(c, c.lay.f);
     const TcScratch sc = tc_scratch(c);
-    launch_tc_decode<PRO_LN, EPI_QKV>(c, sc, h, d, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), r.M,
-                                      tcw(c, wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, d), stream_w,
-                                      epi_cache<bf16>(c, m, l, q));
+    tc_ln_gemm<EPI_QKV>(c, h, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), r.M,
+                        tcw(c, wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, d), stream_w, epi_cache<bf16>(c, m, l, q));
     attention<bf16>(c, m, l, q, o, r);
     launch_tc_decode<PRO_BF16, EPI_RESID>(c, sc, o, d, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_WO), -1, -1, d, d), stream_w,
                                           epi_plain(h, d));
-    launch_tc_decode<PRO_LN, EPI_GELU>(c, sc, h, d, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), r.M,
-                                       tcw(c, wi_layer(m, l, W_W1), -1, -1, dff, d), stream_w, epi_plain(f, dff));
+    tc_ln_gemm<EPI_GELU>(c, h, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), r.M, tcw(c, wi_layer(m, l, W_W1), -1, -1, dff, d),
+                         stream_w, epi_plain(f, dff));
     launch_tc_decode<PRO_BF16, EPI_RESID>(c, sc, f, dff, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_W2), -1, -1, d, dff), stream_w,
                                           epi_plain(h, d));
 }
@@ -706,9 +729,8 @@ void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows
 // Final LayerNorm + output head; leaves fp32 logits and the per-tile (max, index) pairs that the next kernel
 // (the next pass's row set-up, or the verify kernel) turns into token ids.
 void tc_head(tandem_ctx& c, const Model& m, float* h, const Rows& r, float* logits, size_t amax_val_off, size_t amax_idx_off, bool stream_w) {
-    launch_tc_decode<PRO_LN, EPI_ARGMAX>(c, tc_scratch(c), h, m.d.d_model, w_tail(c, m, 0), w_tail(c, m, 1), r.M,
-                                         tcw(c, wi_tail(m, 2), -1, -1, m.d.vocab, m.d.d_model), stream_w, epi_plain(logits, m.d.vocab),
-                                         at<float>(c, amax_val_off), at<int>(c, amax_idx_off), c.lay.vocab_tiles);
+    tc_ln_gemm<EPI_ARGMAX>(c, h, w_tail(c, m, 0), w_tail(c, m, 1), r.M, tcw(c, wi_tail(m, 2), -1, -1, m.d.vocab, m.d.d_model), stream_w,
+                           epi_plain(logits, m.d.vocab), at<float>(c, amax_val_off), at<int>(c, amax_idx_off), c.lay.vocab_tiles);
 }
 
 // FF_Tandem of the block's rows after n large layers (Eq. 2, first line) for every small layer fed from there,
@@ -718,21 +740,32 @@ void tc_project_after(tandem_ctx& c, int n_large_layers_done, const Rows& r) {
     const TcScratch sc = tc_scratch(c);
     float* h = at<float>(c, c.lay.h_large);
     float* yhat = at<float>(c, c.lay.yhat);
+    bool any = false;
+    for (int j = 0; j < c.small.d.n_layers; ++j) any |= (c.layer_map[j] == n_large_layers_done);
+    if (!any) return;
+    const bool fused = tc_fused_prologue(c, dL);
+    bf16* xb = at<bf16>(c, c.lay.xb);
+    if (!fused) {   // one bf16 copy of the rows serves every small layer fed from here
+        const size_t n4 = (size_t)r.M * dL / 4;
+        ProfScope ps(c, PC_ROWS, (double)n4 * 24.0);
+        launch_ex(c, true, 1, cast_rows_bf16_kernel, dim3((unsigned)((n4 + 255) / 256)), dim3(256), 0, (const float*)h, xb, n4);
+    }
     for (int j = 0; j < c.small.d.n_layers; ++j) {
         if (c.layer_map[j] != n_large_layers_done) continue;
         if (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR) {
-            launch_tc_decode<PRO_CAST, EPI_STORE_F32>(c, sc, h, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, dS, dL), true,
-                                                      epi_plain(yhat, dS));
+            const TcW w = tcw(c, wi_tandem(c, j, 0), -1, -1, dS, dL);
+            if (fused) launch_tc_decode<PRO_CAST, EPI_STORE_F32>(c, sc, h, dL, nullptr, nullptr, r.M, w, true, epi_plain(yhat, dS));
+            else launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, xb, dL, nullptr, nullptr, r.M, w, true, epi_plain(yhat, dS));
         } else {
             bf16* t1 = at<bf16>(c, c.lay.t1);
-            launch_tc_decode<PRO_CAST, EPI_GELU>(c, sc, h, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, c.hidden, dL), true,
-                                                 epi_plain(t1, c.hidden));
+            const TcW w = tcw(c, wi_tandem(c, j, 0), -1, -1, c.hidden, dL);
+            if (fused) launch_tc_decode<PRO_CAST, EPI_GELU>(c, sc, h, dL, nullptr, nullptr, r.M, w, true, epi_plain(t1, c.hidden));
+            else launch_tc_decode<PRO_BF16, EPI_GELU>(c, sc, xb, dL, nullptr, nullptr, r.M, w, true, epi_plain(t1, c.hidden));
             launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, t1, c.hidden, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 1), -1, -1, dS, c.hidden),
                                                       true, epi_plain(yhat, dS));
         }
-        launch_tc_decode<PRO_LN, EPI_KV>(c, sc, yhat, dS, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), r.M,
-                                         tcw(c, wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS), true,
-                                         epi_cache<bf16>(c, c.small, j, nullptr));
+        tc_ln_gemm<EPI_KV>(c, yhat, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), r.M,
+                           tcw(c, wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS), true, epi_cache<bf16>(c, c.small, j, nullptr));
     }
 }
 
@@ -1288,16 +1321,12 @@ extern "C" tandem_status tandem_debug_read(tandem_ctx* c, int32_t what, int32_t 
 // ---------------------------------------------------------------------------------------------------
 
 namespace {
-struct AttnScratch { size_t ml, acc, rows, counters, total; int n_chunks; };
-AttnScratch attn_scratch_layout(int batch, int H, int dh, int derived_len, int own_len) {
+struct AttnScratch { size_t rows, total; };
+// The kernel reads each row's sequence and position from two int arrays; that is all the work space it needs.
+AttnScratch attn_scratch_layout(int batch) {
     AttnScratch s;
-    s.n_chunks = cdiv(derived_len + own_len, ATT_CH);
-    size_t off = 0;
-    s.ml = off; off = align_up(off + (size_t)batch * H * s.n_chunks * 2 * 4);
-    s.acc = off; off = align_up(off + (size_t)batch * H * s.n_chunks * dh * 4);
-    s.rows = off; off = align_up(off + (size_t)batch * 2 * 4);
-    s.counters = off; off = align_up(off + (size_t)batch * H * 4);
-    s.total = off;
+    s.rows = 0;
+    s.total = align_up((size_t)batch * 2 * 4);
     return s;
 }
 __global__ void iota_rows_kernel(int* row_seq, int* row_pos, int n, int pos) {
@@ -1308,7 +1337,7 @@ __global__ void iota_rows_kernel(int* row_seq, int* row_pos, int n, int pos) {
 
 extern "C" size_t tandem_decode_attention_scratch_bytes(int32_t batch, int32_t n_heads, int32_t d_head, int32_t derived_len, int32_t own_len) {
     if (batch < 1 || n_heads < 1 || d_head < 1 || derived_len < 0 || own_len < 0 || derived_len + own_len < 1) return 0;
-    return attn_scratch_layout(batch, n_heads, d_head, derived_len, own_len).total;
+    return attn_scratch_layout(batch).total;
 }
 
 extern "C" tandem_status tandem_decode_attention(const void* q, const void* k_derived, const void* v_derived, const void* k_own,
@@ -1321,26 +1350,23 @@ extern "C" tandem_status tandem_decode_attention(const void* q, const void* k_de
     if ((long long)batch * n_heads > 65535 * 16) return TANDEM_ERR_SHAPE;
     if (((uintptr_t)q | (uintptr_t)k_derived | (uintptr_t)v_derived | (uintptr_t)k_own | (uintptr_t)v_own | (uintptr_t)out | (uintptr_t)scratch) & 15)
         return TANDEM_ERR_INVALID_ARG;
-    const AttnScratch sl = attn_scratch_layout(batch, n_heads, d_head, derived_len, own_len);
+    const AttnScratch sl = attn_scratch_layout(batch);
     if (scratch_bytes < sl.total) return TANDEM_ERR_ARENA_TOO_SMALL;
     if (batch > 65535) return TANDEM_ERR_SHAPE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned char* sc = static_cast<unsigned char*>(scratch);
     int* row_seq = reinterpret_cast<int*>(sc + sl.rows);
     int* row_pos = row_seq + batch;
-    CK(cudaMemsetAsync(sc + sl.counters, 0, (size_t)batch * n_heads * 4, s));   // the chunk-merge tickets start at zero
     iota_rows_kernel<<<cdiv(batch, 256), 256, 0, s>>>(row_seq, row_pos, batch, derived_len + own_len - 1);
     AttnArgs a; memset(&a, 0, sizeof(a));
     a.q = q; a.ldq = n_heads * d_head; a.kcache = k_derived; a.vcache = v_derived; a.k2 = k_own; a.v2 = v_own;
     a.split = derived_len; a.t_max = derived_len; a.t_max2 = own_len;
     a.out = out; a.ldo = n_heads * d_head; a.row_seq = row_seq; a.row_pos = row_pos; a.nq = 1; a.n_heads = n_heads;
-    a.part_ml = reinterpret_cast<float*>(sc + sl.ml); a.part_acc = reinterpret_cast<float*>(sc + sl.acc);
-    a.n_chunks_max = sl.n_chunks; a.scale = 1.0f / sqrtf((float)d_head);
-    a.merge_counters = reinterpret_cast<int*>(sc + sl.counters);
+    a.scale = 1.0f / sqrtf((float)d_head);
     tandem_ctx tmp;   // only the stream and the launch counter are used by the launch helpers
     tmp.stream = s;
     tmp.use_pdl = false;
-    launch_attn<bf16>(tmp, d_head, a, batch, false, sl.n_chunks, 0.0);
+    launch_attn_decode(tmp, d_head, a, batch, 0.0);
     return check_launch();
 }
 
@@ -1348,8 +1374,7 @@ extern "C" tandem_status tandem_decode_attention(const void* q, const void* k_de
 // Decode attention for callers that cannot allocate device memory
 // ---------------------------------------------------------------------------------------------------
 
-// Split-K partial results and row indices of tandem_decode_attention_static live here instead of in a
-// caller-provided buffer.  Every GPU that loads this library holds these bytes until the process exits.
+// The per-row index arrays of tandem_decode_attention_static live here instead of in a caller-provided buffer.  Every GPU that loads this library holds these bytes until the process exits.
 static __device__ __align__(256) unsigned char g_static_attn_scratch[TANDEM_STATIC_SCRATCH_BYTES];
 
 namespace {
@@ -1379,10 +1404,10 @@ extern "C" tandem_status tandem_decode_attention_static(const void* q, const voi
                                                         void* stream) {
     if (batch < 1 || n_heads < 1 || d_head < 1 || derived_len < 0 || own_len < 0 || derived_len + own_len < 1)
         return TANDEM_ERR_INVALID_ARG;
-    const size_t need = attn_scratch_layout(batch, n_heads, d_head, derived_len, own_len).total;
+    const size_t need = attn_scratch_layout(batch).total;
     if (need > (size_t)TANDEM_STATIC_SCRATCH_BYTES) {
         snprintf(g_cuda_err, sizeof(g_cuda_err),
-                 "tandem_decode_attention_static: this shape needs %zu bytes of split-K scratch, the built-in buffer holds %d; "
+                 "tandem_decode_attention_static: this batch needs %zu bytes of work space, the built-in buffer holds %d; "
                  "use tandem_decode_attention with your own scratch", need, TANDEM_STATIC_SCRATCH_BYTES);
         return TANDEM_ERR_CAPACITY;
     }

@@ -252,7 +252,8 @@ def test_bf16_small_config_speed_equals_greedy_full_prompt():
 # ------------------------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("B,H,dh,Td,To", [(1, 16, 64, 1024, 4), (3, 4, 64, 129, 4), (2, 2, 32, 0, 3), (2, 3, 128, 127, 0),
-                                          (1, 16, 64, 1, 1), (8, 16, 64, 2048, 4), (1, 2, 64, 128, 1)])
+                                          (1, 16, 64, 1, 1), (8, 16, 64, 2048, 4), (1, 2, 64, 128, 1),
+                                          (2, 4, 64, 5000, 3), (1, 3, 128, 3300, 1), (2, 2, 32, 4100, 0)])
 def test_decode_attention_mixed_context_matches_oracle(B, H, dh, Td, To):
     import torch
     g = torch.Generator().manual_seed(B * 1000 + Td)
@@ -268,7 +269,8 @@ def test_decode_attention_mixed_context_matches_oracle(B, H, dh, Td, To):
             assert np.abs(out[b, h] - want).max() < TOL_BF16
 
 
-@pytest.mark.parametrize("rows,dL,dS", [(4, 256, 64), (13, 4096, 1024), (1, 128, 128)])
+@pytest.mark.parametrize("rows,dL,dS", [(4, 256, 64), (13, 4096, 1024), (1, 128, 128), (29, 512, 256), (40, 1000, 136),
+                                        (64, 1024, 512), (100, 768, 320)])
 def test_ff_tandem_project_matches_oracle(rows, dL, dS):
     import torch
     g = torch.Generator().manual_seed(rows)

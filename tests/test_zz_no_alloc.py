@@ -2,9 +2,9 @@
 
 tandem_decode_attention_static is for callers that cannot call cudaMalloc (host callbacks, processes whose
 device memory belongs to a framework's pool, services that must not touch the allocator once they serve): its
-split-K partial results go to a buffer built into the library instead of a caller-provided one.  It must give
-the same output as tandem_decode_attention, call after call, although every call reuses that one buffer and
-finds the previous call's contents in it.  This file sorts last on purpose: a run that stops at the first
+work space (the per-row index arrays the kernel reads) is a buffer built into the library instead of a
+caller-provided one.  It must give the same output as tandem_decode_attention, call after call, although every
+call reuses that one buffer and finds the previous call's contents in it.  This file sorts last on purpose: a run that stops at the first
 failure has then already run every other test.
 """
 import numpy as np
@@ -28,7 +28,7 @@ def test_static_scratch_entry_point_matches_the_ordinary_one_twice_in_a_row():
     import torch
     build.build()
     binding.load_library()
-    # two different shapes back to back: the second call meets the first call's partial results in the buffer
+    # two different shapes back to back: the second call meets the first call's contents in the buffer
     for B, H, dh, Td, To, seed in ((2, 16, 64, 1000, 4, 1), (3, 4, 128, 300, 2, 2)):
         q, kd, vd, ko, vo = _inputs(B, H, dh, Td, To, seed)
         want = binding.tandem_decode_attention(q, kd, vd, ko, vo)
@@ -45,7 +45,7 @@ def test_static_scratch_entry_point_refuses_shapes_beyond_its_buffer():
     import torch
     build.build()
     lib = binding.load_library()
-    B, H, dh, Td, To = 32, 16, 64, 32768, 4          # needs far more than the built-in 4 MiB
+    B, H, dh, Td, To = 9000, 1, 32, 1, 0             # 8 bytes per sequence: more than the built-in 64 KiB
     assert lib.tandem_decode_attention_scratch_bytes(B, H, dh, Td, To) > binding.STATIC_SCRATCH_BYTES
     q = torch.zeros(B, H, dh, dtype=torch.bfloat16, device="cuda")
     kv = torch.zeros(1, dtype=torch.bfloat16, device="cuda")   # never read: the call must fail before any launch
