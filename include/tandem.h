@@ -200,9 +200,9 @@ TANDEM_API int64_t tandem_launch_count(tandem_ctx* ctx);
  *   scratch          work space of at least tandem_decode_attention_scratch_bytes(...) bytes (the kernel reads
  *                    every row's sequence and position from two int arrays that the call fills there)
  * d_head in {32, 64, 128}; batch <= 65535.  The context is cut into 128-position chunks by absolute position.
- * A cluster of eight CTAs serves one (sequence, head): CTA r takes chunks r, r + 8, ..., each warp keeps an
- * online-softmax state for its share of the positions, and the states are merged in a fixed order through
- * the cluster's shared memory, so a query's result does not depend on what else is in the launch. */
+ * A cluster of 1, 2, 4 or 8 CTAs (chosen from batch * n_heads) serves one (sequence, head): CTA r takes every
+ * cluster-size-th chunk starting at r, each warp keeps an online-softmax state for its share of the positions,
+ * and the states are merged in a fixed order through the cluster's shared memory. */
 TANDEM_API size_t tandem_decode_attention_scratch_bytes(int32_t batch, int32_t n_heads, int32_t d_head,
                                              int32_t derived_len, int32_t own_len);
 TANDEM_API tandem_status tandem_decode_attention(const void* q, const void* k_derived, const void* v_derived,

@@ -231,20 +231,20 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Decode attention, bf16, built for short dependent chains and for streaming: a cluster of ATD_CLUSTER CTAs
-// serves one (sequence, head).  CTA `rank` takes the 128-position chunks rank, rank + 8, ... (anchored at
+// Decode attention, bf16, built for short dependent chains and for streaming: a cluster of CL CTAs (1, 2, 4 or 8,
+// fixed per launch configuration) serves one (sequence, head).  CTA `rank` takes the 128-position chunks rank, rank + CL, ... (anchored at
 // absolute position 0); inside a chunk warp w owns positions 16w .. 16w+15.  Every warp runs on its own: it
 // fetches its rows through a private cp.async ring, keeps an online-softmax state per query in registers and
 // never waits for another warp until the end, where the CTA folds its warps' states in warp order, sends the
-// result to the CTA that finishes the query (remote shared-memory stores), and that CTA merges the eight
+// result to the CTA that finishes the query (remote shared-memory stores), and that CTA merges the CL
 // states in rank order.  No global scratch, no second kernel.  DH / 8 lanes share a key (16 bytes each); a
 // query's arithmetic does not depend on the other queries.  The probabilities use the fast exponential
 // (2^x hardware approximation), well inside the bf16 tolerance.
 // ---------------------------------------------------------------------------------------------------
 constexpr int ATD_THREADS = 256;
 constexpr int ATD_WARPS = ATD_THREADS / 32;
-constexpr int ATD_CLUSTER = 8;
-constexpr int ATD_QPC = (ATT_NQ + ATD_CLUSTER - 1) / ATD_CLUSTER;   // queries a CTA finishes at most
+constexpr int ATD_CLUSTER = 8;                                      // largest cluster; launches use 1, 2, 4 or 8
+constexpr int ATD_SLOTS = ATT_NQ;                                   // inbox states per CTA: cluster size x queries it finishes <= 16
 constexpr int ATD_WROWS = ATT_CH / ATD_WARPS;                       // positions of a chunk per warp (16)
 
 template <int DH> struct AtdCfg {
@@ -259,10 +259,10 @@ template <int DH> struct AtdCfg {
 template <int DH, int QG>
 constexpr size_t attn_decode_smem_bytes() {
     return (size_t)ATD_WARPS * AtdCfg<DH>::STAGES * AtdCfg<DH>::STAGE_ELEMS * sizeof(bf16) +
-           sizeof(float) * ((size_t)ATT_NQ * DH + (size_t)ATD_WARPS * QG * (DH + 2) + (size_t)ATD_CLUSTER * ATD_QPC * (DH + 2));
+           sizeof(float) * ((size_t)ATT_NQ * DH + (size_t)ATD_WARPS * QG * (DH + 2) + (size_t)ATD_SLOTS * (DH + 2));
 }
 
-// grid: (ATD_CLUSTER, heads, sequences) in clusters of ATD_CLUSTER along x; block: ATD_THREADS.
+// grid: (CL, heads, sequences) with the CL CTAs along x forming one cluster, CL in {1, 2, 4, 8}; block: ATD_THREADS.
 template <int DH, int QG>
 __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     using C = AtdCfg<DH>;
@@ -271,11 +271,13 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     bf16* ring_all = reinterpret_cast<bf16*>(smem_raw);
     float* qs = reinterpret_cast<float*>(ring_all + (size_t)NW * C::STAGES * C::STAGE_ELEMS);   // [ATT_NQ][DH]
     float* wst = qs + ATT_NQ * DH;                 // [NW][QG][DH + 2] the warps' states of the current query group
-    float* inbox = wst + NW * QG * (DH + 2);       // [ATD_CLUSTER][ATD_QPC][DH + 2] states sent by the cluster's CTAs
+    float* inbox = wst + NW * QG * (DH + 2);       // [CL][QPC][DH + 2] states sent by the cluster's CTAs
     TC_PROBE_INIT(210);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = blockIdx.x, h = blockIdx.y, g = blockIdx.z;
+    const int CL = gridDim.x;                      // cluster size
+    const int QPC = (ATT_NQ + CL - 1) / CL;        // queries a CTA finishes at most
     const int part = lane % C::TPK, kslot = lane / C::TPK;
     bf16* ring = ring_all + (size_t)warp * C::STAGES * C::STAGE_ELEMS;
     pdl_launch_dependents();
@@ -291,14 +293,14 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     const int pos_first = a.row_pos[row0];
     const int pos_last = pos_first + cnt - 1;
     const int n_chunks = pos_last / ATT_CH + 1;
-    const int n_mine = rank < n_chunks ? (n_chunks - rank + ATD_CLUSTER - 1) / ATD_CLUSTER : 0;
+    const int n_mine = rank < n_chunks ? (n_chunks - rank + CL - 1) / CL : 0;
     const size_t head_base = ((size_t)b * a.n_heads + h) * a.t_max;
     const size_t head_base2 = ((size_t)b * a.n_heads + h) * a.t_max2;
     const int split = a.k2 ? a.split : INT_MAX;
 
     // this warp's rows of its CTA's it-th chunk into stage it % STAGES
     auto issue = [&](int it) {
-        const int t0 = (rank + it * ATD_CLUSTER) * ATT_CH + warp * ATD_WROWS;
+        const int t0 = (rank + it * CL) * ATT_CH + warp * ATD_WROWS;
         bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
         bf16* vs = ks + C::TILE_ELEMS;
 #pragma unroll
@@ -350,7 +352,7 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
             asm volatile("cp.async.wait_group %0;" ::"n"(C::STAGES - 1) : "memory");
             __syncwarp();
             if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(3);
-            const int t0 = (rank + it * ATD_CLUSTER) * ATT_CH + warp * ATD_WROWS;
+            const int t0 = (rank + it * CL) * ATT_CH + warp * ATD_WROWS;
             const bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
             const bf16* vs = ks + C::TILE_ELEMS;
             float sc[QG][C::PPW], mc[QG];
@@ -442,24 +444,23 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
                         val = fmaf(e < DH ? st[e] : st[DH + 1], f, val);
                     }
                 }
-                st_dsmem_f32(smem_u32(inbox + ((size_t)rank * ATD_QPC + qa / ATD_CLUSTER) * (DH + 2) + e), qa % ATD_CLUSTER, val);
+                float* slot = inbox + ((size_t)rank * QPC + qa / CL) * (DH + 2) + e;
+                if (CL > 1) st_dsmem_f32(smem_u32(slot), qa % CL, val);
+                else *slot = val;
             }
         }
         __syncthreads();   // wst is rewritten by the next query group
     }
-    cluster_sync_all();
+    if (CL > 1) cluster_sync_all(); else __syncthreads();
     if (tid == 0) TC_PROBE(5);
-#pragma unroll
-    for (int u = 0; u < ATD_QPC; ++u) {
-        const int qi = rank + u * ATD_CLUSTER;
+    for (int u = 0; u < QPC; ++u) {
+        const int qi = rank + u * CL;
         if (qi < cnt && tid < DH) {
             float mx = -INFINITY;
-#pragma unroll
-            for (int r = 0; r < ATD_CLUSTER; ++r) mx = fmaxf(mx, inbox[((size_t)r * ATD_QPC + u) * (DH + 2) + DH]);
+            for (int r = 0; r < CL; ++r) mx = fmaxf(mx, inbox[((size_t)r * QPC + u) * (DH + 2) + DH]);
             float l = 0.f, o = 0.f;
-#pragma unroll
-            for (int r = 0; r < ATD_CLUSTER; ++r) {
-                const float* st = inbox + ((size_t)r * ATD_QPC + u) * (DH + 2);
+            for (int r = 0; r < CL; ++r) {
+                const float* st = inbox + ((size_t)r * QPC + u) * (DH + 2);
                 const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
                 l = fmaf(st[DH + 1], f, l);
                 o = fmaf(st[tid], f, o);

@@ -460,9 +460,9 @@ void launch_attn(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, bool 
     else launch_attn_dh<T, 128>(c, a, groups, loop, n_chunks, kv_bytes);
 }
 
-// bf16 decode attention: one cluster of ATD_CLUSTER CTAs per (sequence, head); no scratch.
+// bf16 decode attention: one cluster of `cl` CTAs per (sequence, head); no scratch.
 template <int DH, int QG>
-void launch_attn_decode_dq(tandem_ctx& c, const AttnArgs& a, int groups, double kv_bytes) {
+void launch_attn_decode_dq(tandem_ctx& c, const AttnArgs& a, int groups, int cl, double kv_bytes) {
     static bool attr_set[MAX_DEVICES] = {};
     const int dev = cur_dev();
     if (!attr_set[dev]) {
@@ -470,14 +470,21 @@ void launch_attn_decode_dq(tandem_ctx& c, const AttnArgs& a, int groups, double 
         attr_set[dev] = true;
     }
     ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
-    launch_ex(c, true, ATD_CLUSTER, attn_decode_kernel<DH, QG>, dim3(ATD_CLUSTER, a.n_heads, groups), dim3(ATD_THREADS),
-              attn_decode_smem_bytes<DH, QG>(), a);
+    launch_ex(c, true, cl, attn_decode_kernel<DH, QG>, dim3(cl, a.n_heads, groups), dim3(ATD_THREADS), attn_decode_smem_bytes<DH, QG>(), a);
+}
+// Cluster size: enough CTAs to fill the GPU about twice, at most 8.  It depends on the number of sequences and
+// heads only, so every pass of a run (block or one-row) cuts the context the same way.
+int attn_cluster_size(int groups, int n_heads) {
+    int cl = 1;
+    while (cl < ATD_CLUSTER && (long long)groups * n_heads * cl < 296) cl *= 2;
+    return cl;
 }
 void launch_attn_decode(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, double kv_bytes) {
     const bool one = a.nq == 1;
-    if (d_head == 32) { if (one) launch_attn_decode_dq<32, 1>(c, a, groups, kv_bytes); else launch_attn_decode_dq<32, 4>(c, a, groups, kv_bytes); }
-    else if (d_head == 64) { if (one) launch_attn_decode_dq<64, 1>(c, a, groups, kv_bytes); else launch_attn_decode_dq<64, 4>(c, a, groups, kv_bytes); }
-    else { if (one) launch_attn_decode_dq<128, 1>(c, a, groups, kv_bytes); else launch_attn_decode_dq<128, 4>(c, a, groups, kv_bytes); }
+    const int cl = attn_cluster_size(groups, a.n_heads);
+    if (d_head == 32) { if (one) launch_attn_decode_dq<32, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<32, 4>(c, a, groups, cl, kv_bytes); }
+    else if (d_head == 64) { if (one) launch_attn_decode_dq<64, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<64, 4>(c, a, groups, cl, kv_bytes); }
+    else { if (one) launch_attn_decode_dq<128, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<128, 4>(c, a, groups, cl, kv_bytes); }
 }
 
 template <typename T>
@@ -1470,7 +1477,13 @@ extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
         // few rows: weights streamed once per GEMM; LayerNorm fused into the second GEMM's operand load
         TcScratch ts; ts.err = nullptr;
         launch_tc_decode<PRO_BF16, EPI_STORE_F32>(tmp, ts, x, d_large, nullptr, nullptr, rows, wt, true, epi_plain(yhat, d_small));
-        launch_tc_decode<PRO_LN, EPI_KV>(tmp, ts, yhat, d_small, ln_g, ln_b, rows, wkv, true, e);
+        if (rows <= 8 && d_small <= 1024) {
+            launch_tc_decode<PRO_LN, EPI_KV>(tmp, ts, yhat, d_small, ln_g, ln_b, rows, wkv, true, e);
+        } else {
+            launch_ex(tmp, false, 1, layernorm_rows_bf16_kernel, dim3(rows), dim3(128), 0, (const float*)yhat, static_cast<const float*>(ln_g),
+                      static_cast<const float*>(ln_b), a_s, (int)d_small);
+            launch_tc_decode<PRO_BF16, EPI_KV>(tmp, ts, a_s, d_small, nullptr, nullptr, rows, wkv, true, e);
+        }
     } else {
         TRY(launch_tc_tiled<EPI_STORE_F32>(tmp, static_cast<const bf16*>(x), d_large, rows, wt, epi_plain(yhat, d_small), nullptr));
         launch_layernorm<bf16>(tmp, rows, yhat, ln_g, ln_b, a_s, d_small);
