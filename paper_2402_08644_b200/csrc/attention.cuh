@@ -58,8 +58,8 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_last;
     TC_PROBE_INIT(LOOP ? 201 : 200);
-    pdl_launch_dependents();   // the next kernel may start fetching its weights
     pdl_wait();                // queries and keys/values come from earlier kernels
+    pdl_launch_dependents();   // the next kernel may start fetching its weights
     if (threadIdx.x == 0) TC_PROBE(1);
     T* ks = reinterpret_cast<T*>(smem_raw);
     T* vs = ks + ATT_CH * LD;
@@ -280,8 +280,8 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     const int QPC = (ATT_NQ + CL - 1) / CL;        // queries a CTA finishes at most
     const int part = lane % C::TPK, kslot = lane / C::TPK;
     bf16* ring = ring_all + (size_t)warp * C::STAGES * C::STAGE_ELEMS;
-    pdl_launch_dependents();
     pdl_wait();   // queries and the newest keys/values come from earlier kernels
+    pdl_launch_dependents();
     if (tid == 0) TC_PROBE(1);
     const int cnt = a.nq, row0 = g * a.nq;
     const bf16* qg = static_cast<const bf16*>(a.q);

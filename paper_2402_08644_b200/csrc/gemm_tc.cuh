@@ -10,7 +10,9 @@
 //                          The token rows are written into the B stages by the CTA's own threads, which is
 //                          where the LayerNorm (or the fp32 -> bf16 cast) of the residual stream is fused.
 //                          The weight loads are issued before the kernel waits for its predecessor in the
-//                          stream (programmatic dependent launch), so they overlap its tail.
+//                          stream (programmatic dependent launch), so they overlap its run; a kernel lets its
+//                          own successor start once the predecessor is done, which keeps one kernel's worth of
+//                          prefetch in flight (deeper chains of waiting kernels cost more than they hide).
 //  gemm_tc_tiled_kernel    many rows (prompt pass): 128 x 128 output tiles, both operands by TMA.
 //
 // An output element's reduction order depends on (N, K) only, never on the number of rows, so a block
@@ -118,7 +120,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = s_tmem;
-    pdl_launch_dependents();
     if (tid == 0) TC_PROBE(1);
 
     if (warp == 4) {
@@ -177,6 +178,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         }
     }
     pdl_wait();   // x, and everything the epilogue touches, comes from earlier kernels; gains and biases are parameters
+    pdl_launch_dependents();   // only now: one successor at a time sets up and fetches weights behind this kernel
     if (tid == 0) TC_PROBE(5);
     if (EPI == EPI_RESID) {
         // the residual-stream values this thread will add to: fetched now, off the critical path

@@ -86,8 +86,8 @@ __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, i
                                                          const T* __restrict__ pos, float* __restrict__ h, int d) {
     __shared__ int s_tok, s_pos;
     TC_PROBE_INIT(300);
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     if (threadIdx.x == 0) TC_PROBE(1);
     const int m = blockIdx.x;
     const int b = m / nq, r = r0 + (m - b * nq);
@@ -139,8 +139,8 @@ __global__ void __launch_bounds__(128) layernorm_kernel(const float* __restrict_
 __global__ void __launch_bounds__(128) layernorm_rows_bf16_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                                                   const float* __restrict__ bias, bf16* __restrict__ out, int d) {
     __shared__ float red[4];
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     const int d4 = d >> 2;
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)blockIdx.x * d);
     uint2* orow = reinterpret_cast<uint2*>(out + (size_t)blockIdx.x * d);
@@ -194,8 +194,8 @@ __global__ void __launch_bounds__(128) layernorm_rows_bf16_kernel(const float* _
 
 // fp32 rows to bf16, 4 elements per thread; n % 4 == 0.  Decode path (waits for its predecessor in the stream).
 __global__ void cast_rows_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ out, size_t n4) {
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n4) {
         const float4 t = __ldcg(reinterpret_cast<const float4*>(x) + i);
@@ -248,8 +248,8 @@ __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, in
                                                      int max_new, const float* amax_val, const int* amax_idx, int amax_stride,
                                                      int n_tiles) {
     TC_PROBE_INIT(400);
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     if (threadIdx.x == 0) TC_PROBE(1);
     if (amax_val != nullptr) {
         const int rows = batch * (gamma + 1);

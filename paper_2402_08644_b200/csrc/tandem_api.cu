@@ -358,11 +358,15 @@ void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx
     a.x = x; a.ldx = ldx; a.ln_g = static_cast<const float*>(ln_g); a.ln_b = static_cast<const float*>(ln_b);
     a.rows = rows; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
     const int tiles = w.n_segs * a.tiles_per_seg, KB = cdiv(w.K, 64);
-    // K-slices per tile = cluster size: the smallest power of two that puts tiles * S CTAs at or above the target
-    // (about one per SM), at most 8 and at most one per 64-element K-block.  The head GEMM keeps whole tiles.
+    // K-slices per tile = cluster size (a power of two, at most 8, at most one per 64-element K-block): first enough
+    // that a CTA's whole K-slice fits its ring, so every weight tile can be in flight before the predecessor kernel
+    // has finished; then more while the launch has fewer CTAs than the target.  The head GEMM keeps whole tiles.
     int S = 1;
-    if (EPI != EPI_ARGMAX)
-        while (S < 8 && tiles * S < c.tc_target && 2 * S <= KB) S *= 2;
+    if (EPI != EPI_ARGMAX) {
+        const int stages = rows <= 16 ? TcdCfg<16>::STAGES : rows <= 32 ? TcdCfg<32>::STAGES : TcdCfg<64>::STAGES;
+        while (S < 8 && 2 * S <= KB && cdiv(KB, S) > stages) S *= 2;
+        while (S < 8 && 2 * S <= KB && tiles * S < c.tc_target) S *= 2;
+    }
     a.splits = S;
     a.stream_weights = stream_weights ? 1 : 0;
     a.err_flag = sc.err;
