@@ -8,6 +8,7 @@ workload is the "Small Tandem" configuration: bf16, batch 1, 512-token random pr
 tokens, natural acceptance.  The metric is generated tokens per second of the whole job.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload small|tiny|medium]
+  python bench.py --workload micro [--micro-case B,T]     kernel micro-benchmark (decode attention, FF_Tandem projection)
 
 With N > 1 (under torchrun) every rank runs an independent replica (sequences are independent units; there
 is no collective on the path); the value is all ranks' tokens over the slowest rank's time.
@@ -40,7 +41,10 @@ WORKLOADS = {
     "tiny": ("tiny", 1, 32, 4, 64, 128),
     "small": ("small", 1, 512, 3, 256, 1024),
     "medium": ("medium", 8, 2048, 3, 256, 2560),
+    "large": ("large", 1, 8192, 3, 512, 8960),
+    "large4": ("large", 4, 8192, 3, 512, 8960),
 }
+DEVICE_INIT = {"large", "large4"}   # too big to draw on the host in reasonable time: N(0, 0.02^2) drawn on the device
 
 
 def workload_desc(name):
@@ -104,6 +108,20 @@ class ClockSampler:
                     reasons.add(nm)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def device_weights(shape, seed, device):
+    """Random-init weights drawn on the device (timing only; no CPU checker run uses them)."""
+    import torch
+    g = torch.Generator(device=device).manual_seed(seed)
+    out = {}
+    for name in synth.weight_names(shape):
+        shp = synth.weight_shape(shape, name)
+        if synth.is_norm_param(name):
+            out[name] = torch.full(shp, 1.0 if name.endswith("_g") else 0.0, dtype=torch.float32, device=device)
+        else:
+            out[name] = (torch.randn(shp, generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    return out
 
 
 def algorithmic_bytes_per_iteration(shape, B, gamma, T):
@@ -173,18 +191,76 @@ def cpu_baseline(shape, weights, prompt, gamma, new):
                        f"({t2 - t1:.1f} s), decode time scaled to {new} tokens; numpy fp64 with its BLAS threads")}
 
 
+def run_micro(args):
+    """Kernel micro-benchmark: small-model decode attention (16 heads x 64, one query per (sequence, head)) over a
+    large-derived context of T positions plus 4 own positions, and the FF_Tandem projection 4096 -> 1024 with
+    the key/value maps, through the stand-alone C entry points.  L2 is flushed between timed calls."""
+    import torch
+    from paper_2402_08644_b200 import binding, build as _build
+    _build.build()
+    binding.load_library()
+    peak, peak_kind = read_peaks()
+    dev = torch.device("cuda", 0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    g = torch.Generator(device=dev).manual_seed(0)
+
+    def timed(fn):
+        for _ in range(max(3, args.warmup)):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(max(5, args.steps)):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    H, dh, To = 16, 64, 4
+    cases = [(B, T) for B in (1, 8, 32) for T in (1024, 8192, 32768)]
+    if args.micro_case:
+        cases = [tuple(int(v) for v in args.micro_case.split(","))]
+    out = {"metric": "decode_attention_gbs", "unit": "GB/s", "peak": peak, "peak_kind": peak_kind, "dtype": "bf16",
+           "data": "synthetic N(0,1) queries, keys and values", "attention": [], "ff_tandem_project": []}
+    rn = lambda *s: torch.randn(*s, generator=g, device=dev).to(torch.bfloat16)
+    for B, T in cases:
+        q, kd, vd, ko, vo = rn(B, H, dh), rn(B, H, T, dh), rn(B, H, T, dh), rn(B, H, To, dh), rn(B, H, To, dh)
+        o = torch.empty_like(q)
+        scratch = torch.empty(1 << 20, dtype=torch.uint8, device=dev)
+        ms = timed(lambda: binding.tandem_decode_attention(q, kd, vd, ko, vo, o, scratch))
+        byt = 2 * B * H * (T + To) * dh * 2 + 2 * B * H * dh * 2
+        out["attention"].append({"batch": B, "derived_len": T, "own_len": To, "us": ms * 1e3, "algorithmic_bytes": byt,
+                                 "gbs": byt / ms / 1e6, "frac": byt / ms / 1e6 / peak})
+        del q, kd, vd, ko, vo
+    if not args.micro_case:
+        dL, dS = 4096, 1024
+        for rows in (4, 32, 128):
+            x = rn(rows, dL)
+            wt, wk, wv = (rn(dS, k) * 0.02 for k in (dL, dS, dS))
+            lg, lb = torch.ones(dS, device=dev), torch.zeros(dS, device=dev)
+            ms = timed(lambda: binding.tandem_ff_tandem_project(x, wt, lg, lb, wk, wv))
+            byt = (dS * dL + 2 * dS * dS) * 2 + rows * (dL + 2 * dS) * 2
+            out["ff_tandem_project"].append({"rows": rows, "us": ms * 1e3, "algorithmic_bytes": byt, "gbs": byt / ms / 1e6,
+                                             "frac": byt / ms / 1e6 / peak})
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="small", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="small", choices=sorted(WORKLOADS) + ["micro"])
+    ap.add_argument("--micro-case", default="", help="with --workload micro: one attention case 'batch,context'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the accept-all / greedy / per-kernel passes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
+    if args.workload == "micro":
+        run_micro(args)
+        return
     if args.impl == "reference":
         run_reference(args)
         return
@@ -206,7 +282,11 @@ def main():
 
     cfgname, B, P, gamma, new, max_pos = WORKLOADS[args.workload]
     shape = synth.named_config(cfgname, max_pos)
-    weights = synth.make_weights(shape, seed=0)
+    if args.workload in DEVICE_INIT:
+        weights = device_weights(shape, 0, torch.device("cuda", local_rank))
+        args.no_cpu_baseline = True
+    else:
+        weights = synth.make_weights(shape, seed=0)
     prompts = [[int(t) for t in p] for p in synth.make_prompts(B, P, shape.large.vocab, seed=rank)]
     t = binding.Tandem(shape, weights, max_batch=B, max_seq=P + new + gamma + 1, gamma_max=gamma, device=local_rank,
                        max_prefill_rows=B * P)

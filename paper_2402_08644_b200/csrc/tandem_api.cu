@@ -358,15 +358,11 @@ void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx
     a.x = x; a.ldx = ldx; a.ln_g = static_cast<const float*>(ln_g); a.ln_b = static_cast<const float*>(ln_b);
     a.rows = rows; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
     const int tiles = w.n_segs * a.tiles_per_seg, KB = cdiv(w.K, 64);
-    // K-slices per tile = cluster size (a power of two, at most 8, at most one per 64-element K-block): first enough
-    // that a CTA's whole K-slice fits its ring, so every weight tile can be in flight before the predecessor kernel
-    // has finished; then more while the launch has fewer CTAs than the target.  The head GEMM keeps whole tiles.
+    // K-slices per tile = cluster size: the smallest power of two that puts tiles * S CTAs at or above the target
+    // (about one per SM), at most 8 and at most one per 64-element K-block.  The head GEMM keeps whole tiles.
     int S = 1;
-    if (EPI != EPI_ARGMAX) {
-        const int stages = rows <= 16 ? TcdCfg<16>::STAGES : rows <= 32 ? TcdCfg<32>::STAGES : TcdCfg<64>::STAGES;
-        while (S < 8 && 2 * S <= KB && cdiv(KB, S) > stages) S *= 2;
+    if (EPI != EPI_ARGMAX)
         while (S < 8 && 2 * S <= KB && tiles * S < c.tc_target) S *= 2;
-    }
     a.splits = S;
     a.stream_weights = stream_weights ? 1 : 0;
     a.err_flag = sc.err;
@@ -476,16 +472,18 @@ void launch_attn_decode_dq(tandem_ctx& c, const AttnArgs& a, int groups, int cl,
     ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
     launch_ex(c, true, cl, attn_decode_kernel<DH, QG>, dim3(cl, a.n_heads, groups), dim3(ATD_THREADS), attn_decode_smem_bytes<DH, QG>(), a);
 }
-// Cluster size: enough CTAs to fill the GPU about twice, at most 8.  It depends on the number of sequences and
-// heads only, so every pass of a run (block or one-row) cuts the context the same way.
-int attn_cluster_size(int groups, int n_heads) {
+// Cluster size: the largest of 1, 2, 4, 8 that keeps the launch within one wave of resident CTAs (two per SM,
+// one for 128-wide heads).  It depends on the number of sequences and heads only, so every pass of a run
+// (block or one-row) cuts the context the same way.
+int attn_cluster_size(int groups, int n_heads, int d_head) {
+    const long long slots = 148LL * (d_head == 128 ? 1 : 2);
     int cl = 1;
-    while (cl < ATD_CLUSTER && (long long)groups * n_heads * cl < 296) cl *= 2;
+    while (cl < ATD_CLUSTER && (long long)groups * n_heads * cl * 2 <= slots) cl *= 2;
     return cl;
 }
 void launch_attn_decode(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, double kv_bytes) {
     const bool one = a.nq == 1;
-    const int cl = attn_cluster_size(groups, a.n_heads);
+    const int cl = attn_cluster_size(groups, a.n_heads, d_head);
     if (d_head == 32) { if (one) launch_attn_decode_dq<32, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<32, 4>(c, a, groups, cl, kv_bytes); }
     else if (d_head == 64) { if (one) launch_attn_decode_dq<64, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<64, 4>(c, a, groups, cl, kv_bytes); }
     else { if (one) launch_attn_decode_dq<128, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<128, 4>(c, a, groups, cl, kv_bytes); }
