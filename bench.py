@@ -53,6 +53,21 @@ def workload_desc(name):
             f"natural acceptance, random-init N(0,0.02) weights seed 0")
 
 
+# DRAM bytes per launch of the dominant kernel from one ncu capture (profiles/gemm_tc_decode_small_workload_ncu_sections.md),
+# valid only while the kernel's sources are the ones that were profiled.
+NCU_TRAFFIC = {"workload": "small", "kernel": "gemm_tc_decode", "bytes_per_launch": 4971266.0,
+               "sources_sha256_16": "1f421f78c423fd5f"}
+
+
+def kernel_sources_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for fn in ("gemm_tc.cuh", "tc_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2402_08644_b200", "csrc", fn), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
 def read_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -376,8 +391,12 @@ def main():
         dom = max((k for k in prof if k not in flop_classes), key=lambda k: prof[k]["ms"])
         g = prof[dom]
         achieved = g["work"] / 1e9 / (g["ms"] * 1e-3) if g["ms"] > 0 else 0.0
+        traffic = None
+        if (args.workload == NCU_TRAFFIC["workload"] and dom == NCU_TRAFFIC["kernel"]
+                and kernel_sources_hash() == NCU_TRAFFIC["sources_sha256_16"]):
+            traffic = NCU_TRAFFIC["bytes_per_launch"]
         line["roofline"] = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                            "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind,
+                            "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
                             "launches": g["launches"], "avg_launch_us": 1e3 * g["ms"] / max(1, g["launches"]),
                             "algorithmic_bytes_per_launch": g["work"] / max(1, g["launches"])}
         # context: accept-all timing mode and plain greedy decoding of the large model alone
