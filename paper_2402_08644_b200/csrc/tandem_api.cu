@@ -1143,6 +1143,11 @@ extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t
         CK(cudaStreamSynchronize(c->stream));
         c->n_ub = cnt[3];
         c->n_sum = cnt[4];
+        if (cnt[2] != 0) {
+            snprintf(g_cuda_err, sizeof(g_cuda_err), "device-side wait expired (code %d)", cnt[2]);
+            CK(cudaMemsetAsync(c->st.counters + 2, 0, 4, c->stream));
+            return TANDEM_ERR_TIMEOUT;
+        }
         for (int b = 0; b < B; ++b) {
             if (result->drafts) for (int i = 0; i < gamma; ++i) result->drafts[b * gamma + i] = d[(size_t)b * GL + i];
             if (result->targets) for (int i = 0; i <= gamma; ++i) result->targets[b * (gamma + 1) + i] = t[(size_t)b * (GL + 1) + i];
@@ -1199,6 +1204,11 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
     CK(cudaStreamSynchronize(c->stream));
     c->n_ub = cnt[3];
     c->n_sum = cnt[4];
+    if (cnt[2] != 0) {   // a bounded device-side wait gave up somewhere in this call
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "device-side wait expired (code %d)", cnt[2]);
+        CK(cudaMemsetAsync(c->st.counters + 2, 0, 4, c->stream));
+        return TANDEM_ERR_TIMEOUT;
+    }
     const int64_t iters = cnt[5];
     TRY(check_launch());
     CK(cudaMemcpy2DAsync(out_ids, (size_t)max_new * 4, c->st.out_ids, (size_t)c->st.out_cap * 4, (size_t)max_new * 4, B,
