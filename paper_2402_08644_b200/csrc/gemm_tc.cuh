@@ -68,6 +68,22 @@ __device__ __forceinline__ float4 ln_apply(float4 x, float mu, float rs, float4 
     return make_float4((x.x - mu) * rs * g.x + b.x, (x.y - mu) * rs * g.y + b.y, (x.z - mu) * rs * g.z + b.z, (x.w - mu) * rs * g.w + b.w);
 }
 
+// Where column c of weight segment `seg` goes for EPI_QKV / EPI_KV: the query buffer (row stride ldo) or a cache.
+// The address of (row j, column c) is base + row term + col, with the row term j * ldo or the cache row offset.
+struct ScatterCol { bf16* base; long long col; bool is_q; };
+template <int EPI>
+__device__ __forceinline__ ScatterCol scatter_col(const EpiArgs& e, int seg, int c) {
+    ScatterCol sc;
+    int s = seg;
+    if (EPI == EPI_QKV && s == 0) { sc.base = static_cast<bf16*>(e.out); sc.col = c; sc.is_q = true; return sc; }
+    if (EPI == EPI_QKV) s -= 1;
+    const int h = c / e.d_head, el = c - h * e.d_head;
+    sc.base = static_cast<bf16*>(s == 0 ? e.kcache : e.vcache);
+    sc.col = (long long)h * e.t_max * e.d_head + el;
+    sc.is_q = false;
+    return sc;
+}
+
 // grid: tiles * splits CTAs in clusters of `splits` (the K-slices of one tile); dynamic smem TcdCfg<NB>::SMEM_BYTES.
 template <int NB, int PRO, int EPI>
 __global__ void __launch_bounds__(TCD_THREADS)
@@ -82,6 +98,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     __shared__ float s_mu[NB], s_rstd[NB];
     __shared__ float s_av[4][NB];
     __shared__ int s_ai[4][NB];
+    __shared__ long long s_rowoff[NB];   // EPI_QKV / EPI_KV: the row-dependent part of an output's cache index
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t ring0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // shared-space address of stage 0
@@ -180,6 +197,12 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     pdl_wait();   // x, and everything the epilogue touches, comes from earlier kernels; gains and biases are parameters
     pdl_launch_dependents();   // only now: one successor at a time sets up and fetches weights behind this kernel
     if (tid == 0) TC_PROBE(5);
+    if (EPI == EPI_QKV || EPI == EPI_KV) {
+        // cache index of (row j, head h, element el) = ((seq_j * H + h) * t_max + pos_j) * d_head + el: the row part once per row
+        if (tid < a.rows)
+            s_rowoff[tid] = ((long long)a.e.row_seq[tid] * a.e.n_heads * a.e.t_max + a.e.row_pos[tid]) * a.e.d_head;
+        bar_sync(1, 128);
+    }
     if (EPI == EPI_RESID) {
         // the residual-stream values this thread will add to: fetched now, off the critical path
         const float* hp = static_cast<const float*>(a.e.out);
@@ -400,6 +423,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
                 for (int j = 0; j < NB; ++j)
                     if (j < a.rows && valid) out[(size_t)j * a.e.ldo + n] = hres[j] + v[j];
+            } else if (EPI == EPI_QKV || EPI == EPI_KV) {
+                const ScatterCol sc = scatter_col<EPI>(a.e, seg, n_local);
+#pragma unroll
+                for (int j = 0; j < NB; ++j)
+                    if (j < a.rows && valid) sc.base[(sc.is_q ? (long long)j * a.e.ldo : s_rowoff[j]) + sc.col] = __float2bfloat16_rn(v[j]);
             } else {
 #pragma unroll
                 for (int j = 0; j < NB; ++j)
@@ -427,6 +455,8 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             const int n_local = n_local0 + sp * CW + cw;
             const bool valid = n_local < a.seg_rows;
             const int n = seg * a.seg_rows + n_local;
+            ScatterCol sc;
+            if (EPI == EPI_QKV || EPI == EPI_KV) sc = scatter_col<EPI>(a.e, seg, n_local);
 #pragma unroll
             for (int it = 0; it < NB / 2; ++it) {       // 128 / CW = S row groups: rows tid / CW, + S, ...
                 const int j = tid / CW + it * S;
@@ -435,6 +465,8 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
                     for (int ss = 0; ss < 8; ++ss) if (ss < S) acc += inbox[(ss * NB + j) * CW + cw];   // slice order
                     if (EPI == EPI_RESID) static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = hres[it] + acc;
+                    else if (EPI == EPI_QKV || EPI == EPI_KV)
+                        sc.base[(sc.is_q ? (long long)j * a.e.ldo : s_rowoff[j]) + sc.col] = __float2bfloat16_rn(acc);
                     else epilogue<bf16, EPI>(a.e, j, n, acc);
                 }
             }
