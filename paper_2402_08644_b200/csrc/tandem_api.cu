@@ -13,6 +13,7 @@
 
 #include "../../include/tandem.h"
 #include "attention.cuh"
+#include "attention_tc.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
@@ -116,6 +117,9 @@ struct tandem_ctx {
     int tc_target = 148;                 // CTAs a split-K decode GEMM aims for
     std::vector<CUtensorMap> wmap;       // one per weight pointer (matrices only), box 128 rows x 64 columns
     std::vector<char> wmap_ok;
+    std::vector<CUtensorMap> kmap, vmap; // the large model's key / value cache of each layer as [(seq, head, position)][d_head]
+    bool tc_prompt_attn = false;         // prompt attention on the tensor cores (head size 64 or 128)
+    int prompt_group = ATT_NQ;           // queries per attention group of the prompt pass
 };
 
 namespace {
@@ -525,6 +529,33 @@ EpiArgs epi_cache(tandem_ctx& c, const Model& m, int layer, void* q_out) {
     return e;
 }
 
+// Prompt attention of the large model's layer l on the tensor cores; groups of up to 128 queries.
+template <int DH>
+void launch_attn_prompt_tc_dh(tandem_ctx& c, const AttnTcArgs& a, const CUtensorMap& tmq, int l, int groups) {
+    static bool attr_set[MAX_DEVICES] = {};
+    const int dev = cur_dev();
+    if (!attr_set[dev]) {
+        cudaFuncSetAttribute(attn_prefill_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcCfg<DH>::SMEM_BYTES);
+        attr_set[dev] = true;
+    }
+    launch_ex(c, false, 1, attn_prefill_tc_kernel<DH>, dim3(a.n_heads, groups), dim3(ATC_THREADS), (size_t)AtcCfg<DH>::SMEM_BYTES, a, tmq,
+              c.kmap[l], c.vmap[l]);
+}
+void launch_attn_prompt_tc(tandem_ctx& c, int l, const bf16* q, bf16* o, const Rows& r) {
+    const int d = c.large.d.d_model, H = c.large.d.n_heads, dh = d / H;
+    CUtensorMap tmq;
+    if (!make_tmap_bf16(&tmq, q, (uint64_t)r.M, (uint64_t)d, (uint64_t)d)) return;   // cannot fail once the weights' maps were made
+    AttnTcArgs a;
+    memset(&a, 0, sizeof(a));
+    a.out = o; a.ldo = d; a.row_seq = at<int>(c, c.lay.row_seq); a.row_pos = at<int>(c, c.lay.row_pos);
+    a.grp_row0 = at<int>(c, c.lay.grp_row0); a.grp_cnt = at<int>(c, c.lay.grp_cnt);
+    a.n_heads = H; a.t_max = c.cfg.max_seq; a.scale = 1.0f / sqrtf((float)dh); a.err_flag = c.st.counters + 2;
+    // two MMA groups per (128 queries x 128 keys): 4 * 128 * 128 * dh flops, over the causal half of the prompt
+    ProfScope ps(c, PC_ATTN_PROMPT, 0.0);
+    if (dh == 64) launch_attn_prompt_tc_dh<64>(c, a, tmq, l, r.groups);
+    else launch_attn_prompt_tc_dh<128>(c, a, tmq, l, r.groups);
+}
+
 template <typename T>
 void attention(tandem_ctx& c, const Model& m, int l, const T* q, T* o, const Rows& r) {
     const int d = m.d.d_model, H = m.d.n_heads, dh = d / H;
@@ -536,6 +567,10 @@ void attention(tandem_ctx& c, const Model& m, int l, const T* q, T* o, const Row
     aa.part_ml = at<float>(c, c.lay.part_ml); aa.part_acc = at<float>(c, c.lay.part_acc);
     aa.n_chunks_max = c.lay.n_chunks_max; aa.scale = 1.0f / sqrtf((float)dh);
     aa.merge_counters = at<int>(c, c.lay.attn_counters);
+    if (!r.decode && sizeof(T) == 2 && c.tc_prompt_attn && &m == &c.large) {
+        launch_attn_prompt_tc(c, l, reinterpret_cast<const bf16*>(q), reinterpret_cast<bf16*>(o), r);
+        return;
+    }
     if (r.decode && sizeof(T) == 2 && r.groups <= 65535) launch_attn_decode(c, dh, aa, r.groups, r.kv_positions * 2.0 * d * sizeof(T));
     else launch_attn<T>(c, dh, aa, r.groups, !r.decode, r.n_chunks, r.kv_positions * 2.0 * d * sizeof(T));
 }
@@ -1014,8 +1049,21 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
             return TANDEM_ERR_CUDA;
         }
         c->tc = true;
+        const int dhL = cfg->large.d_model / cfg->large.n_heads;
+        if ((dhL == 64 || dhL == 128) && getenv("TANDEM_NO_TC_ATTN") == nullptr) {
+            c->kmap.resize(cfg->large.n_layers);
+            c->vmap.resize(cfg->large.n_layers);
+            bool okm = true;
+            const uint64_t kv_rows = (uint64_t)cfg->max_batch * cfg->large.n_heads * cfg->max_seq;
+            for (int l = 0; l < cfg->large.n_layers && okm; ++l)
+                okm = make_tmap_bf16(&c->kmap[l], kv_ptr<bf16>(*c, c->large, l, 0), kv_rows, (uint64_t)dhL, (uint64_t)dhL) &&
+                      make_tmap_bf16(&c->vmap[l], kv_ptr<bf16>(*c, c->large, l, 1), kv_rows, (uint64_t)dhL, (uint64_t)dhL);
+            if (okm) { c->tc_prompt_attn = true; c->prompt_group = ATC_Q; }
+        }
     }
     if (e == cudaSuccess) e = cudaMemsetAsync(c->arena + lay.st_n, 0, lay.h_large - lay.st_n, c->stream);
+    // positions nobody has written yet are read (and masked, or weighted by zero) by chunked attention: keep them finite
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->arena + lay.kv_large, 0, lay.st_n - lay.kv_large, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "%s in tandem_create", cudaGetErrorString(e));
@@ -1080,7 +1128,7 @@ extern "C" tandem_status tandem_prefill(tandem_ctx* c, int32_t batch, const int3
     for (int b = 0; b < batch; ++b) {
         const int len = prompt_lens[b];
         for (int p = 0; p < len - 1; ++p) {
-            if (p % ATT_NQ == 0) { p_g0[groups] = m; p_gc[groups] = std::min(ATT_NQ, len - 1 - p); ++groups; }
+            if (p % c->prompt_group == 0) { p_g0[groups] = m; p_gc[groups] = std::min(c->prompt_group, len - 1 - p); ++groups; }
             p_tok[m] = prompt_ids[off + p]; p_seq[m] = b; p_pos[m] = p; ++m;
         }
         p_n[b] = len;

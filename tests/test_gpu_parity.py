@@ -206,6 +206,20 @@ def test_bf16_toy_replay_within_tolerance():
     assert flips <= 6
 
 
+@pytest.mark.parametrize("heads_large,heads_small", [(4, 2), (2, 1)])
+def test_bf16_prompt_attention_on_tensor_cores_replay(heads_large, heads_small):
+    """Head sizes 64 and 128 (the tensor-core prompt attention), ragged prompts that span several 128-query tiles
+    and 128-key chunks: logits of the following iterations, accept lengths and counts against the checker."""
+    shape = gpu_toy_shape(dtype=synth.DTYPE_BF16, layer_map=(1, 2), max_pos=400, large=(2, 256, heads_large, 512),
+                          small=(2, 128, heads_small, 256), vocab=211)
+    w = toy_weights(shape, seed=41, std=0.05)
+    for k in w:
+        if not synth.is_norm_param(k):
+            w[k] = synth.round_to_bf16(w[k])
+    flips = _replay_compare(shape, w, prompts_for(shape, [5, 140, 300, 1, 129], seed=8), 3, 3, TOL_BF16, 2 * TOL_BF16)
+    assert flips <= 8
+
+
 def test_bf16_small_config_widths_replay():
     """Config "small" (12x1024 / 4x512, vocab 32000, bf16) with a shortened prompt so the checker stays fast."""
     shape = synth.named_config("small", max_pos=192)
