@@ -206,6 +206,19 @@ def cpu_baseline(shape, weights, prompt, gamma, new):
                        f"({t2 - t1:.1f} s), decode time scaled to {new} tokens; numpy fp64 with its BLAS threads")}
 
 
+def replicas_throughput(local_ms_per_step, units_per_rank, world, device=None):
+    """Whole-job throughput of independent replicas: every rank processes `units_per_rank` units per step, the job
+    takes as long as its slowest rank (MAX over ranks of the per-step time); returns (units / s, that time in ms)."""
+    ms = float(local_ms_per_step)
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        tm = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        ms = float(tm.item())
+    return world * units_per_rank / (ms * 1e-3), ms
+
+
 def run_micro(args):
     """Kernel micro-benchmark: small-model decode attention (16 heads x 64, one query per (sequence, head)) over a
     large-derived context of T positions plus 4 own positions, and the FF_Tandem projection 4096 -> 1024 with
@@ -339,12 +352,7 @@ def main():
     total_ms = ev[0].elapsed_time(ev[-1])
     prefill_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(args.steps)) / args.steps
     decode_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(args.steps)) / args.steps
-    ms_per_step = total_ms / args.steps
-    if world > 1:
-        tm = torch.tensor([ms_per_step], device="cuda")
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        ms_per_step = float(tm.item())
-    value = world * B * new / (ms_per_step * 1e-3)
+    value, ms_per_step = replicas_throughput(total_ms / args.steps, B * new, world, "cuda")
 
     # ---- end to end through the public calls with host buffers, wall clock, copies included ----
     barrier()
@@ -352,15 +360,12 @@ def main():
     for k in range(args.steps):
         out, lens, stats = step()
     torch.cuda.synchronize()
-    e2e_sec = (time.perf_counter() - t0) / args.steps
-    if world > 1:
-        tm = torch.tensor([e2e_sec], device="cuda")
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        e2e_sec = float(tm.item())
+    e2e_value, _ = replicas_throughput(1e3 * (time.perf_counter() - t0) / args.steps, B * new, world, "cuda")
     rows = B * (P - 1)
-    h2d = 4 * (3 * rows + 2 * (rows // 16 + B) + 2 * B)          # row token/sequence/position, query groups, n, pending
+    group = 128 if shape.dtype == synth.DTYPE_BF16 else 16       # queries per attention group of the prompt pass
+    h2d = 4 * (3 * rows + 2 * (rows // group + B) + 2 * B)       # row token/sequence/position, query groups, n, pending
     d2h = 4 * (B * new + B + 16) + stats["iterations"] * 20      # tokens, lengths, histogram; 5 counters per iteration
-    e2e = {"value": world * B * new / e2e_sec, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -65,6 +65,18 @@ __device__ __forceinline__ float warp_max(float v) {
 }
 
 __device__ __forceinline__ float gelu_exact(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f)); }
+// The same GELU with erf from the classical five-term rational approximation (Abramowitz & Stegun 7.1.26,
+// absolute error below 1.5e-7) and the hardware exponential: for outputs that are rounded to bf16 anyway.
+__device__ __forceinline__ float gelu_bf16_out(float x) {
+    const float z = fabsf(x) * 0.70710678118654752440f;
+    const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float erf_abs = 1.0f - poly * t * __expf(-z * z);
+    return 0.5f * x * (1.0f + copysignf(erf_abs, x));
+}
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
     const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));

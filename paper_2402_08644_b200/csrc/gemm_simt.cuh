@@ -44,7 +44,7 @@ __device__ __forceinline__ void epilogue(const EpiArgs& e, int m, int n, float v
     } else if (EPI == EPI_STORE_F32) {
         static_cast<float*>(e.out)[(size_t)m * e.ldo + n] = v;
     } else if (EPI == EPI_GELU) {
-        static_cast<T*>(e.out)[(size_t)m * e.ldo + n] = from_float<T>(gelu_exact(v));
+        static_cast<T*>(e.out)[(size_t)m * e.ldo + n] = from_float<T>(sizeof(T) == 2 ? gelu_bf16_out(v) : gelu_exact(v));
     } else if (EPI == EPI_RESID) {
         float* p = static_cast<float*>(e.out) + (size_t)m * e.ldo + n;
         *p = *p + v;

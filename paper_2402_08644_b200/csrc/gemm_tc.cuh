@@ -519,10 +519,10 @@ __device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int seg, int
     }
     uint4 lo, hi;
     if (EPI == EPI_GELU) {
-        lo.x = pack_bf16x2(gelu_exact(v[0]), gelu_exact(v[1])); lo.y = pack_bf16x2(gelu_exact(v[2]), gelu_exact(v[3]));
-        lo.z = pack_bf16x2(gelu_exact(v[4]), gelu_exact(v[5])); lo.w = pack_bf16x2(gelu_exact(v[6]), gelu_exact(v[7]));
-        hi.x = pack_bf16x2(gelu_exact(v[8]), gelu_exact(v[9])); hi.y = pack_bf16x2(gelu_exact(v[10]), gelu_exact(v[11]));
-        hi.z = pack_bf16x2(gelu_exact(v[12]), gelu_exact(v[13])); hi.w = pack_bf16x2(gelu_exact(v[14]), gelu_exact(v[15]));
+        lo.x = pack_bf16x2(gelu_bf16_out(v[0]), gelu_bf16_out(v[1])); lo.y = pack_bf16x2(gelu_bf16_out(v[2]), gelu_bf16_out(v[3]));
+        lo.z = pack_bf16x2(gelu_bf16_out(v[4]), gelu_bf16_out(v[5])); lo.w = pack_bf16x2(gelu_bf16_out(v[6]), gelu_bf16_out(v[7]));
+        hi.x = pack_bf16x2(gelu_bf16_out(v[8]), gelu_bf16_out(v[9])); hi.y = pack_bf16x2(gelu_bf16_out(v[10]), gelu_bf16_out(v[11]));
+        hi.z = pack_bf16x2(gelu_bf16_out(v[12]), gelu_bf16_out(v[13])); hi.w = pack_bf16x2(gelu_bf16_out(v[14]), gelu_bf16_out(v[15]));
     } else {
         lo.x = pack_bf16x2(v[0], v[1]); lo.y = pack_bf16x2(v[2], v[3]); lo.z = pack_bf16x2(v[4], v[5]); lo.w = pack_bf16x2(v[6], v[7]);
         hi.x = pack_bf16x2(v[8], v[9]); hi.y = pack_bf16x2(v[10], v[11]); hi.z = pack_bf16x2(v[12], v[13]); hi.w = pack_bf16x2(v[14], v[15]);
