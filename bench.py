@@ -270,6 +270,16 @@ def run_micro(args):
             byt = (dS * dL + 2 * dS * dS) * 2 + rows * (dL + 2 * dS) * 2
             out["ff_tandem_project"].append({"rows": rows, "us": ms * 1e3, "algorithmic_bytes": byt, "gbs": byt / ms / 1e6,
                                              "frac": byt / ms / 1e6 / peak})
+        # the streaming GEMM alone at the feed-forward shapes of the four configurations, 4 token rows
+        out["block_linear"] = []
+        for K, N in ((512, 2048), (1024, 4096), (2048, 8192), (4096, 11008), (11008, 4096), (4096, 32000)):
+            x, w = rn(4, K), rn(N, K) * 0.02
+            y = torch.empty(4, N, dtype=torch.bfloat16, device=dev)
+            ms = timed(lambda: binding.tandem_block_linear(x, w, y))
+            byt = 2 * N * K + 2 * 4 * (K + N)
+            out["block_linear"].append({"rows": 4, "in": K, "out": N, "us": ms * 1e3, "algorithmic_bytes": byt,
+                                        "gbs": byt / ms / 1e6, "frac": byt / ms / 1e6 / peak})
+            del x, w, y
     print(json.dumps(out))
 
 

@@ -254,6 +254,15 @@ TANDEM_API tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
                                        void* scratch, size_t scratch_bytes, int32_t rows, int32_t d_large,
                                        int32_t d_small, void* stream);
 
+/* tandem_block_linear: y = x W^T for a block of few token rows, the streaming GEMM behind every projection and
+ * feed-forward map of the draft steps and the block pass (Section 3 "Inference": the large model processes the
+ * gamma+1 tokens of a block together so that each weight is read once for all of them).  All pointers DEVICE,
+ * 16-byte aligned, bf16:  x [rows][in_features];  w [out_features][in_features];  y [rows][out_features].
+ * 1 <= rows <= 64; in_features a multiple of 8.  Needs no work space: the K-slices of an output tile are summed
+ * through the shared memory of a thread-block cluster. */
+TANDEM_API tandem_status tandem_block_linear(const void* x, const void* w, void* y, int32_t rows, int32_t in_features,
+                                             int32_t out_features, void* stream);
+
 TANDEM_API const char* tandem_status_string(tandem_status s);
 /* Name of the last failing CUDA call's error for this thread (valid after TANDEM_ERR_CUDA). */
 TANDEM_API const char* tandem_last_cuda_error(void);

@@ -26,7 +26,7 @@ STATUS_NAMES = ["OK", "INVALID_ARG", "SHAPE", "ARENA_TOO_SMALL", "CAPACITY", "ST
 EXPORTS = ["tandem_query_arena", "tandem_create", "tandem_destroy", "tandem_prefill", "tandem_block_step",
            "tandem_speculative_generate", "tandem_large_greedy_generate", "tandem_debug_read",
            "tandem_decode_attention_scratch_bytes", "tandem_decode_attention", "tandem_ff_tandem_project",
-           "tandem_ff_tandem_project_scratch_bytes",
+           "tandem_ff_tandem_project_scratch_bytes", "tandem_block_linear",
            "tandem_status_string", "tandem_last_cuda_error", "tandem_profile_enable", "tandem_profile_read",
            "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static"]
 
@@ -92,6 +92,7 @@ def load_library():
     lib.tandem_decode_attention_scratch_bytes.restype = sz
     lib.tandem_decode_attention.argtypes = [vp] * 7 + [sz] + [i32] * 5 + [vp]
     lib.tandem_ff_tandem_project.argtypes = [vp] * 9 + [sz] + [i32] * 3 + [vp]
+    lib.tandem_block_linear.argtypes = [vp] * 3 + [i32] * 3 + [vp]
     lib.tandem_ff_tandem_project_scratch_bytes.argtypes = [i32] * 2
     lib.tandem_ff_tandem_project_scratch_bytes.restype = sz
     lib.tandem_decode_attention_static.argtypes = [vp] * 6 + [i32] * 5 + [vp]
@@ -104,7 +105,7 @@ def load_library():
         fn = getattr(lib, name)
         if name.endswith("_string") or name.endswith("_cuda_error") or name.endswith("_class_name"):
             fn.restype = C.c_char_p
-        elif name not in ("tandem_decode_attention_scratch_bytes", "tandem_ff_tandem_project_scratch_bytes",
+        elif name not in ("tandem_decode_attention_scratch_bytes", "tandem_ff_tandem_project_scratch_bytes", "tandem_block_linear",
                           "tandem_launch_count"):
             fn.restype = C.c_int
     lib.tandem_status_string.argtypes = [C.c_int]
@@ -323,3 +324,17 @@ def tandem_ff_tandem_project(x, w_t, ln_g, ln_b, wk, wv, scratch=None):
                                         C.c_void_p(torch.cuda.current_stream(x.device).cuda_stream or None)),
            "tandem_ff_tandem_project")
     return k, v
+
+
+def tandem_block_linear(x, w, y=None):
+    """x [rows][K] bf16, w [N][K] bf16 -> y [rows][N] bf16 (rows <= 64)."""
+    import torch
+    lib = load_library()
+    rows, k = x.shape
+    n = w.shape[0]
+    if y is None:
+        y = torch.empty(rows, n, dtype=torch.bfloat16, device=x.device)
+    _check(lib.tandem_block_linear(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()), rows, k, n,
+                                   C.c_void_p(torch.cuda.current_stream(x.device).cuda_stream or None)),
+           "tandem_block_linear")
+    return y

@@ -1551,3 +1551,23 @@ extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
     }
     return check_launch();
 }
+
+extern "C" tandem_status tandem_block_linear(const void* x, const void* w, void* y, int32_t rows, int32_t in_features,
+                                             int32_t out_features, void* stream) {
+    if (!x || !w || !y) return TANDEM_ERR_INVALID_ARG;
+    if (rows < 1 || rows > 64 || in_features < 8 || out_features < 1) return TANDEM_ERR_INVALID_ARG;
+    if (in_features % 8) return TANDEM_ERR_SHAPE;
+    if (((uintptr_t)x | (uintptr_t)w | (uintptr_t)y) & 15) return TANDEM_ERR_INVALID_ARG;
+    tandem_ctx tmp;   // only the stream, the launch counter and the launch options are used by the launch helpers
+    tmp.stream = static_cast<cudaStream_t>(stream);
+    tmp.use_pdl = false;
+    TcW tw;
+    if (!make_tmap_bf16(&tw.tm[0], w, (uint64_t)out_features, (uint64_t)in_features, (uint64_t)in_features)) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled unavailable or failed");
+        return TANDEM_ERR_CUDA;
+    }
+    tw.tm[1] = tw.tm[2] = tw.tm[0]; tw.n_segs = 1; tw.seg_rows = out_features; tw.K = in_features;
+    TcScratch ts; ts.err = nullptr;
+    launch_tc_decode<PRO_BF16, EPI_STORE>(tmp, ts, x, in_features, nullptr, nullptr, rows, tw, true, epi_plain(y, out_features));
+    return check_launch();
+}

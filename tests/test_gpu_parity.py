@@ -300,6 +300,21 @@ def test_ff_tandem_project_matches_oracle(rows, dL, dS):
     assert np.abs(v.float().cpu().numpy() - a @ f(wv).T).max() < TOL_BF16
 
 
+@pytest.mark.parametrize("rows,K,N", [(1, 64, 128), (4, 1024, 1024), (3, 136, 97), (16, 512, 1536), (17, 4096, 640),
+                                      (33, 264, 1000), (48, 2048, 384), (64, 1024, 4096), (5, 8, 8), (4, 11008, 256)])
+def test_block_linear_matches_matmul(rows, K, N):
+    """The streaming tensor-core GEMM alone: every token-column width (16 / 32 / 48 / 64), ragged tiles along the
+    output features and along K, one K-slice up to clusters of eight, against a float64 product of the same bf16 inputs."""
+    import torch
+    g = torch.Generator().manual_seed(rows * 7 + N)
+    x = torch.randn(rows, K, generator=g).to(torch.bfloat16)
+    w = (torch.randn(N, K, generator=g) * 0.05).to(torch.bfloat16)
+    y = binding.tandem_block_linear(x.cuda(), w.cuda()).float().cpu().numpy()
+    want = x.double().numpy() @ w.double().numpy().T
+    scale = max(1.0, float(np.abs(want).max()))
+    assert np.abs(y - want).max() <= 8e-3 * scale      # bf16 rounding of the output (2^-8 relative)
+
+
 # ------------------------------------------------------------------------------------------------
 # error behaviour: validated on the host, nothing launched
 # ------------------------------------------------------------------------------------------------
