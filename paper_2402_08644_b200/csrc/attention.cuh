@@ -355,6 +355,71 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
             const int t0 = (rank + it * CL) * ATT_CH + warp * ATD_WROWS;
             const bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
             const bf16* vs = ks + C::TILE_ELEMS;
+            if constexpr (QG == 4) {
+                // Four queries: the DH/8 lanes of a key split the four dot products among themselves while they add
+                // them up (a reduce-scatter with the same pairing, hence the same bits, as the one-query butterfly):
+                // the lane whose low position bits are (b0, b1) ends up with query 2*b0 + b1 and does that query's
+                // softmax step; probabilities and rescale factors are then handed round within the key's lanes.
+                const bool b0 = (part & 1) != 0, b1 = (part & 2) != 0;
+                const int qsel = (b0 ? 2 : 0) + (b1 ? 1 : 0);
+                const int key_lane0 = lane & ~(C::TPK - 1);
+                const bool q_live = q0 + qsel < cnt;
+                const int q_pos = pos_first + q0 + qsel;
+                float sp[C::PPW];
+                float mcm = -INFINITY;
+#pragma unroll
+                for (int p = 0; p < C::PPW; ++p) {
+                    const int key = p * C::KPW + kslot;
+                    float kf[8];
+                    load_vec(ks + key * DH + part * 8, kf);
+                    float d[4];
+#pragma unroll
+                    for (int qi = 0; qi < 4; ++qi) {
+                        d[qi] = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) d[qi] = fmaf(qreg[qi][j], kf[j], d[qi]);
+                    }
+                    const float r0 = __shfl_xor_sync(0xffffffffu, b0 ? d[0] : d[2], 1);
+                    const float r1 = __shfl_xor_sync(0xffffffffu, b0 ? d[1] : d[3], 1);
+                    const float e0 = (b0 ? d[2] : d[0]) + r0, e1 = (b0 ? d[3] : d[1]) + r1;
+                    const float r2 = __shfl_xor_sync(0xffffffffu, b1 ? e0 : e1, 2);
+                    float dq = (b1 ? e1 : e0) + r2;
+#pragma unroll
+                    for (int o = 4; o < C::TPK; o <<= 1) dq += __shfl_xor_sync(0xffffffffu, dq, o);
+                    sp[p] = (q_live && t0 + key <= q_pos) ? dq * a.scale : -INFINITY;
+                    mcm = fmaxf(mcm, sp[p]);
+                }
+#pragma unroll
+                for (int o = C::TPK; o < 32; o <<= 1) mcm = fmaxf(mcm, __shfl_xor_sync(0xffffffffu, mcm, o));
+                const float mn = fmaxf(m[0], mcm);
+                const float fm = m[0] > -INFINITY ? __expf(m[0] - mn) : 0.f;
+                m[0] = mn;
+                float ls = 0.f;
+#pragma unroll
+                for (int p = 0; p < C::PPW; ++p) {
+                    sp[p] = mn > -INFINITY ? __expf(sp[p] - mn) : 0.f;
+                    ls += sp[p];
+                }
+                l[0] = l[0] * fm + ls;   // this lane's keys only; the key slots are added up at the end
+#pragma unroll
+                for (int qi = 0; qi < 4; ++qi) {
+                    const float fq = __shfl_sync(0xffffffffu, fm, key_lane0 | ((qi >> 1) | ((qi & 1) << 1)));
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc[qi][j] *= fq;
+                }
+#pragma unroll
+                for (int p = 0; p < C::PPW; ++p) {
+                    const int key = p * C::KPW + kslot;
+                    float vf[8];
+                    load_vec(vs + key * DH + part * 8, vf);
+#pragma unroll
+                    for (int qi = 0; qi < 4; ++qi) {
+                        const float pq = __shfl_sync(0xffffffffu, sp[p], key_lane0 | ((qi >> 1) | ((qi & 1) << 1)));
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) acc[qi][j] = fmaf(pq, vf[j], acc[qi][j]);
+                    }
+                }
+            } else {
             float sc[QG][C::PPW], mc[QG];
 #pragma unroll
             for (int qi = 0; qi < QG; ++qi) mc[qi] = -INFINITY;
@@ -403,15 +468,24 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) acc[qi][j] = fmaf(sc[qi][p], vf[j], acc[qi][j]);
             }
+            }
             __syncwarp();   // the stage may be refilled by this warp's next issue
             if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(8);
         }
         // the warp's state: add up its key slots (lanes that share `part`), lanes 0 .. TPK-1 publish it
+        if constexpr (QG == 4) {   // each lane carries the running maximum and sum of one query only
+#pragma unroll
+            for (int o = C::TPK; o < 32; o <<= 1) l[0] += __shfl_xor_sync(0xffffffffu, l[0], o);
+            if (lane < 4) {        // lane = position bits (b0, b1) of key slot 0: query 2*b0 + b1
+                float* st = wst + (size_t)(warp * QG + (((lane & 1) << 1) | (lane >> 1))) * (DH + 2);
+                st[DH] = m[0]; st[DH + 1] = l[0];
+            }
+        }
 #pragma unroll
         for (int qi = 0; qi < QG; ++qi) {
 #pragma unroll
             for (int o = C::TPK; o < 32; o <<= 1) {
-                l[qi] += __shfl_xor_sync(0xffffffffu, l[qi], o);
+                if (QG != 4) l[qi] += __shfl_xor_sync(0xffffffffu, l[qi], o);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[qi][j] += __shfl_xor_sync(0xffffffffu, acc[qi][j], o);
             }
@@ -419,7 +493,7 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
                 float* st = wst + (size_t)(warp * QG + qi) * (DH + 2);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) st[lane * 8 + j] = acc[qi][j];
-                if (lane == 0) { st[DH] = m[qi]; st[DH + 1] = l[qi]; }
+                if (QG != 4 && lane == 0) { st[DH] = m[qi]; st[DH + 1] = l[qi]; }
             }
         }
         __syncthreads();
