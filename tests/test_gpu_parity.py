@@ -228,6 +228,23 @@ def test_bf16_small_config_widths_replay():
     assert flips <= 3
 
 
+@pytest.mark.parametrize("large,small,batch_lens", [
+    ((2, 2048, 16, 8192), (2, 768, 12, 3072), [70, 33, 9]),        # "medium" widths (head size 128 / 64), batch 3
+    ((1, 4096, 32, 11008), (1, 1024, 16, 4096), [150]),            # "large" widths, batch 1
+])
+def test_bf16_medium_and_large_widths_replay(large, small, batch_lens):
+    """Full widths of the two bigger configurations with few layers and short prompts, so the checker stays fast:
+    rows longer than 1024 (LayerNorm kernel ahead of the GEMMs), 128-wide heads, K up to 11008, vocabulary 32000."""
+    shape = gpu_toy_shape(dtype=synth.DTYPE_BF16, layer_map=None, max_pos=192, large=large, small=small, vocab=32000)
+    w = synth.make_weights(shape, seed=9)
+    # A logit is a sum of d products whose bf16 operand carries a relative rounding error of 2^-9: its absolute error
+    # grows like sqrt(d), and the maximum is taken over 4 x 32000 logits per sequence.  2e-2 is the bound at the
+    # 1024-wide model it was stated for; wider models get the same bound scaled by sqrt(d / 1024).
+    tol = TOL_BF16 * (large[1] / 1024.0) ** 0.5
+    flips = _replay_compare(shape, w, prompts_for(shape, batch_lens, seed=3), 3, 2, tol, 2 * tol)
+    assert flips <= 4
+
+
 @pytest.mark.parametrize("dtype", [synth.DTYPE_FP32, synth.DTYPE_BF16])
 def test_gpu_speed_equals_gpu_greedy_bit_exact(dtype):
     """On the GPU itself: Tandem + SPEED (block passes of gamma+1 rows, ragged rollback) returns exactly the
