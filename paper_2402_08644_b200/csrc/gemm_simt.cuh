@@ -24,6 +24,8 @@ struct EpiArgs {
     const int* row_pos;   // [M] absolute position of each row
     int n_heads, d_head, t_max;
     int seg;              // columns per segment (= d_model) for QKV / KV
+    void* snap;           // EPI_RESID on the tensor-core decode path: optional bf16 copy of the new values [M][snap_ld]
+    int snap_ld;
 };
 
 struct WSegs {            // up to three weight matrices stacked along N, each [seg_rows][K]

@@ -422,7 +422,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 float* out = static_cast<float*>(a.e.out);
 #pragma unroll
                 for (int j = 0; j < NB; ++j)
-                    if (j < a.rows && valid) out[(size_t)j * a.e.ldo + n] = hres[j] + v[j];
+                    if (j < a.rows && valid) {
+                        const float hv = hres[j] + v[j];
+                        out[(size_t)j * a.e.ldo + n] = hv;
+                        if (a.e.snap) static_cast<bf16*>(a.e.snap)[(size_t)j * a.e.snap_ld + n] = __float2bfloat16_rn(hv);
+                    }
             } else if (EPI == EPI_QKV || EPI == EPI_KV) {
                 const ScatterCol sc = scatter_col<EPI>(a.e, seg, n_local);
 #pragma unroll
@@ -464,8 +468,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                     float acc = 0.f;
 #pragma unroll
                     for (int ss = 0; ss < 8; ++ss) if (ss < S) acc += inbox[(ss * NB + j) * CW + cw];   // slice order
-                    if (EPI == EPI_RESID) static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = hres[it] + acc;
-                    else if (EPI == EPI_QKV || EPI == EPI_KV)
+                    if (EPI == EPI_RESID) {
+                        const float hv = hres[it] + acc;
+                        static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = hv;
+                        if (a.e.snap) static_cast<bf16*>(a.e.snap)[(size_t)j * a.e.snap_ld + n] = __float2bfloat16_rn(hv);
+                    } else if (EPI == EPI_QKV || EPI == EPI_KV)
                         sc.base[(sc.is_q ? (long long)j * a.e.ldo : s_rowoff[j]) + sc.col] = __float2bfloat16_rn(acc);
                     else epilogue<bf16, EPI>(a.e, j, n, acc);
                 }

@@ -83,7 +83,7 @@ template <typename T>
 __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, int nq, int fin_r, const float* amax_val,
                                                          const int* amax_idx, int amax_stride, int n_tiles, int* row_tok,
                                                          int* row_seq, int* row_pos, const T* __restrict__ emb,
-                                                         const T* __restrict__ pos, float* __restrict__ h, int d) {
+                                                         const T* __restrict__ pos, float* __restrict__ h, int d, bf16* snap) {
     __shared__ int s_tok, s_pos;
     TC_PROBE_INIT(300);
     pdl_wait();
@@ -106,7 +106,11 @@ __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, i
     __syncthreads();
     const T* er = emb + (size_t)s_tok * d;
     const T* pr = pos + (size_t)s_pos * d;
-    for (int i = threadIdx.x; i < d; i += 128) h[(size_t)m * d + i] = to_float(er[i]) + to_float(pr[i]);
+    for (int i = threadIdx.x; i < d; i += 128) {
+        const float v = to_float(er[i]) + to_float(pr[i]);
+        h[(size_t)m * d + i] = v;
+        if (snap) snap[(size_t)m * d + i] = __float2bfloat16_rn(v);   // bf16 copy for the FF_Tandem projection of x^(0)
+    }
     if (threadIdx.x == 0) TC_PROBE(2);
 }
 

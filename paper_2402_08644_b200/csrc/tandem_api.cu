@@ -51,6 +51,7 @@ struct Layout {   // byte offsets into the arena
     size_t attn_counters;   // inside the zero-filled state block
     size_t h_large, h_small, a, q, o, f, xb, t1, yhat, a_s, logits_large, logits_small, part_ml, part_acc, dbg;
     size_t amax_val_large, amax_idx_large, amax_val_small, amax_idx_small;
+    size_t proj_snap, proj_yhat, proj_a, proj_t1;   // per small layer: the decode projection's own buffers (it runs beside the large pass)
     size_t total;
     int max_rows, dec_rows, max_groups, n_chunks_max, vocab_tiles;
     size_t kv_large_layer, kv_small_layer;   // elements per (layer, k-or-v)
@@ -118,6 +119,12 @@ struct tandem_ctx {
     std::vector<CUtensorMap> wmap;       // one per weight pointer (matrices only), box 128 rows x 64 columns
     std::vector<char> wmap_ok;
     std::vector<CUtensorMap> kmap, vmap; // the large model's key / value cache of each layer as [(seq, head, position)][d_head]
+    cudaStream_t side = nullptr;         // the decode-time FF_Tandem projections run here, beside the large model's later layers
+    std::vector<cudaEvent_t> ev_fork;    // one per small layer
+    cudaEvent_t ev_join = nullptr;
+    bool fork_projection = true;
+    bool next_launch_plain = false;      // the next launch follows a cross-stream wait: no programmatic dependency on a kernel
+    bool setup_failed = false;           // a launch helper could not encode a tensor map: reported by the enclosing call
     bool tc_prompt_attn = false;         // prompt attention on the tensor cores (head size 64 or 128)
     int prompt_group = ATT_NQ;           // queries per attention group of the prompt pass
 };
@@ -209,6 +216,11 @@ Layout make_layout(const tandem_config& c) {
     L.vocab_tiles = cdiv(c.large.vocab, 128);
     L.amax_val_large = take(RD * L.vocab_tiles * 4); L.amax_idx_large = take(RD * L.vocab_tiles * 4);
     L.amax_val_small = take(B * L.vocab_tiles * 4); L.amax_idx_small = take(B * L.vocab_tiles * 4);
+    const size_t nS = c.small.n_layers;
+    L.proj_snap = take(nS * RD * c.large.d_model * 2);
+    L.proj_yhat = take(nS * RD * c.small.d_model * 4);
+    L.proj_a = take(nS * RD * c.small.d_model * 2);
+    L.proj_t1 = take(nS * RD * hidden * 2);
     L.total = off;
     return L;
 }
@@ -323,7 +335,9 @@ void launch_ex(tandem_ctx& c, bool pdl, int cluster, void (*kernel)(KArgs...), d
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c.stream;
     cudaLaunchAttribute attr[2];
     int n = 0;
-    if (pdl && c.use_pdl) {
+    const bool plain = c.next_launch_plain;
+    c.next_launch_plain = false;
+    if (pdl && c.use_pdl && !plain) {
         attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n].val.programmaticStreamSerializationAllowed = 1;
         ++n;
@@ -428,7 +442,9 @@ void launch_gemm(tandem_ctx& c, bool decode, const T* x, int ldx, int M, const L
         else if (M <= 4) launch_smallm<T, 4, EPI>(c, x, ldx, M, K, ws, N, e);
         else launch_smallm<T, 8, EPI>(c, x, ldx, M, K, ws, N, e);
     } else if (sizeof(T) == 2 && c.tc) {
-        launch_tc_tiled<EPI>(c, reinterpret_cast<const bf16*>(x), ldx, M, tcw(c, l.i0, l.i1, l.i2, l.seg_rows, l.K), e, c.st.counters + 2);
+        if (launch_tc_tiled<EPI>(c, reinterpret_cast<const bf16*>(x), ldx, M, tcw(c, l.i0, l.i1, l.i2, l.seg_rows, l.K), e,
+                                 c.st.counters + 2) != TANDEM_OK)
+            c.setup_failed = true;
     } else {
         dim3 grid(cdiv(N, GT_BN), cdiv(M, GT_BM));
         ProfScope ps(c, PC_GEMM_TILED, 2.0 * M * (double)N * K);   // flops, not bytes: this one is compute-bound
@@ -544,7 +560,11 @@ void launch_attn_prompt_tc_dh(tandem_ctx& c, const AttnTcArgs& a, const CUtensor
 void launch_attn_prompt_tc(tandem_ctx& c, int l, const bf16* q, bf16* o, const Rows& r) {
     const int d = c.large.d.d_model, H = c.large.d.n_heads, dh = d / H;
     CUtensorMap tmq;
-    if (!make_tmap_bf16(&tmq, q, (uint64_t)r.M, (uint64_t)d, (uint64_t)d)) return;   // cannot fail once the weights' maps were made
+    if (!make_tmap_bf16(&tmq, q, (uint64_t)r.M, (uint64_t)d, (uint64_t)d)) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed for the query buffer");
+        c.setup_failed = true;
+        return;
+    }
     AttnTcArgs a;
     memset(&a, 0, sizeof(a));
     a.out = o; a.ldo = d; a.row_seq = at<int>(c, c.lay.row_seq); a.row_pos = at<int>(c, c.lay.row_pos);
@@ -721,12 +741,12 @@ void greedy_iteration(tandem_ctx& c, int max_new) {
 
 // Row set-up + embedding for block rows r0 .. r0+nq-1 of every sequence; fin_r: block row whose token is the
 // arg-max the small model's last head GEMM left as per-tile results (-1: none).
-void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r) {
+void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r, bf16* snap = nullptr) {
     ProfScope ps(c, PC_ROWS, (double)c.batch * nq * m.d.d_model * 8.0);
     launch_ex(c, true, 1, step_begin_kernel<bf16>, dim3(c.batch * nq), dim3(128), 0, c.st, r0, nq, fin_r,
               (const float*)at<float>(c, c.lay.amax_val_small), (const int*)at<int>(c, c.lay.amax_idx_small), c.lay.vocab_tiles,
               c.lay.vocab_tiles, at<int>(c, c.lay.row_tok), at<int>(c, c.lay.row_seq), at<int>(c, c.lay.row_pos),
-              (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model);
+              (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model, snap);
 }
 
 // Whether LayerNorm (or the fp32 -> bf16 cast) is fused into the GEMM's operand load.  Fused, every CTA of the
@@ -738,13 +758,13 @@ bool tc_fused_prologue(const tandem_ctx& c, int K) { return c.batch <= 2 && K <=
 // y = LayerNorm(h) W^T with the given epilogue; h fp32 [rows][K].
 template <int EPI>
 void tc_ln_gemm(tandem_ctx& c, const float* h, const void* ln_g, const void* ln_b, int rows, const TcW& w, bool stream_w,
-                const EpiArgs& e, float* amax_val = nullptr, int* amax_idx = nullptr, int amax_stride = 0) {
+                const EpiArgs& e, float* amax_val = nullptr, int* amax_idx = nullptr, int amax_stride = 0, bf16* ln_out = nullptr) {
     const TcScratch sc = tc_scratch(c);
     if (tc_fused_prologue(c, w.K)) {
         launch_tc_decode<PRO_LN, EPI>(c, sc, h, w.K, ln_g, ln_b, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
         return;
     }
-    bf16* a = at<bf16>(c, c.lay.a);
+    bf16* a = ln_out ? ln_out : at<bf16>(c, c.lay.a);
     {
         ProfScope ps(c, PC_LAYERNORM, (double)rows * w.K * 6.0);
         launch_ex(c, true, 1, layernorm_rows_bf16_kernel, dim3(rows), dim3(128), 0, h, static_cast<const float*>(ln_g),
@@ -753,7 +773,7 @@ void tc_ln_gemm(tandem_ctx& c, const float* h, const void* ln_g, const void* ln_
     launch_tc_decode<PRO_BF16, EPI>(c, sc, a, w.K, nullptr, nullptr, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
 }
 
-void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r, bool stream_w) {
+void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r, bool stream_w, bf16* snap = nullptr) {
     const int d = m.d.d_model, dff = m.d.d_ff;
     bf16* q = at<bf16>(c, c.lay.q);
     bf16* o = at<bf16>(c, c.lay.o);
@@ -766,8 +786,9 @@ void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows
                                           epi_plain(h, d));
     tc_ln_gemm<EPI_GELU>(c, h, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), r.M, tcw(c, wi_layer(m, l, W_W1), -1, -1, dff, d),
                          stream_w, epi_plain(f, dff));
-    launch_tc_decode<PRO_BF16, EPI_RESID>(c, sc, f, dff, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_W2), -1, -1, d, dff), stream_w,
-                                          epi_plain(h, d));
+    EpiArgs e2 = epi_plain(h, d);
+    e2.snap = snap; e2.snap_ld = d;   // bf16 copy of x^(l+1) when an FF_Tandem projection reads it
+    launch_tc_decode<PRO_BF16, EPI_RESID>(c, sc, f, dff, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_W2), -1, -1, d, dff), stream_w, e2);
 }
 
 // Final LayerNorm + output head; leaves fp32 logits and the per-tile (max, index) pairs that the next kernel
@@ -822,16 +843,75 @@ void tc_small_step(tandem_ctx& c, int s) {
     tc_head(c, c.small, y, r, logits, c.lay.amax_val_small, c.lay.amax_idx_small, false);
 }
 
+// The same projection on the side stream, from the bf16 copy `snap` of x^(l(j)) that the producing kernel left: it
+// depends on nothing the large model does afterwards (and nothing in the iteration depends on it before the next
+// draft), so it runs beside the large model's later layers instead of in their chain.
+void tc_project_forked(tandem_ctx& c, int n_large_layers_done, int slot, const Rows& r) {
+    const int dL = c.large.d.d_model, dS = c.small.d.d_model;
+    const TcScratch sc = tc_scratch(c);
+    const size_t RD = (size_t)c.lay.dec_rows;
+    const bf16* snap = at<bf16>(c, c.lay.proj_snap) + (size_t)slot * RD * dL;
+    cudaStream_t main_stream = c.stream;
+    cudaEventRecord(c.ev_fork[slot], main_stream);
+    cudaStreamWaitEvent(c.side, c.ev_fork[slot], 0);
+    c.stream = c.side;
+    c.next_launch_plain = true;   // first kernel after a cross-stream wait
+    for (int j = 0; j < c.small.d.n_layers; ++j) {
+        if (c.layer_map[j] != n_large_layers_done) continue;
+        float* yhat = at<float>(c, c.lay.proj_yhat) + (size_t)j * RD * dS;
+        bf16* a_j = at<bf16>(c, c.lay.proj_a) + (size_t)j * RD * dS;
+        if (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR) {
+            launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, snap, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, dS, dL), true,
+                                                      epi_plain(yhat, dS));
+        } else {
+            bf16* t1 = at<bf16>(c, c.lay.proj_t1) + (size_t)j * RD * c.hidden;
+            launch_tc_decode<PRO_BF16, EPI_GELU>(c, sc, snap, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, c.hidden, dL), true,
+                                                 epi_plain(t1, c.hidden));
+            launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, t1, c.hidden, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 1), -1, -1, dS, c.hidden),
+                                                      true, epi_plain(yhat, dS));
+        }
+        tc_ln_gemm<EPI_KV>(c, yhat, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), r.M,
+                           tcw(c, wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS), true, epi_cache<bf16>(c, c.small, j, nullptr),
+                           nullptr, nullptr, 0, a_j);
+    }
+    c.stream = main_stream;
+}
+
+// Slot of the projection buffers for the residual stream after `n` large layers: the first small layer fed from there, or -1.
+int project_slot(const tandem_ctx& c, int n) {
+    for (int j = 0; j < c.small.d.n_layers; ++j)
+        if (c.layer_map[j] == n) return j;
+    return -1;
+}
+
 void tc_large_block(tandem_ctx& c, int gamma, bool project) {
     float* h = at<float>(c, c.lay.h_large);
-    tc_begin(c, c.large, h, 0, gamma + 1, gamma > 0 ? gamma : -1);
+    const bool forked = project && c.fork_projection;
+    const size_t snap_elems = (size_t)c.lay.dec_rows * c.large.d.d_model;
+    auto snap_of = [&](int n) -> bf16* {
+        const int slot = forked ? project_slot(c, n) : -1;
+        return slot >= 0 ? at<bf16>(c, c.lay.proj_snap) + (size_t)slot * snap_elems : nullptr;
+    };
+    bool any_fork = false;
+    tc_begin(c, c.large, h, 0, gamma + 1, gamma > 0 ? gamma : -1, snap_of(0));
     const Rows r = decode_rows(c, gamma, gamma + 1);
-    if (project) tc_project_after(c, 0, r);
+    if (project) {
+        if (forked) { if (project_slot(c, 0) >= 0) { tc_project_forked(c, 0, project_slot(c, 0), r); any_fork = true; } }
+        else tc_project_after(c, 0, r);
+    }
     for (int l = 0; l < c.large.d.n_layers; ++l) {
-        tc_decoder_layer(c, c.large, l, h, r, true);
-        if (project) tc_project_after(c, l + 1, r);
+        tc_decoder_layer(c, c.large, l, h, r, true, snap_of(l + 1));
+        if (project) {
+            if (forked) { if (project_slot(c, l + 1) >= 0) { tc_project_forked(c, l + 1, project_slot(c, l + 1), r); any_fork = true; } }
+            else tc_project_after(c, l + 1, r);
+        }
     }
     tc_head(c, c.large, h, r, at<float>(c, c.lay.logits_large), c.lay.amax_val_large, c.lay.amax_idx_large, true);
+    if (any_fork) {   // the projections join the main stream before the verify kernel
+        cudaEventRecord(c.ev_join, c.side);
+        cudaStreamWaitEvent(c.stream, c.ev_join, 0);
+        c.next_launch_plain = true;
+    }
 }
 
 void tc_iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
@@ -851,6 +931,11 @@ tandem_status check_launch() {
     CK(cudaGetLastError());
     return TANDEM_OK;
 }
+// The same for a context: also reports a launch helper that had to skip its launch.
+tandem_status check_launch(tandem_ctx& c) {
+    if (c.setup_failed) { c.setup_failed = false; return TANDEM_ERR_CUDA; }
+    return check_launch();
+}
 
 void enqueue_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t seed, int max_new) {
     const bool bf = c.cfg.dtype == TANDEM_DTYPE_BF16;
@@ -867,6 +952,8 @@ void enqueue_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t se
 tandem_status launch_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t seed, int max_new) {
     const int need = (c.n_ub - 1 + gamma) / ATT_CH + 1;
     c.chunks_launch = std::min(c.lay.n_chunks_max, (need + 3) / 4 * 4);
+    if (c.cfg.dtype == TANDEM_DTYPE_BF16 && c.tc && tc_nb(c.batch * (gamma + 1)) != 0)
+        c.chunks_launch = 1;   // the cluster attention's grid does not depend on the context length: one graph serves all
     c.ticket++;
     if (c.prof.on || !c.use_graphs) {
         enqueue_iteration(c, kind, gamma, mode, seed, max_new);
@@ -972,6 +1059,15 @@ extern "C" tandem_status tandem_query_arena(const tandem_config* cfg, size_t* by
     return TANDEM_OK;
 }
 
+namespace {
+void release_side(tandem_ctx& c) {
+    for (cudaEvent_t ev : c.ev_fork) cudaEventDestroy(ev);
+    c.ev_fork.clear();
+    if (c.ev_join) { cudaEventDestroy(c.ev_join); c.ev_join = nullptr; }
+    if (c.side) { cudaStreamDestroy(c.side); c.side = nullptr; }
+}
+}  // namespace
+
 extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_weights* weights, void* arena,
                                        size_t arena_bytes, tandem_ctx** out) {
     if (!out || !weights || !weights->ptrs || !arena) return TANDEM_ERR_INVALID_ARG;
@@ -1016,6 +1112,14 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
         st.host_flags = dptr;
     }
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
+    for (int j = 0; j < cfg->small.n_layers && e == cudaSuccess; ++j) {
+        cudaEvent_t ev = nullptr;
+        e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e == cudaSuccess) c->ev_fork.push_back(ev);
+    }
+    c->fork_projection = getenv("TANDEM_NO_FORK") == nullptr;
     c->use_graphs = getenv("TANDEM_NO_GRAPH") == nullptr;
     c->use_pdl = getenv("TANDEM_NO_PDL") == nullptr;
     if (const char* t = getenv("TANDEM_TC_TARGET")) c->tc_target = std::max(1, atoi(t));
@@ -1045,6 +1149,7 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
             if (c->pinned) cudaFreeHost(c->pinned);
             if (c->hflags) cudaFreeHost(c->hflags);
             if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+            release_side(*c);
             delete c;
             return TANDEM_ERR_CUDA;
         }
@@ -1070,6 +1175,7 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
         if (c->pinned) cudaFreeHost(c->pinned);
         if (c->hflags) cudaFreeHost(c->hflags);
         if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+            release_side(*c);
         delete c;
         return TANDEM_ERR_CUDA;
     }
@@ -1086,6 +1192,7 @@ extern "C" tandem_status tandem_destroy(tandem_ctx* c) {
     for (auto& g : c->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
     if (c->hflags) cudaFreeHost(c->hflags);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
+    release_side(*c);
     delete c;
     if (e != cudaSuccess) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "%s in tandem_destroy", cudaGetErrorString(e));
@@ -1154,7 +1261,7 @@ extern "C" tandem_status tandem_prefill(tandem_ctx* c, int32_t batch, const int3
         if (c->cfg.dtype == TANDEM_DTYPE_BF16) large_pass<bf16>(*c, r, true, false);
         else large_pass<float>(*c, r, true, false);
     }
-    return check_launch();
+    return check_launch(*c);
 }
 
 namespace {
