@@ -220,8 +220,8 @@ def replicas_throughput(local_ms_per_step, units_per_rank, world, device=None):
 
 
 def run_micro(args):
-    """Kernel micro-benchmark: small-model decode attention (16 heads x 64, one query per (sequence, head)) over a
-    large-derived context of T positions plus 4 own positions, and the FF_Tandem projection 4096 -> 1024 with
+    """Kernel micro-benchmark: decode attention (16 heads x 64 as in the small models, and the large models' 128-wide
+    heads; one query per (sequence, head)) over a large-derived context of T positions plus 4 own positions, and the FF_Tandem projection 4096 -> 1024 with
     the key/value maps, through the stand-alone C entry points.  L2 is flushed between timed calls."""
     import torch
     from paper_2402_08644_b200 import binding, build as _build
@@ -244,20 +244,22 @@ def run_micro(args):
             ts.append(e0.elapsed_time(e1))
         return float(np.median(ts))
 
-    H, dh, To = 16, 64, 4
-    cases = [(B, T) for B in (1, 8, 32) for T in (1024, 8192, 32768)]
+    To = 4
+    cases = [(B, T, 16, 64) for B in (1, 8, 32) for T in (1024, 8192, 32768)]
+    cases += [(1, 8192, 32, 128), (4, 8192, 32, 128), (8, 2048, 16, 128)]    # the large models' head shapes (128-wide heads)
     if args.micro_case:
-        cases = [tuple(int(v) for v in args.micro_case.split(","))]
+        v = [int(x) for x in args.micro_case.split(",")]
+        cases = [(v[0], v[1], v[2] if len(v) > 2 else 16, v[3] if len(v) > 3 else 64)]
     out = {"metric": "decode_attention_gbs", "unit": "GB/s", "peak": peak, "peak_kind": peak_kind, "dtype": "bf16",
            "data": "synthetic N(0,1) queries, keys and values", "attention": [], "ff_tandem_project": []}
     rn = lambda *s: torch.randn(*s, generator=g, device=dev).to(torch.bfloat16)
-    for B, T in cases:
+    for B, T, H, dh in cases:
         q, kd, vd, ko, vo = rn(B, H, dh), rn(B, H, T, dh), rn(B, H, T, dh), rn(B, H, To, dh), rn(B, H, To, dh)
         o = torch.empty_like(q)
         scratch = torch.empty(1 << 20, dtype=torch.uint8, device=dev)
         ms = timed(lambda: binding.tandem_decode_attention(q, kd, vd, ko, vo, o, scratch))
         byt = 2 * B * H * (T + To) * dh * 2 + 2 * B * H * dh * 2
-        out["attention"].append({"batch": B, "derived_len": T, "own_len": To, "us": ms * 1e3, "algorithmic_bytes": byt,
+        out["attention"].append({"batch": B, "heads": H, "d_head": dh, "derived_len": T, "own_len": To, "us": ms * 1e3, "algorithmic_bytes": byt,
                                  "gbs": byt / ms / 1e6, "frac": byt / ms / 1e6 / peak})
         del q, kd, vd, ko, vo
     if not args.micro_case:
@@ -290,7 +292,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="small", choices=sorted(WORKLOADS) + ["micro"])
-    ap.add_argument("--micro-case", default="", help="with --workload micro: one attention case 'batch,context'")
+    ap.add_argument("--micro-case", default="", help="with --workload micro: one attention case 'batch,context[,heads,d_head]'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the accept-all / greedy / per-kernel passes")
     args = ap.parse_args()

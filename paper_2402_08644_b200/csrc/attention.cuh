@@ -232,13 +232,20 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
 
 // ---------------------------------------------------------------------------------------------------
 // Decode attention, bf16, built for short dependent chains and for streaming: a cluster of CL CTAs (1, 2, 4 or 8,
-// fixed per launch configuration) serves one (sequence, head).  CTA `rank` takes the 128-position chunks rank, rank + CL, ... (anchored at
-// absolute position 0); inside a chunk warp w owns positions 16w .. 16w+15.  Every warp runs on its own: it
-// fetches its rows through a private cp.async ring, keeps an online-softmax state per query in registers and
-// never waits for another warp until the end, where the CTA folds its warps' states in warp order, sends the
-// result to the CTA that finishes the query (remote shared-memory stores), and that CTA merges the CL
-// states in rank order.  No global scratch, no second kernel.  DH / 8 lanes share a key (16 bytes each); a
-// query's arithmetic does not depend on the other queries.  The probabilities use the fast exponential
+// fixed per launch configuration) serves one (sequence, head).  CTA `rank` takes the 128-position chunks rank,
+// rank + CL, ... (anchored at absolute position 0); inside a chunk warp w owns positions 16w .. 16w+15.  Every warp
+// runs on its own: it fetches its rows through a private cp.async ring, keeps the online-softmax state of all the
+// block's queries (up to 16) in registers and never waits for another warp until the end, where the CTA folds its
+// warps' states in warp order, sends the result to the CTA that finishes the query (remote shared-memory stores),
+// and that CTA merges the CL states in rank order.  No global scratch, no second kernel.
+//
+// The two small products of a 16-position tile, S = Q K^T (16 query rows x 16 keys) and O += P V, run on the tensor
+// cores as warp-level m16n8k16 MMAs: with scalar FMAs and shuffles a block of gamma+1 queries is bound by
+// instruction issue at well under half of the memory bandwidth.  The query rows are the MMA's A rows (absent rows
+// are zero), K and V fragments come straight from the ring with ldmatrix (V transposed on the way), the softmax
+// works on the accumulator fragments (a row's 16 scores sit in the four lanes of a quad), and each probability
+// enters the second product as two bf16 numbers (value and remainder).  An output row depends on its own query row
+// only, so a block pass and a one-row pass give the same bits.  The probabilities use the fast exponential
 // (2^x hardware approximation), well inside the bf16 tolerance.
 // ---------------------------------------------------------------------------------------------------
 constexpr int ATD_THREADS = 256;
@@ -246,49 +253,72 @@ constexpr int ATD_WARPS = ATD_THREADS / 32;
 constexpr int ATD_CLUSTER = 8;                                      // largest cluster; launches use 1, 2, 4 or 8
 constexpr int ATD_SLOTS = ATT_NQ;                                   // inbox states per CTA: cluster size x queries it finishes <= 16
 constexpr int ATD_WROWS = ATT_CH / ATD_WARPS;                       // positions of a chunk per warp (16)
+static_assert(ATD_WROWS == 16 && ATT_NQ == 16, "one m16n8k16 tile per warp and chunk");
 
 template <int DH> struct AtdCfg {
-    static constexpr int TPK = DH / 8;               // lanes per key
-    static constexpr int KPW = 32 / TPK;             // keys per warp pass
-    static constexpr int PPW = ATD_WROWS / KPW;      // passes per chunk
+    static constexpr int TPK = DH / 8;               // 16-byte units per key
     static constexpr int STAGES = DH <= 64 ? 3 : 2;
     static constexpr int TILE_ELEMS = ATD_WROWS * DH;   // a warp's keys (or values) of one chunk
     static constexpr int STAGE_ELEMS = 2 * TILE_ELEMS;
     static constexpr int UNITS = ATD_WROWS * TPK / 32;  // 16-byte units per lane per tile
+    static constexpr int KSTEPS = DH / 16;           // MMAs along the head dimension for S
+    static constexpr int NTILES = DH / 8;            // 8-wide output tiles of O
 };
-template <int DH, int QG>
+template <int DH>
 constexpr size_t attn_decode_smem_bytes() {
-    return (size_t)ATD_WARPS * AtdCfg<DH>::STAGES * AtdCfg<DH>::STAGE_ELEMS * sizeof(bf16) +
-           sizeof(float) * ((size_t)ATT_NQ * DH + (size_t)ATD_WARPS * QG * (DH + 2) + (size_t)ATD_SLOTS * (DH + 2));
+    // the warps' rings (reused for the warps' final states) + the inbox of states sent by the cluster's CTAs
+    return (size_t)ATD_WARPS * AtdCfg<DH>::STAGES * AtdCfg<DH>::STAGE_ELEMS * sizeof(bf16) + sizeof(float) * (size_t)ATD_SLOTS * (DH + 2);
+}
+static_assert((size_t)ATD_WARPS * ATT_NQ * (128 + 2) * sizeof(float) <= (size_t)ATD_WARPS * AtdCfg<128>::STAGES * AtdCfg<128>::STAGE_ELEMS * sizeof(bf16) &&
+              (size_t)ATD_WARPS * ATT_NQ * (32 + 2) * sizeof(float) <= (size_t)ATD_WARPS * AtdCfg<32>::STAGES * AtdCfg<32>::STAGE_ELEMS * sizeof(bf16),
+              "the warps' states fit in the ring");
+
+// Where the 16-byte unit u of ring row r lives within the row: XOR-swizzled so that the eight row addresses of
+// one ldmatrix fall into different banks (rows are DH * 2 bytes apart).
+template <int DH>
+__device__ __forceinline__ int atd_swz(int r, int u) { return u ^ (DH >= 64 ? (r & 7) : ((r >> 1) & 3)); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t atd_pack_bf16x2(float lo, float hi) {
+    const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&p);
 }
 
 // grid: (CL, heads, sequences) with the CL CTAs along x forming one cluster, CL in {1, 2, 4, 8}; block: ATD_THREADS.
-template <int DH, int QG>
+template <int DH>
 __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     using C = AtdCfg<DH>;
     constexpr int NW = ATD_WARPS;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    constexpr int SW = DH + 2;                     // a state: DH output sums, the running maximum, the running sum
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     bf16* ring_all = reinterpret_cast<bf16*>(smem_raw);
-    float* qs = reinterpret_cast<float*>(ring_all + (size_t)NW * C::STAGES * C::STAGE_ELEMS);   // [ATT_NQ][DH]
-    float* wst = qs + ATT_NQ * DH;                 // [NW][QG][DH + 2] the warps' states of the current query group
-    float* inbox = wst + NW * QG * (DH + 2);       // [CL][QPC][DH + 2] states sent by the cluster's CTAs
+    float* wst = reinterpret_cast<float*>(smem_raw);                                            // [NW][16][SW], after the main loop
+    float* inbox = reinterpret_cast<float*>(ring_all + (size_t)NW * C::STAGES * C::STAGE_ELEMS);   // [CL][QPC][SW]
     TC_PROBE_INIT(210);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = blockIdx.x, h = blockIdx.y, g = blockIdx.z;
     const int CL = gridDim.x;                      // cluster size
     const int QPC = (ATT_NQ + CL - 1) / CL;        // queries a CTA finishes at most
-    const int part = lane % C::TPK, kslot = lane / C::TPK;
     bf16* ring = ring_all + (size_t)warp * C::STAGES * C::STAGE_ELEMS;
+    const uint32_t ring_s = smem_u32(ring);
     pdl_wait();   // queries and the newest keys/values come from earlier kernels
     pdl_launch_dependents();
     if (tid == 0) TC_PROBE(1);
     const int cnt = a.nq, row0 = g * a.nq;
-    const bf16* qg = static_cast<const bf16*>(a.q);
-    for (int i = tid; i < cnt * DH; i += ATD_THREADS) {
-        const int qi = i / DH, el = i - qi * DH;
-        qs[i] = to_float(qg[(size_t)(row0 + qi) * a.ldq + h * DH + el]);
-    }
     const int b = a.row_seq[row0];
     const int pos_first = a.row_pos[row0];
     const int pos_last = pos_first + cnt - 1;
@@ -298,16 +328,34 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     const size_t head_base2 = ((size_t)b * a.n_heads + h) * a.t_max2;
     const int split = a.k2 ? a.split : INT_MAX;
 
-    // this warp's rows of its CTA's it-th chunk into stage it % STAGES
+    // this warp's rows of its CTA's it-th chunk into stage it % STAGES.  Lane L moves unit L % TPK of rows
+    // L / TPK + (32 / TPK) * u; a tile that lies wholly in one cache and before the last query (all but a
+    // boundary tile or two) takes the short way: one base address, constant steps.
+    constexpr int RSTEP = 32 / C::TPK;             // rows between a lane's consecutive units
+    const int i_row = lane / C::TPK, i_unit = lane - i_row * C::TPK;
     auto issue = [&](int it) {
         const int t0 = (rank + it * CL) * ATT_CH + warp * ATD_WROWS;
         bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
         bf16* vs = ks + C::TILE_ELEMS;
+        const bool first = t0 + ATD_WROWS <= split, second = t0 >= split;
+        if (t0 + ATD_WROWS - 1 <= pos_last && (first || second)) {
+            const size_t src = first ? (head_base + t0 + i_row) * DH : (head_base2 + (t0 - split) + i_row) * DH;
+            const bf16* kg = static_cast<const bf16*>(first ? a.kcache : a.k2) + src + i_unit * 8;
+            const bf16* vg = static_cast<const bf16*>(first ? a.vcache : a.v2) + src + i_unit * 8;
+#pragma unroll
+            for (int u = 0; u < C::UNITS; ++u) {
+                const int t = i_row + RSTEP * u;
+                const int dst = t * DH + atd_swz<DH>(t, i_unit) * 8;
+                cp_async16(ks + dst, kg + (size_t)u * RSTEP * DH);
+                cp_async16(vs + dst, vg + (size_t)u * RSTEP * DH);
+            }
+            return;
+        }
 #pragma unroll
         for (int u = 0; u < C::UNITS; ++u) {
-            const int idx = lane + 32 * u;
-            const int t = idx / C::TPK, v = idx - t * C::TPK;
+            const int t = i_row + RSTEP * u, v = i_unit;
             const int ta = t0 + t;
+            const int dst = t * DH + atd_swz<DH>(t, v) * 8;
             if (ta <= pos_last) {
                 const bf16 *kg, *vg;
                 if (ta < split) {
@@ -317,213 +365,184 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
                     kg = static_cast<const bf16*>(a.k2) + (head_base2 + (ta - split)) * DH;
                     vg = static_cast<const bf16*>(a.v2) + (head_base2 + (ta - split)) * DH;
                 }
-                cp_async16(ks + idx * 8, kg + v * 8);
-                cp_async16(vs + idx * 8, vg + v * 8);
+                cp_async16(ks + dst, kg + v * 8);
+                cp_async16(vs + dst, vg + v * 8);
             } else {   // past the last query: zeros, so that a zero weight times them stays zero
-                *reinterpret_cast<uint4*>(ks + idx * 8) = make_uint4(0u, 0u, 0u, 0u);
-                *reinterpret_cast<uint4*>(vs + idx * 8) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(ks + dst) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(vs + dst) = make_uint4(0u, 0u, 0u, 0u);
             }
         }
     };
-    __syncthreads();   // qs written
+#pragma unroll
+    for (int it = 0; it < C::STAGES - 1; ++it) {
+        if (it < n_mine) issue(it);
+        cp_async_commit();
+    }
+
+    // The queries as A fragments: this lane holds rows lane/4 and lane/4 + 8, columns 2*(lane%4) (+1) (+8) of each
+    // 16-wide step along the head dimension.
+    const int row_lo = lane >> 2, row_hi = row_lo + 8, kc = 2 * (lane & 3);
+    uint32_t qf[C::KSTEPS][4];
+    {
+        const bf16* qg = static_cast<const bf16*>(a.q) + h * DH + kc;
+        const bf16* q_lo = qg + (size_t)(row0 + row_lo) * a.ldq;
+        const bf16* q_hi = qg + (size_t)(row0 + row_hi) * a.ldq;
+#pragma unroll
+        for (int ks = 0; ks < C::KSTEPS; ++ks) {
+            qf[ks][0] = row_lo < cnt ? *reinterpret_cast<const uint32_t*>(q_lo + ks * 16) : 0u;
+            qf[ks][1] = row_hi < cnt ? *reinterpret_cast<const uint32_t*>(q_hi + ks * 16) : 0u;
+            qf[ks][2] = row_lo < cnt ? *reinterpret_cast<const uint32_t*>(q_lo + ks * 16 + 8) : 0u;
+            qf[ks][3] = row_hi < cnt ? *reinterpret_cast<const uint32_t*>(q_hi + ks * 16 + 8) : 0u;
+        }
+    }
+    float o[C::NTILES][4];
+#pragma unroll
+    for (int nt = 0; nt < C::NTILES; ++nt) { o[nt][0] = 0.f; o[nt][1] = 0.f; o[nt][2] = 0.f; o[nt][3] = 0.f; }
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;   // l: this lane's keys only until the end
+    const bool has_hi = cnt > 8;
+
+    // ldmatrix row addresses of this lane (matrix lane/8, row lane%8), relative to the K (or V) tile of a stage
+    const int lm_m = lane >> 3, lm_r = lane & 7;
+    const int lm_sw = DH >= 64 ? lm_r : (lm_r >> 1);
+    const uint32_t k_row = (uint32_t)(lm_r * DH * 2);                           // K: key = 8 * nt + row, unit = 4 * kp + matrix
+    const uint32_t v_row = (uint32_t)((((lm_m & 1) << 3) + lm_r) * DH * 2);     // V: key = 8 * (matrix & 1) + row, unit = 2 * np + matrix / 2
     if (tid == 0) TC_PROBE(2);
 
-    for (int q0 = 0; q0 < cnt; q0 += QG) {
+    for (int it = 0; it < n_mine; ++it) {
+        if (it + C::STAGES - 1 < n_mine) issue(it + C::STAGES - 1);
+        cp_async_commit();
+        asm volatile("cp.async.wait_group %0;" ::"n"(C::STAGES - 1) : "memory");
+        __syncwarp();
+        if (tid == 0 && it == 0) TC_PROBE(3);
+        const int t0 = (rank + it * CL) * ATT_CH + warp * ATD_WROWS;
+        const uint32_t ks_s = ring_s + (uint32_t)((it % C::STAGES) * C::STAGE_ELEMS * 2);
+        const uint32_t vs_s = ks_s + (uint32_t)(C::TILE_ELEMS * 2);
+
+        // S = Q K^T for the tile's 16 keys: two 8-key halves
+        float sc[2][4];
 #pragma unroll
-        for (int it = 0; it < C::STAGES - 1; ++it) {
-            if (it < n_mine) issue(it);
-            cp_async_commit();
-        }
-        float qreg[QG][8];
+        for (int nt = 0; nt < 2; ++nt) {
+            sc[nt][0] = 0.f; sc[nt][1] = 0.f; sc[nt][2] = 0.f; sc[nt][3] = 0.f;
 #pragma unroll
-        for (int qi = 0; qi < QG; ++qi)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) qreg[qi][j] = (q0 + qi < cnt) ? qs[(q0 + qi) * DH + part * 8 + j] : 0.f;
-        float m[QG], l[QG], acc[QG][8];
-#pragma unroll
-        for (int qi = 0; qi < QG; ++qi) {
-            m[qi] = -INFINITY; l[qi] = 0.f;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) acc[qi][j] = 0.f;
-        }
-        for (int it = 0; it < n_mine; ++it) {
-            if (it + C::STAGES - 1 < n_mine) issue(it + C::STAGES - 1);
-            cp_async_commit();
-            asm volatile("cp.async.wait_group %0;" ::"n"(C::STAGES - 1) : "memory");
-            __syncwarp();
-            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(3);
-            const int t0 = (rank + it * CL) * ATT_CH + warp * ATD_WROWS;
-            const bf16* ks = ring + (size_t)(it % C::STAGES) * C::STAGE_ELEMS;
-            const bf16* vs = ks + C::TILE_ELEMS;
-            if constexpr (QG == 4) {
-                // Four queries: the DH/8 lanes of a key split the four dot products among themselves while they add
-                // them up (a reduce-scatter with the same pairing, hence the same bits, as the one-query butterfly):
-                // the lane whose low position bits are (b0, b1) ends up with query 2*b0 + b1 and does that query's
-                // softmax step; probabilities and rescale factors are then handed round within the key's lanes.
-                const bool b0 = (part & 1) != 0, b1 = (part & 2) != 0;
-                const int qsel = (b0 ? 2 : 0) + (b1 ? 1 : 0);
-                const int key_lane0 = lane & ~(C::TPK - 1);
-                const bool q_live = q0 + qsel < cnt;
-                const int q_pos = pos_first + q0 + qsel;
-                float sp[C::PPW];
-                float mcm = -INFINITY;
-#pragma unroll
-                for (int p = 0; p < C::PPW; ++p) {
-                    const int key = p * C::KPW + kslot;
-                    float kf[8];
-                    load_vec(ks + key * DH + part * 8, kf);
-                    float d[4];
-#pragma unroll
-                    for (int qi = 0; qi < 4; ++qi) {
-                        d[qi] = 0.f;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) d[qi] = fmaf(qreg[qi][j], kf[j], d[qi]);
-                    }
-                    const float r0 = __shfl_xor_sync(0xffffffffu, b0 ? d[0] : d[2], 1);
-                    const float r1 = __shfl_xor_sync(0xffffffffu, b0 ? d[1] : d[3], 1);
-                    const float e0 = (b0 ? d[2] : d[0]) + r0, e1 = (b0 ? d[3] : d[1]) + r1;
-                    const float r2 = __shfl_xor_sync(0xffffffffu, b1 ? e0 : e1, 2);
-                    float dq = (b1 ? e1 : e0) + r2;
-#pragma unroll
-                    for (int o = 4; o < C::TPK; o <<= 1) dq += __shfl_xor_sync(0xffffffffu, dq, o);
-                    sp[p] = (q_live && t0 + key <= q_pos) ? dq * a.scale : -INFINITY;
-                    mcm = fmaxf(mcm, sp[p]);
-                }
-#pragma unroll
-                for (int o = C::TPK; o < 32; o <<= 1) mcm = fmaxf(mcm, __shfl_xor_sync(0xffffffffu, mcm, o));
-                const float mn = fmaxf(m[0], mcm);
-                const float fm = m[0] > -INFINITY ? __expf(m[0] - mn) : 0.f;
-                m[0] = mn;
-                float ls = 0.f;
-#pragma unroll
-                for (int p = 0; p < C::PPW; ++p) {
-                    sp[p] = mn > -INFINITY ? __expf(sp[p] - mn) : 0.f;
-                    ls += sp[p];
-                }
-                l[0] = l[0] * fm + ls;   // this lane's keys only; the key slots are added up at the end
-#pragma unroll
-                for (int qi = 0; qi < 4; ++qi) {
-                    const float fq = __shfl_sync(0xffffffffu, fm, key_lane0 | ((qi >> 1) | ((qi & 1) << 1)));
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[qi][j] *= fq;
-                }
-#pragma unroll
-                for (int p = 0; p < C::PPW; ++p) {
-                    const int key = p * C::KPW + kslot;
-                    float vf[8];
-                    load_vec(vs + key * DH + part * 8, vf);
-#pragma unroll
-                    for (int qi = 0; qi < 4; ++qi) {
-                        const float pq = __shfl_sync(0xffffffffu, sp[p], key_lane0 | ((qi >> 1) | ((qi & 1) << 1)));
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) acc[qi][j] = fmaf(pq, vf[j], acc[qi][j]);
-                    }
-                }
-            } else {
-            float sc[QG][C::PPW], mc[QG];
-#pragma unroll
-            for (int qi = 0; qi < QG; ++qi) mc[qi] = -INFINITY;
-#pragma unroll
-            for (int p = 0; p < C::PPW; ++p) {
-                const int key = p * C::KPW + kslot;
-                float kf[8];
-                load_vec(ks + key * DH + part * 8, kf);
-#pragma unroll
-                for (int qi = 0; qi < QG; ++qi) {
-                    float d = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) d = fmaf(qreg[qi][j], kf[j], d);
-#pragma unroll
-                    for (int o = 1; o < C::TPK; o <<= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-                    const bool live = (q0 + qi < cnt) && (t0 + key <= pos_first + q0 + qi);
-                    sc[qi][p] = live ? d * a.scale : -INFINITY;
-                    mc[qi] = fmaxf(mc[qi], sc[qi][p]);
-                }
-            }
-#pragma unroll
-            for (int qi = 0; qi < QG; ++qi) {
-#pragma unroll
-                for (int o = C::TPK; o < 32; o <<= 1) mc[qi] = fmaxf(mc[qi], __shfl_xor_sync(0xffffffffu, mc[qi], o));
-                const float mn = fmaxf(m[qi], mc[qi]);
-                const float f = m[qi] > -INFINITY ? __expf(m[qi] - mn) : 0.f;
-                m[qi] = mn;
-                float ls = 0.f;
-#pragma unroll
-                for (int p = 0; p < C::PPW; ++p) {
-                    const float pr = mn > -INFINITY ? __expf(sc[qi][p] - mn) : 0.f;
-                    sc[qi][p] = pr;
-                    ls += pr;
-                }
-                l[qi] = l[qi] * f + ls;   // this lane's keys only; the key slots are added up at the end
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc[qi][j] *= f;
-            }
-#pragma unroll
-            for (int p = 0; p < C::PPW; ++p) {
-                const int key = p * C::KPW + kslot;
-                float vf[8];
-                load_vec(vs + key * DH + part * 8, vf);
-#pragma unroll
-                for (int qi = 0; qi < QG; ++qi)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[qi][j] = fmaf(sc[qi][p], vf[j], acc[qi][j]);
-            }
-            }
-            __syncwarp();   // the stage may be refilled by this warp's next issue
-            if (tid == 0 && it == 0 && q0 == 0) TC_PROBE(8);
-        }
-        // the warp's state: add up its key slots (lanes that share `part`), lanes 0 .. TPK-1 publish it
-        if constexpr (QG == 4) {   // each lane carries the running maximum and sum of one query only
-#pragma unroll
-            for (int o = C::TPK; o < 32; o <<= 1) l[0] += __shfl_xor_sync(0xffffffffu, l[0], o);
-            if (lane < 4) {        // lane = position bits (b0, b1) of key slot 0: query 2*b0 + b1
-                float* st = wst + (size_t)(warp * QG + (((lane & 1) << 1) | (lane >> 1))) * (DH + 2);
-                st[DH] = m[0]; st[DH + 1] = l[0];
+            for (int kp = 0; kp < C::KSTEPS / 2; ++kp) {
+                uint32_t kf[4];
+                ldmatrix_x4(ks_s + (uint32_t)(nt * 8 * DH * 2) + k_row + (uint32_t)((((kp * 4 + lm_m) ^ lm_sw)) << 4), kf);
+                mma_bf16_16816(sc[nt], qf[2 * kp], kf[0], kf[1]);
+                mma_bf16_16816(sc[nt], qf[2 * kp + 1], kf[2], kf[3]);
             }
         }
+        // scale, causal mask, running maxima (a row's scores sit in the four lanes of a quad).  Rows 8-15 are
+        // skipped when the block has at most eight queries: their state stays (-inf, 0, 0) and is never read.
+        float mc_lo = -INFINITY, mc_hi = -INFINITY;
 #pragma unroll
-        for (int qi = 0; qi < QG; ++qi) {
+        for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
-            for (int o = C::TPK; o < 32; o <<= 1) {
-                if (QG != 4) l[qi] += __shfl_xor_sync(0xffffffffu, l[qi], o);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc[qi][j] += __shfl_xor_sync(0xffffffffu, acc[qi][j], o);
-            }
-            if (lane < C::TPK) {
-                float* st = wst + (size_t)(warp * QG + qi) * (DH + 2);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) st[lane * 8 + j] = acc[qi][j];
-                if (QG != 4 && lane == 0) { st[DH] = m[qi]; st[DH + 1] = l[qi]; }
-            }
-        }
-        __syncthreads();
-        if (tid == 0 && q0 == 0) TC_PROBE(4);
-        // fold the warps' states in warp order and send the CTA's state of query qi to CTA qi % 8
-        for (int i = tid; i < QG * (DH + 2); i += ATD_THREADS) {
-            const int qi = i / (DH + 2), e = i - qi * (DH + 2);
-            const int qa = q0 + qi;
-            if (qa < cnt) {
-                float mx = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < NW; ++w) mx = fmaxf(mx, wst[(size_t)(w * QG + qi) * (DH + 2) + DH]);
-                float val;
-                if (e == DH) {
-                    val = mx;
-                } else {
-                    val = 0.f;
-#pragma unroll
-                    for (int w = 0; w < NW; ++w) {
-                        const float* st = wst + (size_t)(w * QG + qi) * (DH + 2);
-                        const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
-                        val = fmaf(e < DH ? st[e] : st[DH + 1], f, val);
-                    }
+            for (int e = 0; e < 2; ++e) {
+                const int ta = t0 + nt * 8 + kc + e;
+                sc[nt][e] = (row_lo < cnt && ta <= pos_first + row_lo) ? sc[nt][e] * a.scale : -INFINITY;
+                mc_lo = fmaxf(mc_lo, sc[nt][e]);
+                if (has_hi) {
+                    sc[nt][2 + e] = (row_hi < cnt && ta <= pos_first + row_hi) ? sc[nt][2 + e] * a.scale : -INFINITY;
+                    mc_hi = fmaxf(mc_hi, sc[nt][2 + e]);
                 }
-                float* slot = inbox + ((size_t)rank * QPC + qa / CL) * (DH + 2) + e;
-                if (CL > 1) st_dsmem_f32(smem_u32(slot), qa % CL, val);
-                else *slot = val;
             }
         }
-        __syncthreads();   // wst is rewritten by the next query group
+        mc_lo = fmaxf(mc_lo, __shfl_xor_sync(0xffffffffu, mc_lo, 1));
+        mc_lo = fmaxf(mc_lo, __shfl_xor_sync(0xffffffffu, mc_lo, 2));
+        const float mn_lo = fmaxf(m_lo, mc_lo);
+        const float f_lo = m_lo > -INFINITY ? __expf(m_lo - mn_lo) : 0.f;
+        m_lo = mn_lo;
+        float mn_hi = -INFINITY, f_hi = 1.f;
+        if (has_hi) {
+            mc_hi = fmaxf(mc_hi, __shfl_xor_sync(0xffffffffu, mc_hi, 1));
+            mc_hi = fmaxf(mc_hi, __shfl_xor_sync(0xffffffffu, mc_hi, 2));
+            mn_hi = fmaxf(m_hi, mc_hi);
+            f_hi = m_hi > -INFINITY ? __expf(m_hi - mn_hi) : 0.f;
+            m_hi = mn_hi;
+        }
+        // probabilities as the sum of two bf16 numbers (the rounded value and the rounded remainder): the second
+        // product then sees them to about 16 significant bits instead of 8, at the price of a second MMA
+        uint32_t pf[4], pr[4];
+        float ls_lo = 0.f, ls_hi = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            const float p0 = mn_lo > -INFINITY ? __expf(sc[nt][0] - mn_lo) : 0.f, p1 = mn_lo > -INFINITY ? __expf(sc[nt][1] - mn_lo) : 0.f;
+            ls_lo += p0 + p1;
+            const __nv_bfloat162 h_lo = __floats2bfloat162_rn(p0, p1);
+            pf[2 * nt] = *reinterpret_cast<const uint32_t*>(&h_lo);       // keys 8 nt + kc (+1): A columns of the same numbers
+            pr[2 * nt] = atd_pack_bf16x2(p0 - __low2float(h_lo), p1 - __high2float(h_lo));
+            pf[2 * nt + 1] = 0u; pr[2 * nt + 1] = 0u;
+            if (has_hi) {
+                const float p2 = mn_hi > -INFINITY ? __expf(sc[nt][2] - mn_hi) : 0.f, p3 = mn_hi > -INFINITY ? __expf(sc[nt][3] - mn_hi) : 0.f;
+                ls_hi += p2 + p3;
+                const __nv_bfloat162 h_hi = __floats2bfloat162_rn(p2, p3);
+                pf[2 * nt + 1] = *reinterpret_cast<const uint32_t*>(&h_hi);
+                pr[2 * nt + 1] = atd_pack_bf16x2(p2 - __low2float(h_hi), p3 - __high2float(h_hi));
+            }
+        }
+        l_lo = l_lo * f_lo + ls_lo;
+        l_hi = l_hi * f_hi + ls_hi;
+        // O = O * f + P V; the rescaling is skipped while no row of the warp has a new maximum (a factor of exactly 1)
+        const bool rescale = __any_sync(0xffffffffu, f_lo != 1.f || f_hi != 1.f);
+#pragma unroll
+        for (int np = 0; np < C::NTILES / 2; ++np) {
+            uint32_t vf[4];
+            ldmatrix_x4_trans(vs_s + v_row + (uint32_t)((((2 * np + (lm_m >> 1)) ^ lm_sw)) << 4), vf);
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                float (&acc)[4] = o[2 * np + hh];
+                if (rescale) { acc[0] *= f_lo; acc[1] *= f_lo; acc[2] *= f_hi; acc[3] *= f_hi; }
+                mma_bf16_16816(acc, pf, vf[2 * hh], vf[2 * hh + 1]);
+                mma_bf16_16816(acc, pr, vf[2 * hh], vf[2 * hh + 1]);
+            }
+        }
+        __syncwarp();   // the stage may be refilled by this warp's next issue
+        if (tid == 0 && it == 0) TC_PROBE(8);
+    }
+    // a row's sum: add the quad's lanes
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();   // every warp is done with its ring: the warps' states go where the rings were
+    {
+        float* st_lo = wst + (size_t)(warp * ATT_NQ + row_lo) * SW;
+        float* st_hi = wst + (size_t)(warp * ATT_NQ + row_hi) * SW;
+        if (row_lo < cnt) {
+#pragma unroll
+            for (int nt = 0; nt < C::NTILES; ++nt) *reinterpret_cast<float2*>(st_lo + nt * 8 + kc) = make_float2(o[nt][0], o[nt][1]);
+            if ((lane & 3) == 0) { st_lo[DH] = m_lo; st_lo[DH + 1] = l_lo; }
+        }
+        if (row_hi < cnt) {
+#pragma unroll
+            for (int nt = 0; nt < C::NTILES; ++nt) *reinterpret_cast<float2*>(st_hi + nt * 8 + kc) = make_float2(o[nt][2], o[nt][3]);
+            if ((lane & 3) == 0) { st_hi[DH] = m_hi; st_hi[DH + 1] = l_hi; }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) TC_PROBE(4);
+    // fold the warps' states in warp order and send the CTA's state of query qa to CTA qa % CL
+    for (int i = tid; i < cnt * SW; i += ATD_THREADS) {
+        const int qa = i / SW, e = i - qa * SW;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) mx = fmaxf(mx, wst[(size_t)(w * ATT_NQ + qa) * SW + DH]);
+        float val;
+        if (e == DH) {
+            val = mx;
+        } else {
+            val = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const float* st = wst + (size_t)(w * ATT_NQ + qa) * SW;
+                const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
+                val = fmaf(e < DH ? st[e] : st[DH + 1], f, val);
+            }
+        }
+        float* slot = inbox + ((size_t)rank * QPC + qa / CL) * SW + e;
+        if (CL > 1) st_dsmem_f32(smem_u32(slot), qa % CL, val);
+        else *slot = val;
     }
     if (CL > 1) cluster_sync_all(); else __syncthreads();
     if (tid == 0) TC_PROBE(5);
@@ -531,15 +550,15 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
         const int qi = rank + u * CL;
         if (qi < cnt && tid < DH) {
             float mx = -INFINITY;
-            for (int r = 0; r < CL; ++r) mx = fmaxf(mx, inbox[((size_t)r * QPC + u) * (DH + 2) + DH]);
-            float l = 0.f, o = 0.f;
+            for (int r = 0; r < CL; ++r) mx = fmaxf(mx, inbox[((size_t)r * QPC + u) * SW + DH]);
+            float l = 0.f, ov = 0.f;
             for (int r = 0; r < CL; ++r) {
-                const float* st = inbox + ((size_t)r * QPC + u) * (DH + 2);
+                const float* st = inbox + ((size_t)r * QPC + u) * SW;
                 const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
                 l = fmaf(st[DH + 1], f, l);
-                o = fmaf(st[tid], f, o);
+                ov = fmaf(st[tid], f, ov);
             }
-            static_cast<bf16*>(a.out)[(size_t)(row0 + qi) * a.ldo + h * DH + tid] = __float2bfloat16_rn(o / l);
+            static_cast<bf16*>(a.out)[(size_t)(row0 + qi) * a.ldo + h * DH + tid] = __float2bfloat16_rn(ov / l);
         }
     }
     if (tid == 0) TC_PROBE(6);

@@ -481,16 +481,16 @@ void launch_attn(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, bool 
 }
 
 // bf16 decode attention: one cluster of `cl` CTAs per (sequence, head); no scratch.
-template <int DH, int QG>
+template <int DH>
 void launch_attn_decode_dq(tandem_ctx& c, const AttnArgs& a, int groups, int cl, double kv_bytes) {
     static bool attr_set[MAX_DEVICES] = {};
     const int dev = cur_dev();
     if (!attr_set[dev]) {
-        cudaFuncSetAttribute(attn_decode_kernel<DH, QG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_decode_smem_bytes<DH, QG>());
+        cudaFuncSetAttribute(attn_decode_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_decode_smem_bytes<DH>());
         attr_set[dev] = true;
     }
     ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
-    launch_ex(c, true, cl, attn_decode_kernel<DH, QG>, dim3(cl, a.n_heads, groups), dim3(ATD_THREADS), attn_decode_smem_bytes<DH, QG>(), a);
+    launch_ex(c, true, cl, attn_decode_kernel<DH>, dim3(cl, a.n_heads, groups), dim3(ATD_THREADS), attn_decode_smem_bytes<DH>(), a);
 }
 // Cluster size: the largest of 1, 2, 4, 8 that keeps the launch within one wave of resident CTAs (two per SM,
 // one for 128-wide heads).  It depends on the number of sequences and heads only, so every pass of a run
@@ -502,11 +502,10 @@ int attn_cluster_size(int groups, int n_heads, int d_head) {
     return cl;
 }
 void launch_attn_decode(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, double kv_bytes) {
-    const bool one = a.nq == 1;
     const int cl = attn_cluster_size(groups, a.n_heads, d_head);
-    if (d_head == 32) { if (one) launch_attn_decode_dq<32, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<32, 4>(c, a, groups, cl, kv_bytes); }
-    else if (d_head == 64) { if (one) launch_attn_decode_dq<64, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<64, 4>(c, a, groups, cl, kv_bytes); }
-    else { if (one) launch_attn_decode_dq<128, 1>(c, a, groups, cl, kv_bytes); else launch_attn_decode_dq<128, 4>(c, a, groups, cl, kv_bytes); }
+    if (d_head == 32) launch_attn_decode_dq<32>(c, a, groups, cl, kv_bytes);
+    else if (d_head == 64) launch_attn_decode_dq<64>(c, a, groups, cl, kv_bytes);
+    else launch_attn_decode_dq<128>(c, a, groups, cl, kv_bytes);
 }
 
 template <typename T>
