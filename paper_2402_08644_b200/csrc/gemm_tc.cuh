@@ -5,8 +5,10 @@
 //                          The job is streaming W once from HBM: every CTA owns one (tile, K-slice) unit so
 //                          that all SMs pull weights, tiles arrive by TMA through a ring of stages, and the
 //                          K-slices of a tile sit in one thread-block cluster: each CTA sends its partial
-//                          sums to the CTA that finishes those columns (remote shared-memory stores), which
-//                          adds them in slice order.
+//                          sums to the CTA that finishes those token rows (remote shared-memory stores), which
+//                          adds them in slice order.  Epilogues that write the fp32 residual stream can also
+//                          leave, per row and 128-feature tile, the mean and the sum of squared deviations of
+//                          what they wrote; the next LayerNorm prologue merges those instead of re-reading rows.
 //                          The token rows are written into the B stages by the CTA's own threads, which is
 //                          where the LayerNorm (or the fp32 -> bf16 cast) of the residual stream is fused.
 //                          The weight loads are issued before the kernel waits for its predecessor in the
@@ -34,6 +36,8 @@ struct TcDecodeArgs {
     int ldx;
     const float* ln_g;      // PRO_LN: LayerNorm gain / bias [K]
     const float* ln_b;
+    const float* ln_part;   // PRO_LN, nullable: (mean, sum of squared deviations) of consecutive ln_pw-element pieces of each
+    int ln_ld, ln_pw;       //   row of x, piece p of row r at ln_part[2 * (r * ln_ld + p)]; null: the kernel reads whole rows
     int rows, K, N;         // N = output features over all segments
     int seg_rows;           // output features per weight segment (one tensor map each)
     int tiles_per_seg;      // ceil(seg_rows / 128)
@@ -52,7 +56,7 @@ template <int NB> struct TcdCfg {
     static constexpr int A_BYTES = 128 * 128;       // 128 weight rows x 64 bf16
     static constexpr int B_BYTES = NB * 128;        // NB token rows x 64 bf16
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int INBOX_BYTES = NB * 128 * 4;   // the K-slices' partial sums for this CTA's share of the columns
+    static constexpr int INBOX_BYTES = NB * 128 * 4;   // the K-slices' partial sums for the token rows this CTA finishes
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + INBOX_BYTES + 1024;   // + slack to align the ring to 1024
     static constexpr int TMEM_COLS = NB <= 32 ? 32 : 64;
 };
@@ -66,6 +70,15 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 __device__ __forceinline__ float4 ln_apply(float4 x, float mu, float rs, float4 g, float4 b) {
     return make_float4((x.x - mu) * rs * g.x + b.x, (x.y - mu) * rs * g.y + b.y, (x.z - mu) * rs * g.z + b.z, (x.w - mu) * rs * g.w + b.w);
+}
+
+// Merges the (count, mean, sum of squared deviations) of a second set of values into the first (pairwise update of
+// Chan, Golub and LeVeque); nb > 0.
+__device__ __forceinline__ void moments_merge(float& na, float& mean, float& m2, float nb, float mb, float qb) {
+    const float n = na + nb, dl = mb - mean;
+    mean += dl * (nb / n);
+    m2 += qb + dl * dl * (na * nb / n);
+    na = n;
 }
 
 // Where column c of weight segment `seg` goes for EPI_QKV / EPI_KV: the query buffer (row stride ldo) or a cache.
@@ -99,6 +112,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     __shared__ float s_av[4][NB];
     __shared__ int s_ai[4][NB];
     __shared__ long long s_rowoff[NB];   // EPI_QKV / EPI_KV: the row-dependent part of an output's cache index
+    __shared__ __align__(16) float s_gb[PRO == PRO_LN ? C::STAGES * 128 : 4];   // gains then biases of a ring's worth of K-blocks
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t ring0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // shared-space address of stage 0
@@ -116,7 +130,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     const int K4 = a.K >> 2;
     // LayerNorm rows short enough to sit in registers (8 float4 per lane) and a K-slice that fits the ring
     // without reuse: the B operand is then written straight from the registers that gave the statistics.
-    const bool ln_regs = PRO == PRO_LN && K4 <= 256 && nkb <= C::STAGES;
+    const bool ln_regs = PRO == PRO_LN && K4 <= 256 && nkb <= C::STAGES && a.ln_part == nullptr;
+    // Token rows whose outputs this CTA finishes: all of them without split-K, else a contiguous share of ceil(rows / S).
+    const int rpc = S == 1 ? a.rows : (a.rows + S - 1) / S;
+    const int j_first = S == 1 ? 0 : sp * rpc;
+    const int j_count = max(0, min(rpc, a.rows - j_first));
     float hres[EPI == EPI_RESID ? NB : 1];   // EPI_RESID: the residual values this thread's outputs are added to
     TC_PROBE_INIT(100 + PRO * 10 + EPI);
 
@@ -206,19 +224,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     if (EPI == EPI_RESID) {
         // the residual-stream values this thread will add to: fetched now, off the critical path
         const float* hp = static_cast<const float*>(a.e.out);
-        if (S == 1) {
-            const int nl = n_local0 + tid;
+        const int nl = n_local0 + tid;
 #pragma unroll
-            for (int j = 0; j < NB; ++j)
-                hres[j] = (j < a.rows && nl < a.seg_rows) ? __ldcg(hp + (size_t)j * a.e.ldo + seg * a.seg_rows + nl) : 0.f;
-        } else {
-            const int CW = 128 / S;
-            const int nl = n_local0 + sp * CW + (tid & (CW - 1));
-#pragma unroll
-            for (int it = 0; it < NB / 2; ++it) {
-                const int j = tid / CW + it * S;
-                hres[it] = (j < a.rows && nl < a.seg_rows) ? __ldcg(hp + (size_t)j * a.e.ldo + seg * a.seg_rows + nl) : 0.f;
-            }
+        for (int s = 0; s < NB; ++s) {
+            if (s >= j_count) break;   // (every loop over rows leaves at the last row: the unrolled rest is never fetched)
+            hres[s] = nl < a.seg_rows ? ld_cg_pinned(hp + (size_t)(j_first + s) * a.e.ldo + seg * a.seg_rows + nl) : 0.f;
         }
     }
     if (ln_regs) {
@@ -272,7 +282,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         if (tid == 0) TC_PROBE(6);
     } else {
         // general case: statistics (LayerNorm), then the K-blocks a ring's worth at a time
-        if (PRO == PRO_LN) {
+        if (PRO == PRO_LN && a.ln_part == nullptr) {
             for (int r = warp; r < a.rows; r += 4) {   // one warp per row, fixed lane-strided order
                 const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx);
                 float mu, var;
@@ -315,17 +325,53 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         for (int i0 = 0; i0 < nkb; i0 += C::STAGES) {
             // a ring's worth of K-blocks at a time: all loads first, so their latencies overlap
             uint4 raw[PRO == PRO_BF16 ? C::STAGES : 1][CPT];
-            if (PRO == PRO_BF16) {
+            float4 xf[PRO == PRO_BF16 ? 1 : C::STAGES][CPT][2];
 #pragma unroll
-                for (int g = 0; g < C::STAGES; ++g)
+            for (int g = 0; g < C::STAGES; ++g)
 #pragma unroll
-                    for (int ch = 0; ch < CPT; ++ch) {
-                        const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
-                        const int k = (kb0 + i0 + g) * 64 + c * 8;
-                        raw[g][ch] = (i0 + g < nkb && r < a.rows && k < a.K)
-                                         ? __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k))
-                                         : make_uint4(0u, 0u, 0u, 0u);
+                for (int ch = 0; ch < CPT; ++ch) {
+                    const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
+                    const int k = (kb0 + i0 + g) * 64 + c * 8;
+                    const bool in = i0 + g < nkb && r < a.rows && k < a.K;
+                    if (PRO == PRO_BF16) {
+                        raw[g][ch] = in ? __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k))
+                                        : make_uint4(0u, 0u, 0u, 0u);
+                    } else {
+                        const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
+                        xf[g][ch][0] = in ? __ldcg(xp) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        xf[g][ch][1] = in ? __ldcg(xp + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
+                }
+            if (PRO == PRO_LN) {
+                // gains and biases of these K-blocks go through shared memory: thread t fetches floats 4t .. 4t+3
+                float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), b4 = g4;
+                const int kg = (kb0 + i0) * 64 + tid * 4;
+                if (tid < C::STAGES * 16 && i0 + (tid >> 4) < nkb && kg < a.K) {
+                    g4 = __ldg(reinterpret_cast<const float4*>(a.ln_g + kg));
+                    b4 = __ldg(reinterpret_cast<const float4*>(a.ln_b + kg));
+                }
+                if (i0 == 0 && a.ln_part != nullptr && tid < a.rows) {
+                    // row statistics from the pieces the producing kernels left, merged in piece order
+                    const float2* pr = reinterpret_cast<const float2*>(a.ln_part) + (size_t)tid * a.ln_ld;
+                    const int P = (a.K + a.ln_pw - 1) / a.ln_pw;
+                    float na = 0.f, mean = 0.f, m2 = 0.f;
+                    for (int p0 = 0; p0 < P; p0 += 16) {
+                        float2 t[16];
+#pragma unroll
+                        for (int u = 0; u < 16; ++u) t[u] = p0 + u < P ? __ldcg(pr + p0 + u) : make_float2(0.f, 0.f);
+#pragma unroll
+                        for (int u = 0; u < 16; ++u)
+                            if (p0 + u < P) moments_merge(na, mean, m2, (float)min(a.ln_pw, a.K - (p0 + u) * a.ln_pw), t[u].x, t[u].y);
+                    }
+                    s_mu[tid] = mean;
+                    s_rstd[tid] = 1.0f / sqrtf(m2 / (float)a.K + 1e-5f);
+                }
+                bar_sync(1, 128);   // the previous round's readers are done with s_gb; s_mu / s_rstd are written
+                if (tid < C::STAGES * 16) {
+                    *reinterpret_cast<float4*>(&s_gb[tid * 4]) = g4;
+                    *reinterpret_cast<float4*>(&s_gb[C::STAGES * 64 + tid * 4]) = b4;
+                }
+                bar_sync(1, 128);
             }
             bool dead = false;
 #pragma unroll
@@ -345,19 +391,17 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                     uint4 val = make_uint4(0u, 0u, 0u, 0u);
                     if (PRO == PRO_BF16) {
                         val = raw[g][ch];
-                    } else {
-                        const int k = (kb0 + i) * 64 + c * 8;
-                        if (r < a.rows && k < a.K) {
-                            const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
-                            float4 u0 = __ldcg(xp), u1 = __ldcg(xp + 1);
-                            if (PRO == PRO_LN) {
-                                const float mu = s_mu[r], rs = s_rstd[r];
-                                u0 = ln_apply(u0, mu, rs, __ldg(reinterpret_cast<const float4*>(a.ln_g + k)), __ldg(reinterpret_cast<const float4*>(a.ln_b + k)));
-                                u1 = ln_apply(u1, mu, rs, __ldg(reinterpret_cast<const float4*>(a.ln_g + k) + 1), __ldg(reinterpret_cast<const float4*>(a.ln_b + k) + 1));
-                            }
-                            val.x = pack_bf16x2(u0.x, u0.y); val.y = pack_bf16x2(u0.z, u0.w);
-                            val.z = pack_bf16x2(u1.x, u1.y); val.w = pack_bf16x2(u1.z, u1.w);
+                    } else if (r < a.rows && (kb0 + i) * 64 + c * 8 < a.K) {
+                        float4 u0 = xf[g][ch][0], u1 = xf[g][ch][1];
+                        if (PRO == PRO_LN) {
+                            const float mu = s_mu[r], rs = s_rstd[r];
+                            const float4* gp = reinterpret_cast<const float4*>(&s_gb[g * 64 + c * 8]);
+                            const float4* bp = reinterpret_cast<const float4*>(&s_gb[C::STAGES * 64 + g * 64 + c * 8]);
+                            u0 = ln_apply(u0, mu, rs, gp[0], bp[0]);
+                            u1 = ln_apply(u1, mu, rs, gp[1], bp[1]);
                         }
+                        val.x = pack_bf16x2(u0.x, u0.y); val.y = pack_bf16x2(u0.z, u0.w);
+                        val.z = pack_bf16x2(u1.x, u1.y); val.w = pack_bf16x2(u1.z, u1.w);
                     }
                     // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
                     *reinterpret_cast<uint4*>(bt + r * 128 + ((c ^ (r & 7)) << 4)) = val;
@@ -387,94 +431,111 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         }
         if (tid == 0) TC_PROBE(8);
     }
-    if (S == 1) {
+    const int n_local = n_local0 + tl;                 // warps 0-3: this thread's output feature
+    const bool valid = n_local < a.seg_rows;
+    const int n = seg * a.seg_rows + n_local;
+    if (EPI == EPI_ARGMAX) {                            // whole tiles only (S == 1)
         if (warp < 4) {
-            const int n_local = n_local0 + tl;
-            const bool valid = n_local < a.seg_rows;
-            const int n = seg * a.seg_rows + n_local;
-            if (EPI == EPI_ARGMAX) {
-                float* out = static_cast<float*>(a.e.out);
+            float* out = static_cast<float*>(a.e.out);
 #pragma unroll
-                for (int j = 0; j < NB; ++j) {
-                    if (j < a.rows) {
-                        float bv = valid ? v[j] : -INFINITY;
-                        int bi = valid ? n : INT_MAX;
-                        if (valid) out[(size_t)j * a.e.ldo + n] = v[j];
+            for (int j = 0; j < NB; ++j) {
+                if (j >= a.rows) break;
+                {
+                    float bv = valid ? v[j] : -INFINITY;
+                    int bi = valid ? n : INT_MAX;
+                    if (valid) out[(size_t)j * a.e.ldo + n] = v[j];
 #pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) {
-                            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-                        }
-                        if (lane == 0) { s_av[warp][j] = bv; s_ai[warp][j] = bi; }
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
                     }
+                    if (lane == 0) { s_av[warp][j] = bv; s_ai[warp][j] = bi; }
                 }
-                bar_sync(1, 128);
-                if (tid < a.rows) {
-                    float bv = s_av[0][tid];
-                    int bi = s_ai[0][tid];
-                    for (int w = 1; w < 4; ++w)
-                        if (s_av[w][tid] > bv || (s_av[w][tid] == bv && s_ai[w][tid] < bi)) { bv = s_av[w][tid]; bi = s_ai[w][tid]; }
-                    a.amax_val[(size_t)tid * a.amax_stride + tile] = bv;
-                    a.amax_idx[(size_t)tid * a.amax_stride + tile] = bi;
-                }
-            } else if (EPI == EPI_RESID) {
-                float* out = static_cast<float*>(a.e.out);
-#pragma unroll
-                for (int j = 0; j < NB; ++j)
-                    if (j < a.rows && valid) {
-                        const float hv = hres[j] + v[j];
-                        out[(size_t)j * a.e.ldo + n] = hv;
-                        if (a.e.snap) static_cast<bf16*>(a.e.snap)[(size_t)j * a.e.snap_ld + n] = __float2bfloat16_rn(hv);
-                    }
-            } else if (EPI == EPI_QKV || EPI == EPI_KV) {
-                const ScatterCol sc = scatter_col<EPI>(a.e, seg, n_local);
-#pragma unroll
-                for (int j = 0; j < NB; ++j)
-                    if (j < a.rows && valid) sc.base[(sc.is_q ? (long long)j * a.e.ldo : s_rowoff[j]) + sc.col] = __float2bfloat16_rn(v[j]);
-            } else {
-#pragma unroll
-                for (int j = 0; j < NB; ++j)
-                    if (j < a.rows && valid) epilogue<bf16, EPI>(a.e, j, n, v[j]);
+            }
+            bar_sync(1, 128);
+            if (tid < a.rows) {
+                float bv = s_av[0][tid];
+                int bi = s_ai[0][tid];
+                for (int w = 1; w < 4; ++w)
+                    if (s_av[w][tid] > bv || (s_av[w][tid] == bv && s_ai[w][tid] < bi)) { bv = s_av[w][tid]; bi = s_ai[w][tid]; }
+                a.amax_val[(size_t)tid * a.amax_stride + tile] = bv;
+                a.amax_idx[(size_t)tid * a.amax_stride + tile] = bi;
             }
         }
     } else {
-        // The cluster's CTAs hold the K-slices of one tile, and CTA `r` finishes columns [r*128/S, (r+1)*128/S).
-        // Every CTA sends each column's partial sums to the inbox of the CTA that finishes it (remote shared-memory
-        // stores), one cluster barrier makes them visible, and each CTA sums its inbox in slice order.  Nobody
-        // touches a peer's shared memory after the barrier, so CTAs may leave as they finish.
-        const int CW = 128 / S;
-        const uint32_t inbox0 = ring0 + C::STAGES * C::STAGE_BYTES;           // [S][NB][CW] fp32
-        if (warp < 4) {
-            const int dst = tl / CW, cw = tl & (CW - 1);
+        if (S > 1) {
+            // The cluster's CTAs hold the K-slices of one tile, and CTA r finishes token rows [r * rpc, (r + 1) * rpc).
+            // Every CTA sends each row's partial sums to the inbox of the CTA that finishes it (remote shared-memory
+            // stores), one cluster barrier makes them visible, and each CTA sums its inbox in slice order.  Nobody
+            // touches a peer's shared memory after the barrier, so CTAs may leave as they finish.
+            const uint32_t inbox0 = ring0 + C::STAGES * C::STAGE_BYTES;           // [S][rpc][128] fp32
+            if (warp < 4) {
+                int dst = 0, jj = 0;
 #pragma unroll
-            for (int j = 0; j < NB; ++j)
-                if (j < a.rows) st_dsmem_f32(inbox0 + ((sp * NB + j) * CW + cw) * 4, dst, v[j]);
+                for (int j = 0; j < NB; ++j) {
+                    if (j >= a.rows) break;
+                    st_dsmem_f32(inbox0 + ((sp * rpc + jj) * 128 + tl) * 4, dst, v[j]);
+                    if (++jj == rpc) { jj = 0; ++dst; }
+                }
+            }
+            cluster_sync_all();
+            if (tid == 0) TC_PROBE(9);
+            if (warp < 4) {
+                const float* inbox = reinterpret_cast<const float*>(ring + C::STAGES * C::STAGE_BYTES);
+#pragma unroll
+                for (int s = 0; s < NB / 2; ++s) {
+                    if (s >= j_count) break;
+                    float acc = 0.f;
+#pragma unroll
+                    for (int ss = 0; ss < 8; ++ss) if (ss < S) acc += inbox[((ss * rpc + s) * 128) + tl];   // slice order
+                    v[s] = acc;
+                }
+            }
         }
-        cluster_sync_all();
-        if (tid == 0) TC_PROBE(9);
-        if (warp < 4 && EPI != EPI_ARGMAX) {
-            const float* inbox = reinterpret_cast<const float*>(ring + C::STAGES * C::STAGE_BYTES);
-            const int cw = tid & (CW - 1);
-            const int n_local = n_local0 + sp * CW + cw;
-            const bool valid = n_local < a.seg_rows;
-            const int n = seg * a.seg_rows + n_local;
+        // v[s] is now the finished product of token row j_first + s and this thread's feature
+        if (warp < 4) {
+            constexpr bool STAT = EPI == EPI_RESID || EPI == EPI_STORE_F32;
+            const bool stat = STAT && a.e.stat != nullptr;
+            const int cnt_w = min(32, max(0, a.seg_rows - (n_local0 + warp * 32)));   // valid features in this warp
             ScatterCol sc;
             if (EPI == EPI_QKV || EPI == EPI_KV) sc = scatter_col<EPI>(a.e, seg, n_local);
 #pragma unroll
-            for (int it = 0; it < NB / 2; ++it) {       // 128 / CW = S row groups: rows tid / CW, + S, ...
-                const int j = tid / CW + it * S;
-                if (j < a.rows && valid) {
-                    float acc = 0.f;
+            for (int s = 0; s < NB; ++s) {
+                if (s >= j_count) break;
+                {
+                    const int j = j_first + s;
+                    float hv = v[s];
+                    if (EPI == EPI_RESID) hv += hres[s];
+                    if (valid) {
+                        if (EPI == EPI_RESID || EPI == EPI_STORE_F32) {
+                            static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = hv;
+                            if (EPI == EPI_RESID && a.e.snap) static_cast<bf16*>(a.e.snap)[(size_t)j * a.e.snap_ld + n] = __float2bfloat16_rn(hv);
+                        } else if (EPI == EPI_QKV || EPI == EPI_KV) {
+                            sc.base[(sc.is_q ? (long long)j * a.e.ldo : s_rowoff[j]) + sc.col] = __float2bfloat16_rn(hv);
+                        } else {
+                            epilogue<bf16, EPI>(a.e, j, n, hv);
+                        }
+                    }
+                    if (stat) {
+                        // mean and squared deviations of what this warp wrote of row j (two passes over registers)
+                        const float mw = cnt_w > 0 ? warp_sum(valid ? hv : 0.f) / (float)cnt_w : 0.f;
+                        const float dv = valid ? hv - mw : 0.f;
+                        const float qw = warp_sum(dv * dv);
+                        if (lane == 0) { s_av[warp][s] = mw; s_ai[warp][s] = __float_as_int(qw); }
+                    }
+                }
+            }
+            if (stat) {
+                bar_sync(1, 128);
+                if (tid < j_count) {   // the four warps' pieces merged in warp order: one piece per (row, tile)
+                    float na = 0.f, mean = 0.f, m2 = 0.f;
 #pragma unroll
-                    for (int ss = 0; ss < 8; ++ss) if (ss < S) acc += inbox[(ss * NB + j) * CW + cw];   // slice order
-                    if (EPI == EPI_RESID) {
-                        const float hv = hres[it] + acc;
-                        static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = hv;
-                        if (a.e.snap) static_cast<bf16*>(a.e.snap)[(size_t)j * a.e.snap_ld + n] = __float2bfloat16_rn(hv);
-                    } else if (EPI == EPI_QKV || EPI == EPI_KV)
-                        sc.base[(sc.is_q ? (long long)j * a.e.ldo : s_rowoff[j]) + sc.col] = __float2bfloat16_rn(acc);
-                    else epilogue<bf16, EPI>(a.e, j, n, acc);
+                    for (int w = 0; w < 4; ++w) {
+                        const int cw = min(32, max(0, a.seg_rows - (n_local0 + w * 32)));
+                        if (cw > 0) moments_merge(na, mean, m2, (float)cw, s_av[w][tid], __int_as_float(s_ai[w][tid]));
+                    }
+                    reinterpret_cast<float2*>(a.e.stat)[(size_t)(j_first + tid) * a.e.stat_ld + tile] = make_float2(mean, m2);
                 }
             }
         }
