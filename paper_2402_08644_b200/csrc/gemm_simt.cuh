@@ -26,8 +26,6 @@ struct EpiArgs {
     int seg;              // columns per segment (= d_model) for QKV / KV
     void* snap;           // EPI_RESID on the tensor-core decode path: optional bf16 copy of the new values [M][snap_ld]
     int snap_ld;
-    float* stat;          // EPI_RESID / EPI_STORE_F32 on the tensor-core decode path: optional (mean, sum of squared deviations)
-    int stat_ld;          //   of each 128-feature tile of each row written, tile t of row m at stat[2 * (m * stat_ld + t)]
 };
 
 struct WSegs {            // up to three weight matrices stacked along N, each [seg_rows][K]

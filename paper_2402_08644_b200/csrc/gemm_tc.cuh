@@ -6,9 +6,7 @@
 //                          that all SMs pull weights, tiles arrive by TMA through a ring of stages, and the
 //                          K-slices of a tile sit in one thread-block cluster: each CTA sends its partial
 //                          sums to the CTA that finishes those token rows (remote shared-memory stores), which
-//                          adds them in slice order.  Epilogues that write the fp32 residual stream can also
-//                          leave, per row and 128-feature tile, the mean and the sum of squared deviations of
-//                          what they wrote; the next LayerNorm prologue merges those instead of re-reading rows.
+//                          adds them in slice order.
 //                          The token rows are written into the B stages by the CTA's own threads, which is
 //                          where the LayerNorm (or the fp32 -> bf16 cast) of the residual stream is fused.
 //                          The weight loads are issued before the kernel waits for its predecessor in the
@@ -36,8 +34,6 @@ struct TcDecodeArgs {
     int ldx;
     const float* ln_g;      // PRO_LN: LayerNorm gain / bias [K]
     const float* ln_b;
-    const float* ln_part;   // PRO_LN, nullable: (mean, sum of squared deviations) of consecutive ln_pw-element pieces of each
-    int ln_ld, ln_pw;       //   row of x, piece p of row r at ln_part[2 * (r * ln_ld + p)]; null: the kernel reads whole rows
     int rows, K, N;         // N = output features over all segments
     int seg_rows;           // output features per weight segment (one tensor map each)
     int tiles_per_seg;      // ceil(seg_rows / 128)
@@ -72,15 +68,6 @@ __device__ __forceinline__ float4 ln_apply(float4 x, float mu, float rs, float4 
     return make_float4((x.x - mu) * rs * g.x + b.x, (x.y - mu) * rs * g.y + b.y, (x.z - mu) * rs * g.z + b.z, (x.w - mu) * rs * g.w + b.w);
 }
 
-// Merges the (count, mean, sum of squared deviations) of a second set of values into the first (pairwise update of
-// Chan, Golub and LeVeque); nb > 0.
-__device__ __forceinline__ void moments_merge(float& na, float& mean, float& m2, float nb, float mb, float qb) {
-    const float n = na + nb, dl = mb - mean;
-    mean += dl * (nb / n);
-    m2 += qb + dl * dl * (na * nb / n);
-    na = n;
-}
-
 // Where column c of weight segment `seg` goes for EPI_QKV / EPI_KV: the query buffer (row stride ldo) or a cache.
 // The address of (row j, column c) is base + row term + col, with the row term j * ldo or the cache row offset.
 struct ScatterCol { bf16* base; long long col; bool is_q; };
@@ -112,7 +99,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     __shared__ float s_av[4][NB];
     __shared__ int s_ai[4][NB];
     __shared__ long long s_rowoff[NB];   // EPI_QKV / EPI_KV: the row-dependent part of an output's cache index
-    __shared__ __align__(16) float s_gb[PRO == PRO_LN ? C::STAGES * 128 : 4];   // gains then biases of a ring's worth of K-blocks
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t ring0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;          // shared-space address of stage 0
@@ -130,7 +116,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     const int K4 = a.K >> 2;
     // LayerNorm rows short enough to sit in registers (8 float4 per lane) and a K-slice that fits the ring
     // without reuse: the B operand is then written straight from the registers that gave the statistics.
-    const bool ln_regs = PRO == PRO_LN && K4 <= 256 && nkb <= C::STAGES && a.ln_part == nullptr;
+    const bool ln_regs = PRO == PRO_LN && K4 <= 256 && nkb <= C::STAGES;
     // Token rows whose outputs this CTA finishes: all of them without split-K, else a contiguous share of ceil(rows / S).
     const int rpc = S == 1 ? a.rows : (a.rows + S - 1) / S;
     const int j_first = S == 1 ? 0 : sp * rpc;
@@ -228,7 +214,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
         for (int s = 0; s < NB; ++s) {
             if (s >= j_count) break;   // (every loop over rows leaves at the last row: the unrolled rest is never fetched)
-            hres[s] = nl < a.seg_rows ? ld_cg_pinned(hp + (size_t)(j_first + s) * a.e.ldo + seg * a.seg_rows + nl) : 0.f;
+            hres[s] = nl < a.seg_rows ? __ldcg(hp + (size_t)(j_first + s) * a.e.ldo + seg * a.seg_rows + nl) : 0.f;
         }
     }
     if (ln_regs) {
@@ -257,7 +243,8 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
             for (int i = 0; i < C::STAGES; ++i) {
                 const int kb = kb0 + i;
-                if (i < nkb && (kb & 1) == (lane >> 4)) {
+                if (i >= nkb) break;
+                if ((kb & 1) == (lane >> 4)) {
                     const int u = kb >> 1;
                     float4 xv = t[0];
 #pragma unroll
@@ -282,7 +269,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         if (tid == 0) TC_PROBE(6);
     } else {
         // general case: statistics (LayerNorm), then the K-blocks a ring's worth at a time
-        if (PRO == PRO_LN && a.ln_part == nullptr) {
+        if (PRO == PRO_LN) {
             for (int r = warp; r < a.rows; r += 4) {   // one warp per row, fixed lane-strided order
                 const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx);
                 float mu, var;
@@ -325,64 +312,28 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         for (int i0 = 0; i0 < nkb; i0 += C::STAGES) {
             // a ring's worth of K-blocks at a time: all loads first, so their latencies overlap
             uint4 raw[PRO == PRO_BF16 ? C::STAGES : 1][CPT];
-            float4 xf[PRO == PRO_BF16 ? 1 : C::STAGES][CPT][2];
+            if (PRO == PRO_BF16) {
 #pragma unroll
-            for (int g = 0; g < C::STAGES; ++g)
+                for (int g = 0; g < C::STAGES; ++g)
 #pragma unroll
-                for (int ch = 0; ch < CPT; ++ch) {
-                    const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
-                    const int k = (kb0 + i0 + g) * 64 + c * 8;
-                    const bool in = i0 + g < nkb && r < a.rows && k < a.K;
-                    if (PRO == PRO_BF16) {
-                        raw[g][ch] = in ? __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k))
-                                        : make_uint4(0u, 0u, 0u, 0u);
-                    } else {
-                        const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
-                        xf[g][ch][0] = in ? __ldcg(xp) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        xf[g][ch][1] = in ? __ldcg(xp + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int ch = 0; ch < CPT; ++ch) {
+                        const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
+                        const int k = (kb0 + i0 + g) * 64 + c * 8;
+                        raw[g][ch] = (i0 + g < nkb && r < a.rows && k < a.K)
+                                         ? __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k))
+                                         : make_uint4(0u, 0u, 0u, 0u);
                     }
-                }
-            if (PRO == PRO_LN) {
-                // gains and biases of these K-blocks go through shared memory: thread t fetches floats 4t .. 4t+3
-                float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), b4 = g4;
-                const int kg = (kb0 + i0) * 64 + tid * 4;
-                if (tid < C::STAGES * 16 && i0 + (tid >> 4) < nkb && kg < a.K) {
-                    g4 = __ldg(reinterpret_cast<const float4*>(a.ln_g + kg));
-                    b4 = __ldg(reinterpret_cast<const float4*>(a.ln_b + kg));
-                }
-                if (i0 == 0 && a.ln_part != nullptr && tid < a.rows) {
-                    // row statistics from the pieces the producing kernels left, merged in piece order
-                    const float2* pr = reinterpret_cast<const float2*>(a.ln_part) + (size_t)tid * a.ln_ld;
-                    const int P = (a.K + a.ln_pw - 1) / a.ln_pw;
-                    float na = 0.f, mean = 0.f, m2 = 0.f;
-                    for (int p0 = 0; p0 < P; p0 += 16) {
-                        float2 t[16];
-#pragma unroll
-                        for (int u = 0; u < 16; ++u) t[u] = p0 + u < P ? __ldcg(pr + p0 + u) : make_float2(0.f, 0.f);
-#pragma unroll
-                        for (int u = 0; u < 16; ++u)
-                            if (p0 + u < P) moments_merge(na, mean, m2, (float)min(a.ln_pw, a.K - (p0 + u) * a.ln_pw), t[u].x, t[u].y);
-                    }
-                    s_mu[tid] = mean;
-                    s_rstd[tid] = 1.0f / sqrtf(m2 / (float)a.K + 1e-5f);
-                }
-                bar_sync(1, 128);   // the previous round's readers are done with s_gb; s_mu / s_rstd are written
-                if (tid < C::STAGES * 16) {
-                    *reinterpret_cast<float4*>(&s_gb[tid * 4]) = g4;
-                    *reinterpret_cast<float4*>(&s_gb[C::STAGES * 64 + tid * 4]) = b4;
-                }
-                bar_sync(1, 128);
             }
             bool dead = false;
 #pragma unroll
             for (int g = 0; g < C::STAGES; ++g) {
                 const int i = i0 + g;
-                if (i >= nkb || dead) continue;
+                if (i >= nkb || dead) break;
                 const int st = g;   // i0 is a multiple of STAGES
                 if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
                     tc_report(a.err_flag, TC_ERR_SLOT);
                     dead = true;
-                    continue;
+                    break;
                 }
                 unsigned char* bt = ring + st * C::STAGE_BYTES + C::A_BYTES;
 #pragma unroll
@@ -391,17 +342,19 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                     uint4 val = make_uint4(0u, 0u, 0u, 0u);
                     if (PRO == PRO_BF16) {
                         val = raw[g][ch];
-                    } else if (r < a.rows && (kb0 + i) * 64 + c * 8 < a.K) {
-                        float4 u0 = xf[g][ch][0], u1 = xf[g][ch][1];
-                        if (PRO == PRO_LN) {
-                            const float mu = s_mu[r], rs = s_rstd[r];
-                            const float4* gp = reinterpret_cast<const float4*>(&s_gb[g * 64 + c * 8]);
-                            const float4* bp = reinterpret_cast<const float4*>(&s_gb[C::STAGES * 64 + g * 64 + c * 8]);
-                            u0 = ln_apply(u0, mu, rs, gp[0], bp[0]);
-                            u1 = ln_apply(u1, mu, rs, gp[1], bp[1]);
+                    } else {
+                        const int k = (kb0 + i) * 64 + c * 8;
+                        if (r < a.rows && k < a.K) {
+                            const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
+                            float4 u0 = __ldcg(xp), u1 = __ldcg(xp + 1);
+                            if (PRO == PRO_LN) {
+                                const float mu = s_mu[r], rs = s_rstd[r];
+                                u0 = ln_apply(u0, mu, rs, __ldg(reinterpret_cast<const float4*>(a.ln_g + k)), __ldg(reinterpret_cast<const float4*>(a.ln_b + k)));
+                                u1 = ln_apply(u1, mu, rs, __ldg(reinterpret_cast<const float4*>(a.ln_g + k) + 1), __ldg(reinterpret_cast<const float4*>(a.ln_b + k) + 1));
+                            }
+                            val.x = pack_bf16x2(u0.x, u0.y); val.y = pack_bf16x2(u0.z, u0.w);
+                            val.z = pack_bf16x2(u1.x, u1.y); val.w = pack_bf16x2(u1.z, u1.w);
                         }
-                        val.x = pack_bf16x2(u0.x, u0.y); val.y = pack_bf16x2(u0.z, u0.w);
-                        val.z = pack_bf16x2(u1.x, u1.y); val.w = pack_bf16x2(u1.z, u1.w);
                     }
                     // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
                     *reinterpret_cast<uint4*>(bt + r * 128 + ((c ^ (r & 7)) << 4)) = val;
@@ -495,9 +448,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         }
         // v[s] is now the finished product of token row j_first + s and this thread's feature
         if (warp < 4) {
-            constexpr bool STAT = EPI == EPI_RESID || EPI == EPI_STORE_F32;
-            const bool stat = STAT && a.e.stat != nullptr;
-            const int cnt_w = min(32, max(0, a.seg_rows - (n_local0 + warp * 32)));   // valid features in this warp
             ScatterCol sc;
             if (EPI == EPI_QKV || EPI == EPI_KV) sc = scatter_col<EPI>(a.e, seg, n_local);
 #pragma unroll
@@ -517,25 +467,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                             epilogue<bf16, EPI>(a.e, j, n, hv);
                         }
                     }
-                    if (stat) {
-                        // mean and squared deviations of what this warp wrote of row j (two passes over registers)
-                        const float mw = cnt_w > 0 ? warp_sum(valid ? hv : 0.f) / (float)cnt_w : 0.f;
-                        const float dv = valid ? hv - mw : 0.f;
-                        const float qw = warp_sum(dv * dv);
-                        if (lane == 0) { s_av[warp][s] = mw; s_ai[warp][s] = __float_as_int(qw); }
-                    }
-                }
-            }
-            if (stat) {
-                bar_sync(1, 128);
-                if (tid < j_count) {   // the four warps' pieces merged in warp order: one piece per (row, tile)
-                    float na = 0.f, mean = 0.f, m2 = 0.f;
-#pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        const int cw = min(32, max(0, a.seg_rows - (n_local0 + w * 32)));
-                        if (cw > 0) moments_merge(na, mean, m2, (float)cw, s_av[w][tid], __int_as_float(s_ai[w][tid]));
-                    }
-                    reinterpret_cast<float2*>(a.e.stat)[(size_t)(j_first + tid) * a.e.stat_ld + tile] = make_float2(mean, m2);
                 }
             }
         }

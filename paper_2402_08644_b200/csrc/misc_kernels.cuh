@@ -75,14 +75,6 @@ __device__ __forceinline__ int argmax_from_tiles(const float* val, const int* id
     return bi == INT_MAX ? 0 : bi;
 }
 
-__device__ __forceinline__ float block_sum_128(float v, float* red) {
-    v = warp_sum(v);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    return red[0] + red[1] + red[2] + red[3];
-}
-
 // Start of a pass over decode rows: row set-up and x^(0) = Emb(t) + Pos(index) in one kernel (Eq. 1).
 // Row m = b*nq + (r - r0) carries block row r of sequence b (row 0 = pending token, row r = draft r).
 // The token of block row fin_r is not known yet as an id: it is the arg-max of the small model's last
@@ -91,10 +83,8 @@ template <typename T>
 __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, int nq, int fin_r, const float* amax_val,
                                                          const int* amax_idx, int amax_stride, int n_tiles, int* row_tok,
                                                          int* row_seq, int* row_pos, const T* __restrict__ emb,
-                                                         const T* __restrict__ pos, float* __restrict__ h, int d, bf16* snap,
-                                                         float* stat, int stat_ld) {
+                                                         const T* __restrict__ pos, float* __restrict__ h, int d, bf16* snap) {
     __shared__ int s_tok, s_pos;
-    __shared__ float s_red[4];
     TC_PROBE_INIT(300);
     pdl_wait();
     pdl_launch_dependents();
@@ -116,25 +106,20 @@ __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, i
     __syncthreads();
     const T* er = emb + (size_t)s_tok * d;
     const T* pr = pos + (size_t)s_pos * d;
-    float sum = 0.f;
     for (int i = threadIdx.x; i < d; i += 128) {
         const float v = to_float(er[i]) + to_float(pr[i]);
         h[(size_t)m * d + i] = v;
         if (snap) snap[(size_t)m * d + i] = __float2bfloat16_rn(v);   // bf16 copy for the FF_Tandem projection of x^(0)
-        sum += v;
-    }
-    if (stat) {
-        // mean and sum of squared deviations of the row, as one piece, for the first LayerNorm that reads it
-        const float mean = block_sum_128(sum, s_red) / (float)d;
-        float q = 0.f;
-        for (int i = threadIdx.x; i < d; i += 128) {
-            const float dv = to_float(er[i]) + to_float(pr[i]) - mean;
-            q = fmaf(dv, dv, q);
-        }
-        q = block_sum_128(q, s_red);
-        if (threadIdx.x == 0) reinterpret_cast<float2*>(stat)[(size_t)m * stat_ld] = make_float2(mean, q);
     }
     if (threadIdx.x == 0) TC_PROBE(2);
+}
+
+__device__ __forceinline__ float block_sum_128(float v, float* red) {
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    return red[0] + red[1] + red[2] + red[3];
 }
 
 // LayerNorm of fp32 rows (biased variance, eps 1e-5), output in the storage type.  grid: rows; block: 128.

@@ -745,7 +745,7 @@ void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r
     launch_ex(c, true, 1, step_begin_kernel<bf16>, dim3(c.batch * nq), dim3(128), 0, c.st, r0, nq, fin_r,
               (const float*)at<float>(c, c.lay.amax_val_small), (const int*)at<int>(c, c.lay.amax_idx_small), c.lay.vocab_tiles,
               c.lay.vocab_tiles, at<int>(c, c.lay.row_tok), at<int>(c, c.lay.row_seq), at<int>(c, c.lay.row_pos),
-              (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model, snap, (float*)nullptr, 0);
+              (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model, snap);
 }
 
 // Whether LayerNorm (or the fp32 -> bf16 cast) is fused into the GEMM's operand load.  Fused, every CTA of the

@@ -19,14 +19,6 @@ namespace tandem {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
-// A global load (L2 only) that is issued where it is written: plain loads are free to sink to their first use,
-// which defeats fetching a value early, behind other work.
-__device__ __forceinline__ float ld_cg_pinned(const float* p) {
-    float v;
-    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
-    return v;
-}
-
 // ---- programmatic dependent launch --------------------------------------------------------------
 // pdl_wait: blocks until every grid this one depends on has finished and its writes are visible.
 // pdl_launch_dependents: lets the next grid in the stream start its independent prologue early.
