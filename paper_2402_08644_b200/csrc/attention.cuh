@@ -315,9 +315,9 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     const int QPC = (ATT_NQ + CL - 1) / CL;        // queries a CTA finishes at most
     bf16* ring = ring_all + (size_t)warp * C::STAGES * C::STAGE_ELEMS;
     const uint32_t ring_s = smem_u32(ring);
-    pdl_wait();   // queries and the newest keys/values come from earlier kernels
-    pdl_launch_dependents();
-    if (tid == 0) TC_PROBE(1);
+    // The row arrays were written at the start of the pass, at least two kernels back in the stream, so they may be
+    // read before the wait below: a kernel lets its successor start only after its own wait has returned, that is
+    // after its predecessor has finished, hence everything older than the immediate predecessor is complete.
     const int cnt = a.nq, row0 = g * a.nq;
     const int b = a.row_seq[row0];
     const int pos_first = a.row_pos[row0];
@@ -373,10 +373,26 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
             }
         }
     };
+    // Tiles that end before the block's first position hold committed keys and values from earlier iterations (or
+    // earlier steps of this one): they are fetched before the wait; what the predecessor may have written, after it.
+    int pre = 0;
 #pragma unroll
     for (int it = 0; it < C::STAGES - 1; ++it) {
-        if (it < n_mine) issue(it);
-        cp_async_commit();
+        if (it == pre && it < n_mine && (rank + it * CL) * ATT_CH + (warp + 1) * ATD_WROWS <= pos_first) {
+            issue(it);
+            cp_async_commit();
+            ++pre;
+        }
+    }
+    pdl_wait();   // queries and the newest keys/values come from the kernel before this one
+    pdl_launch_dependents();
+    if (tid == 0) TC_PROBE(1);
+#pragma unroll
+    for (int it = 0; it < C::STAGES - 1; ++it) {
+        if (it >= pre) {
+            if (it < n_mine) issue(it);
+            cp_async_commit();
+        }
     }
 
     // The queries as A fragments: this lane holds rows lane/4 and lane/4 + 8, columns 2*(lane%4) (+1) (+8) of each
