@@ -143,12 +143,20 @@ __global__ void __launch_bounds__(128) layernorm_kernel(const float* __restrict_
 __global__ void __launch_bounds__(128) layernorm_rows_bf16_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                                                   const float* __restrict__ bias, bf16* __restrict__ out, int d) {
     __shared__ float red[4];
-    pdl_wait();
-    pdl_launch_dependents();
     const int d4 = d >> 2;
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)blockIdx.x * d);
     uint2* orow = reinterpret_cast<uint2*>(out + (size_t)blockIdx.x * d);
     if (d4 <= 8 * 128) {
+        // gains and biases are parameters: fetched while the kernel that writes x is still running
+        float4 gq[8], bq[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int k4 = threadIdx.x + 128 * u;
+            gq[u] = k4 < d4 ? __ldg(reinterpret_cast<const float4*>(gain) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            bq[u] = k4 < d4 ? __ldg(reinterpret_cast<const float4*>(bias) + k4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        pdl_wait();
+        pdl_launch_dependents();
         float4 t[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) t[u] = (threadIdx.x + 128 * u < d4) ? __ldcg(xr + threadIdx.x + 128 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -169,13 +177,15 @@ __global__ void __launch_bounds__(128) layernorm_rows_bf16_kernel(const float* _
         for (int u = 0; u < 8; ++u) {
             const int k4 = threadIdx.x + 128 * u;
             if (k4 < d4) {
-                const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + k4), b = __ldg(reinterpret_cast<const float4*>(bias) + k4);
+                const float4 g = gq[u], b = bq[u];
                 const __nv_bfloat162 lo = __floats2bfloat162_rn((t[u].x - mu) * rs * g.x + b.x, (t[u].y - mu) * rs * g.y + b.y);
                 const __nv_bfloat162 hi = __floats2bfloat162_rn((t[u].z - mu) * rs * g.z + b.z, (t[u].w - mu) * rs * g.w + b.w);
                 orow[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
             }
         }
     } else {
+        pdl_wait();
+        pdl_launch_dependents();
         float s = 0.f;
         for (int k4 = threadIdx.x; k4 < d4; k4 += 128) { const float4 t = __ldcg(xr + k4); s += (t.x + t.y) + (t.z + t.w); }
         const float mu = block_sum_128(s, red) / d;
