@@ -262,6 +262,31 @@ def test_gpu_speed_equals_gpu_greedy_bit_exact(dtype):
     t.close()
 
 
+@pytest.mark.parametrize("gamma,large,small", [(9, (3, 128, 4, 256), (2, 64, 2, 136)),      # head size 32
+                                               (15, (2, 256, 4, 512), (2, 128, 2, 256)),    # head size 64
+                                               (11, (2, 256, 2, 512), (2, 128, 1, 256))])   # head size 128
+def test_bf16_long_blocks_replay_and_equal_greedy(gamma, large, small):
+    """Blocks of more than eight rows (both halves of the attention's 16-row tile carry queries), every head size:
+    logits against the checker, and GPU SPEED == GPU greedy."""
+    shape = gpu_toy_shape(dtype=synth.DTYPE_BF16, layer_map=(1, 2), large=large, small=small)
+    w = toy_weights(shape, seed=53, std=0.05)
+    for k in w:
+        if not synth.is_norm_param(k):
+            w[k] = synth.round_to_bf16(w[k])
+    prompts = prompts_for(shape, [131, 7], seed=12)
+    flips = _replay_compare(shape, w, prompts, gamma, 2, TOL_BF16, 2 * TOL_BF16)
+    assert flips <= 2 * (gamma + 1)
+    t = binding.Tandem(shape, w, max_batch=2, max_seq=shape.large.max_pos, gamma_max=gamma)
+    t.tandem_prefill(prompts)
+    greedy, _, _ = t.tandem_large_greedy_generate(40)
+    for mode in (0, 1):
+        t.tandem_prefill(prompts)
+        got, _, _ = t.tandem_speculative_generate(gamma, 40, mode)
+        if mode == 0:
+            assert got.tolist() == greedy.tolist()
+    t.close()
+
+
 def test_bf16_small_config_speed_equals_greedy_full_prompt():
     """Config "small" at its full prompt length (512) and gamma 3: GPU SPEED == GPU greedy, and the natural
     accept histogram is what the call reports."""
