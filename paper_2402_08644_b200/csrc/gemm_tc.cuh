@@ -13,7 +13,7 @@
 //                          stream (programmatic dependent launch), so they overlap its run; a kernel lets its
 //                          own successor start once the predecessor is done, which keeps one kernel's worth of
 //                          prefetch in flight (deeper chains of waiting kernels cost more than they hide).
-//  gemm_tc_tiled_kernel    many rows (prompt pass): 128 x 128 output tiles, both operands by TMA.
+//  gemm_tc_tiled_kernel    many rows (prompt pass): 128 x 256 output tiles, both operands by TMA.
 //
 // An output element's reduction order depends on (N, K) only, never on the number of rows, so a block
 // pass and a one-row pass give identical bits.
@@ -480,7 +480,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Many rows: 128 x 128 output tiles, A = token rows, B = weight rows, both by TMA.
+// Many rows: 128 x 256 output tiles, A = token rows, B = weight rows, both by TMA.
 // ---------------------------------------------------------------------------------------------------
 
 struct TcTiledArgs {
@@ -491,11 +491,15 @@ struct TcTiledArgs {
 };
 
 constexpr int TCT_THREADS = 192;
-constexpr int TCT_STAGES = 6;
-constexpr int TCT_TILE_BYTES = 128 * 128;
-constexpr int TCT_STAGE_BYTES = 2 * TCT_TILE_BYTES;
-constexpr int TCT_SMEM_BYTES = TCT_STAGES * TCT_STAGE_BYTES + 1024;
-constexpr int TCT_TMEM_COLS = 128;
+constexpr int TCT_TILE_BYTES = 128 * 128;          // one TMA box: 128 rows x 64 bf16
+// BN = output features per tile: 256 when that still fills the GPU (each token-row tile read from shared memory then
+// feeds twice the MMA work of a square tile), else 128.
+template <int BN> struct TctCfg {
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int STAGE_BYTES = (1 + BN / 128) * TCT_TILE_BYTES;   // token rows, then the weight rows (one box per 128)
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
+    static constexpr int TMEM_COLS = BN;
+};
 
 // Sixteen consecutive output features of one row.  n_local0 is a multiple of 16.
 template <int EPI>
@@ -544,14 +548,15 @@ __device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int seg, int
     reinterpret_cast<uint4*>(dst)[1] = hi;
 }
 
-// grid: (tiles over all segments, ceil(M / 128)); dynamic smem TCT_SMEM_BYTES.
-template <int EPI>
+// grid: (tiles of BN output features over all segments, ceil(M / 128)); dynamic smem TctCfg<BN>::SMEM_BYTES.
+template <int EPI, int BN>
 __global__ void __launch_bounds__(TCT_THREADS)
 gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tm0,
                      const __grid_constant__ CUtensorMap tm1, const __grid_constant__ CUtensorMap tm2) {
+    using C = TctCfg<BN>;
     extern __shared__ __align__(1024) unsigned char smem_dyn[];
-    __shared__ __align__(8) uint64_t s_full[TCT_STAGES];
-    __shared__ __align__(8) uint64_t s_empty[TCT_STAGES];
+    __shared__ __align__(8) uint64_t s_full[C::STAGES];
+    __shared__ __align__(8) uint64_t s_empty[C::STAGES];
     __shared__ __align__(8) uint64_t s_accum;
     __shared__ uint32_t s_tmem;
 
@@ -559,18 +564,18 @@ gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tm
     const uint32_t ring0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     const int tile = blockIdx.x;
     const int seg = tile / a.tiles_per_seg;
-    const int n_local0 = (tile - seg * a.tiles_per_seg) * 128;
+    const int n_local0 = (tile - seg * a.tiles_per_seg) * BN;
     const int m0 = blockIdx.y * 128;
     const int KB = (a.K + 63) >> 6;
 
     if (warp == 5) {
         if (lane == 0) {
-            for (int s = 0; s < TCT_STAGES; ++s) { mbar_init(smem_u32(&s_full[s]), 1); mbar_init(smem_u32(&s_empty[s]), 1); }
+            for (int s = 0; s < C::STAGES; ++s) { mbar_init(smem_u32(&s_full[s]), 1); mbar_init(smem_u32(&s_empty[s]), 1); }
             mbar_init(smem_u32(&s_accum), 1);
             mbar_init_fence();
         }
         __syncwarp();
-        tmem_alloc(smem_u32(&s_tmem), TCT_TMEM_COLS);
+        tmem_alloc(smem_u32(&s_tmem), C::TMEM_COLS);
         tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -584,30 +589,32 @@ gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tm
             tma_prefetch_desc(&tmx);
             tma_prefetch_desc(tw);
             for (int i = 0; i < KB; ++i) {
-                const int st = i % TCT_STAGES;
-                if (i >= TCT_STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / TCT_STAGES) - 1) & 1)) {
+                const int st = i % C::STAGES;
+                if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
                     tc_report(a.err_flag, TC_ERR_SLOT);
                     break;
                 }
                 const uint32_t bar = smem_u32(&s_full[st]);
-                mbar_arrive_expect_tx(bar, TCT_STAGE_BYTES);
-                tma_load_2d_nohint(ring0 + st * TCT_STAGE_BYTES, &tmx, i * 64, m0, bar);
-                tma_load_2d_nohint(ring0 + st * TCT_STAGE_BYTES + TCT_TILE_BYTES, tw, i * 64, n_local0, bar);
+                mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+                tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES, &tmx, i * 64, m0, bar);
+#pragma unroll
+                for (int hb = 0; hb < BN / 128; ++hb)   // rows past the segment's end arrive as zeros
+                    tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES + (1 + hb) * TCT_TILE_BYTES, tw, i * 64, n_local0 + hb * 128, bar);
             }
         }
         __syncwarp();
     } else if (warp == 5) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
+            constexpr uint32_t idesc = umma_idesc_bf16(128, BN);
             for (int i = 0; i < KB; ++i) {
-                const int st = i % TCT_STAGES;
-                if (!mbar_wait(smem_u32(&s_full[st]), (i / TCT_STAGES) & 1)) {
+                const int st = i % C::STAGES;
+                if (!mbar_wait(smem_u32(&s_full[st]), (i / C::STAGES) & 1)) {
                     tc_report(a.err_flag, TC_ERR_OPERANDS);
                     break;
                 }
                 tc_fence_after_sync();
-                const uint64_t da = umma_desc_k_sw128(ring0 + st * TCT_STAGE_BYTES);
-                const uint64_t db = umma_desc_k_sw128(ring0 + st * TCT_STAGE_BYTES + TCT_TILE_BYTES);
+                const uint64_t da = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES);
+                const uint64_t db = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES + TCT_TILE_BYTES);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
                 umma_commit(smem_u32(&s_empty[st]));
@@ -620,7 +627,7 @@ gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tm
         tc_fence_after_sync();
         const int m = m0 + warp * 32 + lane;   // output row = TMEM lane
 #pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 16) {
+        for (int c0 = 0; c0 < BN; c0 += 16) {
             float t[16];
             tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c0, t);   // warp-wide: every lane takes part
             if (m < a.M && n_local0 + c0 < a.seg_rows) epilogue16<EPI>(a.e, m, seg, a.seg_rows, n_local0 + c0, t);
@@ -628,7 +635,7 @@ gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tm
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem, TCT_TMEM_COLS);
+    if (warp == 5) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 }  // namespace tandem

@@ -396,15 +396,23 @@ void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx
 }
 
 // y = x W^T for many rows on the tensor cores; x bf16 [M][ldx].
-template <int EPI>
-tandem_status launch_tc_tiled(tandem_ctx& c, const bf16* x, int ldx, int M, const TcW& w, const EpiArgs& e, int* err) {
-    if (M <= 0) return TANDEM_OK;
+template <int EPI, int BN>
+void launch_tc_tiled_bn(tandem_ctx& c, TcTiledArgs& a, const CUtensorMap& tmx, const TcW& w, int M) {
+    using C = TctCfg<BN>;
     static bool attr_set[MAX_DEVICES] = {};
     const int dev = cur_dev();
     if (!attr_set[dev]) {
-        cudaFuncSetAttribute(gemm_tc_tiled_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TCT_SMEM_BYTES);
+        cudaFuncSetAttribute(gemm_tc_tiled_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
         attr_set[dev] = true;
     }
+    a.tiles_per_seg = cdiv(w.seg_rows, BN);
+    launch_ex(c, false, 1, gemm_tc_tiled_kernel<EPI, BN>, dim3(w.n_segs * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)C::SMEM_BYTES,
+              a, tmx, w.tm[0], w.tm[1], w.tm[2]);
+}
+
+template <int EPI>
+tandem_status launch_tc_tiled(tandem_ctx& c, const bf16* x, int ldx, int M, const TcW& w, const EpiArgs& e, int* err) {
+    if (M <= 0) return TANDEM_OK;
     CUtensorMap tmx;
     if (!make_tmap_bf16(&tmx, x, (uint64_t)M, (uint64_t)w.K, (uint64_t)ldx)) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled failed for an activation buffer");
@@ -412,11 +420,12 @@ tandem_status launch_tc_tiled(tandem_ctx& c, const bf16* x, int ldx, int M, cons
     }
     TcTiledArgs a;
     memset(&a, 0, sizeof(a));
-    a.M = M; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
+    a.M = M; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows;
     a.err_flag = err; a.e = e;
     ProfScope ps(c, PC_GEMM_TC_TILED, 2.0 * M * (double)a.N * w.K);   // flops
-    launch_ex(c, false, 1, gemm_tc_tiled_kernel<EPI>, dim3(w.n_segs * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)TCT_SMEM_BYTES,
-              a, tmx, w.tm[0], w.tm[1], w.tm[2]);
+    // 256-wide tiles when they still give every SM a tile, else square ones
+    if ((long long)w.n_segs * cdiv(w.seg_rows, 256) * cdiv(M, 128) >= 148) launch_tc_tiled_bn<EPI, 256>(c, a, tmx, w, M);
+    else launch_tc_tiled_bn<EPI, 128>(c, a, tmx, w, M);
     return TANDEM_OK;
 }
 
