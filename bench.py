@@ -402,8 +402,11 @@ def main():
         prof = t.tandem_profile_read()
         t.tandem_profile_enable(0)
         tot = sum(v["ms"] for v in prof.values()) or 1.0
+        # work: algorithmic bytes per second (GB/s) for the streaming kernels, flops per second (TFLOP/s) for the prompt pass
         line["kernels"] = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / tot, 4),
-                               "avg_us": round(1e3 * v["ms"] / max(1, v["launches"]), 3)} for k, v in prof.items()}
+                               "avg_us": round(1e3 * v["ms"] / max(1, v["launches"]), 3),
+                               "rate": round(v["work"] / (v["ms"] * 1e-3) / (1e12 if k in ("gemm_tiled", "gemm_tc_tiled", "attn_prompt") else 1e9), 1)
+                               if v["ms"] > 0 else 0.0} for k, v in prof.items()}
         flop_classes = ("gemm_tiled", "gemm_tc_tiled", "attn_prompt")     # prompt-pass kernels: work counted in flops
         dom = max((k for k in prof if k not in flop_classes), key=lambda k: prof[k]["ms"])
         g = prof[dom]

@@ -161,15 +161,22 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
         for (int c = 0; c < n_chunks && ok; ++c) {
             if (!mbar_wait(smem_u32(&s_sfull), c & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); ok = false; break; }
             tc_fence_after_sync();
-            // pass 1: the row's maximum over this chunk
+            // pass 1: the row's maximum over this chunk (every chunk but the tile's last one or two lies wholly before
+            // the tile's first query: no key of it is masked for any row)
+            const bool full = c * 128 + 127 <= pos_first;
             float mc = -INFINITY;
 #pragma unroll 1
             for (int c0 = 0; c0 < 128; c0 += 16) {
                 float t[16];
                 tmem_ld16(lane_addr + c0, t);
+                if (full) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (c * 128 + c0 + i <= qpos) mc = fmaxf(mc, t[i] * a.scale);
+                    for (int i = 0; i < 16; ++i) mc = fmaxf(mc, t[i] * a.scale);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (c * 128 + c0 + i <= qpos) mc = fmaxf(mc, t[i] * a.scale);
+                }
             }
             const float mn = fmaxf(m, mc);
             const float f = m > -INFINITY ? __expf(m - mn) : 0.f;
@@ -184,8 +191,8 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
                 uint32_t pk[8];
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
-                    const float p0v = (c * 128 + c0 + i <= qpos && mn > -INFINITY) ? __expf(t[i] * a.scale - mn) : 0.f;
-                    const float p1v = (c * 128 + c0 + i + 1 <= qpos && mn > -INFINITY) ? __expf(t[i + 1] * a.scale - mn) : 0.f;
+                    const float p0v = (full || (c * 128 + c0 + i <= qpos && mn > -INFINITY)) ? __expf(t[i] * a.scale - mn) : 0.f;
+                    const float p1v = (full || (c * 128 + c0 + i + 1 <= qpos && mn > -INFINITY)) ? __expf(t[i + 1] * a.scale - mn) : 0.f;
                     const __nv_bfloat162 pb = __floats2bfloat162_rn(p0v, p1v);
                     // the sum uses the rounded values, the same ones the tensor core multiplies with V
                     ls += __bfloat162float(pb.x) + __bfloat162float(pb.y);
@@ -197,8 +204,10 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
                 *reinterpret_cast<uint4*>(prow + (((ch + 1) ^ (qi & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
             }
             l = l * f + ls;
+            if (f != 1.f) {   // a factor of exactly 1 (no new maximum) changes nothing
 #pragma unroll
-            for (int e = 0; e < DH; ++e) o[e] *= f;
+                for (int e = 0; e < DH; ++e) o[e] *= f;
+            }
             tc_fence_before_sync();      // the TMEM reads of S are done before the next chunk's MMA may overwrite it
             fence_proxy_async_smem();
             __syncwarp();
