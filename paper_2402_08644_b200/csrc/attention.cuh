@@ -319,8 +319,8 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     // read before the wait below: a kernel lets its successor start only after its own wait has returned, that is
     // after its predecessor has finished, hence everything older than the immediate predecessor is complete.
     const int cnt = a.nq, row0 = g * a.nq;
-    const int b = a.row_seq[row0];
-    const int pos_first = a.row_pos[row0];
+    const int b = __ldcg(a.row_seq + row0);          // from L2: nothing an earlier kernel on this SM may have cached
+    const int pos_first = __ldcg(a.row_pos + row0);
     const int pos_last = pos_first + cnt - 1;
     const int n_chunks = pos_last / ATT_CH + 1;
     const int n_mine = rank < n_chunks ? (n_chunks - rank + CL - 1) / CL : 0;
