@@ -9,7 +9,9 @@
 //                       ([key][element], i.e. MN-major for the B operand)
 //     O  = O * f + PV   in the thread's registers (f rescales to the new maximum)
 // Warp 4 streams K and V chunks by TMA through a two-stage ring, warp 5 allocates TMEM and issues the MMAs,
-// warps 0-3 do the softmax and the epilogue.  Every wait is bounded.
+// warps 0-3 do the softmax and the epilogue.  The tensor work hides behind the softmax: S of chunk c+1 (a second S
+// buffer in TMEM) is computed while the softmax warps work on chunk c, and PV of chunk c while they take the maximum
+// of chunk c+1; they add PV of chunk c only then.  Every wait is bounded.
 #pragma once
 #include "common.cuh"
 #include "gemm_tc.cuh"
@@ -35,7 +37,7 @@ template <int DH> struct AtcCfg {
     static constexpr int KV_BYTES = 2 * NSUB * ATC_SUB;        // K and V of one chunk
     static constexpr int P_BYTES = 2 * ATC_SUB;                // 128 queries x 128 keys bf16
     static constexpr int SMEM_BYTES = Q_BYTES + 2 * KV_BYTES + P_BYTES + 1024;
-    static constexpr int TMEM_COLS = 256;                      // S: columns 0..127, PV: 128..128+DH-1
+    static constexpr int TMEM_COLS = 512;                      // S of even chunks: columns 0..127, PV: 128..128+DH-1, S of odd chunks: 256..383
 };
 
 // Instruction descriptor: bf16 A (K-major) and B, fp32 accumulation; b_mn = 1 when B is MN-major.
@@ -62,7 +64,7 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
                        const __grid_constant__ CUtensorMap tmv) {
     using C = AtcCfg<DH>;
     extern __shared__ __align__(1024) unsigned char smem_dyn[];
-    __shared__ __align__(8) uint64_t s_qfull, s_kvfull[2], s_kvfree[2], s_sfull, s_pready, s_ofull;
+    __shared__ __align__(8) uint64_t s_qfull, s_kvfull[2], s_kvfree[2], s_sfull[2], s_pready, s_ofull;
     __shared__ uint32_t s_tmem;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -84,7 +86,8 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
         if (lane == 0) {
             mbar_init(smem_u32(&s_qfull), 1);
             for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&s_kvfull[s]), 1); mbar_init(smem_u32(&s_kvfree[s]), 1); }
-            mbar_init(smem_u32(&s_sfull), 1);
+            mbar_init(smem_u32(&s_sfull[0]), 1);
+            mbar_init(smem_u32(&s_sfull[1]), 1);
             mbar_init(smem_u32(&s_pready), 4);   // one arrive per softmax warp
             mbar_init(smem_u32(&s_ofull), 1);
             mbar_init_fence();
@@ -122,21 +125,30 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
             constexpr uint32_t idesc_o = umma_idesc_bf16_b(128, DH, 1);
             bool ok = mbar_wait(smem_u32(&s_qfull), 0);
             if (!ok) tc_report(a.err_flag, TC_ERR_OPERANDS);
-            for (int c = 0; c < n_chunks && ok; ++c) {
+            // S = Q K^T of chunk c into the S buffer c & 1: both K-major, 16 elements of the head dimension per instruction
+            auto issue_s = [&](int c) -> bool {
                 const int st = c & 1;
-                if (!mbar_wait(smem_u32(&s_kvfull[st]), (c >> 1) & 1)) { tc_report(a.err_flag, TC_ERR_OPERANDS); break; }
+                if (!mbar_wait(smem_u32(&s_kvfull[st]), (c >> 1) & 1)) { tc_report(a.err_flag, TC_ERR_OPERANDS); return false; }
                 tc_fence_after_sync();
-                const uint32_t kaddr = kv0 + st * C::KV_BYTES, vaddr = kaddr + C::NSUB * ATC_SUB;
-                // S = Q K^T: both K-major, 16 elements of the head dimension per instruction
+                const uint32_t kaddr = kv0 + st * C::KV_BYTES;
 #pragma unroll
                 for (int sb = 0; sb < C::NSUB; ++sb)
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem, umma_desc_k_sw128(q0 + sb * ATC_SUB) + 2 * k, umma_desc_k_sw128(kaddr + sb * ATC_SUB) + 2 * k, idesc_s,
+                        umma_bf16(tmem + st * 256, umma_desc_k_sw128(q0 + sb * ATC_SUB) + 2 * k, umma_desc_k_sw128(kaddr + sb * ATC_SUB) + 2 * k, idesc_s,
                                   (sb | k) != 0 ? 1u : 0u);
-                umma_commit(smem_u32(&s_sfull));
+                umma_commit(smem_u32(&s_sfull[st]));
+                return true;
+            };
+            ok = ok && issue_s(0);
+            for (int c = 0; c < n_chunks && ok; ++c) {
+                const int st = c & 1;
+                // the next chunk's scores are computed while the softmax warps work on this one (its S buffer was
+                // released with the probabilities of chunk c - 1)
+                if (c + 1 < n_chunks && !issue_s(c + 1)) break;
                 if (!mbar_wait(smem_u32(&s_pready), c & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); break; }
                 tc_fence_after_sync();
+                const uint32_t vaddr = kv0 + st * C::KV_BYTES + C::NSUB * ATC_SUB;
                 // PV = P V: P K-major (two 64-key sub-tiles), V MN-major; 16 keys per instruction
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -159,8 +171,9 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         for (int c = 0; c < n_chunks && ok; ++c) {
-            if (!mbar_wait(smem_u32(&s_sfull), c & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); ok = false; break; }
+            if (!mbar_wait(smem_u32(&s_sfull[c & 1]), (c >> 1) & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); ok = false; break; }
             tc_fence_after_sync();
+            const uint32_t s_addr = lane_addr + (c & 1) * 256;
             // pass 1: the row's maximum over this chunk (every chunk but the tile's last one or two lies wholly before
             // the tile's first query: no key of it is masked for any row)
             const bool full = c * 128 + 127 <= pos_first;
@@ -168,7 +181,7 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
 #pragma unroll 1
             for (int c0 = 0; c0 < 128; c0 += 16) {
                 float t[16];
-                tmem_ld16(lane_addr + c0, t);
+                tmem_ld16(s_addr + c0, t);
                 if (full) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) mc = fmaxf(mc, t[i] * a.scale);
@@ -181,13 +194,25 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
             const float mn = fmaxf(m, mc);
             const float f = m > -INFINITY ? __expf(m - mn) : 0.f;
             m = mn;
-            // (the previous chunk's P tile is free: its PV was awaited at the end of the last iteration)
+            // O += PV of the previous chunk (it ran during pass 1; it is on the scale of the previous maximum, like o),
+            // which also frees the P tile
+            if (c > 0) {
+                if (!mbar_wait(smem_u32(&s_ofull), (c - 1) & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); ok = false; break; }
+                tc_fence_after_sync();
+#pragma unroll
+                for (int e0 = 0; e0 < DH; e0 += 16) {
+                    float t[16];
+                    tmem_ld16(lane_addr + 128 + e0, t);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o[e0 + i] += t[i];
+                }
+            }
             // pass 2: probabilities, row sum, bf16 P tile (row qi: 128 keys = two sub-tiles of 64, 128-byte swizzle)
             float ls = 0.f;
 #pragma unroll 1
             for (int c0 = 0; c0 < 128; c0 += 16) {
                 float t[16];
-                tmem_ld16(lane_addr + c0, t);
+                tmem_ld16(s_addr + c0, t);
                 uint32_t pk[8];
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
@@ -212,15 +237,18 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&s_pready));
-            // O += PV of this chunk
-            if (!mbar_wait(smem_u32(&s_ofull), c & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); ok = false; break; }
+        }
+        if (ok) {   // the last chunk's PV
+            if (!mbar_wait(smem_u32(&s_ofull), (n_chunks - 1) & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); ok = false; }
             tc_fence_after_sync();
+            if (ok) {
 #pragma unroll
-            for (int e0 = 0; e0 < DH; e0 += 16) {
-                float t[16];
-                tmem_ld16(lane_addr + 128 + e0, t);
+                for (int e0 = 0; e0 < DH; e0 += 16) {
+                    float t[16];
+                    tmem_ld16(lane_addr + 128 + e0, t);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) o[e0 + i] += t[i];
+                    for (int i = 0; i < 16; ++i) o[e0 + i] += t[i];
+                }
             }
             tc_fence_before_sync();
         }
