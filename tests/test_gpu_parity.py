@@ -262,6 +262,22 @@ def test_gpu_speed_equals_gpu_greedy_bit_exact(dtype):
     t.close()
 
 
+@pytest.mark.parametrize("heads_large,heads_small", [(18, 6), (9, 3)])     # head size 64 / 128
+def test_bf16_long_prompt_wide_gemm_tiles_replay(heads_large, heads_small):
+    """A prompt long enough (1301 rows, eleven key chunks in the prompt attention) that the prompt-pass GEMMs with
+    many output features take their 256-wide tiles, with a model width (1152) that leaves a ragged last tile per
+    weight segment: the iterations that follow are compared with the checker, which has read the same prompt."""
+    shape = gpu_toy_shape(dtype=synth.DTYPE_BF16, layer_map=(1, 2), max_pos=1408, large=(2, 1152, heads_large, 4608),
+                          small=(2, 384, heads_small, 1536), vocab=499)
+    w = toy_weights(shape, seed=61, std=0.03)
+    for k in w:
+        if not synth.is_norm_param(k):
+            w[k] = synth.round_to_bf16(w[k])
+    flips = _replay_compare(shape, w, prompts_for(shape, [1301], seed=14), 3, 2, TOL_BF16 * (1152 / 1024.0) ** 0.5,
+                            2 * TOL_BF16 * (1152 / 1024.0) ** 0.5)
+    assert flips <= 3
+
+
 @pytest.mark.parametrize("gamma,large,small", [(9, (3, 128, 4, 256), (2, 64, 2, 136)),      # head size 32
                                                (15, (2, 256, 4, 512), (2, 128, 2, 256)),    # head size 64
                                                (11, (2, 256, 2, 512), (2, 128, 1, 256))])   # head size 128
