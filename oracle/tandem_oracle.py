@@ -18,7 +18,7 @@ representations, y_hat = projected large representations, gamma = block length):
   * Section 3.1: draft gamma tokens, verify the block, first mismatch, take the large model's token
     there, continue with the large model's representations of all previous tokens.
 
-Readings taken where the paper is silent or inconsistent (numbers match the design notes):
+Readings taken where the paper is silent or inconsistent:
   R1  Boundary.  Eq. 2 prints k = floor(i/gamma)*gamma, which would let a token at a multiple of gamma
       attend the large model's representation of itself.  The training bullets of Section 3 and
       Figure 3 say that the current block, including the query token, uses the small model's own
@@ -41,8 +41,8 @@ Readings taken where the paper is silent or inconsistent (numbers match the desi
       with the free token, Figure 2); accept_mode 2 takes a pseudo-random accept length from a
       counter-based hash (test only).
 
-Pins: every function here is pinned by tests/test_oracle_*.py (library decoder layer, brute force vs
-cache, SPEED == plain greedy, self-tandem, block == single-token passes, schedule fixtures from
+Pins: every function here is pinned by tests/test_oracle_*.py (library decoder layer, both FF_Tandem
+branches against library modules and closed forms, brute force vs cache, SPEED == plain greedy, self-tandem, block == single-token passes, schedule fixtures from
 Figures 2 and 3, hand-made accept cases).  The absolute logit values of a random-init *Tandem* pair
 have no value printed in the paper to compare with: for those, parity unpinned beyond the invariants.
 """

@@ -132,3 +132,58 @@ def test_splitmix64_matches_published_sequence_head():
     for g in (1, 3, 7):
         vals = {O.hashed_accept_length(11, 0, it, g) for it in range(200)}
         assert vals == set(range(g + 1))
+
+
+def _projection(kind, d_large, d_small, hidden, seed):
+    rng = np.random.default_rng(seed)
+    if kind == synth.FF_TANDEM_LINEAR:
+        w = {"T.0.w_t": rng.normal(size=(d_small, d_large))}
+    else:
+        w = {"T.0.w_t1": rng.normal(size=(hidden, d_large)), "T.0.w_t2": rng.normal(size=(d_small, hidden))}
+    return O.TandemProjection(w, 1, kind), w
+
+
+def test_ff_tandem_mlp_matches_a_library_two_layer_module():
+    """Eq. 2, first line, with the two-layer FF_Tandem: Linear -> GELU -> Linear without biases, built
+    separately from torch modules.  Non-square widths so that a transposed matrix cannot pass."""
+    proj, w = _projection(synth.FF_TANDEM_MLP, d_large=24, d_small=10, hidden=17, seed=5)
+    lin1 = torch.nn.Linear(24, 17, bias=False, dtype=torch.float64)
+    lin2 = torch.nn.Linear(17, 10, bias=False, dtype=torch.float64)
+    with torch.no_grad():
+        lin1.weight.copy_(torch.tensor(w["T.0.w_t1"]))
+        lin2.weight.copy_(torch.tensor(w["T.0.w_t2"]))
+    module = torch.nn.Sequential(lin1, torch.nn.GELU(), lin2)
+    x = np.random.default_rng(6).normal(size=(9, 24)) * 2
+    with torch.no_grad():
+        want = module(torch.tensor(x)).numpy()
+    assert np.allclose(proj(0, x), want, atol=1e-12)
+    assert np.allclose(proj(0, x[3]), want[3], atol=1e-12)      # a single row, as the cached path calls it
+
+
+def test_ff_tandem_mlp_hand_cases():
+    """First map = identity: the projection is GELU(x) W_T2^T, so dropping the GELU, applying it after the
+    second map, or swapping the two matrices all give something else.  Closed-form values at x = 1 and x = 0."""
+    d = 6
+    rng = np.random.default_rng(7)
+    w2 = rng.normal(size=(4, d))
+    proj = O.TandemProjection({"T.0.w_t1": np.eye(d), "T.0.w_t2": w2}, 1, synth.FF_TANDEM_MLP)
+    x = rng.normal(size=(5, d)) * 2
+    phi = 0.5 * (1 + np.vectorize(math.erf)(x / math.sqrt(2)))
+    want = (x * phi) @ w2.T
+    assert np.allclose(proj(0, x), want, atol=1e-13)
+    assert not np.allclose(proj(0, x), x @ w2.T, atol=1e-3)                   # GELU dropped
+    assert np.allclose(proj(0, np.zeros(d)), 0.0)
+    ones = proj(0, np.ones(d))
+    assert np.allclose(ones, 0.8413447460685429 * w2.sum(axis=1), atol=1e-13)     # Phi(1) * row sums
+    # second map = identity instead: GELU applies to the first map's output, not to x
+    w1 = rng.normal(size=(d, d))
+    proj2 = O.TandemProjection({"T.0.w_t1": w1, "T.0.w_t2": np.eye(d)}, 1, synth.FF_TANDEM_MLP)
+    h = x @ w1.T
+    assert np.allclose(proj2(0, x), h * 0.5 * (1 + np.vectorize(math.erf)(h / math.sqrt(2))), atol=1e-13)
+
+
+def test_ff_tandem_linear_is_one_matrix_product():
+    proj, w = _projection(synth.FF_TANDEM_LINEAR, d_large=24, d_small=10, hidden=0, seed=8)
+    x = np.random.default_rng(9).normal(size=(4, 24))
+    want = torch.nn.functional.linear(torch.tensor(x), torch.tensor(w["T.0.w_t"])).numpy()
+    assert np.allclose(proj(0, x), want, atol=1e-13)
