@@ -125,20 +125,6 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def device_weights(shape, seed, device):
-    """Random-init weights drawn on the device (timing only; no CPU checker run uses them)."""
-    import torch
-    g = torch.Generator(device=device).manual_seed(seed)
-    out = {}
-    for name in synth.weight_names(shape):
-        shp = synth.weight_shape(shape, name)
-        if synth.is_norm_param(name):
-            out[name] = torch.full(shp, 1.0 if name.endswith("_g") else 0.0, dtype=torch.float32, device=device)
-        else:
-            out[name] = (torch.randn(shp, generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
-    return out
-
-
 def algorithmic_bytes_per_iteration(shape, B, gamma, T):
     """Weights of the large model once, of the small model gamma times, FF_Tandem and the small key/value maps
     once, plus both KV streams at context length T (bf16)."""
@@ -323,7 +309,7 @@ def main():
     cfgname, B, P, gamma, new, max_pos = WORKLOADS[args.workload]
     shape = synth.named_config(cfgname, max_pos)
     if args.workload in DEVICE_INIT:
-        weights = device_weights(shape, 0, torch.device("cuda", local_rank))
+        weights = synth.device_weights(shape, 0, torch.device("cuda", local_rank))
         args.no_cpu_baseline = True
     else:
         weights = synth.make_weights(shape, seed=0)

@@ -22,6 +22,12 @@
  *  - A context is bound to one device and one stream and is not thread-safe.  All GPU work is enqueued
  *    on that stream.
  *  - Greedy decisions: arg-max over fp32 logits, lowest token id on ties.
+ *  - bf16 contexts: weights, queries and both KV caches are bf16; everything else between the kernels of a
+ *    decode pass (residual stream, normalised rows, attention and GELU outputs) is fp32, and enters each
+ *    tensor-core product as the sum of two bf16 numbers.  The prompt pass keeps bf16 activations.
+ *  - Two environment variables are read once by tandem_create, for diagnosis only; neither changes a result:
+ *    TANDEM_NO_GRAPH (set to anything) launches every kernel of an iteration eagerly instead of replaying a CUDA
+ *    graph; TANDEM_NO_PDL orders the kernels by plain stream order instead of programmatic dependent launch.
  */
 #ifndef TANDEM_B200_H
 #define TANDEM_B200_H
@@ -117,7 +123,8 @@ TANDEM_API tandem_status tandem_query_arena(const tandem_config* cfg, size_t* by
 
 /* Builds a context over caller-owned weights and arena (DEVICE, 256-byte aligned, arena_bytes >= the
  * queried size).  Supported shapes: d_model % n_heads == 0; head size 32, 64 or 128; d_model, d_ff and
- * ff_tandem_hidden multiples of 8; max_batch * (gamma_max + 1) <= 256.  Zero-fills the arena's state. */
+ * ff_tandem_hidden multiples of 8; max_batch * (gamma_max + 1) <= 256 (up to 64 block rows every weight is
+ * read once per pass; beyond that once per group of 64 rows).  Zero-fills the arena's state. */
 TANDEM_API tandem_status tandem_create(const tandem_config* cfg, const tandem_weights* weights,
                             void* arena /* DEVICE */, size_t arena_bytes, tandem_ctx** out /* HOST out */);
 
@@ -175,6 +182,14 @@ TANDEM_API tandem_status tandem_large_greedy_generate(tandem_ctx* ctx, int32_t m
  * bytes must equal the size of the selected item. */
 TANDEM_API tandem_status tandem_debug_read(tandem_ctx* ctx, int32_t what, int32_t layer, int32_t seq,
                                 void* host_dst, size_t bytes);
+
+/* Test hook for the give-up path of the bounded device-side waits (bf16 contexts).  Enqueues one thread block of
+ * the decode GEMM whose weight loads are withheld and whose waits give up after 1024 polls instead of 2^22: its
+ * wait for operands runs out, it records the code in the context's error word, frees its tensor memory and
+ * returns like any other kernel (nothing faults, nothing is left in flight).  The next tandem_block_step with a
+ * result, or the next generate call, then returns TANDEM_ERR_TIMEOUT, leaves the caller's buffers untouched and
+ * clears the word; the context stays usable.  The model's state is not touched. */
+TANDEM_API tandem_status tandem_debug_expire_wait(tandem_ctx* ctx);
 
 /* Measurement hooks.  tandem_profile_enable(ctx, n > 0) brackets each of the next n kernel launches with a
  * pair of CUDA events on the context's stream (this slows the stream down: never leave it on while timing
@@ -244,10 +259,11 @@ TANDEM_API tandem_status tandem_decode_attention_static(const void* q, const voi
  *   x [rows][d_large] bf16;  w_t [d_small][d_large] bf16;  ln_g, ln_b [d_small] fp32;
  *   wk, wv [d_small][d_small] bf16;  k_out, v_out [rows][d_small] bf16;
  *   scratch: at least tandem_ff_tandem_project_scratch_bytes(rows, d_small) bytes (the fp32 projection
- *   and, above 64 rows, its normalised bf16 copy).  rows <= 256; d_large, d_small multiples of 8.
- * Up to 64 rows the two GEMMs stream their weights once on the tensor cores with the LayerNorm fused into
- * the second one's operand load and the key/value write as its epilogue; above that they are tiled GEMMs
- * with a LayerNorm kernel in between. */
+ *   and its normalised fp32 copy).  rows <= 256; d_large, d_small multiples of 8.
+ * The two GEMMs stream their weights on the tensor cores (once up to 64 rows, else once per group of 64 rows)
+ * with the key/value write as the second one's epilogue; the LayerNorm is fused into the second one's operand
+ * load for up to 8 rows of up to 1024 elements and runs as a kernel of its own otherwise.  Asynchronous; a
+ * bounded device-side wait that ran out is reported by tandem_standalone_check. */
 TANDEM_API size_t tandem_ff_tandem_project_scratch_bytes(int32_t rows, int32_t d_small);
 TANDEM_API tandem_status tandem_ff_tandem_project(const void* x, const void* w_t, const void* ln_g, const void* ln_b,
                                        const void* wk, const void* wv, void* k_out, void* v_out,
@@ -259,9 +275,14 @@ TANDEM_API tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
  * gamma+1 tokens of a block together so that each weight is read once for all of them).  All pointers DEVICE,
  * 16-byte aligned, bf16:  x [rows][in_features];  w [out_features][in_features];  y [rows][out_features].
  * 1 <= rows <= 64; in_features a multiple of 8.  Needs no work space: the K-slices of an output tile are summed
- * through the shared memory of a thread-block cluster. */
+ * through the shared memory of a thread-block cluster.  Asynchronous; see tandem_standalone_check. */
 TANDEM_API tandem_status tandem_block_linear(const void* x, const void* w, void* y, int32_t rows, int32_t in_features,
                                              int32_t out_features, void* stream);
+
+/* Waits for `stream` and reports whether a bounded device-side wait ran out in a tandem_ff_tandem_project or
+ * tandem_block_linear call on the current device since the last check: TANDEM_ERR_TIMEOUT (the outputs of those
+ * calls are then not valid; the record is cleared), else TANDEM_OK. */
+TANDEM_API tandem_status tandem_standalone_check(void* stream);
 
 TANDEM_API const char* tandem_status_string(tandem_status s);
 /* Name of the last failing CUDA call's error for this thread (valid after TANDEM_ERR_CUDA). */

@@ -28,7 +28,8 @@ EXPORTS = ["tandem_query_arena", "tandem_create", "tandem_destroy", "tandem_pref
            "tandem_decode_attention_scratch_bytes", "tandem_decode_attention", "tandem_ff_tandem_project",
            "tandem_ff_tandem_project_scratch_bytes", "tandem_block_linear",
            "tandem_status_string", "tandem_last_cuda_error", "tandem_profile_enable", "tandem_profile_read",
-           "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static"]
+           "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static",
+           "tandem_debug_expire_wait", "tandem_standalone_check"]
 
 
 class TandemError(RuntimeError):
@@ -96,6 +97,8 @@ def load_library():
     lib.tandem_ff_tandem_project_scratch_bytes.argtypes = [i32] * 2
     lib.tandem_ff_tandem_project_scratch_bytes.restype = sz
     lib.tandem_decode_attention_static.argtypes = [vp] * 6 + [i32] * 5 + [vp]
+    lib.tandem_debug_expire_wait.argtypes = [vp]
+    lib.tandem_standalone_check.argtypes = [vp]
     lib.tandem_profile_enable.argtypes = [vp, i32]
     lib.tandem_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(C.c_int64), C.POINTER(C.c_double)]
     lib.tandem_profile_class_name.argtypes = [i32]
@@ -234,6 +237,9 @@ class Tandem:
                "tandem_large_greedy_generate")
         return out, lens, self._stats(st, 0)
 
+    def tandem_debug_expire_wait(self) -> None:
+        _check(self.lib.tandem_debug_expire_wait(self.ctx), "tandem_debug_expire_wait")
+
     def tandem_launch_count(self) -> int:
         return int(self.lib.tandem_launch_count(self.ctx))
 
@@ -338,3 +344,12 @@ def tandem_block_linear(x, w, y=None):
                                    C.c_void_p(torch.cuda.current_stream(x.device).cuda_stream or None)),
            "tandem_block_linear")
     return y
+
+
+def tandem_standalone_check(device=None) -> None:
+    """Waits for the current stream; raises TandemError(TIMEOUT) if a bounded device-side wait ran out in a
+    stand-alone GEMM call since the last check."""
+    import torch
+    lib = load_library()
+    _check(lib.tandem_standalone_check(C.c_void_p(torch.cuda.current_stream(device).cuda_stream or None)),
+           "tandem_standalone_check")

@@ -29,7 +29,8 @@ struct AttnArgs {
     const void* kcache; const void* vcache;   // [seq][head][t_max][DH]
     const void* k2; const void* v2;            // optional second segment [seq][head][t_max2][DH] holding
     int split, t_max2;                         //   positions >= split (used when k2 != nullptr)
-    void* out; int ldo;                  // T [M][ldo]
+    void* out; int ldo;                  // T [M][ldo]; float when out_f32 is set (attn_decode_kernel only)
+    int out_f32;
     const int* row_seq; const int* row_pos;
     const int* grp_row0; const int* grp_cnt;   // nullable: then group g = rows g*nq .. g*nq+nq-1
     int nq;
@@ -57,10 +58,8 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
     constexpr int QPT = (ATT_NQ + QS - 1) / QS; // queries per thread in the value phase
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_last;
-    TC_PROBE_INIT(LOOP ? 201 : 200);
     pdl_wait();                // queries and keys/values come from earlier kernels
     pdl_launch_dependents();   // the next kernel may start fetching its weights
-    if (threadIdx.x == 0) TC_PROBE(1);
     T* ks = reinterpret_cast<T*>(smem_raw);
     T* vs = ks + ATT_CH * LD;
     float* qs = reinterpret_cast<float*>(vs + ATT_CH * LD);
@@ -116,7 +115,6 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
         cp_async_commit();
         cp_async_wait_all();
         __syncthreads();
-        if (threadIdx.x == 0) TC_PROBE(2);
 
         // scores: thread t owns key t0+t for every query
         for (int t = tid; t < nt; t += ATT_THREADS) {
@@ -141,7 +139,6 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
         }
         __syncthreads();
 
-        if (threadIdx.x == 0) TC_PROBE(3);
         // per query: chunk max, exponentials, chunk sum
         for (int qi = warp; qi < cnt; qi += ATT_THREADS / 32) {
             float m = -INFINITY;
@@ -160,7 +157,6 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
         }
         __syncthreads();
 
-        if (threadIdx.x == 0) TC_PROBE(4);
         // weighted values: thread owns element e for queries qsub, qsub+QS, ...
 #pragma unroll
         for (int i = 0; i < QPT; ++i) {
@@ -191,10 +187,8 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
         }
     } else {
         // The CTA that finishes last for this (group, head) merges every query's chunks in position order.
-        if (threadIdx.x == 0) TC_PROBE(5);
         __threadfence();
         __syncthreads();
-        if (threadIdx.x == 0) TC_PROBE(6);
         if (tid == 0) {
             const int active = min((int)gridDim.x, pos_last / ATT_CH + 1);   // CTAs that got this far
             int* counter = a.merge_counters + (size_t)g * a.n_heads + h;
@@ -203,7 +197,6 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
             if (t == active - 1) *counter = 0;   // ready for the next launch
         }
         __syncthreads();
-        if (threadIdx.x == 0) TC_PROBE(7);
         if (!s_last) return;
         __threadfence();
 #pragma unroll
@@ -226,7 +219,6 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
             }
             og[(size_t)(row0 + qi) * a.ldo + h * DH + e] = from_float<T>(o / l);
         }
-        if (threadIdx.x == 0) TC_PROBE(8);
     }
 }
 
@@ -307,12 +299,12 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     bf16* ring_all = reinterpret_cast<bf16*>(smem_raw);
     float* wst = reinterpret_cast<float*>(smem_raw);                                            // [NW][16][SW], after the main loop
     float* inbox = reinterpret_cast<float*>(ring_all + (size_t)NW * C::STAGES * C::STAGE_ELEMS);   // [CL][QPC][SW]
-    TC_PROBE_INIT(210);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = blockIdx.x, h = blockIdx.y, g = blockIdx.z;
     const int CL = gridDim.x;                      // cluster size
     const int QPC = (ATT_NQ + CL - 1) / CL;        // queries a CTA finishes at most
+    if (CL > 1) cluster_arrive_relaxed();          // opening handshake: waited for just before the first remote store
     bf16* ring = ring_all + (size_t)warp * C::STAGES * C::STAGE_ELEMS;
     const uint32_t ring_s = smem_u32(ring);
     // The row arrays were written at the start of the pass, at least two kernels back in the stream, so they may be
@@ -386,7 +378,6 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     }
     pdl_wait();   // queries and the newest keys/values come from the kernel before this one
     pdl_launch_dependents();
-    if (tid == 0) TC_PROBE(1);
 #pragma unroll
     for (int it = 0; it < C::STAGES - 1; ++it) {
         if (it >= pre) {
@@ -422,14 +413,12 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     const int lm_sw = DH >= 64 ? lm_r : (lm_r >> 1);
     const uint32_t k_row = (uint32_t)(lm_r * DH * 2);                           // K: key = 8 * nt + row, unit = 4 * kp + matrix
     const uint32_t v_row = (uint32_t)((((lm_m & 1) << 3) + lm_r) * DH * 2);     // V: key = 8 * (matrix & 1) + row, unit = 2 * np + matrix / 2
-    if (tid == 0) TC_PROBE(2);
 
     for (int it = 0; it < n_mine; ++it) {
         if (it + C::STAGES - 1 < n_mine) issue(it + C::STAGES - 1);
         cp_async_commit();
         asm volatile("cp.async.wait_group %0;" ::"n"(C::STAGES - 1) : "memory");
         __syncwarp();
-        if (tid == 0 && it == 0) TC_PROBE(3);
         const int t0 = (rank + it * CL) * ATT_CH + warp * ATD_WROWS;
         const uint32_t ks_s = ring_s + (uint32_t)((it % C::STAGES) * C::STAGE_ELEMS * 2);
         const uint32_t vs_s = ks_s + (uint32_t)(C::TILE_ELEMS * 2);
@@ -513,7 +502,6 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
             }
         }
         __syncwarp();   // the stage may be refilled by this warp's next issue
-        if (tid == 0 && it == 0) TC_PROBE(8);
     }
     // a row's sum: add the quad's lanes
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
@@ -537,8 +525,8 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
         }
     }
     __syncthreads();
-    if (tid == 0) TC_PROBE(4);
     // fold the warps' states in warp order and send the CTA's state of query qa to CTA qa % CL
+    if (CL > 1) cluster_wait();   // closes the opening handshake: every CTA of the cluster is running
     for (int i = tid; i < cnt * SW; i += ATD_THREADS) {
         const int qa = i / SW, e = i - qa * SW;
         float mx = -INFINITY;
@@ -561,7 +549,6 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
         else *slot = val;
     }
     if (CL > 1) cluster_sync_all(); else __syncthreads();
-    if (tid == 0) TC_PROBE(5);
     for (int u = 0; u < QPC; ++u) {
         const int qi = rank + u * CL;
         if (qi < cnt && tid < DH) {
@@ -574,10 +561,11 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
                 l = fmaf(st[DH + 1], f, l);
                 ov = fmaf(st[tid], f, ov);
             }
-            static_cast<bf16*>(a.out)[(size_t)(row0 + qi) * a.ldo + h * DH + tid] = __float2bfloat16_rn(ov / l);
+            const size_t oi = (size_t)(row0 + qi) * a.ldo + h * DH + tid;
+            if (a.out_f32) static_cast<float*>(a.out)[oi] = ov / l;
+            else static_cast<bf16*>(a.out)[oi] = __float2bfloat16_rn(ov / l);
         }
     }
-    if (tid == 0) TC_PROBE(6);
 }
 
 }  // namespace tandem

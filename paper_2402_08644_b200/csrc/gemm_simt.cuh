@@ -6,8 +6,7 @@
 //                      number of rows, so a block pass and a one-row pass give identical bits.
 //  gemm_tiled_kernel   prompt path (many rows), classic shared-memory tiling.
 //
-// Both are the exact-arithmetic (fp32 FMA) paths: they serve the fp32 test mode and are the fall-back
-// shapes of the bf16 mode.
+// Both are the exact-arithmetic (fp32 FMA) paths of the fp32 test mode.
 #pragma once
 #include "common.cuh"
 
@@ -16,7 +15,7 @@ namespace tandem {
 enum { EPI_STORE = 0, EPI_STORE_F32 = 1, EPI_GELU = 2, EPI_RESID = 3, EPI_QKV = 4, EPI_KV = 5 };
 
 struct EpiArgs {
-    void* out;            // EPI_STORE/GELU: T [M][ldo];  STORE_F32/RESID: float [M][ldo];  QKV: q as T [M][ldo]
+    void* out;            // EPI_STORE/GELU: T [M][ldo] (GELU on the tensor-core decode path: float);  STORE_F32/RESID: float [M][ldo];  QKV: q as T [M][ldo]
     int ldo;
     void* kcache;         // QKV / KV: this layer's keys   [B][H][t_max][d_head] (T)
     void* vcache;         //           this layer's values
@@ -24,7 +23,7 @@ struct EpiArgs {
     const int* row_pos;   // [M] absolute position of each row
     int n_heads, d_head, t_max;
     int seg;              // columns per segment (= d_model) for QKV / KV
-    void* snap;           // EPI_RESID on the tensor-core decode path: optional bf16 copy of the new values [M][snap_ld]
+    void* snap;           // EPI_RESID on the tensor-core decode path: optional fp32 copy of the new values [M][snap_ld]
     int snap_ld;
 };
 

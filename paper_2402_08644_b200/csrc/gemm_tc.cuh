@@ -8,7 +8,12 @@
 //                          sums to the CTA that finishes those token rows (remote shared-memory stores), which
 //                          adds them in slice order.
 //                          The token rows are written into the B stages by the CTA's own threads, which is
-//                          where the LayerNorm (or the fp32 -> bf16 cast) of the residual stream is fused.
+//                          where the LayerNorm of the residual stream is fused.  Activations arrive in fp32 and
+//                          enter the product as the sum of two bf16 numbers (the rounded value and the rounded
+//                          remainder, about 16 significant bits): the B tile holds the NB value rows followed
+//                          by the NB remainder rows, one MMA of N = 2 NB covers both (the weight tile is read
+//                          from shared memory once), and the epilogue adds the two accumulator columns of a
+//                          token row.  The kernel streams weights, so the wider B operand costs no bandwidth.
 //                          The weight loads are issued before the kernel waits for its predecessor in the
 //                          stream (programmatic dependent launch), so they overlap its run; a kernel lets its
 //                          own successor start once the predecessor is done, which keeps one kernel's worth of
@@ -25,12 +30,14 @@
 
 namespace tandem {
 
-enum { PRO_BF16 = 0, PRO_LN = 1, PRO_CAST = 2 };   // how the token rows become the bf16 B operand
+// How the token rows become the B operand: PRO_BF16: bf16 rows as they are (remainder rows zero); PRO_LN: fp32 rows,
+// LayerNorm, then value + remainder; PRO_F32: fp32 rows as value + remainder.
+enum { PRO_BF16 = 0, PRO_LN = 1, PRO_F32 = 2 };
 constexpr int EPI_ARGMAX = 6;                       // fp32 store plus the (max, index) of each row within the tile
 enum { TC_ERR_SLOT = 1, TC_ERR_OPERANDS = 2, TC_ERR_ACCUM = 3 };   // which bounded wait gave up
 
 struct TcDecodeArgs {
-    const void* x;          // PRO_BF16: bf16 [rows][ldx];  PRO_LN / PRO_CAST: float [rows][ldx]
+    const void* x;          // PRO_BF16: bf16 [rows][ldx];  PRO_LN / PRO_F32: float [rows][ldx]
     int ldx;
     const float* ln_g;      // PRO_LN: LayerNorm gain / bias [K]
     const float* ln_b;
@@ -40,6 +47,9 @@ struct TcDecodeArgs {
     int splits;             // K-slices per tile: 1, 2, 4 or 8 = the cluster size; grid = tiles * splits
     int stream_weights;     // 1: weights are read once per pass and should not stay in L2
     int* err_flag;          // nullable
+    unsigned poll_limit;    // polls before a wait on an mbarrier gives up; 0 = MBAR_POLL_LIMIT
+    int withhold_weights;   // test hook for the give-up path: the TMA thread issues no loads, so the wait for
+                            // operands must run out (nothing is in flight when the kernel leaves)
     float* amax_val;        // EPI_ARGMAX: [rows][amax_stride] best value per tile
     int* amax_idx;          //             and its output feature
     int amax_stride;
@@ -48,14 +58,23 @@ struct TcDecodeArgs {
 
 constexpr int TCD_THREADS = 192;   // warps 0-3: B operand + epilogue; warp 4: TMA; warp 5: TMEM + MMA issue
 template <int NB> struct TcdCfg {
-    static constexpr int STAGES = NB <= 16 ? 5 : (NB <= 32 ? 4 : 3);   // two CTAs fit on an SM
+    static constexpr int NB2 = 2 * NB;              // B-operand rows = accumulator columns: values, then remainders
+    static constexpr int STAGES = NB <= 16 ? 5 : (NB <= 32 ? 4 : 3);   // two CTAs fit on an SM up to NB = 48
     static constexpr int A_BYTES = 128 * 128;       // 128 weight rows x 64 bf16
-    static constexpr int B_BYTES = NB * 128;        // NB token rows x 64 bf16
+    static constexpr int B_BYTES = NB2 * 128;       // 2 NB rows x 64 bf16
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int INBOX_BYTES = NB * 128 * 4;   // the K-slices' partial sums for the token rows this CTA finishes
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + INBOX_BYTES + 1024;   // + slack to align the ring to 1024
-    static constexpr int TMEM_COLS = NB <= 32 ? 32 : 64;
+    static constexpr int TMEM_COLS = NB2 <= 32 ? 32 : (NB2 <= 64 ? 64 : 128);
 };
+
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): the pair carries x to about 16 significant bits.
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __low2float(h), x1 - __high2float(h));
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+}
 
 __device__ __forceinline__ void tc_report(int* err_flag, int code) {
     if (err_flag) atomicExch(err_flag, code);
@@ -105,6 +124,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     unsigned char* ring = smem_dyn + (ring0 - smem_u32(smem_dyn));         // the same place as a generic pointer
 
     const int S = a.splits;
+    const uint32_t poll_limit = a.poll_limit ? a.poll_limit : MBAR_POLL_LIMIT;
     const int unit = blockIdx.x;
     const int tile = unit / S, sp = unit - tile * S;                       // sp = this CTA's rank in its cluster
     const int seg = tile / a.tiles_per_seg;
@@ -122,7 +142,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     const int j_first = S == 1 ? 0 : sp * rpc;
     const int j_count = max(0, min(rpc, a.rows - j_first));
     float hres[EPI == EPI_RESID ? NB : 1];   // EPI_RESID: the residual values this thread's outputs are added to
-    TC_PROBE_INIT(100 + PRO * 10 + EPI);
 
     if (warp == 5) {
         if (lane == 0) {
@@ -141,17 +160,17 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = s_tmem;
-    if (tid == 0) TC_PROBE(1);
+    if (S > 1) cluster_arrive_relaxed();   // opening handshake: waited for just before the first remote store
 
     if (warp == 4) {
         // ---- weight tiles: independent of every earlier kernel, so no wait on the predecessor here ----
-        if (lane == 0) {
+        if (lane == 0 && !a.withhold_weights) {
             const CUtensorMap* tm = seg == 0 ? &tm0 : (seg == 1 ? &tm1 : &tm2);
             tma_prefetch_desc(tm);
             const uint64_t pol = l2_policy_evict_first();
             for (int i = 0; i < nkb; ++i) {
                 const int st = i % C::STAGES;
-                if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
+                if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1, poll_limit)) {
                     tc_report(a.err_flag, TC_ERR_SLOT);
                     break;
                 }
@@ -160,21 +179,19 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 if (a.stream_weights) tma_load_2d(ring0 + st * C::STAGE_BYTES, tm, (kb0 + i) * 64, n_local0, bar, pol);
                 else tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES, tm, (kb0 + i) * 64, n_local0, bar);
             }
-            TC_PROBE(2);
         }
         __syncwarp();
     } else if (warp == 5) {
         // ---- MMA issue: one thread ----
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(128, NB);
+            constexpr uint32_t idesc = umma_idesc_bf16(128, C::NB2);
             for (int i = 0; i < nkb; ++i) {
                 const int st = i % C::STAGES;
-                if (!mbar_wait(smem_u32(&s_full[st]), (i / C::STAGES) & 1)) {
+                if (!mbar_wait(smem_u32(&s_full[st]), (i / C::STAGES) & 1, poll_limit)) {
                     tc_report(a.err_flag, TC_ERR_OPERANDS);
                     break;
                 }
                 tc_fence_after_sync();
-                if (i == 0) TC_PROBE(3);
                 const uint64_t da = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES);
                 const uint64_t db = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES + C::A_BYTES);
 #pragma unroll
@@ -183,7 +200,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 umma_commit(smem_u32(&s_empty[st]));
             }
             umma_commit(smem_u32(&s_accum));
-            TC_PROBE(4);
         }
         __syncwarp();
     } else {
@@ -200,7 +216,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     }
     pdl_wait();   // x, and everything the epilogue touches, comes from earlier kernels; gains and biases are parameters
     pdl_launch_dependents();   // only now: one successor at a time sets up and fetches weights behind this kernel
-    if (tid == 0) TC_PROBE(5);
     if (EPI == EPI_QKV || EPI == EPI_KV) {
         // cache index of (row j, head h, element el) = ((seq_j * H + h) * t_max + pos_j) * d_head + el: the row part once per row
         if (tid < a.rows)
@@ -229,7 +244,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
             for (int u = 0; u < 8; ++u) s += (t[u].x + t[u].y) + (t[u].z + t[u].w);
             const float mu = warp_sum(s) / (float)a.K;
-            if (tid == 0) TC_PROBE(13);
             float q = 0.f;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -239,7 +253,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 }
             }
             const float rs = 1.0f / sqrtf(warp_sum(q) / (float)a.K + 1e-5f);
-            if (tid == 0) TC_PROBE(14);
 #pragma unroll
             for (int i = 0; i < C::STAGES; ++i) {
                 const int kb = kb0 + i;
@@ -249,24 +262,24 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                     float4 xv = t[0];
 #pragma unroll
                     for (int uu = 1; uu < 8; ++uu) if (u == uu) xv = t[uu];
-                    uint2 val = make_uint2(0u, 0u);   // beyond K the weights are zero-filled; so is x
+                    uint2 val = make_uint2(0u, 0u), rem = make_uint2(0u, 0u);   // beyond K the weights are zero-filled; so is x
                     if (u * 32 + lane < K4) {
                         const float4 y = ln_apply(xv, mu, rs, gq[i], bq[i]);
-                        val.x = pack_bf16x2(y.x, y.y); val.y = pack_bf16x2(y.z, y.w);
+                        split_bf16x2(y.x, y.y, val.x, rem.x);
+                        split_bf16x2(y.z, y.w, val.y, rem.y);
                     }
                     const int c = (lane & 15) >> 1;
-                    unsigned char* bt = ring + i * C::STAGE_BYTES + C::A_BYTES;
-                    *reinterpret_cast<uint2*>(bt + r * 128 + ((c ^ (r & 7)) << 4) + ((lane & 1) << 3)) = val;
+                    unsigned char* bt = ring + i * C::STAGE_BYTES + C::A_BYTES + r * 128 + ((c ^ (r & 7)) << 4) + ((lane & 1) << 3);
+                    *reinterpret_cast<uint2*>(bt) = val;
+                    *reinterpret_cast<uint2*>(bt + NB * 128) = rem;   // NB is a multiple of 8: the same swizzle phase
                 }
             }
         }
         // rows >= a.rows of the B tiles stay as they are: a column of the product depends on its own row only
-        if (tid == 0) TC_PROBE(15);
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0)
             for (int i = 0; i < nkb; ++i) mbar_arrive(smem_u32(&s_full[i]));
-        if (tid == 0) TC_PROBE(6);
     } else {
         // general case: statistics (LayerNorm), then the K-blocks a ring's worth at a time
         if (PRO == PRO_LN) {
@@ -308,29 +321,34 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             }
             bar_sync(1, 128);
         }
-        constexpr int CPT = NB * 8 / 128;   // 16-byte chunks of one B tile per thread
+        constexpr int CPT = NB * 8 / 128;   // 8-element chunks of the NB token rows of one K-block per thread
         for (int i0 = 0; i0 < nkb; i0 += C::STAGES) {
             // a ring's worth of K-blocks at a time: all loads first, so their latencies overlap
             uint4 raw[PRO == PRO_BF16 ? C::STAGES : 1][CPT];
-            if (PRO == PRO_BF16) {
+            float4 raw32[PRO == PRO_BF16 ? 1 : C::STAGES][CPT][2];
 #pragma unroll
-                for (int g = 0; g < C::STAGES; ++g)
+            for (int g = 0; g < C::STAGES; ++g)
 #pragma unroll
-                    for (int ch = 0; ch < CPT; ++ch) {
-                        const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
-                        const int k = (kb0 + i0 + g) * 64 + c * 8;
-                        raw[g][ch] = (i0 + g < nkb && r < a.rows && k < a.K)
-                                         ? __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k))
-                                         : make_uint4(0u, 0u, 0u, 0u);
+                for (int ch = 0; ch < CPT; ++ch) {
+                    const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
+                    const int k = (kb0 + i0 + g) * 64 + c * 8;
+                    const bool live = i0 + g < nkb && r < a.rows && k < a.K;
+                    if (PRO == PRO_BF16) {
+                        raw[g][ch] = live ? __ldcg(reinterpret_cast<const uint4*>(static_cast<const bf16*>(a.x) + (size_t)r * a.ldx + k))
+                                          : make_uint4(0u, 0u, 0u, 0u);
+                    } else {
+                        const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
+                        raw32[g][ch][0] = live ? __ldcg(xp) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        raw32[g][ch][1] = live ? __ldcg(xp + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
-            }
+                }
             bool dead = false;
 #pragma unroll
             for (int g = 0; g < C::STAGES; ++g) {
                 const int i = i0 + g;
                 if (i >= nkb || dead) break;
                 const int st = g;   // i0 is a multiple of STAGES
-                if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
+                if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1, poll_limit)) {
                     tc_report(a.err_flag, TC_ERR_SLOT);
                     dead = true;
                     break;
@@ -339,32 +357,32 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
                 for (int ch = 0; ch < CPT; ++ch) {
                     const int idx = tid + ch * 128, r = idx >> 3, c = idx & 7;
-                    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                    uint4 val = make_uint4(0u, 0u, 0u, 0u), rem = make_uint4(0u, 0u, 0u, 0u);
                     if (PRO == PRO_BF16) {
                         val = raw[g][ch];
                     } else {
                         const int k = (kb0 + i) * 64 + c * 8;
                         if (r < a.rows && k < a.K) {
-                            const float4* xp = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx + k);
-                            float4 u0 = __ldcg(xp), u1 = __ldcg(xp + 1);
+                            float4 u0 = raw32[g][ch][0], u1 = raw32[g][ch][1];
                             if (PRO == PRO_LN) {
                                 const float mu = s_mu[r], rs = s_rstd[r];
                                 u0 = ln_apply(u0, mu, rs, __ldg(reinterpret_cast<const float4*>(a.ln_g + k)), __ldg(reinterpret_cast<const float4*>(a.ln_b + k)));
                                 u1 = ln_apply(u1, mu, rs, __ldg(reinterpret_cast<const float4*>(a.ln_g + k) + 1), __ldg(reinterpret_cast<const float4*>(a.ln_b + k) + 1));
                             }
-                            val.x = pack_bf16x2(u0.x, u0.y); val.y = pack_bf16x2(u0.z, u0.w);
-                            val.z = pack_bf16x2(u1.x, u1.y); val.w = pack_bf16x2(u1.z, u1.w);
+                            split_bf16x2(u0.x, u0.y, val.x, rem.x); split_bf16x2(u0.z, u0.w, val.y, rem.y);
+                            split_bf16x2(u1.x, u1.y, val.z, rem.z); split_bf16x2(u1.z, u1.w, val.w, rem.w);
                         }
                     }
                     // 128-byte swizzle: the 16-byte chunk index is XORed with the row index modulo 8
-                    *reinterpret_cast<uint4*>(bt + r * 128 + ((c ^ (r & 7)) << 4)) = val;
+                    unsigned char* dst = bt + r * 128 + ((c ^ (r & 7)) << 4);
+                    *reinterpret_cast<uint4*>(dst) = val;
+                    *reinterpret_cast<uint4*>(dst + NB * 128) = rem;   // the remainder row of token row r (same swizzle phase)
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s_full[st]));
             }
         }
-        if (tid == 0) TC_PROBE(6);
     }
     }
 
@@ -372,17 +390,17 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     float v[NB];
     const int tl = warp * 32 + lane;
     if (warp < 4) {
-        if (!mbar_wait(smem_u32(&s_accum), 0)) tc_report(a.err_flag, TC_ERR_ACCUM);
+        if (!mbar_wait(smem_u32(&s_accum), 0, poll_limit)) tc_report(a.err_flag, TC_ERR_ACCUM);
         tc_fence_after_sync();
-        if (tid == 0) TC_PROBE(7);
 #pragma unroll
         for (int c0 = 0; c0 < NB; c0 += 16) {
-            float t[16];
-            tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c0, t);
+            if (c0 >= a.rows) break;                  // columns of absent token rows are never read
+            float t[16], u[16];
+            tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c0, t);        // x's values times W
+            tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + NB + c0, u);   // x's remainders times W
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[c0 + i] = t[i];
+            for (int i = 0; i < 16; ++i) v[c0 + i] = t[i] + u[i];
         }
-        if (tid == 0) TC_PROBE(8);
     }
     const int n_local = n_local0 + tl;                 // warps 0-3: this thread's output feature
     const bool valid = n_local < a.seg_rows;
@@ -423,6 +441,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             // stores), one cluster barrier makes them visible, and each CTA sums its inbox in slice order.  Nobody
             // touches a peer's shared memory after the barrier, so CTAs may leave as they finish.
             const uint32_t inbox0 = ring0 + C::STAGES * C::STAGE_BYTES;           // [S][rpc][128] fp32
+            cluster_wait();   // closes the opening handshake: every CTA of the cluster is running
             if (warp < 4) {
                 int dst = 0, jj = 0;
 #pragma unroll
@@ -433,7 +452,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 }
             }
             cluster_sync_all();
-            if (tid == 0) TC_PROBE(9);
             if (warp < 4) {
                 const float* inbox = reinterpret_cast<const float*>(ring + C::STAGES * C::STAGE_BYTES);
 #pragma unroll
@@ -460,7 +478,9 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                     if (valid) {
                         if (EPI == EPI_RESID || EPI == EPI_STORE_F32) {
                             static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = hv;
-                            if (EPI == EPI_RESID && a.e.snap) static_cast<bf16*>(a.e.snap)[(size_t)j * a.e.snap_ld + n] = __float2bfloat16_rn(hv);
+                            if (EPI == EPI_RESID && a.e.snap) static_cast<float*>(a.e.snap)[(size_t)j * a.e.snap_ld + n] = hv;
+                        } else if (EPI == EPI_GELU) {   // activations between the decode kernels stay fp32
+                            static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = gelu_bf16_out(hv);
                         } else if (EPI == EPI_QKV || EPI == EPI_KV) {
                             sc.base[(sc.is_q ? (long long)j * a.e.ldo : s_rowoff[j]) + sc.col] = __float2bfloat16_rn(hv);
                         } else {
@@ -470,13 +490,10 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 }
             }
         }
-        if (tid == 0) TC_PROBE(10);
     }
-    if (tid == 0) TC_PROBE(11);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 5) tmem_dealloc(tmem, C::TMEM_COLS);
-    if (tid == 0) TC_PROBE(12);
 }
 
 // ---------------------------------------------------------------------------------------------------

@@ -83,12 +83,10 @@ template <typename T>
 __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, int nq, int fin_r, const float* amax_val,
                                                          const int* amax_idx, int amax_stride, int n_tiles, int* row_tok,
                                                          int* row_seq, int* row_pos, const T* __restrict__ emb,
-                                                         const T* __restrict__ pos, float* __restrict__ h, int d, bf16* snap) {
+                                                         const T* __restrict__ pos, float* __restrict__ h, int d, float* snap) {
     __shared__ int s_tok, s_pos;
-    TC_PROBE_INIT(300);
     pdl_wait();
     pdl_launch_dependents();
-    if (threadIdx.x == 0) TC_PROBE(1);
     const int m = blockIdx.x;
     const int b = m / nq, r = r0 + (m - b * nq);
     if (threadIdx.x < 32) {
@@ -109,9 +107,8 @@ __global__ void __launch_bounds__(128) step_begin_kernel(LoopState st, int r0, i
     for (int i = threadIdx.x; i < d; i += 128) {
         const float v = to_float(er[i]) + to_float(pr[i]);
         h[(size_t)m * d + i] = v;
-        if (snap) snap[(size_t)m * d + i] = __float2bfloat16_rn(v);   // bf16 copy for the FF_Tandem projection of x^(0)
+        if (snap) snap[(size_t)m * d + i] = v;   // copy for the FF_Tandem projection of x^(0)
     }
-    if (threadIdx.x == 0) TC_PROBE(2);
 }
 
 __device__ __forceinline__ float block_sum_128(float v, float* red) {
@@ -138,14 +135,25 @@ __global__ void __launch_bounds__(128) layernorm_kernel(const float* __restrict_
         out[(size_t)blockIdx.x * d + i] = from_float<T>((xr[i] - mu) * rstd * gain[i] + bias[i]);
 }
 
-// Decode-path LayerNorm of fp32 rows to bf16 for the tensor-core GEMMs: the row sits in registers between the
-// passes (up to 4096 elements), loads and stores are 16 / 8 bytes wide.  grid: rows; block: 128; d % 4 == 0.
-__global__ void __launch_bounds__(128) layernorm_rows_bf16_kernel(const float* __restrict__ x, const float* __restrict__ gain,
-                                                                  const float* __restrict__ bias, bf16* __restrict__ out, int d) {
+// Four normalised values to the output row: fp32 as they are, bf16 rounded.
+__device__ __forceinline__ void ln_store4(float* orow, int k4, float y0, float y1, float y2, float y3) {
+    reinterpret_cast<float4*>(orow)[k4] = make_float4(y0, y1, y2, y3);
+}
+__device__ __forceinline__ void ln_store4(bf16* orow, int k4, float y0, float y1, float y2, float y3) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(y0, y1), hi = __floats2bfloat162_rn(y2, y3);
+    reinterpret_cast<uint2*>(orow)[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+}
+
+// Decode-path LayerNorm of fp32 rows ahead of the tensor-core GEMMs (fp32 out; bf16 out for the stand-alone
+// projection above 64 rows): the row sits in registers between the passes (up to 4096 elements), loads and stores
+// are 16 bytes wide.  grid: rows; block: 128; d % 4 == 0.
+template <typename TO>
+__global__ void __launch_bounds__(128) layernorm_rows_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+                                                             const float* __restrict__ bias, TO* __restrict__ out, int d) {
     __shared__ float red[4];
     const int d4 = d >> 2;
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)blockIdx.x * d);
-    uint2* orow = reinterpret_cast<uint2*>(out + (size_t)blockIdx.x * d);
+    TO* orow = out + (size_t)blockIdx.x * d;
     if (d4 <= 8 * 128) {
         // gains and biases are parameters: fetched while the kernel that writes x is still running
         float4 gq[8], bq[8];
@@ -178,9 +186,8 @@ __global__ void __launch_bounds__(128) layernorm_rows_bf16_kernel(const float* _
             const int k4 = threadIdx.x + 128 * u;
             if (k4 < d4) {
                 const float4 g = gq[u], b = bq[u];
-                const __nv_bfloat162 lo = __floats2bfloat162_rn((t[u].x - mu) * rs * g.x + b.x, (t[u].y - mu) * rs * g.y + b.y);
-                const __nv_bfloat162 hi = __floats2bfloat162_rn((t[u].z - mu) * rs * g.z + b.z, (t[u].w - mu) * rs * g.w + b.w);
-                orow[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+                ln_store4(orow, k4, (t[u].x - mu) * rs * g.x + b.x, (t[u].y - mu) * rs * g.y + b.y,
+                          (t[u].z - mu) * rs * g.z + b.z, (t[u].w - mu) * rs * g.w + b.w);
             }
         }
     } else {
@@ -199,22 +206,9 @@ __global__ void __launch_bounds__(128) layernorm_rows_bf16_kernel(const float* _
         for (int k4 = threadIdx.x; k4 < d4; k4 += 128) {
             const float4 t = __ldcg(xr + k4);
             const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + k4), b = __ldg(reinterpret_cast<const float4*>(bias) + k4);
-            const __nv_bfloat162 lo = __floats2bfloat162_rn((t.x - mu) * rs * g.x + b.x, (t.y - mu) * rs * g.y + b.y);
-            const __nv_bfloat162 hi = __floats2bfloat162_rn((t.z - mu) * rs * g.z + b.z, (t.w - mu) * rs * g.w + b.w);
-            orow[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+            ln_store4(orow, k4, (t.x - mu) * rs * g.x + b.x, (t.y - mu) * rs * g.y + b.y, (t.z - mu) * rs * g.z + b.z,
+                      (t.w - mu) * rs * g.w + b.w);
         }
-    }
-}
-
-// fp32 rows to bf16, 4 elements per thread; n % 4 == 0.  Decode path (waits for its predecessor in the stream).
-__global__ void cast_rows_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ out, size_t n4) {
-    pdl_wait();
-    pdl_launch_dependents();
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n4) {
-        const float4 t = __ldcg(reinterpret_cast<const float4*>(x) + i);
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(t.x, t.y), hi = __floats2bfloat162_rn(t.z, t.w);
-        reinterpret_cast<uint2*>(out)[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
     }
 }
 
@@ -261,10 +255,8 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restric
 __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed,
                                                      int max_new, const float* amax_val, const int* amax_idx, int amax_stride,
                                                      int n_tiles) {
-    TC_PROBE_INIT(400);
     pdl_wait();
     pdl_launch_dependents();
-    if (threadIdx.x == 0) TC_PROBE(1);
     if (amax_val != nullptr) {
         const int rows = batch * (gamma + 1);
         for (int m = threadIdx.x >> 5; m < rows; m += 8) {
@@ -315,7 +307,6 @@ __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, in
         st.host_flags[4] = st.counters[5];
         __threadfence_system();
         st.host_flags[0] = ticket;
-        TC_PROBE(2);
     }
 }
 

@@ -7,6 +7,7 @@
 #include <time.h>
 
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -41,8 +42,6 @@ thread_local char g_cuda_err[256] = "";
 
 size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 int cdiv(int a, int b) { return (a + b - 1) / b; }
-// Columns of the tensor-core decode GEMM's B operand for a number of token rows (0: too many rows for it).
-int tc_nb(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 48 ? 48 : rows <= 64 ? 64 : 0; }
 
 struct Layout {   // byte offsets into the arena
     size_t kv_large, kv_small;
@@ -51,6 +50,7 @@ struct Layout {   // byte offsets into the arena
     size_t attn_counters;   // inside the zero-filled state block
     size_t h_large, h_small, a, q, o, f, xb, t1, yhat, a_s, logits_large, logits_small, part_ml, part_acc, dbg;
     size_t amax_val_large, amax_idx_large, amax_val_small, amax_idx_small;
+    size_t a32, o32, f32;                           // fp32 activations between the bf16 decode kernels: LayerNorm / attention / GELU outputs
     size_t proj_snap, proj_yhat, proj_a, proj_t1;   // per small layer: the decode projection's own buffers (it runs beside the large pass)
     size_t total;
     int max_rows, dec_rows, max_groups, n_chunks_max, vocab_tiles;
@@ -97,7 +97,7 @@ struct tandem_ctx {
     size_t pinned_ints;
     int64_t launches = 0;
     int last_gamma = 0;
-    LoopState st;
+    LoopState st{};
     // CUDA graphs of one iteration, keyed by everything baked into the captured launches
     struct GraphEntry {
         int kind, gamma, mode, max_new, batch, chunks;
@@ -115,14 +115,13 @@ struct tandem_ctx {
     // tensor-core path (bf16 only)
     bool tc = false;                     // weights have tensor maps; GEMMs run on tcgen05
     bool use_pdl = true;                 // programmatic dependent launch between the decode kernels
-    int tc_target = 148;                 // CTAs a split-K decode GEMM aims for
+    int n_sms = 0;                       // multiprocessors of the context's device: split-K decode GEMMs aim for about one CTA each
     std::vector<CUtensorMap> wmap;       // one per weight pointer (matrices only), box 128 rows x 64 columns
     std::vector<char> wmap_ok;
     std::vector<CUtensorMap> kmap, vmap; // the large model's key / value cache of each layer as [(seq, head, position)][d_head]
     cudaStream_t side = nullptr;         // the decode-time FF_Tandem projections run here, beside the large model's later layers
     std::vector<cudaEvent_t> ev_fork;    // one per small layer
     cudaEvent_t ev_join = nullptr;
-    bool fork_projection = true;
     bool next_launch_plain = false;      // the next launch follows a cross-stream wait: no programmatic dependency on a kernel
     bool setup_failed = false;           // a launch helper could not encode a tensor map: reported by the enclosing call
     bool tc_prompt_attn = false;         // prompt attention on the tensor cores (head size 64 or 128)
@@ -217,10 +216,11 @@ Layout make_layout(const tandem_config& c) {
     L.amax_val_large = take(RD * L.vocab_tiles * 4); L.amax_idx_large = take(RD * L.vocab_tiles * 4);
     L.amax_val_small = take(B * L.vocab_tiles * 4); L.amax_idx_small = take(B * L.vocab_tiles * 4);
     const size_t nS = c.small.n_layers;
-    L.proj_snap = take(nS * RD * c.large.d_model * 2);
+    L.a32 = take(RD * dmax * 4); L.o32 = take(RD * dmax * 4); L.f32 = take(RD * fmax * 4);
+    L.proj_snap = take(nS * RD * c.large.d_model * 4);
     L.proj_yhat = take(nS * RD * c.small.d_model * 4);
-    L.proj_a = take(nS * RD * c.small.d_model * 2);
-    L.proj_t1 = take(nS * RD * hidden * 2);
+    L.proj_a = take(nS * RD * c.small.d_model * 4);
+    L.proj_t1 = take(nS * RD * hidden * 4);
     L.total = off;
     return L;
 }
@@ -259,15 +259,32 @@ int cur_dev() {   // opt-in shared-memory sizes are per device
 // launch helpers
 // ---------------------------------------------------------------------------------------------------
 
+// Opt-in dynamic shared memory of a kernel, requested once per device (`done`: one bit per device, one word per
+// kernel instantiation).  The attribute call is idempotent, so two threads racing to be first is harmless.
+template <typename K>
+void ensure_dyn_smem(K kernel, size_t bytes, std::atomic<unsigned long long>& done) {
+    const unsigned long long bit = 1ull << cur_dev();
+    if (done.load(std::memory_order_acquire) & bit) return;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    done.fetch_or(bit, std::memory_order_release);
+}
+
+// Multiprocessors of the current device (asked once per device).
+int sm_count() {
+    static std::atomic<int> cache[MAX_DEVICES];
+    const int dev = cur_dev();
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 1;
+    cache[dev].store(n, std::memory_order_relaxed);
+    return n;
+}
+
 template <typename T, int MT, int EPI>
 void launch_smallm(tandem_ctx& c, const T* x, int ldx, int M, int K, const WSegs& ws, int N, const EpiArgs& e) {
-    static bool attr_set[MAX_DEVICES] = {};
+    static std::atomic<unsigned long long> attr_done{0};
     const size_t smem = (size_t)MT * GS_KC * sizeof(T);
-    const int dev = cur_dev();
-    if (!attr_set[dev]) {
-        cudaFuncSetAttribute(gemm_smallm_kernel<T, MT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_set[dev] = true;
-    }
+    ensure_dyn_smem(gemm_smallm_kernel<T, MT, EPI>, smem, attr_done);
     dim3 grid(cdiv(N, GS_WARPS * GS_COLS), cdiv(M, MT));
     ProfScope ps(c, PC_GEMM_SMALLM, ((double)N * K + (double)M * K + (double)M * N) * sizeof(T));
     gemm_smallm_kernel<T, MT, EPI><<<grid, GS_THREADS, smem, c.stream>>>(x, ldx, M, K, ws, N, e);
@@ -310,7 +327,11 @@ struct TcW {              // up to three weight matrices stacked along the outpu
     CUtensorMap tm[3];
     int n_segs, seg_rows, K;
 };
-struct TcScratch { int* err; };
+struct TcScratch {
+    int* err;                  // where a bounded wait that ran out records its code (nullable)
+    unsigned poll_limit = 0;   // 0: the kernels' default
+    int withhold_weights = 0;  // test hook, see TcDecodeArgs
+};
 
 TcW tcw(const tandem_ctx& c, int i0, int i1, int i2, int seg_rows, int K) {
     TcW w;
@@ -324,7 +345,7 @@ TcW tcw(const tandem_ctx& c, int i0, int i1, int i2, int seg_rows, int K) {
 
 TcScratch tc_scratch(tandem_ctx& c) {
     TcScratch s;
-    s.err = c.st.counters + 2;
+    s.err = c.st.counters ? c.st.counters + 2 : nullptr;
     return s;
 }
 
@@ -356,16 +377,13 @@ void launch_ex(tandem_ctx& c, bool pdl, int cluster, void (*kernel)(KArgs...), d
 template <int NB, int PRO, int EPI>
 void launch_tc_decode_nb(tandem_ctx& c, const TcDecodeArgs& a, const TcW& w, int units) {
     using C = TcdCfg<NB>;
-    static bool attr_set[MAX_DEVICES] = {};
-    const int dev = cur_dev();
-    if (!attr_set[dev]) {
-        cudaFuncSetAttribute(gemm_tc_decode_kernel<NB, PRO, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-        attr_set[dev] = true;
-    }
+    static std::atomic<unsigned long long> attr_done{0};
+    ensure_dyn_smem(gemm_tc_decode_kernel<NB, PRO, EPI>, C::SMEM_BYTES, attr_done);
     launch_ex(c, true, a.splits, gemm_tc_decode_kernel<NB, PRO, EPI>, dim3(units), dim3(TCD_THREADS), (size_t)C::SMEM_BYTES, a, w.tm[0], w.tm[1], w.tm[2]);
 }
 
-// y = prologue(x) W^T for rows <= 64 on the tensor cores, streaming W once.
+// y = prologue(x) W^T for few rows on the tensor cores, streaming W once per group of up to 64 rows (one group in
+// every benchmark configuration; more rows than that re-read the weights per group, with unchanged arithmetic).
 template <int PRO, int EPI>
 void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx, const void* ln_g, const void* ln_b, int rows,
                       const TcW& w, bool stream_weights, const EpiArgs& e, float* amax_val = nullptr, int* amax_idx = nullptr,
@@ -373,38 +391,47 @@ void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx
     if (rows <= 0) return;
     TcDecodeArgs a;
     memset(&a, 0, sizeof(a));
-    a.x = x; a.ldx = ldx; a.ln_g = static_cast<const float*>(ln_g); a.ln_b = static_cast<const float*>(ln_b);
-    a.rows = rows; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
+    a.ldx = ldx; a.ln_g = static_cast<const float*>(ln_g); a.ln_b = static_cast<const float*>(ln_b);
+    a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
     const int tiles = w.n_segs * a.tiles_per_seg, KB = cdiv(w.K, 64);
-    // K-slices per tile = cluster size: the smallest power of two that puts tiles * S CTAs at or above the target
-    // (about one per SM), at most 8 and at most one per 64-element K-block.  The head GEMM keeps whole tiles.
+    // K-slices per tile = cluster size: the smallest power of two that puts tiles * S CTAs at or above one per
+    // multiprocessor, at most 8 and at most one per 64-element K-block.  The head GEMM keeps whole tiles.
     int S = 1;
     if (EPI != EPI_ARGMAX)
-        while (S < 8 && 2 * S <= KB && tiles * S < c.tc_target) S *= 2;
+        while (S < 8 && 2 * S <= KB && tiles * S < c.n_sms) S *= 2;
     a.splits = S;
     a.stream_weights = stream_weights ? 1 : 0;
     a.err_flag = sc.err;
-    a.amax_val = amax_val; a.amax_idx = amax_idx; a.amax_stride = amax_stride;
-    a.e = e;
+    a.poll_limit = sc.poll_limit;
+    a.withhold_weights = sc.withhold_weights;
+    a.amax_stride = amax_stride;
     const size_t xsz = PRO == PRO_BF16 ? 2 : 4;
-    ProfScope ps(c, PC_GEMM_TC_DECODE, 2.0 * a.N * w.K + (double)rows * w.K * xsz + (double)rows * a.N * (EPI == EPI_STORE_F32 || EPI == EPI_ARGMAX || EPI == EPI_RESID ? 4.0 : 2.0));
+    const size_t osz = EPI == EPI_STORE ? 2 : 4;       // EPI_QKV: the query buffer is bf16 too (below)
     const int units = tiles * S;
-    if (rows <= 16) launch_tc_decode_nb<16, PRO, EPI>(c, a, w, units);
-    else if (rows <= 32) launch_tc_decode_nb<32, PRO, EPI>(c, a, w, units);
-    else if (rows <= 48) launch_tc_decode_nb<48, PRO, EPI>(c, a, w, units);
-    else launch_tc_decode_nb<64, PRO, EPI>(c, a, w, units);
+    for (int r0 = 0; r0 < rows; r0 += 64) {
+        const int nr = std::min(64, rows - r0);
+        a.rows = nr;
+        a.x = static_cast<const unsigned char*>(x) + (size_t)r0 * ldx * xsz;
+        a.amax_val = amax_val ? amax_val + (size_t)r0 * amax_stride : nullptr;
+        a.amax_idx = amax_idx ? amax_idx + (size_t)r0 * amax_stride : nullptr;
+        a.e = e;
+        if (e.out) a.e.out = static_cast<unsigned char*>(e.out) + (size_t)r0 * e.ldo * (EPI == EPI_QKV ? 2 : osz);
+        if (e.row_seq) { a.e.row_seq = e.row_seq + r0; a.e.row_pos = e.row_pos + r0; }
+        if (e.snap) a.e.snap = static_cast<float*>(e.snap) + (size_t)r0 * e.snap_ld;
+        ProfScope ps(c, PC_GEMM_TC_DECODE, 2.0 * a.N * w.K + (double)nr * w.K * xsz + (double)nr * a.N * (EPI == EPI_QKV || EPI == EPI_KV || EPI == EPI_STORE ? 2.0 : 4.0));
+        if (nr <= 16) launch_tc_decode_nb<16, PRO, EPI>(c, a, w, units);
+        else if (nr <= 32) launch_tc_decode_nb<32, PRO, EPI>(c, a, w, units);
+        else if (nr <= 48) launch_tc_decode_nb<48, PRO, EPI>(c, a, w, units);
+        else launch_tc_decode_nb<64, PRO, EPI>(c, a, w, units);
+    }
 }
 
 // y = x W^T for many rows on the tensor cores; x bf16 [M][ldx].
 template <int EPI, int BN>
 void launch_tc_tiled_bn(tandem_ctx& c, TcTiledArgs& a, const CUtensorMap& tmx, const TcW& w, int M) {
     using C = TctCfg<BN>;
-    static bool attr_set[MAX_DEVICES] = {};
-    const int dev = cur_dev();
-    if (!attr_set[dev]) {
-        cudaFuncSetAttribute(gemm_tc_tiled_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-        attr_set[dev] = true;
-    }
+    static std::atomic<unsigned long long> attr_done{0};
+    ensure_dyn_smem(gemm_tc_tiled_kernel<EPI, BN>, C::SMEM_BYTES, attr_done);
     a.tiles_per_seg = cdiv(w.seg_rows, BN);
     launch_ex(c, false, 1, gemm_tc_tiled_kernel<EPI, BN>, dim3(w.n_segs * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)C::SMEM_BYTES,
               a, tmx, w.tm[0], w.tm[1], w.tm[2]);
@@ -424,7 +451,7 @@ tandem_status launch_tc_tiled(tandem_ctx& c, const bf16* x, int ldx, int M, cons
     a.err_flag = err; a.e = e;
     ProfScope ps(c, PC_GEMM_TC_TILED, 2.0 * M * (double)a.N * w.K);   // flops
     // 256-wide tiles when they still give every SM a tile, else square ones
-    if ((long long)w.n_segs * cdiv(w.seg_rows, 256) * cdiv(M, 128) >= 148) launch_tc_tiled_bn<EPI, 256>(c, a, tmx, w, M);
+    if ((long long)w.n_segs * cdiv(w.seg_rows, 256) * cdiv(M, 128) >= c.n_sms) launch_tc_tiled_bn<EPI, 256>(c, a, tmx, w, M);
     else launch_tc_tiled_bn<EPI, 128>(c, a, tmx, w, M);
     return TANDEM_OK;
 }
@@ -463,16 +490,10 @@ void launch_gemm(tandem_ctx& c, bool decode, const T* x, int ldx, int M, const L
 }
 
 template <typename T, int DH>
-void set_attn_attrs() {
-    cudaFuncSetAttribute(attn_kernel<T, DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<T, DH>());
-    cudaFuncSetAttribute(attn_kernel<T, DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<T, DH>());
-}
-
-template <typename T, int DH>
 void launch_attn_dh(tandem_ctx& c, const AttnArgs& a, int groups, bool loop, int n_chunks, double kv_bytes) {
-    static bool attr_set[MAX_DEVICES] = {};
-    const int dev = cur_dev();
-    if (!attr_set[dev]) { set_attn_attrs<T, DH>(); attr_set[dev] = true; }
+    static std::atomic<unsigned long long> attr_done_split{0}, attr_done_loop{0};
+    ensure_dyn_smem(attn_kernel<T, DH, false>, attn_smem_bytes<T, DH>(), attr_done_split);
+    ensure_dyn_smem(attn_kernel<T, DH, true>, attn_smem_bytes<T, DH>(), attr_done_loop);
     if (loop) {
         ProfScope ps(c, PC_ATTN_PROMPT, kv_bytes);
         launch_ex(c, false, 1, attn_kernel<T, DH, true>, dim3(1, a.n_heads, groups), dim3(ATT_THREADS), attn_smem_bytes<T, DH>(), a);
@@ -492,26 +513,22 @@ void launch_attn(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, bool 
 // bf16 decode attention: one cluster of `cl` CTAs per (sequence, head); no scratch.
 template <int DH>
 void launch_attn_decode_dq(tandem_ctx& c, const AttnArgs& a, int groups, int cl, double kv_bytes) {
-    static bool attr_set[MAX_DEVICES] = {};
-    const int dev = cur_dev();
-    if (!attr_set[dev]) {
-        cudaFuncSetAttribute(attn_decode_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_decode_smem_bytes<DH>());
-        attr_set[dev] = true;
-    }
+    static std::atomic<unsigned long long> attr_done{0};
+    ensure_dyn_smem(attn_decode_kernel<DH>, attn_decode_smem_bytes<DH>(), attr_done);
     ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
     launch_ex(c, true, cl, attn_decode_kernel<DH>, dim3(cl, a.n_heads, groups), dim3(ATD_THREADS), attn_decode_smem_bytes<DH>(), a);
 }
 // Cluster size: the largest of 1, 2, 4, 8 that keeps the launch within one wave of resident CTAs (two per SM,
 // one for 128-wide heads).  It depends on the number of sequences and heads only, so every pass of a run
 // (block or one-row) cuts the context the same way.
-int attn_cluster_size(int groups, int n_heads, int d_head) {
-    const long long slots = 148LL * (d_head == 128 ? 1 : 2);
+int attn_cluster_size(int n_sms, int groups, int n_heads, int d_head) {
+    const long long slots = (long long)n_sms * (d_head == 128 ? 1 : 2);
     int cl = 1;
     while (cl < ATD_CLUSTER && (long long)groups * n_heads * cl * 2 <= slots) cl *= 2;
     return cl;
 }
 void launch_attn_decode(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, double kv_bytes) {
-    const int cl = attn_cluster_size(groups, a.n_heads, d_head);
+    const int cl = attn_cluster_size(c.n_sms, groups, a.n_heads, d_head);
     if (d_head == 32) launch_attn_decode_dq<32>(c, a, groups, cl, kv_bytes);
     else if (d_head == 64) launch_attn_decode_dq<64>(c, a, groups, cl, kv_bytes);
     else launch_attn_decode_dq<128>(c, a, groups, cl, kv_bytes);
@@ -556,12 +573,8 @@ EpiArgs epi_cache(tandem_ctx& c, const Model& m, int layer, void* q_out) {
 // Prompt attention of the large model's layer l on the tensor cores; groups of up to 128 queries.
 template <int DH>
 void launch_attn_prompt_tc_dh(tandem_ctx& c, const AttnTcArgs& a, const CUtensorMap& tmq, int l, int groups) {
-    static bool attr_set[MAX_DEVICES] = {};
-    const int dev = cur_dev();
-    if (!attr_set[dev]) {
-        cudaFuncSetAttribute(attn_prefill_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtcCfg<DH>::SMEM_BYTES);
-        attr_set[dev] = true;
-    }
+    static std::atomic<unsigned long long> attr_done{0};
+    ensure_dyn_smem(attn_prefill_tc_kernel<DH>, AtcCfg<DH>::SMEM_BYTES, attr_done);
     launch_ex(c, false, 1, attn_prefill_tc_kernel<DH>, dim3(a.n_heads, groups), dim3(ATC_THREADS), (size_t)AtcCfg<DH>::SMEM_BYTES, a, tmq,
               c.kmap[l], c.vmap[l]);
 }
@@ -599,8 +612,17 @@ void attention(tandem_ctx& c, const Model& m, int l, const T* q, T* o, const Row
         launch_attn_prompt_tc(c, l, reinterpret_cast<const bf16*>(q), reinterpret_cast<bf16*>(o), r);
         return;
     }
-    if (r.decode && sizeof(T) == 2 && r.groups <= 65535) launch_attn_decode(c, dh, aa, r.groups, r.kv_positions * 2.0 * d * sizeof(T));
-    else launch_attn<T>(c, dh, aa, r.groups, !r.decode, r.n_chunks, r.kv_positions * 2.0 * d * sizeof(T));
+    launch_attn<T>(c, dh, aa, r.groups, !r.decode, r.n_chunks, r.kv_positions * 2.0 * d * sizeof(T));
+}
+
+// bf16 decode / block attention over the cache of layer l: bf16 queries, fp32 output rows.
+void attention_decode(tandem_ctx& c, const Model& m, int l, const bf16* q, float* o, const Rows& r) {
+    const int d = m.d.d_model, H = m.d.n_heads, dh = d / H;
+    AttnArgs aa; memset(&aa, 0, sizeof(aa));
+    aa.q = q; aa.ldq = d; aa.kcache = kv_ptr<bf16>(c, m, l, 0); aa.vcache = kv_ptr<bf16>(c, m, l, 1);
+    aa.out = o; aa.ldo = d; aa.out_f32 = 1; aa.row_seq = at<int>(c, c.lay.row_seq); aa.row_pos = at<int>(c, c.lay.row_pos);
+    aa.nq = r.nq; aa.n_heads = H; aa.t_max = c.cfg.max_seq; aa.scale = 1.0f / sqrtf((float)dh);
+    launch_attn_decode(c, dh, aa, r.groups, r.kv_positions * 2.0 * d * 2.0);
 }
 
 // Eq. 2, first line, for small layer j, then that layer's LayerNorm and key/value maps: writes the
@@ -749,7 +771,7 @@ void greedy_iteration(tandem_ctx& c, int max_new) {
 
 // Row set-up + embedding for block rows r0 .. r0+nq-1 of every sequence; fin_r: block row whose token is the
 // arg-max the small model's last head GEMM left as per-tile results (-1: none).
-void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r, bf16* snap = nullptr) {
+void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r, float* snap = nullptr) {
     ProfScope ps(c, PC_ROWS, (double)c.batch * nq * m.d.d_model * 8.0);
     launch_ex(c, true, 1, step_begin_kernel<bf16>, dim3(c.batch * nq), dim3(128), 0, c.st, r0, nq, fin_r,
               (const float*)at<float>(c, c.lay.amax_val_small), (const int*)at<int>(c, c.lay.amax_idx_small), c.lay.vocab_tiles,
@@ -757,46 +779,48 @@ void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r
               (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model, snap);
 }
 
-// Whether LayerNorm (or the fp32 -> bf16 cast) is fused into the GEMM's operand load.  Fused, every CTA of the
-// GEMM normalises the rows it needs itself: right for a couple of sequences and short rows, wasteful beyond.
-// The choice depends on the batch and the model only, never on the number of rows, so a block pass and a
-// one-row pass take the same route.
+// Whether LayerNorm is fused into the GEMM's operand load.  Fused, every CTA of the GEMM normalises the rows it
+// needs itself: right for a couple of sequences and short rows, wasteful beyond.  The choice depends on the batch
+// and the model only, never on the number of rows, so a block pass and a one-row pass take the same route.
 bool tc_fused_prologue(const tandem_ctx& c, int K) { return c.batch <= 2 && K <= 1024; }
 
-// y = LayerNorm(h) W^T with the given epilogue; h fp32 [rows][K].
+// y = LayerNorm(h) W^T with the given epilogue; h fp32 [rows][K].  ln_out: where the normalised rows go when the
+// LayerNorm runs as its own kernel (default: the pass's activation buffer).
 template <int EPI>
 void tc_ln_gemm(tandem_ctx& c, const float* h, const void* ln_g, const void* ln_b, int rows, const TcW& w, bool stream_w,
-                const EpiArgs& e, float* amax_val = nullptr, int* amax_idx = nullptr, int amax_stride = 0, bf16* ln_out = nullptr) {
+                const EpiArgs& e, float* amax_val = nullptr, int* amax_idx = nullptr, int amax_stride = 0, float* ln_out = nullptr) {
     const TcScratch sc = tc_scratch(c);
     if (tc_fused_prologue(c, w.K)) {
         launch_tc_decode<PRO_LN, EPI>(c, sc, h, w.K, ln_g, ln_b, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
         return;
     }
-    bf16* a = ln_out ? ln_out : at<bf16>(c, c.lay.a);
+    float* a = ln_out ? ln_out : at<float>(c, c.lay.a32);
     {
-        ProfScope ps(c, PC_LAYERNORM, (double)rows * w.K * 6.0);
-        launch_ex(c, true, 1, layernorm_rows_bf16_kernel, dim3(rows), dim3(128), 0, h, static_cast<const float*>(ln_g),
+        ProfScope ps(c, PC_LAYERNORM, (double)rows * w.K * 8.0);
+        launch_ex(c, true, 1, layernorm_rows_kernel<float>, dim3(rows), dim3(128), 0, h, static_cast<const float*>(ln_g),
                   static_cast<const float*>(ln_b), a, w.K);
     }
-    launch_tc_decode<PRO_BF16, EPI>(c, sc, a, w.K, nullptr, nullptr, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
+    launch_tc_decode<PRO_F32, EPI>(c, sc, a, w.K, nullptr, nullptr, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
 }
 
-void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r, bool stream_w, bf16* snap = nullptr) {
+// One decoder layer of a decode pass.  Between the kernels the activations are fp32 (attention and GELU outputs,
+// normalised rows); only the queries and the cached keys / values are bf16.
+void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r, bool stream_w, float* snap = nullptr) {
     const int d = m.d.d_model, dff = m.d.d_ff;
     bf16* q = at<bf16>(c, c.lay.q);
-    bf16* o = at<bf16>(c, c.lay.o);
-    bf16* f = at<bf16>(c, c.lay.f);
+    float* o = at<float>(c, c.lay.o32);
+    float* f = at<float>(c, c.lay.f32);
     const TcScratch sc = tc_scratch(c);
     tc_ln_gemm<EPI_QKV>(c, h, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), r.M,
                         tcw(c, wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, d), stream_w, epi_cache<bf16>(c, m, l, q));
-    attention<bf16>(c, m, l, q, o, r);
-    launch_tc_decode<PRO_BF16, EPI_RESID>(c, sc, o, d, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_WO), -1, -1, d, d), stream_w,
-                                          epi_plain(h, d));
+    attention_decode(c, m, l, q, o, r);
+    launch_tc_decode<PRO_F32, EPI_RESID>(c, sc, o, d, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_WO), -1, -1, d, d), stream_w,
+                                         epi_plain(h, d));
     tc_ln_gemm<EPI_GELU>(c, h, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), r.M, tcw(c, wi_layer(m, l, W_W1), -1, -1, dff, d),
                          stream_w, epi_plain(f, dff));
     EpiArgs e2 = epi_plain(h, d);
-    e2.snap = snap; e2.snap_ld = d;   // bf16 copy of x^(l+1) when an FF_Tandem projection reads it
-    launch_tc_decode<PRO_BF16, EPI_RESID>(c, sc, f, dff, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_W2), -1, -1, d, dff), stream_w, e2);
+    e2.snap = snap; e2.snap_ld = d;   // copy of x^(l+1) when an FF_Tandem projection reads it
+    launch_tc_decode<PRO_F32, EPI_RESID>(c, sc, f, dff, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_W2), -1, -1, d, dff), stream_w, e2);
 }
 
 // Final LayerNorm + output head; leaves fp32 logits and the per-tile (max, index) pairs that the next kernel
@@ -804,42 +828,6 @@ void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows
 void tc_head(tandem_ctx& c, const Model& m, float* h, const Rows& r, float* logits, size_t amax_val_off, size_t amax_idx_off, bool stream_w) {
     tc_ln_gemm<EPI_ARGMAX>(c, h, w_tail(c, m, 0), w_tail(c, m, 1), r.M, tcw(c, wi_tail(m, 2), -1, -1, m.d.vocab, m.d.d_model), stream_w,
                            epi_plain(logits, m.d.vocab), at<float>(c, amax_val_off), at<int>(c, amax_idx_off), c.lay.vocab_tiles);
-}
-
-// FF_Tandem of the block's rows after n large layers (Eq. 2, first line) for every small layer fed from there,
-// then that layer's LayerNorm and key/value maps with the cache write as the GEMM epilogue.
-void tc_project_after(tandem_ctx& c, int n_large_layers_done, const Rows& r) {
-    const int dL = c.large.d.d_model, dS = c.small.d.d_model;
-    const TcScratch sc = tc_scratch(c);
-    float* h = at<float>(c, c.lay.h_large);
-    float* yhat = at<float>(c, c.lay.yhat);
-    bool any = false;
-    for (int j = 0; j < c.small.d.n_layers; ++j) any |= (c.layer_map[j] == n_large_layers_done);
-    if (!any) return;
-    const bool fused = tc_fused_prologue(c, dL);
-    bf16* xb = at<bf16>(c, c.lay.xb);
-    if (!fused) {   // one bf16 copy of the rows serves every small layer fed from here
-        const size_t n4 = (size_t)r.M * dL / 4;
-        ProfScope ps(c, PC_ROWS, (double)n4 * 24.0);
-        launch_ex(c, true, 1, cast_rows_bf16_kernel, dim3((unsigned)((n4 + 255) / 256)), dim3(256), 0, (const float*)h, xb, n4);
-    }
-    for (int j = 0; j < c.small.d.n_layers; ++j) {
-        if (c.layer_map[j] != n_large_layers_done) continue;
-        if (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR) {
-            const TcW w = tcw(c, wi_tandem(c, j, 0), -1, -1, dS, dL);
-            if (fused) launch_tc_decode<PRO_CAST, EPI_STORE_F32>(c, sc, h, dL, nullptr, nullptr, r.M, w, true, epi_plain(yhat, dS));
-            else launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, xb, dL, nullptr, nullptr, r.M, w, true, epi_plain(yhat, dS));
-        } else {
-            bf16* t1 = at<bf16>(c, c.lay.t1);
-            const TcW w = tcw(c, wi_tandem(c, j, 0), -1, -1, c.hidden, dL);
-            if (fused) launch_tc_decode<PRO_CAST, EPI_GELU>(c, sc, h, dL, nullptr, nullptr, r.M, w, true, epi_plain(t1, c.hidden));
-            else launch_tc_decode<PRO_BF16, EPI_GELU>(c, sc, xb, dL, nullptr, nullptr, r.M, w, true, epi_plain(t1, c.hidden));
-            launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, t1, c.hidden, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 1), -1, -1, dS, c.hidden),
-                                                      true, epi_plain(yhat, dS));
-        }
-        tc_ln_gemm<EPI_KV>(c, yhat, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), r.M,
-                           tcw(c, wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS), true, epi_cache<bf16>(c, c.small, j, nullptr));
-    }
 }
 
 void tc_small_step(tandem_ctx& c, int s) {
@@ -851,14 +839,16 @@ void tc_small_step(tandem_ctx& c, int s) {
     tc_head(c, c.small, y, r, logits, c.lay.amax_val_small, c.lay.amax_idx_small, false);
 }
 
-// The same projection on the side stream, from the bf16 copy `snap` of x^(l(j)) that the producing kernel left: it
-// depends on nothing the large model does afterwards (and nothing in the iteration depends on it before the next
-// draft), so it runs beside the large model's later layers instead of in their chain.
+// FF_Tandem of the block's rows after n large layers (Eq. 2, first line) for every small layer fed from there, then
+// that layer's LayerNorm and key/value maps with the cache write as the GEMM epilogue.  It runs on the side stream,
+// from the copy `snap` of x^(l(j)) that the producing kernel left: it depends on nothing the large model does
+// afterwards (and nothing in the iteration depends on it before the next draft), so it runs beside the large model's
+// later layers instead of in their chain.
 void tc_project_forked(tandem_ctx& c, int n_large_layers_done, int slot, const Rows& r) {
     const int dL = c.large.d.d_model, dS = c.small.d.d_model;
     const TcScratch sc = tc_scratch(c);
     const size_t RD = (size_t)c.lay.dec_rows;
-    const bf16* snap = at<bf16>(c, c.lay.proj_snap) + (size_t)slot * RD * dL;
+    const float* snap = at<float>(c, c.lay.proj_snap) + (size_t)slot * RD * dL;
     cudaStream_t main_stream = c.stream;
     cudaEventRecord(c.ev_fork[slot], main_stream);
     cudaStreamWaitEvent(c.side, c.ev_fork[slot], 0);
@@ -867,16 +857,16 @@ void tc_project_forked(tandem_ctx& c, int n_large_layers_done, int slot, const R
     for (int j = 0; j < c.small.d.n_layers; ++j) {
         if (c.layer_map[j] != n_large_layers_done) continue;
         float* yhat = at<float>(c, c.lay.proj_yhat) + (size_t)j * RD * dS;
-        bf16* a_j = at<bf16>(c, c.lay.proj_a) + (size_t)j * RD * dS;
+        float* a_j = at<float>(c, c.lay.proj_a) + (size_t)j * RD * dS;
         if (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR) {
-            launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, snap, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, dS, dL), true,
-                                                      epi_plain(yhat, dS));
+            launch_tc_decode<PRO_F32, EPI_STORE_F32>(c, sc, snap, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, dS, dL), true,
+                                                     epi_plain(yhat, dS));
         } else {
-            bf16* t1 = at<bf16>(c, c.lay.proj_t1) + (size_t)j * RD * c.hidden;
-            launch_tc_decode<PRO_BF16, EPI_GELU>(c, sc, snap, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, c.hidden, dL), true,
-                                                 epi_plain(t1, c.hidden));
-            launch_tc_decode<PRO_BF16, EPI_STORE_F32>(c, sc, t1, c.hidden, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 1), -1, -1, dS, c.hidden),
-                                                      true, epi_plain(yhat, dS));
+            float* t1 = at<float>(c, c.lay.proj_t1) + (size_t)j * RD * c.hidden;
+            launch_tc_decode<PRO_F32, EPI_GELU>(c, sc, snap, dL, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 0), -1, -1, c.hidden, dL), true,
+                                                epi_plain(t1, c.hidden));
+            launch_tc_decode<PRO_F32, EPI_STORE_F32>(c, sc, t1, c.hidden, nullptr, nullptr, r.M, tcw(c, wi_tandem(c, j, 1), -1, -1, dS, c.hidden),
+                                                     true, epi_plain(yhat, dS));
         }
         tc_ln_gemm<EPI_KV>(c, yhat, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), r.M,
                            tcw(c, wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS), true, epi_cache<bf16>(c, c.small, j, nullptr),
@@ -894,25 +884,18 @@ int project_slot(const tandem_ctx& c, int n) {
 
 void tc_large_block(tandem_ctx& c, int gamma, bool project) {
     float* h = at<float>(c, c.lay.h_large);
-    const bool forked = project && c.fork_projection;
     const size_t snap_elems = (size_t)c.lay.dec_rows * c.large.d.d_model;
-    auto snap_of = [&](int n) -> bf16* {
-        const int slot = forked ? project_slot(c, n) : -1;
-        return slot >= 0 ? at<bf16>(c, c.lay.proj_snap) + (size_t)slot * snap_elems : nullptr;
+    auto snap_of = [&](int n) -> float* {
+        const int slot = project ? project_slot(c, n) : -1;
+        return slot >= 0 ? at<float>(c, c.lay.proj_snap) + (size_t)slot * snap_elems : nullptr;
     };
     bool any_fork = false;
     tc_begin(c, c.large, h, 0, gamma + 1, gamma > 0 ? gamma : -1, snap_of(0));
     const Rows r = decode_rows(c, gamma, gamma + 1);
-    if (project) {
-        if (forked) { if (project_slot(c, 0) >= 0) { tc_project_forked(c, 0, project_slot(c, 0), r); any_fork = true; } }
-        else tc_project_after(c, 0, r);
-    }
+    if (project && project_slot(c, 0) >= 0) { tc_project_forked(c, 0, project_slot(c, 0), r); any_fork = true; }
     for (int l = 0; l < c.large.d.n_layers; ++l) {
         tc_decoder_layer(c, c.large, l, h, r, true, snap_of(l + 1));
-        if (project) {
-            if (forked) { if (project_slot(c, l + 1) >= 0) { tc_project_forked(c, l + 1, project_slot(c, l + 1), r); any_fork = true; } }
-            else tc_project_after(c, l + 1, r);
-        }
+        if (project && project_slot(c, l + 1) >= 0) { tc_project_forked(c, l + 1, project_slot(c, l + 1), r); any_fork = true; }
     }
     tc_head(c, c.large, h, r, at<float>(c, c.lay.logits_large), c.lay.amax_val_large, c.lay.amax_idx_large, true);
     if (any_fork) {   // the projections join the main stream before the verify kernel
@@ -946,13 +929,12 @@ tandem_status check_launch(tandem_ctx& c) {
 }
 
 void enqueue_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t seed, int max_new) {
-    const bool bf = c.cfg.dtype == TANDEM_DTYPE_BF16;
-    if (bf && c.tc && tc_nb(c.batch * (gamma + 1)) != 0) {
+    if (c.cfg.dtype == TANDEM_DTYPE_BF16) {   // one bf16 path: the tensor-core kernels (a bf16 context always has tensor maps)
         if (kind == 0) tc_iteration(c, gamma, mode, seed, max_new); else tc_greedy_iteration(c, max_new);
         return;
     }
-    if (kind == 0) { if (bf) iteration<bf16>(c, gamma, mode, seed, max_new); else iteration<float>(c, gamma, mode, seed, max_new); }
-    else { if (bf) greedy_iteration<bf16>(c, max_new); else greedy_iteration<float>(c, max_new); }
+    if (kind == 0) iteration<float>(c, gamma, mode, seed, max_new);
+    else greedy_iteration<float>(c, max_new);
 }
 
 // Enqueues one iteration on the context's stream: eagerly the first time a launch shape is seen (and whenever
@@ -960,7 +942,7 @@ void enqueue_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t se
 tandem_status launch_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t seed, int max_new) {
     const int need = (c.n_ub - 1 + gamma) / ATT_CH + 1;
     c.chunks_launch = std::min(c.lay.n_chunks_max, (need + 3) / 4 * 4);
-    if (c.cfg.dtype == TANDEM_DTYPE_BF16 && c.tc && tc_nb(c.batch * (gamma + 1)) != 0)
+    if (c.cfg.dtype == TANDEM_DTYPE_BF16)
         c.chunks_launch = 1;   // the cluster attention's grid does not depend on the context length: one graph serves all
     c.ticket++;
     if (c.prof.on || !c.use_graphs) {
@@ -1127,11 +1109,12 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
         e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
         if (e == cudaSuccess) c->ev_fork.push_back(ev);
     }
-    c->fork_projection = getenv("TANDEM_NO_FORK") == nullptr;
+    // Two diagnostic switches, read here once (see tandem.h): launch every kernel eagerly instead of replaying a
+    // graph, and plain stream order instead of programmatic dependent launch.  Neither changes any result.
     c->use_graphs = getenv("TANDEM_NO_GRAPH") == nullptr;
     c->use_pdl = getenv("TANDEM_NO_PDL") == nullptr;
-    if (const char* t = getenv("TANDEM_TC_TARGET")) c->tc_target = std::max(1, atoi(t));
-    if (e == cudaSuccess && cfg->dtype == TANDEM_DTYPE_BF16 && getenv("TANDEM_NO_TC") == nullptr) {
+    c->n_sms = sm_count();
+    if (e == cudaSuccess && cfg->dtype == TANDEM_DTYPE_BF16) {
         // one tensor map per weight matrix: [out_features][in_features], 128 x 64 tiles
         c->wmap.resize(c->w.size());
         c->wmap_ok.assign(c->w.size(), 0);
@@ -1163,7 +1146,7 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
         }
         c->tc = true;
         const int dhL = cfg->large.d_model / cfg->large.n_heads;
-        if ((dhL == 64 || dhL == 128) && getenv("TANDEM_NO_TC_ATTN") == nullptr) {
+        if (dhL == 64 || dhL == 128) {
             c->kmap.resize(cfg->large.n_layers);
             c->vmap.resize(cfg->large.n_layers);
             bool okm = true;
@@ -1298,11 +1281,12 @@ extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t
         int32_t* cnt = c->pinned;   // staging is idle outside prefill
         CK(cudaMemcpyAsync(cnt, c->st.counters, 5 * 4, cudaMemcpyDeviceToHost, c->stream));
         const int B = c->batch, GL = TANDEM_GAMMA_LIMIT;
-        std::vector<int32_t> d((size_t)B * GL), t((size_t)B * (GL + 1));
+        // everything lands in private buffers first: the caller's arrays are written only once the iteration is known to be good
+        std::vector<int32_t> d((size_t)B * GL), t((size_t)B * (GL + 1)), acc((size_t)B), ncm((size_t)B);
         if (result->drafts) CK(cudaMemcpyAsync(d.data(), c->st.drafts, d.size() * 4, cudaMemcpyDeviceToHost, c->stream));
         if (result->targets) CK(cudaMemcpyAsync(t.data(), c->st.targets, t.size() * 4, cudaMemcpyDeviceToHost, c->stream));
-        if (result->accept_len) CK(cudaMemcpyAsync(result->accept_len, c->st.accept_len, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
-        if (result->n_committed) CK(cudaMemcpyAsync(result->n_committed, c->st.n, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+        if (result->accept_len) CK(cudaMemcpyAsync(acc.data(), c->st.accept_len, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+        if (result->n_committed) CK(cudaMemcpyAsync(ncm.data(), c->st.n, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
         CK(cudaStreamSynchronize(c->stream));
         c->n_ub = cnt[3];
         c->n_sum = cnt[4];
@@ -1314,6 +1298,8 @@ extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t
         for (int b = 0; b < B; ++b) {
             if (result->drafts) for (int i = 0; i < gamma; ++i) result->drafts[b * gamma + i] = d[(size_t)b * GL + i];
             if (result->targets) for (int i = 0; i <= gamma; ++i) result->targets[b * (gamma + 1) + i] = t[(size_t)b * (GL + 1) + i];
+            if (result->accept_len) result->accept_len[b] = acc[b];
+            if (result->n_committed) result->n_committed[b] = ncm[b];
         }
     }
     return TANDEM_OK;
@@ -1453,6 +1439,24 @@ extern "C" tandem_status tandem_profile_read(tandem_ctx* c, int32_t n_classes, d
     return TANDEM_OK;
 }
 
+extern "C" tandem_status tandem_debug_expire_wait(tandem_ctx* c) {
+    TRY(begin_call(c));
+    if (c->cfg.dtype != TANDEM_DTYPE_BF16) return TANDEM_ERR_UNIMPLEMENTED;
+    // One CTA of the decode GEMM over the first 128 x 64 corner of the large model's first query matrix, with the
+    // weight loads withheld and a poll limit of 1024: the MMA thread's wait for operands runs out, the kernel
+    // records the code in the context's error word and leaves through its normal tear-down.  The (meaningless)
+    // product goes to the debug scratch area.
+    TcScratch sc = tc_scratch(*c);
+    sc.poll_limit = 1024;
+    sc.withhold_weights = 1;
+    const int d = c->large.d.d_model;
+    TcW w = tcw(*c, wi_layer(c->large, 0, W_WQ), -1, -1, std::min(128, d), 64);
+    c->next_launch_plain = true;
+    launch_tc_decode<PRO_F32, EPI_STORE_F32>(*c, sc, at<float>(*c, c->lay.h_large), d, nullptr, nullptr, 1, w, false,
+                                             epi_plain(at<float>(*c, c->lay.dbg), 128));
+    return check_launch(*c);
+}
+
 extern "C" tandem_status tandem_debug_read(tandem_ctx* c, int32_t what, int32_t layer, int32_t seq, void* host_dst, size_t bytes) {
     TRY(begin_call(c));
     if (!host_dst) return TANDEM_ERR_INVALID_ARG;
@@ -1545,9 +1549,10 @@ extern "C" tandem_status tandem_decode_attention(const void* q, const void* k_de
     a.split = derived_len; a.t_max = derived_len; a.t_max2 = own_len;
     a.out = out; a.ldo = n_heads * d_head; a.row_seq = row_seq; a.row_pos = row_pos; a.nq = 1; a.n_heads = n_heads;
     a.scale = 1.0f / sqrtf((float)d_head);
-    tandem_ctx tmp;   // only the stream and the launch counter are used by the launch helpers
+    tandem_ctx tmp;   // only the stream, the launch counter and the launch options are used by the launch helpers
     tmp.stream = s;
     tmp.use_pdl = false;
+    tmp.n_sms = sm_count();
     launch_attn_decode(tmp, d_head, a, batch, 0.0);
     return check_launch();
 }
@@ -1599,18 +1604,52 @@ extern "C" tandem_status tandem_decode_attention_static(const void* q, const voi
                                    n_heads, d_head, derived_len, own_len, stream);
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Stand-alone GEMM entry points: their bounded waits report into one word per device
+// ---------------------------------------------------------------------------------------------------
+
+static __device__ int g_standalone_err;
+
 namespace {
+int* g_standalone_err_addr[MAX_DEVICES] = {};
+std::mutex g_standalone_err_mutex;
+
+// Device address of the current device's error word (looked up once per device); null if the lookup fails, in
+// which case the kernels run without reporting.
+int* standalone_err_word() {
+    const int dev = cur_dev();
+    std::lock_guard<std::mutex> lock(g_standalone_err_mutex);
+    if (!g_standalone_err_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_standalone_err) == cudaSuccess) g_standalone_err_addr[dev] = static_cast<int*>(p);
+    }
+    return g_standalone_err_addr[dev];
+}
+
 struct ProjScratch { size_t yhat, a_s, rows, total; };
 ProjScratch proj_scratch_layout(int rows, int d_small) {
     ProjScratch p;
     size_t off = 0;
     p.yhat = off; off = align_up(off + (size_t)rows * d_small * 4);
-    p.a_s = off; off = align_up(off + (size_t)rows * d_small * 2);
+    p.a_s = off; off = align_up(off + (size_t)rows * d_small * 4);
     p.rows = off; off = align_up(off + (size_t)rows * 8);
     p.total = off;
     return p;
 }
 }  // namespace
+
+extern "C" tandem_status tandem_standalone_check(void* stream) {
+    int* word = standalone_err_word();
+    if (!word) return TANDEM_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int code = 0;
+    CK(cudaMemcpyAsync(&code, word, sizeof(int), cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    if (code == 0) return TANDEM_OK;
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "device-side wait expired (code %d)", code);
+    CK(cudaMemsetAsync(word, 0, sizeof(int), s));
+    return TANDEM_ERR_TIMEOUT;
+}
 
 extern "C" size_t tandem_ff_tandem_project_scratch_bytes(int32_t rows, int32_t d_small) {
     if (rows < 1 || rows > 256 || d_small < 8) return 0;
@@ -1631,9 +1670,10 @@ extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
     tandem_ctx tmp;   // only the stream, the launch counter and the launch options are used by the launch helpers
     tmp.stream = static_cast<cudaStream_t>(stream);
     tmp.use_pdl = false;
+    tmp.n_sms = sm_count();
     unsigned char* sc = static_cast<unsigned char*>(scratch);
     float* yhat = reinterpret_cast<float*>(sc + pl.yhat);
-    bf16* a_s = reinterpret_cast<bf16*>(sc + pl.a_s);
+    float* a_s = reinterpret_cast<float*>(sc + pl.a_s);
     int* row_seq = reinterpret_cast<int*>(sc + pl.rows);
     int* row_pos = row_seq + rows;
     TcW wt, wkv;
@@ -1648,21 +1688,16 @@ extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
     iota_rows_kernel<<<cdiv(rows, 256), 256, 0, tmp.stream>>>(row_seq, row_pos, rows, 0);
     EpiArgs e; memset(&e, 0, sizeof(e));
     e.kcache = k_out; e.vcache = v_out; e.row_seq = row_seq; e.row_pos = row_pos; e.n_heads = 1; e.d_head = d_small; e.t_max = 1; e.seg = d_small;
-    if (tc_nb(rows) != 0) {
-        // few rows: weights streamed once per GEMM; LayerNorm fused into the second GEMM's operand load
-        TcScratch ts; ts.err = nullptr;
-        launch_tc_decode<PRO_BF16, EPI_STORE_F32>(tmp, ts, x, d_large, nullptr, nullptr, rows, wt, true, epi_plain(yhat, d_small));
-        if (rows <= 8 && d_small <= 1024) {
-            launch_tc_decode<PRO_LN, EPI_KV>(tmp, ts, yhat, d_small, ln_g, ln_b, rows, wkv, true, e);
-        } else {
-            launch_ex(tmp, false, 1, layernorm_rows_bf16_kernel, dim3(rows), dim3(128), 0, (const float*)yhat, static_cast<const float*>(ln_g),
-                      static_cast<const float*>(ln_b), a_s, (int)d_small);
-            launch_tc_decode<PRO_BF16, EPI_KV>(tmp, ts, a_s, d_small, nullptr, nullptr, rows, wkv, true, e);
-        }
+    // weights streamed once per GEMM and group of 64 rows; for a few short rows the LayerNorm is fused into the
+    // second GEMM's operand load
+    TcScratch ts; ts.err = standalone_err_word();
+    launch_tc_decode<PRO_BF16, EPI_STORE_F32>(tmp, ts, x, d_large, nullptr, nullptr, rows, wt, true, epi_plain(yhat, d_small));
+    if (rows <= 8 && d_small <= 1024) {
+        launch_tc_decode<PRO_LN, EPI_KV>(tmp, ts, yhat, d_small, ln_g, ln_b, rows, wkv, true, e);
     } else {
-        TRY(launch_tc_tiled<EPI_STORE_F32>(tmp, static_cast<const bf16*>(x), d_large, rows, wt, epi_plain(yhat, d_small), nullptr));
-        launch_layernorm<bf16>(tmp, rows, yhat, ln_g, ln_b, a_s, d_small);
-        TRY(launch_tc_tiled<EPI_KV>(tmp, a_s, d_small, rows, wkv, e, nullptr));
+        launch_ex(tmp, false, 1, layernorm_rows_kernel<float>, dim3(rows), dim3(128), 0, (const float*)yhat, static_cast<const float*>(ln_g),
+                  static_cast<const float*>(ln_b), a_s, (int)d_small);
+        launch_tc_decode<PRO_F32, EPI_KV>(tmp, ts, a_s, d_small, nullptr, nullptr, rows, wkv, true, e);
     }
     return check_launch();
 }
@@ -1676,13 +1711,14 @@ extern "C" tandem_status tandem_block_linear(const void* x, const void* w, void*
     tandem_ctx tmp;   // only the stream, the launch counter and the launch options are used by the launch helpers
     tmp.stream = static_cast<cudaStream_t>(stream);
     tmp.use_pdl = false;
+    tmp.n_sms = sm_count();
     TcW tw;
     if (!make_tmap_bf16(&tw.tm[0], w, (uint64_t)out_features, (uint64_t)in_features, (uint64_t)in_features)) {
         snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled unavailable or failed");
         return TANDEM_ERR_CUDA;
     }
     tw.tm[1] = tw.tm[2] = tw.tm[0]; tw.n_segs = 1; tw.seg_rows = out_features; tw.K = in_features;
-    TcScratch ts; ts.err = nullptr;
+    TcScratch ts; ts.err = standalone_err_word();
     launch_tc_decode<PRO_BF16, EPI_STORE>(tmp, ts, x, in_features, nullptr, nullptr, rows, tw, true, epi_plain(y, out_features));
     return check_launch();
 }

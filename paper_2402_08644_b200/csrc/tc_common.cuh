@@ -9,12 +9,6 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-// Measurement hooks: checkpoints that a profiling build may define to record timestamps; nothing otherwise.
-#ifndef TC_PROBE
-#define TC_PROBE_INIT(tag)
-#define TC_PROBE(slot)
-#endif
-
 namespace tandem {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -48,8 +42,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 constexpr uint32_t MBAR_POLL_LIMIT = 1u << 22;   // a healthy wait ends within a few polls
 // Waits for the phase with the given parity; false when the poll limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < MBAR_POLL_LIMIT; ++i)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = MBAR_POLL_LIMIT) {
+    for (uint32_t i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -143,8 +137,11 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
 }
-// The same barrier in two halves: arrive once this CTA no longer reads its peers' shared memory, wait before exit.
-__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+// The same barrier in two halves.  cluster_arrive_relaxed + cluster_wait is the opening handshake of a kernel that
+// writes into its peers' shared memory: a CTA arrives right after its set-up and waits just before its first
+// remote store, by which time every CTA of the cluster has started (remote shared memory may not be touched
+// before that).  No memory ordering is needed for it.
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
 // Reads a float at the same shared-memory offset in the cluster's CTA number `rank`.
 __device__ __forceinline__ float ld_dsmem_f32(uint32_t local_smem_addr, int rank) {

@@ -190,3 +190,19 @@ def make_self_tandem_weights(shape: TandemShape, seed: int, std: float = 0.02) -
         elif name.startswith("T."):
             w[name] = np.eye(shape.small.d_model, shape.large.d_model, dtype=np.float32)
     return w
+
+
+def device_weights(shape: TandemShape, seed: int, device) -> Dict[str, "torch.Tensor"]:
+    """Random-init weights of the same distribution drawn directly on a CUDA device as torch tensors (bf16
+    matrices, fp32 LayerNorm parameters), for shapes too large to draw on the host in reasonable time.  No CPU
+    checker run can use them: they serve timing and GPU-internal invariants only."""
+    import torch
+    g = torch.Generator(device=device).manual_seed(seed)
+    out = {}
+    for name in weight_names(shape):
+        shp = weight_shape(shape, name)
+        if is_norm_param(name):
+            out[name] = torch.full(shp, 1.0 if name.endswith("_g") else 0.0, dtype=torch.float32, device=device)
+        else:
+            out[name] = (torch.randn(shp, generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    return out

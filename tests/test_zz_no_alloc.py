@@ -10,6 +10,7 @@ failure has then already run every other test.
 import numpy as np
 import pytest
 
+from oracle import tandem_oracle as O
 from paper_2402_08644_b200 import binding, build
 
 pytestmark = pytest.mark.gpu
@@ -39,6 +40,13 @@ def test_static_scratch_entry_point_matches_the_ordinary_one_twice_in_a_row():
             diff = (out.float() - want.float()).abs().max().item()
             assert diff <= TOL_BF16, (B, H, dh, Td, To, call, diff)
             assert torch.equal(out, want)       # same kernels, same order: in fact bit-identical
+        # and against the CPU checker directly, so that the two entry points cannot be wrong together
+        f = lambda x: x.float().cpu().numpy().astype(np.float64)
+        for b in range(B):
+            for h in range(H):
+                K = np.concatenate([f(kd[b, h]), f(ko[b, h])], 0)
+                V = np.concatenate([f(vd[b, h]), f(vo[b, h])], 0)
+                assert np.abs(f(out[b, h]) - O.attend(f(q[b, h]), K, V, 1)).max() < TOL_BF16
 
 
 def test_static_scratch_entry_point_refuses_shapes_beyond_its_buffer():
