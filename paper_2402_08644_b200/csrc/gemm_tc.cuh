@@ -59,7 +59,7 @@ struct TcDecodeArgs {
 constexpr int TCD_THREADS = 192;   // warps 0-3: B operand + epilogue; warp 4: TMA; warp 5: TMEM + MMA issue
 template <int NB> struct TcdCfg {
     static constexpr int NB2 = 2 * NB;              // B-operand rows = accumulator columns: values, then remainders
-    static constexpr int STAGES = NB <= 16 ? 5 : (NB <= 32 ? 4 : 3);   // two CTAs fit on an SM up to NB = 48
+    static constexpr int STAGES = NB <= 16 ? 5 : 3;   // two CTAs fit on an SM up to NB = 48 (at most 113 KB each with the static part)
     static constexpr int A_BYTES = 128 * 128;       // 128 weight rows x 64 bf16
     static constexpr int B_BYTES = NB2 * 128;       // 2 NB rows x 64 bf16
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -67,6 +67,8 @@ template <int NB> struct TcdCfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + INBOX_BYTES + 1024;   // + slack to align the ring to 1024
     static constexpr int TMEM_COLS = NB2 <= 32 ? 32 : (NB2 <= 64 ? 64 : 128);
 };
+static_assert(TcdCfg<16>::SMEM_BYTES + 3072 <= 113 * 1024 && TcdCfg<32>::SMEM_BYTES + 3072 <= 113 * 1024 &&
+              TcdCfg<48>::SMEM_BYTES + 3072 <= 113 * 1024, "two CTAs per SM: a kernel and its prefetching successor");
 
 // x = hi + lo with hi = bf16(x), lo = bf16(x - hi): the pair carries x to about 16 significant bits.
 __device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
