@@ -5,7 +5,9 @@ A step is one pass of the whole path over one batch of synthetic input: the prom
 the prompt, FF_Tandem projection of every prompt position) followed by Tandem + SPEED greedy decoding of
 `max_new` tokens per sequence (draft, block verify, projection, accept/rollback, repeated).  The default
 workload is the "Small Tandem" configuration: bf16, batch 1, 512-token random prompt, gamma 3, 256 new
-tokens, natural acceptance.  The metric is generated tokens per second of the whole job.
+tokens, natural acceptance.  The metric is generated tokens per second of the decode phase over all ranks (the
+step's prompt pass is timed in the same step and reported beside it); the default line also carries compact records
+of the medium (batch 8) and large (batch 1) configurations.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload small|tiny|medium]
   python bench.py --workload micro [--micro-case B,T]     kernel micro-benchmark (decode attention, FF_Tandem projection)
@@ -53,17 +55,17 @@ def workload_desc(name):
             f"natural acceptance, random-init N(0,0.02) weights seed 0")
 
 
-# DRAM bytes per launch of the dominant kernel from one ncu capture (profiles/gemm_tc_decode_small_workload_ncu_sections.md),
-# valid only while the kernel's sources are the ones that were profiled.
-NCU_TRAFFIC = {"workload": "small", "kernel": "gemm_tc_decode", "bytes_per_launch": 4960588.4,
-               "sources_sha256_16": "3d412ad8e4eca612"}
+# DRAM bytes (read + write) of one decode iteration from one ncu capture of every kernel of an iteration, valid only
+# while the kernel sources are the ones that were profiled (else the line reports null).
+NCU_TRAFFIC = {"workload": "small", "bytes_per_iteration": None, "sources_sha256_16": ""}
 
 
 def kernel_sources_hash():
     import hashlib
     h = hashlib.sha256()
-    for fn in ("gemm_tc.cuh", "tc_common.cuh"):
-        with open(os.path.join(ROOT, "paper_2402_08644_b200", "csrc", fn), "rb") as f:
+    csrc = os.path.join(ROOT, "paper_2402_08644_b200", "csrc")
+    for fn in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, fn), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:16]
 
@@ -271,6 +273,202 @@ def run_micro(args):
     print(json.dumps(out))
 
 
+def measure_workload(name, steps, warmup, rank, local_rank, world, extras, keep_for_cpu=False):
+    """Times `steps` steps of one workload on this rank's GPU.  Returns a dict of raw timings (ms, per step unless
+    stated) plus, with `extras`, the accept-all and plain-greedy decode rates and the per-kernel pass."""
+    import torch
+    import torch.distributed as dist
+    from paper_2402_08644_b200 import binding
+
+    cfgname, B, P, gamma, new, max_pos = WORKLOADS[name]
+    shape = synth.named_config(cfgname, max_pos)
+    dev = torch.device("cuda", local_rank)
+    if name in DEVICE_INIT:
+        weights = synth.device_weights(shape, 0, dev)
+    else:
+        weights = synth.make_weights(shape, seed=0)
+    prompts = [[int(t) for t in p] for p in synth.make_prompts(B, P, shape.large.vocab, seed=rank)]
+    t = binding.Tandem(shape, weights, max_batch=B, max_seq=P + new + gamma + 1, gamma_max=gamma, device=local_rank,
+                       max_prefill_rows=B * P)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_decode(fn, reps):
+        """Mean device time (ms) of fn() after a fresh prompt pass, events on the library's stream."""
+        tot = 0.0
+        for _ in range(reps):
+            t.tandem_prefill(prompts)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream); fn(); e1.record(stream)
+            torch.cuda.synchronize()
+            tot += e0.elapsed_time(e1)
+        return tot / reps
+
+    for _ in range(warmup):
+        t.tandem_prefill(prompts)
+        t.tandem_speculative_generate(gamma, new, 0)
+
+    # ---- device-timed region: K steps between events on the stream the library launches on ----
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    barrier()
+    launches0 = t.tandem_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps + 1)]
+    ev[0].record(stream)
+    iters = 0
+    for k in range(steps):
+        t.tandem_prefill(prompts)
+        ev[2 * k + 1].record(stream)
+        out, lens, stats = t.tandem_speculative_generate(gamma, new, 0)
+        ev[2 * k + 2].record(stream)
+        iters += stats["iterations"]
+    barrier()
+    clocks = sampler.stop()
+    r = {"name": name, "shape": shape, "B": B, "P": P, "gamma": gamma, "new": new, "clocks": clocks,
+         "launches": t.tandem_launch_count() - launches0, "accept_hist": stats["accept_hist"],
+         "step_ms": ev[0].elapsed_time(ev[-1]) / steps,
+         "prefill_ms": sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(steps)) / steps,
+         "decode_ms": sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(steps)) / steps,
+         "iters_per_step": iters / steps}
+
+    # ---- end to end through the public calls with host buffers, wall clock, copies included ----
+    barrier()
+    t0 = time.perf_counter()
+    for k in range(steps):
+        t.tandem_prefill(prompts)
+        out, lens, stats = t.tandem_speculative_generate(gamma, new, 0)
+    torch.cuda.synchronize()
+    r["e2e_step_ms"] = 1e3 * (time.perf_counter() - t0) / steps
+    rows = B * (P - 1)
+    group = 128 if shape.dtype == synth.DTYPE_BF16 else 16       # queries per attention group of the prompt pass
+    r["h2d"] = 4 * (3 * rows + 2 * (rows // group + B) + 2 * B)  # row token/sequence/position, query groups, n, pending
+    r["d2h"] = 4 * (B * new + B + 16) + stats["iterations"] * 20  # tokens, lengths, histogram; 5 counters per iteration
+
+    if extras:
+        # context: accept-all timing mode and plain greedy decoding of the large model alone (graphs warmed first)
+        for fn in (lambda: t.tandem_speculative_generate(gamma, new, 1), lambda: t.tandem_large_greedy_generate(new)):
+            t.tandem_prefill(prompts); fn(); t.tandem_prefill(prompts); fn()
+        r["accept_all_decode_ms"] = timed_decode(lambda: t.tandem_speculative_generate(gamma, new, 1), 2)
+        r["greedy_decode_ms"] = timed_decode(lambda: t.tandem_large_greedy_generate(new), 2)
+        # per-kernel pass: the same step with every launch bracketed by events (serialises the stream: shares only)
+        t.tandem_profile_enable(400000)
+        t.tandem_prefill(prompts)
+        t.tandem_speculative_generate(gamma, new, 0)
+        r["prof"] = t.tandem_profile_read()
+        t.tandem_profile_enable(0)
+    t.close()
+    if keep_for_cpu:
+        r["weights"], r["prompt0"] = weights, prompts[0]
+    del t, weights
+    torch.cuda.empty_cache()
+    return r
+
+
+FLOP_CLASSES = ("gemm_tiled", "gemm_tc_tiled", "attn_prompt")     # prompt-pass kernels: work counted in flops
+
+
+def iteration_roofline(r, peak):
+    """Whole-iteration view of the decode phase: algorithmic bytes of one draft / verify iteration (weights of the
+    large model once, of the small model gamma times, projection and key/value maps once, both KV streams at the
+    mean context length) over the measured device time per iteration."""
+    T_avg = r["P"] + r["new"] / 2
+    it_bytes = algorithmic_bytes_per_iteration(r["shape"], r["B"], r["gamma"], T_avg)
+    it_ms = r["decode_ms"] / r["iters_per_step"]
+    gbs = it_bytes / 1e9 / (it_ms * 1e-3)
+    return {"algorithmic_gb": it_bytes / 1e9, "us": 1e3 * it_ms, "achieved_gbs": gbs, "frac_of_peak": gbs / peak}
+
+
+def sub_record(r, peak):
+    """Compact record of one workload for the default line."""
+    it = iteration_roofline(r, peak)
+    toks = r["B"] * r["new"]
+    rec = {"workload": workload_desc(r["name"]), "decode_tokens_per_s": toks / (r["decode_ms"] * 1e-3),
+           "step_tokens_per_s": toks / (r["step_ms"] * 1e-3), "prefill_ms": r["prefill_ms"], "decode_ms": r["decode_ms"],
+           "us_per_iteration": it["us"], "algorithmic_gb_per_iteration": it["algorithmic_gb"],
+           "achieved_gbs": it["achieved_gbs"], "frac_of_peak": it["frac_of_peak"], "accept_hist": r["accept_hist"],
+           "gpu_launches": int(r["launches"]), "clocks": r["clocks"]}
+    if "accept_all_decode_ms" in r:
+        rec["accept_all_decode_tokens_per_s"] = toks / (r["accept_all_decode_ms"] * 1e-3)
+        rec["large_greedy_decode_tokens_per_s"] = toks / (r["greedy_decode_ms"] * 1e-3)
+    return rec
+
+
+def run_ours(args, rank, local_rank, world):
+    import torch
+    import torch.distributed as dist
+    extras = rank == 0 and not args.no_extras
+    want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload not in DEVICE_INIT
+    r = measure_workload(args.workload, args.steps, args.warmup, rank, local_rank, world, extras, keep_for_cpu=want_cpu)
+    B, new, shape = r["B"], r["new"], r["shape"]
+    toks = B * new
+    # value: generated tokens per second of the decode phase (all ranks' tokens over the slowest rank's time); the
+    # prompt pass of the same step is timed separately (prefill_ms) and included in ms_per_step and step_tokens_per_s
+    value, decode_ms = replicas_throughput(r["decode_ms"], toks, world, "cuda")
+    step_value, ms_per_step = replicas_throughput(r["step_ms"], toks, world, "cuda")
+    e2e_value, _ = replicas_throughput(r["e2e_step_ms"], toks, world, "cuda")
+    peak, peak_kind = read_peaks()
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if shape.dtype == synth.DTYPE_BF16 else "f32", "data": "synthetic",
+            "config": {"workload": workload_desc(args.workload), "parallelism": f"replicas x{world}",
+                       "value_scope": "decode phase (draft, verify, project, accept) of each step; the step's prompt pass is "
+                                      "in ms_per_step, prefill_ms and step_tokens_per_s",
+                       "l2": "per-iteration working set (weights + KV) exceeds the 126 MB L2; no flush needed"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"],
+                    "scope": "whole step through the C calls with host buffers (prompt pass + decode), wall clock"},
+            "gpu_launches": int(r["launches"]), "clocks": r["clocks"], "prefill_ms": r["prefill_ms"], "decode_ms": decode_ms,
+            "step_tokens_per_s": step_value, "iterations_per_step": r["iters_per_step"], "accept_hist": r["accept_hist"]}
+
+    if extras:
+        it = iteration_roofline(r, peak)
+        prof = r["prof"]
+        line["accept_all_decode_tokens_per_s"] = toks / (r["accept_all_decode_ms"] * 1e-3)
+        line["large_greedy_decode_tokens_per_s"] = toks / (r["greedy_decode_ms"] * 1e-3)
+        tot = sum(v["ms"] for v in prof.values()) or 1.0
+        # bracketed pass: work = algorithmic bytes (GB/s) for the streaming kernels, flops (TFLOP/s) for the prompt pass
+        line["kernels_bracketed"] = {
+            k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / tot, 4),
+                "avg_us": round(1e3 * v["ms"] / max(1, v["launches"]), 3),
+                "rate": round(v["work"] / (v["ms"] * 1e-3) / (1e12 if k in FLOP_CLASSES else 1e9), 1) if v["ms"] > 0 else 0.0}
+            for k, v in prof.items() if v["launches"]}
+        decode_classes = [k for k in prof if k not in FLOP_CLASSES]
+        dec_tot = sum(prof[k]["ms"] for k in decode_classes) or 1.0
+        dom = max(decode_classes, key=lambda k: prof[k]["ms"])
+        g = prof[dom]
+        # the dominant kernel inside the timed region: its share of the bracketed decode time applied to the
+        # device-timed decode phase (graph replay, overlapped launches), so launches x time never exceeds the step
+        piped_ms = r["decode_ms"] * g["ms"] / dec_tot
+        traffic = None
+        if args.workload == NCU_TRAFFIC["workload"] and kernel_sources_hash() == NCU_TRAFFIC["sources_sha256_16"]:
+            traffic = NCU_TRAFFIC["bytes_per_iteration"]
+        line["roofline"] = {
+            "bound": "hbm", "scope": "one draft / verify iteration of the decode phase, all kernels",
+            "achieved": it["achieved_gbs"], "peak": peak, "unit": "GB/s", "frac": it["frac_of_peak"], "traffic": traffic,
+            "peak_kind": peak_kind, "algorithmic_bytes": it["algorithmic_gb"] * 1e9, "us": it["us"],
+            "dominant_kernel": {"kernel": dom, "launches": g["launches"], "share_of_decode": g["ms"] / dec_tot,
+                                "avg_launch_us": 1e3 * piped_ms / max(1, g["launches"]),
+                                "algorithmic_bytes_per_launch": g["work"] / max(1, g["launches"]),
+                                "achieved": g["work"] / 1e9 / (piped_ms * 1e-3),
+                                "frac": g["work"] / 1e9 / (piped_ms * 1e-3) / peak}}
+    if want_cpu:
+        line["cpu_baseline"] = cpu_baseline(shape, r.pop("weights"), r.pop("prompt0"), r["gamma"], new)
+    if extras and world == 1 and args.workload == "small" and not args.no_subrecords:
+        # the other batch sizes of the metric: batch 8 (medium) and the bandwidth-bound batch 1 (large), few steps each
+        line["workloads"] = {}
+        for name in ("medium", "large"):
+            rr = measure_workload(name, 2, 3, rank, local_rank, world, extras=True)
+            rr.pop("prof", None)
+            line["workloads"][name] = sub_record(rr, peak)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -281,6 +479,7 @@ def main():
     ap.add_argument("--micro-case", default="", help="with --workload micro: one attention case 'batch,context[,heads,d_head]'")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the accept-all / greedy / per-kernel passes")
+    ap.add_argument("--no-subrecords", action="store_true", help="skip the medium / large sub-records of the default line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -306,127 +505,7 @@ def main():
     if world > 1:
         dist.barrier()
 
-    cfgname, B, P, gamma, new, max_pos = WORKLOADS[args.workload]
-    shape = synth.named_config(cfgname, max_pos)
-    if args.workload in DEVICE_INIT:
-        weights = synth.device_weights(shape, 0, torch.device("cuda", local_rank))
-        args.no_cpu_baseline = True
-    else:
-        weights = synth.make_weights(shape, seed=0)
-    prompts = [[int(t) for t in p] for p in synth.make_prompts(B, P, shape.large.vocab, seed=rank)]
-    t = binding.Tandem(shape, weights, max_batch=B, max_seq=P + new + gamma + 1, gamma_max=gamma, device=local_rank,
-                       max_prefill_rows=B * P)
-    stream = torch.cuda.current_stream()
-
-    def step(mode=0):
-        t.tandem_prefill(prompts)
-        return t.tandem_speculative_generate(gamma, new, mode)
-
-    for _ in range(args.warmup):
-        out, lens, stats = step()
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    # ---- device-timed region: K steps between events on the stream the library launches on ----
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    barrier()
-    launches0 = t.tandem_launch_count()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
-    ev[0].record(stream)
-    iters = 0
-    for k in range(args.steps):
-        t.tandem_prefill(prompts)
-        ev[2 * k + 1].record(stream)
-        out, lens, stats = t.tandem_speculative_generate(gamma, new, 0)
-        ev[2 * k + 2].record(stream)
-        iters += stats["iterations"]
-    barrier()
-    clocks = sampler.stop()
-    launches = t.tandem_launch_count() - launches0
-    total_ms = ev[0].elapsed_time(ev[-1])
-    prefill_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(args.steps)) / args.steps
-    decode_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(args.steps)) / args.steps
-    value, ms_per_step = replicas_throughput(total_ms / args.steps, B * new, world, "cuda")
-
-    # ---- end to end through the public calls with host buffers, wall clock, copies included ----
-    barrier()
-    t0 = time.perf_counter()
-    for k in range(args.steps):
-        out, lens, stats = step()
-    torch.cuda.synchronize()
-    e2e_value, _ = replicas_throughput(1e3 * (time.perf_counter() - t0) / args.steps, B * new, world, "cuda")
-    rows = B * (P - 1)
-    group = 128 if shape.dtype == synth.DTYPE_BF16 else 16       # queries per attention group of the prompt pass
-    h2d = 4 * (3 * rows + 2 * (rows // group + B) + 2 * B)       # row token/sequence/position, query groups, n, pending
-    d2h = 4 * (B * new + B + 16) + stats["iterations"] * 20      # tokens, lengths, histogram; 5 counters per iteration
-    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
-
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if shape.dtype == synth.DTYPE_BF16 else "f32", "data": "synthetic",
-            "config": {"workload": workload_desc(args.workload), "parallelism": f"replicas x{world}",
-                       "l2": "per-iteration working set (weights + KV) exceeds the 126 MB L2; no flush needed"},
-            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "prefill_ms": prefill_ms, "decode_ms": decode_ms, "decode_tokens_per_s": B * new / (decode_ms * 1e-3),
-            "iterations_per_step": iters / args.steps, "accept_hist": stats["accept_hist"]}
-
-    if rank == 0 and not args.no_extras:
-        peak, peak_kind = read_peaks()
-        # whole-iteration view: algorithmic bytes of one draft/verify iteration over the measured time per iteration
-        T_avg = P + new / 2
-        it_bytes = algorithmic_bytes_per_iteration(shape, B, gamma, T_avg)
-        it_ms = decode_ms / (iters / args.steps)
-        line["iteration"] = {"algorithmic_gb": it_bytes / 1e9, "ms": it_ms, "achieved_gbs": it_bytes / 1e9 / (it_ms * 1e-3),
-                             "frac_of_peak": it_bytes / 1e9 / (it_ms * 1e-3) / peak}
-        # per-kernel pass: the same step with every launch bracketed by events (slower; not the timed value)
-        t.tandem_profile_enable(200000)
-        step()
-        prof = t.tandem_profile_read()
-        t.tandem_profile_enable(0)
-        tot = sum(v["ms"] for v in prof.values()) or 1.0
-        # work: algorithmic bytes per second (GB/s) for the streaming kernels, flops per second (TFLOP/s) for the prompt pass
-        line["kernels"] = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / tot, 4),
-                               "avg_us": round(1e3 * v["ms"] / max(1, v["launches"]), 3),
-                               "rate": round(v["work"] / (v["ms"] * 1e-3) / (1e12 if k in ("gemm_tiled", "gemm_tc_tiled", "attn_prompt") else 1e9), 1)
-                               if v["ms"] > 0 else 0.0} for k, v in prof.items()}
-        flop_classes = ("gemm_tiled", "gemm_tc_tiled", "attn_prompt")     # prompt-pass kernels: work counted in flops
-        dom = max((k for k in prof if k not in flop_classes), key=lambda k: prof[k]["ms"])
-        g = prof[dom]
-        achieved = g["work"] / 1e9 / (g["ms"] * 1e-3) if g["ms"] > 0 else 0.0
-        traffic = None
-        if (args.workload == NCU_TRAFFIC["workload"] and dom == NCU_TRAFFIC["kernel"]
-                and kernel_sources_hash() == NCU_TRAFFIC["sources_sha256_16"]):
-            traffic = NCU_TRAFFIC["bytes_per_launch"]
-        line["roofline"] = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                            "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
-                            "launches": g["launches"], "avg_launch_us": 1e3 * g["ms"] / max(1, g["launches"]),
-                            "algorithmic_bytes_per_launch": g["work"] / max(1, g["launches"])}
-        # The bracketing events serialise the stream and add their own latency to every launch.  For context: the
-        # kernel's share of the bracketed pass applied to the timed region itself (graph replay, launches overlapped).
-        decode_classes = [k for k in prof if k not in flop_classes]
-        dec_tot = sum(prof[k]["ms"] for k in decode_classes) or 1.0
-        piped_ms = decode_ms * g["ms"] / dec_tot
-        line["roofline"]["in_pipeline"] = {"avg_launch_us": 1e3 * piped_ms / max(1, g["launches"]),
-                                           "achieved": g["work"] / 1e9 / (piped_ms * 1e-3),
-                                           "frac": g["work"] / 1e9 / (piped_ms * 1e-3) / peak}
-        # context: accept-all timing mode and plain greedy decoding of the large model alone
-        t.tandem_prefill(prompts); torch.cuda.synchronize()
-        t0 = time.perf_counter(); t.tandem_speculative_generate(gamma, new, 1); torch.cuda.synchronize()
-        line["accept_all_decode_tokens_per_s"] = B * new / (time.perf_counter() - t0)
-        t.tandem_prefill(prompts); torch.cuda.synchronize()
-        t0 = time.perf_counter(); t.tandem_large_greedy_generate(new); torch.cuda.synchronize()
-        line["large_greedy_decode_tokens_per_s"] = B * new / (time.perf_counter() - t0)
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(shape, weights, prompts[0], gamma, new)
-    t.close()
-    if rank == 0:
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    run_ours(args, rank, local_rank, world)
 
 
 if __name__ == "__main__":
