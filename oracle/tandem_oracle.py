@@ -40,9 +40,17 @@ Readings taken where the paper is silent or inconsistent:
   R13 accept_mode 1 keeps all gamma drafts whatever the comparison says (equal to stand-alone Tandem
       with the free token, Figure 2); accept_mode 2 takes a pseudo-random accept length from a
       counter-based hash (test only).
+  R16 Stand-alone Tandem (Section 3, "Inference", the two configurations; Figures 2 and 3).
+      "Representation Generation Only": per round the small model appends gamma tokens starting from the
+      pending token, then the large model reads the pending token and the first gamma-1 new tokens as one
+      block of gamma rows, without an output head; the last new token becomes pending (Figure 3, right).
+      "Representation Generation + Token Prediction" for the prompt too (Figure 2, left): the large model
+      reads all P prompt tokens and its prediction is the first response token, which becomes pending.
+      A response that is not a whole number of blocks long drops the surplus of the last round (as R12).
 
 Pins: every function here is pinned by tests/test_oracle_*.py (library decoder layer, both FF_Tandem
-branches against library modules and closed forms, brute force vs cache, SPEED == plain greedy, self-tandem, block == single-token passes, schedule fixtures from
+branches against library modules and closed forms, brute force vs cache, the stand-alone variants against
+brute-force loops, Figure 3's schedule and the self-tandem collapse, SPEED == plain greedy, self-tandem, block == single-token passes, schedule fixtures from
 Figures 2 and 3, hand-made accept cases).  The absolute logit values of a random-init *Tandem* pair
 have no value printed in the paper to compare with: for those, parity unpinned beyond the invariants.
 """
@@ -298,6 +306,54 @@ class TandemOracle:
             self._project_rows(reps, range(m))
             self.schedule.append(("L", list(range(m))))
 
+    def prefill_all_tokens(self, prompt: Sequence[int]) -> int:
+        """Figure 2, left (R16): the large model reads the whole prompt; its prediction for the next position is
+        the first response token, which is appended and becomes the pending token.  Returns that token."""
+        assert len(prompt) >= 1
+        self.tokens = [int(t) for t in prompt]
+        P = len(prompt)
+        reps, logits = large_block_pass(self.large, self.large_cache, self.tokens, 0)
+        self._project_rows(reps, range(P))
+        self.n_large_runs += 1
+        self.schedule.append(("L", list(range(P))))
+        first = argmax_decision(logits[P - 1])
+        self.tokens.append(first)
+        return first
+
+    def step_representation_only(self, gamma: int, forced: Optional[Sequence[int]] = None) -> dict:
+        """One round of stand-alone Tandem without the free token (Figure 3, R16): gamma small-model steps from the
+        pending token; all gamma tokens are kept; the large model then reads the pending token and the first
+        gamma-1 new tokens as one block (no output head) and those rows are projected for the small model."""
+        assert gamma >= 1
+        n = len(self.tokens)
+        drafts, s_logits = self.draft(gamma, forced)
+        kept = [int(t) for t in (forced if forced is not None else drafts)]
+        rows = [self.tokens[-1]] + kept[:-1]
+        reps, _ = large_block_pass(self.large, self.large_cache, rows, n - 1)
+        self.n_large_runs += 1
+        self.schedule.append(("L", list(range(n - 1, n - 1 + gamma))))
+        self.tokens += kept
+        self._project_rows(reps, range(gamma))
+        self.own.truncate(0)
+        self.iteration += 1
+        return {"drafts": drafts, "emitted": kept, "small_logits": s_logits, "n_committed": len(self.tokens), "reps": reps}
+
+    def generate_representation_only(self, prompt: Sequence[int], gamma: int, max_new: int) -> List[int]:
+        self.prefill(prompt)
+        P = len(prompt)
+        while len(self.tokens) - P < max_new:
+            self.step_representation_only(gamma)
+        return self.tokens[P:P + max_new]
+
+    def generate_free_token_full_prompt(self, prompt: Sequence[int], gamma: int, max_new: int) -> List[int]:
+        """Figure 2 as drawn: the first response token comes from the large model reading the whole prompt, then
+        rounds of gamma small-model tokens followed by one large-model token (accept-all rounds)."""
+        self.prefill_all_tokens(prompt)
+        P = len(prompt)
+        while len(self.tokens) - P < max_new:
+            self.step(gamma, ACCEPT_ALL)
+        return self.tokens[P:P + max_new]
+
     # --- one token through the small model over the mixed context (Eq. 2, lines 2-3) --------------
     def _small_step(self, token: int, index: int) -> np.ndarray:
         sm = self.small
@@ -443,6 +499,48 @@ def standalone_tandem_free_token(shape, weights: Dict[str, np.ndarray], prompt: 
             seq.append(argmax_decision(lg[-1]))
         _, logits = decoder_full_forward(large, seq)
         seq.append(argmax_decision(logits[-1]))
+    return seq[P:P + max_new]
+
+
+def standalone_tandem_representation_only(shape, weights: Dict[str, np.ndarray], prompt: Sequence[int], gamma: int,
+                                          max_new: int, dtype=np.float64) -> List[int]:
+    """Stand-alone Tandem decoding without the free token, written directly from Figure 3 and the
+    "Representation Generation Only" variant of Section 3, by brute force (no cache).
+
+    Each round: the large model's representations of everything but the last token are recomputed from
+    scratch; the small model, attending them, appends gamma tokens one at a time.  The large model never
+    predicts a token."""
+    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
+    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype)
+    proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
+    seq = [int(t) for t in prompt]
+    P = len(seq)
+    while len(seq) - P < max_new:
+        boundary = len(seq) - 1
+        reps, _ = decoder_full_forward(large, seq[:boundary])
+        for _ in range(gamma):
+            lg = tandem_small_full_forward(small, proj, shape.layer_map, reps, boundary, seq)
+            seq.append(argmax_decision(lg[-1]))
+    return seq[P:P + max_new]
+
+
+def standalone_tandem_free_token_full_prompt(shape, weights: Dict[str, np.ndarray], prompt: Sequence[int], gamma: int,
+                                             max_new: int, dtype=np.float64) -> List[int]:
+    """Figure 2 as drawn, by brute force: the large model reads the whole sequence and appends its prediction;
+    the small model, attending the large model's representations of everything before that token, appends
+    gamma tokens; repeat."""
+    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
+    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype)
+    proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
+    seq = [int(t) for t in prompt]
+    P = len(seq)
+    while len(seq) - P < max_new:
+        reps, logits = decoder_full_forward(large, seq)
+        boundary = len(seq)
+        seq.append(argmax_decision(logits[-1]))
+        for _ in range(gamma):
+            lg = tandem_small_full_forward(small, proj, shape.layer_map, reps, boundary, seq)
+            seq.append(argmax_decision(lg[-1]))
     return seq[P:P + max_new]
 
 

@@ -232,3 +232,92 @@ def test_hash_mode_still_emits_valid_lengths_and_counts_runs():
     for a, (nl, ns) in zip(accs, runs):
         assert nl == len(a) and ns == 3 * len(a)   # one large run and gamma small runs per iteration
         assert sum(x + 1 for x in a) >= 10 > sum(x + 1 for x in a[:-1])
+
+
+# ------------------------------------------------------------------------------------------------
+# Stand-alone Tandem variants (Section 3 "Inference"; Figures 2 and 3)
+# ------------------------------------------------------------------------------------------------
+
+def test_representation_only_cached_equals_brute_force_figure3():
+    for kind, gamma, new in ((synth.FF_TANDEM_LINEAR, 2, 9), (synth.FF_TANDEM_MLP, 3, 8), (synth.FF_TANDEM_LINEAR, 1, 4)):
+        shape = toy_shape(kind=kind, hidden=12 if kind else 0)
+        w = toy_weights(shape, seed=40 + gamma)
+        prompt = _prompt(shape, 5, seed=gamma)
+        got = O.TandemOracle(shape, w).generate_representation_only(prompt, gamma, new)
+        assert got == O.standalone_tandem_representation_only(shape, w, prompt, gamma, new)
+        assert len(got) == new
+    # it is neither the large model's greedy decoding nor the free-token variant
+    assert got != O.plain_greedy(shape, w, prompt, new)
+
+
+def test_representation_only_schedule_matches_figure3_for_three_blocks():
+    shape = toy_shape()
+    w = toy_weights(shape, seed=1)
+    o = O.TandemOracle(shape, w)
+    o.prefill(_prompt(shape, 8))
+    for _ in range(3):
+        o.step_representation_only(2)
+    assert o.schedule == _read_schedule("fig3_schedule_three_blocks_gamma2.txt")
+    assert (o.n_large_runs, o.n_small_runs) == (3, 6)
+    assert o.large_cache.length() == o.derived.length() == len(o.tokens) - 1 and o.own.length() == 0
+
+
+def _derived_boundaries(schedule):
+    """For every small-model run: (its position, number of positions the large model had read before it)."""
+    seen, out = 0, []
+    for model, positions in schedule:
+        if model == "L":
+            seen = max(seen, positions[-1] + 1)
+        else:
+            out.append((positions[0], seen))
+    return out
+
+
+def test_both_variants_agree_on_which_positions_are_large_derived():
+    """Whenever the small model runs at position p inside a block that starts at position s, the large model has
+    read exactly positions 0..s-1 — with and without the free token (the training bullets of Section 3)."""
+    shape = toy_shape()
+    w = toy_weights(shape, seed=3)
+    for gamma in (1, 2, 4):
+        a, b = O.TandemOracle(shape, w), O.TandemOracle(shape, w)
+        a.prefill(_prompt(shape, 6)); b.prefill(_prompt(shape, 6))
+        for _ in range(3):
+            a.step_representation_only(gamma)
+            b.step(gamma, mode=O.ACCEPT_ALL)
+        for sched, per_round in ((a.schedule, gamma), (b.schedule, gamma + 1)):
+            runs = _derived_boundaries(sched)
+            assert len(runs) == 3 * gamma
+            for i, (pos, seen) in enumerate(runs):
+                block_start = 5 + (i // gamma) * per_round
+                assert seen == block_start and block_start <= pos < block_start + gamma
+
+
+def test_self_tandem_representation_only_is_plain_greedy():
+    """Small = large, identity FF_Tandem, l(j) = j: Eq. 2 is Eq. 1 for any boundary, so the small model's tokens are
+    the large model's greedy tokens although the large model never predicts anything."""
+    dims = synth.ModelDims(2, 32, 4, 64, 50, 64)
+    shape = synth.self_tandem_shape(dims)
+    w = synth.make_self_tandem_weights(shape, seed=6, std=0.35)
+    prompt = _prompt(shape, 4, seed=9)
+    got = O.TandemOracle(shape, w).generate_representation_only(prompt, 3, 10)
+    assert got == O.plain_greedy(shape, w, prompt, 10)
+
+
+def test_full_prompt_free_token_variant_matches_brute_force_and_figure2():
+    shape = toy_shape(kind=synth.FF_TANDEM_MLP, hidden=12)
+    w = toy_weights(shape, seed=23)
+    prompt = _prompt(shape, 8, seed=2)
+    o = O.TandemOracle(shape, w)
+    got = o.generate_free_token_full_prompt(prompt, 2, 9)
+    assert got == O.standalone_tandem_free_token_full_prompt(shape, w, prompt, 2, 9)
+    assert got[0] == O.plain_greedy(shape, w, prompt, 1)[0]          # the first token is the large model's own
+    # Figure 2's schedule: the golden file describes it from the 9-token prompt (query + free token) onwards
+    fig2 = _read_schedule("fig2_schedule_gamma2.txt")
+    assert o.schedule[: len(fig2)] == fig2
+    # reading the whole prompt at once equals the Figure-3 prompt pass followed by a one-row large step
+    a, b = O.TandemOracle(shape, w), O.TandemOracle(shape, w)
+    first = a.prefill_all_tokens(prompt)
+    b.prefill(prompt)
+    assert b.step(0)["emitted"] == [first] and a.tokens == b.tokens
+    for layer in range(shape.small.n_layers):
+        assert np.allclose(np.stack(a.derived.k[layer]), np.stack(b.derived.k[layer]), atol=1e-10)
