@@ -354,6 +354,10 @@ def measure_workload(name, steps, warmup, rank, local_rank, world, extras, keep_
             t.tandem_prefill(prompts); fn(); t.tandem_prefill(prompts); fn()
         r["accept_all_decode_ms"] = timed_decode(lambda: t.tandem_speculative_generate(gamma, new, 1), 2)
         r["greedy_decode_ms"] = timed_decode(lambda: t.tandem_large_greedy_generate(new), 2)
+        # stand-alone Tandem without the free token (the small model writes the response; Figure 3)
+        rep_only = lambda: t.tandem_standalone_generate(gamma, binding.STANDALONE_REPRESENTATION_ONLY, new)
+        t.tandem_prefill(prompts); rep_only(); t.tandem_prefill(prompts); rep_only()
+        r["representation_only_decode_ms"] = timed_decode(rep_only, 2)
         # per-kernel pass: the same step with every launch bracketed by events (serialises the stream: shares only)
         t.tandem_profile_enable(400000)
         t.tandem_prefill(prompts)
@@ -394,6 +398,7 @@ def sub_record(r, peak):
     if "accept_all_decode_ms" in r:
         rec["accept_all_decode_tokens_per_s"] = toks / (r["accept_all_decode_ms"] * 1e-3)
         rec["large_greedy_decode_tokens_per_s"] = toks / (r["greedy_decode_ms"] * 1e-3)
+        rec["standalone_representation_only_decode_tokens_per_s"] = toks / (r["representation_only_decode_ms"] * 1e-3)
     return rec
 
 
@@ -428,6 +433,7 @@ def run_ours(args, rank, local_rank, world):
         prof = r["prof"]
         line["accept_all_decode_tokens_per_s"] = toks / (r["accept_all_decode_ms"] * 1e-3)
         line["large_greedy_decode_tokens_per_s"] = toks / (r["greedy_decode_ms"] * 1e-3)
+        line["standalone_representation_only_decode_tokens_per_s"] = toks / (r["representation_only_decode_ms"] * 1e-3)
         tot = sum(v["ms"] for v in prof.values()) or 1.0
         # bracketed pass: work = algorithmic bytes (GB/s) for the streaming kernels, flops (TFLOP/s) for the prompt pass
         line["kernels_bracketed"] = {

@@ -64,7 +64,15 @@ enum { TANDEM_FF_LINEAR = 0, TANDEM_FF_MLP = 1 };
 /* accept_mode: 0 = compare drafts with M_L's arg-max (Section 3.1); 1 = keep all gamma drafts (equals
  * stand-alone Tandem with the free token, Figure 2); 2 = accept length drawn from a counter-based hash
  * of (mode_seed, sequence, iteration), for tests of ragged accept lengths. */
-enum { TANDEM_ACCEPT_NATURAL = 0, TANDEM_ACCEPT_ALL = 1, TANDEM_ACCEPT_HASH = 2 };
+enum { TANDEM_ACCEPT_NATURAL = 0, TANDEM_ACCEPT_ALL = 1, TANDEM_ACCEPT_HASH = 2,
+       /* 3 = a round of stand-alone Tandem without the free token ("Representation Generation Only", Section 3
+        * "Inference", Figure 3): M_L reads the pending token and the first gamma-1 drafts as gamma rows and
+        * predicts nothing, all gamma drafts are kept, the last one becomes pending.  Needs gamma >= 1; a step
+        * result's targets are -1. */
+       TANDEM_ACCEPT_REPRESENTATION_ONLY = 3 };
+/* variants of tandem_standalone_generate */
+enum { TANDEM_STANDALONE_FREE_TOKEN = 0, TANDEM_STANDALONE_REPRESENTATION_ONLY = 1,
+       TANDEM_STANDALONE_FREE_TOKEN_FULL_PROMPT = 2 };
 
 #define TANDEM_GAMMA_LIMIT 15 /* largest block length gamma a context can be created for */
 
@@ -151,7 +159,7 @@ TANDEM_API tandem_status tandem_prefill(tandem_ctx* ctx, int32_t batch, const in
  *   accept  per sequence: a = length of the longest prefix of drafts equal to M_L's arg-max; the sequence
  *           gains d_1..d_a and M_L's token for the next position, which becomes pending; both caches
  *           roll back to the kept positions (a length update; no data moves).
- * 0 <= gamma <= gamma_max.  result may be NULL (the call is then asynchronous); filling it waits for
+ * 0 <= gamma <= gamma_max; accept_mode: TANDEM_ACCEPT_*.  result may be NULL (the call is then asynchronous); filling it waits for
  * the stream.  Fails with TANDEM_ERR_CAPACITY, launching nothing, if a sequence could outgrow max_seq. */
 TANDEM_API tandem_status tandem_block_step(tandem_ctx* ctx, int32_t gamma, int32_t accept_mode, uint64_t mode_seed,
                                 tandem_step_result* result /* HOST, nullable */);
@@ -163,6 +171,22 @@ TANDEM_API tandem_status tandem_block_step(tandem_ctx* ctx, int32_t gamma, int32
 TANDEM_API tandem_status tandem_speculative_generate(tandem_ctx* ctx, int32_t gamma, int32_t max_new_tokens,
                                           int32_t accept_mode, uint64_t mode_seed, int32_t* out_ids,
                                           int32_t* out_lens, tandem_stats* stats);
+
+/* Stand-alone Tandem decoding (Section 3 "Inference"; Table 3's latency row): M_S writes the response, M_L only
+ * supplies representations (and, with the free token, one token per block); nothing is verified.  Must follow
+ * tandem_prefill; same buffers and stop rule as tandem_speculative_generate; 1 <= gamma <= gamma_max.
+ *   TANDEM_STANDALONE_FREE_TOKEN              "Representation Generation + Token Prediction" (Figure 2) for the
+ *       response blocks after the prompt pass of tandem_prefill (which is Figure 3's): per round M_S appends gamma
+ *       tokens, M_L reads the pending token and those gamma tokens and appends its own next token.
+ *   TANDEM_STANDALONE_REPRESENTATION_ONLY     "Representation Generation Only" (Figure 3): per round M_S appends
+ *       gamma tokens, M_L reads gamma rows (the pending token and the first gamma-1 new ones) without its
+ *       output head; the last new token is M_S's next input.
+ *   TANDEM_STANDALONE_FREE_TOKEN_FULL_PROMPT  Figure 2 as drawn: M_L first reads the last prompt token too and
+ *       its prediction is the first response token; then rounds as in TANDEM_STANDALONE_FREE_TOKEN.
+ * stats->accept_hist counts rounds by the number of M_S tokens kept (gamma; 0 for the leading M_L round). */
+TANDEM_API tandem_status tandem_standalone_generate(tandem_ctx* ctx, int32_t gamma, int32_t variant,
+                                                    int32_t max_new_tokens, int32_t* out_ids, int32_t* out_lens,
+                                                    tandem_stats* stats);
 
 /* Baseline and invariant hook: plain greedy decoding of M_L alone, one token per pass (the output that
  * Tandem + SPEED must reproduce; abstract and Section 3.1).  Same buffers as above.  Leaves the small

@@ -18,7 +18,8 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtandem_
 _lib = None
 
 GAMMA_LIMIT = 15
-ACCEPT_NATURAL, ACCEPT_ALL, ACCEPT_HASH = 0, 1, 2
+ACCEPT_NATURAL, ACCEPT_ALL, ACCEPT_HASH, ACCEPT_REPRESENTATION_ONLY = 0, 1, 2, 3
+STANDALONE_FREE_TOKEN, STANDALONE_REPRESENTATION_ONLY, STANDALONE_FREE_TOKEN_FULL_PROMPT = 0, 1, 2
 STATUS_NAMES = ["OK", "INVALID_ARG", "SHAPE", "ARENA_TOO_SMALL", "CAPACITY", "STATE", "CUDA", "TIMEOUT", "UNIMPLEMENTED"]
 (READ_LARGE_LOGITS, READ_SMALL_LOGITS, READ_LARGE_HIDDEN, READ_LARGE_K, READ_LARGE_V, READ_SMALL_K, READ_SMALL_V,
  READ_COMMITTED) = range(8)
@@ -29,7 +30,7 @@ EXPORTS = ["tandem_query_arena", "tandem_create", "tandem_destroy", "tandem_pref
            "tandem_ff_tandem_project_scratch_bytes", "tandem_block_linear",
            "tandem_status_string", "tandem_last_cuda_error", "tandem_profile_enable", "tandem_profile_read",
            "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static",
-           "tandem_debug_expire_wait", "tandem_standalone_check"]
+           "tandem_debug_expire_wait", "tandem_standalone_check", "tandem_standalone_generate"]
 
 
 class TandemError(RuntimeError):
@@ -88,6 +89,7 @@ def load_library():
     lib.tandem_block_step.argtypes = [vp, i32, i32, u64, C.POINTER(StepResult)]
     lib.tandem_speculative_generate.argtypes = [vp, i32, i32, i32, u64, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_large_greedy_generate.argtypes = [vp, i32, pi32, pi32, C.POINTER(Stats)]
+    lib.tandem_standalone_generate.argtypes = [vp, i32, i32, i32, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_debug_read.argtypes = [vp, i32, i32, i32, vp, sz]
     lib.tandem_decode_attention_scratch_bytes.argtypes = [i32] * 5
     lib.tandem_decode_attention_scratch_bytes.restype = sz
@@ -226,6 +228,15 @@ class Tandem:
         p = lambda x: x.ctypes.data_as(C.POINTER(C.c_int32))
         _check(self.lib.tandem_speculative_generate(self.ctx, gamma, max_new, accept_mode, mode_seed, p(out), p(lens),
                                                     C.byref(st)), "tandem_speculative_generate")
+        return out, lens, self._stats(st, gamma)
+
+    def tandem_standalone_generate(self, gamma: int, variant: int, max_new: int):
+        out = np.zeros((self.batch, max_new), np.int32)
+        lens = np.zeros(self.batch, np.int32)
+        st = Stats()
+        p = lambda x: x.ctypes.data_as(C.POINTER(C.c_int32))
+        _check(self.lib.tandem_standalone_generate(self.ctx, gamma, variant, max_new, p(out), p(lens), C.byref(st)),
+               "tandem_standalone_generate")
         return out, lens, self._stats(st, gamma)
 
     def tandem_large_greedy_generate(self, max_new: int):

@@ -251,13 +251,26 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restric
 //   the sequence gains d_1..d_a and g_{a+1}; n advances; g_{a+1} becomes pending.
 // Rolling the caches back is the update of n: positions >= n-1 are rewritten by the next iteration.
 // When amax_val is given, the large model's arg-max per block row is first finished from the per-tile results of
-// its output-head GEMM.  block: 256.
+// its output-head GEMM.
+// mode 3 is the round of stand-alone Tandem without the free token (Section 3 "Inference", "Representation
+// Generation Only"; Figure 3): the large model has read gamma rows and predicted nothing, all gamma tokens of the
+// small model are kept and the last one becomes pending.  The last draft is then not a block row, so nobody has
+// turned it into a token id yet: when fin_val is given it is finished here from the small head's per-tile results.
+// block: 256.
 __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed,
                                                      int max_new, const float* amax_val, const int* amax_idx, int amax_stride,
-                                                     int n_tiles) {
+                                                     int n_tiles, const float* fin_val, const int* fin_idx) {
     pdl_wait();
     pdl_launch_dependents();
-    if (amax_val != nullptr) {
+    if (mode == 3) {
+        if (fin_val != nullptr && gamma > 0) {
+            for (int b = threadIdx.x >> 5; b < batch; b += 8) {
+                const int tok = argmax_from_tiles(fin_val + (size_t)b * amax_stride, fin_idx + (size_t)b * amax_stride, n_tiles);
+                if ((threadIdx.x & 31) == 0) st.drafts[b * st.gamma_limit + gamma - 1] = tok;
+            }
+        }
+        __syncthreads();
+    } else if (amax_val != nullptr) {
         const int rows = batch * (gamma + 1);
         for (int m = threadIdx.x >> 5; m < rows; m += 8) {
             const int tok = argmax_from_tiles(amax_val + (size_t)m * amax_stride, amax_idx + (size_t)m * amax_stride, n_tiles);
@@ -273,14 +286,14 @@ __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, in
         const int* d = st.drafts + b * st.gamma_limit;
         const int* g = st.targets + b * (st.gamma_limit + 1);
         int a = 0;
-        if (mode == 1) a = gamma;
+        if (mode == 1 || mode == 3) a = gamma;
         else if (mode == 2) a = (int)(splitmix64(splitmix64(splitmix64(seed) ^ (unsigned long long)b) ^ (unsigned long long)iteration) % (unsigned long long)(gamma + 1));
         else { while (a < gamma && d[a] == g[a]) ++a; }
         st.accept_len[b] = a;
         atomicAdd(st.hist + a, 1ull);
         const int em = st.emitted[b];
         const int room = max_new - em;
-        const int take = min(a + 1, room);
+        const int take = min(mode == 3 ? a : a + 1, room);
         int last = st.pending[b];
         for (int i = 0; i < take; ++i) {
             last = (i < a) ? d[i] : g[a];

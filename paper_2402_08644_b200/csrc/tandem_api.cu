@@ -745,14 +745,21 @@ void launch_verify(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_ne
     ProfScope ps(c, PC_VERIFY, (double)c.batch * (2 * gamma + 8) * 4.0);
     launch_ex(c, true, 1, verify_kernel, dim3(1), dim3(256), 0, c.st, c.batch, gamma, mode, (unsigned long long)seed, max_new,
               from_tiles ? (const float*)at<float>(c, c.lay.amax_val_large) : (const float*)nullptr,
-              from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_large) : (const int*)nullptr, c.lay.vocab_tiles, c.lay.vocab_tiles);
+              from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_large) : (const int*)nullptr, c.lay.vocab_tiles, c.lay.vocab_tiles,
+              from_tiles ? (const float*)at<float>(c, c.lay.amax_val_small) : (const float*)nullptr,
+              from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_small) : (const int*)nullptr);
 }
 
 template <typename T>
 void iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
     for (int s = 0; s < gamma; ++s) small_step<T>(c, s);
-    setup_rows(c, 0, gamma + 1);
-    large_pass<T>(c, decode_rows(c, gamma, gamma + 1), true, true);
+    if (mode == 3) {   // stand-alone Tandem without the free token: gamma rows, no output head
+        setup_rows(c, 0, gamma);
+        large_pass<T>(c, decode_rows(c, gamma - 1, gamma), true, false);
+    } else {
+        setup_rows(c, 0, gamma + 1);
+        large_pass<T>(c, decode_rows(c, gamma, gamma + 1), true, true);
+    }
     launch_verify(c, gamma, mode, seed, max_new, false);
     c.last_gamma = gamma;
 }
@@ -882,7 +889,9 @@ int project_slot(const tandem_ctx& c, int n) {
     return -1;
 }
 
-void tc_large_block(tandem_ctx& c, int gamma, bool project) {
+// The large model over nq block rows per sequence (row 0 = pending token, row r = draft r); fin_r: block row whose
+// token the small model's last head GEMM left as per-tile results (-1: none); head: final LayerNorm + output head.
+void tc_large_block(tandem_ctx& c, int nq, int fin_r, bool project, bool head) {
     float* h = at<float>(c, c.lay.h_large);
     const size_t snap_elems = (size_t)c.lay.dec_rows * c.large.d.d_model;
     auto snap_of = [&](int n) -> float* {
@@ -890,14 +899,14 @@ void tc_large_block(tandem_ctx& c, int gamma, bool project) {
         return slot >= 0 ? at<float>(c, c.lay.proj_snap) + (size_t)slot * snap_elems : nullptr;
     };
     bool any_fork = false;
-    tc_begin(c, c.large, h, 0, gamma + 1, gamma > 0 ? gamma : -1, snap_of(0));
-    const Rows r = decode_rows(c, gamma, gamma + 1);
+    tc_begin(c, c.large, h, 0, nq, fin_r, snap_of(0));
+    const Rows r = decode_rows(c, nq - 1, nq);
     if (project && project_slot(c, 0) >= 0) { tc_project_forked(c, 0, project_slot(c, 0), r); any_fork = true; }
     for (int l = 0; l < c.large.d.n_layers; ++l) {
         tc_decoder_layer(c, c.large, l, h, r, true, snap_of(l + 1));
         if (project && project_slot(c, l + 1) >= 0) { tc_project_forked(c, l + 1, project_slot(c, l + 1), r); any_fork = true; }
     }
-    tc_head(c, c.large, h, r, at<float>(c, c.lay.logits_large), c.lay.amax_val_large, c.lay.amax_idx_large, true);
+    if (head) tc_head(c, c.large, h, r, at<float>(c, c.lay.logits_large), c.lay.amax_val_large, c.lay.amax_idx_large, true);
     if (any_fork) {   // the projections join the main stream before the verify kernel
         cudaEventRecord(c.ev_join, c.side);
         cudaStreamWaitEvent(c.stream, c.ev_join, 0);
@@ -907,13 +916,14 @@ void tc_large_block(tandem_ctx& c, int gamma, bool project) {
 
 void tc_iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
     for (int s = 0; s < gamma; ++s) tc_small_step(c, s);
-    tc_large_block(c, gamma, true);
+    if (mode == 3) tc_large_block(c, gamma, -1, true, false);   // gamma rows, no head: the last draft is finished by the verify kernel
+    else tc_large_block(c, gamma + 1, gamma > 0 ? gamma : -1, true, true);
     launch_verify(c, gamma, mode, seed, max_new, true);
     c.last_gamma = gamma;
 }
 
 void tc_greedy_iteration(tandem_ctx& c, int max_new) {
-    tc_large_block(c, 0, false);
+    tc_large_block(c, 1, -1, false, true);
     launch_verify(c, 0, 0, 0ull, max_new, true);
     c.last_gamma = 0;
 }
@@ -1269,7 +1279,8 @@ tandem_status capacity_for(tandem_ctx* c, int extra_tokens, int gamma) {
 extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t accept_mode, uint64_t mode_seed,
                                            tandem_step_result* result) {
     TRY(begin_call(c));
-    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 2) return TANDEM_ERR_INVALID_ARG;
+    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 3) return TANDEM_ERR_INVALID_ARG;
+    if (accept_mode == TANDEM_ACCEPT_REPRESENTATION_ONLY && gamma < 1) return TANDEM_ERR_INVALID_ARG;
     if (c->batch == 0) return TANDEM_ERR_STATE;
     TRY(capacity_for(c, 0, gamma));
     reset_call_kernel<<<1, 256, 0, c->stream>>>(c->st, c->batch);
@@ -1297,7 +1308,8 @@ extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t
         }
         for (int b = 0; b < B; ++b) {
             if (result->drafts) for (int i = 0; i < gamma; ++i) result->drafts[b * gamma + i] = d[(size_t)b * GL + i];
-            if (result->targets) for (int i = 0; i <= gamma; ++i) result->targets[b * (gamma + 1) + i] = t[(size_t)b * (GL + 1) + i];
+            if (result->targets) for (int i = 0; i <= gamma; ++i)   // no predictions of the large model in a representation-only round
+                result->targets[b * (gamma + 1) + i] = accept_mode == TANDEM_ACCEPT_REPRESENTATION_ONLY ? -1 : t[(size_t)b * (GL + 1) + i];
             if (result->accept_len) result->accept_len[b] = acc[b];
             if (result->n_committed) result->n_committed[b] = ncm[b];
         }
@@ -1307,8 +1319,10 @@ extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t
 
 namespace {
 
+// lead_large_step: the call starts with one round of the large model alone over the pending token (a block of one
+// row with projection and output head), which gives the first new token (Figure 2, left).
 tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_new, int mode, uint64_t seed,
-                           int32_t* out_ids, int32_t* out_lens, tandem_stats* stats) {
+                           int32_t* out_ids, int32_t* out_lens, tandem_stats* stats, bool lead_large_step = false) {
     if (!out_ids || max_new < 1) return TANDEM_ERR_INVALID_ARG;
     if (c->batch == 0) return TANDEM_ERR_STATE;
     if (max_new > c->cfg.max_seq) return TANDEM_ERR_CAPACITY;
@@ -1324,7 +1338,9 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
     const int DEPTH = 3;
     const int kind = speculative ? 0 : 1;
     const int64_t ticket0 = c->ticket;
-    const int min_iters = (max_new + gamma) / (gamma + 1);
+    const int per_iter = mode == TANDEM_ACCEPT_REPRESENTATION_ONLY ? gamma : gamma + 1;   // most tokens one iteration can emit
+    const int lead = lead_large_step ? 1 : 0;
+    const int min_iters = lead + (max_new - lead + per_iter - 1) / per_iter;
     const int n_known0 = c->n_ub;
     int64_t enq = 0, seen = 0;   // iterations of this call enqueued / observed
     int n_known = n_known0;      // max_b n_b after the last observed iteration
@@ -1345,7 +1361,8 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
         if (finished) break;
         if (enq > (int64_t)max_new + DEPTH + 1) return TANDEM_ERR_STATE;   // every live iteration emits a token
         c->n_ub = std::min<long long>((long long)n_known + (enq - seen) * (gamma + 1), (long long)n_known0 + max_new);
-        TRY(launch_iteration(*c, kind, gamma, mode, seed, max_new));
+        if (lead && enq == 0) TRY(launch_iteration(*c, 0, 0, TANDEM_ACCEPT_NATURAL, 0ull, max_new));
+        else TRY(launch_iteration(*c, kind, gamma, mode, seed, max_new));
         ++enq;
     }
     int32_t* cnt = c->pinned;   // staging is idle outside prefill
@@ -1370,7 +1387,7 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
         memset(stats, 0, sizeof(*stats));
         stats->iterations = iters;
         stats->large_runs = iters;
-        stats->small_runs = speculative ? iters * gamma : 0;
+        stats->small_runs = speculative ? std::max<int64_t>(0, iters - lead) * gamma : 0;
         stats->emitted = (int64_t)B * max_new;
         for (int i = 0; i <= TANDEM_GAMMA_LIMIT; ++i) stats->accept_hist[i] = (int64_t)hist[i];
         stats->kernel_launches = c->launches - launches0;
@@ -1383,8 +1400,24 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
 extern "C" tandem_status tandem_speculative_generate(tandem_ctx* c, int32_t gamma, int32_t max_new_tokens, int32_t accept_mode,
                                                      uint64_t mode_seed, int32_t* out_ids, int32_t* out_lens, tandem_stats* stats) {
     TRY(begin_call(c));
-    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 2) return TANDEM_ERR_INVALID_ARG;
+    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 3) return TANDEM_ERR_INVALID_ARG;
+    if (accept_mode == TANDEM_ACCEPT_REPRESENTATION_ONLY && gamma < 1) return TANDEM_ERR_INVALID_ARG;
     return run_generate(c, true, gamma, max_new_tokens, accept_mode, mode_seed, out_ids, out_lens, stats);
+}
+
+extern "C" tandem_status tandem_standalone_generate(tandem_ctx* c, int32_t gamma, int32_t variant, int32_t max_new_tokens,
+                                                    int32_t* out_ids, int32_t* out_lens, tandem_stats* stats) {
+    TRY(begin_call(c));
+    if (gamma < 1 || gamma > c->cfg.gamma_max) return TANDEM_ERR_INVALID_ARG;
+    switch (variant) {
+        case TANDEM_STANDALONE_FREE_TOKEN:
+            return run_generate(c, true, gamma, max_new_tokens, TANDEM_ACCEPT_ALL, 0ull, out_ids, out_lens, stats);
+        case TANDEM_STANDALONE_REPRESENTATION_ONLY:
+            return run_generate(c, true, gamma, max_new_tokens, TANDEM_ACCEPT_REPRESENTATION_ONLY, 0ull, out_ids, out_lens, stats);
+        case TANDEM_STANDALONE_FREE_TOKEN_FULL_PROMPT:
+            return run_generate(c, true, gamma, max_new_tokens, TANDEM_ACCEPT_ALL, 0ull, out_ids, out_lens, stats, true);
+        default: return TANDEM_ERR_INVALID_ARG;
+    }
 }
 
 extern "C" tandem_status tandem_large_greedy_generate(tandem_ctx* c, int32_t max_new_tokens, int32_t* out_ids, int32_t* out_lens,

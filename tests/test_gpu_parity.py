@@ -151,6 +151,66 @@ def test_fp32_self_tandem_accepts_every_draft():
 
 
 # ------------------------------------------------------------------------------------------------
+# stand-alone Tandem (Section 3 "Inference"; Figures 2 and 3)
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kind,gamma,new", [(synth.FF_TANDEM_LINEAR, 2, 13), (synth.FF_TANDEM_MLP, 3, 10),
+                                            (synth.FF_TANDEM_LINEAR, 1, 5), (synth.FF_TANDEM_MLP, 5, 17)])
+def test_fp32_standalone_variants_match_oracle_bit_exact(kind, gamma, new):
+    """All three stand-alone variants on a ragged batch, token for token, with the run counts of each."""
+    shape = gpu_toy_shape(kind=kind, hidden=40 if kind else 0, layer_map=(1, 3))
+    w = toy_weights(shape, seed=60 + gamma)
+    prompts = prompts_for(shape, [1, 6, 131, 17], seed=gamma)
+    t = binding.Tandem(shape, w, max_batch=4, max_seq=200, gamma_max=gamma)
+    for variant in (binding.STANDALONE_FREE_TOKEN, binding.STANDALONE_REPRESENTATION_ONLY,
+                    binding.STANDALONE_FREE_TOKEN_FULL_PROMPT):
+        want, runs = [], []
+        for p in prompts:
+            o = O.TandemOracle(shape, w)
+            if variant == binding.STANDALONE_FREE_TOKEN:
+                want.append(o.generate(p, gamma, new, mode=O.ACCEPT_ALL)[0])
+            elif variant == binding.STANDALONE_REPRESENTATION_ONLY:
+                want.append(o.generate_representation_only(p, gamma, new))
+            else:
+                want.append(o.generate_free_token_full_prompt(p, gamma, new))
+            runs.append((o.n_large_runs, o.n_small_runs))
+        t.tandem_prefill(prompts)
+        got, lens, stats = t.tandem_standalone_generate(gamma, variant, new)
+        assert got.tolist() == want, variant
+        assert lens.tolist() == [new] * 4
+        assert stats["large_runs"] == max(r[0] for r in runs) and stats["small_runs"] == max(r[1] for r in runs)
+    t.close()
+
+
+def test_fp32_representation_only_steps_match_oracle():
+    """Round by round: drafts and committed counts bit-exact, small logits and both caches within 1e-4."""
+    shape = gpu_toy_shape(kind=synth.FF_TANDEM_LINEAR, layer_map=(1, 3))
+    w = toy_weights(shape, seed=66)
+    prompts = prompts_for(shape, [3, 129], seed=5)
+    t = binding.Tandem(shape, w, max_batch=2, max_seq=200, gamma_max=4)
+    t.tandem_prefill(prompts)
+    oracles = [O.TandemOracle(shape, w) for _ in prompts]
+    for o, p in zip(oracles, prompts):
+        o.prefill(p)
+    for it in range(4):
+        res = t.tandem_block_step(4, binding.ACCEPT_REPRESENTATION_ONLY)
+        s_logits = t.tandem_debug_read(binding.READ_SMALL_LOGITS, 4)
+        for b, o in enumerate(oracles):
+            r = o.step_representation_only(4)
+            assert res["drafts"][b].tolist() == r["drafts"] and res["accept_len"][b] == 4
+            assert res["n_committed"][b] == r["n_committed"] and (res["targets"][b] == -1).all()
+            for s in range(4):
+                assert np.abs(s_logits[s, b] - r["small_logits"][s]).max() < TOL_FP32
+    for b, o in enumerate(oracles):
+        for layer in range(shape.small.n_layers):
+            k = t.tandem_debug_read(binding.READ_SMALL_K, layer=layer, seq=b)
+            assert k.shape[0] == o.derived.length() and np.abs(k - np.stack(o.derived.k[layer])).max() < TOL_FP32
+        k = t.tandem_debug_read(binding.READ_LARGE_K, layer=1, seq=b)
+        assert np.abs(k - np.stack(o.large_cache.k[1])).max() < TOL_FP32
+    t.close()
+
+
+# ------------------------------------------------------------------------------------------------
 # bf16 mode
 # ------------------------------------------------------------------------------------------------
 
@@ -366,6 +426,48 @@ def test_bf16_replay_with_kept_drafts(gamma, mode, large, small):
                             mode=mode, mode_seed=4242, accepts=accepts, check_kv=True)
     assert flips <= 8
     assert max(accepts) == gamma and (mode == 1 or min(accepts) < gamma)     # the hash really gives ragged lengths
+
+
+@pytest.mark.parametrize("gamma,large,small", [(3, (3, 128, 4, 256), (2, 64, 2, 136)), (4, (2, 256, 4, 512), (2, 128, 2, 256)),
+                                               (2, (2, 256, 2, 512), (2, 128, 1, 256))])
+def test_bf16_representation_only_replay(gamma, large, small):
+    """Stand-alone Tandem without the free token on the tensor-core path: the checker is fed the GPU's tokens; small
+    logits of every round within tolerance, differing choices only at near-ties, caches at the end."""
+    shape = gpu_toy_shape(dtype=synth.DTYPE_BF16, layer_map=(1, 2), large=large, small=small)
+    w = _bf16_weights(shape, seed=90 + gamma, std=0.05)
+    prompts = prompts_for(shape, [11, 1, 140], seed=31)
+    t = binding.Tandem(shape, w, max_batch=3, max_seq=shape.large.max_pos, gamma_max=gamma)
+    t.tandem_prefill(prompts)
+    oracles = [O.TandemOracle(shape, w) for _ in prompts]
+    for o, p in zip(oracles, prompts):
+        o.prefill(p)
+    flips = 0
+    for it in range(6):
+        res = t.tandem_block_step(gamma, binding.ACCEPT_REPRESENTATION_ONLY)
+        s_logits = t.tandem_debug_read(binding.READ_SMALL_LOGITS, gamma)
+        for b, o in enumerate(oracles):
+            g_drafts = res["drafts"][b].tolist()
+            r = o.step_representation_only(gamma, forced=g_drafts)
+            for s in range(gamma):
+                assert np.abs(s_logits[s, b] - r["small_logits"][s]).max() < TOL_BF16
+                if r["drafts"][s] != g_drafts[s]:
+                    assert _near_tie(r["small_logits"][s], g_drafts[s], 2 * TOL_BF16)
+                    flips += 1
+            assert res["n_committed"][b] == r["n_committed"] and res["accept_len"][b] == gamma
+    assert flips <= 6
+    for b, o in enumerate(oracles):
+        for layer in range(shape.small.n_layers):
+            k = t.tandem_debug_read(binding.READ_SMALL_K, layer=layer, seq=b)
+            want = np.stack(o.derived.k[layer])
+            assert k.shape == want.shape and (np.abs(k - want) <= TOL_BF16 * np.maximum(1.0, np.abs(want))).all()
+    # the whole response through the generate call equals the step-by-step rounds on the GPU
+    t.tandem_prefill(prompts)
+    a, _, st = t.tandem_standalone_generate(gamma, binding.STANDALONE_REPRESENTATION_ONLY, 3 * gamma + 1)
+    t.tandem_prefill(prompts)
+    steps = [t.tandem_block_step(gamma, binding.ACCEPT_REPRESENTATION_ONLY)["drafts"] for _ in range(4)]
+    b_ = np.concatenate(steps, axis=1)[:, : 3 * gamma + 1]
+    assert a.tolist() == b_.tolist() and st["large_runs"] == 4 and st["small_runs"] == 4 * gamma
+    t.close()
 
 
 def test_bf16_self_tandem_accepts_drafts_naturally():
