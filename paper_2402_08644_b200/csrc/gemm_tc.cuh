@@ -237,11 +237,22 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     if (ln_regs) {
         // short LayerNorm rows: one pass over x.  Lane L holds the row's float4 number L + 32u in
         // t[u], i.e. K-block 2u + (L >= 16), 16-byte chunk (L & 15) / 2, half L & 1.
+        // A warp's rows are fetched one row ahead, so the loads of its rows overlap.
+        float4 tn[8];
+        if (warp < a.rows) {
+            const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)warp * a.ldx);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) tn[u] = (lane + 32 * u < K4) ? __ldcg(xr + lane + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         for (int r = warp; r < a.rows; r += 4) {
-            const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)r * a.ldx);
             float4 t[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) t[u] = (lane + 32 * u < K4) ? __ldcg(xr + lane + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int u = 0; u < 8; ++u) t[u] = tn[u];
+            if (r + 4 < a.rows) {
+                const float4* xr = reinterpret_cast<const float4*>(static_cast<const float*>(a.x) + (size_t)(r + 4) * a.ldx);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) tn[u] = (lane + 32 * u < K4) ? __ldcg(xr + lane + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
             float s = 0.f;
 #pragma unroll
             for (int u = 0; u < 8; ++u) s += (t[u].x + t[u].y) + (t[u].z + t[u].w);
