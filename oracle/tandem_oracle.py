@@ -27,6 +27,9 @@ Readings taken where the paper is silent or inconsistent:
       the previous tokens").
   R2  x^(l) is the residual stream after l large layers; l = 0 is the embedding output.
   R3  y_hat replaces y as the *layer input* at that position: K = LN1_S(y_hat) Wk^T, V likewise.
+  R17 Multi-query / grouped-query attention ("whether the attention is multi-head or multi-query", Section 3):
+      n_kv_heads key/value heads of the same head size; query head h reads key/value head
+      h // (n_heads / n_kv_heads); W_k and W_v map d_model to n_kv_heads * d_head.  Either model, independently.
   R4  Pre-LayerNorm blocks (gain and bias, eps 1e-5, biased variance), exact-erf GELU, no linear
       biases, learned absolute position embeddings, untied output head.
   R6  FF_Tandem MLP variant: hidden width given by the shape, GELU, no biases.
@@ -91,16 +94,22 @@ def softmax(s: np.ndarray) -> np.ndarray:
     return e / e.sum(axis=-1, keepdims=True)
 
 
-def attend(q: np.ndarray, K: np.ndarray, V: np.ndarray, n_heads: int) -> np.ndarray:
-    """Multi-head attention of ONE query q[d] over a context K[n][d], V[n][d]: per head,
-    softmax(q_h . k_h / sqrt(d_h)) weighted sum of v_h; heads concatenated."""
+def attend(q: np.ndarray, K: np.ndarray, V: np.ndarray, n_heads: int, n_kv_heads: Optional[int] = None) -> np.ndarray:
+    """Multi-head attention of ONE query q[d] over a context K[n][d_kv], V[n][d_kv]: per head,
+    softmax(q_h . k_g / sqrt(d_h)) weighted sum of v_g; heads concatenated.  With fewer key/value heads than
+    query heads (multi-query / grouped-query attention, which Section 3 allows for either model), query head h
+    reads key/value head g = h // (n_heads / n_kv_heads); by default g = h and d_kv = d."""
     d = q.shape[0]
     dh = d // n_heads
+    kv = n_heads if n_kv_heads is None else n_kv_heads
+    group = n_heads // kv
     out = np.empty(d, dtype=q.dtype)
     for h in range(n_heads):
         sl = slice(h * dh, (h + 1) * dh)
-        scores = K[:, sl] @ q[sl] / math.sqrt(dh)
-        out[sl] = softmax(scores) @ V[:, sl]
+        g = h // group
+        sg = slice(g * dh, (g + 1) * dh)
+        scores = K[:, sg] @ q[sl] / math.sqrt(dh)
+        out[sl] = softmax(scores) @ V[:, sg]
     return out
 
 
@@ -132,9 +141,10 @@ class Decoder:
     """Weights of one decoder (prefix 'L' or 'S' in the weight dict), cast to the compute dtype."""
 
     def __init__(self, weights: Dict[str, np.ndarray], prefix: str, n_layers: int, n_heads: int,
-                 dtype=np.float64):
+                 dtype=np.float64, n_kv_heads: Optional[int] = None):
         g = lambda name: np.asarray(weights[f"{prefix}.{name}"], dtype=dtype)
         self.n_layers, self.n_heads = n_layers, n_heads
+        self.n_kv_heads = n_heads if not n_kv_heads else n_kv_heads
         self.emb, self.pos = g("emb"), g("pos")
         self.layers = []
         for l in range(n_layers):
@@ -188,7 +198,7 @@ def decoder_full_forward(dec: Decoder, ids: Sequence[int]) -> Tuple[List[np.ndar
         p = dec.layers[l]
         a = layer_norm(h, p["ln1_g"], p["ln1_b"])
         q, k, v = a @ p["wq"].T, a @ p["wk"].T, a @ p["wv"].T
-        o = np.stack([attend(q[i], k[: i + 1], v[: i + 1], dec.n_heads) for i in range(S)]) if S else h
+        o = np.stack([attend(q[i], k[: i + 1], v[: i + 1], dec.n_heads, dec.n_kv_heads) for i in range(S)]) if S else h
         h = h + o @ p["wo"].T
         h = dec.feed_forward(l, h)
         reps.append(h)
@@ -215,7 +225,7 @@ def tandem_small_full_forward(small: Decoder, proj: TandemProjection, layer_map:
         a_ctx = layer_norm(ctx, p_["ln1_g"], p_["ln1_b"])
         k, v = a_ctx @ p_["wk"].T, a_ctx @ p_["wv"].T
         q = layer_norm(y, p_["ln1_g"], p_["ln1_b"]) @ p_["wq"].T
-        o = np.stack([attend(q[r], k[: p + 1], v[: p + 1], small.n_heads) for r, p in enumerate(own)])
+        o = np.stack([attend(q[r], k[: p + 1], v[: p + 1], small.n_heads, small.n_kv_heads) for r, p in enumerate(own)])
         y = y + o @ p_["wo"].T
         y = small.feed_forward(j, y)
     return small.logits(y)
@@ -262,7 +272,7 @@ def large_block_pass(dec: Decoder, cache: KVCache, tokens: Sequence[int], start:
         for r in range(R):
             cache.append(l, k[r], v[r])
         K, V = np.stack(cache.k[l]), np.stack(cache.v[l])
-        o = np.stack([attend(q[r], K[: start + r + 1], V[: start + r + 1], dec.n_heads) for r in range(R)])
+        o = np.stack([attend(q[r], K[: start + r + 1], V[: start + r + 1], dec.n_heads, dec.n_kv_heads) for r in range(R)])
         h = h + o @ p["wo"].T
         h = dec.feed_forward(l, h)
         reps.append(h)
@@ -274,8 +284,8 @@ class TandemOracle:
 
     def __init__(self, shape, weights: Dict[str, np.ndarray], dtype=np.float64):
         self.shape = shape
-        self.large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
-        self.small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype)
+        self.large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype, shape.large.kv_heads)
+        self.small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype, shape.small.kv_heads)
         self.proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
         self.layer_map = list(shape.layer_map)
         self.tokens: List[int] = []           # committed tokens c[0..n-1]; c[n-1] is pending
@@ -365,7 +375,7 @@ class TandemOracle:
             K = np.stack(self.derived.k[j] + self.own.k[j])
             V = np.stack(self.derived.v[j] + self.own.v[j])
             assert K.shape[0] == index + 1
-            y = y + attend(a @ p["wq"].T, K, V, sm.n_heads) @ p["wo"].T
+            y = y + attend(a @ p["wq"].T, K, V, sm.n_heads, sm.n_kv_heads) @ p["wo"].T
             y = sm.feed_forward(j, y)
         self.n_small_runs += 1
         self.schedule.append(("S", [index]))
@@ -452,7 +462,7 @@ def plain_greedy(shape, weights: Dict[str, np.ndarray], prompt: Sequence[int], m
                  dtype=np.float64) -> List[int]:
     """Greedy decoding of the large model alone by full recompute: tok[t] = argmax M_L(prompt ++ tok[<t]).
     This is the definition that SPEED's output must equal (abstract; Section 3.1)."""
-    dec = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
+    dec = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype, shape.large.kv_heads)
     seq = [int(t) for t in prompt]
     for _ in range(max_new):
         _, logits = decoder_full_forward(dec, seq)
@@ -464,7 +474,7 @@ def plain_greedy_cached(shape, weights: Dict[str, np.ndarray], prompt: Sequence[
                         dtype=np.float64) -> List[int]:
     """The same tokens with a key/value cache and one-row block passes (used where full recompute
     is too slow; pinned against `plain_greedy` on small cases)."""
-    dec = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
+    dec = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype, shape.large.kv_heads)
     cache = KVCache(dec.n_layers)
     seq = [int(t) for t in prompt]
     if len(seq) > 1:
@@ -486,8 +496,8 @@ def standalone_tandem_free_token(shape, weights: Dict[str, np.ndarray], prompt: 
     Each round: the small model, reading the large model's representations of everything but the
     last token, appends gamma tokens one at a time; then the large model reads the whole sequence
     and appends its own prediction of the next token."""
-    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
-    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype)
+    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype, shape.large.kv_heads)
+    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype, shape.small.kv_heads)
     proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
     seq = [int(t) for t in prompt]
     P = len(seq)
@@ -510,8 +520,8 @@ def standalone_tandem_representation_only(shape, weights: Dict[str, np.ndarray],
     Each round: the large model's representations of everything but the last token are recomputed from
     scratch; the small model, attending them, appends gamma tokens one at a time.  The large model never
     predicts a token."""
-    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
-    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype)
+    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype, shape.large.kv_heads)
+    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype, shape.small.kv_heads)
     proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
     seq = [int(t) for t in prompt]
     P = len(seq)
@@ -529,8 +539,8 @@ def standalone_tandem_free_token_full_prompt(shape, weights: Dict[str, np.ndarra
     """Figure 2 as drawn, by brute force: the large model reads the whole sequence and appends its prediction;
     the small model, attending the large model's representations of everything before that token, appends
     gamma tokens; repeat."""
-    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype)
-    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype)
+    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype, shape.large.kv_heads)
+    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype, shape.small.kv_heads)
     proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
     seq = [int(t) for t in prompt]
     P = len(seq)

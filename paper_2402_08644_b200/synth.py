@@ -33,10 +33,20 @@ class ModelDims:
     d_ff: int
     vocab: int
     max_pos: int
+    n_kv_heads: int = 0     # key/value heads (multi-query / grouped-query attention); 0 = n_heads (multi-head)
 
     @property
     def d_head(self) -> int:
         return self.d_model // self.n_heads
+
+    @property
+    def kv_heads(self) -> int:
+        return self.n_kv_heads if self.n_kv_heads > 0 else self.n_heads
+
+    @property
+    def d_kv(self) -> int:
+        """Width of a position's keys (or values): kv_heads * d_head."""
+        return self.kv_heads * self.d_head
 
 
 @dataclass(frozen=True)
@@ -123,7 +133,7 @@ def weight_shape(shape: TandemShape, name: str) -> tuple:
     d, f, v = dims.d_model, dims.d_ff, dims.vocab
     leaf = parts[-1]
     table = {"emb": (v, d), "pos": (dims.max_pos, d), "w_out": (v, d),
-             "wq": (d, d), "wk": (d, d), "wv": (d, d), "wo": (d, d), "w1": (f, d), "w2": (d, f)}
+             "wq": (d, d), "wk": (dims.d_kv, d), "wv": (dims.d_kv, d), "wo": (d, d), "w1": (f, d), "w2": (d, f)}
     if leaf in table:
         return table[leaf]
     return (d,)   # LayerNorm gain / bias

@@ -321,3 +321,21 @@ def test_full_prompt_free_token_variant_matches_brute_force_and_figure2():
     assert b.step(0)["emitted"] == [first] and a.tokens == b.tokens
     for layer in range(shape.small.n_layers):
         assert np.allclose(np.stack(a.derived.k[layer]), np.stack(b.derived.k[layer]), atol=1e-10)
+
+
+def test_grouped_query_models_keep_every_invariant():
+    """Multi-query large model and grouped-query small model (Section 3): SPEED == plain greedy, block == single
+    passes, cached == brute force, and keys/values have the narrower width."""
+    L = synth.ModelDims(3, 32, 4, 64, 50, 64, n_kv_heads=1)
+    S = synth.ModelDims(2, 24, 6, 48, 50, 64, n_kv_heads=2)
+    shape = synth.make_shape(L, S, synth.FF_TANDEM_LINEAR, 0, (1, 3), synth.DTYPE_FP32)
+    w = toy_weights(shape, seed=12)
+    assert w["L.0.wk"].shape == (8, 32) and w["S.1.wv"].shape == (8, 24) and w["L.0.wq"].shape == (32, 32)
+    prompt = _prompt(shape, 6, seed=4)
+    o = O.TandemOracle(shape, w)
+    got, accepts = o.generate(prompt, 3, 9)
+    assert got == O.plain_greedy(shape, w, prompt, 9)
+    assert o.large_cache.k[0][0].shape == (8,) and o.derived.k[0][0].shape == (8,)
+    assert O.TandemOracle(shape, w).generate(prompt, 2, 7, mode=O.ACCEPT_ALL)[0] == O.standalone_tandem_free_token(shape, w, prompt, 2, 7)
+    assert O.TandemOracle(shape, w).generate_representation_only(prompt, 2, 6) == \
+        O.standalone_tandem_representation_only(shape, w, prompt, 2, 6)

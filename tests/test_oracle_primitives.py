@@ -187,3 +187,26 @@ def test_ff_tandem_linear_is_one_matrix_product():
     x = np.random.default_rng(9).normal(size=(4, 24))
     want = torch.nn.functional.linear(torch.tensor(x), torch.tensor(w["T.0.w_t"])).numpy()
     assert np.allclose(proj(0, x), want, atol=1e-13)
+
+
+@pytest.mark.parametrize("n_heads,n_kv_heads", [(8, 1), (8, 2), (6, 3), (4, 4)])
+def test_attend_grouped_query_matches_library(n_heads, n_kv_heads):
+    """Multi-query / grouped-query attention against torch's scaled_dot_product_attention with enable_gqa, and
+    against multi-head attention over keys/values repeated per group (the definition)."""
+    rng = np.random.default_rng(n_heads * 10 + n_kv_heads)
+    dh, n = 5, 11
+    q = rng.normal(size=n_heads * dh)
+    K = rng.normal(size=(n, n_kv_heads * dh))
+    V = rng.normal(size=(n, n_kv_heads * dh))
+    got = O.attend(q, K, V, n_heads, n_kv_heads)
+    tq = torch.tensor(q).reshape(1, n_heads, 1, dh)
+    tk = torch.tensor(K).reshape(n, n_kv_heads, dh).permute(1, 0, 2).unsqueeze(0)
+    tv = torch.tensor(V).reshape(n, n_kv_heads, dh).permute(1, 0, 2).unsqueeze(0)
+    want = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, enable_gqa=True).reshape(-1).numpy()
+    assert np.allclose(got, want, atol=1e-12)
+    rep = n_heads // n_kv_heads
+    K_full = K.reshape(n, n_kv_heads, dh).repeat(rep, axis=1).reshape(n, n_heads * dh)
+    V_full = V.reshape(n, n_kv_heads, dh).repeat(rep, axis=1).reshape(n, n_heads * dh)
+    assert np.allclose(got, O.attend(q, K_full, V_full, n_heads), atol=1e-13)
+    if 1 < n_kv_heads < n_heads:  # the grouping matters: a rotated head-to-group map gives something else
+        assert not np.allclose(got, O.attend(q, np.roll(K_full, dh, axis=1), np.roll(V_full, dh, axis=1), n_heads), atol=1e-3)
