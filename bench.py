@@ -132,11 +132,11 @@ def algorithmic_bytes_per_iteration(shape, B, gamma, T):
     once, plus both KV streams at context length T (bf16)."""
     esz = 2 if shape.dtype == synth.DTYPE_BF16 else 4
     def model(d):
-        return d.n_layers * (4 * d.d_model ** 2 + 2 * d.d_model * d.d_ff) + d.d_model * d.vocab
+        return d.n_layers * (2 * d.d_model ** 2 + 2 * d.d_model * d.d_kv + 2 * d.d_model * d.d_ff) + d.d_model * d.vocab
     L, S = shape.large, shape.small
-    proj = S.n_layers * (S.d_model * L.d_model + 2 * S.d_model ** 2) if shape.ff_tandem_kind == 0 else \
-        S.n_layers * (shape.hidden * L.d_model + S.d_model * shape.hidden + 2 * S.d_model ** 2)
-    kv = B * T * (L.n_layers * 2 * L.d_model + gamma * S.n_layers * 2 * S.d_model)
+    proj = S.n_layers * (S.d_model * L.d_model + 2 * S.d_model * S.d_kv) if shape.ff_tandem_kind == 0 else \
+        S.n_layers * (shape.hidden * L.d_model + S.d_model * shape.hidden + 2 * S.d_model * S.d_kv)
+    kv = B * T * (L.n_layers * 2 * L.d_kv + gamma * S.n_layers * 2 * S.d_kv)
     return esz * (model(L) + gamma * model(S) + proj + kv)
 
 

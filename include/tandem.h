@@ -78,6 +78,10 @@ enum { TANDEM_STANDALONE_FREE_TOKEN = 0, TANDEM_STANDALONE_REPRESENTATION_ONLY =
 
 typedef struct {
     int32_t n_layers, d_model, n_heads, d_ff, vocab, max_pos;
+    int32_t n_kv_heads; /* key/value heads: multi-query (1) or grouped-query attention, which Section 3 allows for
+                           either model.  0 = n_heads (multi-head).  Must divide n_heads; query head h reads key/value
+                           head h / (n_heads / n_kv_heads); wk and wv are then [n_kv_heads * d_head][d_model] and a
+                           cached position holds n_kv_heads * d_head keys (values). */
 } tandem_dims;
 
 typedef struct {
@@ -98,7 +102,7 @@ typedef struct {
 
 /* DEVICE pointers in this fixed order (n_ptrs must match):
  *   for model in (large, small):  emb[V][d], pos[max_pos][d],
- *       per layer: ln1_g[d], ln1_b[d], wq[d][d], wk[d][d], wv[d][d], wo[d][d], ln2_g[d], ln2_b[d],
+ *       per layer: ln1_g[d], ln1_b[d], wq[d][d], wk[d_kv][d], wv[d_kv][d], wo[d][d], ln2_g[d], ln2_b[d],
  *                  w1[d_ff][d], w2[d][d_ff],
  *       lnf_g[d], lnf_b[d], w_out[V][d]
  *   then per small layer j:  linear: w_t[d_S][d_L]      MLP: w_t1[hidden][d_L], w_t2[d_S][hidden]
@@ -198,9 +202,9 @@ TANDEM_API tandem_status tandem_large_greedy_generate(tandem_ctx* ctx, int32_t m
  *   what = 0  large logits      [batch][gamma+1][vocab]              (last verify pass)
  *   what = 1  small logits      [gamma][batch][vocab]                (last draft steps)
  *   what = 2  large hidden      [batch][gamma+1][d_large]            (final residual stream, last verify)
- *   what = 3  large keys        [n][d_large]  for (layer, seq), n = positions M_L has processed
+ *   what = 3  large keys        [n][d_kv_large]  for (layer, seq), n = positions M_L has processed
  *   what = 4  large values      same
- *   what = 5  small keys        [n][d_small]  for (layer, seq): the large-derived region
+ *   what = 5  small keys        [n][d_kv_small]  for (layer, seq): the large-derived region
  *   what = 6  small values      same
  *   what = 7  committed counts  int32 [batch]
  * bytes must equal the size of the selected item. */

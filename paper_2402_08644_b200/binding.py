@@ -44,7 +44,7 @@ class TandemError(RuntimeError):
 
 
 class Dims(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "d_ff", "vocab", "max_pos")]
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "d_ff", "vocab", "max_pos", "n_kv_heads")]
 
 
 class Config(C.Structure):
@@ -125,7 +125,7 @@ def _check(status: int, where: str) -> None:
 
 
 def _dims(d: synth.ModelDims) -> Dims:
-    return Dims(d.n_layers, d.d_model, d.n_heads, d.d_ff, d.vocab, d.max_pos)
+    return Dims(d.n_layers, d.d_model, d.n_heads, d.d_ff, d.vocab, d.max_pos, d.n_kv_heads)
 
 
 def make_config(shape: synth.TandemShape, max_batch: int, max_seq: int, gamma_max: int, device: int = 0,
@@ -279,7 +279,7 @@ class Tandem:
             out = np.zeros(B, np.int32)
         else:
             n = int(self.tandem_debug_read(READ_COMMITTED)[seq]) - 1
-            d = self.shape.large.d_model if what in (READ_LARGE_K, READ_LARGE_V) else self.shape.small.d_model
+            d = self.shape.large.d_kv if what in (READ_LARGE_K, READ_LARGE_V) else self.shape.small.d_kv
             out = np.zeros((n, d), np.float32)
         _check(self.lib.tandem_debug_read(self.ctx, what, layer, seq, out.ctypes.data_as(C.c_void_p), out.nbytes),
                "tandem_debug_read")

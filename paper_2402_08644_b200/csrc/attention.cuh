@@ -35,6 +35,7 @@ struct AttnArgs {
     const int* grp_row0; const int* grp_cnt;   // nullable: then group g = rows g*nq .. g*nq+nq-1
     int nq;
     int n_heads, t_max;
+    int n_kv_heads;                      // key/value heads of the caches; 0 = n_heads.  Query head h reads kv head h / (n_heads / n_kv_heads)
     float* part_ml;                      // split mode: [M][H][n_chunks_max][2]
     float* part_acc;                     //             [M][H][n_chunks_max][DH]
     int n_chunks_max;
@@ -90,8 +91,10 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
 #pragma unroll
     for (int i = 0; i < QPT; ++i) { racc[i] = 0.f; rm[i] = -INFINITY; rl[i] = 0.f; }
 
-    const size_t head_base = ((size_t)b * a.n_heads + h) * a.t_max;
-    const size_t head_base2 = ((size_t)b * a.n_heads + h) * a.t_max2;
+    const int n_kv = a.n_kv_heads > 0 ? a.n_kv_heads : a.n_heads;
+    const int kvh = h / (a.n_heads / n_kv);            // grouped-query attention: several query heads share one key/value head
+    const size_t head_base = ((size_t)b * n_kv + kvh) * a.t_max;
+    const size_t head_base2 = ((size_t)b * n_kv + kvh) * a.t_max2;
     const int split = a.k2 ? a.split : INT_MAX;
     for (int c = c_begin; c < c_end; ++c) {
         const int t0 = c * ATT_CH;
@@ -316,8 +319,10 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     const int pos_last = pos_first + cnt - 1;
     const int n_chunks = pos_last / ATT_CH + 1;
     const int n_mine = rank < n_chunks ? (n_chunks - rank + CL - 1) / CL : 0;
-    const size_t head_base = ((size_t)b * a.n_heads + h) * a.t_max;
-    const size_t head_base2 = ((size_t)b * a.n_heads + h) * a.t_max2;
+    const int n_kv = a.n_kv_heads > 0 ? a.n_kv_heads : a.n_heads;
+    const int kvh = h / (a.n_heads / n_kv);            // grouped-query attention: several query heads share one key/value head
+    const size_t head_base = ((size_t)b * n_kv + kvh) * a.t_max;
+    const size_t head_base2 = ((size_t)b * n_kv + kvh) * a.t_max2;
     const int split = a.k2 ? a.split : INT_MAX;
 
     // this warp's rows of its CTA's it-th chunk into stage it % STAGES.  Lane L moves unit L % TPK of rows

@@ -24,6 +24,7 @@ struct AttnTcArgs {
     const int* row_seq; const int* row_pos;
     const int* grp_row0; const int* grp_cnt;
     int n_heads, t_max;
+    int n_kv_heads;                       // key/value heads of the cache (<= n_heads, divides it)
     float scale;
     int* err_flag;
 };
@@ -80,7 +81,7 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
     const int pos_first = a.row_pos[row0];
     const int pos_last = pos_first + cnt - 1;
     const int n_chunks = pos_last / 128 + 1;
-    const int kv_row0 = (b * a.n_heads + h) * a.t_max;     // row of position 0 in the cache's 2-D view
+    const int kv_row0 = (b * a.n_kv_heads + h / (a.n_heads / a.n_kv_heads)) * a.t_max;     // row of position 0 of this head's key/value head in the cache's 2-D view
 
     if (warp == 5) {
         if (lane == 0) {

@@ -21,21 +21,24 @@ struct EpiArgs {
     void* vcache;         //           this layer's values
     const int* row_seq;   // [M] sequence of each row
     const int* row_pos;   // [M] absolute position of each row
-    int n_heads, d_head, t_max;
-    int seg;              // columns per segment (= d_model) for QKV / KV
+    int n_heads, d_head, t_max;   // n_heads: key/value heads of the cache
+    int seg0;             // QKV / KV: columns of the first segment (QKV: the queries, d_model; KV: the keys)
+    int seg;              //           columns of every further segment (keys / values: kv heads * d_head)
     void* snap;           // EPI_RESID on the tensor-core decode path: optional fp32 copy of the new values [M][snap_ld]
     int snap_ld;
 };
 
-struct WSegs {            // up to three weight matrices stacked along N, each [seg_rows][K]
+struct WSegs {            // up to three weight matrices stacked along N: [seg_rows0][K], then [seg_rows][K] each
     const void* w[3];
+    int seg_rows0;
     int seg_rows;
 };
 
 template <typename T>
 __device__ __forceinline__ const T* weight_row(const WSegs& ws, int n, int K) {
-    const int s = n / ws.seg_rows;
-    return static_cast<const T*>(ws.w[s]) + (size_t)(n - s * ws.seg_rows) * K;
+    if (n < ws.seg_rows0) return static_cast<const T*>(ws.w[0]) + (size_t)n * K;
+    const int r = n - ws.seg_rows0, s = r / ws.seg_rows;
+    return static_cast<const T*>(ws.w[1 + s]) + (size_t)(r - s * ws.seg_rows) * K;
 }
 
 template <typename T, int EPI>
@@ -50,8 +53,8 @@ __device__ __forceinline__ void epilogue(const EpiArgs& e, int m, int n, float v
         float* p = static_cast<float*>(e.out) + (size_t)m * e.ldo + n;
         *p = *p + v;
     } else {
-        int s = n / e.seg;
-        const int c = n - s * e.seg;
+        int s = 0, c = n;
+        if (n >= e.seg0) { s = 1 + (n - e.seg0) / e.seg; c = (n - e.seg0) - (s - 1) * e.seg; }
         if (EPI == EPI_QKV) {
             if (s == 0) {
                 static_cast<T*>(e.out)[(size_t)m * e.ldo + c] = from_float<T>(v);

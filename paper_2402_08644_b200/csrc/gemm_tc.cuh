@@ -42,7 +42,8 @@ struct TcDecodeArgs {
     const float* ln_g;      // PRO_LN: LayerNorm gain / bias [K]
     const float* ln_b;
     int rows, K, N;         // N = output features over all segments
-    int seg_rows;           // output features per weight segment (one tensor map each)
+    int seg_rows0, tiles0;  // output features and tiles of the first weight segment (one tensor map per segment)
+    int seg_rows;           // output features of every further segment
     int tiles_per_seg;      // ceil(seg_rows / 128)
     int splits;             // K-slices per tile: 1, 2, 4 or 8 = the cluster size; grid = tiles * splits
     int stream_weights;     // 1: weights are read once per pass and should not stay in L2
@@ -129,8 +130,10 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     const uint32_t poll_limit = a.poll_limit ? a.poll_limit : MBAR_POLL_LIMIT;
     const int unit = blockIdx.x;
     const int tile = unit / S, sp = unit - tile * S;                       // sp = this CTA's rank in its cluster
-    const int seg = tile / a.tiles_per_seg;
-    const int n_local0 = (tile - seg * a.tiles_per_seg) * 128;
+    const int seg = tile < a.tiles0 ? 0 : 1 + (tile - a.tiles0) / a.tiles_per_seg;
+    const int n_local0 = (seg == 0 ? tile : tile - a.tiles0 - (seg - 1) * a.tiles_per_seg) * 128;
+    const int seg_rows = seg == 0 ? a.seg_rows0 : a.seg_rows;               // output features of this tile's segment
+    const int seg_base = seg == 0 ? 0 : a.seg_rows0 + (seg - 1) * a.seg_rows;   // and its first output feature
     const int KB = (a.K + 63) >> 6;
     const int kb_base = KB / S, kb_rem = KB - kb_base * S;
     const int kb0 = sp * kb_base + min(sp, kb_rem);
@@ -231,7 +234,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
         for (int s = 0; s < NB; ++s) {
             if (s >= j_count) break;   // (every loop over rows leaves at the last row: the unrolled rest is never fetched)
-            hres[s] = nl < a.seg_rows ? __ldcg(hp + (size_t)(j_first + s) * a.e.ldo + seg * a.seg_rows + nl) : 0.f;
+            hres[s] = nl < seg_rows ? __ldcg(hp + (size_t)(j_first + s) * a.e.ldo + seg_base + nl) : 0.f;
         }
     }
     if (ln_regs) {
@@ -416,8 +419,8 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         }
     }
     const int n_local = n_local0 + tl;                 // warps 0-3: this thread's output feature
-    const bool valid = n_local < a.seg_rows;
-    const int n = seg * a.seg_rows + n_local;
+    const bool valid = n_local < seg_rows;
+    const int n = seg_base + n_local;
     if (EPI == EPI_ARGMAX) {                            // whole tiles only (S == 1)
         if (warp < 4) {
             float* out = static_cast<float*>(a.e.out);
@@ -515,6 +518,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 
 struct TcTiledArgs {
     int M, K, N;
+    int seg_rows0, tiles0;   // first segment: output features, tiles of BN
     int seg_rows, tiles_per_seg;
     int* err_flag;
     EpiArgs e;
@@ -533,8 +537,8 @@ template <int BN> struct TctCfg {
 
 // Sixteen consecutive output features of one row.  n_local0 is a multiple of 16.
 template <int EPI>
-__device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int seg, int seg_rows, int n_local0, const float (&v)[16]) {
-    const int n0 = seg * seg_rows + n_local0;
+__device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int seg, int seg_base, int seg_rows, int n_local0, const float (&v)[16]) {
+    const int n0 = seg_base + n_local0;
     if (n_local0 + 16 > seg_rows || (e.ldo & 7) || (seg_rows & 7)) {
         for (int i = 0; i < 16; ++i)
             if (n_local0 + i < seg_rows) epilogue<bf16, EPI>(e, m, n0 + i, v[i]);
@@ -593,8 +597,10 @@ gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tm
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t ring0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     const int tile = blockIdx.x;
-    const int seg = tile / a.tiles_per_seg;
-    const int n_local0 = (tile - seg * a.tiles_per_seg) * BN;
+    const int seg = tile < a.tiles0 ? 0 : 1 + (tile - a.tiles0) / a.tiles_per_seg;
+    const int n_local0 = (seg == 0 ? tile : tile - a.tiles0 - (seg - 1) * a.tiles_per_seg) * BN;
+    const int seg_rows = seg == 0 ? a.seg_rows0 : a.seg_rows;
+    const int seg_base = seg == 0 ? 0 : a.seg_rows0 + (seg - 1) * a.seg_rows;
     const int m0 = blockIdx.y * 128;
     const int KB = (a.K + 63) >> 6;
 
@@ -660,7 +666,7 @@ gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tm
         for (int c0 = 0; c0 < BN; c0 += 16) {
             float t[16];
             tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c0, t);   // warp-wide: every lane takes part
-            if (m < a.M && n_local0 + c0 < a.seg_rows) epilogue16<EPI>(a.e, m, seg, a.seg_rows, n_local0 + c0, t);
+            if (m < a.M && n_local0 + c0 < seg_rows) epilogue16<EPI>(a.e, m, seg, seg_base, seg_rows, n_local0 + c0, t);
         }
     }
     tc_fence_before_sync();

@@ -59,9 +59,10 @@ struct Layout {   // byte offsets into the arena
 
 struct Model {
     tandem_dims d;
+    int kv_heads, d_kv;     // key/value heads and the width of a position's keys (kv_heads * d_head)
     int wbase;
     size_t kv_off;          // arena offset of this model's KV cache
-    size_t kv_layer_elems;  // elements per (layer, K or V): B * H * T * dh
+    size_t kv_layer_elems;  // elements per (layer, K or V): B * kv_heads * T * dh
 };
 
 }  // namespace
@@ -156,8 +157,11 @@ int dims_ok(const tandem_dims& d) {
     const int dh = d.d_model / d.n_heads;
     if (dh != 32 && dh != 64 && dh != 128) return 0;
     if (d.d_model % 8 || d.d_ff % 8) return 0;
+    if (d.n_kv_heads < 0 || (d.n_kv_heads > 0 && d.n_heads % d.n_kv_heads)) return 0;
     return 1;
 }
+int kv_heads_of(const tandem_dims& d) { return d.n_kv_heads > 0 ? d.n_kv_heads : d.n_heads; }
+int d_kv_of(const tandem_dims& d) { return kv_heads_of(d) * (d.d_model / d.n_heads); }
 
 tandem_status validate(const tandem_config* c) {
     if (!c || !c->layer_map) return TANDEM_ERR_INVALID_ARG;
@@ -191,8 +195,8 @@ Layout make_layout(const tandem_config& c) {
     const size_t R = L.max_rows, RD = L.dec_rows, V = c.large.vocab;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
-    L.kv_large_layer = B * T * c.large.d_model;
-    L.kv_small_layer = B * T * c.small.d_model;
+    L.kv_large_layer = B * T * d_kv_of(c.large);
+    L.kv_small_layer = B * T * d_kv_of(c.small);
     L.kv_large = take((size_t)c.large.n_layers * 2 * L.kv_large_layer * esz);
     L.kv_small = take((size_t)c.small.n_layers * 2 * L.kv_small_layer * esz);
     L.st_n = take(B * 4); L.st_pending = take(B * 4); L.st_drafts = take(B * GL * 4);
@@ -241,10 +245,11 @@ inline int wi_tail(const Model& m, int k) { return m.wbase + 2 + 10 * m.d.n_laye
 inline int wi_tandem(const tandem_ctx& c, int j, int k) { return c.tbase + (c.cfg.ff_tandem_kind == TANDEM_FF_LINEAR ? j : 2 * j + k); }
 
 // A linear map given by the indices of up to three weight matrices stacked along the output features.
-struct Lin { int i0, i1, i2, seg_rows, K; };
-inline Lin lin1(int i0, int rows, int K) { Lin l = {i0, -1, -1, rows, K}; return l; }
-inline Lin lin3(int i0, int i1, int i2, int rows, int K) { Lin l = {i0, i1, i2, rows, K}; return l; }
-inline int lin_n(const Lin& l) { return (1 + (l.i1 >= 0) + (l.i2 >= 0)) * l.seg_rows; }
+// (the first matrix has seg_rows0 rows, the others seg_rows each: queries next to narrower keys / values)
+struct Lin { int i0, i1, i2, seg_rows0, seg_rows, K; };
+inline Lin lin1(int i0, int rows, int K) { Lin l = {i0, -1, -1, rows, rows, K}; return l; }
+inline Lin lin3(int i0, int i1, int i2, int rows0, int rows, int K) { Lin l = {i0, i1, i2, rows0, rows, K}; return l; }
+inline int lin_n(const Lin& l) { return l.seg_rows0 + ((l.i1 >= 0) + (l.i2 >= 0)) * l.seg_rows; }
 
 template <typename P> P* at(tandem_ctx& c, size_t off) { return reinterpret_cast<P*>(c.arena + off); }
 
@@ -325,23 +330,25 @@ bool make_tmap_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t c
 
 struct TcW {              // up to three weight matrices stacked along the output features
     CUtensorMap tm[3];
-    int n_segs, seg_rows, K;
+    int n_segs, seg_rows0, seg_rows, K;   // rows of the first segment, rows of every further one
 };
+inline int tcw_n(const TcW& w) { return w.seg_rows0 + (w.n_segs - 1) * w.seg_rows; }
 struct TcScratch {
     int* err;                  // where a bounded wait that ran out records its code (nullable)
     unsigned poll_limit = 0;   // 0: the kernels' default
     int withhold_weights = 0;  // test hook, see TcDecodeArgs
 };
 
-TcW tcw(const tandem_ctx& c, int i0, int i1, int i2, int seg_rows, int K) {
+TcW tcw3(const tandem_ctx& c, int i0, int i1, int i2, int seg_rows0, int seg_rows, int K) {
     TcW w;
     w.tm[0] = c.wmap[i0];
     w.tm[1] = c.wmap[i1 >= 0 ? i1 : i0];
     w.tm[2] = c.wmap[i2 >= 0 ? i2 : i0];
     w.n_segs = 1 + (i1 >= 0) + (i2 >= 0);
-    w.seg_rows = seg_rows; w.K = K;
+    w.seg_rows0 = seg_rows0; w.seg_rows = seg_rows; w.K = K;
     return w;
 }
+TcW tcw(const tandem_ctx& c, int i0, int i1, int i2, int seg_rows, int K) { return tcw3(c, i0, i1, i2, seg_rows, seg_rows, K); }
 
 TcScratch tc_scratch(tandem_ctx& c) {
     TcScratch s;
@@ -392,8 +399,9 @@ void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx
     TcDecodeArgs a;
     memset(&a, 0, sizeof(a));
     a.ldx = ldx; a.ln_g = static_cast<const float*>(ln_g); a.ln_b = static_cast<const float*>(ln_b);
-    a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
-    const int tiles = w.n_segs * a.tiles_per_seg, KB = cdiv(w.K, 64);
+    a.K = w.K; a.N = tcw_n(w); a.seg_rows0 = w.seg_rows0; a.tiles0 = cdiv(w.seg_rows0, 128);
+    a.seg_rows = w.seg_rows; a.tiles_per_seg = cdiv(w.seg_rows, 128);
+    const int tiles = a.tiles0 + (w.n_segs - 1) * a.tiles_per_seg, KB = cdiv(w.K, 64);
     // K-slices per tile = cluster size: the smallest power of two that puts tiles * S CTAs at or above one per
     // multiprocessor, at most 8 and at most one per 64-element K-block.  The head GEMM keeps whole tiles.
     int S = 1;
@@ -432,8 +440,9 @@ void launch_tc_tiled_bn(tandem_ctx& c, TcTiledArgs& a, const CUtensorMap& tmx, c
     using C = TctCfg<BN>;
     static std::atomic<unsigned long long> attr_done{0};
     ensure_dyn_smem(gemm_tc_tiled_kernel<EPI, BN>, C::SMEM_BYTES, attr_done);
+    a.tiles0 = cdiv(w.seg_rows0, BN);
     a.tiles_per_seg = cdiv(w.seg_rows, BN);
-    launch_ex(c, false, 1, gemm_tc_tiled_kernel<EPI, BN>, dim3(w.n_segs * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)C::SMEM_BYTES,
+    launch_ex(c, false, 1, gemm_tc_tiled_kernel<EPI, BN>, dim3(a.tiles0 + (w.n_segs - 1) * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)C::SMEM_BYTES,
               a, tmx, w.tm[0], w.tm[1], w.tm[2]);
 }
 
@@ -447,11 +456,11 @@ tandem_status launch_tc_tiled(tandem_ctx& c, const bf16* x, int ldx, int M, cons
     }
     TcTiledArgs a;
     memset(&a, 0, sizeof(a));
-    a.M = M; a.K = w.K; a.N = w.n_segs * w.seg_rows; a.seg_rows = w.seg_rows;
+    a.M = M; a.K = w.K; a.N = tcw_n(w); a.seg_rows0 = w.seg_rows0; a.seg_rows = w.seg_rows;
     a.err_flag = err; a.e = e;
     ProfScope ps(c, PC_GEMM_TC_TILED, 2.0 * M * (double)a.N * w.K);   // flops
     // 256-wide tiles when they still give every SM a tile, else square ones
-    if ((long long)w.n_segs * cdiv(w.seg_rows, 256) * cdiv(M, 128) >= c.n_sms) launch_tc_tiled_bn<EPI, 256>(c, a, tmx, w, M);
+    if ((long long)(cdiv(w.seg_rows0, 256) + (w.n_segs - 1) * cdiv(w.seg_rows, 256)) * cdiv(M, 128) >= c.n_sms) launch_tc_tiled_bn<EPI, 256>(c, a, tmx, w, M);
     else launch_tc_tiled_bn<EPI, 128>(c, a, tmx, w, M);
     return TANDEM_OK;
 }
@@ -461,6 +470,7 @@ WSegs segs_of(const tandem_ctx& c, const Lin& l) {
     s.w[0] = c.w[l.i0];
     s.w[1] = l.i1 >= 0 ? c.w[l.i1] : nullptr;
     s.w[2] = l.i2 >= 0 ? c.w[l.i2] : nullptr;
+    s.seg_rows0 = l.seg_rows0;
     s.seg_rows = l.seg_rows;
     return s;
 }
@@ -478,7 +488,7 @@ void launch_gemm(tandem_ctx& c, bool decode, const T* x, int ldx, int M, const L
         else if (M <= 4) launch_smallm<T, 4, EPI>(c, x, ldx, M, K, ws, N, e);
         else launch_smallm<T, 8, EPI>(c, x, ldx, M, K, ws, N, e);
     } else if (sizeof(T) == 2 && c.tc) {
-        if (launch_tc_tiled<EPI>(c, reinterpret_cast<const bf16*>(x), ldx, M, tcw(c, l.i0, l.i1, l.i2, l.seg_rows, l.K), e,
+        if (launch_tc_tiled<EPI>(c, reinterpret_cast<const bf16*>(x), ldx, M, tcw3(c, l.i0, l.i1, l.i2, l.seg_rows0, l.seg_rows, l.K), e,
                                  c.st.counters + 2) != TANDEM_OK)
             c.setup_failed = true;
     } else {
@@ -567,7 +577,8 @@ EpiArgs epi_cache(tandem_ctx& c, const Model& m, int layer, void* q_out) {
     e.out = q_out; e.ldo = m.d.d_model;
     e.kcache = kv_ptr<T>(c, m, layer, 0); e.vcache = kv_ptr<T>(c, m, layer, 1);
     e.row_seq = at<int>(c, c.lay.row_seq); e.row_pos = at<int>(c, c.lay.row_pos);
-    e.n_heads = m.d.n_heads; e.d_head = m.d.d_model / m.d.n_heads; e.t_max = c.cfg.max_seq; e.seg = m.d.d_model;
+    e.n_heads = m.kv_heads; e.d_head = m.d.d_model / m.d.n_heads; e.t_max = c.cfg.max_seq;
+    e.seg0 = q_out ? m.d.d_model : m.d_kv; e.seg = m.d_kv;   // with queries: [d_model | d_kv | d_kv]; keys / values alone: [d_kv | d_kv]
     return e;
 }
 
@@ -591,7 +602,7 @@ void launch_attn_prompt_tc(tandem_ctx& c, int l, const bf16* q, bf16* o, const R
     memset(&a, 0, sizeof(a));
     a.out = o; a.ldo = d; a.row_seq = at<int>(c, c.lay.row_seq); a.row_pos = at<int>(c, c.lay.row_pos);
     a.grp_row0 = at<int>(c, c.lay.grp_row0); a.grp_cnt = at<int>(c, c.lay.grp_cnt);
-    a.n_heads = H; a.t_max = c.cfg.max_seq; a.scale = 1.0f / sqrtf((float)dh); a.err_flag = c.st.counters + 2;
+    a.n_heads = H; a.n_kv_heads = c.large.kv_heads; a.t_max = c.cfg.max_seq; a.scale = 1.0f / sqrtf((float)dh); a.err_flag = c.st.counters + 2;
     // two MMA groups per (128 queries x 128 keys): 4 * 128 * 128 * dh flops, over the causal half of the prompt
     ProfScope ps(c, PC_ATTN_PROMPT, 0.0);
     if (dh == 64) launch_attn_prompt_tc_dh<64>(c, a, tmq, l, r.groups);
@@ -605,7 +616,7 @@ void attention(tandem_ctx& c, const Model& m, int l, const T* q, T* o, const Row
     aa.q = q; aa.ldq = d; aa.kcache = kv_ptr<T>(c, m, l, 0); aa.vcache = kv_ptr<T>(c, m, l, 1);
     aa.out = o; aa.ldo = d; aa.row_seq = at<int>(c, c.lay.row_seq); aa.row_pos = at<int>(c, c.lay.row_pos);
     if (!r.decode) { aa.grp_row0 = at<int>(c, c.lay.grp_row0); aa.grp_cnt = at<int>(c, c.lay.grp_cnt); }
-    aa.nq = r.nq; aa.n_heads = H; aa.t_max = c.cfg.max_seq;
+    aa.nq = r.nq; aa.n_heads = H; aa.n_kv_heads = m.kv_heads; aa.t_max = c.cfg.max_seq;
     aa.part_ml = at<float>(c, c.lay.part_ml); aa.part_acc = at<float>(c, c.lay.part_acc);
     aa.n_chunks_max = c.lay.n_chunks_max; aa.scale = 1.0f / sqrtf((float)dh);
     aa.merge_counters = at<int>(c, c.lay.attn_counters);
@@ -622,7 +633,7 @@ void attention_decode(tandem_ctx& c, const Model& m, int l, const bf16* q, float
     AttnArgs aa; memset(&aa, 0, sizeof(aa));
     aa.q = q; aa.ldq = d; aa.kcache = kv_ptr<bf16>(c, m, l, 0); aa.vcache = kv_ptr<bf16>(c, m, l, 1);
     aa.out = o; aa.ldo = d; aa.out_f32 = 1; aa.row_seq = at<int>(c, c.lay.row_seq); aa.row_pos = at<int>(c, c.lay.row_pos);
-    aa.nq = r.nq; aa.n_heads = H; aa.t_max = c.cfg.max_seq; aa.scale = 1.0f / sqrtf((float)dh);
+    aa.nq = r.nq; aa.n_heads = H; aa.n_kv_heads = m.kv_heads; aa.t_max = c.cfg.max_seq; aa.scale = 1.0f / sqrtf((float)dh);
     launch_attn_decode(c, dh, aa, r.groups, r.kv_positions * 2.0 * d * 2.0);
 }
 
@@ -642,7 +653,7 @@ void project_layer(tandem_ctx& c, int j, const Rows& r) {
         launch_gemm<T, EPI_STORE_F32>(c, r.decode, t1, c.hidden, r.M, lin1(wi_tandem(c, j, 1), dS, c.hidden), epi_plain(yhat, dS));
     }
     launch_layernorm<T>(c, r.M, yhat, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), a_s, dS);
-    launch_gemm<T, EPI_KV>(c, r.decode, a_s, dS, r.M, lin3(wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS),
+    launch_gemm<T, EPI_KV>(c, r.decode, a_s, dS, r.M, lin3(wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, c.small.d_kv, c.small.d_kv, dS),
                            epi_cache<T>(c, c.small, j, nullptr));
 }
 
@@ -670,7 +681,7 @@ void decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows& r
     T* o = at<T>(c, c.lay.o);
     T* f = at<T>(c, c.lay.f);
     launch_layernorm<T>(c, r.M, h, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), a, d);
-    launch_gemm<T, EPI_QKV>(c, r.decode, a, d, r.M, lin3(wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, d),
+    launch_gemm<T, EPI_QKV>(c, r.decode, a, d, r.M, lin3(wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, m.d_kv, d),
                             epi_cache<T>(c, m, l, q));
     attention<T>(c, m, l, q, o, r);
     launch_gemm<T, EPI_RESID>(c, r.decode, o, d, r.M, lin1(wi_layer(m, l, W_WO), d, d), epi_plain(h, d));
@@ -821,7 +832,7 @@ void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows
     float* f = at<float>(c, c.lay.f32);
     const TcScratch sc = tc_scratch(c);
     tc_ln_gemm<EPI_QKV>(c, h, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), r.M,
-                        tcw(c, wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, d), stream_w, epi_cache<bf16>(c, m, l, q));
+                        tcw3(c, wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, m.d_kv, d), stream_w, epi_cache<bf16>(c, m, l, q));
     attention_decode(c, m, l, q, o, r);
     launch_tc_decode<PRO_F32, EPI_RESID>(c, sc, o, d, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_WO), -1, -1, d, d), stream_w,
                                          epi_plain(h, d));
@@ -878,7 +889,7 @@ void tc_project_forked(tandem_ctx& c, int n_large_layers_done, int slot, const R
                                                      true, epi_plain(yhat, dS));
         }
         tc_ln_gemm<EPI_KV>(c, yhat, w_layer(c, c.small, j, W_LN1G), w_layer(c, c.small, j, W_LN1B), r.M,
-                           tcw(c, wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, dS, dS), true, epi_cache<bf16>(c, c.small, j, nullptr),
+                           tcw(c, wi_layer(c.small, j, W_WK), wi_layer(c.small, j, W_WV), -1, c.small.d_kv, dS), true, epi_cache<bf16>(c, c.small, j, nullptr),
                            nullptr, nullptr, 0, a_j);
     }
     c.stream = main_stream;
@@ -1093,6 +1104,8 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
     c->stream = static_cast<cudaStream_t>(cfg->stream);
     c->esz = cfg->dtype == TANDEM_DTYPE_BF16 ? 2 : 4;
     c->hidden = cfg->ff_tandem_hidden > 0 ? cfg->ff_tandem_hidden : cfg->small.d_model;
+    c->large.kv_heads = kv_heads_of(cfg->large); c->large.d_kv = d_kv_of(cfg->large);
+    c->small.kv_heads = kv_heads_of(cfg->small); c->small.d_kv = d_kv_of(cfg->small);
     c->large.d = cfg->large; c->large.wbase = 0; c->large.kv_off = lay.kv_large; c->large.kv_layer_elems = lay.kv_large_layer;
     c->small.d = cfg->small; c->small.wbase = 5 + 10 * cfg->large.n_layers; c->small.kv_off = lay.kv_small; c->small.kv_layer_elems = lay.kv_small_layer;
     c->tbase = c->small.wbase + 5 + 10 * cfg->small.n_layers;
@@ -1138,7 +1151,7 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
         for (const Model* m : {&c->large, &c->small}) {
             const int d = m->d.d_model, dff = m->d.d_ff;
             for (int l = 0; l < m->d.n_layers; ++l) {
-                add(wi_layer(*m, l, W_WQ), d, d); add(wi_layer(*m, l, W_WK), d, d); add(wi_layer(*m, l, W_WV), d, d);
+                add(wi_layer(*m, l, W_WQ), d, d); add(wi_layer(*m, l, W_WK), m->d_kv, d); add(wi_layer(*m, l, W_WV), m->d_kv, d);
                 add(wi_layer(*m, l, W_WO), d, d); add(wi_layer(*m, l, W_W1), dff, d); add(wi_layer(*m, l, W_W2), d, dff);
             }
             add(wi_tail(*m, 2), m->d.vocab, d);
@@ -1162,7 +1175,7 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
             c->kmap.resize(cfg->large.n_layers);
             c->vmap.resize(cfg->large.n_layers);
             bool okm = true;
-            const uint64_t kv_rows = (uint64_t)cfg->max_batch * cfg->large.n_heads * cfg->max_seq;
+            const uint64_t kv_rows = (uint64_t)cfg->max_batch * c->large.kv_heads * cfg->max_seq;
             for (int l = 0; l < cfg->large.n_layers && okm; ++l)
                 okm = make_tmap_bf16(&c->kmap[l], kv_ptr<bf16>(*c, c->large, l, 0), kv_rows, (uint64_t)dhL, (uint64_t)dhL) &&
                       make_tmap_bf16(&c->vmap[l], kv_ptr<bf16>(*c, c->large, l, 1), kv_rows, (uint64_t)dhL, (uint64_t)dhL);
@@ -1513,7 +1526,7 @@ extern "C" tandem_status tandem_debug_read(tandem_ctx* c, int32_t what, int32_t 
         if (layer < 0 || layer >= m.d.n_layers || seq < 0 || seq >= B) return TANDEM_ERR_INVALID_ARG;
         int n_b = 0;
         CK(cudaMemcpy(&n_b, c->st.n + seq, 4, cudaMemcpyDeviceToHost));
-        const int n = n_b - 1, d = m.d.d_model, H = m.d.n_heads, dh = d / H;
+        const int n = n_b - 1, H = m.kv_heads, dh = m.d.d_model / m.d.n_heads, d = m.d_kv;
         if (bytes != (size_t)n * d * 4) return TANDEM_ERR_INVALID_ARG;
         if (n == 0) return TANDEM_OK;
         const int which = (what == 3 || what == 5) ? 0 : 1;
@@ -1718,11 +1731,11 @@ extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
         snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled unavailable or failed");
         return TANDEM_ERR_CUDA;
     }
-    wt.tm[1] = wt.tm[2] = wt.tm[0]; wt.n_segs = 1; wt.seg_rows = d_small; wt.K = d_large;
-    wkv.tm[2] = wkv.tm[0]; wkv.n_segs = 2; wkv.seg_rows = d_small; wkv.K = d_small;
+    wt.tm[1] = wt.tm[2] = wt.tm[0]; wt.n_segs = 1; wt.seg_rows0 = wt.seg_rows = d_small; wt.K = d_large;
+    wkv.tm[2] = wkv.tm[0]; wkv.n_segs = 2; wkv.seg_rows0 = wkv.seg_rows = d_small; wkv.K = d_small;
     iota_rows_kernel<<<cdiv(rows, 256), 256, 0, tmp.stream>>>(row_seq, row_pos, rows, 0);
     EpiArgs e; memset(&e, 0, sizeof(e));
-    e.kcache = k_out; e.vcache = v_out; e.row_seq = row_seq; e.row_pos = row_pos; e.n_heads = 1; e.d_head = d_small; e.t_max = 1; e.seg = d_small;
+    e.kcache = k_out; e.vcache = v_out; e.row_seq = row_seq; e.row_pos = row_pos; e.n_heads = 1; e.d_head = d_small; e.t_max = 1; e.seg0 = e.seg = d_small;
     // weights streamed once per GEMM and group of 64 rows; for a few short rows the LayerNorm is fused into the
     // second GEMM's operand load
     TcScratch ts; ts.err = standalone_err_word();
@@ -1752,7 +1765,7 @@ extern "C" tandem_status tandem_block_linear(const void* x, const void* w, void*
         snprintf(g_cuda_err, sizeof(g_cuda_err), "cuTensorMapEncodeTiled unavailable or failed");
         return TANDEM_ERR_CUDA;
     }
-    tw.tm[1] = tw.tm[2] = tw.tm[0]; tw.n_segs = 1; tw.seg_rows = out_features; tw.K = in_features;
+    tw.tm[1] = tw.tm[2] = tw.tm[0]; tw.n_segs = 1; tw.seg_rows0 = tw.seg_rows = out_features; tw.K = in_features;
     TcScratch ts; ts.err = standalone_err_word();
     launch_tc_decode<PRO_BF16, EPI_STORE>(tmp, ts, x, in_features, nullptr, nullptr, rows, tw, true, epi_plain(y, out_features));
     return check_launch();
