@@ -45,14 +45,17 @@ WORKLOADS = {
     "medium": ("medium", 8, 2048, 3, 256, 2560),
     "large": ("large", 1, 8192, 3, 512, 8960),
     "large4": ("large", 4, 8192, 3, 512, 8960),
+    "large_gqa": ("large", 1, 8192, 3, 512, 8960),   # the large pair with grouped-query attention: 8 key/value heads of 32 (16 -> 4 in the small model)
 }
-DEVICE_INIT = {"large", "large4"}   # too big to draw on the host in reasonable time: N(0, 0.02^2) drawn on the device
+KV_HEADS = {"large_gqa": (8, 4)}
+DEVICE_INIT = {"large", "large4", "large_gqa"}   # too big to draw on the host in reasonable time: N(0, 0.02^2) drawn on the device
 
 
 def workload_desc(name):
     cfgname, B, P, gamma, new, _ = WORKLOADS[name]
+    kv = f", key/value heads {KV_HEADS[name][0]} (large) / {KV_HEADS[name][1]} (small)" if name in KV_HEADS else ""
     return (f"{cfgname}: batch {B}, prompt {P} uniform-random ids, gamma {gamma}, {new} new tokens, "
-            f"natural acceptance, random-init N(0,0.02) weights seed 0")
+            f"natural acceptance, random-init N(0,0.02) weights seed 0{kv}")
 
 
 # DRAM bytes (read + write) of one decode iteration from one ncu capture of every kernel of an iteration, valid only
@@ -282,6 +285,10 @@ def measure_workload(name, steps, warmup, rank, local_rank, world, extras, keep_
 
     cfgname, B, P, gamma, new, max_pos = WORKLOADS[name]
     shape = synth.named_config(cfgname, max_pos)
+    if name in KV_HEADS:
+        from dataclasses import replace
+        shape = replace(shape, large=replace(shape.large, n_kv_heads=KV_HEADS[name][0]),
+                        small=replace(shape.small, n_kv_heads=KV_HEADS[name][1]))
     dev = torch.device("cuda", local_rank)
     if name in DEVICE_INIT:
         weights = synth.device_weights(shape, 0, dev)
@@ -465,7 +472,7 @@ def run_ours(args, rank, local_rank, world):
     if extras and world == 1 and args.workload == "small" and not args.no_subrecords:
         # the other batch sizes of the metric: batch 8 (medium) and the bandwidth-bound batch 1 (large), few steps each
         line["workloads"] = {}
-        for name in ("medium", "large"):
+        for name in ("medium", "large", "large_gqa"):
             rr = measure_workload(name, 2, 3, rank, local_rank, world, extras=True)
             rr.pop("prof", None)
             line["workloads"][name] = sub_record(rr, peak)

@@ -36,6 +36,8 @@ struct AttnArgs {
     int nq;
     int n_heads, t_max;
     int n_kv_heads;                      // key/value heads of the caches; 0 = n_heads.  Query head h reads kv head h / (n_heads / n_kv_heads)
+    int heads_per_cta;                   // attn_decode_kernel: query heads of one key/value head served by one CTA (their rows share
+                                         // the 16-row tile: heads_per_cta * nq <= 16); 0 = 1.  grid.y = n_heads / heads_per_cta
     float* part_ml;                      // split mode: [M][H][n_chunks_max][2]
     float* part_acc;                     //             [M][H][n_chunks_max][DH]
     int n_chunks_max;
@@ -304,7 +306,11 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     float* inbox = reinterpret_cast<float*>(ring_all + (size_t)NW * C::STAGES * C::STAGE_ELEMS);   // [CL][QPC][SW]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int rank = blockIdx.x, h = blockIdx.y, g = blockIdx.z;
+    const int rank = blockIdx.x, g = blockIdx.z;
+    // Grouped-query attention: the tile's 16 rows hold the block's queries of `gpc` query heads that share one
+    // key/value head (row = head * nq + block row), so their keys and values are streamed once for all of them.
+    const int gpc = a.heads_per_cta > 0 ? a.heads_per_cta : 1;
+    const int h = blockIdx.y * gpc;                // first query head of this CTA
     const int CL = gridDim.x;                      // cluster size
     const int QPC = (ATT_NQ + CL - 1) / CL;        // queries a CTA finishes at most
     if (CL > 1) cluster_arrive_relaxed();          // opening handshake: waited for just before the first remote store
@@ -313,10 +319,10 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     // The row arrays were written at the start of the pass, at least two kernels back in the stream, so they may be
     // read before the wait below: a kernel lets its successor start only after its own wait has returned, that is
     // after its predecessor has finished, hence everything older than the immediate predecessor is complete.
-    const int cnt = a.nq, row0 = g * a.nq;
+    const int nq = a.nq, cnt = gpc * nq, row0 = g * nq;   // cnt: rows of the tile in use
     const int b = __ldcg(a.row_seq + row0);          // from L2: nothing an earlier kernel on this SM may have cached
     const int pos_first = __ldcg(a.row_pos + row0);
-    const int pos_last = pos_first + cnt - 1;
+    const int pos_last = pos_first + nq - 1;
     const int n_chunks = pos_last / ATT_CH + 1;
     const int n_mine = rank < n_chunks ? (n_chunks - rank + CL - 1) / CL : 0;
     const int n_kv = a.n_kv_heads > 0 ? a.n_kv_heads : a.n_heads;
@@ -394,11 +400,14 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     // The queries as A fragments: this lane holds rows lane/4 and lane/4 + 8, columns 2*(lane%4) (+1) (+8) of each
     // 16-wide step along the head dimension.
     const int row_lo = lane >> 2, row_hi = row_lo + 8, kc = 2 * (lane & 3);
+    // tile row -> (query head within the CTA, block row); rows beyond cnt are absent (zero queries, never stored)
+    const int hq_lo = row_lo < cnt ? row_lo / nq : 0, hq_hi = row_hi < cnt ? row_hi / nq : 0;
+    const int i_lo = row_lo < cnt ? row_lo - hq_lo * nq : 0, i_hi = row_hi < cnt ? row_hi - hq_hi * nq : 0;
     uint32_t qf[C::KSTEPS][4];
     {
         const bf16* qg = static_cast<const bf16*>(a.q) + h * DH + kc;
-        const bf16* q_lo = qg + (size_t)(row0 + row_lo) * a.ldq;
-        const bf16* q_hi = qg + (size_t)(row0 + row_hi) * a.ldq;
+        const bf16* q_lo = qg + (size_t)(row0 + i_lo) * a.ldq + hq_lo * DH;
+        const bf16* q_hi = qg + (size_t)(row0 + i_hi) * a.ldq + hq_hi * DH;
 #pragma unroll
         for (int ks = 0; ks < C::KSTEPS; ++ks) {
             qf[ks][0] = row_lo < cnt ? *reinterpret_cast<const uint32_t*>(q_lo + ks * 16) : 0u;
@@ -449,10 +458,10 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 const int ta = t0 + nt * 8 + kc + e;
-                sc[nt][e] = (row_lo < cnt && ta <= pos_first + row_lo) ? sc[nt][e] * a.scale : -INFINITY;
+                sc[nt][e] = (row_lo < cnt && ta <= pos_first + i_lo) ? sc[nt][e] * a.scale : -INFINITY;
                 mc_lo = fmaxf(mc_lo, sc[nt][e]);
                 if (has_hi) {
-                    sc[nt][2 + e] = (row_hi < cnt && ta <= pos_first + row_hi) ? sc[nt][2 + e] * a.scale : -INFINITY;
+                    sc[nt][2 + e] = (row_hi < cnt && ta <= pos_first + i_hi) ? sc[nt][2 + e] * a.scale : -INFINITY;
                     mc_hi = fmaxf(mc_hi, sc[nt][2 + e]);
                 }
             }
@@ -566,7 +575,8 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
                 l = fmaf(st[DH + 1], f, l);
                 ov = fmaf(st[tid], f, ov);
             }
-            const size_t oi = (size_t)(row0 + qi) * a.ldo + h * DH + tid;
+            const int hq = qi / nq;                  // tile row qi = query head hq of this CTA, block row qi - hq * nq
+            const size_t oi = (size_t)(row0 + qi - hq * nq) * a.ldo + (h + hq) * DH + tid;
             if (a.out_f32) static_cast<float*>(a.out)[oi] = ov / l;
             else static_cast<bf16*>(a.out)[oi] = __float2bfloat16_rn(ov / l);
         }

@@ -526,7 +526,8 @@ void launch_attn_decode_dq(tandem_ctx& c, const AttnArgs& a, int groups, int cl,
     static std::atomic<unsigned long long> attr_done{0};
     ensure_dyn_smem(attn_decode_kernel<DH>, attn_decode_smem_bytes<DH>(), attr_done);
     ProfScope ps(c, PC_ATTN_SPLIT, kv_bytes);
-    launch_ex(c, true, cl, attn_decode_kernel<DH>, dim3(cl, a.n_heads, groups), dim3(ATD_THREADS), attn_decode_smem_bytes<DH>(), a);
+    launch_ex(c, true, cl, attn_decode_kernel<DH>, dim3(cl, a.n_heads / std::max(1, a.heads_per_cta), groups), dim3(ATD_THREADS),
+              attn_decode_smem_bytes<DH>(), a);
 }
 // Cluster size: the largest of 1, 2, 4, 8 that keeps the launch within one wave of resident CTAs (two per SM,
 // one for 128-wide heads).  It depends on the number of sequences and heads only, so every pass of a run
@@ -538,8 +539,18 @@ int attn_cluster_size(int n_sms, int groups, int n_heads, int d_head) {
     while (cl < ATD_CLUSTER && (long long)groups * n_heads * cl * 2 <= slots) cl *= 2;
     return cl;
 }
-void launch_attn_decode(tandem_ctx& c, int d_head, const AttnArgs& a, int groups, double kv_bytes) {
-    const int cl = attn_cluster_size(c.n_sms, groups, a.n_heads, d_head);
+void launch_attn_decode(tandem_ctx& c, int d_head, const AttnArgs& a0, int groups, double kv_bytes) {
+    AttnArgs a = a0;
+    // Grouped-query attention: the query heads of one key/value head ride in one CTA as far as the 16-row tile has
+    // room (heads * queries per block <= 16; a power of two that divides the group).  The cluster size is taken
+    // from the key/value heads, which do not depend on the number of queries: a block pass and a one-row pass cut
+    // the context the same way.
+    const int n_kv = a.n_kv_heads > 0 ? a.n_kv_heads : a.n_heads;
+    const int group = a.n_heads / n_kv;
+    int gpc = 1;
+    while (gpc * 2 <= group && group % (gpc * 2) == 0 && gpc * 2 * a.nq <= ATT_NQ) gpc *= 2;
+    a.heads_per_cta = gpc;
+    const int cl = attn_cluster_size(c.n_sms, groups, n_kv, d_head);
     if (d_head == 32) launch_attn_decode_dq<32>(c, a, groups, cl, kv_bytes);
     else if (d_head == 64) launch_attn_decode_dq<64>(c, a, groups, cl, kv_bytes);
     else launch_attn_decode_dq<128>(c, a, groups, cl, kv_bytes);
