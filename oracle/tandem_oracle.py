@@ -30,6 +30,14 @@ Readings taken where the paper is silent or inconsistent:
   R17 Multi-query / grouped-query attention ("whether the attention is multi-head or multi-query", Section 3):
       n_kv_heads key/value heads of the same head size; query head h reads key/value head
       h // (n_heads / n_kv_heads); W_k and W_v map d_model to n_kv_heads * d_head.  Either model, independently.
+  R18 Sampling inside SPEED (Section 3.1 builds on the SPEED / speculative-decoding framework and its
+      experiments use sampled responses, num-samples 1 and 4).  The rule of that framework: draft d_r is drawn
+      from the small model's distribution q_r = softmax(logits_S / T_S); it is kept with probability
+      min(1, p_r(d_r) / q_r(d_r)), p_r = softmax(logits_L / T_L); at the first rejection the token is redrawn
+      from the normalised positive part of p_r - q_r; if all gamma drafts are kept, one more token is drawn from
+      p_{gamma+1}.  Every draw uses one uniform variate from a counter-based generator keyed by
+      (seed, sequence, iteration, slot): slots 0..gamma-1 draw the drafts, 16+r tests draft r, 48 redraws.
+      A draw from weights w with variate u returns the first index whose running sum exceeds u * sum(w).
   R4  Pre-LayerNorm blocks (gain and bias, eps 1e-5, biased variance), exact-erf GELU, no linear
       biases, learned absolute position embeddings, untied output head.
   R6  FF_Tandem MLP variant: hidden width given by the shape, GELU, no biases.
@@ -131,6 +139,47 @@ def splitmix64(x: int) -> int:
 def hashed_accept_length(mode_seed: int, seq: int, iteration: int, gamma: int) -> int:
     """accept_mode 2 (R13): a = mix(mix(mix(seed) ^ seq) ^ iteration) mod (gamma + 1)."""
     return splitmix64(splitmix64(splitmix64(mode_seed) ^ seq) ^ iteration) % (gamma + 1)
+
+
+# ----------------------------------------------------------------------------------------------
+# Sampling (R18)
+# ----------------------------------------------------------------------------------------------
+
+SLOT_ACCEPT = 16      # slot of the variate that tests draft r: SLOT_ACCEPT + r
+SLOT_REDRAW = 48      # slot of the variate that redraws (or draws the extra token)
+
+
+def uniform_variate(seed: int, seq: int, iteration: int, slot: int) -> float:
+    """Counter-based uniform in [0, 1) with 24 bits: the top 24 bits of
+    mix(mix(mix(mix(seed) ^ seq) ^ iteration) ^ slot), exactly representable in float32 and float64."""
+    x = splitmix64(splitmix64(splitmix64(splitmix64(seed) ^ seq) ^ iteration) ^ slot)
+    return (x >> 40) / float(1 << 24)
+
+
+def temperature_softmax(logits: np.ndarray, temperature: float) -> np.ndarray:
+    """softmax(logits / T) over the last axis."""
+    return softmax(np.asarray(logits, dtype=np.float64) / temperature)
+
+
+def draw_index(weights: np.ndarray, u: float) -> int:
+    """Inverse-CDF draw from non-negative (unnormalised) weights: the first index whose running sum exceeds
+    u * sum(weights); the last index with a positive weight if rounding leaves none."""
+    c = np.cumsum(weights)
+    target = u * c[-1]
+    for i in range(len(c)):
+        if c[i] > target:
+            return i
+    return int(np.nonzero(weights > 0)[0][-1])
+
+
+def accept_probability(p: np.ndarray, q: np.ndarray, token: int) -> float:
+    """Probability of keeping a draft drawn from q when the target distribution is p: min(1, p / q)."""
+    return min(1.0, p[token] / q[token]) if q[token] > 0 else 1.0
+
+
+def residual_weights(p: np.ndarray, q: np.ndarray) -> np.ndarray:
+    """Unnormalised distribution of the redrawn token after a rejection: the positive part of p - q."""
+    return np.maximum(p - q, 0.0)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -434,6 +483,60 @@ class TandemOracle:
         self.own.truncate(0)
         self.iteration += 1
         return emitted
+
+    def step_sampling(self, gamma: int, temp_large: float, temp_small: float, seed: int, seq: int = 0,
+                      forced: Optional[dict] = None) -> dict:
+        """One sampled Tandem + SPEED iteration (R18).  Returns the drafts, the accept length, the token emitted
+        after the kept drafts, and the distributions / variates behind every decision.  With `forced`
+        ({"drafts", "accept_len", "final"}: another implementation's choices) those choices are followed instead
+        of this function's own, so that the caller can check each of them against the returned records."""
+        n = len(self.tokens)
+        it = self.iteration
+        assert self.derived.length() == n - 1 and self.own.length() == 0
+        u_in = self.tokens[-1]
+        drafts, own_drafts, q_list, s_logits = [], [], [], []
+        for s_ in range(gamma):
+            lg = self._small_step(u_in, n - 1 + s_)
+            q = temperature_softmax(lg, temp_small)
+            d = draw_index(q, uniform_variate(seed, seq, it, s_))
+            own_drafts.append(d)
+            u_in = int(forced["drafts"][s_]) if forced is not None else d
+            drafts.append(u_in)
+            q_list.append(q)
+            s_logits.append(lg)
+        rows = [self.tokens[-1]] + drafts
+        reps, l_logits = large_block_pass(self.large, self.large_cache, rows, n - 1)
+        self.n_large_runs += 1
+        p_list = [temperature_softmax(l_logits[r], temp_large) for r in range(gamma + 1)]
+        ratios = [accept_probability(p_list[r], q_list[r], drafts[r]) for r in range(gamma)]
+        tests = [uniform_variate(seed, seq, it, SLOT_ACCEPT + r) for r in range(gamma)]
+        own_a = 0
+        while own_a < gamma and tests[own_a] < ratios[own_a]:
+            own_a += 1
+        a = int(forced["accept_len"]) if forced is not None else own_a
+        final_w = residual_weights(p_list[a], q_list[a]) if a < gamma else p_list[gamma]
+        u_final = uniform_variate(seed, seq, it, SLOT_REDRAW)
+        own_final = draw_index(final_w, u_final)
+        final = int(forced["final"]) if forced is not None else own_final
+        emitted = drafts[:a] + [final]
+        self.tokens += emitted
+        self.large_cache.truncate(n + a)
+        self._project_rows(reps, range(a + 1))
+        self.own.truncate(0)
+        self.iteration += 1
+        return {"drafts": drafts, "own_drafts": own_drafts, "accept_len": a, "own_accept_len": own_a, "final": final,
+                "own_final": own_final, "emitted": emitted, "q": q_list, "p": p_list, "ratios": ratios, "tests": tests,
+                "final_weights": final_w, "u_final": u_final, "small_logits": s_logits, "large_logits": l_logits,
+                "n_committed": len(self.tokens)}
+
+    def generate_sampling(self, prompt: Sequence[int], gamma: int, max_new: int, temp_large: float, temp_small: float,
+                          seed: int, seq: int = 0) -> Tuple[List[int], List[int]]:
+        self.prefill(prompt)
+        P = len(prompt)
+        accepts = []
+        while len(self.tokens) - P < max_new:
+            accepts.append(self.step_sampling(gamma, temp_large, temp_small, seed, seq)["accept_len"])
+        return self.tokens[P:P + max_new], accepts
 
     def step(self, gamma: int, mode: int = ACCEPT_NATURAL, mode_seed: int = 0, seq: int = 0) -> dict:
         drafts, s_logits = self.draft(gamma)
