@@ -365,6 +365,13 @@ def measure_workload(name, steps, warmup, rank, local_rank, world, extras, keep_
         rep_only = lambda: t.tandem_standalone_generate(gamma, binding.STANDALONE_REPRESENTATION_ONLY, new)
         t.tandem_prefill(prompts); rep_only(); t.tandem_prefill(prompts); rep_only()
         r["representation_only_decode_ms"] = timed_decode(rep_only, 2)
+        # sampled SPEED at temperature 1 / 1 (two independent random models still overlap in distribution, so the
+        # accept lengths are spread out, unlike the arg-max comparison)
+        sampled = lambda: t.tandem_speculative_generate(gamma, new, binding.ACCEPT_SAMPLE, 1)
+        t.tandem_prefill(prompts); sampled(); t.tandem_prefill(prompts); sampled()
+        r["sampled_decode_ms"] = timed_decode(sampled, 2)
+        t.tandem_prefill(prompts)
+        r["sampled_accept_hist"] = sampled()[2]["accept_hist"]
         # per-kernel pass: the same step with every launch bracketed by events (serialises the stream: shares only)
         t.tandem_profile_enable(400000)
         t.tandem_prefill(prompts)
@@ -406,6 +413,8 @@ def sub_record(r, peak):
         rec["accept_all_decode_tokens_per_s"] = toks / (r["accept_all_decode_ms"] * 1e-3)
         rec["large_greedy_decode_tokens_per_s"] = toks / (r["greedy_decode_ms"] * 1e-3)
         rec["standalone_representation_only_decode_tokens_per_s"] = toks / (r["representation_only_decode_ms"] * 1e-3)
+        rec["sampled_decode_tokens_per_s"] = toks / (r["sampled_decode_ms"] * 1e-3)
+        rec["sampled_accept_hist"] = r["sampled_accept_hist"]
     return rec
 
 
@@ -441,6 +450,8 @@ def run_ours(args, rank, local_rank, world):
         line["accept_all_decode_tokens_per_s"] = toks / (r["accept_all_decode_ms"] * 1e-3)
         line["large_greedy_decode_tokens_per_s"] = toks / (r["greedy_decode_ms"] * 1e-3)
         line["standalone_representation_only_decode_tokens_per_s"] = toks / (r["representation_only_decode_ms"] * 1e-3)
+        line["sampled_decode_tokens_per_s"] = toks / (r["sampled_decode_ms"] * 1e-3)
+        line["sampled_accept_hist"] = r["sampled_accept_hist"]
         tot = sum(v["ms"] for v in prof.values()) or 1.0
         # bracketed pass: work = algorithmic bytes (GB/s) for the streaming kernels, flops (TFLOP/s) for the prompt pass
         line["kernels_bracketed"] = {

@@ -69,7 +69,15 @@ enum { TANDEM_ACCEPT_NATURAL = 0, TANDEM_ACCEPT_ALL = 1, TANDEM_ACCEPT_HASH = 2,
         * "Inference", Figure 3): M_L reads the pending token and the first gamma-1 drafts as gamma rows and
         * predicts nothing, all gamma drafts are kept, the last one becomes pending.  Needs gamma >= 1; a step
         * result's targets are -1. */
-       TANDEM_ACCEPT_REPRESENTATION_ONLY = 3 };
+       TANDEM_ACCEPT_REPRESENTATION_ONLY = 3,
+       /* 4 = sampled SPEED (Section 3.1 builds on the SPEED / speculative-decoding framework; the paper's latency
+        * tables are on sampled responses): draft r is drawn from softmax(logits_S / T_S); it is kept with probability
+        * min(1, p(d_r) / q(d_r)) with p = softmax(logits_L / T_L); at the first rejection the token is redrawn from
+        * the positive part of p - q; if all drafts are kept one more token is drawn from M_L's next distribution.
+        * Temperatures: tandem_set_sampling; mode_seed seeds the counter-based uniform variates, keyed by
+        * (seed, sequence, iteration, slot).  A step result's targets then hold, at index accept_len, the token that
+        * follows the kept drafts (other entries: M_L's arg-max, for information). */
+       TANDEM_ACCEPT_SAMPLE = 4 };
 /* variants of tandem_standalone_generate */
 enum { TANDEM_STANDALONE_FREE_TOKEN = 0, TANDEM_STANDALONE_REPRESENTATION_ONLY = 1,
        TANDEM_STANDALONE_FREE_TOKEN_FULL_PROMPT = 2 };
@@ -154,6 +162,16 @@ TANDEM_API tandem_status tandem_destroy(tandem_ctx* ctx);
 TANDEM_API tandem_status tandem_prefill(tandem_ctx* ctx, int32_t batch, const int32_t* prompt_ids,
                              const int32_t* prompt_lens);
 
+/* The same prompt pass for several responses per query ("num-samples" of Section 3.1 and Section 4.2, e.g. 4
+ * sampled responses that are ranked afterwards): n_queries prompts, each starting num_samples sequences; query q
+ * owns sequences q * num_samples .. (q + 1) * num_samples - 1 of the batch, n_queries * num_samples <= max_batch.
+ * M_L reads each prompt ONCE; its keys / values and the small model's large-derived keys / values are then copied
+ * to the query's other sequences, which start from the same pending token and diverge through their own random
+ * variates (TANDEM_ACCEPT_SAMPLE keys them by sequence).  prompt_ids / prompt_lens as in tandem_prefill, per query.
+ * (The copies make the samples ordinary sequences: decode attention reads each sequence's own cache.) */
+TANDEM_API tandem_status tandem_prefill_samples(tandem_ctx* ctx, int32_t n_queries, int32_t num_samples,
+                                                const int32_t* prompt_ids, const int32_t* prompt_lens);
+
 /* One Tandem + SPEED iteration for every sequence (Section 3.1):
  *   draft   M_S runs gamma times from the pending token; each step attends the large-derived keys/values
  *           of positions M_L has processed plus M_S's own keys/values of the current block (Eq. 2);
@@ -175,6 +193,10 @@ TANDEM_API tandem_status tandem_block_step(tandem_ctx* ctx, int32_t gamma, int32
 TANDEM_API tandem_status tandem_speculative_generate(tandem_ctx* ctx, int32_t gamma, int32_t max_new_tokens,
                                           int32_t accept_mode, uint64_t mode_seed, int32_t* out_ids,
                                           int32_t* out_lens, tandem_stats* stats);
+
+/* Temperatures of the two models for accept mode TANDEM_ACCEPT_SAMPLE (both > 0; default 1 and 1).  Applies to the
+ * iterations enqueued afterwards; waits for the context's stream when a value changes. */
+TANDEM_API tandem_status tandem_set_sampling(tandem_ctx* ctx, float temp_large, float temp_small);
 
 /* Stand-alone Tandem decoding (Section 3 "Inference"; Table 3's latency row): M_S writes the response, M_L only
  * supplies representations (and, with the free token, one token per block); nothing is verified.  Must follow

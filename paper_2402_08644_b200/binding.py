@@ -18,7 +18,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtandem_
 _lib = None
 
 GAMMA_LIMIT = 15
-ACCEPT_NATURAL, ACCEPT_ALL, ACCEPT_HASH, ACCEPT_REPRESENTATION_ONLY = 0, 1, 2, 3
+ACCEPT_NATURAL, ACCEPT_ALL, ACCEPT_HASH, ACCEPT_REPRESENTATION_ONLY, ACCEPT_SAMPLE = 0, 1, 2, 3, 4
 STANDALONE_FREE_TOKEN, STANDALONE_REPRESENTATION_ONLY, STANDALONE_FREE_TOKEN_FULL_PROMPT = 0, 1, 2
 STATUS_NAMES = ["OK", "INVALID_ARG", "SHAPE", "ARENA_TOO_SMALL", "CAPACITY", "STATE", "CUDA", "TIMEOUT", "UNIMPLEMENTED"]
 (READ_LARGE_LOGITS, READ_SMALL_LOGITS, READ_LARGE_HIDDEN, READ_LARGE_K, READ_LARGE_V, READ_SMALL_K, READ_SMALL_V,
@@ -30,7 +30,8 @@ EXPORTS = ["tandem_query_arena", "tandem_create", "tandem_destroy", "tandem_pref
            "tandem_ff_tandem_project_scratch_bytes", "tandem_block_linear",
            "tandem_status_string", "tandem_last_cuda_error", "tandem_profile_enable", "tandem_profile_read",
            "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static",
-           "tandem_debug_expire_wait", "tandem_standalone_check", "tandem_standalone_generate"]
+           "tandem_debug_expire_wait", "tandem_standalone_check", "tandem_standalone_generate",
+           "tandem_set_sampling", "tandem_prefill_samples"]
 
 
 class TandemError(RuntimeError):
@@ -86,10 +87,12 @@ def load_library():
     lib.tandem_create.argtypes = [C.POINTER(Config), C.POINTER(Weights), vp, sz, C.POINTER(vp)]
     lib.tandem_destroy.argtypes = [vp]
     lib.tandem_prefill.argtypes = [vp, i32, pi32, pi32]
+    lib.tandem_prefill_samples.argtypes = [vp, i32, i32, pi32, pi32]
     lib.tandem_block_step.argtypes = [vp, i32, i32, u64, C.POINTER(StepResult)]
     lib.tandem_speculative_generate.argtypes = [vp, i32, i32, i32, u64, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_large_greedy_generate.argtypes = [vp, i32, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_standalone_generate.argtypes = [vp, i32, i32, i32, pi32, pi32, C.POINTER(Stats)]
+    lib.tandem_set_sampling.argtypes = [vp, C.c_float, C.c_float]
     lib.tandem_debug_read.argtypes = [vp, i32, i32, i32, vp, sz]
     lib.tandem_decode_attention_scratch_bytes.argtypes = [i32] * 5
     lib.tandem_decode_attention_scratch_bytes.restype = sz
@@ -202,6 +205,13 @@ class Tandem:
                                        lens.ctypes.data_as(C.POINTER(C.c_int32))), "tandem_prefill")
         self.batch = len(prompts)
 
+    def tandem_prefill_samples(self, prompts: Sequence[Sequence[int]], num_samples: int) -> None:
+        lens = np.asarray([len(p) for p in prompts], dtype=np.int32)
+        ids = np.ascontiguousarray(np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts]))
+        _check(self.lib.tandem_prefill_samples(self.ctx, len(prompts), num_samples, ids.ctypes.data_as(C.POINTER(C.c_int32)),
+                                               lens.ctypes.data_as(C.POINTER(C.c_int32))), "tandem_prefill_samples")
+        self.batch = len(prompts) * num_samples
+
     def tandem_block_step(self, gamma: int, accept_mode: int = 0, mode_seed: int = 0, want_result: bool = True):
         if not want_result:
             _check(self.lib.tandem_block_step(self.ctx, gamma, accept_mode, mode_seed, None), "tandem_block_step")
@@ -229,6 +239,9 @@ class Tandem:
         _check(self.lib.tandem_speculative_generate(self.ctx, gamma, max_new, accept_mode, mode_seed, p(out), p(lens),
                                                     C.byref(st)), "tandem_speculative_generate")
         return out, lens, self._stats(st, gamma)
+
+    def tandem_set_sampling(self, temp_large: float, temp_small: float) -> None:
+        _check(self.lib.tandem_set_sampling(self.ctx, temp_large, temp_small), "tandem_set_sampling")
 
     def tandem_standalone_generate(self, gamma: int, variant: int, max_new: int):
         out = np.zeros((self.batch, max_new), np.int32)

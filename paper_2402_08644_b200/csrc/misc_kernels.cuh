@@ -256,6 +256,8 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restric
 // Generation Only"; Figure 3): the large model has read gamma rows and predicted nothing, all gamma tokens of the
 // small model are kept and the last one becomes pending.  The last draft is then not a block row, so nobody has
 // turned it into a token id yet: when fin_val is given it is finished here from the small head's per-tile results.
+// mode 4 is sampled SPEED: sample_verify_kernel has already written each sequence's accept length and, at that index
+// of its targets, the token drawn after the kept drafts; this kernel only does the bookkeeping.
 // block: 256.
 __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed,
                                                      int max_new, const float* amax_val, const int* amax_idx, int amax_stride,
@@ -270,7 +272,7 @@ __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, in
             }
         }
         __syncthreads();
-    } else if (amax_val != nullptr) {
+    } else if (amax_val != nullptr && mode != 4) {   // (mode 4: the sampled decisions are already in place)
         const int rows = batch * (gamma + 1);
         for (int m = threadIdx.x >> 5; m < rows; m += 8) {
             const int tok = argmax_from_tiles(amax_val + (size_t)m * amax_stride, amax_idx + (size_t)m * amax_stride, n_tiles);
@@ -287,6 +289,7 @@ __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, in
         const int* g = st.targets + b * (st.gamma_limit + 1);
         int a = 0;
         if (mode == 1 || mode == 3) a = gamma;
+        else if (mode == 4) a = min(max(st.accept_len[b], 0), gamma);   // sampled SPEED: decided by sample_verify_kernel, with g[a] the token it drew
         else if (mode == 2) a = (int)(splitmix64(splitmix64(splitmix64(seed) ^ (unsigned long long)b) ^ (unsigned long long)iteration) % (unsigned long long)(gamma + 1));
         else { while (a < gamma && d[a] == g[a]) ++a; }
         st.accept_len[b] = a;

@@ -19,6 +19,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "misc_kernels.cuh"
+#include "sampling.cuh"
 
 using namespace tandem;
 
@@ -127,6 +128,7 @@ struct tandem_ctx {
     bool setup_failed = false;           // a launch helper could not encode a tensor map: reported by the enclosing call
     bool tc_prompt_attn = false;         // prompt attention on the tensor cores (head size 64 or 128)
     int prompt_group = ATT_NQ;           // queries per attention group of the prompt pass
+    float temp_large = 1.0f, temp_small = 1.0f;   // sampled SPEED (accept mode 4): temperatures of the two models
 };
 
 namespace {
@@ -773,9 +775,27 @@ void launch_verify(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_ne
               from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_small) : (const int*)nullptr);
 }
 
+// Sampled SPEED: draft s of every sequence drawn from the small model's logits of step s.
+void launch_sample_draft(tandem_ctx& c, int s, uint64_t seed) {
+    const float* logits = at<float>(c, c.lay.logits_small) + (size_t)s * c.batch * c.small.d.vocab;
+    ProfScope ps(c, PC_ARGMAX, (double)c.batch * c.small.d.vocab * 8.0);
+    launch_ex(c, true, 1, sample_draft_kernel, dim3(c.batch), dim3(SMP_THREADS), 0, c.st, logits, (int)c.small.d.vocab, s, c.temp_small,
+              (unsigned long long)seed);
+}
+// Sampled SPEED: accept / redraw decisions of the iteration, ahead of the verify kernel's bookkeeping.
+void launch_sample_verify(tandem_ctx& c, int gamma, uint64_t seed) {
+    ProfScope ps(c, PC_ARGMAX, (double)c.batch * (2 * gamma + 1) * c.large.d.vocab * 8.0);
+    launch_ex(c, true, 1, sample_verify_kernel, dim3(c.batch), dim3(SMP_THREADS), 0, c.st, c.batch, gamma,
+              (const float*)at<float>(c, c.lay.logits_large), (const float*)at<float>(c, c.lay.logits_small), (int)c.large.d.vocab,
+              c.temp_large, c.temp_small, (unsigned long long)seed);
+}
+
 template <typename T>
 void iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
-    for (int s = 0; s < gamma; ++s) small_step<T>(c, s);
+    for (int s = 0; s < gamma; ++s) {
+        small_step<T>(c, s);
+        if (mode == 4) launch_sample_draft(c, s, seed);   // replaces the arg-max draft of this step
+    }
     if (mode == 3) {   // stand-alone Tandem without the free token: gamma rows, no output head
         setup_rows(c, 0, gamma);
         large_pass<T>(c, decode_rows(c, gamma - 1, gamma), true, false);
@@ -783,6 +803,7 @@ void iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
         setup_rows(c, 0, gamma + 1);
         large_pass<T>(c, decode_rows(c, gamma, gamma + 1), true, true);
     }
+    if (mode == 4) launch_sample_verify(c, gamma, seed);
     launch_verify(c, gamma, mode, seed, max_new, false);
     c.last_gamma = gamma;
 }
@@ -861,9 +882,11 @@ void tc_head(tandem_ctx& c, const Model& m, float* h, const Rows& r, float* logi
                            epi_plain(logits, m.d.vocab), at<float>(c, amax_val_off), at<int>(c, amax_idx_off), c.lay.vocab_tiles);
 }
 
-void tc_small_step(tandem_ctx& c, int s) {
+// sampled: the previous draft was drawn by sample_draft_kernel (it is in the loop state already), not left as per-tile
+// arg-max results.
+void tc_small_step(tandem_ctx& c, int s, bool sampled) {
     float* y = at<float>(c, c.lay.h_small);
-    tc_begin(c, c.small, y, s, 1, s > 0 ? s : -1);
+    tc_begin(c, c.small, y, s, 1, (s > 0 && !sampled) ? s : -1);
     const Rows r = decode_rows(c, s, 1);
     for (int j = 0; j < c.small.d.n_layers; ++j) tc_decoder_layer(c, c.small, j, y, r, false);
     float* logits = at<float>(c, c.lay.logits_small) + (size_t)s * c.batch * c.small.d.vocab;
@@ -939,9 +962,14 @@ void tc_large_block(tandem_ctx& c, int nq, int fin_r, bool project, bool head) {
 }
 
 void tc_iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
-    for (int s = 0; s < gamma; ++s) tc_small_step(c, s);
+    const bool sampled = mode == 4;
+    for (int s = 0; s < gamma; ++s) {
+        tc_small_step(c, s, sampled);
+        if (sampled) launch_sample_draft(c, s, seed);
+    }
     if (mode == 3) tc_large_block(c, gamma, -1, true, false);   // gamma rows, no head: the last draft is finished by the verify kernel
-    else tc_large_block(c, gamma + 1, gamma > 0 ? gamma : -1, true, true);
+    else tc_large_block(c, gamma + 1, (gamma > 0 && !sampled) ? gamma : -1, true, true);
+    if (sampled) launch_sample_verify(c, gamma, seed);
     launch_verify(c, gamma, mode, seed, max_new, true);
     c.last_gamma = gamma;
 }
@@ -1228,22 +1256,29 @@ extern "C" tandem_status tandem_destroy(tandem_ctx* c) {
     return TANDEM_OK;
 }
 
-extern "C" tandem_status tandem_prefill(tandem_ctx* c, int32_t batch, const int32_t* prompt_ids, const int32_t* prompt_lens) {
-    TRY(begin_call(c));
-    if (!prompt_ids || !prompt_lens || batch < 1) return TANDEM_ERR_INVALID_ARG;
-    if (batch > c->cfg.max_batch) return TANDEM_ERR_CAPACITY;
+namespace {
+
+// Prompt pass for n_queries prompts, each the start of `samples` sequences (query q owns sequences q * samples ..
+// q * samples + samples - 1).  The large model reads each prompt once, into the first sequence of its query; the
+// other sequences of the query get copies of the keys / values it produced (both caches) and the same pending token.
+tandem_status prefill_impl(tandem_ctx* c, int n_queries, int samples, const int32_t* prompt_ids, const int32_t* prompt_lens) {
+    if (!prompt_ids || !prompt_lens || n_queries < 1 || samples < 1) return TANDEM_ERR_INVALID_ARG;
+    const long long batch_ll = (long long)n_queries * samples;
+    if (batch_ll > c->cfg.max_batch) return TANDEM_ERR_CAPACITY;
+    const int batch = (int)batch_ll;
     const int pos_cap = std::min(c->cfg.max_seq, std::min(c->cfg.large.max_pos, c->cfg.small.max_pos));
-    long long rows = 0, total = 0;
+    long long rows = 0, total = 0, total_ids = 0;
     int n_max = 0;
-    for (int b = 0; b < batch; ++b) {
-        if (prompt_lens[b] < 1) return TANDEM_ERR_INVALID_ARG;
-        if (prompt_lens[b] > pos_cap) return TANDEM_ERR_CAPACITY;
-        rows += prompt_lens[b] - 1;
-        total += prompt_lens[b];
-        n_max = std::max(n_max, prompt_lens[b]);
+    for (int q = 0; q < n_queries; ++q) {
+        if (prompt_lens[q] < 1) return TANDEM_ERR_INVALID_ARG;
+        if (prompt_lens[q] > pos_cap) return TANDEM_ERR_CAPACITY;
+        rows += prompt_lens[q] - 1;
+        total += (long long)prompt_lens[q] * samples;
+        total_ids += prompt_lens[q];
+        n_max = std::max(n_max, prompt_lens[q]);
     }
     if (rows > c->lay.max_rows) return TANDEM_ERR_CAPACITY;
-    for (long long i = 0; i < total; ++i)
+    for (long long i = 0; i < total_ids; ++i)
         if (prompt_ids[i] < 0 || prompt_ids[i] >= c->cfg.large.vocab) return TANDEM_ERR_INVALID_ARG;
 
     CK(cudaStreamSynchronize(c->stream));   // staging buffer free again; no verify kernel in flight
@@ -1259,14 +1294,16 @@ extern "C" tandem_status tandem_prefill(tandem_ctx* c, int32_t batch, const int3
     int32_t* p_pend = p_n + c->cfg.max_batch;
     int m = 0, groups = 0;
     long long off = 0;
-    for (int b = 0; b < batch; ++b) {
-        const int len = prompt_lens[b];
+    for (int q = 0; q < n_queries; ++q) {
+        const int len = prompt_lens[q];
         for (int p = 0; p < len - 1; ++p) {
             if (p % c->prompt_group == 0) { p_g0[groups] = m; p_gc[groups] = std::min(c->prompt_group, len - 1 - p); ++groups; }
-            p_tok[m] = prompt_ids[off + p]; p_seq[m] = b; p_pos[m] = p; ++m;
+            p_tok[m] = prompt_ids[off + p]; p_seq[m] = q * samples; p_pos[m] = p; ++m;
         }
-        p_n[b] = len;
-        p_pend[b] = prompt_ids[off + len - 1];
+        for (int j = 0; j < samples; ++j) {
+            p_n[q * samples + j] = len;
+            p_pend[q * samples + j] = prompt_ids[off + len - 1];
+        }
         off += len;
     }
     cudaStream_t s = c->stream;
@@ -1288,7 +1325,42 @@ extern "C" tandem_status tandem_prefill(tandem_ctx* c, int32_t batch, const int3
         if (c->cfg.dtype == TANDEM_DTYPE_BF16) large_pass<bf16>(*c, r, true, false);
         else large_pass<float>(*c, r, true, false);
     }
-    return check_launch(*c);
+    TRY(check_launch(*c));
+    if (samples > 1) {
+        // the prompt's keys / values, per (model, layer, K or V, key/value head): positions 0 .. len - 2 of sequence
+        // q * samples go to the query's other sequences (one strided copy per destination)
+        for (const Model* mdl : {&c->large, &c->small}) {
+            const int dh = mdl->d.d_model / mdl->d.n_heads;
+            const size_t pitch = (size_t)c->cfg.max_seq * dh * c->esz;            // one head's positions
+            const size_t seq_bytes = pitch * mdl->kv_heads;
+            for (int l = 0; l < mdl->d.n_layers; ++l)
+                for (int which = 0; which < 2; ++which) {
+                    unsigned char* base = c->arena + mdl->kv_off + ((size_t)l * 2 + which) * mdl->kv_layer_elems * c->esz;
+                    for (int q = 0; q < n_queries; ++q) {
+                        const size_t width = (size_t)(prompt_lens[q] - 1) * dh * c->esz;
+                        if (width == 0) continue;
+                        const unsigned char* src = base + (size_t)q * samples * seq_bytes;
+                        for (int j = 1; j < samples; ++j)
+                            CK(cudaMemcpy2DAsync(base + ((size_t)q * samples + j) * seq_bytes, pitch, src, pitch, width, mdl->kv_heads,
+                                                 cudaMemcpyDeviceToDevice, s));
+                    }
+                }
+        }
+    }
+    return TANDEM_OK;
+}
+
+}  // namespace
+
+extern "C" tandem_status tandem_prefill(tandem_ctx* c, int32_t batch, const int32_t* prompt_ids, const int32_t* prompt_lens) {
+    TRY(begin_call(c));
+    return prefill_impl(c, batch, 1, prompt_ids, prompt_lens);
+}
+
+extern "C" tandem_status tandem_prefill_samples(tandem_ctx* c, int32_t n_queries, int32_t num_samples, const int32_t* prompt_ids,
+                                                const int32_t* prompt_lens) {
+    TRY(begin_call(c));
+    return prefill_impl(c, n_queries, num_samples, prompt_ids, prompt_lens);
 }
 
 namespace {
@@ -1305,7 +1377,7 @@ tandem_status capacity_for(tandem_ctx* c, int extra_tokens, int gamma) {
 extern "C" tandem_status tandem_block_step(tandem_ctx* c, int32_t gamma, int32_t accept_mode, uint64_t mode_seed,
                                            tandem_step_result* result) {
     TRY(begin_call(c));
-    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 3) return TANDEM_ERR_INVALID_ARG;
+    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 4) return TANDEM_ERR_INVALID_ARG;
     if (accept_mode == TANDEM_ACCEPT_REPRESENTATION_ONLY && gamma < 1) return TANDEM_ERR_INVALID_ARG;
     if (c->batch == 0) return TANDEM_ERR_STATE;
     TRY(capacity_for(c, 0, gamma));
@@ -1426,9 +1498,22 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
 extern "C" tandem_status tandem_speculative_generate(tandem_ctx* c, int32_t gamma, int32_t max_new_tokens, int32_t accept_mode,
                                                      uint64_t mode_seed, int32_t* out_ids, int32_t* out_lens, tandem_stats* stats) {
     TRY(begin_call(c));
-    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 3) return TANDEM_ERR_INVALID_ARG;
+    if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 4) return TANDEM_ERR_INVALID_ARG;
     if (accept_mode == TANDEM_ACCEPT_REPRESENTATION_ONLY && gamma < 1) return TANDEM_ERR_INVALID_ARG;
     return run_generate(c, true, gamma, max_new_tokens, accept_mode, mode_seed, out_ids, out_lens, stats);
+}
+
+extern "C" tandem_status tandem_set_sampling(tandem_ctx* c, float temp_large, float temp_small) {
+    TRY(begin_call(c));
+    if (!(temp_large > 0.f) || !(temp_small > 0.f)) return TANDEM_ERR_INVALID_ARG;
+    if (temp_large == c->temp_large && temp_small == c->temp_small) return TANDEM_OK;
+    // the temperatures are kernel arguments baked into the captured iterations: drop the sampled ones
+    CK(cudaStreamSynchronize(c->stream));
+    for (auto& g : c->graphs)
+        if (g.mode == TANDEM_ACCEPT_SAMPLE && g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+    c->temp_large = temp_large;
+    c->temp_small = temp_small;
+    return TANDEM_OK;
 }
 
 extern "C" tandem_status tandem_standalone_generate(tandem_ctx* c, int32_t gamma, int32_t variant, int32_t max_new_tokens,

@@ -566,6 +566,152 @@ def test_expired_device_wait_is_reported_and_the_context_survives():
 
 
 # ------------------------------------------------------------------------------------------------
+# sampled SPEED (Section 3.1 on the SPEED framework)
+# ------------------------------------------------------------------------------------------------
+
+def _cdf_valid(weights, u, token, eps):
+    """Whether `token` is a correct inverse-CDF draw from `weights` for the variate u, up to eps of probability mass
+    (the GPU sums in fp32, the checker in fp64: near a boundary of the running sum both neighbours are correct)."""
+    c = np.cumsum(weights) / weights.sum()
+    lo = c[token - 1] if token > 0 else 0.0
+    return weights[token] > 0 and lo - eps <= u <= c[token] + eps
+
+
+def _sampled_replay(shape, w, prompts, gamma, iters, tl, ts, seed, tol, eps):
+    """GPU iterations in sampled mode; the checker follows the GPU's choices and every choice must be a correct one
+    under the checker's distributions.  Returns (choices that equal the checker's own, all choices, accept lengths)."""
+    t = binding.Tandem(shape, w, max_batch=len(prompts), max_seq=shape.large.max_pos, gamma_max=gamma)
+    t.tandem_set_sampling(tl, ts)
+    t.tandem_prefill(prompts)
+    oracles = [O.TandemOracle(shape, w) for _ in prompts]
+    for o, p in zip(oracles, prompts):
+        o.prefill(p)
+    same = total = 0
+    accepts = []
+    for it in range(iters):
+        res = t.tandem_block_step(gamma, binding.ACCEPT_SAMPLE, seed)
+        s_logits = t.tandem_debug_read(binding.READ_SMALL_LOGITS, gamma)
+        l_logits = t.tandem_debug_read(binding.READ_LARGE_LOGITS, gamma)
+        for b, o in enumerate(oracles):
+            a = int(res["accept_len"][b])
+            forced = {"drafts": res["drafts"][b].tolist(), "accept_len": a, "final": int(res["targets"][b][a])}
+            iteration = o.iteration
+            r = o.step_sampling(gamma, tl, ts, seed, b, forced=forced)
+            for s_ in range(gamma):
+                assert np.abs(s_logits[s_, b] - r["small_logits"][s_]).max() < tol
+                assert _cdf_valid(r["q"][s_], O.uniform_variate(seed, b, iteration, s_), forced["drafts"][s_], eps)
+            assert np.abs(l_logits[b] - r["large_logits"]).max() < tol
+            for i in range(a):                                      # kept drafts passed their test
+                assert r["tests"][i] < r["ratios"][i] + eps
+            if a < gamma:                                           # the first rejected one failed it
+                assert r["tests"][a] >= r["ratios"][a] - eps
+            assert _cdf_valid(r["final_weights"], r["u_final"], forced["final"], eps)
+            assert res["n_committed"][b] == r["n_committed"]
+            same += (r["own_drafts"] == forced["drafts"]) + (r["own_accept_len"] == a) + (r["own_final"] == forced["final"])
+            total += 3
+            accepts.append(a)
+    t.close()
+    return same, total, accepts
+
+
+def test_fp32_sampled_speed_choices_are_the_checkers():
+    """fp32 mode, ragged batch, temperatures 0.9 / 1.1: every draft, every accept / reject decision and every
+    redrawn token is a correct draw under the checker's distributions, and nearly all equal the checker's own."""
+    shape = gpu_toy_shape(kind=synth.FF_TANDEM_MLP, hidden=40, layer_map=(1, 3))
+    w = toy_weights(shape, seed=91)
+    same, total, accepts = _sampled_replay(shape, w, prompts_for(shape, [3, 130, 17], seed=9), 3, 6, 0.9, 1.1, 777, TOL_FP32, 1e-4)
+    assert same >= total - 2
+    assert len(set(accepts)) >= 2
+
+
+def test_bf16_sampled_speed_choices_are_valid_draws():
+    shape = gpu_toy_shape(dtype=synth.DTYPE_BF16, layer_map=(1, 2), large=(2, 256, 4, 512), small=(2, 128, 2, 256))
+    w = _bf16_weights(shape, seed=92, std=0.05)
+    same, total, accepts = _sampled_replay(shape, w, prompts_for(shape, [5, 140, 1], seed=19), 4, 6, 0.8, 1.0, 4242, TOL_BF16, 0.05)
+    assert same >= 0.8 * total
+
+
+@pytest.mark.parametrize("dtype", [synth.DTYPE_FP32, synth.DTYPE_BF16])
+def test_cold_sampling_is_greedy_and_sampling_is_reproducible(dtype):
+    """Temperatures near zero turn every draw into an arg-max: the sampled loop then returns the tokens of plain
+    greedy decoding of the large model on the GPU.  At ordinary temperatures two runs with one seed agree token for
+    token, another seed gives another response, and self-tandem keeps every draft."""
+    shape = gpu_toy_shape(dtype=dtype)
+    w = toy_weights(shape, seed=77)
+    prompts = prompts_for(shape, [3, 129, 64], seed=1)
+    t = binding.Tandem(shape, w, max_batch=3, max_seq=320, gamma_max=4)
+    t.tandem_prefill(prompts)
+    greedy, _, _ = t.tandem_large_greedy_generate(30)
+    t.tandem_set_sampling(1e-3, 1e-3)
+    t.tandem_prefill(prompts)
+    cold, _, _ = t.tandem_speculative_generate(4, 30, binding.ACCEPT_SAMPLE, 5)
+    assert cold.tolist() == greedy.tolist()
+    t.tandem_set_sampling(1.0, 1.0)
+    runs = []
+    for seed in (5, 5, 6):
+        t.tandem_prefill(prompts)
+        got, lens, st = t.tandem_speculative_generate(4, 30, binding.ACCEPT_SAMPLE, seed)
+        assert lens.tolist() == [30, 30, 30]
+        runs.append(got.tolist())
+    assert runs[0] == runs[1] and runs[0] != runs[2] and runs[0] != greedy.tolist()
+    t.close()
+    dims = synth.ModelDims(3, 128, 4, 256, 97, 128)
+    st_shape = synth.self_tandem_shape(dims, dtype)
+    ws = synth.make_self_tandem_weights(st_shape, seed=4, std=0.08)
+    if dtype == synth.DTYPE_BF16:
+        for k in ws:
+            if not synth.is_norm_param(k):
+                ws[k] = synth.round_to_bf16(ws[k])
+    t = binding.Tandem(st_shape, ws, max_batch=2, max_seq=128, gamma_max=4)
+    t.tandem_set_sampling(0.9, 0.9)
+    t.tandem_prefill(prompts_for(st_shape, [7, 40], seed=2))
+    kept = [int(a) for _ in range(5) for a in t.tandem_block_step(4, binding.ACCEPT_SAMPLE, 3)["accept_len"]]
+    assert sum(a == 4 for a in kept) >= (10 if dtype == synth.DTYPE_FP32 else 7)
+    t.close()
+
+
+@pytest.mark.parametrize("dtype", [synth.DTYPE_FP32, synth.DTYPE_BF16])
+def test_num_samples_share_one_prompt_pass(dtype):
+    """Several sampled responses per query: the prompt is read once per query and its keys / values copied to the
+    query's other sequences.  Everything afterwards must be exactly what a batch of repeated prompts gives: both
+    caches bit for bit, and the sampled responses token for token; the samples of one query differ from each other.
+    In fp32 the first sampled iteration is also replayed against the checker."""
+    shape = gpu_toy_shape(dtype=dtype, layer_map=(1, 3))
+    w = toy_weights(shape, seed=93) if dtype == synth.DTYPE_FP32 else _bf16_weights(shape, seed=93, std=0.06)
+    queries = prompts_for(shape, [131, 1, 18], seed=23)
+    S = 3
+    repeated = [q for q in queries for _ in range(S)]
+    t = binding.Tandem(shape, w, max_batch=9, max_seq=320, gamma_max=3)
+    t.tandem_set_sampling(0.9, 1.0)
+    results = []
+    for shared in (True, False):
+        if shared:
+            t.tandem_prefill_samples(queries, S)
+        else:
+            t.tandem_prefill(repeated)
+        caches = [t.tandem_debug_read(what, layer=1, seq=b) for what in (binding.READ_LARGE_K, binding.READ_SMALL_V) for b in range(9)]
+        first = t.tandem_block_step(3, binding.ACCEPT_SAMPLE, 31)
+        got, lens, _ = t.tandem_speculative_generate(3, 20, binding.ACCEPT_SAMPLE, 31)
+        results.append((caches, first, got.tolist()))
+    for a, b in zip(results[0][0], results[1][0]):
+        assert np.array_equal(a, b)
+    assert results[0][2] == results[1][2]
+    for k in ("drafts", "accept_len", "targets", "n_committed"):
+        assert np.array_equal(results[0][1][k], results[1][1][k])
+    resp = results[0][2]
+    assert resp[0] != resp[1] and resp[3] != resp[4]         # samples of one query diverge (sequence-keyed variates)
+    if dtype == synth.DTYPE_FP32:
+        first = results[0][1]
+        for b, p in enumerate(repeated):
+            o = O.TandemOracle(shape, w)
+            o.prefill(p)
+            r = o.step_sampling(3, 0.9, 1.0, 31, b)
+            assert first["drafts"][b].tolist() == r["drafts"] and first["accept_len"][b] == r["accept_len"]
+            assert first["targets"][b][r["accept_len"]] == r["final"]
+    t.close()
+
+
+# ------------------------------------------------------------------------------------------------
 # multi-query / grouped-query attention (Section 3: either model may use it)
 # ------------------------------------------------------------------------------------------------
 
