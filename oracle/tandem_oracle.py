@@ -38,6 +38,14 @@ Readings taken where the paper is silent or inconsistent:
       p_{gamma+1}.  Every draw uses one uniform variate from a counter-based generator keyed by
       (seed, sequence, iteration, slot): slots 0..gamma-1 draw the drafts, 16+r tests draft r, 48 redraws.
       A draw from weights w with variate u returns the first index whose running sum exceeds u * sum(w).
+  R19 Adaptive block length (Section 3.1 "Adaptive Block Length", Section 4: tau = 0.8).  After every draft the
+      router looks at the small model's distribution q = softmax(logits_S) for that draft: features
+      [entropy of q (nats), the k largest probabilities in descending order (lowest id first on ties), the small
+      model's embedding rows of those k tokens], a two-layer perceptron hidden = relu(W1 x + b1),
+      s = sigmoid(w2 . hidden + b2) = predicted probability that the large model disagrees (what the paper trains
+      it to predict).  The small model goes on drafting while 1 - s >= tau and fewer than gamma_max drafts exist;
+      otherwise the drafts made so far (at least one) are verified as a block of that length.  k, the hidden width
+      and the weights are inputs (the paper gives none); decisions are per sequence.
   R4  Pre-LayerNorm blocks (gain and bias, eps 1e-5, biased variance), exact-erf GELU, no linear
       biases, learned absolute position embeddings, untied output head.
   R6  FF_Tandem MLP variant: hidden width given by the shape, GELU, no biases.
@@ -180,6 +188,36 @@ def accept_probability(p: np.ndarray, q: np.ndarray, token: int) -> float:
 def residual_weights(p: np.ndarray, q: np.ndarray) -> np.ndarray:
     """Unnormalised distribution of the redrawn token after a rejection: the positive part of p - q."""
     return np.maximum(p - q, 0.0)
+
+
+# ----------------------------------------------------------------------------------------------
+# Router of the adaptive block length (R19)
+# ----------------------------------------------------------------------------------------------
+
+class Router:
+    """Two-layer perceptron on [entropy, top-k probabilities, top-k embedding rows] (R19)."""
+
+    def __init__(self, k: int, w1: np.ndarray, b1: np.ndarray, w2: np.ndarray, b2: float, tau: float, dtype=np.float64):
+        self.k, self.tau = int(k), float(tau)
+        self.w1, self.b1 = np.asarray(w1, dtype=dtype), np.asarray(b1, dtype=dtype)
+        self.w2, self.b2 = np.asarray(w2, dtype=dtype), float(b2)
+
+    def features(self, logits: np.ndarray, emb: np.ndarray) -> np.ndarray:
+        q = softmax(np.asarray(logits, dtype=np.float64))
+        nz = q[q > 0]
+        entropy = -(nz * np.log(nz)).sum()
+        top = np.argsort(-q, kind="stable")[: self.k]          # descending probability, lowest id first on ties
+        return np.concatenate([[entropy], q[top]] + [emb[t] for t in top])
+
+    def disagreement(self, logits: np.ndarray, emb: np.ndarray) -> float:
+        x = self.features(logits, emb)
+        hidden = np.maximum(self.w1 @ x + self.b1, 0.0)
+        return float(1.0 / (1.0 + np.exp(-(self.w2 @ hidden + self.b2))))
+
+    def keep_drafting(self, logits: np.ndarray, emb: np.ndarray) -> Tuple[bool, float]:
+        """(whether the small model may go on, the confidence 1 - s compared with tau)."""
+        conf = 1.0 - self.disagreement(logits, emb)
+        return conf >= self.tau, conf
 
 
 # ----------------------------------------------------------------------------------------------
@@ -537,6 +575,48 @@ class TandemOracle:
         while len(self.tokens) - P < max_new:
             accepts.append(self.step_sampling(gamma, temp_large, temp_small, seed, seq)["accept_len"])
         return self.tokens[P:P + max_new], accepts
+
+    def step_adaptive(self, gamma_max: int, router: "Router", forced_len: Optional[int] = None,
+                      forced_drafts: Optional[Sequence[int]] = None) -> dict:
+        """One greedy Tandem + SPEED iteration whose block length the router chooses (R19): draft, ask the router,
+        stop at its first "verify now" or at gamma_max, then verify exactly the drafts made.  With `forced_len` /
+        `forced_drafts` (another implementation's block length and draft ids) those are followed; the router's
+        confidences are returned either way so that the caller can check each decision."""
+        n = len(self.tokens)
+        assert self.derived.length() == n - 1 and self.own.length() == 0 and gamma_max >= 1
+        u = self.tokens[-1]
+        drafts, own_drafts, s_logits, confs = [], [], [], []
+        own_len = None
+        s_ = 0
+        while True:
+            lg = self._small_step(u, n - 1 + s_)
+            d = argmax_decision(lg)
+            own_drafts.append(d)
+            u = int(forced_drafts[s_]) if forced_drafts is not None else d
+            drafts.append(u)
+            s_logits.append(lg)
+            go_on, conf = router.keep_drafting(lg, self.small.emb)
+            confs.append(conf)
+            s_ += 1
+            if own_len is None and (not go_on or s_ == gamma_max):
+                own_len = s_
+            if (forced_len is None and own_len is not None) or (forced_len is not None and s_ == forced_len):
+                break
+        targets, l_logits, reps = self.verify(drafts)
+        a = self.accept_length(drafts, targets)
+        emitted = self.commit(a, drafts, targets, reps)
+        return {"drafts": drafts, "own_drafts": own_drafts, "block_len": len(drafts), "own_block_len": own_len,
+                "confidences": confs, "targets": targets, "accept_len": a, "emitted": emitted, "small_logits": s_logits,
+                "large_logits": l_logits, "n_committed": len(self.tokens)}
+
+    def generate_adaptive(self, prompt: Sequence[int], gamma_max: int, max_new: int, router: "Router") -> Tuple[List[int], List[int]]:
+        """Full response with the adaptive block length; returns (tokens, block length of every iteration)."""
+        self.prefill(prompt)
+        P = len(prompt)
+        lens = []
+        while len(self.tokens) - P < max_new:
+            lens.append(self.step_adaptive(gamma_max, router)["block_len"])
+        return self.tokens[P:P + max_new], lens
 
     def step(self, gamma: int, mode: int = ACCEPT_NATURAL, mode_seed: int = 0, seq: int = 0) -> dict:
         drafts, s_logits = self.draft(gamma)

@@ -216,3 +216,15 @@ def device_weights(shape: TandemShape, seed: int, device) -> Dict[str, "torch.Te
         else:
             out[name] = (torch.randn(shp, generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
     return out
+
+
+def make_router(shape: TandemShape, k: int, hidden: int, seed: int) -> Dict[str, np.ndarray]:
+    """Random-init weights of the adaptive-block-length router (a stand-in for the trained router of Section 3.1):
+    w1 [hidden][1 + k + k * d_small] ~ N(0, 1 / fan_in), b1 [hidden] ~ N(0, 0.1^2), w2 [hidden] ~ N(0, 1 / hidden),
+    b2 scalar 0.  float32."""
+    f = 1 + k + k * shape.small.d_model
+    gen = np.random.Generator(np.random.Philox(key=[seed & 0xFFFFFFFFFFFFFFFF, 0xA6]))
+    return {"k": k, "w1": (gen.standard_normal((hidden, f), dtype=np.float32) / np.float32(np.sqrt(f))).astype(np.float32),
+            "b1": (gen.standard_normal(hidden, dtype=np.float32) * np.float32(0.1)).astype(np.float32),
+            "w2": (gen.standard_normal(hidden, dtype=np.float32) / np.float32(np.sqrt(hidden))).astype(np.float32),
+            "b2": np.float32(0.0)}
