@@ -295,7 +295,8 @@ def measure_workload(name, steps, warmup, rank, local_rank, world, extras, keep_
     else:
         weights = synth.make_weights(shape, seed=0)
     prompts = [[int(t) for t in p] for p in synth.make_prompts(B, P, shape.large.vocab, seed=rank)]
-    t = binding.Tandem(shape, weights, max_batch=B, max_seq=P + new + gamma + 1, gamma_max=gamma, device=local_rank,
+    gmax = 2 * gamma if extras else gamma     # the adaptive block length of the extras drafts up to 2 gamma tokens
+    t = binding.Tandem(shape, weights, max_batch=B, max_seq=P + new + gmax + 1, gamma_max=gmax, device=local_rank,
                        max_prefill_rows=B * P)
     stream = torch.cuda.current_stream()
 
@@ -372,6 +373,15 @@ def measure_workload(name, steps, warmup, rank, local_rank, world, extras, keep_
         r["sampled_decode_ms"] = timed_decode(sampled, 2)
         t.tandem_prefill(prompts)
         r["sampled_accept_hist"] = sampled()[2]["accept_hist"]
+        # adaptive block length with a random-init router (mechanism only: the paper's router is trained); gamma_max = 2 gamma
+        if t.gamma_max >= 2 * gamma:
+            t.tandem_set_router(synth.make_router(shape, 4, 64, seed=0), 0.5)
+            adaptive = lambda: t.tandem_adaptive_generate(2 * gamma, new)
+            t.tandem_prefill(prompts); adaptive(); t.tandem_prefill(prompts); adaptive()
+            r["adaptive_decode_ms"] = timed_decode(adaptive, 2)
+            t.tandem_prefill(prompts)
+            st = adaptive()[2]
+            r["adaptive_runs"] = {"large_runs": st["large_runs"], "small_runs": st["small_runs"], "gamma_max": 2 * gamma, "tau": 0.5}
         # per-kernel pass: the same step with every launch bracketed by events (serialises the stream: shares only)
         t.tandem_profile_enable(400000)
         t.tandem_prefill(prompts)
@@ -415,6 +425,9 @@ def sub_record(r, peak):
         rec["standalone_representation_only_decode_tokens_per_s"] = toks / (r["representation_only_decode_ms"] * 1e-3)
         rec["sampled_decode_tokens_per_s"] = toks / (r["sampled_decode_ms"] * 1e-3)
         rec["sampled_accept_hist"] = r["sampled_accept_hist"]
+        if "adaptive_decode_ms" in r:
+            rec["adaptive_decode_tokens_per_s"] = toks / (r["adaptive_decode_ms"] * 1e-3)
+            rec["adaptive_runs"] = r["adaptive_runs"]
     return rec
 
 
@@ -452,6 +465,9 @@ def run_ours(args, rank, local_rank, world):
         line["standalone_representation_only_decode_tokens_per_s"] = toks / (r["representation_only_decode_ms"] * 1e-3)
         line["sampled_decode_tokens_per_s"] = toks / (r["sampled_decode_ms"] * 1e-3)
         line["sampled_accept_hist"] = r["sampled_accept_hist"]
+        if "adaptive_decode_ms" in r:
+            line["adaptive_decode_tokens_per_s"] = toks / (r["adaptive_decode_ms"] * 1e-3)
+            line["adaptive_runs"] = r["adaptive_runs"]
         tot = sum(v["ms"] for v in prof.values()) or 1.0
         # bracketed pass: work = algorithmic bytes (GB/s) for the streaming kernels, flops (TFLOP/s) for the prompt pass
         line["kernels_bracketed"] = {

@@ -198,6 +198,30 @@ TANDEM_API tandem_status tandem_speculative_generate(tandem_ctx* ctx, int32_t ga
  * iterations enqueued afterwards; waits for the context's stream when a value changes. */
 TANDEM_API tandem_status tandem_set_sampling(tandem_ctx* ctx, float temp_large, float temp_small);
 
+/* Adaptive block length (Section 3.1 "Adaptive Block Length"; Section 4: tau = 0.8; Tables 5-6).  After every
+ * draft a router looks at M_S's distribution q = softmax(logits_S) for that draft and decides, per sequence, whether
+ * M_S goes on drafting or the drafts made so far are verified.  Features: [entropy of q in nats, the top_k largest
+ * probabilities in descending order (lowest id first on ties), M_S's embedding rows of those top_k tokens], length
+ * F = 1 + top_k + top_k * d_small.  Router: hidden = relu(w1 x + b1), s = sigmoid(w2 . hidden + b2) = predicted
+ * probability that M_L disagrees; drafting continues while 1 - s >= tau and fewer than gamma_max drafts exist.
+ *
+ * tandem_set_router: w1 [hidden][F], b1 [hidden], w2 [hidden]: DEVICE, fp32, caller-owned, valid until replaced or
+ * the context is destroyed; 1 <= top_k <= 8.  (The paper's router is trained; any weights can be passed.)
+ * tandem_adaptive_step: one iteration with the natural (arg-max) comparison.  result arrays are sized by gamma_max
+ * ([batch][gamma_max] drafts, [batch][gamma_max+1] targets); entries beyond a sequence's own block are -1.
+ * block_len: HOST [batch], drafts each sequence made; confidence: HOST [batch][gamma_max], the router's 1 - s per
+ * draft (0 beyond the block); both nullable.  Synchronous: the host reads, after every draft step, how many
+ * sequences still draft, launches no further draft step once none does, and sizes M_L's block by the longest block
+ * of the batch (rows beyond a sequence's own block are computed and ignored).
+ * tandem_adaptive_generate: repeats it until every sequence has max_new_tokens; stats->small_runs counts the draft
+ * steps executed, stats->large_runs the verify passes (the two columns of Table 6). */
+TANDEM_API tandem_status tandem_set_router(tandem_ctx* ctx, int32_t top_k, int32_t hidden, const void* w1, const void* b1,
+                                           const void* w2, float b2, float tau);
+TANDEM_API tandem_status tandem_adaptive_step(tandem_ctx* ctx, int32_t gamma_max, tandem_step_result* result,
+                                              int32_t* block_len, float* confidence);
+TANDEM_API tandem_status tandem_adaptive_generate(tandem_ctx* ctx, int32_t gamma_max, int32_t max_new_tokens,
+                                                  int32_t* out_ids, int32_t* out_lens, tandem_stats* stats);
+
 /* Stand-alone Tandem decoding (Section 3 "Inference"; Table 3's latency row): M_S writes the response, M_L only
  * supplies representations (and, with the free token, one token per block); nothing is verified.  Must follow
  * tandem_prefill; same buffers and stop rule as tandem_speculative_generate; 1 <= gamma <= gamma_max.

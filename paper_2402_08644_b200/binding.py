@@ -31,7 +31,8 @@ EXPORTS = ["tandem_query_arena", "tandem_create", "tandem_destroy", "tandem_pref
            "tandem_status_string", "tandem_last_cuda_error", "tandem_profile_enable", "tandem_profile_read",
            "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static",
            "tandem_debug_expire_wait", "tandem_standalone_check", "tandem_standalone_generate",
-           "tandem_set_sampling", "tandem_prefill_samples"]
+           "tandem_set_sampling", "tandem_prefill_samples", "tandem_set_router", "tandem_adaptive_step",
+           "tandem_adaptive_generate"]
 
 
 class TandemError(RuntimeError):
@@ -93,6 +94,9 @@ def load_library():
     lib.tandem_large_greedy_generate.argtypes = [vp, i32, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_standalone_generate.argtypes = [vp, i32, i32, i32, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_set_sampling.argtypes = [vp, C.c_float, C.c_float]
+    lib.tandem_set_router.argtypes = [vp, i32, i32, vp, vp, vp, C.c_float, C.c_float]
+    lib.tandem_adaptive_step.argtypes = [vp, i32, C.POINTER(StepResult), pi32, C.POINTER(C.c_float)]
+    lib.tandem_adaptive_generate.argtypes = [vp, i32, i32, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_debug_read.argtypes = [vp, i32, i32, i32, vp, sz]
     lib.tandem_decode_attention_scratch_bytes.argtypes = [i32] * 5
     lib.tandem_decode_attention_scratch_bytes.restype = sz
@@ -242,6 +246,33 @@ class Tandem:
 
     def tandem_set_sampling(self, temp_large: float, temp_small: float) -> None:
         _check(self.lib.tandem_set_sampling(self.ctx, temp_large, temp_small), "tandem_set_sampling")
+
+    def tandem_set_router(self, router: Dict[str, np.ndarray], tau: float) -> None:
+        """router: {"k", "w1" [hidden][F], "b1", "w2", "b2"} as made by synth.make_router; kept on the device here."""
+        import torch
+        self._router = {n: torch.from_numpy(np.ascontiguousarray(router[n], dtype=np.float32)).to(self.device) for n in ("w1", "b1", "w2")}
+        _check(self.lib.tandem_set_router(self.ctx, int(router["k"]), int(router["w1"].shape[0]), C.c_void_p(self._router["w1"].data_ptr()),
+                                          C.c_void_p(self._router["b1"].data_ptr()), C.c_void_p(self._router["w2"].data_ptr()),
+                                          float(router["b2"]), float(tau)), "tandem_set_router")
+
+    def tandem_adaptive_step(self, gamma_max: int):
+        B = self.batch
+        d = np.zeros((B, gamma_max), np.int32); t = np.zeros((B, gamma_max + 1), np.int32)
+        a = np.zeros(B, np.int32); n = np.zeros(B, np.int32); bl = np.zeros(B, np.int32)
+        cf = np.zeros((B, gamma_max), np.float32)
+        p = lambda x: x.ctypes.data_as(C.POINTER(C.c_int32))
+        res = StepResult(p(d), p(t), p(a), p(n))
+        _check(self.lib.tandem_adaptive_step(self.ctx, gamma_max, C.byref(res), p(bl), cf.ctypes.data_as(C.POINTER(C.c_float))),
+               "tandem_adaptive_step")
+        return {"drafts": d, "targets": t, "accept_len": a, "n_committed": n, "block_len": bl, "confidence": cf}
+
+    def tandem_adaptive_generate(self, gamma_max: int, max_new: int):
+        out = np.zeros((self.batch, max_new), np.int32)
+        lens = np.zeros(self.batch, np.int32)
+        st = Stats()
+        p = lambda x: x.ctypes.data_as(C.POINTER(C.c_int32))
+        _check(self.lib.tandem_adaptive_generate(self.ctx, gamma_max, max_new, p(out), p(lens), C.byref(st)), "tandem_adaptive_generate")
+        return out, lens, self._stats(st, gamma_max)
 
     def tandem_standalone_generate(self, gamma: int, variant: int, max_new: int):
         out = np.zeros((self.batch, max_new), np.int32)

@@ -19,8 +19,14 @@ struct LoopState {
     int* out_ids;      // [B][out_cap]
     int* counters;     // [0] iteration index since prefill (advances while sequences are live), [1] live sequences,
                        // [2] error flags, [3] max_b n_b, [4] sum_b n_b, [5] live iterations of the current call,
-                       // [6] verify kernels executed since the context was created (the host's ticket)
-    volatile int* host_flags;   // mapped pinned host memory: [0] ticket, [1] live, [2] n_max, [3] n_sum, [4] iterations
+                       // [6] verify kernels executed since the context was created (the host's ticket),
+                       // [7] sequences still drafting (adaptive block length), [8] router launches since the prompt pass,
+                       // [9] CTAs of the running router launch that have finished
+    volatile int* host_flags;   // mapped pinned host memory: [0] ticket, [1] live, [2] n_max, [3] n_sum, [4] iterations,
+                                // [5] router ticket, [6] sequences still drafting
+    int* block_len;    // [B] adaptive block length: drafts made in the current iteration
+    int* drafting;     // [B] adaptive block length: 1 while the router lets the sequence go on drafting
+    float* confidence; // [B][gamma_limit] the router's 1 - s for every draft of the current iteration
     unsigned long long* hist;   // [gamma_limit+1] accept-length histogram of live sequences
     int out_cap;
     int gamma_limit;
@@ -258,10 +264,11 @@ __global__ void __launch_bounds__(256) argmax_rows_kernel(const float* __restric
 // turned it into a token id yet: when fin_val is given it is finished here from the small head's per-tile results.
 // mode 4 is sampled SPEED: sample_verify_kernel has already written each sequence's accept length and, at that index
 // of its targets, the token drawn after the kept drafts; this kernel only does the bookkeeping.
+// block_len (nullable): per-sequence number of drafts of this iteration when the router chose it.
 // block: 256.
 __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, int gamma, int mode, unsigned long long seed,
                                                      int max_new, const float* amax_val, const int* amax_idx, int amax_stride,
-                                                     int n_tiles, const float* fin_val, const int* fin_idx) {
+                                                     int n_tiles, const float* fin_val, const int* fin_idx, const int* block_len) {
     pdl_wait();
     pdl_launch_dependents();
     if (mode == 3) {
@@ -291,7 +298,10 @@ __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, in
         if (mode == 1 || mode == 3) a = gamma;
         else if (mode == 4) a = min(max(st.accept_len[b], 0), gamma);   // sampled SPEED: decided by sample_verify_kernel, with g[a] the token it drew
         else if (mode == 2) a = (int)(splitmix64(splitmix64(splitmix64(seed) ^ (unsigned long long)b) ^ (unsigned long long)iteration) % (unsigned long long)(gamma + 1));
-        else { while (a < gamma && d[a] == g[a]) ++a; }
+        else {   // adaptive block length: only the drafts the sequence really made count (later rows are dead)
+            const int gamma_b = block_len ? min(block_len[b], gamma) : gamma;
+            while (a < gamma_b && d[a] == g[a]) ++a;
+        }
         st.accept_len[b] = a;
         atomicAdd(st.hist + a, 1ull);
         const int em = st.emitted[b];

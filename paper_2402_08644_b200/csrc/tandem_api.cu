@@ -19,6 +19,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "misc_kernels.cuh"
+#include "router.cuh"
 #include "sampling.cuh"
 
 using namespace tandem;
@@ -47,6 +48,7 @@ int cdiv(int a, int b) { return (a + b - 1) / b; }
 struct Layout {   // byte offsets into the arena
     size_t kv_large, kv_small;
     size_t st_n, st_pending, st_drafts, st_targets, st_accept, st_emitted, st_done, st_out, st_counters, st_hist;
+    size_t st_block_len, st_drafting, st_confidence;
     size_t row_tok, row_seq, row_pos, grp_row0, grp_cnt;
     size_t attn_counters;   // inside the zero-filled state block
     size_t h_large, h_small, a, q, o, f, xb, t1, yhat, a_s, logits_large, logits_small, part_ml, part_acc, dbg;
@@ -129,6 +131,9 @@ struct tandem_ctx {
     bool tc_prompt_attn = false;         // prompt attention on the tensor cores (head size 64 or 128)
     int prompt_group = ATT_NQ;           // queries per attention group of the prompt pass
     float temp_large = 1.0f, temp_small = 1.0f;   // sampled SPEED (accept mode 4): temperatures of the two models
+    RouterArgs router{};                 // adaptive block length: the router's weights (caller-owned, DEVICE) and threshold
+    bool has_router = false;
+    int64_t router_ticket = 0;           // router launches since the prompt pass
 };
 
 namespace {
@@ -204,6 +209,7 @@ Layout make_layout(const tandem_config& c) {
     L.st_n = take(B * 4); L.st_pending = take(B * 4); L.st_drafts = take(B * GL * 4);
     L.st_targets = take(B * (GL + 1) * 4); L.st_accept = take(B * 4); L.st_emitted = take(B * 4);
     L.st_done = take(B * 4); L.st_out = take(B * T * 4); L.st_counters = take(16 * 4); L.st_hist = take((GL + 1) * 8);
+    L.st_block_len = take(B * 4); L.st_drafting = take(B * 4); L.st_confidence = take(B * GL * 4);
     L.row_tok = take(R * 4); L.row_seq = take(R * 4); L.row_pos = take(R * 4);
     L.grp_row0 = take((size_t)L.max_groups * 4); L.grp_cnt = take((size_t)L.max_groups * 4);
     L.attn_counters = take(B * hmax * 4);
@@ -766,13 +772,30 @@ void small_step(tandem_ctx& c, int s) {
     head_argmax<T>(c, c.small, y, r, logits, c.st.drafts, TANDEM_GAMMA_LIMIT, s);
 }
 
-void launch_verify(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new, bool from_tiles) {
+void launch_verify(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new, bool from_tiles, bool adaptive = false) {
     ProfScope ps(c, PC_VERIFY, (double)c.batch * (2 * gamma + 8) * 4.0);
     launch_ex(c, true, 1, verify_kernel, dim3(1), dim3(256), 0, c.st, c.batch, gamma, mode, (unsigned long long)seed, max_new,
               from_tiles ? (const float*)at<float>(c, c.lay.amax_val_large) : (const float*)nullptr,
               from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_large) : (const int*)nullptr, c.lay.vocab_tiles, c.lay.vocab_tiles,
               from_tiles ? (const float*)at<float>(c, c.lay.amax_val_small) : (const float*)nullptr,
-              from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_small) : (const int*)nullptr);
+              from_tiles ? (const int*)at<int>(c, c.lay.amax_idx_small) : (const int*)nullptr,
+              adaptive ? (const int*)c.st.block_len : (const int*)nullptr);
+}
+
+// Adaptive block length: the router's decision after draft step s, for every sequence that is still drafting.
+void launch_router(tandem_ctx& c, int s, int gamma_max) {
+    const float* logits = at<float>(c, c.lay.logits_small) + (size_t)s * c.batch * c.small.d.vocab;
+    ProfScope ps(c, PC_ARGMAX, (double)c.batch * c.small.d.vocab * 4.0 * (2 + c.router.k));
+    if (c.cfg.dtype == TANDEM_DTYPE_BF16)
+        launch_ex(c, true, 1, router_kernel<bf16>, dim3(c.batch), dim3(RT_THREADS), 0, c.st, c.batch, logits, (int)c.small.d.vocab, s, gamma_max,
+                  (const bf16*)w_emb(c, c.small), (int)c.small.d.d_model, c.router);
+    else
+        launch_ex(c, true, 1, router_kernel<float>, dim3(c.batch), dim3(RT_THREADS), 0, c.st, c.batch, logits, (int)c.small.d.vocab, s, gamma_max,
+                  (const float*)w_emb(c, c.small), (int)c.small.d.d_model, c.router);
+}
+void launch_adaptive_begin(tandem_ctx& c) {
+    ProfScope ps(c, PC_ROWS, (double)c.batch * 8.0);
+    launch_ex(c, true, 1, adaptive_begin_kernel, dim3(1), dim3(256), 0, c.st, c.batch);
 }
 
 // Sampled SPEED: draft s of every sequence drawn from the small model's logits of step s.
@@ -990,8 +1013,29 @@ tandem_status check_launch(tandem_ctx& c) {
     return check_launch();
 }
 
+// kind 0: draft + verify (gamma drafts, accept mode);  1: plain greedy M_L;
+// kind 3: one draft step of the adaptive block length (gamma = step index, mode = gamma_max) followed by the router;
+// kind 4: the verify half of an adaptive iteration (gamma = longest block of the batch).
 void enqueue_iteration(tandem_ctx& c, int kind, int gamma, int mode, uint64_t seed, int max_new) {
-    if (c.cfg.dtype == TANDEM_DTYPE_BF16) {   // one bf16 path: the tensor-core kernels (a bf16 context always has tensor maps)
+    const bool bf = c.cfg.dtype == TANDEM_DTYPE_BF16;   // one bf16 path: the tensor-core kernels (a bf16 context always has tensor maps)
+    if (kind == 3) {
+        if (gamma == 0) launch_adaptive_begin(c);
+        if (bf) tc_small_step(c, gamma, false); else small_step<float>(c, gamma);
+        launch_router(c, gamma, mode);
+        return;
+    }
+    if (kind == 4) {
+        if (bf) {
+            tc_large_block(c, gamma + 1, gamma, true, true);
+        } else {
+            setup_rows(c, 0, gamma + 1);
+            large_pass<float>(c, decode_rows(c, gamma, gamma + 1), true, true);
+        }
+        launch_verify(c, gamma, TANDEM_ACCEPT_NATURAL, 0ull, max_new, bf, true);
+        c.last_gamma = gamma;
+        return;
+    }
+    if (bf) {
         if (kind == 0) tc_iteration(c, gamma, mode, seed, max_new); else tc_greedy_iteration(c, max_new);
         return;
     }
@@ -1006,7 +1050,8 @@ tandem_status launch_iteration(tandem_ctx& c, int kind, int gamma, int mode, uin
     c.chunks_launch = std::min(c.lay.n_chunks_max, (need + 3) / 4 * 4);
     if (c.cfg.dtype == TANDEM_DTYPE_BF16)
         c.chunks_launch = 1;   // the cluster attention's grid does not depend on the context length: one graph serves all
-    c.ticket++;
+    if (kind == 3) c.router_ticket++; else c.ticket++;   // what the host will wait for: the router's or the verify kernel's publication
+    if (kind != 3) c.last_gamma = kind == 1 ? 0 : gamma;   // (set here, not while enqueueing: a replayed graph enqueues nothing on the host)
     if (c.prof.on || !c.use_graphs) {
         enqueue_iteration(c, kind, gamma, mode, seed, max_new);
         return check_launch();
@@ -1048,9 +1093,10 @@ tandem_status launch_iteration(tandem_ctx& c, int kind, int gamma, int mode, uin
     return TANDEM_OK;
 }
 
-// Waits (bounded) until the verify kernel with the given ticket has published its results to the host.
-tandem_status wait_ticket(tandem_ctx& c, int64_t ticket) {
-    volatile int32_t* hf = c.hflags;
+// Waits (bounded) until the kernel that publishes into slot `slot` of the host flags (0: verify kernel, 5: router)
+// has reached the given ticket.
+tandem_status wait_ticket(tandem_ctx& c, int64_t ticket, int slot = 0) {
+    volatile int32_t* hf = c.hflags + slot;
     struct timespec t0, t1;
     clock_gettime(CLOCK_MONOTONIC, &t0);
     for (unsigned spin = 0; (int64_t)hf[0] < ticket; ++spin) {
@@ -1156,6 +1202,8 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
     st.targets = at<int>(*c, lay.st_targets); st.accept_len = at<int>(*c, lay.st_accept); st.emitted = at<int>(*c, lay.st_emitted);
     st.done = at<int>(*c, lay.st_done); st.out_ids = at<int>(*c, lay.st_out); st.counters = at<int>(*c, lay.st_counters);
     st.hist = at<unsigned long long>(*c, lay.st_hist);
+    st.block_len = at<int>(*c, lay.st_block_len); st.drafting = at<int>(*c, lay.st_drafting);
+    st.confidence = at<float>(*c, lay.st_confidence);
     st.out_cap = cfg->max_seq; st.gamma_limit = TANDEM_GAMMA_LIMIT;
     cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&c->pinned), c->pinned_ints * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaHostAlloc(reinterpret_cast<void**>(&c->hflags), 16 * sizeof(int32_t), cudaHostAllocMapped);
@@ -1282,8 +1330,10 @@ tandem_status prefill_impl(tandem_ctx* c, int n_queries, int samples, const int3
         if (prompt_ids[i] < 0 || prompt_ids[i] >= c->cfg.large.vocab) return TANDEM_ERR_INVALID_ARG;
 
     CK(cudaStreamSynchronize(c->stream));   // staging buffer free again; no verify kernel in flight
-    c->ticket = 0;                          // the device-side ticket is cleared with the rest of the loop state below
+    c->ticket = 0;                          // the device-side tickets are cleared with the rest of the loop state below
+    c->router_ticket = 0;
     c->hflags[0] = 0;
+    c->hflags[5] = 0;
     const int M = (int)rows;
     int32_t* p_tok = c->pinned;
     int32_t* p_seq = p_tok + c->lay.max_rows;
@@ -1494,6 +1544,129 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
 }
 
 }  // namespace
+
+namespace {
+
+// One adaptive iteration, synchronous: draft steps until the router has stopped every sequence (the host reads the
+// count the router publishes after each step) or gamma_max drafts exist, then one verify pass over the longest block.
+tandem_status adaptive_iteration(tandem_ctx* c, int gamma_max, int max_new, int* block_max) {
+    int s = 0;
+    for (; s < gamma_max; ++s) {
+        TRY(launch_iteration(*c, 3, s, gamma_max, 0ull, max_new));
+        TRY(wait_ticket(*c, c->router_ticket, 5));
+        if (c->hflags[6] <= 0) { ++s; break; }
+    }
+    *block_max = s;
+    TRY(launch_iteration(*c, 4, s, 0, 0ull, max_new));
+    TRY(wait_ticket(*c, c->ticket, 0));
+    c->n_ub = c->hflags[2];
+    c->n_sum = c->hflags[3];
+    return TANDEM_OK;
+}
+
+tandem_status check_error_word(tandem_ctx* c) {
+    int32_t* cnt = c->pinned;   // staging is idle outside prefill
+    CK(cudaMemcpyAsync(cnt, c->st.counters, 8 * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (cnt[2] != 0) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "device-side wait expired (code %d)", cnt[2]);
+        CK(cudaMemsetAsync(c->st.counters + 2, 0, 4, c->stream));
+        return TANDEM_ERR_TIMEOUT;
+    }
+    return TANDEM_OK;
+}
+
+}  // namespace
+
+extern "C" tandem_status tandem_set_router(tandem_ctx* c, int32_t top_k, int32_t hidden, const void* w1, const void* b1, const void* w2,
+                                           float b2, float tau) {
+    TRY(begin_call(c));
+    if (!w1 || !b1 || !w2 || top_k < 1 || top_k > RT_MAX_K || hidden < 1 || top_k > c->cfg.small.vocab) return TANDEM_ERR_INVALID_ARG;
+    if (((uintptr_t)w1 | (uintptr_t)b1 | (uintptr_t)w2) & 3) return TANDEM_ERR_INVALID_ARG;
+    CK(cudaStreamSynchronize(c->stream));
+    for (auto& g : c->graphs)   // the router's arguments are baked into the captured draft steps
+        if (g.kind == 3 && g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+    c->router.w1 = static_cast<const float*>(w1); c->router.b1 = static_cast<const float*>(b1); c->router.w2 = static_cast<const float*>(w2);
+    c->router.b2 = b2; c->router.tau = tau; c->router.k = top_k; c->router.hidden = hidden;
+    c->has_router = true;
+    return TANDEM_OK;
+}
+
+extern "C" tandem_status tandem_adaptive_step(tandem_ctx* c, int32_t gamma_max, tandem_step_result* result, int32_t* block_len,
+                                              float* confidence) {
+    TRY(begin_call(c));
+    if (gamma_max < 1 || gamma_max > c->cfg.gamma_max) return TANDEM_ERR_INVALID_ARG;
+    if (c->batch == 0 || !c->has_router) return TANDEM_ERR_STATE;
+    TRY(capacity_for(c, 0, gamma_max));
+    reset_call_kernel<<<1, 256, 0, c->stream>>>(c->st, c->batch);
+    c->launches++;
+    int block_max = 0;
+    TRY(adaptive_iteration(c, gamma_max, INT_MAX, &block_max));
+    TRY(check_error_word(c));
+    const int B = c->batch, GL = TANDEM_GAMMA_LIMIT;
+    std::vector<int32_t> d((size_t)B * GL), t((size_t)B * (GL + 1)), acc((size_t)B), ncm((size_t)B), bl((size_t)B);
+    std::vector<float> cf((size_t)B * GL);
+    CK(cudaMemcpyAsync(d.data(), c->st.drafts, d.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(t.data(), c->st.targets, t.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(acc.data(), c->st.accept_len, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(ncm.data(), c->st.n, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(bl.data(), c->st.block_len, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(cf.data(), c->st.confidence, cf.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    for (int b = 0; b < B; ++b) {
+        for (int i = 0; i < gamma_max; ++i) {   // entries beyond a sequence's own block length are -1 / 0
+            const bool own = i < bl[b];
+            if (result && result->drafts) result->drafts[b * gamma_max + i] = own ? d[(size_t)b * GL + i] : -1;
+            if (confidence) confidence[b * gamma_max + i] = own ? cf[(size_t)b * GL + i] : 0.f;
+        }
+        if (result && result->targets) for (int i = 0; i <= gamma_max; ++i)
+            result->targets[b * (gamma_max + 1) + i] = i <= bl[b] ? t[(size_t)b * (GL + 1) + i] : -1;
+        if (result && result->accept_len) result->accept_len[b] = acc[b];
+        if (result && result->n_committed) result->n_committed[b] = ncm[b];
+        if (block_len) block_len[b] = bl[b];
+    }
+    return TANDEM_OK;
+}
+
+extern "C" tandem_status tandem_adaptive_generate(tandem_ctx* c, int32_t gamma_max, int32_t max_new, int32_t* out_ids, int32_t* out_lens,
+                                                  tandem_stats* stats) {
+    TRY(begin_call(c));
+    if (gamma_max < 1 || gamma_max > c->cfg.gamma_max || !out_ids || max_new < 1) return TANDEM_ERR_INVALID_ARG;
+    if (c->batch == 0 || !c->has_router) return TANDEM_ERR_STATE;
+    if (max_new > c->cfg.max_seq) return TANDEM_ERR_CAPACITY;
+    TRY(capacity_for(c, max_new, gamma_max));
+    const int B = c->batch;
+    const int64_t launches0 = c->launches;
+    reset_call_kernel<<<1, 256, 0, c->stream>>>(c->st, B);
+    c->launches++;
+    CK(cudaMemsetAsync(c->st.hist, 0, (TANDEM_GAMMA_LIMIT + 1) * 8, c->stream));
+    int64_t iters = 0, small_runs = 0;
+    for (;;) {
+        if (iters > max_new) return TANDEM_ERR_STATE;   // every live iteration emits a token
+        int block_max = 0;
+        TRY(adaptive_iteration(c, gamma_max, max_new, &block_max));
+        ++iters;
+        small_runs += block_max;
+        if (c->hflags[1] <= 0) break;
+    }
+    TRY(check_error_word(c));
+    CK(cudaMemcpy2DAsync(out_ids, (size_t)max_new * 4, c->st.out_ids, (size_t)c->st.out_cap * 4, (size_t)max_new * 4, B,
+                         cudaMemcpyDeviceToHost, c->stream));
+    std::vector<unsigned long long> hist(TANDEM_GAMMA_LIMIT + 1);
+    CK(cudaMemcpyAsync(hist.data(), c->st.hist, hist.size() * 8, cudaMemcpyDeviceToHost, c->stream));
+    if (out_lens) CK(cudaMemcpyAsync(out_lens, c->st.emitted, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (stats) {
+        memset(stats, 0, sizeof(*stats));
+        stats->iterations = iters;
+        stats->large_runs = iters;
+        stats->small_runs = small_runs;
+        stats->emitted = (int64_t)B * max_new;
+        for (int i = 0; i <= TANDEM_GAMMA_LIMIT; ++i) stats->accept_hist[i] = (int64_t)hist[i];
+        stats->kernel_launches = c->launches - launches0;
+    }
+    return TANDEM_OK;
+}
 
 extern "C" tandem_status tandem_speculative_generate(tandem_ctx* c, int32_t gamma, int32_t max_new_tokens, int32_t accept_mode,
                                                      uint64_t mode_seed, int32_t* out_ids, int32_t* out_lens, tandem_stats* stats) {

@@ -712,6 +712,111 @@ def test_num_samples_share_one_prompt_pass(dtype):
 
 
 # ------------------------------------------------------------------------------------------------
+# adaptive block length (Section 3.1)
+# ------------------------------------------------------------------------------------------------
+
+def _median_tau(shape, w, prompts, router, gamma_max):
+    """A threshold in the middle of the confidences this router shows on these prompts, so that both of its
+    decisions occur (the paper's router is trained; a random one needs its threshold placed)."""
+    always = O.Router(router["k"], router["w1"], router["b1"], router["w2"], router["b2"], -1.0)
+    confs = []
+    for p in prompts:
+        o = O.TandemOracle(shape, w)
+        o.prefill(p)
+        for _ in range(2):
+            confs += o.step_adaptive(gamma_max, always)["confidences"]
+    return float(np.median(confs))
+
+
+def _adaptive_replay(shape, w, prompts, gamma_max, iters, tol, eps):
+    router = synth.make_router(shape, 3, 16, seed=7)
+    tau = _median_tau(shape, w, prompts, router, gamma_max)
+    orouter = O.Router(router["k"], router["w1"], router["b1"], router["w2"], router["b2"], tau)
+    t = binding.Tandem(shape, w, max_batch=len(prompts), max_seq=shape.large.max_pos, gamma_max=gamma_max)
+    t.tandem_set_router(router, tau)
+    t.tandem_prefill(prompts)
+    oracles = [O.TandemOracle(shape, w) for _ in prompts]
+    for o, p in zip(oracles, prompts):
+        o.prefill(p)
+    lens, same = [], 0
+    for it in range(iters):
+        res = t.tandem_adaptive_step(gamma_max)
+        gmax = int(res["block_len"].max())
+        s_logits = t.tandem_debug_read(binding.READ_SMALL_LOGITS, gmax)
+        for b, o in enumerate(oracles):
+            n = int(res["block_len"][b])
+            g_drafts = res["drafts"][b][:n].tolist()
+            assert 1 <= n <= gamma_max and (res["drafts"][b][n:] == -1).all() and (res["targets"][b][n + 1:] == -1).all()
+            r = o.step_adaptive(gamma_max, orouter, forced_len=n, forced_drafts=g_drafts)
+            for s_ in range(n):
+                assert np.abs(s_logits[s_, b] - r["small_logits"][s_]).max() < tol
+                assert abs(res["confidence"][b][s_] - r["confidences"][s_]) < eps
+                if r["own_drafts"][s_] != g_drafts[s_]:
+                    assert _near_tie(r["small_logits"][s_], g_drafts[s_], 2 * tol)
+            # the router's decisions, up to eps around the threshold: go on before the last draft, stop at it
+            assert all(r["confidences"][i] >= tau - eps for i in range(n - 1))
+            assert n == gamma_max or r["confidences"][n - 1] < tau + eps
+            g_targets = res["targets"][b][: n + 1].tolist()
+            for i in range(n + 1):
+                if r["targets"][i] != g_targets[i]:
+                    assert _near_tie(r["large_logits"][i], g_targets[i], 2 * tol)
+            same += (r["own_block_len"] == n)
+            lens.append(n)
+            if r["targets"] == g_targets:
+                assert res["accept_len"][b] == r["accept_len"] and res["n_committed"][b] == r["n_committed"]
+            else:   # a near-tie flipped a target: follow the GPU's ids from here on
+                a = O.TandemOracle.accept_length(g_drafts, g_targets)
+                assert res["accept_len"][b] == a
+                del o.tokens[len(o.tokens) - len(r["emitted"]):]
+                o.tokens += g_drafts[:a] + [g_targets[a]]
+                o.large_cache.truncate(len(o.tokens) - 1)
+                o.derived.truncate(len(o.tokens) - 1)
+    t.close()
+    return lens, same
+
+
+def test_fp32_adaptive_block_length_matches_oracle():
+    shape = gpu_toy_shape(kind=synth.FF_TANDEM_LINEAR, layer_map=(1, 3))
+    w = toy_weights(shape, seed=95)
+    prompts = prompts_for(shape, [4, 130, 19], seed=29)
+    lens, same = _adaptive_replay(shape, w, prompts, 5, 6, TOL_FP32, 1e-4)
+    assert same == len(lens) and len(set(lens)) >= 2          # every block length is the checker's own; they vary
+
+
+def test_bf16_adaptive_block_length_replay():
+    shape = gpu_toy_shape(dtype=synth.DTYPE_BF16, layer_map=(1, 2), large=(2, 256, 4, 512), small=(2, 128, 2, 256))
+    w = _bf16_weights(shape, seed=96, std=0.05)
+    lens, same = _adaptive_replay(shape, w, prompts_for(shape, [6, 141, 1], seed=33), 5, 6, TOL_BF16, 2e-2)
+    assert same >= 0.8 * len(lens) and len(set(lens)) >= 2
+
+
+@pytest.mark.parametrize("dtype", [synth.DTYPE_FP32, synth.DTYPE_BF16])
+def test_adaptive_generate_is_exact_and_counts_runs(dtype):
+    """With any router the response is the large model's greedy decoding (verification is unchanged); a router that
+    always stops gives one draft per iteration, one that never stops gamma_max; the run counts say so."""
+    shape = gpu_toy_shape(dtype=dtype)
+    w = toy_weights(shape, seed=77)
+    prompts = prompts_for(shape, [3, 129, 64], seed=1)
+    router = synth.make_router(shape, 2, 8, seed=3)
+    t = binding.Tandem(shape, w, max_batch=3, max_seq=320, gamma_max=4)
+    t.tandem_prefill(prompts)
+    greedy, _, _ = t.tandem_large_greedy_generate(24)
+    for tau, per_iter in ((2.0, 1), (-1.0, 4), (None, None)):
+        if tau is None:
+            tau = _median_tau(shape, w, prompts[:1], router, 4) if dtype == synth.DTYPE_FP32 else 0.5
+        t.tandem_set_router(router, tau)
+        t.tandem_prefill(prompts)
+        got, lens, st = t.tandem_adaptive_generate(4, 24)
+        assert got.tolist() == greedy.tolist() and lens.tolist() == [24, 24, 24]
+        assert st["large_runs"] == st["iterations"]
+        if per_iter:
+            assert st["small_runs"] == per_iter * st["iterations"]
+        else:
+            assert st["iterations"] <= st["small_runs"] <= 4 * st["iterations"]
+    t.close()
+
+
+# ------------------------------------------------------------------------------------------------
 # multi-query / grouped-query attention (Section 3: either model may use it)
 # ------------------------------------------------------------------------------------------------
 
