@@ -206,7 +206,7 @@ TANDEM_API tandem_status tandem_set_sampling(tandem_ctx* ctx, float temp_large, 
  * probability that M_L disagrees; drafting continues while 1 - s >= tau and fewer than gamma_max drafts exist.
  *
  * tandem_set_router: w1 [hidden][F], b1 [hidden], w2 [hidden]: DEVICE, fp32, caller-owned, valid until replaced or
- * the context is destroyed; 1 <= top_k <= 8.  (The paper's router is trained; any weights can be passed.)
+ * the context is destroyed; 1 <= top_k <= 8 and F * 4 bytes <= 48 KB (else TANDEM_ERR_SHAPE).  (The paper's router is trained; any weights can be passed.)
  * tandem_adaptive_step: one iteration with the natural (arg-max) comparison.  result arrays are sized by gamma_max
  * ([batch][gamma_max] drafts, [batch][gamma_max+1] targets); entries beyond a sequence's own block are -1.
  * block_len: HOST [batch], drafts each sequence made; confidence: HOST [batch][gamma_max], the router's 1 - s per

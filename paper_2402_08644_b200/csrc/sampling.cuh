@@ -5,9 +5,9 @@
 //
 // Every draw uses one uniform variate from a counter-based generator keyed by (seed, sequence, iteration, slot):
 // slots 0..gamma-1 draw the drafts, 16 + r tests draft r, 48 redraws.  A draw from weights w with variate u returns
-// the first index whose running sum exceeds u * sum(w).  The running sums are fp32: thread t of the block owns the
-// contiguous segment [t * seg, (t + 1) * seg) and adds it front to back, the segments' sums are scanned in thread
-// order, and the thread whose segment contains the target walks it again in the same order.
+// the first index whose running sum exceeds u * sum(w).  The running sums are fp32: each warp of the block owns a
+// contiguous range of the row, the ranges' sums are scanned in warp order, and the warp whose range contains the
+// target walks it again 32 weights at a time.
 #pragma once
 #include <math.h>
 #include "common.cuh"
@@ -16,7 +16,8 @@
 
 namespace tandem {
 
-constexpr int SMP_THREADS = 256;
+constexpr int SMP_THREADS = 1024;   // one CTA walks a whole row of logits several times: many loads in flight
+constexpr int SMP_WARPS = SMP_THREADS / 32;
 constexpr int SMP_SLOT_ACCEPT = 16;
 constexpr int SMP_SLOT_REDRAW = 48;
 
@@ -26,7 +27,7 @@ __device__ __forceinline__ float uniform_variate(unsigned long long seed, int se
     return (float)(x >> 40) * (1.0f / 16777216.0f);   // 24 bits: exact in fp32
 }
 
-// Block-wide reductions over SMP_THREADS threads; `red` holds 8 floats.  Every thread gets the result.
+// Block-wide reductions over SMP_THREADS threads; `red` holds SMP_WARPS floats.  Every thread gets the result.
 __device__ __forceinline__ float smp_block_max(float v, float* red) {
     v = warp_max(v);
     __syncthreads();
@@ -34,56 +35,81 @@ __device__ __forceinline__ float smp_block_max(float v, float* red) {
     __syncthreads();
     float r = red[0];
 #pragma unroll
-    for (int w = 1; w < SMP_THREADS / 32; ++w) r = fmaxf(r, red[w]);
+    for (int w = 1; w < SMP_WARPS; ++w) r = fmaxf(r, red[w]);
     return r;
 }
 
 // Maximum of row[0..V).
 __device__ __forceinline__ float smp_row_max(const float* row, int V, float* red) {
     float m = -INFINITY;
-    for (int i = threadIdx.x; i < V; i += SMP_THREADS) m = fmaxf(m, __ldcg(row + i));
+    const bool vec = (V & 3) == 0 && (reinterpret_cast<uintptr_t>(row) & 15) == 0;   // 16 bytes at a time, several loads in flight
+    const int V4 = vec ? V >> 2 : 0;
+#pragma unroll 4
+    for (int i4 = threadIdx.x; i4 < V4; i4 += SMP_THREADS) {
+        const float4 x = __ldcg(reinterpret_cast<const float4*>(row) + i4);
+        m = fmaxf(fmaxf(m, fmaxf(x.x, x.y)), fmaxf(x.z, x.w));
+    }
+    for (int i = 4 * V4 + threadIdx.x; i < V; i += SMP_THREADS) m = fmaxf(m, __ldcg(row + i));
     return smp_block_max(m, red);
 }
 
 // Inverse-CDF draw from the non-negative weights w(i), i in [0, V), with variate u in [0, 1).
-// scan: SMP_THREADS floats of shared memory; s_pick: one int.  Every thread returns the drawn index.
-// Also returns the total of the weights through *total_out (nullable).
+// Warp j of the block owns the contiguous range [j * chunk, (j + 1) * chunk).  Pass A: every warp sums its range
+// (lanes stride over it, coalesced), the warps' sums are scanned in warp order.  Pass B: the warp whose range
+// contains the target u * total walks it again, 32 consecutive weights at a time with a warp-wide running sum, and
+// takes the first index whose running sum exceeds the target.
+// wsum: SMP_WARPS floats of shared memory; s_pick: one int.  Every thread returns the drawn index; *total_out
+// (nullable) receives the total of the weights.
 template <typename W>
-__device__ __forceinline__ int smp_draw(W w, int V, float u, float* scan, int* s_pick, float* total_out) {
-    const int tid = threadIdx.x;
-    const int seg = (V + SMP_THREADS - 1) / SMP_THREADS;
-    const int i0 = min(V, tid * seg), i1 = min(V, i0 + seg);
+__device__ __forceinline__ int smp_draw(W w, int V, float u, float* wsum, int* s_pick, float* total_out) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int chunk = (((V + SMP_WARPS - 1) / SMP_WARPS) + 31) & ~31;
+    const int i0 = min(V, warp * chunk), i1 = min(V, i0 + chunk);
     float local = 0.f;
     int last_pos = -1;
-    for (int i = i0; i < i1; ++i) {
+    for (int i = i0 + lane; i < i1; i += 32) {
         const float x = w(i);
         local += x;
         if (x > 0.f) last_pos = i;
     }
+    local = warp_sum(local);
     __syncthreads();
-    scan[tid] = local;
+    if (lane == 0) wsum[warp] = local;
     if (tid == 0) *s_pick = -1;
     __syncthreads();
-    if (tid == 0) {   // inclusive scan of the segments' sums in thread order (256 additions, one thread: a fixed order)
+    if (tid == 0) {   // inclusive scan of the warps' sums in warp order
         float run = 0.f;
-        for (int t = 0; t < SMP_THREADS; ++t) { run += scan[t]; scan[t] = run; }
+        for (int t = 0; t < SMP_WARPS; ++t) { run += wsum[t]; wsum[t] = run; }
     }
     __syncthreads();
-    const float total = scan[SMP_THREADS - 1];
+    const float total = wsum[SMP_WARPS - 1];
     const float target = u * total;
-    const float incl = scan[tid], excl = tid > 0 ? scan[tid - 1] : 0.f;
-    if (incl > target && excl <= target) {   // exactly one segment contains the target
+    const float incl = wsum[warp], excl = warp > 0 ? wsum[warp - 1] : 0.f;
+    if (incl > target && excl <= target) {   // exactly one warp's range contains the target (warp-uniform condition)
         float run = excl;
         int pick = -1;
-        for (int i = i0; i < i1; ++i) {
-            run += w(i);
-            if (run > target) { pick = i; break; }
+        for (int base = i0; base < i1 && pick < 0; base += 32) {
+            const int i = base + lane;
+            float p = i < i1 ? w(i) : 0.f;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {   // inclusive running sum over the 32 lanes
+                const float q = __shfl_up_sync(0xffffffffu, p, o);
+                if (lane >= o) p += q;
+            }
+            const unsigned hit = __ballot_sync(0xffffffffu, run + p > target);
+            if (hit) pick = base + __ffs(hit) - 1;
+            run += __shfl_sync(0xffffffffu, p, 31);
         }
-        if (pick < 0) pick = last_pos;       // rounding: the segment's own walk fell just short
-        *s_pick = pick;
+        if (pick < 0) {   // rounding: the second walk fell just short of the target: the range's last positive weight
+            int lp = last_pos;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) lp = max(lp, __shfl_xor_sync(0xffffffffu, lp, o));
+            pick = lp;
+        }
+        if (lane == 0) *s_pick = pick;
     }
     __syncthreads();
-    if (*s_pick < 0) {   // rounding left no index beyond the target: the last index with a positive weight
+    if (*s_pick < 0) {   // rounding left no range beyond the target: the last index with a positive weight
         __syncthreads();
         atomicMax(s_pick, last_pos);
         __syncthreads();
@@ -96,7 +122,7 @@ __device__ __forceinline__ int smp_draw(W w, int V, float u, float* scan, int* s
 // grid: batch; block: SMP_THREADS.
 __global__ void __launch_bounds__(SMP_THREADS) sample_draft_kernel(LoopState st, const float* __restrict__ logits, int V, int s,
                                                                    float temp, unsigned long long seed) {
-    __shared__ float red[8], scan[SMP_THREADS];
+    __shared__ float red[SMP_WARPS], scan[SMP_WARPS];
     __shared__ int s_pick;
     pdl_wait();
     pdl_launch_dependents();
@@ -116,7 +142,7 @@ __global__ void __launch_bounds__(SMP_THREADS) sample_draft_kernel(LoopState st,
 __global__ void __launch_bounds__(SMP_THREADS) sample_verify_kernel(LoopState st, int batch, int gamma, const float* __restrict__ logits_large,
                                                                     const float* __restrict__ logits_small, int V, float temp_large,
                                                                     float temp_small, unsigned long long seed) {
-    __shared__ float red[8], scan[SMP_THREADS];
+    __shared__ float red[SMP_WARPS], scan[SMP_WARPS];
     __shared__ int s_pick;
     pdl_wait();
     pdl_launch_dependents();

@@ -785,12 +785,13 @@ void launch_verify(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_ne
 // Adaptive block length: the router's decision after draft step s, for every sequence that is still drafting.
 void launch_router(tandem_ctx& c, int s, int gamma_max) {
     const float* logits = at<float>(c, c.lay.logits_small) + (size_t)s * c.batch * c.small.d.vocab;
-    ProfScope ps(c, PC_ARGMAX, (double)c.batch * c.small.d.vocab * 4.0 * (2 + c.router.k));
+    ProfScope ps(c, PC_ARGMAX, (double)c.batch * c.small.d.vocab * 8.0);
+    const size_t feat_bytes = sizeof(float) * (size_t)(1 + c.router.k + c.router.k * c.small.d.d_model);   // <= 48 KB, checked by tandem_set_router
     if (c.cfg.dtype == TANDEM_DTYPE_BF16)
-        launch_ex(c, true, 1, router_kernel<bf16>, dim3(c.batch), dim3(RT_THREADS), 0, c.st, c.batch, logits, (int)c.small.d.vocab, s, gamma_max,
+        launch_ex(c, true, 1, router_kernel<bf16>, dim3(c.batch), dim3(RT_THREADS), feat_bytes, c.st, c.batch, logits, (int)c.small.d.vocab, s, gamma_max,
                   (const bf16*)w_emb(c, c.small), (int)c.small.d.d_model, c.router);
     else
-        launch_ex(c, true, 1, router_kernel<float>, dim3(c.batch), dim3(RT_THREADS), 0, c.st, c.batch, logits, (int)c.small.d.vocab, s, gamma_max,
+        launch_ex(c, true, 1, router_kernel<float>, dim3(c.batch), dim3(RT_THREADS), feat_bytes, c.st, c.batch, logits, (int)c.small.d.vocab, s, gamma_max,
                   (const float*)w_emb(c, c.small), (int)c.small.d.d_model, c.router);
 }
 void launch_adaptive_begin(tandem_ctx& c) {
@@ -1583,6 +1584,7 @@ extern "C" tandem_status tandem_set_router(tandem_ctx* c, int32_t top_k, int32_t
     TRY(begin_call(c));
     if (!w1 || !b1 || !w2 || top_k < 1 || top_k > RT_MAX_K || hidden < 1 || top_k > c->cfg.small.vocab) return TANDEM_ERR_INVALID_ARG;
     if (((uintptr_t)w1 | (uintptr_t)b1 | (uintptr_t)w2) & 3) return TANDEM_ERR_INVALID_ARG;
+    if (sizeof(float) * (size_t)(1 + top_k + (size_t)top_k * c->cfg.small.d_model) > 48 * 1024) return TANDEM_ERR_SHAPE;   // the feature vector sits in shared memory
     CK(cudaStreamSynchronize(c->stream));
     for (auto& g : c->graphs)   // the router's arguments are baked into the captured draft steps
         if (g.kind == 3 && g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
