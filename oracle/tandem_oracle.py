@@ -46,6 +46,12 @@ Readings taken where the paper is silent or inconsistent:
       it to predict).  The small model goes on drafting while 1 - s >= tau and fewer than gamma_max drafts exist;
       otherwise the drafts made so far (at least one) are verified as a block of that length.  k, the hidden width
       and the weights are inputs (the paper gives none); decisions are per sequence.
+  R20 Teacher-forced Tandem forward (Eq. 2 over a whole given sequence, as in training and in the accuracy /
+      cross-entropy evaluation of Section 4.1): blocks of gamma positions anchored at position 0; the token at
+      position i is the small model's input at i, its context holds the projected large representations of
+      positions below the block's start floor(i / gamma) * gamma and the small model's own representations from
+      there to i (R1); its logits predict the token at i + 1.  Per position: the negative log-likelihood of the
+      true next token (natural log) and the arg-max.
   R4  Pre-LayerNorm blocks (gain and bias, eps 1e-5, biased variance), exact-erf GELU, no linear
       biases, learned absolute position embeddings, untied output head.
   R6  FF_Tandem MLP variant: hidden width given by the shape, GELU, no biases.
@@ -435,6 +441,19 @@ class TandemOracle:
         self.iteration += 1
         return {"drafts": drafts, "emitted": kept, "small_logits": s_logits, "n_committed": len(self.tokens), "reps": reps}
 
+    def teacher_forced_logits(self, ids: Sequence[int], gamma: int) -> np.ndarray:
+        """The same logits as `teacher_forced_tandem_logits` through the caches: the first token is the pending
+        token of an empty prompt pass, then representation-only rounds fed the given tokens (R20)."""
+        seq = [int(t) for t in ids]
+        self.prefill(seq[:1])
+        out = []
+        while len(out) < len(seq):
+            g = min(gamma, len(seq) - len(out))
+            nxt = seq[len(out) + 1: len(out) + 1 + g]
+            forced = nxt + [0] * (g - len(nxt))          # the token after the last position does not exist: any id, never used
+            out += self.step_representation_only(g, forced=forced)["small_logits"]
+        return np.stack(out)
+
     def generate_representation_only(self, prompt: Sequence[int], gamma: int, max_new: int) -> List[int]:
         self.prefill(prompt)
         P = len(prompt)
@@ -735,6 +754,36 @@ def standalone_tandem_free_token_full_prompt(shape, weights: Dict[str, np.ndarra
             lg = tandem_small_full_forward(small, proj, shape.layer_map, reps, boundary, seq)
             seq.append(argmax_decision(lg[-1]))
     return seq[P:P + max_new]
+
+
+def teacher_forced_tandem_logits(shape, weights: Dict[str, np.ndarray], ids: Sequence[int], gamma: int,
+                                 dtype=np.float64) -> np.ndarray:
+    """Eq. 2 over a whole given sequence by brute force (R20): for every block, the large model's representations of
+    everything before the block are recomputed from scratch and the small model reads the block on top of them.
+    Returns the small model's logits for positions 0 .. len(ids) - 1, shape [S][V]."""
+    large = Decoder(weights, "L", shape.large.n_layers, shape.large.n_heads, dtype, shape.large.kv_heads)
+    small = Decoder(weights, "S", shape.small.n_layers, shape.small.n_heads, dtype, shape.small.kv_heads)
+    proj = TandemProjection(weights, shape.small.n_layers, shape.ff_tandem_kind, dtype)
+    seq = [int(t) for t in ids]
+    out = []
+    for start in range(0, len(seq), gamma):
+        end = min(len(seq), start + gamma)
+        reps, _ = decoder_full_forward(large, seq[:start])
+        out.append(tandem_small_full_forward(small, proj, shape.layer_map, reps, start, seq[:end]))
+    return np.concatenate(out, axis=0)
+
+
+def next_token_scores(logits: np.ndarray, ids: Sequence[int]) -> Tuple[np.ndarray, np.ndarray]:
+    """For positions 0 .. S-2: (negative log-likelihood of the true next token under softmax(logits), arg-max)."""
+    S = len(ids)
+    nll = np.empty(S - 1)
+    top = np.empty(S - 1, dtype=np.int64)
+    for i in range(S - 1):
+        row = np.asarray(logits[i], dtype=np.float64)
+        m = row.max()
+        nll[i] = m + math.log(np.exp(row - m).sum()) - row[int(ids[i + 1])]
+        top[i] = argmax_decision(logits[i])
+    return nll, top
 
 
 def generate_batch(shape, weights: Dict[str, np.ndarray], prompts: Sequence[Sequence[int]], gamma: int,

@@ -11,6 +11,7 @@ plus the schedule of Figures 2 and 3, hand-made accept cases, forced modes and r
 import os
 
 import numpy as np
+import torch
 import pytest
 
 from oracle import tandem_oracle as O
@@ -339,3 +340,39 @@ def test_grouped_query_models_keep_every_invariant():
     assert O.TandemOracle(shape, w).generate(prompt, 2, 7, mode=O.ACCEPT_ALL)[0] == O.standalone_tandem_free_token(shape, w, prompt, 2, 7)
     assert O.TandemOracle(shape, w).generate_representation_only(prompt, 2, 6) == \
         O.standalone_tandem_representation_only(shape, w, prompt, 2, 6)
+
+
+# ------------------------------------------------------------------------------------------------
+# Teacher-forced Tandem forward (Eq. 2 over a given sequence)
+# ------------------------------------------------------------------------------------------------
+
+def test_teacher_forced_forward_limits_and_cached_path():
+    shape = toy_shape(kind=synth.FF_TANDEM_MLP, hidden=12)
+    w = toy_weights(shape, seed=31)
+    ids = _prompt(shape, 11, seed=6)
+    small = O.Decoder(w, "S", shape.small.n_layers, shape.small.n_heads)
+    # one block over the whole sequence: no large-derived context, a plain decoder (Eq. 1 with the small model's weights)
+    assert np.allclose(O.teacher_forced_tandem_logits(shape, w, ids, 64), O.decoder_full_forward(small, ids)[1], atol=1e-10)
+    for gamma in (1, 2, 3, 4):
+        brute = O.teacher_forced_tandem_logits(shape, w, ids, gamma)
+        cached = O.TandemOracle(shape, w).teacher_forced_logits(ids, gamma)
+        assert brute.shape == (11, shape.small.vocab) and np.allclose(brute, cached, atol=1e-9)
+        # positions of the first block see no large model at all
+        assert np.allclose(brute[:gamma], O.decoder_full_forward(small, ids[:gamma])[1], atol=1e-10)
+    assert np.abs(O.teacher_forced_tandem_logits(shape, w, ids, 2) - O.teacher_forced_tandem_logits(shape, w, ids, 3)).max() > 1e-3
+    # self-tandem: Eq. 2 is Eq. 1 of the large model for any block length
+    dims = synth.ModelDims(2, 32, 4, 64, 50, 64)
+    st = synth.self_tandem_shape(dims)
+    ws = synth.make_self_tandem_weights(st, seed=6, std=0.35)
+    large = O.Decoder(ws, "L", 2, 4)
+    assert np.allclose(O.teacher_forced_tandem_logits(st, ws, ids, 3), O.decoder_full_forward(large, ids)[1], atol=1e-9)
+
+
+def test_next_token_scores_against_library_cross_entropy():
+    rng = np.random.default_rng(2)
+    logits = rng.normal(size=(6, 9)) * 3
+    ids = [3, 1, 4, 1, 5, 8]
+    nll, top = O.next_token_scores(logits, ids)
+    want = torch.nn.functional.cross_entropy(torch.tensor(logits[:5]), torch.tensor(ids[1:]), reduction="none").numpy()
+    assert np.allclose(nll, want, atol=1e-12) and top.tolist() == logits[:5].argmax(1).tolist()
+    assert np.isclose(O.next_token_scores(np.zeros((2, 7)), [0, 3])[0][0], np.log(7.0))
