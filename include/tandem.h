@@ -194,6 +194,18 @@ TANDEM_API tandem_status tandem_speculative_generate(tandem_ctx* ctx, int32_t ga
                                           int32_t accept_mode, uint64_t mode_seed, int32_t* out_ids,
                                           int32_t* out_lens, tandem_stats* stats);
 
+/* Teacher-forced Tandem forward: Eq. 2 over whole given sequences with block length gamma, as in training (Section 3
+ * "Training": the key/value pairs of earlier blocks come from M_L through FF_Tandem, those of the current block from
+ * M_S) and in the accuracy / cross-entropy evaluation of Section 4.1.  Blocks of gamma positions are anchored at
+ * position 0; the token at position i is M_S's input at i and its logits predict the token at i + 1.
+ *   ids: HOST, the sequences concatenated; lens: HOST [batch], each >= 2; max(lens) + gamma <= max_seq and max_pos.
+ *   nll:  HOST [sum(lens[b] - 1)], per sequence and position 0 .. len-2 the negative log-likelihood (natural log) of
+ *         the true next token under softmax of M_S's logits;  top1: HOST, same shape, M_S's arg-max (nullable).
+ * Synchronous.  Replaces the context's sequences (it runs an empty prompt pass and representation-only rounds whose
+ * drafts are the given tokens); call tandem_prefill before decoding again. */
+TANDEM_API tandem_status tandem_teacher_forced_forward(tandem_ctx* ctx, int32_t gamma, int32_t batch, const int32_t* ids,
+                                                       const int32_t* lens, float* nll, int32_t* top1);
+
 /* Temperatures of the two models for accept mode TANDEM_ACCEPT_SAMPLE (both > 0; default 1 and 1).  Applies to the
  * iterations enqueued afterwards; waits for the context's stream when a value changes. */
 TANDEM_API tandem_status tandem_set_sampling(tandem_ctx* ctx, float temp_large, float temp_small);

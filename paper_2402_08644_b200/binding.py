@@ -32,7 +32,7 @@ EXPORTS = ["tandem_query_arena", "tandem_create", "tandem_destroy", "tandem_pref
            "tandem_profile_class_name", "tandem_launch_count", "tandem_decode_attention_static",
            "tandem_debug_expire_wait", "tandem_standalone_check", "tandem_standalone_generate",
            "tandem_set_sampling", "tandem_prefill_samples", "tandem_set_router", "tandem_adaptive_step",
-           "tandem_adaptive_generate"]
+           "tandem_adaptive_generate", "tandem_teacher_forced_forward"]
 
 
 class TandemError(RuntimeError):
@@ -94,6 +94,7 @@ def load_library():
     lib.tandem_large_greedy_generate.argtypes = [vp, i32, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_standalone_generate.argtypes = [vp, i32, i32, i32, pi32, pi32, C.POINTER(Stats)]
     lib.tandem_set_sampling.argtypes = [vp, C.c_float, C.c_float]
+    lib.tandem_teacher_forced_forward.argtypes = [vp, i32, i32, pi32, pi32, C.POINTER(C.c_float), pi32]
     lib.tandem_set_router.argtypes = [vp, i32, i32, vp, vp, vp, C.c_float, C.c_float]
     lib.tandem_adaptive_step.argtypes = [vp, i32, C.POINTER(StepResult), pi32, C.POINTER(C.c_float)]
     lib.tandem_adaptive_generate.argtypes = [vp, i32, i32, pi32, pi32, C.POINTER(Stats)]
@@ -243,6 +244,19 @@ class Tandem:
         _check(self.lib.tandem_speculative_generate(self.ctx, gamma, max_new, accept_mode, mode_seed, p(out), p(lens),
                                                     C.byref(st)), "tandem_speculative_generate")
         return out, lens, self._stats(st, gamma)
+
+    def tandem_teacher_forced_forward(self, sequences: Sequence[Sequence[int]], gamma: int):
+        """Returns ([nll per sequence], [top1 per sequence]): arrays of len(seq) - 1 entries each."""
+        lens = np.asarray([len(p) for p in sequences], dtype=np.int32)
+        ids = np.ascontiguousarray(np.concatenate([np.asarray(p, dtype=np.int32) for p in sequences]))
+        n = int((lens - 1).sum())
+        nll = np.zeros(n, np.float32); top = np.zeros(n, np.int32)
+        p = lambda x: x.ctypes.data_as(C.POINTER(C.c_int32))
+        _check(self.lib.tandem_teacher_forced_forward(self.ctx, gamma, len(sequences), p(ids), p(lens),
+                                                      nll.ctypes.data_as(C.POINTER(C.c_float)), p(top)), "tandem_teacher_forced_forward")
+        self.batch = len(sequences)
+        cuts = np.cumsum(lens - 1)[:-1]
+        return np.split(nll, cuts), np.split(top, cuts)
 
     def tandem_set_sampling(self, temp_large: float, temp_small: float) -> None:
         _check(self.lib.tandem_set_sampling(self.ctx, temp_large, temp_small), "tandem_set_sampling")

@@ -336,6 +336,65 @@ __global__ void __launch_bounds__(256) verify_kernel(LoopState st, int batch, in
     }
 }
 
+// Teacher-forced Tandem forward (Eq. 2 over a given sequence): the next gamma tokens of every sequence become the
+// "drafts" of the round, so that draft step s reads the true token of its position.  forced: [batch][stride] token
+// ids; positions at or beyond forced_len[b] read as token 0 (rows past a sequence's end are computed and ignored).
+// grid: 1; block: 256.
+__global__ void __launch_bounds__(256) forced_fill_kernel(LoopState st, int batch, int gamma, const int* __restrict__ forced,
+                                                          const int* __restrict__ forced_len, int stride) {
+    pdl_wait();
+    pdl_launch_dependents();
+    for (int i = threadIdx.x; i < batch * gamma; i += 256) {
+        const int b = i / gamma, r = i - b * gamma;
+        const int p = st.n[b] + r;                       // position of the token that draft r + 1 stands for
+        st.drafts[b * st.gamma_limit + r] = p < forced_len[b] ? forced[(size_t)b * stride + p] : 0;
+    }
+}
+
+// Scores of a teacher-forced round: for draft step s of sequence b, at position p = n_b - 1 + s, the negative
+// log-likelihood of the true token at p + 1 under softmax(logits) and the arg-max (lowest id on ties).
+// logits: [gamma][batch][V].  grid: (gamma, batch); block: 256.
+__global__ void __launch_bounds__(256) score_rows_kernel(LoopState st, int batch, const float* __restrict__ logits, int V,
+                                                         const int* __restrict__ forced, const int* __restrict__ forced_len, int stride,
+                                                         float* __restrict__ nll, int* __restrict__ top1) {
+    __shared__ float sv[8], ss[8];
+    __shared__ int si[8];
+    pdl_wait();
+    pdl_launch_dependents();
+    const int s = blockIdx.x, b = blockIdx.y;
+    const int p = st.n[b] - 1 + s;
+    if (p + 1 >= forced_len[b]) return;                  // no true next token: nothing to score
+    const float* row = logits + ((size_t)s * batch + b) * V;
+    float best = -INFINITY;
+    int bi = INT_MAX;
+    for (int i = threadIdx.x; i < V; i += 256) {
+        const float v = __ldcg(row + i);
+        if (v > best || (v == best && i < bi)) { best = v; bi = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = best; si[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    for (int w = 0; w < 8; ++w)
+        if (sv[w] > best || (sv[w] == best && si[w] < bi)) { best = sv[w]; bi = si[w]; }
+    float z = 0.f;
+    for (int i = threadIdx.x; i < V; i += 256) z += expf(__ldcg(row + i) - best);
+    z = warp_sum(z);
+    if ((threadIdx.x & 31) == 0) ss[threadIdx.x >> 5] = z;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < 8; ++w) tot += ss[w];
+        const int truth = forced[(size_t)b * stride + p + 1];
+        nll[(size_t)b * stride + p] = best + logf(tot) - __ldcg(row + truth);
+        top1[(size_t)b * stride + p] = bi;
+    }
+}
+
 // Test hook: gathers K or V of one (layer, sequence) from [H][t_max][dh] into fp32 [n][H*dh].
 template <typename T>
 __global__ void gather_kv_kernel(const T* __restrict__ cache_seq, float* __restrict__ dst, int n, int n_heads, int d_head, int t_max) {

@@ -49,6 +49,7 @@ struct Layout {   // byte offsets into the arena
     size_t kv_large, kv_small;
     size_t st_n, st_pending, st_drafts, st_targets, st_accept, st_emitted, st_done, st_out, st_counters, st_hist;
     size_t st_block_len, st_drafting, st_confidence;
+    size_t forced_ids, forced_len, forced_nll, forced_top;   // teacher-forced forward: given tokens [B][T], lengths [B], scores [B][T]
     size_t row_tok, row_seq, row_pos, grp_row0, grp_cnt;
     size_t attn_counters;   // inside the zero-filled state block
     size_t h_large, h_small, a, q, o, f, xb, t1, yhat, a_s, logits_large, logits_small, part_ml, part_acc, dbg;
@@ -224,6 +225,7 @@ Layout make_layout(const tandem_config& c) {
     L.part_ml = take(RD * hmax * L.n_chunks_max * 2 * 4);
     L.part_acc = take(RD * dmax * L.n_chunks_max * 4);
     L.dbg = take(T * dmax * 4);
+    L.forced_ids = take(B * T * 4); L.forced_len = take(B * 4); L.forced_nll = take(B * T * 4); L.forced_top = take(B * T * 4);
     L.vocab_tiles = cdiv(c.large.vocab, 128);
     L.amax_val_large = take(RD * L.vocab_tiles * 4); L.amax_idx_large = take(RD * L.vocab_tiles * 4);
     L.amax_val_small = take(B * L.vocab_tiles * 4); L.amax_idx_small = take(B * L.vocab_tiles * 4);
@@ -756,8 +758,10 @@ void setup_rows(tandem_ctx& c, int r0, int nq) {
 }
 
 // Draft step s: one token per sequence through the small model over the mixed context (Eq. 2, lines 2-3).
+// dst: where the step's arg-max goes (default: draft s of the loop state; a teacher-forced round keeps its given
+// drafts and sends the arg-max to the unused target array).
 template <typename T>
-void small_step(tandem_ctx& c, int s) {
+void small_step(tandem_ctx& c, int s, bool keep_drafts = false) {
     setup_rows(c, s, 1);
     Rows r = decode_rows(c, s, 1);
     float* y = at<float>(c, c.lay.h_small);
@@ -769,7 +773,22 @@ void small_step(tandem_ctx& c, int s) {
     }
     for (int j = 0; j < c.small.d.n_layers; ++j) decoder_layer<T>(c, c.small, j, y, r);
     float* logits = at<float>(c, c.lay.logits_small) + (size_t)s * c.batch * c.small.d.vocab;
-    head_argmax<T>(c, c.small, y, r, logits, c.st.drafts, TANDEM_GAMMA_LIMIT, s);
+    if (keep_drafts) head_argmax<T>(c, c.small, y, r, logits, c.st.targets, TANDEM_GAMMA_LIMIT + 1, s);
+    else head_argmax<T>(c, c.small, y, r, logits, c.st.drafts, TANDEM_GAMMA_LIMIT, s);
+}
+
+// Teacher-forced round (accept mode 5): the given tokens become the round's drafts; after the draft steps their
+// logits are scored against the given next tokens.
+void launch_forced_fill(tandem_ctx& c, int gamma) {
+    ProfScope ps(c, PC_ROWS, (double)c.batch * gamma * 8.0);
+    launch_ex(c, true, 1, forced_fill_kernel, dim3(1), dim3(256), 0, c.st, c.batch, gamma, (const int*)at<int>(c, c.lay.forced_ids),
+              (const int*)at<int>(c, c.lay.forced_len), (int)c.cfg.max_seq);
+}
+void launch_score_rows(tandem_ctx& c, int gamma) {
+    ProfScope ps(c, PC_ARGMAX, (double)c.batch * gamma * c.small.d.vocab * 8.0);
+    launch_ex(c, true, 1, score_rows_kernel, dim3(gamma, c.batch), dim3(256), 0, c.st, c.batch, (const float*)at<float>(c, c.lay.logits_small),
+              (int)c.small.d.vocab, (const int*)at<int>(c, c.lay.forced_ids), (const int*)at<int>(c, c.lay.forced_len), (int)c.cfg.max_seq,
+              at<float>(c, c.lay.forced_nll), at<int>(c, c.lay.forced_top));
 }
 
 void launch_verify(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new, bool from_tiles, bool adaptive = false) {
@@ -816,11 +835,13 @@ void launch_sample_verify(tandem_ctx& c, int gamma, uint64_t seed) {
 
 template <typename T>
 void iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
+    if (mode == 5) launch_forced_fill(c, gamma);
     for (int s = 0; s < gamma; ++s) {
-        small_step<T>(c, s);
+        small_step<T>(c, s, mode == 5);
         if (mode == 4) launch_sample_draft(c, s, seed);   // replaces the arg-max draft of this step
     }
-    if (mode == 3) {   // stand-alone Tandem without the free token: gamma rows, no output head
+    if (mode == 5) launch_score_rows(c, gamma);
+    if (mode == 3 || mode == 5) {   // stand-alone Tandem without the free token: gamma rows, no output head
         setup_rows(c, 0, gamma);
         large_pass<T>(c, decode_rows(c, gamma - 1, gamma), true, false);
     } else {
@@ -828,7 +849,7 @@ void iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
         large_pass<T>(c, decode_rows(c, gamma, gamma + 1), true, true);
     }
     if (mode == 4) launch_sample_verify(c, gamma, seed);
-    launch_verify(c, gamma, mode, seed, max_new, false);
+    launch_verify(c, gamma, mode == 5 ? 3 : mode, seed, max_new, false);
     c.last_gamma = gamma;
 }
 
@@ -986,10 +1007,18 @@ void tc_large_block(tandem_ctx& c, int nq, int fin_r, bool project, bool head) {
 }
 
 void tc_iteration(tandem_ctx& c, int gamma, int mode, uint64_t seed, int max_new) {
-    const bool sampled = mode == 4;
+    const bool sampled = mode == 4, forced = mode == 5;
+    if (forced) launch_forced_fill(c, gamma);
     for (int s = 0; s < gamma; ++s) {
-        tc_small_step(c, s, sampled);
+        tc_small_step(c, s, sampled || forced);   // (both find their drafts in the loop state, not in per-tile arg-max results)
         if (sampled) launch_sample_draft(c, s, seed);
+    }
+    if (forced) {   // teacher-forced round: score the logits, then a representation-only block whose drafts are the given tokens
+        launch_score_rows(c, gamma);
+        tc_large_block(c, gamma, -1, true, false);
+        launch_verify(c, gamma, 3, seed, max_new, false);
+        c.last_gamma = gamma;
+        return;
     }
     if (mode == 3) tc_large_block(c, gamma, -1, true, false);   // gamma rows, no head: the last draft is finished by the verify kernel
     else tc_large_block(c, gamma + 1, (gamma > 0 && !sampled) ? gamma : -1, true, true);
@@ -1487,7 +1516,7 @@ tandem_status run_generate(tandem_ctx* c, bool speculative, int gamma, int max_n
     const int DEPTH = 3;
     const int kind = speculative ? 0 : 1;
     const int64_t ticket0 = c->ticket;
-    const int per_iter = mode == TANDEM_ACCEPT_REPRESENTATION_ONLY ? gamma : gamma + 1;   // most tokens one iteration can emit
+    const int per_iter = (mode == TANDEM_ACCEPT_REPRESENTATION_ONLY || mode == 5) ? gamma : gamma + 1;   // most tokens one iteration can emit
     const int lead = lead_large_step ? 1 : 0;
     const int min_iters = lead + (max_new - lead + per_iter - 1) / per_iter;
     const int n_known0 = c->n_ub;
@@ -1676,6 +1705,50 @@ extern "C" tandem_status tandem_speculative_generate(tandem_ctx* c, int32_t gamm
     if (gamma < 0 || gamma > c->cfg.gamma_max || accept_mode < 0 || accept_mode > 4) return TANDEM_ERR_INVALID_ARG;
     if (accept_mode == TANDEM_ACCEPT_REPRESENTATION_ONLY && gamma < 1) return TANDEM_ERR_INVALID_ARG;
     return run_generate(c, true, gamma, max_new_tokens, accept_mode, mode_seed, out_ids, out_lens, stats);
+}
+
+extern "C" tandem_status tandem_teacher_forced_forward(tandem_ctx* c, int32_t gamma, int32_t batch, const int32_t* ids, const int32_t* lens,
+                                                       float* nll, int32_t* top1) {
+    TRY(begin_call(c));
+    if (!ids || !lens || !nll || batch < 1 || gamma < 1 || gamma > c->cfg.gamma_max) return TANDEM_ERR_INVALID_ARG;
+    if (batch > c->cfg.max_batch) return TANDEM_ERR_CAPACITY;
+    int max_len = 0;
+    long long total = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (lens[b] < 2) return TANDEM_ERR_INVALID_ARG;
+        max_len = std::max(max_len, lens[b]);
+        total += lens[b];
+    }
+    const int pos_cap = std::min(c->cfg.max_seq, std::min(c->cfg.large.max_pos, c->cfg.small.max_pos));
+    if ((long long)max_len + gamma > pos_cap) return TANDEM_ERR_CAPACITY;
+    for (long long i = 0; i < total; ++i)
+        if (ids[i] < 0 || ids[i] >= c->cfg.large.vocab) return TANDEM_ERR_INVALID_ARG;
+    // an empty prompt pass: the first token of every sequence is its pending token
+    std::vector<int32_t> first((size_t)batch), ones((size_t)batch, 1), padded((size_t)batch * c->cfg.max_seq, 0);
+    long long off = 0;
+    for (int b = 0; b < batch; ++b) {
+        first[b] = ids[off];
+        memcpy(padded.data() + (size_t)b * c->cfg.max_seq, ids + off, (size_t)lens[b] * 4);
+        off += lens[b];
+    }
+    TRY(prefill_impl(c, batch, 1, first.data(), ones.data()));
+    CK(cudaMemcpyAsync(c->arena + c->lay.forced_ids, padded.data(), padded.size() * 4, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->arena + c->lay.forced_len, lens, (size_t)batch * 4, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));   // the host arrays above go out of scope
+    std::vector<int32_t> scratch_ids((size_t)batch * (max_len - 1));
+    TRY(run_generate(c, true, gamma, max_len - 1, 5, 0ull, scratch_ids.data(), nullptr, nullptr));
+    std::vector<float> h_nll((size_t)batch * c->cfg.max_seq);
+    std::vector<int32_t> h_top((size_t)batch * c->cfg.max_seq);
+    CK(cudaMemcpyAsync(h_nll.data(), c->arena + c->lay.forced_nll, h_nll.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(h_top.data(), c->arena + c->lay.forced_top, h_top.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    long long o = 0;
+    for (int b = 0; b < batch; ++b)
+        for (int p = 0; p + 1 < lens[b]; ++p, ++o) {
+            nll[o] = h_nll[(size_t)b * c->cfg.max_seq + p];
+            if (top1) top1[o] = h_top[(size_t)b * c->cfg.max_seq + p];
+        }
+    return TANDEM_OK;
 }
 
 extern "C" tandem_status tandem_set_sampling(tandem_ctx* c, float temp_large, float temp_small) {

@@ -817,6 +817,38 @@ def test_adaptive_generate_is_exact_and_counts_runs(dtype):
 
 
 # ------------------------------------------------------------------------------------------------
+# teacher-forced Tandem forward (Eq. 2 over given sequences)
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype,gamma", [(synth.DTYPE_FP32, 3), (synth.DTYPE_FP32, 1), (synth.DTYPE_BF16, 4), (synth.DTYPE_BF16, 2)])
+def test_teacher_forced_forward_scores_match_oracle(dtype, gamma):
+    """Ragged batch of given sequences (one crosses a 128-position chunk): per-position negative log-likelihood of
+    the true next token within tolerance of the checker's brute-force Eq. 2, arg-max equal (near-ties aside)."""
+    shape = gpu_toy_shape(kind=synth.FF_TANDEM_MLP if dtype == synth.DTYPE_FP32 else synth.FF_TANDEM_LINEAR, hidden=40, dtype=dtype,
+                          layer_map=(1, 3), max_pos=200)
+    w = toy_weights(shape, seed=97) if dtype == synth.DTYPE_FP32 else _bf16_weights(shape, seed=97, std=0.06)
+    seqs = prompts_for(shape, [2, 140, 23], seed=41)
+    tol = TOL_FP32 if dtype == synth.DTYPE_FP32 else TOL_BF16
+    t = binding.Tandem(shape, w, max_batch=3, max_seq=200, gamma_max=4)
+    nll, top = t.tandem_teacher_forced_forward(seqs, gamma)
+    for b, ids in enumerate(seqs):
+        logits = O.teacher_forced_tandem_logits(shape, w, ids, gamma)
+        want_nll, want_top = O.next_token_scores(logits, ids)
+        assert nll[b].shape == (len(ids) - 1,)
+        assert np.abs(nll[b] - want_nll).max() < 2 * tol          # a difference of two logit-sized quantities
+        for i in np.nonzero(top[b] != want_top)[0]:
+            assert _near_tie(logits[i], top[b][i], 2 * tol)
+        assert (top[b] != want_top).sum() <= (0 if dtype == synth.DTYPE_FP32 else 4)
+    # the context is usable for decoding afterwards
+    t.tandem_prefill(seqs)
+    got, _, _ = t.tandem_speculative_generate(3, 5)
+    t.tandem_prefill(seqs)
+    greedy, _, _ = t.tandem_large_greedy_generate(5)
+    assert got.tolist() == greedy.tolist()
+    t.close()
+
+
+# ------------------------------------------------------------------------------------------------
 # multi-query / grouped-query attention (Section 3: either model may use it)
 # ------------------------------------------------------------------------------------------------
 
