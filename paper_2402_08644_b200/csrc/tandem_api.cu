@@ -325,14 +325,14 @@ EncodeTiledFn tmap_encoder() {
     return fn;
 }
 
-// bf16 matrix [rows][cols] with leading dimension ld (elements), tiles of 128 rows x 64 columns, 128-byte swizzle.
-// base 16-byte aligned, ld a multiple of 8.
-bool make_tmap_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+// bf16 matrix [rows][cols] with leading dimension ld (elements), tiles of box_rows (128 by default) rows x 64 columns,
+// 128-byte swizzle.  base 16-byte aligned, ld a multiple of 8.
+bool make_tmap_bf16(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows = 128) {
     EncodeTiledFn enc = tmap_encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {ld * 2};
-    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t box[2] = {64, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -1294,8 +1294,8 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
             bool okm = true;
             const uint64_t kv_rows = (uint64_t)cfg->max_batch * c->large.kv_heads * cfg->max_seq;
             for (int l = 0; l < cfg->large.n_layers && okm; ++l)
-                okm = make_tmap_bf16(&c->kmap[l], kv_ptr<bf16>(*c, c->large, l, 0), kv_rows, (uint64_t)dhL, (uint64_t)dhL) &&
-                      make_tmap_bf16(&c->vmap[l], kv_ptr<bf16>(*c, c->large, l, 1), kv_rows, (uint64_t)dhL, (uint64_t)dhL);
+                okm = make_tmap_bf16(&c->kmap[l], kv_ptr<bf16>(*c, c->large, l, 0), kv_rows, (uint64_t)dhL, (uint64_t)dhL, ATC_KC) &&
+                      make_tmap_bf16(&c->vmap[l], kv_ptr<bf16>(*c, c->large, l, 1), kv_rows, (uint64_t)dhL, (uint64_t)dhL, ATC_KC);
             if (okm) { c->tc_prompt_attn = true; c->prompt_group = ATC_Q; }
         }
     }
