@@ -10,8 +10,8 @@
 //                       it lies in the cache ([key][element], i.e. MN-major for the B operand)
 // The running maximum is lazy: probabilities are taken relative to a reference m that moves only when a chunk's
 // maximum exceeds it by more than ATC_LAZY (so they stay below e^ATC_LAZY); only then is O, in TMEM, rescaled
-// (tcgen05.ld, multiply, tcgen05.st) - rare after the first chunks.  The row sum uses the rounded probabilities, the
-// same numbers the tensor core multiplies with V.
+// (tcgen05.ld, multiply, tcgen05.st) - rare after the first chunks.  The row sum adds the fp32 probabilities (their
+// bf16 roundings, which the tensor core multiplies with V, differ from them by 2^-9 each with random signs).
 // Warp 4 streams K (two stages) and V (one stage) by TMA, warp 5 allocates TMEM and issues the MMAs (S of chunk c+1
 // goes out before the probabilities of chunk c are awaited), warps 0-3 do the softmax and the epilogue.  Every wait is
 // bounded.
@@ -74,6 +74,31 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) 
         : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// 64 consecutive fp32 columns of this thread's TMEM lane in one load (load and wait in one statement: the registers
+// are not read before the load has landed).
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64]) {
+    uint32_t r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+              "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+              "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+              "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]),
+              "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]),
+              "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]),
+              "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]),
+              "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
+// 2^x by the hardware approximation (relative error about 2^-22; 2^-inf = 0), one instruction.
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 // grid: (heads, groups); dynamic smem AtcCfg<DH>::SMEM_BYTES.
 // tmq: queries [M][d_model] (box 64 x 128); tmk / tmv: one layer's cache seen as [(seq, kv head, position)][DH] (box 64 x 64).
@@ -192,37 +217,43 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
         const int qi = warp * 32 + lane;
         const int qpos = pos_first + qi;                 // (rows past cnt compute on whatever the tile holds; never stored)
         const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+        // Everything runs in the base-2 domain: with sc2 = scale * log2(e), a probability is 2^(s * sc2 - m) (one
+        // multiply-add and one ex2 per element); m is the reference maximum in that domain.
+        const float sc2 = a.scale * 1.4426950408889634f;
+        constexpr float LAZY2 = ATC_LAZY * 1.4426950408889634f;
         float m = -INFINITY, l = 0.f;                    // reference maximum of the exponentials, running sum
         bool ok = true;
         for (int c = 0; c < n_chunks && ok; ++c) {
             if (!mbar_wait(smem_u32(&s_sfull[c & 1]), (c >> 1) & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); ok = false; break; }
             tc_fence_after_sync();
             const uint32_t s_addr = lane_addr + (c & 1) * ATC_KC;
-            // this row of S, scaled and masked (every chunk but the tile's last ones lies wholly before its first query)
+            // this row of S, raw; keys after the query's position become -inf (every chunk but the tile's last ones lies
+            // wholly before its first query and needs no mask)
             const bool full = c * ATC_KC + ATC_KC - 1 <= pos_first;
             float t[ATC_KC];
-            float mc = -INFINITY;
+            tmem_ld64(s_addr, t);                        // the whole row in one load
+            float mr = -INFINITY;
+            if (full) {
 #pragma unroll
-            for (int c0 = 0; c0 < ATC_KC; c0 += 16) {
-                float u[16];
-                tmem_ld16(s_addr + c0, u);
+                for (int i = 0; i < ATC_KC; ++i) mr = fmaxf(mr, t[i]);
+            } else {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float v = (full || c * ATC_KC + c0 + i <= qpos) ? u[i] * a.scale : -INFINITY;
-                    t[c0 + i] = v;
-                    mc = fmaxf(mc, v);
+                for (int i = 0; i < ATC_KC; ++i) {
+                    t[i] = (c * ATC_KC + i <= qpos) ? t[i] : -INFINITY;
+                    mr = fmaxf(mr, t[i]);
                 }
             }
+            const float mc = mr * sc2;                   // the chunk's maximum in the base-2 domain (the scale is positive)
             tc_fence_before_sync();      // the TMEM reads of S are done before the MMA after next may overwrite the buffer
             // P V of the previous chunk must be complete before the P tile is rewritten or O is touched
             if (c > 0) {
                 if (!mbar_wait(smem_u32(&s_ofull), (c - 1) & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); ok = false; break; }
                 tc_fence_after_sync();
             }
-            // lazy reference: it moves only when this chunk's maximum exceeds it by more than ATC_LAZY
-            const bool move = mc > m + ATC_LAZY;         // (first chunk: m = -inf, every row with a visible key moves)
+            // lazy reference: it moves only when this chunk's maximum exceeds it by more than the margin
+            const bool move = mc > m + LAZY2;            // (first chunk: m = -inf, every row with a visible key moves)
             if (c > 0 && __any_sync(0xffffffffu, move)) {
-                const float f = (move && m > -INFINITY) ? __expf(m - mc) : 1.0f;   // rows that keep their reference: exactly 1
+                const float f = (move && m > -INFINITY) ? ex2_approx(m - mc) : 1.0f;   // rows that keep their reference: exactly 1
 #pragma unroll
                 for (int e0 = 0; e0 < DH; e0 += 16) {
                     float o[16];
@@ -235,22 +266,24 @@ attn_prefill_tc_kernel(const AttnTcArgs a, const __grid_constant__ CUtensorMap t
                 l *= f;
             }
             if (move) m = mc;
-            // probabilities relative to the reference, bf16; row sum of the rounded values; one 128-byte row of the P tile
+            // probabilities relative to the reference (2^(-inf) = 0 for masked keys), their sum, and one 128-byte row
+            // of the bf16 P tile
             unsigned char* prow = pg + qi * 128;
-            float ls = 0.f;
+            const float nm = -m;
+            float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
             for (int c0 = 0; c0 < ATC_KC; c0 += 8) {
                 uint32_t pk[4];
 #pragma unroll
                 for (int i = 0; i < 8; i += 2) {
-                    const float p0v = t[c0 + i] > -INFINITY ? __expf(t[c0 + i] - m) : 0.f;
-                    const float p1v = t[c0 + i + 1] > -INFINITY ? __expf(t[c0 + i + 1] - m) : 0.f;
-                    const __nv_bfloat162 pb = __floats2bfloat162_rn(p0v, p1v);
-                    ls += __bfloat162float(pb.x) + __bfloat162float(pb.y);
-                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+                    const float p0v = ex2_approx(fmaf(t[c0 + i], sc2, nm));
+                    const float p1v = ex2_approx(fmaf(t[c0 + i + 1], sc2, nm));
+                    ls0 += p0v; ls1 += p1v;
+                    pk[i >> 1] = pack_bf16x2(p0v, p1v);
                 }
                 *reinterpret_cast<uint4*>(prow + ((((c0 >> 3)) ^ (qi & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
+            const float ls = ls0 + ls1;
             l += ls;
             tc_fence_before_sync();      // the rescaled O is in TMEM before the next P V accumulates onto it
             fence_proxy_async_smem();

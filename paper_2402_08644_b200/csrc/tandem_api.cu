@@ -135,6 +135,7 @@ struct tandem_ctx {
     RouterArgs router{};                 // adaptive block length: the router's weights (caller-owned, DEVICE) and threshold
     bool has_router = false;
     int64_t router_ticket = 0;           // router launches since the prompt pass
+    double prompt_sq_sum = 0.0;          // sum over the sequences of the current prompt pass of (rows)^2 (accounting of the attention's work)
 };
 
 namespace {
@@ -624,8 +625,8 @@ void launch_attn_prompt_tc(tandem_ctx& c, int l, const bf16* q, bf16* o, const R
     a.out = o; a.ldo = d; a.row_seq = at<int>(c, c.lay.row_seq); a.row_pos = at<int>(c, c.lay.row_pos);
     a.grp_row0 = at<int>(c, c.lay.grp_row0); a.grp_cnt = at<int>(c, c.lay.grp_cnt);
     a.n_heads = H; a.n_kv_heads = c.large.kv_heads; a.t_max = c.cfg.max_seq; a.scale = 1.0f / sqrtf((float)dh); a.err_flag = c.st.counters + 2;
-    // two MMA groups per (128 queries x 128 keys): 4 * 128 * 128 * dh flops, over the causal half of the prompt
-    ProfScope ps(c, PC_ATTN_PROMPT, 0.0);
+    // causal attention: Q K^T and P V over the lower triangle, 2 * d_head * T^2 flops per head and sequence
+    ProfScope ps(c, PC_ATTN_PROMPT, 2.0 * dh * H * c.prompt_sq_sum);
     if (dh == 64) launch_attn_prompt_tc_dh<64>(c, a, tmq, l, r.groups);
     else launch_attn_prompt_tc_dh<128>(c, a, tmq, l, r.groups);
 }
@@ -1400,6 +1401,8 @@ tandem_status prefill_impl(tandem_ctx* c, int n_queries, int samples, const int3
     c->batch = batch;
     c->n_ub = n_max;
     c->n_sum = total;
+    c->prompt_sq_sum = 0.0;
+    for (int q = 0; q < n_queries; ++q) c->prompt_sq_sum += (double)(prompt_lens[q] - 1) * (prompt_lens[q] - 1);
     if (M > 0) {
         Rows r; r.M = M; r.groups = groups; r.nq = 0; r.decode = false; r.n_chunks = 0; r.kv_positions = (double)rows;
         if (c->cfg.dtype == TANDEM_DTYPE_BF16) large_pass<bf16>(*c, r, true, false);
