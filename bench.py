@@ -431,6 +431,44 @@ def sub_record(r, peak):
     return rec
 
 
+def run_prefill_only(args, local_rank):
+    """The prompt pass alone (large model over the prompt, FF_Tandem projection of every position): device time per
+    pass and the tensor-core rate over its algorithmic flops (2 x parameters x rows for the linear maps, 2 d T^2 per
+    layer and sequence for the causal attention)."""
+    import torch
+    from dataclasses import replace
+    from paper_2402_08644_b200 import binding
+    cfgname, B, P, gamma, new, max_pos = WORKLOADS[args.workload]
+    shape = synth.named_config(cfgname, max_pos)
+    if args.layers > 0:
+        shape = synth.make_shape(replace(shape.large, n_layers=args.layers), replace(shape.small, n_layers=min(args.layers, shape.small.n_layers)),
+                                 shape.ff_tandem_kind, shape.ff_tandem_hidden, None, shape.dtype)
+    dev = torch.device("cuda", local_rank)
+    weights = synth.device_weights(shape, 0, dev)
+    prompts = [[int(t) for t in p] for p in synth.make_prompts(B, P, shape.large.vocab, seed=0)]
+    t = binding.Tandem(shape, weights, max_batch=B, max_seq=P + 8, gamma_max=gamma, device=local_rank, max_prefill_rows=B * P)
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        t.tandem_prefill(prompts)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        t.tandem_prefill(prompts)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    L, S = shape.large, shape.small
+    rows = B * (P - 1)
+    lin = L.n_layers * (2 * L.d_model ** 2 + 2 * L.d_model * L.d_kv + 2 * L.d_model * L.d_ff) + \
+        S.n_layers * (S.d_model * L.d_model + 2 * S.d_model * S.d_kv)
+    flops = 2.0 * lin * rows + L.n_layers * 2.0 * L.d_model * B * float(P - 1) ** 2
+    t.close()
+    print(json.dumps({"metric": "prompt_pass_ms", "value": ms, "unit": "ms", "workload": workload_desc(args.workload),
+                      "layers": [L.n_layers, S.n_layers], "rows": rows, "algorithmic_tflop": flops / 1e12,
+                      "tflops": flops / 1e12 / (ms * 1e-3), "steps": args.steps, "warmup": args.warmup}))
+
+
 def run_ours(args, rank, local_rank, world):
     import torch
     import torch.distributed as dist
@@ -520,6 +558,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the accept-all / greedy / per-kernel passes")
     ap.add_argument("--no-subrecords", action="store_true", help="skip the medium / large sub-records of the default line")
+    ap.add_argument("--prefill-only", action="store_true", help="time the prompt pass alone (steps = prompt passes); prints its own JSON line")
+    ap.add_argument("--layers", type=int, default=0, help="with --prefill-only: cut both models to this many layers (small cases for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -545,7 +585,10 @@ def main():
     if world > 1:
         dist.barrier()
 
-    run_ours(args, rank, local_rank, world)
+    if args.prefill_only:
+        run_prefill_only(args, local_rank)
+    else:
+        run_ours(args, rank, local_rank, world)
 
 
 if __name__ == "__main__":
