@@ -18,7 +18,8 @@
 //                          stream (programmatic dependent launch), so they overlap its run; a kernel lets its
 //                          own successor start once the predecessor is done, which keeps one kernel's worth of
 //                          prefetch in flight (deeper chains of waiting kernels cost more than they hide).
-//  gemm_tc_tiled_kernel    many rows (prompt pass): 128 x 256 output tiles, both operands by TMA.
+//  gemm_tc_tiled_kernel    many rows (prompt pass): 128 x 256 output tiles, both operands by TMA; persistent CTAs with two
+//                          accumulators in TMEM, so that a tile's epilogue runs under the next tile's MMAs.
 //
 // An output element's reduction order depends on (N, K) only, never on the number of rows, so a block
 // pass and a one-row pass give identical bits.
@@ -520,6 +521,7 @@ struct TcTiledArgs {
     int M, K, N;
     int seg_rows0, tiles0;   // first segment: output features, tiles of BN
     int seg_rows, tiles_per_seg;
+    int tiles_n, tiles_m;    // BN-wide feature tiles over all segments, 128-row tiles
     int* err_flag;
     EpiArgs e;
 };
@@ -532,7 +534,7 @@ template <int BN> struct TctCfg {
     static constexpr int STAGES = BN == 256 ? 4 : 6;
     static constexpr int STAGE_BYTES = (1 + BN / 128) * TCT_TILE_BYTES;   // token rows, then the weight rows (one box per 128)
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
-    static constexpr int TMEM_COLS = BN;
+    static constexpr int TMEM_COLS = 2 * BN;   // two accumulators
 };
 
 // Sixteen consecutive output features of one row.  n_local0 is a multiple of 16.
@@ -582,7 +584,10 @@ __device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int seg, int
     reinterpret_cast<uint4*>(dst)[1] = hi;
 }
 
-// grid: (tiles of BN output features over all segments, ceil(M / 128)); dynamic smem TctCfg<BN>::SMEM_BYTES.
+// Persistent: grid = min(tiles, SMs) CTAs, CTA b takes output tiles b, b + grid, ... (tile = (row tile, BN-wide feature
+// tile), feature tiles fastest).  The TMA ring runs on across tile boundaries, and two accumulators in TMEM alternate,
+// so that the epilogue of one tile (TMEM -> registers -> global) overlaps the MMAs of the next.
+// dynamic smem TctCfg<BN>::SMEM_BYTES.
 template <int EPI, int BN>
 __global__ void __launch_bounds__(TCT_THREADS)
 gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tm0,
@@ -591,23 +596,24 @@ gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tm
     extern __shared__ __align__(1024) unsigned char smem_dyn[];
     __shared__ __align__(8) uint64_t s_full[C::STAGES];
     __shared__ __align__(8) uint64_t s_empty[C::STAGES];
-    __shared__ __align__(8) uint64_t s_accum;
+    __shared__ __align__(8) uint64_t s_acc_full[2], s_acc_free[2];
     __shared__ uint32_t s_tmem;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t ring0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-    const int tile = blockIdx.x;
-    const int seg = tile < a.tiles0 ? 0 : 1 + (tile - a.tiles0) / a.tiles_per_seg;
-    const int n_local0 = (seg == 0 ? tile : tile - a.tiles0 - (seg - 1) * a.tiles_per_seg) * BN;
-    const int seg_rows = seg == 0 ? a.seg_rows0 : a.seg_rows;
-    const int seg_base = seg == 0 ? 0 : a.seg_rows0 + (seg - 1) * a.seg_rows;
-    const int m0 = blockIdx.y * 128;
     const int KB = (a.K + 63) >> 6;
+    const int total = a.tiles_n * a.tiles_m;
+    // feature tile -> (segment, first feature within it)
+    auto seg_of = [&](int tile_n, int& n_local0) {
+        const int seg = tile_n < a.tiles0 ? 0 : 1 + (tile_n - a.tiles0) / a.tiles_per_seg;
+        n_local0 = (seg == 0 ? tile_n : tile_n - a.tiles0 - (seg - 1) * a.tiles_per_seg) * BN;
+        return seg;
+    };
 
     if (warp == 5) {
         if (lane == 0) {
             for (int s = 0; s < C::STAGES; ++s) { mbar_init(smem_u32(&s_full[s]), 1); mbar_init(smem_u32(&s_empty[s]), 1); }
-            mbar_init(smem_u32(&s_accum), 1);
+            for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&s_acc_full[s]), 1); mbar_init(smem_u32(&s_acc_free[s]), 4); }   // free: one arrive per epilogue warp
             mbar_init_fence();
         }
         __syncwarp();
@@ -621,52 +627,110 @@ gemm_tc_tiled_kernel(const TcTiledArgs a, const __grid_constant__ CUtensorMap tm
 
     if (warp == 4) {
         if (lane == 0) {
-            const CUtensorMap* tw = seg == 0 ? &tm0 : (seg == 1 ? &tm1 : &tm2);
             tma_prefetch_desc(&tmx);
-            tma_prefetch_desc(tw);
-            for (int i = 0; i < KB; ++i) {
-                const int st = i % C::STAGES;
-                if (i >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1)) {
-                    tc_report(a.err_flag, TC_ERR_SLOT);
-                    break;
-                }
-                const uint32_t bar = smem_u32(&s_full[st]);
-                mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
-                tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES, &tmx, i * 64, m0, bar);
+            tma_prefetch_desc(&tm0);
+            long long g = 0;   // k-blocks issued by this CTA over all of its tiles: ring position
+            bool ok = true;
+            for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+                int n_local0;
+                const int seg = seg_of(t % a.tiles_n, n_local0);
+                const int m0 = (t / a.tiles_n) * 128;
+                const CUtensorMap* tw = seg == 0 ? &tm0 : (seg == 1 ? &tm1 : &tm2);
+                for (int i = 0; i < KB; ++i, ++g) {
+                    const int st = (int)(g % C::STAGES);
+                    if (g >= C::STAGES && !mbar_wait(smem_u32(&s_empty[st]), (uint32_t)((g / C::STAGES) - 1) & 1)) {
+                        tc_report(a.err_flag, TC_ERR_SLOT);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t bar = smem_u32(&s_full[st]);
+                    mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+                    tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES, &tmx, i * 64, m0, bar);
 #pragma unroll
-                for (int hb = 0; hb < BN / 128; ++hb)   // rows past the segment's end arrive as zeros
-                    tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES + (1 + hb) * TCT_TILE_BYTES, tw, i * 64, n_local0 + hb * 128, bar);
+                    for (int hb = 0; hb < BN / 128; ++hb)   // rows past the segment's end arrive as zeros
+                        tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES + (1 + hb) * TCT_TILE_BYTES, tw, i * 64, n_local0 + hb * 128, bar);
+                }
             }
         }
         __syncwarp();
     } else if (warp == 5) {
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(128, BN);
-            for (int i = 0; i < KB; ++i) {
-                const int st = i % C::STAGES;
-                if (!mbar_wait(smem_u32(&s_full[st]), (i / C::STAGES) & 1)) {
-                    tc_report(a.err_flag, TC_ERR_OPERANDS);
+            long long g = 0;
+            bool ok = true;
+            int it = 0;
+            for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
+                const int buf = it & 1;
+                // the accumulator's previous tile (two tiles back) must have been read out
+                if (it >= 2 && !mbar_wait(smem_u32(&s_acc_free[buf]), (uint32_t)((it >> 1) - 1) & 1)) {
+                    tc_report(a.err_flag, TC_ERR_ACCUM);
                     break;
                 }
                 tc_fence_after_sync();
-                const uint64_t da = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES);
-                const uint64_t db = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES + TCT_TILE_BYTES);
+                for (int i = 0; i < KB; ++i, ++g) {
+                    const int st = (int)(g % C::STAGES);
+                    if (!mbar_wait(smem_u32(&s_full[st]), (uint32_t)(g / C::STAGES) & 1)) {
+                        tc_report(a.err_flag, TC_ERR_OPERANDS);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint64_t da = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES);
+                    const uint64_t db = umma_desc_k_sw128(ring0 + st * C::STAGE_BYTES + TCT_TILE_BYTES);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
-                umma_commit(smem_u32(&s_empty[st]));
+                    for (int k = 0; k < 4; ++k) umma_bf16(tmem + buf * BN, da + 2 * k, db + 2 * k, idesc, (i | k) != 0 ? 1u : 0u);
+                    umma_commit(smem_u32(&s_empty[st]));
+                }
+                umma_commit(smem_u32(&s_acc_full[buf]));   // (also after a failed wait: the epilogue warps must not be left waiting)
             }
-            umma_commit(smem_u32(&s_accum));
         }
         __syncwarp();
     } else {
-        if (!mbar_wait(smem_u32(&s_accum), 0)) tc_report(a.err_flag, TC_ERR_ACCUM);
-        tc_fence_after_sync();
-        const int m = m0 + warp * 32 + lane;   // output row = TMEM lane
+        int it = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+            const int buf = it & 1;
+            int n_local0;
+            const int seg = seg_of(t % a.tiles_n, n_local0);
+            const int seg_rows = seg == 0 ? a.seg_rows0 : a.seg_rows;
+            const int seg_base = seg == 0 ? 0 : a.seg_rows0 + (seg - 1) * a.seg_rows;
+            if (!mbar_wait(smem_u32(&s_acc_full[buf]), (uint32_t)(it >> 1) & 1)) { tc_report(a.err_flag, TC_ERR_ACCUM); break; }
+            tc_fence_after_sync();
+            const int m = (t / a.tiles_n) * 128 + warp * 32 + lane;   // output row = TMEM lane
+            const uint32_t acc = tmem + (static_cast<uint32_t>(warp * 32) << 16) + buf * BN;
+            if (EPI == EPI_RESID && n_local0 + BN <= seg_rows && (a.e.ldo & 3) == 0 && (seg_base & 3) == 0) {
+                // residual add on whole tiles: the old values of 64 columns are fetched together (sixteen 16-byte loads in
+                // flight) before the accumulator is read, instead of one exposed round trip per 16 columns
+                float* prow = static_cast<float*>(a.e.out) + (size_t)min(m, a.M - 1) * a.e.ldo + seg_base + n_local0;
 #pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 16) {
-            float t[16];
-            tmem_ld16(tmem + (static_cast<uint32_t>(warp * 32) << 16) + c0, t);   // warp-wide: every lane takes part
-            if (m < a.M && n_local0 + c0 < seg_rows) epilogue16<EPI>(a.e, m, seg, seg_base, seg_rows, n_local0 + c0, t);
+                for (int c0 = 0; c0 < BN; c0 += 64) {
+                    float4 old[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) old[j] = __ldcg(reinterpret_cast<const float4*>(prow + c0) + j);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float v[16];
+                        tmem_ld16(acc + c0 + 16 * q, v);   // warp-wide: every lane takes part
+                        if (m < a.M) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float4 o = old[4 * q + i];
+                                reinterpret_cast<float4*>(prow + c0 + 16 * q)[i] =
+                                    make_float4(v[4 * i] + o.x, v[4 * i + 1] + o.y, v[4 * i + 2] + o.z, v[4 * i + 3] + o.w);
+                            }
+                        }
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 16) {
+                    float v[16];
+                    tmem_ld16(acc + c0, v);   // warp-wide: every lane takes part
+                    if (m < a.M && n_local0 + c0 < seg_rows) epilogue16<EPI>(a.e, m, seg, seg_base, seg_rows, n_local0 + c0, v);
+                }
+            }
+            tc_fence_before_sync();   // this warp's TMEM reads are done: the accumulator may be overwritten
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_acc_free[buf]));
         }
     }
     tc_fence_before_sync();

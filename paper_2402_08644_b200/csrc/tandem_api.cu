@@ -453,7 +453,9 @@ void launch_tc_tiled_bn(tandem_ctx& c, TcTiledArgs& a, const CUtensorMap& tmx, c
     ensure_dyn_smem(gemm_tc_tiled_kernel<EPI, BN>, C::SMEM_BYTES, attr_done);
     a.tiles0 = cdiv(w.seg_rows0, BN);
     a.tiles_per_seg = cdiv(w.seg_rows, BN);
-    launch_ex(c, false, 1, gemm_tc_tiled_kernel<EPI, BN>, dim3(a.tiles0 + (w.n_segs - 1) * a.tiles_per_seg, cdiv(M, 128)), dim3(TCT_THREADS), (size_t)C::SMEM_BYTES,
+    a.tiles_n = a.tiles0 + (w.n_segs - 1) * a.tiles_per_seg;
+    a.tiles_m = cdiv(M, 128);
+    launch_ex(c, false, 1, gemm_tc_tiled_kernel<EPI, BN>, dim3(std::min(a.tiles_n * a.tiles_m, std::max(1, c.n_sms))), dim3(TCT_THREADS), (size_t)C::SMEM_BYTES,
               a, tmx, w.tm[0], w.tm[1], w.tm[2]);
 }
 
