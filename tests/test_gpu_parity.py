@@ -486,7 +486,7 @@ def test_bf16_self_tandem_accepts_drafts_naturally():
     assert sum(a == 4 for a in accepts) >= 0.75 * len(accepts)
 
 
-@pytest.mark.parametrize("batch,gamma", [(16, 3), (12, 5), (23, 2)])      # 64, 72 and 69 block rows
+@pytest.mark.parametrize("batch,gamma", [(16, 3), (12, 5), (23, 2), (16, 15)])      # 64, 72, 69 and 256 block rows (the longest block: 16 rows per sequence)
 def test_bf16_many_block_rows_replay_and_equal_greedy(batch, gamma):
     """Blocks of exactly 64 rows (the widest single pass over the weights) and of more than 64 rows (the weights
     are then read once per group of 64 rows): logits, accept lengths and counts against the checker with hashed
