@@ -148,6 +148,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     const int j_first = S == 1 ? 0 : sp * rpc;
     const int j_count = max(0, min(rpc, a.rows - j_first));
     float hres[EPI == EPI_RESID ? NB : 1];   // EPI_RESID: the residual values this thread's outputs are added to
+    int my_seq = 0, my_pos = 0;              // EPI_QKV / EPI_KV, threads below a.rows: this token row's sequence and position
 
     if (warp == 5) {
         if (lane == 0) {
@@ -223,10 +224,10 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     pdl_wait();   // x, and everything the epilogue touches, comes from earlier kernels; gains and biases are parameters
     pdl_launch_dependents();   // only now: one successor at a time sets up and fetches weights behind this kernel
     if (EPI == EPI_QKV || EPI == EPI_KV) {
-        // cache index of (row j, head h, element el) = ((seq_j * H + h) * t_max + pos_j) * d_head + el: the row part once per row
-        if (tid < a.rows)
-            s_rowoff[tid] = ((long long)a.e.row_seq[tid] * a.e.n_heads * a.e.t_max + a.e.row_pos[tid]) * a.e.d_head;
-        bar_sync(1, 128);
+        // cache index of (row j, head h, element el) = ((seq_j * H + h) * t_max + pos_j) * d_head + el: the row part once
+        // per row.  Only the epilogue needs it: the two loads are in flight while the B operand is produced, and the
+        // barrier that publishes the offsets sits after that.
+        if (tid < a.rows) { my_seq = a.e.row_seq[tid]; my_pos = a.e.row_pos[tid]; }   // first used ahead of the epilogue
     }
     if (EPI == EPI_RESID) {
         // the residual-stream values this thread will add to: fetched now, off the critical path
@@ -407,6 +408,10 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     float v[NB];
     const int tl = warp * 32 + lane;
     if (warp < 4) {
+        if (EPI == EPI_QKV || EPI == EPI_KV) {
+            if (tid < a.rows) s_rowoff[tid] = ((long long)my_seq * a.e.n_heads * a.e.t_max + my_pos) * a.e.d_head;
+            bar_sync(1, 128);
+        }
         if (!mbar_wait(smem_u32(&s_accum), 0, poll_limit)) tc_report(a.err_flag, TC_ERR_ACCUM);
         tc_fence_after_sync();
 #pragma unroll
