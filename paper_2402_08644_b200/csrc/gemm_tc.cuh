@@ -222,7 +222,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         }
     }
     pdl_wait();   // x, and everything the epilogue touches, comes from earlier kernels; gains and biases are parameters
-    pdl_launch_dependents();   // only now: one successor at a time sets up and fetches weights behind this kernel
     if (EPI == EPI_QKV || EPI == EPI_KV) {
         // cache index of (row j, head h, element el) = ((seq_j * H + h) * t_max + pos_j) * d_head + el: the row part once
         // per row.  Only the epilogue needs it: the two loads are in flight while the B operand is produced, and the
@@ -408,6 +407,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     float v[NB];
     const int tl = warp * 32 + lane;
     if (warp < 4) {
+        // Only now may the successor start: it sets up and fetches its first weight tiles behind this kernel's MMAs and
+        // epilogue.  Letting it start right after the wait above measured 2-3 % slower per iteration (its CTAs'
+        // set-up and loads then compete with this kernel's token-row loads); later than here (after the accumulator
+        // is ready, or after the exchange) slower again (the successor's head start shrinks).
+        pdl_launch_dependents();
         if (EPI == EPI_QKV || EPI == EPI_KV) {
             if (tid < a.rows) s_rowoff[tid] = ((long long)my_seq * a.e.n_heads * a.e.t_max + my_pos) * a.e.d_head;
             bar_sync(1, 128);
