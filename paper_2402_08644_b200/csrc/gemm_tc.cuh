@@ -35,7 +35,7 @@ namespace tandem {
 // LayerNorm, then value + remainder; PRO_F32: fp32 rows as value + remainder.
 enum { PRO_BF16 = 0, PRO_LN = 1, PRO_F32 = 2 };
 constexpr int EPI_ARGMAX = 6;                       // fp32 store plus the (max, index) of each row within the tile
-enum { TC_ERR_SLOT = 1, TC_ERR_OPERANDS = 2, TC_ERR_ACCUM = 3 };   // which bounded wait gave up
+enum { TC_ERR_SLOT = 1, TC_ERR_OPERANDS = 2, TC_ERR_ACCUM = 3, TC_ERR_EXCHANGE = 4 };   // which bounded wait gave up
 
 struct TcDecodeArgs {
     const void* x;          // PRO_BF16: bf16 [rows][ldx];  PRO_LN / PRO_F32: float [rows][ldx]
@@ -117,6 +117,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     __shared__ __align__(8) uint64_t s_full[C::STAGES];
     __shared__ __align__(8) uint64_t s_empty[C::STAGES];
     __shared__ __align__(8) uint64_t s_accum;
+    __shared__ __align__(8) uint64_t s_inbox;   // counts the bytes of the K-slices' partial sums sent to this CTA
     __shared__ uint32_t s_tmem;
     __shared__ float s_mu[NB], s_rstd[NB];
     __shared__ float s_av[4][NB];
@@ -157,6 +158,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                 mbar_init(smem_u32(&s_empty[s]), 1);   // the MMA thread's commit
             }
             mbar_init(smem_u32(&s_accum), 1);
+            mbar_init(smem_u32(&s_inbox), 1);
             mbar_init_fence();
         }
         __syncwarp();
@@ -463,21 +465,25 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     } else {
         if (S > 1) {
             // The cluster's CTAs hold the K-slices of one tile, and CTA r finishes token rows [r * rpc, (r + 1) * rpc).
-            // Every CTA sends each row's partial sums to the inbox of the CTA that finishes it (remote shared-memory
-            // stores), one cluster barrier makes them visible, and each CTA sums its inbox in slice order.  Nobody
-            // touches a peer's shared memory after the barrier, so CTAs may leave as they finish.
+            // Every CTA sends each row's partial sums to the inbox of the CTA that finishes it, with stores that count
+            // their bytes on the receiver's inbox barrier; a CTA that finishes rows waits until S x rows x 128 floats
+            // have arrived and sums its inbox in slice order.  No cluster-wide barrier: a CTA without rows of its own
+            // leaves right after sending, the others once everything addressed to them has arrived (nothing is
+            // written into a CTA's shared memory after that).
             const uint32_t inbox0 = ring0 + C::STAGES * C::STAGE_BYTES;           // [S][rpc][128] fp32
             cluster_wait();   // closes the opening handshake: every CTA of the cluster is running
             if (warp < 4) {
+                const uint32_t ibar = smem_u32(&s_inbox);
+                if (tid == 0 && j_count > 0) mbar_arrive_expect_tx(ibar, (uint32_t)(S * j_count * 128 * 4));
                 int dst = 0, jj = 0;
 #pragma unroll
                 for (int j = 0; j < NB; ++j) {
                     if (j >= a.rows) break;
-                    st_dsmem_f32(inbox0 + ((sp * rpc + jj) * 128 + tl) * 4, dst, v[j]);
+                    st_async_dsmem_f32(inbox0 + ((sp * rpc + jj) * 128 + tl) * 4, ibar, dst, v[j]);
                     if (++jj == rpc) { jj = 0; ++dst; }
                 }
+                if (j_count > 0 && !mbar_wait(ibar, 0, poll_limit)) tc_report(a.err_flag, TC_ERR_EXCHANGE);
             }
-            cluster_sync_all();
             if (warp < 4) {
                 const float* inbox = reinterpret_cast<const float*>(ring + C::STAGES * C::STAGE_BYTES);
 #pragma unroll

@@ -159,6 +159,17 @@ __device__ __forceinline__ void st_dsmem_f32(uint32_t local_smem_addr, int rank,
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
 }
 
+// Writes a float to the same shared-memory offset in the cluster's CTA number `rank` and counts its four bytes on the
+// mbarrier at `local_bar`'s offset in that CTA: the receiver learns of the data from its own barrier, with no fence
+// and no cluster-wide barrier in between.
+__device__ __forceinline__ void st_async_dsmem_f32(uint32_t local_smem_addr, uint32_t local_bar, int rank, float v) {
+    uint32_t ra, rb;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_smem_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rb) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(ra), "r"(__float_as_uint(v)), "r"(rb) : "memory");
+}
+
 // Named barrier among a subset of the CTA's warps.
 __device__ __forceinline__ void bar_sync(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 
