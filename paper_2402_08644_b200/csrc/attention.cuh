@@ -36,6 +36,7 @@ struct AttnArgs {
     int nq;
     int n_heads, t_max;
     int n_kv_heads;                      // key/value heads of the caches; 0 = n_heads.  Query head h reads kv head h / (n_heads / n_kv_heads)
+    int* err_flag;                       // attn_decode_kernel: where a bounded wait that ran out records its code (nullable)
     int heads_per_cta;                   // attn_decode_kernel: query heads of one key/value head served by one CTA (their rows share
                                          // the 16-row tile: heads_per_cta * nq <= 16); 0 = 1.  grid.y = n_heads / heads_per_cta
     float* part_ml;                      // split mode: [M][H][n_chunks_max][2]
@@ -247,6 +248,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(AttnArgs a) {
 // ---------------------------------------------------------------------------------------------------
 constexpr int ATD_THREADS = 256;
 constexpr int ATD_WARPS = ATD_THREADS / 32;
+constexpr int ATD_ERR_EXCHANGE = 5;                                 // error code: the wait for the cluster's states gave up
 constexpr int ATD_CLUSTER = 8;                                      // largest cluster; launches use 1, 2, 4 or 8
 constexpr int ATD_SLOTS = ATT_NQ;                                   // inbox states per CTA: cluster size x queries it finishes <= 16
 constexpr int ATD_WROWS = ATT_CH / ATD_WARPS;                       // positions of a chunk per warp (16)
@@ -313,6 +315,8 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     const int h = blockIdx.y * gpc;                // first query head of this CTA
     const int CL = gridDim.x;                      // cluster size
     const int QPC = (ATT_NQ + CL - 1) / CL;        // queries a CTA finishes at most
+    __shared__ __align__(8) uint64_t s_inbox_bar;  // counts the bytes of the states sent to this CTA by the cluster's CTAs
+    if (CL > 1 && tid == 0) { mbar_init(smem_u32(&s_inbox_bar), 1); mbar_init_fence(); }
     if (CL > 1) cluster_arrive_relaxed();          // opening handshake: waited for just before the first remote store
     bf16* ring = ring_all + (size_t)warp * C::STAGES * C::STAGE_ELEMS;
     const uint32_t ring_s = smem_u32(ring);
@@ -559,10 +563,20 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
             }
         }
         float* slot = inbox + ((size_t)rank * QPC + qa / CL) * SW + e;
-        if (CL > 1) st_dsmem_f32(smem_u32(slot), qa % CL, val);
+        if (CL > 1) st_async_dsmem_f32(smem_u32(slot), smem_u32(&s_inbox_bar), qa % CL, val);   // counted on the receiver's barrier
         else *slot = val;
     }
-    if (CL > 1) cluster_sync_all(); else __syncthreads();
+    if (CL > 1) {
+        // This CTA finishes queries rank, rank + CL, ...: it waits (bounded) until every CTA's state of each of them
+        // has arrived.  No cluster-wide barrier: a CTA without queries of its own leaves right after sending.
+        const int n_fin = rank < cnt ? (cnt - rank + CL - 1) / CL : 0;
+        if (n_fin > 0) {
+            if (tid == 0) mbar_arrive_expect_tx(smem_u32(&s_inbox_bar), (uint32_t)(CL * n_fin * SW * 4));
+            if (!mbar_wait(smem_u32(&s_inbox_bar), 0) && a.err_flag) atomicExch(a.err_flag, ATD_ERR_EXCHANGE);
+        }
+    } else {
+        __syncthreads();
+    }
     for (int u = 0; u < QPC; ++u) {
         const int qi = rank + u * CL;
         if (qi < cnt && tid < DH) {

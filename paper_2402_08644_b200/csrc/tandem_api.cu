@@ -658,6 +658,7 @@ void attention_decode(tandem_ctx& c, const Model& m, int l, const bf16* q, float
     aa.q = q; aa.ldq = d; aa.kcache = kv_ptr<bf16>(c, m, l, 0); aa.vcache = kv_ptr<bf16>(c, m, l, 1);
     aa.out = o; aa.ldo = d; aa.out_f32 = 1; aa.row_seq = at<int>(c, c.lay.row_seq); aa.row_pos = at<int>(c, c.lay.row_pos);
     aa.nq = r.nq; aa.n_heads = H; aa.n_kv_heads = m.kv_heads; aa.t_max = c.cfg.max_seq; aa.scale = 1.0f / sqrtf((float)dh);
+    aa.err_flag = tc_scratch(c).err;
     launch_attn_decode(c, dh, aa, r.groups, r.kv_positions * 2.0 * d * 2.0);
 }
 
