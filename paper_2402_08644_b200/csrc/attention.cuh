@@ -580,14 +580,25 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     for (int u = 0; u < QPC; ++u) {
         const int qi = rank + u * CL;
         if (qi < cnt && tid < DH) {
+            // the CTAs' states in rank order; all loads and exponentials first, then the two sums (same order as a plain loop)
+            float mr[ATD_CLUSTER], lr[ATD_CLUSTER], orr[ATD_CLUSTER];
             float mx = -INFINITY;
-            for (int r = 0; r < CL; ++r) mx = fmaxf(mx, inbox[((size_t)r * QPC + u) * SW + DH]);
-            float l = 0.f, ov = 0.f;
-            for (int r = 0; r < CL; ++r) {
+#pragma unroll
+            for (int r = 0; r < ATD_CLUSTER; ++r) {
                 const float* st = inbox + ((size_t)r * QPC + u) * SW;
-                const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
-                l = fmaf(st[DH + 1], f, l);
-                ov = fmaf(st[tid], f, ov);
+                mr[r] = r < CL ? st[DH] : -INFINITY;
+                lr[r] = r < CL ? st[DH + 1] : 0.f;
+                orr[r] = r < CL ? st[tid] : 0.f;
+                mx = fmaxf(mx, mr[r]);
+            }
+            float l = 0.f, ov = 0.f;
+#pragma unroll
+            for (int r = 0; r < ATD_CLUSTER; ++r) {
+                if (r < CL) {
+                    const float f = mr[r] > -INFINITY ? __expf(mr[r] - mx) : 0.f;
+                    l = fmaf(lr[r], f, l);
+                    ov = fmaf(orr[r], f, ov);
+                }
             }
             const int hq = qi / nq;                  // tile row qi = query head hq of this CTA, block row qi - hq * nq
             const size_t oi = (size_t)(row0 + qi - hq * nq) * a.ldo + (h + hq) * DH + tid;
