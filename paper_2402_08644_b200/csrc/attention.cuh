@@ -392,7 +392,6 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
         }
     }
     pdl_wait();   // queries and the newest keys/values come from the kernel before this one
-    pdl_launch_dependents();
 #pragma unroll
     for (int it = 0; it < C::STAGES - 1; ++it) {
         if (it >= pre) {
@@ -521,6 +520,7 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
         }
         __syncwarp();   // the stage may be refilled by this warp's next issue
     }
+    pdl_launch_dependents();   // the successor starts behind the merge, not behind this kernel's loads (measured: a little faster)
     // a row's sum: add the quad's lanes
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
     l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
