@@ -250,6 +250,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
             for (int u = 0; u < 8; ++u) tn[u] = (lane + 32 * u < K4) ? __ldcg(xr + lane + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        pdl_launch_dependents();   // (a K-slice that fits the ring: see the note at the epilogue)
         for (int r = warp; r < a.rows; r += 4) {
             float4 t[8];
 #pragma unroll
@@ -361,6 +362,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                         raw32[g][ch][1] = live ? __ldcg(xp + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
+            if (nkb <= C::STAGES) pdl_launch_dependents();   // (a K-slice that fits the ring: see the note at the epilogue)
             bool dead = false;
 #pragma unroll
             for (int g = 0; g < C::STAGES; ++g) {
@@ -409,10 +411,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     float v[NB];
     const int tl = warp * 32 + lane;
     if (warp < 4) {
-        // Only now may the successor start: it sets up and fetches its first weight tiles behind this kernel's MMAs and
-        // epilogue.  Letting it start right after the wait above measured 2-3 % slower per iteration (its CTAs'
-        // set-up and loads then compete with this kernel's token-row loads); later than here (after the accumulator
-        // is ready, or after the exchange) slower again (the successor's head start shrinks).
+        // The successor may start (set up, fetch its first weight tiles) once this kernel's token-row loads are out of
+        // its way: right after they have been issued when the K-slice fits the ring (one round of loads; see above),
+        // else here, after the last round has been written.  Letting it start right after the wait measured 2-3 %
+        // slower per iteration (its CTAs' set-up and loads compete with the row loads); later than here (after the
+        // accumulator is ready, or after the exchange) slower again (the successor's head start shrinks).
         pdl_launch_dependents();
         if (EPI == EPI_QKV || EPI == EPI_KV) {
             if (tid < a.rows) s_rowoff[tid] = ((long long)my_seq * a.e.n_heads * a.e.t_max + my_pos) * a.e.d_head;
