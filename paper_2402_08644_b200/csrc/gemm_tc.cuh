@@ -211,6 +211,11 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             umma_commit(smem_u32(&s_accum));
         }
         __syncwarp();
+        // TMEM goes back as soon as the epilogue warps have read the accumulator (they arrive on barrier 2 right after
+        // their loads), not at the end of the kernel: nothing is left to do for this warp after that.
+        asm volatile("bar.sync 2, 160;" ::: "memory");
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, C::TMEM_COLS);
     } else {
     // ---- warps 0-3: token rows into the B stages (then the epilogue) ----
     float4 gq[C::STAGES], bq[C::STAGES];   // register path: gain / bias of this lane's slot in each of the CTA's K-blocks
@@ -432,6 +437,8 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[c0 + i] = t[i] + u[i];
         }
+        tc_fence_before_sync();
+        asm volatile("bar.arrive 2, 160;" ::: "memory");   // the accumulator has been read: warp 5 may free the TMEM columns
     }
     const int n_local = n_local0 + tl;                 // warps 0-3: this thread's output feature
     const bool valid = n_local < seg_rows;
@@ -526,9 +533,6 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
             }
         }
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
 // ---------------------------------------------------------------------------------------------------
