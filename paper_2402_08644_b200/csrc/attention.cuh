@@ -37,6 +37,8 @@ struct AttnArgs {
     int n_heads, t_max;
     int n_kv_heads;                      // key/value heads of the caches; 0 = n_heads.  Query head h reads kv head h / (n_heads / n_kv_heads)
     int* err_flag;                       // attn_decode_kernel: where a bounded wait that ran out records its code (nullable)
+    void* out_lo;                        // attn_decode_kernel, optional: `out` is then the bf16 plane of the values and this the bf16
+                                         // plane of the remainders (fp32 result = value + remainder), both [M][ldo]
     int heads_per_cta;                   // attn_decode_kernel: query heads of one key/value head served by one CTA (their rows share
                                          // the 16-row tile: heads_per_cta * nq <= 16); 0 = 1.  grid.y = n_heads / heads_per_cta
     float* part_ml;                      // split mode: [M][H][n_chunks_max][2]
@@ -602,8 +604,13 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
             }
             const int hq = qi / nq;                  // tile row qi = query head hq of this CTA, block row qi - hq * nq
             const size_t oi = (size_t)(row0 + qi - hq * nq) * a.ldo + (h + hq) * DH + tid;
-            if (a.out_f32) static_cast<float*>(a.out)[oi] = ov / l;
-            else static_cast<bf16*>(a.out)[oi] = __float2bfloat16_rn(ov / l);
+            const float res = ov / l;
+            if (a.out_lo) {
+                const bf16 hi = __float2bfloat16_rn(res);
+                static_cast<bf16*>(a.out)[oi] = hi;
+                static_cast<bf16*>(a.out_lo)[oi] = __float2bfloat16_rn(res - __bfloat162float(hi));
+            } else if (a.out_f32) static_cast<float*>(a.out)[oi] = res;
+            else static_cast<bf16*>(a.out)[oi] = __float2bfloat16_rn(res);
         }
     }
 }

@@ -24,6 +24,8 @@ struct EpiArgs {
     int n_heads, d_head, t_max;   // n_heads: key/value heads of the cache
     int seg0;             // QKV / KV: columns of the first segment (QKV: the queries, d_model; KV: the keys)
     int seg;              //           columns of every further segment (keys / values: kv heads * d_head)
+    void* out_lo;         // EPI_GELU on the tensor-core decode path, optional: `out` is then the bf16 plane of the values and this
+                          // the bf16 plane of the remainders (x = value + remainder), both [M][ldo], for a consumer that loads them by TMA
     void* snap;           // EPI_RESID on the tensor-core decode path: optional fp32 copy of the new values [M][snap_ld]
     int snap_ld;
 };

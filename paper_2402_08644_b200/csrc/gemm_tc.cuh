@@ -32,14 +32,19 @@
 namespace tandem {
 
 // How the token rows become the B operand: PRO_BF16: bf16 rows as they are (remainder rows zero); PRO_LN: fp32 rows,
-// LayerNorm, then value + remainder; PRO_F32: fp32 rows as value + remainder.
-enum { PRO_BF16 = 0, PRO_LN = 1, PRO_F32 = 2 };
+// LayerNorm, then value + remainder; PRO_F32: fp32 rows as value + remainder; PRO_TMA: the producer of the rows has
+// already written them as two bf16 planes (values, remainders), and TMA brings them into the B stages beside the
+// weights (no registers, no rounds, nothing for warps 0-3 to do before the epilogue).
+enum { PRO_BF16 = 0, PRO_LN = 1, PRO_F32 = 2, PRO_TMA = 3 };
 constexpr int EPI_ARGMAX = 6;                       // fp32 store plus the (max, index) of each row within the tile
 enum { TC_ERR_SLOT = 1, TC_ERR_OPERANDS = 2, TC_ERR_ACCUM = 3, TC_ERR_EXCHANGE = 4 };   // which bounded wait gave up
 
 struct TcDecodeArgs {
-    const void* x;          // PRO_BF16: bf16 [rows][ldx];  PRO_LN / PRO_F32: float [rows][ldx]
+    const void* x;          // PRO_BF16: bf16 [rows][ldx];  PRO_LN / PRO_F32: float [rows][ldx];  PRO_TMA: unused (tensor map)
     int ldx;
+    int x_row0, x_plane_rows;   // PRO_TMA: first token row of this launch; rows between the value and the remainder plane
+    int release_early;          // PRO_TMA: the successor is released right after the wait on the predecessor (a small matrix:
+                                // a chain of dependent steps, nothing to protect) instead of after the last token-row loads
     const float* ln_g;      // PRO_LN: LayerNorm gain / bias [K]
     const float* ln_b;
     int rows, K, N;         // N = output features over all segments
@@ -111,7 +116,7 @@ __device__ __forceinline__ ScatterCol scatter_col(const EpiArgs& e, int seg, int
 template <int NB, int PRO, int EPI>
 __global__ void __launch_bounds__(TCD_THREADS)
 gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap tm0, const __grid_constant__ CUtensorMap tm1,
-                      const __grid_constant__ CUtensorMap tm2) {
+                      const __grid_constant__ CUtensorMap tm2, const __grid_constant__ CUtensorMap tmx) {
     using C = TcdCfg<NB>;
     extern __shared__ __align__(1024) unsigned char smem_dyn[];
     __shared__ __align__(8) uint64_t s_full[C::STAGES];
@@ -154,7 +159,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
     if (warp == 5) {
         if (lane == 0) {
             for (int s = 0; s < C::STAGES; ++s) {
-                mbar_init(smem_u32(&s_full[s]), 5);    // the TMA thread's arrive + one arrive per B-operand warp
+                mbar_init(smem_u32(&s_full[s]), PRO == PRO_TMA ? 2 : 5);   // the TMA thread's arrive + one per B-operand warp (PRO_TMA: its second arrive)
                 mbar_init(smem_u32(&s_empty[s]), 1);   // the MMA thread's commit
             }
             mbar_init(smem_u32(&s_accum), 1);
@@ -173,7 +178,44 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
 
     if (warp == 4) {
         // ---- weight tiles: independent of every earlier kernel, so no wait on the predecessor here ----
-        if (lane == 0 && !a.withhold_weights) {
+        if (PRO == PRO_TMA && lane == 0 && !a.withhold_weights) {
+            // Weights of the first ring-ful before the wait on the predecessor, then the wait, then their token rows
+            // (two planes, 16-row boxes), then weights and rows together as stages come free.
+            const CUtensorMap* tm = seg == 0 ? &tm0 : (seg == 1 ? &tm1 : &tm2);
+            tma_prefetch_desc(tm);
+            tma_prefetch_desc(&tmx);
+            const uint64_t pol = l2_policy_evict_first();
+            auto load_a = [&](int i, int st) {
+                const uint32_t bar = smem_u32(&s_full[st]);
+                mbar_arrive_expect_tx(bar, C::A_BYTES);
+                if (a.stream_weights) tma_load_2d(ring0 + st * C::STAGE_BYTES, tm, (kb0 + i) * 64, n_local0, bar, pol);
+                else tma_load_2d_nohint(ring0 + st * C::STAGE_BYTES, tm, (kb0 + i) * 64, n_local0, bar);
+            };
+            auto load_b = [&](int i, int st) {
+                const uint32_t bar = smem_u32(&s_full[st]);
+                const uint32_t dst = ring0 + st * C::STAGE_BYTES + C::A_BYTES;
+                mbar_arrive_expect_tx(bar, C::B_BYTES);
+#pragma unroll
+                for (int r16 = 0; r16 < NB; r16 += 16) {
+                    tma_load_2d_nohint(dst + r16 * 128, &tmx, (kb0 + i) * 64, a.x_row0 + r16, bar);                          // values
+                    tma_load_2d_nohint(dst + (NB + r16) * 128, &tmx, (kb0 + i) * 64, a.x_plane_rows + a.x_row0 + r16, bar);   // remainders
+                }
+            };
+            const int n_pre = min(nkb, C::STAGES);
+            for (int i = 0; i < n_pre; ++i) load_a(i, i);
+            pdl_wait();
+            for (int i = 0; i < n_pre; ++i) load_b(i, i);
+            for (int i = n_pre; i < nkb; ++i) {
+                const int st = i % C::STAGES;
+                if (!mbar_wait(smem_u32(&s_empty[st]), ((i / C::STAGES) - 1) & 1, poll_limit)) {
+                    tc_report(a.err_flag, TC_ERR_SLOT);
+                    break;
+                }
+                load_a(i, st);
+                load_b(i, st);
+            }
+            pdl_launch_dependents();   // the last token rows are on their way: the successor may start (see the note at the epilogue)
+        } else if (lane == 0 && !a.withhold_weights) {
             const CUtensorMap* tm = seg == 0 ? &tm0 : (seg == 1 ? &tm1 : &tm2);
             tma_prefetch_desc(tm);
             const uint64_t pol = l2_policy_evict_first();
@@ -305,7 +347,7 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         __syncwarp();
         if (lane == 0)
             for (int i = 0; i < nkb; ++i) mbar_arrive(smem_u32(&s_full[i]));
-    } else {
+    } else if (PRO != PRO_TMA) {
         // general case: statistics (LayerNorm), then the K-blocks a ring's worth at a time
         if (PRO == PRO_LN) {
             for (int r = warp; r < a.rows; r += 4) {   // one warp per row, fixed lane-strided order
@@ -421,7 +463,9 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
         // else here, after the last round has been written.  Letting it start right after the wait measured 2-3 %
         // slower per iteration (its CTAs' set-up and loads compete with the row loads); later than here (after the
         // accumulator is ready, or after the exchange) slower again (the successor's head start shrinks).
-        pdl_launch_dependents();
+        // (PRO_TMA with a K-slice longer than the ring and a matrix large enough to be a stream: the TMA thread does it, after
+        // its last loads; otherwise there is nothing of this kernel's in the successor's way, and it is released at once)
+        if (PRO != PRO_TMA || nkb <= C::STAGES || a.release_early) pdl_launch_dependents();
         if (EPI == EPI_QKV || EPI == EPI_KV) {
             if (tid < a.rows) s_rowoff[tid] = ((long long)my_seq * a.e.n_heads * a.e.t_max + my_pos) * a.e.d_head;
             bar_sync(1, 128);
@@ -521,8 +565,15 @@ gemm_tc_decode_kernel(const TcDecodeArgs a, const __grid_constant__ CUtensorMap 
                         if (EPI == EPI_RESID || EPI == EPI_STORE_F32) {
                             static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = hv;
                             if (EPI == EPI_RESID && a.e.snap) static_cast<float*>(a.e.snap)[(size_t)j * a.e.snap_ld + n] = hv;
-                        } else if (EPI == EPI_GELU) {   // activations between the decode kernels stay fp32
-                            static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = gelu_bf16_out(hv);
+                        } else if (EPI == EPI_GELU) {   // activations between the decode kernels stay fp32, or value + remainder planes
+                            const float gv = gelu_bf16_out(hv);
+                            if (a.e.out_lo) {
+                                const bf16 hi = __float2bfloat16_rn(gv);
+                                static_cast<bf16*>(a.e.out)[(size_t)j * a.e.ldo + n] = hi;
+                                static_cast<bf16*>(a.e.out_lo)[(size_t)j * a.e.ldo + n] = __float2bfloat16_rn(gv - __bfloat162float(hi));
+                            } else {
+                                static_cast<float*>(a.e.out)[(size_t)j * a.e.ldo + n] = gv;
+                            }
                         } else if (EPI == EPI_QKV || EPI == EPI_KV) {
                             sc.base[(sc.is_q ? (long long)j * a.e.ldo : s_rowoff[j]) + sc.col] = __float2bfloat16_rn(hv);
                         } else {

@@ -149,17 +149,32 @@ __device__ __forceinline__ void ln_store4(bf16* orow, int k4, float y0, float y1
     const __nv_bfloat162 lo = __floats2bfloat162_rn(y0, y1), hi = __floats2bfloat162_rn(y2, y3);
     reinterpret_cast<uint2*>(orow)[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
 }
+// value plane + remainder plane (x = bf16(x) + bf16(x - bf16(x))), for a GEMM that loads its token rows by TMA
+__device__ __forceinline__ void ln_store4_split(bf16* vrow, bf16* rrow, int k4, float y0, float y1, float y2, float y3) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(y0, y1), b = __floats2bfloat162_rn(y2, y3);
+    const __nv_bfloat162 ra = __floats2bfloat162_rn(y0 - __low2float(a), y1 - __high2float(a));
+    const __nv_bfloat162 rb = __floats2bfloat162_rn(y2 - __low2float(b), y3 - __high2float(b));
+    reinterpret_cast<uint2*>(vrow)[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+    reinterpret_cast<uint2*>(rrow)[k4] = make_uint2(*reinterpret_cast<const uint32_t*>(&ra), *reinterpret_cast<const uint32_t*>(&rb));
+}
+__device__ __forceinline__ void ln_store4(float* orow, bf16*, int k4, float y0, float y1, float y2, float y3) { ln_store4(orow, k4, y0, y1, y2, y3); }
+__device__ __forceinline__ void ln_store4(bf16* orow, bf16* rrow, int k4, float y0, float y1, float y2, float y3) {
+    if (rrow) ln_store4_split(orow, rrow, k4, y0, y1, y2, y3);
+    else ln_store4(orow, k4, y0, y1, y2, y3);
+}
 
 // Decode-path LayerNorm of fp32 rows ahead of the tensor-core GEMMs (fp32 out; bf16 out for the stand-alone
 // projection above 64 rows): the row sits in registers between the passes (up to 4096 elements), loads and stores
 // are 16 bytes wide.  grid: rows; block: 128; d % 4 == 0.
 template <typename TO>
 __global__ void __launch_bounds__(128) layernorm_rows_kernel(const float* __restrict__ x, const float* __restrict__ gain,
-                                                             const float* __restrict__ bias, TO* __restrict__ out, int d) {
+                                                             const float* __restrict__ bias, TO* __restrict__ out, int d,
+                                                             bf16* out_lo = nullptr) {
     __shared__ float red[4];
     const int d4 = d >> 2;
     const float4* xr = reinterpret_cast<const float4*>(x + (size_t)blockIdx.x * d);
     TO* orow = out + (size_t)blockIdx.x * d;
+    bf16* rrow = out_lo ? out_lo + (size_t)blockIdx.x * d : nullptr;   // TO = bf16 only: the remainder plane's row
     if (d4 <= 8 * 128) {
         // gains and biases are parameters: fetched while the kernel that writes x is still running
         float4 gq[8], bq[8];
@@ -192,7 +207,7 @@ __global__ void __launch_bounds__(128) layernorm_rows_kernel(const float* __rest
             const int k4 = threadIdx.x + 128 * u;
             if (k4 < d4) {
                 const float4 g = gq[u], b = bq[u];
-                ln_store4(orow, k4, (t[u].x - mu) * rs * g.x + b.x, (t[u].y - mu) * rs * g.y + b.y,
+                ln_store4(orow, rrow, k4, (t[u].x - mu) * rs * g.x + b.x, (t[u].y - mu) * rs * g.y + b.y,
                           (t[u].z - mu) * rs * g.z + b.z, (t[u].w - mu) * rs * g.w + b.w);
             }
         }
@@ -212,7 +227,7 @@ __global__ void __launch_bounds__(128) layernorm_rows_kernel(const float* __rest
         for (int k4 = threadIdx.x; k4 < d4; k4 += 128) {
             const float4 t = __ldcg(xr + k4);
             const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + k4), b = __ldg(reinterpret_cast<const float4*>(bias) + k4);
-            ln_store4(orow, k4, (t.x - mu) * rs * g.x + b.x, (t.y - mu) * rs * g.y + b.y, (t.z - mu) * rs * g.z + b.z,
+            ln_store4(orow, rrow, k4, (t.x - mu) * rs * g.x + b.x, (t.y - mu) * rs * g.y + b.y, (t.z - mu) * rs * g.z + b.z,
                       (t.w - mu) * rs * g.w + b.w);
         }
     }

@@ -122,6 +122,10 @@ struct tandem_ctx {
     bool use_pdl = true;                 // programmatic dependent launch between the decode kernels
     int n_sms = 0;                       // multiprocessors of the context's device: split-K decode GEMMs aim for about one CTA each
     std::vector<CUtensorMap> wmap;       // one per weight pointer (matrices only), box 128 rows x 64 columns
+    // Decode activations as two bf16 planes (values, then remainders, dec_rows rows each) that the consuming GEMM loads by
+    // TMA: maps of the LayerNorm / attention / GELU buffers, [buffer 0..2][0 large, 1 small], 16-row boxes.
+    CUtensorMap xmap[3][2];
+    bool xmap_ok = false;
     std::vector<char> wmap_ok;
     std::vector<CUtensorMap> kmap, vmap; // the large model's key / value cache of each layer as [(seq, head, position)][d_head]
     cudaStream_t side = nullptr;         // the decode-time FF_Tandem projections run here, beside the large model's later layers
@@ -393,11 +397,12 @@ void launch_ex(tandem_ctx& c, bool pdl, int cluster, void (*kernel)(KArgs...), d
 }
 
 template <int NB, int PRO, int EPI>
-void launch_tc_decode_nb(tandem_ctx& c, const TcDecodeArgs& a, const TcW& w, int units) {
+void launch_tc_decode_nb(tandem_ctx& c, const TcDecodeArgs& a, const TcW& w, int units, const CUtensorMap* xmap) {
     using C = TcdCfg<NB>;
     static std::atomic<unsigned long long> attr_done{0};
     ensure_dyn_smem(gemm_tc_decode_kernel<NB, PRO, EPI>, C::SMEM_BYTES, attr_done);
-    launch_ex(c, true, a.splits, gemm_tc_decode_kernel<NB, PRO, EPI>, dim3(units), dim3(TCD_THREADS), (size_t)C::SMEM_BYTES, a, w.tm[0], w.tm[1], w.tm[2]);
+    launch_ex(c, true, a.splits, gemm_tc_decode_kernel<NB, PRO, EPI>, dim3(units), dim3(TCD_THREADS), (size_t)C::SMEM_BYTES, a, w.tm[0], w.tm[1], w.tm[2],
+              xmap ? *xmap : w.tm[0]);
 }
 
 // y = prologue(x) W^T for few rows on the tensor cores, streaming W once per group of up to 64 rows (one group in
@@ -405,7 +410,7 @@ void launch_tc_decode_nb(tandem_ctx& c, const TcDecodeArgs& a, const TcW& w, int
 template <int PRO, int EPI>
 void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx, const void* ln_g, const void* ln_b, int rows,
                       const TcW& w, bool stream_weights, const EpiArgs& e, float* amax_val = nullptr, int* amax_idx = nullptr,
-                      int amax_stride = 0) {
+                      int amax_stride = 0, const CUtensorMap* xmap = nullptr, int x_plane_rows = 0) {
     if (rows <= 0) return;
     TcDecodeArgs a;
     memset(&a, 0, sizeof(a));
@@ -430,18 +435,21 @@ void launch_tc_decode(tandem_ctx& c, const TcScratch& sc, const void* x, int ldx
     for (int r0 = 0; r0 < rows; r0 += 64) {
         const int nr = std::min(64, rows - r0);
         a.rows = nr;
+        a.x_row0 = r0; a.x_plane_rows = x_plane_rows;
+        a.release_early = (size_t)a.N * (size_t)w.K * 2 <= ((size_t)16 << 20) ? 1 : 0;
         a.x = static_cast<const unsigned char*>(x) + (size_t)r0 * ldx * xsz;
         a.amax_val = amax_val ? amax_val + (size_t)r0 * amax_stride : nullptr;
         a.amax_idx = amax_idx ? amax_idx + (size_t)r0 * amax_stride : nullptr;
         a.e = e;
-        if (e.out) a.e.out = static_cast<unsigned char*>(e.out) + (size_t)r0 * e.ldo * (EPI == EPI_QKV ? 2 : osz);
+        if (e.out) a.e.out = static_cast<unsigned char*>(e.out) + (size_t)r0 * e.ldo * ((EPI == EPI_QKV || e.out_lo) ? 2 : osz);
+        if (e.out_lo) a.e.out_lo = static_cast<unsigned char*>(e.out_lo) + (size_t)r0 * e.ldo * 2;   // (value / remainder planes are bf16)
         if (e.row_seq) { a.e.row_seq = e.row_seq + r0; a.e.row_pos = e.row_pos + r0; }
         if (e.snap) a.e.snap = static_cast<float*>(e.snap) + (size_t)r0 * e.snap_ld;
         ProfScope ps(c, PC_GEMM_TC_DECODE, 2.0 * a.N * w.K + (double)nr * w.K * xsz + (double)nr * a.N * (EPI == EPI_QKV || EPI == EPI_KV || EPI == EPI_STORE ? 2.0 : 4.0));
-        if (nr <= 16) launch_tc_decode_nb<16, PRO, EPI>(c, a, w, units);
-        else if (nr <= 32) launch_tc_decode_nb<32, PRO, EPI>(c, a, w, units);
-        else if (nr <= 48) launch_tc_decode_nb<48, PRO, EPI>(c, a, w, units);
-        else launch_tc_decode_nb<64, PRO, EPI>(c, a, w, units);
+        if (nr <= 16) launch_tc_decode_nb<16, PRO, EPI>(c, a, w, units, xmap);
+        else if (nr <= 32) launch_tc_decode_nb<32, PRO, EPI>(c, a, w, units, xmap);
+        else if (nr <= 48) launch_tc_decode_nb<48, PRO, EPI>(c, a, w, units, xmap);
+        else launch_tc_decode_nb<64, PRO, EPI>(c, a, w, units, xmap);
     }
 }
 
@@ -652,13 +660,14 @@ void attention(tandem_ctx& c, const Model& m, int l, const T* q, T* o, const Row
 }
 
 // bf16 decode / block attention over the cache of layer l: bf16 queries, fp32 output rows.
-void attention_decode(tandem_ctx& c, const Model& m, int l, const bf16* q, float* o, const Rows& r) {
+void attention_decode(tandem_ctx& c, const Model& m, int l, const bf16* q, float* o, const Rows& r, bf16* o_lo = nullptr) {
     const int d = m.d.d_model, H = m.d.n_heads, dh = d / H;
     AttnArgs aa; memset(&aa, 0, sizeof(aa));
     aa.q = q; aa.ldq = d; aa.kcache = kv_ptr<bf16>(c, m, l, 0); aa.vcache = kv_ptr<bf16>(c, m, l, 1);
     aa.out = o; aa.ldo = d; aa.out_f32 = 1; aa.row_seq = at<int>(c, c.lay.row_seq); aa.row_pos = at<int>(c, c.lay.row_pos);
     aa.nq = r.nq; aa.n_heads = H; aa.n_kv_heads = m.kv_heads; aa.t_max = c.cfg.max_seq; aa.scale = 1.0f / sqrtf((float)dh);
     aa.err_flag = tc_scratch(c).err;
+    aa.out_lo = o_lo;   // non-null: o is the bf16 value plane, o_lo the remainder plane
     launch_attn_decode(c, dh, aa, r.groups, r.kv_positions * 2.0 * d * 2.0);
 }
 
@@ -879,6 +888,19 @@ void tc_begin(tandem_ctx& c, const Model& m, float* h, int r0, int nq, int fin_r
               (const bf16*)w_emb(c, m), (const bf16*)w_pos(c, m), h, m.d.d_model, snap);
 }
 
+// The decode activations' value / remainder planes (see tandem_ctx::xmap): buffer 0 = LayerNorm output, 1 = attention
+// output, 2 = GELU output; K = the row length in use (the model's width, or its FFN width for buffer 2).
+struct XPlanes { bf16* hi; bf16* lo; const CUtensorMap* map; };
+XPlanes x_planes(tandem_ctx& c, int buf, const Model& m) {
+    const size_t off = buf == 0 ? c.lay.a32 : (buf == 1 ? c.lay.o32 : c.lay.f32);
+    const size_t K = buf == 2 ? m.d.d_ff : m.d.d_model;
+    XPlanes p;
+    p.hi = reinterpret_cast<bf16*>(c.arena + off);
+    p.lo = p.hi + (size_t)c.lay.dec_rows * K;
+    p.map = &c.xmap[buf][&m == &c.large ? 0 : 1];
+    return p;
+}
+
 // Whether LayerNorm is fused into the GEMM's operand load.  Fused, every CTA of the GEMM normalises the rows it
 // needs itself: right for a couple of sequences and short rows, wasteful beyond (eight sequences of 768 elements
 // already measured 2 % slower per iteration than the LayerNorm kernel).  The choice depends on the batch
@@ -895,11 +917,25 @@ void tc_ln_gemm(tandem_ctx& c, const float* h, const void* ln_g, const void* ln_
         launch_tc_decode<PRO_LN, EPI>(c, sc, h, w.K, ln_g, ln_b, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
         return;
     }
+    const Model* hm = h == reinterpret_cast<const float*>(c.arena + c.lay.h_large) ? &c.large :
+                      (h == reinterpret_cast<const float*>(c.arena + c.lay.h_small) ? &c.small : nullptr);
+    if (!ln_out && c.xmap_ok && hm && hm->d.d_model == w.K) {
+        // the LayerNorm kernel leaves value and remainder planes, the GEMM loads them by TMA beside its weights
+        const XPlanes xp = x_planes(c, 0, *hm);
+        {
+            ProfScope ps(c, PC_LAYERNORM, (double)rows * w.K * 8.0);
+            launch_ex(c, true, 1, layernorm_rows_kernel<bf16>, dim3(rows), dim3(128), 0, h, static_cast<const float*>(ln_g),
+                      static_cast<const float*>(ln_b), xp.hi, w.K, xp.lo);
+        }
+        launch_tc_decode<PRO_TMA, EPI>(c, sc, xp.hi, w.K, nullptr, nullptr, rows, w, stream_w, e, amax_val, amax_idx, amax_stride, xp.map,
+                                       c.lay.dec_rows);
+        return;
+    }
     float* a = ln_out ? ln_out : at<float>(c, c.lay.a32);
     {
         ProfScope ps(c, PC_LAYERNORM, (double)rows * w.K * 8.0);
         launch_ex(c, true, 1, layernorm_rows_kernel<float>, dim3(rows), dim3(128), 0, h, static_cast<const float*>(ln_g),
-                  static_cast<const float*>(ln_b), a, w.K);
+                  static_cast<const float*>(ln_b), a, w.K, (bf16*)nullptr);
     }
     launch_tc_decode<PRO_F32, EPI>(c, sc, a, w.K, nullptr, nullptr, rows, w, stream_w, e, amax_val, amax_idx, amax_stride);
 }
@@ -914,13 +950,27 @@ void tc_decoder_layer(tandem_ctx& c, const Model& m, int l, float* h, const Rows
     const TcScratch sc = tc_scratch(c);
     tc_ln_gemm<EPI_QKV>(c, h, w_layer(c, m, l, W_LN1G), w_layer(c, m, l, W_LN1B), r.M,
                         tcw3(c, wi_layer(m, l, W_WQ), wi_layer(m, l, W_WK), wi_layer(m, l, W_WV), d, m.d_kv, d), stream_w, epi_cache<bf16>(c, m, l, q));
+    EpiArgs e2 = epi_plain(h, d);
+    e2.snap = snap; e2.snap_ld = d;   // copy of x^(l+1) when an FF_Tandem projection reads it
+    if (c.xmap_ok) {
+        // attention and GELU outputs as value / remainder planes that the next GEMM loads by TMA
+        const XPlanes xo = x_planes(c, 1, m), xf = x_planes(c, 2, m);
+        attention_decode(c, m, l, q, reinterpret_cast<float*>(xo.hi), r, xo.lo);
+        launch_tc_decode<PRO_TMA, EPI_RESID>(c, sc, xo.hi, d, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_WO), -1, -1, d, d), stream_w,
+                                             epi_plain(h, d), nullptr, nullptr, 0, xo.map, c.lay.dec_rows);
+        EpiArgs e1 = epi_plain(xf.hi, dff);
+        e1.out_lo = xf.lo;
+        tc_ln_gemm<EPI_GELU>(c, h, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), r.M, tcw(c, wi_layer(m, l, W_W1), -1, -1, dff, d),
+                             stream_w, e1);
+        launch_tc_decode<PRO_TMA, EPI_RESID>(c, sc, xf.hi, dff, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_W2), -1, -1, d, dff), stream_w, e2,
+                                             nullptr, nullptr, 0, xf.map, c.lay.dec_rows);
+        return;
+    }
     attention_decode(c, m, l, q, o, r);
     launch_tc_decode<PRO_F32, EPI_RESID>(c, sc, o, d, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_WO), -1, -1, d, d), stream_w,
                                          epi_plain(h, d));
     tc_ln_gemm<EPI_GELU>(c, h, w_layer(c, m, l, W_LN2G), w_layer(c, m, l, W_LN2B), r.M, tcw(c, wi_layer(m, l, W_W1), -1, -1, dff, d),
                          stream_w, epi_plain(f, dff));
-    EpiArgs e2 = epi_plain(h, d);
-    e2.snap = snap; e2.snap_ld = d;   // copy of x^(l+1) when an FF_Tandem projection reads it
     launch_tc_decode<PRO_F32, EPI_RESID>(c, sc, f, dff, nullptr, nullptr, r.M, tcw(c, wi_layer(m, l, W_W2), -1, -1, d, dff), stream_w, e2);
 }
 
@@ -1291,6 +1341,18 @@ extern "C" tandem_status tandem_create(const tandem_config* cfg, const tandem_we
             return TANDEM_ERR_CUDA;
         }
         c->tc = true;
+        {
+            bool okx = true;
+            const uint64_t RDx = (uint64_t)lay.dec_rows;
+            for (int buf = 0; buf < 3 && okx; ++buf)
+                for (int mi = 0; mi < 2 && okx; ++mi) {
+                    const Model& mm = mi == 0 ? c->large : c->small;
+                    const uint64_t K = buf == 2 ? mm.d.d_ff : mm.d.d_model;
+                    const size_t off = buf == 0 ? lay.a32 : (buf == 1 ? lay.o32 : lay.f32);
+                    okx = K % 8 == 0 && make_tmap_bf16(&c->xmap[buf][mi], c->arena + off, 2 * RDx, K, K, 16);
+                }
+            c->xmap_ok = okx;
+        }
         const int dhL = cfg->large.d_model / cfg->large.n_heads;
         if (dhL == 64 || dhL == 128) {
             c->kmap.resize(cfg->large.n_layers);
@@ -2094,7 +2156,7 @@ extern "C" tandem_status tandem_ff_tandem_project(const void* x, const void* w_t
         launch_tc_decode<PRO_LN, EPI_KV>(tmp, ts, yhat, d_small, ln_g, ln_b, rows, wkv, true, e);
     } else {
         launch_ex(tmp, false, 1, layernorm_rows_kernel<float>, dim3(rows), dim3(128), 0, (const float*)yhat, static_cast<const float*>(ln_g),
-                  static_cast<const float*>(ln_b), a_s, (int)d_small);
+                  static_cast<const float*>(ln_b), a_s, (int)d_small, (bf16*)nullptr);
         launch_tc_decode<PRO_F32, EPI_KV>(tmp, ts, a_s, d_small, nullptr, nullptr, rows, wkv, true, e);
     }
     return check_launch();
