@@ -547,26 +547,32 @@ __global__ void __launch_bounds__(ATD_THREADS) attn_decode_kernel(AttnArgs a) {
     __syncthreads();
     // fold the warps' states in warp order and send the CTA's state of query qa to CTA qa % CL
     if (CL > 1) cluster_wait();   // closes the opening handshake: every CTA of the cluster is running
-    for (int i = tid; i < cnt * SW; i += ATD_THREADS) {
-        const int qa = i / SW, e = i - qa * SW;
+    // One thread per (query, output element); the thread of element 0 also folds the query's running sum and sends its
+    // maximum (with 4 queries of 64 elements that is one pass over the block's 256 threads).
+    for (int i = tid; i < cnt * DH; i += ATD_THREADS) {
+        const int qa = i / DH, e = i - qa * DH;
         float mx = -INFINITY;
 #pragma unroll
         for (int w = 0; w < NW; ++w) mx = fmaxf(mx, wst[(size_t)(w * ATT_NQ + qa) * SW + DH]);
-        float val;
-        if (e == DH) {
-            val = mx;
-        } else {
-            val = 0.f;
+        float val = 0.f, lsum = 0.f;
 #pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                const float* st = wst + (size_t)(w * ATT_NQ + qa) * SW;
-                const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
-                val = fmaf(e < DH ? st[e] : st[DH + 1], f, val);
-            }
+        for (int w = 0; w < NW; ++w) {
+            const float* st = wst + (size_t)(w * ATT_NQ + qa) * SW;
+            const float f = st[DH] > -INFINITY ? __expf(st[DH] - mx) : 0.f;
+            val = fmaf(st[e], f, val);
+            if (e == 0) lsum = fmaf(st[DH + 1], f, lsum);
         }
-        float* slot = inbox + ((size_t)rank * QPC + qa / CL) * SW + e;
-        if (CL > 1) st_async_dsmem_f32(smem_u32(slot), smem_u32(&s_inbox_bar), qa % CL, val);   // counted on the receiver's barrier
-        else *slot = val;
+        float* slot = inbox + ((size_t)rank * QPC + qa / CL) * SW;
+        if (CL > 1) {   // counted on the receiver's barrier
+            st_async_dsmem_f32(smem_u32(slot + e), smem_u32(&s_inbox_bar), qa % CL, val);
+            if (e == 0) {
+                st_async_dsmem_f32(smem_u32(slot + DH), smem_u32(&s_inbox_bar), qa % CL, mx);
+                st_async_dsmem_f32(smem_u32(slot + DH + 1), smem_u32(&s_inbox_bar), qa % CL, lsum);
+            }
+        } else {
+            slot[e] = val;
+            if (e == 0) { slot[DH] = mx; slot[DH + 1] = lsum; }
+        }
     }
     if (CL > 1) {
         // This CTA finishes queries rank, rank + CL, ...: it waits (bounded) until every CTA's state of each of them
